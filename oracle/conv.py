@@ -1,0 +1,137 @@
+"""Oracle: convolution / tensor-product entry points (test infrastructure only).
+
+conv_fwd / conv_bwd call the plain C loops of conv_naive.c (float64 sums of the
+paper's message-passing-convolution and message-passing-backward equations).
+tp_fwd / tp_bwd are the tensor-product formula followed by the edge-scalar
+weighting ("Mathematical operations") and the tensor-product backward rule
+("Differentiation"), written as dense numpy contractions in float64.
+
+The C file is compiled on first use with gcc (and by the repository build
+step); nothing here touches the CUDA library.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+from . import cg
+
+_HERE = Path(__file__).resolve().parent
+_SO = _HERE / "libe3j_oracle.so"
+_SRC = _HERE / "conv_naive.c"
+_lib = None
+
+
+def build(force: bool = False) -> Path:
+    """Compile conv_naive.c into libe3j_oracle.so next to it."""
+    if force or not _SO.exists() or _SO.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _SO.with_suffix(f".tmp{os.getpid()}.so")
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", str(tmp), str(_SRC)])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(str(_SO))
+        i64, i32 = ctypes.c_int64, ctypes.c_int
+        ptr = ctypes.c_void_p
+        lib.e3j_oracle_conv_fwd.argtypes = [i64, i64, i32, i32, i32, i32, i32] + [ptr] * 8
+        lib.e3j_oracle_conv_fwd.restype = i32
+        lib.e3j_oracle_conv_bwd.argtypes = [i64, i64, i32, i32, i32, i32, i32] + [ptr] * 11
+        lib.e3j_oracle_conv_bwd.restype = i32
+        lib.e3j_oracle_threads.restype = i32
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    """Number of OpenMP threads the C loops will use."""
+    return int(_load().e3j_oracle_threads())
+
+
+class Coupling:
+    """Dense coupling tensor and shapes of one (irreps_in, sh_lmax, irreps_out) signature."""
+
+    def __init__(self, irreps_in: str, sh_lmax: int, irreps_out: str | None = None,
+                 out_lmax: int | None = None):
+        self.C, self.i3, self.paths, self.nq = cg.dense_coupling(irreps_in, sh_lmax, irreps_out, out_lmax)
+        self.D, self.d, self.dp = self.C.shape
+        self.P = len(self.paths)
+        self.C = np.ascontiguousarray(self.C)
+        self.i3 = np.ascontiguousarray(self.i3, dtype=np.int32)
+
+    @property
+    def nnz(self) -> int:
+        return int(np.count_nonzero(self.C))
+
+
+def _f32(a, shape):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    assert a.shape == tuple(shape), (a.shape, shape)
+    return a
+
+
+def _i32(a, n):
+    a = np.ascontiguousarray(a, dtype=np.int32)
+    assert a.shape == (n,)
+    return a
+
+
+def _p(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def conv_fwd(cp: Coupling, x, y, s, senders, receivers) -> np.ndarray:
+    """m[N, D, N_q] in float64."""
+    n, e = x.shape[0], len(senders)
+    x = _f32(x, (n, cp.d, cp.nq)); y = _f32(y, (e, cp.dp)); s = _f32(s, (e, cp.P, cp.nq))
+    senders, receivers = _i32(senders, e), _i32(receivers, e)
+    out = np.zeros((n, cp.D, cp.nq))
+    rc = _load().e3j_oracle_conv_fwd(n, e, cp.d, cp.dp, cp.P, cp.D, cp.nq, _p(cp.C), _p(cp.i3),
+                                     _p(x), _p(y), _p(s), _p(senders), _p(receivers), _p(out))
+    if rc != 0:
+        raise ValueError("oracle: receivers not sorted or index out of range")
+    return out
+
+
+def conv_bwd(cp: Coupling, x, y, s, senders, receivers, dm):
+    """(dx[N,d,N_q], dy[E,d'], ds[E,P,N_q]) in float64."""
+    n, e = x.shape[0], len(senders)
+    x = _f32(x, (n, cp.d, cp.nq)); y = _f32(y, (e, cp.dp)); s = _f32(s, (e, cp.P, cp.nq))
+    dm = _f32(dm, (n, cp.D, cp.nq))
+    senders, receivers = _i32(senders, e), _i32(receivers, e)
+    dx = np.zeros((n, cp.d, cp.nq)); dy = np.zeros((e, cp.dp)); ds = np.zeros((e, cp.P, cp.nq))
+    rc = _load().e3j_oracle_conv_bwd(n, e, cp.d, cp.dp, cp.P, cp.D, cp.nq, _p(cp.C), _p(cp.i3),
+                                     _p(x), _p(y), _p(s), _p(senders), _p(receivers), _p(dm),
+                                     _p(dx), _p(dy), _p(ds))
+    if rc != 0:
+        raise ValueError("oracle: receivers not sorted or index out of range")
+    return dx, dy, ds
+
+
+def tp_fwd(cp: Coupling, x1, x2, w) -> np.ndarray:
+    """z[r,i0,q] = w[r,i3(i0),q] * sum_{i1,i2} C[i0,i1,i2] x1[r,i1,q] x2[r,i2]  (float64)."""
+    x1 = np.asarray(x1, dtype=np.float64); x2 = np.asarray(x2, dtype=np.float64)
+    w = np.asarray(w, dtype=np.float64)
+    z = np.einsum("ijk,rjq,rk->riq", cp.C, x1, x2)
+    return z * w[:, cp.i3, :]
+
+
+def tp_bwd(cp: Coupling, x1, x2, w, dz):
+    """(dx1, dx2, dw) of tp_fwd for the output cotangent dz, float64."""
+    x1 = np.asarray(x1, dtype=np.float64); x2 = np.asarray(x2, dtype=np.float64)
+    w = np.asarray(w, dtype=np.float64); dz = np.asarray(dz, dtype=np.float64)
+    wdz = dz * w[:, cp.i3, :]
+    dx1 = np.einsum("ijk,rk,riq->rjq", cp.C, x2, wdz)
+    dx2 = np.einsum("ijk,rjq,riq->rk", cp.C, x1, wdz)
+    z = np.einsum("ijk,rjq,rk->riq", cp.C, x1, x2)
+    dw = np.zeros_like(w)
+    np.add.at(dw, (slice(None), cp.i3, slice(None)), z * dz)
+    return dx1, dx2, dw
