@@ -1,0 +1,176 @@
+/* e3j.h -- C ABI of the B200 (sm_100a) fused equivariant message-passing convolution.
+ *
+ * The operation (paper: appendix "Tensor Product and Message Passing Convolution
+ * kernels", section "Mathematical Details"):
+ *
+ *   forward  (message-passing-convolution equation)
+ *     out[b,i0,q] = sum_{edges e with receiver b} w[e,i3(i0),q]
+ *                   * sum_{i1,i2} C[i0,i1,i2] * x[sender(e),i1,q] * sh[e,i2]
+ *   backward (message-passing-backward equation, ds per irreducible block)
+ *     grad_x[a,i1,q] = sum_{edges e with sender a} sum C * sh[e,i2] * w[e,k,q] * grad_out[b,i0,q]
+ *     grad_sh[e,i2]  = sum_q sum C * x[a,i1,q] * w[e,k,q] * grad_out[b,i0,q]
+ *     grad_w[e,k,q]  = sum_{i0 in block k} grad_out[b,i0,q] * sum C * x[a,i1,q] * sh[e,i2]
+ *
+ * C is the real Clebsch-Gordan coupling tensor of every allowed path
+ * (l1,p1) x (l2,(-1)^l2) -> (L, p1*(-1)^l2), |l1-l2| <= L <= l1+l2, kept as a
+ * sparse list of records (i0,i1,i2,i3,value) sorted by output coordinate i0
+ * (paper: "CUDA kernels", sparse COO records).  One output block and one weight
+ * block per path (output multiplicities are not collapsed).
+ *
+ * Conventions
+ *   - Layout is the paper's trailing-channel layout: [batch, feature coordinate,
+ *     channel], channel fastest.  (The multiplicity-major layout of e3nn is not
+ *     accepted; transpose first.)
+ *   - Components of a degree-l block are ordered m = -l..l.
+ *   - Coefficients: unitary real CG (sum over (m1,m2) of C^2 = 1 per output
+ *     component), real basis Y_{l,m>0} = sqrt2 (-1)^m Re Y_l^m,
+ *     Y_{l,m<0} = sqrt2 (-1)^m Im Y_l^{|m|}; each path's sign is chosen so that
+ *     its first non-zero entry in (M,m1,m2) order is positive
+ *     (so 1 x 1 -> 0 is +dot/sqrt(3), l x 0 -> l is +identity).
+ *   - Paths are ordered by the position of their output irrep in `irreps_out`
+ *     (default 0e,0o,1o,1e,2e,2o,3o,3e,...), ties by (input irrep index, l2).
+ *     Output block k and weight block k belong to path k.
+ *   - All tensors are float32, all graph indices int32, all pointers DEVICE
+ *     pointers unless stated otherwise.  The caller owns every tensor and every
+ *     workspace; a plan owns only its coefficient tables.
+ *   - Every compute call enqueues work on `stream` (a cudaStream_t passed as
+ *     void*) and returns without synchronising.  Outputs are fully overwritten.
+ *   - Results are bit-identical from run to run on the same device: no
+ *     floating-point atomics are used anywhere.
+ *   - There is no CPU fallback.  Without a usable CUDA device every compute call
+ *     returns E3J_ERR_CUDA.
+ *
+ * Errors: every function returns an int status (0 = E3J_OK, negative = error);
+ * nothing throws across this boundary.  e3j_status_string() names a status,
+ * e3j_last_cuda_error() returns the cudaError_t behind the last E3J_ERR_CUDA
+ * on the calling thread.
+ */
+#ifndef E3J_H_
+#define E3J_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    E3J_OK = 0,
+    E3J_ERR_INVALID_ARG = -1,   /* NULL pointer, negative size, capacity too small        */
+    E3J_ERR_BAD_IRREPS = -2,    /* descriptor string does not parse                         */
+    E3J_ERR_MUL_NOT_UNIFORM = -3, /* input irreps must share one multiplicity (= N_q)       */
+    E3J_ERR_UNSUPPORTED = -4,   /* a dimension exceeds 255, l > 8, or nothing couples        */
+    E3J_ERR_WORKSPACE = -5,     /* workspace NULL, misaligned (256 B) or too small            */
+    E3J_ERR_CUDA = -6,          /* a CUDA runtime call failed; see e3j_last_cuda_error()      */
+    E3J_ERR_GRAPH = -7          /* written by e3j_graph_validate into its device status word */
+};
+
+/* plan flags */
+#define E3J_PLAN_GENERIC_ONLY 1u /* never pick a signature-specialised kernel */
+
+typedef struct e3j_plan e3j_plan; /* opaque; immutable after creation; usable from several streams */
+
+typedef struct {
+    int n_channels; /* N_q : uniform multiplicity of the input irreps                  */
+    int d_in;       /* d   : input feature coordinates, sum (2 l1 + 1)                 */
+    int d_sh;       /* d'  : (sh_lmax + 1)^2                                           */
+    int n_paths;    /* P   : paths = output blocks = weight blocks                     */
+    int d_out;      /* D   : output coordinates, sum over paths (2L + 1)               */
+    int nnz;        /* non-zero coefficient records                                    */
+    int n_pairs;    /* distinct (i0,i1) pairs with a non-zero coefficient              */
+    int specialised;/* 1 if signature-specialised kernels exist and are enabled        */
+} e3j_plan_info_t;
+
+typedef struct {
+    int in_index;   /* which input irrep                */
+    int l1, p1;     /* its degree and parity (+1 / -1)  */
+    int l2;         /* harmonic degree                  */
+    int L, p;       /* output degree and parity         */
+    int x_off;      /* first i1 coordinate              */
+    int y_off;      /* first i2 coordinate (= l2^2)     */
+    int out_off;    /* first i0 coordinate              */
+} e3j_path_info_t;
+
+/* Plan builder (host only; paper: "Reconstruction of Clebsch Gordan coefficients",
+ * ladder-operator construction, and "CUDA kernels", sparse records and index packing).
+ *   irreps_in   e.g. "128x0e+128x1o"; one multiplicity for all irreps (= N_q)
+ *   sh_lmax     harmonics are 1x0e + 1x1o + ... + 1x(sh_lmax)
+ *   irreps_out  filter and block order, e.g. "0e+1o+1e+2e+2o"; NULL = every
+ *               reachable (L,p) with L <= out_lmax in the default order
+ *   out_lmax    used only when irreps_out is NULL; negative = no limit
+ * Creates host tables only; device copies are made on first use on each device.
+ * The plan must be released with e3j_plan_destroy. */
+int e3j_plan_create(e3j_plan** out, const char* irreps_in, int sh_lmax, const char* irreps_out,
+                    int out_lmax, unsigned flags);
+int e3j_plan_destroy(e3j_plan* plan);
+int e3j_plan_info(const e3j_plan* plan, e3j_plan_info_t* info);
+/* Copies up to `capacity` path descriptors (host memory); returns P or an error. */
+int e3j_plan_paths(const e3j_plan* plan, e3j_path_info_t* paths, int capacity);
+/* Copies the coefficient records, sorted by (i0,i1,i2), into HOST arrays of
+ * `capacity` entries each (val in float64 as built, before rounding to float32);
+ * returns nnz or an error. */
+int e3j_plan_records(const e3j_plan* plan, int32_t* i0, int32_t* i1, int32_t* i2, int32_t* i3,
+                     double* val, int capacity);
+
+/* Graph preparation (paper: the forward algorithm takes receiver CSR pointers as
+ * data; the backward is "message passing on the transposed graph").  Integer work
+ * only, all on the device:
+ *   rowptr[n_nodes+1]   rowptr[b] = first edge with receiver >= b
+ *   sender_perm[n_edges] edge ids sorted by (sender, edge id)
+ *   colptr[n_nodes+1]   sender_perm[colptr[a] .. colptr[a+1]) are the edges sent by a
+ * receivers must be non-decreasing.  Any output pointer may be NULL (skipped);
+ * sender_perm and colptr are produced together. */
+int e3j_graph_prepare(int64_t n_nodes, int64_t n_edges, const int32_t* senders,
+                      const int32_t* receivers, int32_t* rowptr, int32_t* sender_perm,
+                      int32_t* colptr, void* stream);
+/* Writes 0 (fine) or E3J_ERR_GRAPH (receivers decrease somewhere, or an index is
+ * outside [0, n_nodes)) into the DEVICE word *status; read it after synchronising. */
+int e3j_graph_validate(int64_t n_nodes, int64_t n_edges, const int32_t* senders,
+                       const int32_t* receivers, int32_t* status, void* stream);
+
+/* Convolution forward.  Shapes: x [n_nodes,d,N_q], sh [n_edges,d'], w [n_edges,P,N_q],
+ * senders/receivers [n_edges] (receivers non-decreasing), rowptr [n_nodes+1] or NULL
+ * (then it is derived into the workspace), out [n_nodes,D,N_q].  Receivers without
+ * edges get a row of zeros.  workspace: 256-byte aligned, at least
+ * e3j_conv_fwd_workspace_bytes(); its contents need not be preserved between calls,
+ * and two calls that overlap on the GPU must not share it. */
+size_t e3j_conv_fwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges);
+int e3j_conv_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                 const float* sh, const float* w, const int32_t* senders,
+                 const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                 size_t workspace_bytes, void* stream);
+
+/* Convolution backward.  grad_out [n_nodes,D,N_q]; grad_x [n_nodes,d,N_q],
+ * grad_sh [n_edges,d'], grad_w [n_edges,P,N_q]; any of the three may be NULL (not
+ * computed).  rowptr, sender_perm, colptr as produced by e3j_graph_prepare, or NULL
+ * (then derived into the workspace on every call).  A node that sends nothing gets
+ * a zero grad_x row. */
+size_t e3j_conv_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges);
+int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                 const float* sh, const float* w, const int32_t* senders,
+                 const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                 const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
+                 float* grad_w, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Standalone channelwise tensor product with per-row, per-path weights (paper:
+ * tensor-product formula followed by the edge-scalar weighting; backward: the
+ * tensor-product backward rule, one streaming pass).  Rows are their own receivers:
+ *   out[r,i0,q] = w[r,i3(i0),q] * sum C[i0,i1,i2] * x1[r,i1,q] * x2[r,i2]
+ * x1 [rows,d,N_q], x2 [rows,d'], w [rows,P,N_q], out/grad_out [rows,D,N_q].
+ * Any of grad_x1, grad_x2, grad_w may be NULL. */
+int e3j_tp_fwd(const e3j_plan* plan, int64_t rows, const float* x1, const float* x2,
+               const float* w, float* out, void* stream);
+int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float* x2,
+               const float* w, const float* grad_out, float* grad_x1, float* grad_x2,
+               float* grad_w, void* stream);
+
+const char* e3j_status_string(int status);
+int e3j_last_cuda_error(void);
+/* Number of kernel launches this library has enqueued from the calling process. */
+int64_t e3j_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* E3J_H_ */

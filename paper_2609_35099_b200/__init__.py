@@ -1,1 +1,320 @@
-"""placeholder, replaced below"""
+"""Python binding of libe3j (the sm_100a fused equivariant convolution).
+
+Argument marshalling only: every function below has the name of the C entry point
+it calls (see include/e3j.h) and passes device pointers of torch tensors straight
+through.  torch is used for device memory and streams, nothing else; there is no
+CPU or PyTorch fallback -- if the compiled library is missing, or a call fails,
+an exception is raised.
+
+    plan = e3j_plan_create("128x0e+128x1o", 3, None, 3)
+    rowptr, sender_perm, colptr = e3j_graph_prepare(n_nodes, senders, receivers)
+    out = e3j_conv_fwd(plan, x, sh, w, senders, receivers, rowptr)
+    gx, gsh, gw = e3j_conv_bwd(plan, x, sh, w, senders, receivers, grad_out,
+                               rowptr, sender_perm, colptr)
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+__all__ = [
+    "E3JError", "Plan", "library_path", "e3j_plan_create", "e3j_plan_destroy", "e3j_plan_info",
+    "e3j_plan_paths", "e3j_plan_records", "e3j_graph_prepare", "e3j_graph_validate",
+    "e3j_conv_fwd_workspace_bytes", "e3j_conv_bwd_workspace_bytes", "e3j_conv_fwd", "e3j_conv_bwd",
+    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_status_string", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
+]
+
+E3J_PLAN_GENERIC_ONLY = 1
+_LIB_PATH = Path(__file__).resolve().parent / "libe3j.so"
+_lib = None
+
+
+class E3JError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        lib = _load()
+        msg = lib.e3j_status_string(status).decode()
+        if status == -6:
+            msg += f" (cudaError {lib.e3j_last_cuda_error()})"
+        super().__init__(f"{where}: {msg} [status {status}]")
+        self.status = status
+
+
+class _PlanInfo(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("n_channels", "d_in", "d_sh", "n_paths", "d_out", "nnz", "n_pairs", "specialised")]
+
+
+class _PathInfo(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("in_index", "l1", "p1", "l2", "L", "p", "x_off", "y_off", "out_off")]
+
+
+def library_path() -> Path:
+    return _LIB_PATH
+
+
+def _load():
+    """Loads libe3j.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2609_35099_b200.build` "
+            "(nvcc, sm_100a). There is no CPU or PyTorch fallback.")
+    lib = ctypes.CDLL(str(_LIB_PATH))
+    vp, i64, i32, sz, u32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t, ctypes.c_uint
+    lib.e3j_plan_create.argtypes = [ctypes.POINTER(vp), ctypes.c_char_p, i32, ctypes.c_char_p, i32, u32]
+    lib.e3j_plan_destroy.argtypes = [vp]
+    lib.e3j_plan_info.argtypes = [vp, ctypes.POINTER(_PlanInfo)]
+    lib.e3j_plan_paths.argtypes = [vp, ctypes.POINTER(_PathInfo), i32]
+    lib.e3j_plan_records.argtypes = [vp, vp, vp, vp, vp, vp, i32]
+    lib.e3j_graph_prepare.argtypes = [i64, i64, vp, vp, vp, vp, vp, vp]
+    lib.e3j_graph_validate.argtypes = [i64, i64, vp, vp, vp, vp]
+    lib.e3j_conv_fwd_workspace_bytes.argtypes = [vp, i64, i64]
+    lib.e3j_conv_fwd_workspace_bytes.restype = sz
+    lib.e3j_conv_bwd_workspace_bytes.argtypes = [vp, i64, i64]
+    lib.e3j_conv_bwd_workspace_bytes.restype = sz
+    lib.e3j_conv_fwd.argtypes = [vp, i64, i64] + [vp] * 8 + [sz, vp]
+    lib.e3j_conv_bwd.argtypes = [vp, i64, i64] + [vp] * 13 + [sz, vp]
+    lib.e3j_tp_fwd.argtypes = [vp, i64] + [vp] * 5
+    lib.e3j_tp_bwd.argtypes = [vp, i64] + [vp] * 8
+    lib.e3j_status_string.argtypes = [i32]
+    lib.e3j_status_string.restype = ctypes.c_char_p
+    lib.e3j_last_cuda_error.restype = i32
+    lib.e3j_launch_count.restype = i64
+    for name in ("e3j_plan_create", "e3j_plan_destroy", "e3j_plan_info", "e3j_plan_paths", "e3j_plan_records",
+                 "e3j_graph_prepare", "e3j_graph_validate", "e3j_conv_fwd", "e3j_conv_bwd", "e3j_tp_fwd",
+                 "e3j_tp_bwd"):
+        getattr(lib, name).restype = i32
+    _lib = lib
+    return lib
+
+
+def _check(status: int, where: str) -> int:
+    if status < 0:
+        raise E3JError(status, where)
+    return status
+
+
+class Plan:
+    """Owner of one e3j_plan handle (released when the object is collected)."""
+
+    def __init__(self, handle: int):
+        self.handle = ctypes.c_void_p(handle)
+        info = _PlanInfo()
+        _check(_load().e3j_plan_info(self.handle, ctypes.byref(info)), "e3j_plan_info")
+        for name, _ in _PlanInfo._fields_:
+            setattr(self, name, getattr(info, name))
+
+    def __del__(self):
+        try:
+            e3j_plan_destroy(self)
+        except Exception:
+            pass
+
+
+def e3j_plan_create(irreps_in: str, sh_lmax: int, irreps_out: str | None = None, out_lmax: int = -1,
+                    flags: int = 0) -> Plan:
+    h = ctypes.c_void_p()
+    out = irreps_out.encode() if irreps_out is not None else None
+    _check(_load().e3j_plan_create(ctypes.byref(h), irreps_in.encode(), sh_lmax, out, out_lmax, flags),
+           "e3j_plan_create")
+    return Plan(h.value)
+
+
+def e3j_plan_destroy(plan: Plan) -> None:
+    if plan.handle is not None and plan.handle.value:
+        _load().e3j_plan_destroy(plan.handle)
+        plan.handle = ctypes.c_void_p()
+
+
+def e3j_plan_info(plan: Plan) -> dict:
+    return {name: getattr(plan, name) for name, _ in _PlanInfo._fields_}
+
+
+def e3j_plan_paths(plan: Plan) -> list[dict]:
+    arr = (_PathInfo * plan.n_paths)()
+    _check(_load().e3j_plan_paths(plan.handle, arr, plan.n_paths), "e3j_plan_paths")
+    return [{name: getattr(p, name) for name, _ in _PathInfo._fields_} for p in arr]
+
+
+def e3j_plan_records(plan: Plan):
+    """(i0, i1, i2, i3, val) numpy arrays of the coefficient records (host side)."""
+    import numpy as np
+    n = plan.nnz
+    idx = [np.zeros(n, dtype=np.int32) for _ in range(4)]
+    val = np.zeros(n, dtype=np.float64)
+    ptr = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    _check(_load().e3j_plan_records(plan.handle, *map(ptr, idx), ptr(val), n), "e3j_plan_records")
+    return (*idx, val)
+
+
+# ----------------------------------------------------------------- marshalling
+def _torch():
+    import torch
+    return torch
+
+
+def _dev_ptr(t, dtype, shape, name):
+    torch = _torch()
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name} must be contiguous {dtype}")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    torch = _torch()
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _workspace(nbytes: int, like, workspace):
+    torch = _torch()
+    if workspace is None:
+        workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=like.device)
+    if workspace.dtype != torch.uint8 or not workspace.is_cuda or workspace.numel() < nbytes:
+        raise ValueError("workspace must be a CUDA uint8 tensor of sufficient size")
+    return workspace
+
+
+def e3j_graph_prepare(n_nodes: int, senders, receivers, want_transpose: bool = True, stream=None):
+    """(rowptr, sender_perm, colptr) int32 CUDA tensors; the last two are None unless want_transpose."""
+    torch = _torch()
+    e = senders.numel()
+    rowptr = torch.empty(n_nodes + 1, dtype=torch.int32, device=senders.device)
+    perm = torch.empty(max(e, 1), dtype=torch.int32, device=senders.device) if want_transpose else None
+    colptr = torch.empty(n_nodes + 1, dtype=torch.int32, device=senders.device) if want_transpose else None
+    _check(_load().e3j_graph_prepare(n_nodes, e, _dev_ptr(senders, torch.int32, (e,), "senders"),
+                                     _dev_ptr(receivers, torch.int32, (e,), "receivers"),
+                                     _dev_ptr(rowptr, torch.int32, None, "rowptr"),
+                                     _dev_ptr(perm, torch.int32, None, "sender_perm"),
+                                     _dev_ptr(colptr, torch.int32, None, "colptr"), _stream(stream)),
+           "e3j_graph_prepare")
+    if perm is not None:
+        perm = perm[:e]
+    return rowptr, perm, colptr
+
+
+def e3j_graph_validate(n_nodes: int, senders, receivers, stream=None) -> int:
+    """0 if the graph is usable, else the (negative) E3J_ERR_GRAPH status.  Synchronises."""
+    torch = _torch()
+    e = senders.numel()
+    status = torch.zeros(1, dtype=torch.int32, device=senders.device)
+    _check(_load().e3j_graph_validate(n_nodes, e, _dev_ptr(senders, torch.int32, (e,), "senders"),
+                                      _dev_ptr(receivers, torch.int32, (e,), "receivers"),
+                                      _dev_ptr(status, torch.int32, None, "status"), _stream(stream)),
+           "e3j_graph_validate")
+    return int(status.item())
+
+
+def e3j_conv_fwd_workspace_bytes(plan: Plan, n_nodes: int, n_edges: int) -> int:
+    return int(_load().e3j_conv_fwd_workspace_bytes(plan.handle, n_nodes, n_edges))
+
+
+def e3j_conv_bwd_workspace_bytes(plan: Plan, n_nodes: int, n_edges: int) -> int:
+    return int(_load().e3j_conv_bwd_workspace_bytes(plan.handle, n_nodes, n_edges))
+
+
+def e3j_conv_fwd(plan: Plan, x, sh, w, senders, receivers, rowptr=None, out=None, workspace=None,
+                 stream=None):
+    torch = _torch()
+    n, e = x.shape[0], senders.numel()
+    f32, i32 = torch.float32, torch.int32
+    if out is None:
+        out = torch.empty((n, plan.d_out, plan.n_channels), dtype=f32, device=x.device)
+    nbytes = e3j_conv_fwd_workspace_bytes(plan, n, e)
+    workspace = _workspace(nbytes, x, workspace)
+    _check(_load().e3j_conv_fwd(
+        plan.handle, n, e,
+        _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"),
+        _dev_ptr(sh, f32, (e, plan.d_sh), "sh"),
+        _dev_ptr(w, f32, (e, plan.n_paths, plan.n_channels), "w"),
+        _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
+        _dev_ptr(rowptr, i32, (n + 1,), "rowptr"),
+        _dev_ptr(out, f32, (n, plan.d_out, plan.n_channels), "out"),
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_fwd")
+    return out
+
+
+def e3j_conv_bwd(plan: Plan, x, sh, w, senders, receivers, grad_out, rowptr=None, sender_perm=None,
+                 colptr=None, grad_x=True, grad_sh=True, grad_w=True, workspace=None, stream=None):
+    """Returns (grad_x, grad_sh, grad_w).  Each grad_* argument is True (allocate), False/None
+    (not wanted) or a preallocated tensor."""
+    torch = _torch()
+    n, e = x.shape[0], senders.numel()
+    f32, i32 = torch.float32, torch.int32
+
+    def alloc(flag, shape):
+        if flag is True:
+            return torch.empty(shape, dtype=f32, device=x.device)
+        return flag if isinstance(flag, torch.Tensor) else None
+
+    grad_x = alloc(grad_x, (n, plan.d_in, plan.n_channels))
+    grad_sh = alloc(grad_sh, (e, plan.d_sh))
+    grad_w = alloc(grad_w, (e, plan.n_paths, plan.n_channels))
+    nbytes = e3j_conv_bwd_workspace_bytes(plan, n, e)
+    workspace = _workspace(nbytes, x, workspace)
+    _check(_load().e3j_conv_bwd(
+        plan.handle, n, e,
+        _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"),
+        _dev_ptr(sh, f32, (e, plan.d_sh), "sh"),
+        _dev_ptr(w, f32, (e, plan.n_paths, plan.n_channels), "w"),
+        _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
+        _dev_ptr(rowptr, i32, (n + 1,), "rowptr"),
+        _dev_ptr(sender_perm, i32, (e,), "sender_perm"), _dev_ptr(colptr, i32, (n + 1,), "colptr"),
+        _dev_ptr(grad_out, f32, (n, plan.d_out, plan.n_channels), "grad_out"),
+        _dev_ptr(grad_x, f32, (n, plan.d_in, plan.n_channels), "grad_x"),
+        _dev_ptr(grad_sh, f32, (e, plan.d_sh), "grad_sh"),
+        _dev_ptr(grad_w, f32, (e, plan.n_paths, plan.n_channels), "grad_w"),
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_bwd")
+    return grad_x, grad_sh, grad_w
+
+
+def e3j_tp_fwd(plan: Plan, x1, x2, w, out=None, stream=None):
+    torch = _torch()
+    rows, f32 = x1.shape[0], torch.float32
+    if out is None:
+        out = torch.empty((rows, plan.d_out, plan.n_channels), dtype=f32, device=x1.device)
+    _check(_load().e3j_tp_fwd(
+        plan.handle, rows, _dev_ptr(x1, f32, (rows, plan.d_in, plan.n_channels), "x1"),
+        _dev_ptr(x2, f32, (rows, plan.d_sh), "x2"),
+        _dev_ptr(w, f32, (rows, plan.n_paths, plan.n_channels), "w"),
+        _dev_ptr(out, f32, (rows, plan.d_out, plan.n_channels), "out"), _stream(stream)), "e3j_tp_fwd")
+    return out
+
+
+def e3j_tp_bwd(plan: Plan, x1, x2, w, grad_out, grad_x1=True, grad_x2=True, grad_w=True, stream=None):
+    torch = _torch()
+    rows, f32 = x1.shape[0], torch.float32
+
+    def alloc(flag, shape):
+        if flag is True:
+            return torch.empty(shape, dtype=f32, device=x1.device)
+        return flag if isinstance(flag, torch.Tensor) else None
+
+    grad_x1 = alloc(grad_x1, (rows, plan.d_in, plan.n_channels))
+    grad_x2 = alloc(grad_x2, (rows, plan.d_sh))
+    grad_w = alloc(grad_w, (rows, plan.n_paths, plan.n_channels))
+    _check(_load().e3j_tp_bwd(
+        plan.handle, rows, _dev_ptr(x1, f32, (rows, plan.d_in, plan.n_channels), "x1"),
+        _dev_ptr(x2, f32, (rows, plan.d_sh), "x2"),
+        _dev_ptr(w, f32, (rows, plan.n_paths, plan.n_channels), "w"),
+        _dev_ptr(grad_out, f32, (rows, plan.d_out, plan.n_channels), "grad_out"),
+        _dev_ptr(grad_x1, f32, None, "grad_x1"), _dev_ptr(grad_x2, f32, None, "grad_x2"),
+        _dev_ptr(grad_w, f32, None, "grad_w"), _stream(stream)), "e3j_tp_bwd")
+    return grad_x1, grad_x2, grad_w
+
+
+def e3j_status_string(status: int) -> str:
+    return _load().e3j_status_string(status).decode()
+
+
+def e3j_launch_count() -> int:
+    return int(_load().e3j_launch_count())

@@ -1,0 +1,358 @@
+// C ABI of libe3j: argument checking, device-table upload, kernel dispatch.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "fast_registry.hpp"
+#include "generic_kernels.cuh"
+
+namespace e3j {
+
+thread_local int g_last_cuda_error = 0;
+std::atomic<int64_t> g_launch_count{0};
+
+int graph_prepare(int64_t, int64_t, const int32_t*, const int32_t*, int32_t*, int32_t*, int32_t*,
+                  cudaStream_t);
+int graph_validate(int64_t, int64_t, const int32_t*, const int32_t*, int32_t*, cudaStream_t);
+
+namespace {
+
+template <class Key>
+void pack_sorted(const std::vector<Record>& rec, int n_keys, Key key, std::vector<PackedRecord>& out,
+                 std::vector<int32_t>& start, int which) {
+    std::vector<Record> r = rec;
+    std::stable_sort(r.begin(), r.end(), [&](const Record& a, const Record& b) { return key(a) < key(b); });
+    out.clear();
+    start.assign(n_keys + 1, 0);
+    for (const Record& x : r) {
+        PackedRecord p{};
+        if (which == 0) { p.a = (uint8_t)x.i1; p.b = (uint8_t)x.i2; }
+        if (which == 1) { p.a = (uint8_t)x.i0; p.b = (uint8_t)x.i2; }
+        if (which == 2) { p.a = (uint8_t)x.i0; p.b = (uint8_t)x.i1; }
+        p.c = (uint8_t)x.i3;
+        p.val = (float)x.val;
+        out.push_back(p);
+        start[key(x) + 1] += 1;
+    }
+    for (int i = 0; i < n_keys; ++i) start[i + 1] += start[i];
+}
+
+}  // namespace
+
+int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
+    int device = 0;
+    E3J_CUDA_TRY(cudaGetDevice(&device));
+    std::lock_guard<std::mutex> lock(plan->mu);
+    for (const DeviceTables& t : plan->dev)
+        if (t.device == device) { out = t; return E3J_OK; }
+
+    std::vector<PackedRecord> r0, r1, r2;
+    std::vector<int32_t> s0, s1, s2, i0_path(plan->D), path_off(plan->P + 1);
+    pack_sorted(plan->rec, plan->D, [](const Record& r) { return r.i0; }, r0, s0, 0);
+    pack_sorted(plan->rec, plan->d, [](const Record& r) { return r.i1; }, r1, s1, 1);
+    pack_sorted(plan->rec, plan->dp, [](const Record& r) { return r.i2; }, r2, s2, 2);
+    for (int k = 0; k < plan->P; ++k) {
+        path_off[k] = plan->paths[k].out_off;
+        for (int m = 0; m < 2 * plan->paths[k].L + 1; ++m) i0_path[plan->paths[k].out_off + m] = k;
+    }
+    path_off[plan->P] = plan->D;
+
+    // one allocation, 256-byte aligned sections
+    size_t off = 0;
+    auto reserve = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t nb = sizeof(PackedRecord) * plan->rec.size();
+    const size_t o_r0 = reserve(nb), o_r1 = reserve(nb), o_r2 = reserve(nb);
+    const size_t o_s0 = reserve(4 * s0.size()), o_s1 = reserve(4 * s1.size()), o_s2 = reserve(4 * s2.size());
+    const size_t o_ip = reserve(4 * i0_path.size()), o_po = reserve(4 * path_off.size());
+    std::vector<char> host(off, 0);
+    std::memcpy(host.data() + o_r0, r0.data(), nb);
+    std::memcpy(host.data() + o_r1, r1.data(), nb);
+    std::memcpy(host.data() + o_r2, r2.data(), nb);
+    std::memcpy(host.data() + o_s0, s0.data(), 4 * s0.size());
+    std::memcpy(host.data() + o_s1, s1.data(), 4 * s1.size());
+    std::memcpy(host.data() + o_s2, s2.data(), 4 * s2.size());
+    std::memcpy(host.data() + o_ip, i0_path.data(), 4 * i0_path.size());
+    std::memcpy(host.data() + o_po, path_off.data(), 4 * path_off.size());
+
+    DeviceTables t;
+    t.device = device;
+    E3J_CUDA_TRY(cudaMalloc(&t.base, off));
+    const cudaError_t err = cudaMemcpy(t.base, host.data(), off, cudaMemcpyHostToDevice);
+    if (err != cudaSuccess) { cudaFree(t.base); return cuda_status(err); }
+    char* b = (char*)t.base;
+    t.by_i0 = (const PackedRecord*)(b + o_r0);
+    t.by_i1 = (const PackedRecord*)(b + o_r1);
+    t.by_i2 = (const PackedRecord*)(b + o_r2);
+    t.i0_start = (const int32_t*)(b + o_s0);
+    t.i1_start = (const int32_t*)(b + o_s1);
+    t.i2_start = (const int32_t*)(b + o_s2);
+    t.i0_path = (const int32_t*)(b + o_ip);
+    t.path_out_off = (const int32_t*)(b + o_po);
+    plan->dev.push_back(t);
+    out = t;
+    return E3J_OK;
+}
+
+namespace {
+
+inline int grid_for(int64_t n) {
+    int64_t g = std::min<int64_t>(std::max<int64_t>(n, 1), 148 * 32);
+    return (int)g;
+}
+
+inline Dims dims_of(const e3j_plan* p) { return Dims{p->nq, p->d, p->dp, p->P, p->D}; }
+
+// workspace layout shared by fwd and bwd: [rowptr | colptr | sender_perm | kernel scratch]
+struct WorkspaceLayout {
+    size_t rowptr, colptr, perm, scratch, total;
+};
+WorkspaceLayout layout(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, bool bwd) {
+    WorkspaceLayout L{};
+    size_t off = 0;
+    L.rowptr = off; off = align_up(off + 4 * (size_t)(n_nodes + 1), 256);
+    L.colptr = off; if (bwd) off = align_up(off + 4 * (size_t)(n_nodes + 1), 256);
+    L.perm = off;   if (bwd) off = align_up(off + 4 * (size_t)std::max<int64_t>(n_edges, 1), 256);
+    L.scratch = off;
+    const FastKernels* fk = fast_lookup(plan);
+    if (fk) off += bwd ? fk->bwd_scratch_bytes(n_nodes, n_edges) : fk->fwd_scratch_bytes(n_nodes, n_edges);
+    L.total = align_up(off, 256);
+    return L;
+}
+
+int check_workspace(const void* ws, size_t have, size_t need) {
+    if (need == 0) return E3J_OK;
+    if (!ws || ((uintptr_t)ws & 255u) || have < need) return E3J_ERR_WORKSPACE;
+    return E3J_OK;
+}
+
+}  // namespace
+}  // namespace e3j
+
+using namespace e3j;
+
+extern "C" {
+
+int e3j_plan_create(e3j_plan** out, const char* irreps_in, int sh_lmax, const char* irreps_out,
+                    int out_lmax, unsigned flags) {
+    if (!out || !irreps_in) return E3J_ERR_INVALID_ARG;
+    *out = nullptr;
+    e3j_plan* plan = new (std::nothrow) e3j_plan();
+    if (!plan) return E3J_ERR_INVALID_ARG;
+    int st = E3J_ERR_INVALID_ARG;
+    try {
+        st = build_plan(*plan, irreps_in, sh_lmax, irreps_out, out_lmax, flags);
+        if (st == E3J_OK && !(flags & E3J_PLAN_GENERIC_ONLY)) plan->fast_id = fast_find(plan->signature.c_str());
+    } catch (...) {
+        st = E3J_ERR_INVALID_ARG;
+    }
+    if (st != E3J_OK) { delete plan; return st; }
+    *out = plan;
+    return E3J_OK;
+}
+
+int e3j_plan_destroy(e3j_plan* plan) {
+    if (!plan) return E3J_OK;
+    int prev = 0;
+    const bool have_dev = cudaGetDevice(&prev) == cudaSuccess;
+    for (DeviceTables& t : plan->dev) {
+        if (t.base && cudaSetDevice(t.device) == cudaSuccess) cudaFree(t.base);
+    }
+    if (have_dev && !plan->dev.empty()) cudaSetDevice(prev);
+    delete plan;
+    return E3J_OK;
+}
+
+int e3j_plan_info(const e3j_plan* plan, e3j_plan_info_t* info) {
+    if (!plan || !info) return E3J_ERR_INVALID_ARG;
+    info->n_channels = plan->nq; info->d_in = plan->d; info->d_sh = plan->dp;
+    info->n_paths = plan->P; info->d_out = plan->D; info->nnz = (int)plan->rec.size();
+    info->n_pairs = plan->n_pairs; info->specialised = plan->fast_id >= 0 ? 1 : 0;
+    return E3J_OK;
+}
+
+int e3j_plan_paths(const e3j_plan* plan, e3j_path_info_t* paths, int capacity) {
+    if (!plan || !paths || capacity < plan->P) return E3J_ERR_INVALID_ARG;
+    std::copy(plan->paths.begin(), plan->paths.end(), paths);
+    return plan->P;
+}
+
+int e3j_plan_records(const e3j_plan* plan, int32_t* i0, int32_t* i1, int32_t* i2, int32_t* i3,
+                     double* val, int capacity) {
+    if (!plan || !i0 || !i1 || !i2 || !i3 || !val) return E3J_ERR_INVALID_ARG;
+    const int n = (int)plan->rec.size();
+    if (capacity < n) return E3J_ERR_INVALID_ARG;
+    for (int r = 0; r < n; ++r) {
+        i0[r] = plan->rec[r].i0; i1[r] = plan->rec[r].i1; i2[r] = plan->rec[r].i2;
+        i3[r] = plan->rec[r].i3; val[r] = plan->rec[r].val;
+    }
+    return n;
+}
+
+int e3j_graph_prepare(int64_t n_nodes, int64_t n_edges, const int32_t* senders,
+                      const int32_t* receivers, int32_t* rowptr, int32_t* sender_perm,
+                      int32_t* colptr, void* stream) {
+    if (n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
+        return E3J_ERR_INVALID_ARG;
+    if (n_edges > 0 && (!senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    if ((sender_perm == nullptr) != (colptr == nullptr)) return E3J_ERR_INVALID_ARG;
+    return graph_prepare(n_nodes, n_edges, senders, receivers, rowptr, sender_perm, colptr,
+                         (cudaStream_t)stream);
+}
+
+int e3j_graph_validate(int64_t n_nodes, int64_t n_edges, const int32_t* senders,
+                       const int32_t* receivers, int32_t* status, void* stream) {
+    if (n_nodes < 0 || n_edges < 0 || !status) return E3J_ERR_INVALID_ARG;
+    if (n_edges > 0 && (!senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    return graph_validate(n_nodes, n_edges, senders, receivers, status, (cudaStream_t)stream);
+}
+
+size_t e3j_conv_fwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges) {
+    if (!plan || n_nodes < 0 || n_edges < 0) return 0;
+    return layout(plan, n_nodes, n_edges, false).total;
+}
+
+size_t e3j_conv_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges) {
+    if (!plan || n_nodes < 0 || n_edges < 0) return 0;
+    return layout(plan, n_nodes, n_edges, true).total;
+}
+
+int e3j_conv_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                 const float* sh, const float* w, const int32_t* senders,
+                 const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                 size_t workspace_bytes, void* stream) {
+    if (!plan || n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
+        return E3J_ERR_INVALID_ARG;
+    if (n_nodes == 0) return E3J_OK;
+    if (!out || !x) return E3J_ERR_INVALID_ARG;
+    if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const WorkspaceLayout L = layout(plan, n_nodes, n_edges, false);
+    if (int s = check_workspace(workspace, workspace_bytes, L.total)) return s;
+    char* ws = (char*)workspace;
+
+    const FastKernels* fk = fast_lookup(plan);
+    if (fk && n_edges > 0) {
+        ConvArgs a{};
+        a.n_nodes = n_nodes; a.n_edges = n_edges; a.x = x; a.sh = sh; a.w = w;
+        a.senders = senders; a.receivers = receivers; a.rowptr = rowptr; a.out = out;
+        a.workspace = ws + L.scratch; a.workspace_bytes = workspace_bytes - L.scratch; a.stream = st;
+        return fk->conv_fwd(a);
+    }
+    if (!rowptr) {
+        int32_t* rp = (int32_t*)(ws + L.rowptr);
+        if (int s = graph_prepare(n_nodes, n_edges, senders, receivers, rp, nullptr, nullptr, st)) return s;
+        rowptr = rp;
+    }
+    DeviceTables t;
+    if (int s = get_device_tables(plan, t)) return s;
+    generic::conv_fwd_kernel<false><<<grid_for(n_nodes), 256, 0, st>>>(t, dims_of(plan), n_nodes, x, sh, w,
+                                                                      senders, rowptr, out);
+    return after_launch();
+}
+
+int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                 const float* sh, const float* w, const int32_t* senders,
+                 const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                 const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
+                 float* grad_w, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!plan || n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
+        return E3J_ERR_INVALID_ARG;
+    if (n_nodes == 0) return E3J_OK;
+    if (!x || !grad_out) return E3J_ERR_INVALID_ARG;
+    if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    if ((sender_perm == nullptr) != (colptr == nullptr)) return E3J_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const WorkspaceLayout L = layout(plan, n_nodes, n_edges, true);
+    if (int s = check_workspace(workspace, workspace_bytes, L.total)) return s;
+    char* ws = (char*)workspace;
+    if (grad_x && !sender_perm) {
+        int32_t* cp = (int32_t*)(ws + L.colptr);
+        int32_t* pm = (int32_t*)(ws + L.perm);
+        if (int s = graph_prepare(n_nodes, n_edges, senders, receivers, nullptr, pm, cp, st)) return s;
+        sender_perm = pm; colptr = cp;
+    }
+    const FastKernels* fk = fast_lookup(plan);
+    if (fk && n_edges > 0) {
+        ConvArgs a{};
+        a.n_nodes = n_nodes; a.n_edges = n_edges; a.x = x; a.sh = sh; a.w = w;
+        a.senders = senders; a.receivers = receivers; a.rowptr = rowptr;
+        a.sender_perm = sender_perm; a.colptr = colptr; a.grad_out = grad_out;
+        a.grad_x = grad_x; a.grad_sh = grad_sh; a.grad_w = grad_w;
+        a.workspace = ws + L.scratch; a.workspace_bytes = workspace_bytes - L.scratch; a.stream = st;
+        return fk->conv_bwd(a);
+    }
+    DeviceTables t;
+    if (int s = get_device_tables(plan, t)) return s;
+    const Dims dm = dims_of(plan);
+    if ((grad_w || grad_sh) && n_edges > 0) {
+        generic::conv_bwd_edge_kernel<false><<<grid_for(n_edges), 256, 0, st>>>(
+            t, dm, n_edges, x, sh, w, senders, receivers, grad_out, grad_w, grad_sh);
+        if (int s = after_launch()) return s;
+    }
+    if (grad_x) {
+        generic::conv_bwd_node_kernel<false><<<grid_for(n_nodes), 256, 0, st>>>(
+            t, dm, n_nodes, sh, w, receivers, sender_perm, colptr, grad_out, grad_x);
+        if (int s = after_launch()) return s;
+    }
+    return E3J_OK;
+}
+
+int e3j_tp_fwd(const e3j_plan* plan, int64_t rows, const float* x1, const float* x2,
+               const float* w, float* out, void* stream) {
+    if (!plan || rows < 0) return E3J_ERR_INVALID_ARG;
+    if (rows == 0) return E3J_OK;
+    if (!x1 || !x2 || !w || !out) return E3J_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const FastKernels* fk = fast_lookup(plan);
+    if (fk && fk->tp_fwd) return fk->tp_fwd(rows, x1, x2, w, out, st);
+    DeviceTables t;
+    if (int s = get_device_tables(plan, t)) return s;
+    generic::conv_fwd_kernel<true><<<grid_for(rows), 256, 0, st>>>(t, dims_of(plan), rows, x1, x2, w, nullptr,
+                                                                  nullptr, out);
+    return after_launch();
+}
+
+int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float* x2,
+               const float* w, const float* grad_out, float* grad_x1, float* grad_x2,
+               float* grad_w, void* stream) {
+    if (!plan || rows < 0) return E3J_ERR_INVALID_ARG;
+    if (rows == 0) return E3J_OK;
+    if (!x1 || !x2 || !w || !grad_out) return E3J_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const FastKernels* fk = fast_lookup(plan);
+    if (fk && fk->tp_bwd) return fk->tp_bwd(rows, x1, x2, w, grad_out, grad_x1, grad_x2, grad_w, st);
+    DeviceTables t;
+    if (int s = get_device_tables(plan, t)) return s;
+    const Dims dm = dims_of(plan);
+    if (grad_w || grad_x2) {
+        generic::conv_bwd_edge_kernel<true><<<grid_for(rows), 256, 0, st>>>(t, dm, rows, x1, x2, w, nullptr,
+                                                                           nullptr, grad_out, grad_w, grad_x2);
+        if (int s = after_launch()) return s;
+    }
+    if (grad_x1) {
+        generic::conv_bwd_node_kernel<true><<<grid_for(rows), 256, 0, st>>>(t, dm, rows, x2, w, nullptr, nullptr,
+                                                                           nullptr, grad_out, grad_x1);
+        if (int s = after_launch()) return s;
+    }
+    return E3J_OK;
+}
+
+const char* e3j_status_string(int status) {
+    switch (status) {
+        case E3J_OK: return "ok";
+        case E3J_ERR_INVALID_ARG: return "invalid argument";
+        case E3J_ERR_BAD_IRREPS: return "irreps descriptor does not parse";
+        case E3J_ERR_MUL_NOT_UNIFORM: return "input irreps must share one multiplicity";
+        case E3J_ERR_UNSUPPORTED: return "unsupported plan (a dimension exceeds 255, l > 8, or no path couples)";
+        case E3J_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case E3J_ERR_CUDA: return "CUDA runtime error";
+        case E3J_ERR_GRAPH: return "graph invalid (receivers not sorted or index out of range)";
+        default: return "unknown status";
+    }
+}
+
+int e3j_last_cuda_error(void) { return g_last_cuda_error; }
+int64_t e3j_launch_count(void) { return g_launch_count.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,54 @@
+// Internal helpers shared by the CUDA translation units of libe3j.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+
+#include "plan.hpp"
+
+namespace e3j {
+
+extern thread_local int g_last_cuda_error;
+extern std::atomic<int64_t> g_launch_count;
+
+inline int cuda_status(cudaError_t err) {
+    if (err == cudaSuccess) return E3J_OK;
+    g_last_cuda_error = (int)err;
+    return E3J_ERR_CUDA;
+}
+
+#define E3J_CUDA_TRY(expr)                                   \
+    do {                                                     \
+        const int _st = ::e3j::cuda_status((expr));          \
+        if (_st != E3J_OK) return _st;                       \
+    } while (0)
+
+// Call after every kernel launch: counts it and converts a launch error to a status.
+inline int after_launch() {
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return cuda_status(cudaGetLastError());
+}
+
+// Device tables of `plan` on the current device (uploaded on first use).
+int get_device_tables(const e3j_plan* plan, DeviceTables& out);
+
+struct Dims {
+    int nq, d, dp, P, D;
+};
+
+// Scalar description of a graph launch shared by the generic and specialised paths.
+struct ConvArgs {
+    int64_t n_nodes, n_edges;
+    const float *x, *sh, *w;
+    const int32_t *senders, *receivers, *rowptr, *sender_perm, *colptr;
+    const float* grad_out;
+    float *out, *grad_x, *grad_sh, *grad_w;
+    void* workspace;
+    size_t workspace_bytes;
+    cudaStream_t stream;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace e3j

@@ -1,0 +1,26 @@
+// Internal: registry of signature-specialised kernels (generated, compiled ahead of time).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+
+#include "common.cuh"
+
+namespace e3j {
+
+struct FastKernels {
+    const char* signature;  // plan signature this entry was generated for
+    size_t (*fwd_scratch_bytes)(int64_t n_nodes, int64_t n_edges);
+    size_t (*bwd_scratch_bytes)(int64_t n_nodes, int64_t n_edges);
+    int (*conv_fwd)(const ConvArgs&);
+    int (*conv_bwd)(const ConvArgs&);
+    int (*tp_fwd)(int64_t rows, const float* x1, const float* x2, const float* w, float* out, cudaStream_t);
+    int (*tp_bwd)(int64_t rows, const float* x1, const float* x2, const float* w, const float* g,
+                  float* gx1, float* gx2, float* gw, cudaStream_t);
+};
+
+// Index of the entry generated for `signature`, or -1.
+int fast_find(const char* signature);
+// Entry selected at plan creation, or nullptr (generic kernels).
+const FastKernels* fast_lookup(const e3j_plan* plan);
+
+}  // namespace e3j

@@ -1,0 +1,194 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle, element by element.
+
+Tolerance (fp32 arithmetic against an fp64 reference): max abs error <= 1e-5 * max|oracle| per
+irreducible block; results must be bit-identical from run to run.
+"""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+import paper_2609_35099_b200 as e3j
+from oracle import conv as oconv
+from paper_2609_35099_b200 import workloads
+from parity_util import assert_blockwise_close, blocks_of_paths
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _cuda(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def make_case(config, n_atoms=None, irreps_out="default", flags=0):
+    c = workloads.CONFIGS[config]
+    iro = c["irreps_out"] if irreps_out == "default" else irreps_out
+    olm = c["out_lmax"] if iro is None else -1
+    wl = workloads.make_graph(config, n_atoms)
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], iro, olm, flags)
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], iro, None if olm < 0 else olm)
+    x, y, w, g = workloads.make_features(wl, plan.n_paths, plan.d_out)
+    return wl, plan, cp, x, y, w, g
+
+
+def run_conv_parity(wl, plan, cp, x, y, w, g, prepared=True):
+    n, e = wl.n_nodes, wl.n_edges
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    dx, dy, dw, dg = _cuda(x), _cuda(y), _cuda(w), _cuda(g)
+    if prepared:
+        rowptr, perm, colptr = e3j.e3j_graph_prepare(n, snd, rcv)
+    else:
+        rowptr = perm = colptr = None
+    out = e3j.e3j_conv_fwd(plan, dx, dy, dw, snd, rcv, rowptr)
+    gx, gy, gw = e3j.e3j_conv_bwd(plan, dx, dy, dw, snd, rcv, dg, rowptr, perm, colptr)
+    out2 = e3j.e3j_conv_fwd(plan, dx, dy, dw, snd, rcv, rowptr)
+    gx2, gy2, gw2 = e3j.e3j_conv_bwd(plan, dx, dy, dw, snd, rcv, dg, rowptr, perm, colptr)
+    torch.cuda.synchronize()
+    for a, b in ((out, out2), (gx, gx2), (gy, gy2), (gw, gw2)):
+        assert torch.equal(a, b), "results differ between two runs"
+    ref = oconv.conv_fwd(cp, x, y, w, wl.senders, wl.receivers)
+    rx, ry, rw = oconv.conv_bwd(cp, x, y, w, wl.senders, wl.receivers, g)
+    worst = [
+        assert_blockwise_close(out.cpu().numpy(), ref, blocks_of_paths(cp.paths, "out"), what="out"),
+        assert_blockwise_close(gx.cpu().numpy(), rx, blocks_of_paths(cp.paths, "x"), what="grad_x"),
+        assert_blockwise_close(gy.cpu().numpy(), ry, blocks_of_paths(cp.paths, "sh"), what="grad_sh"),
+        assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="grad_w"),
+    ]
+    return worst
+
+
+@pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
+@pytest.mark.parametrize("config,n_atoms", [(1, None), (2, 192), (3, 300), (5, 3000)])
+def test_conv_small(config, n_atoms, flags):
+    worst = run_conv_parity(*make_case(config, n_atoms, flags=flags))
+    assert max(worst) < 1e-5
+
+
+@pytest.mark.parametrize("config", [2, 3])
+def test_conv_full_size(config):
+    """Configs 2 and 3 at their full size, every element."""
+    worst = run_conv_parity(*make_case(config))
+    assert max(worst) < 1e-5
+
+
+def test_conv_natural_parity_outputs():
+    worst = run_conv_parity(*make_case(2, 192, irreps_out=workloads.NATURAL_PARITY_OUT))
+    assert max(worst) < 1e-5
+
+
+def test_conv_without_prepared_graph():
+    worst = run_conv_parity(*make_case(1), prepared=False)
+    assert max(worst) < 1e-5
+
+
+@pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
+def test_isolated_nodes_ragged_rows_and_duplicates(flags):
+    """Receivers without edges get zero rows; silent senders zero gradients; duplicate edges
+    and self-loops are ordinary edges; one very long row."""
+    rng = np.random.default_rng(42)
+    c = workloads.CONFIGS[2]
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], None, 3, flags)
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], None, 3)
+    n = 41
+    deg = rng.integers(0, 9, size=n)
+    deg[[0, 7, 8, 40]] = 0
+    deg[20] = 700  # a hub
+    rcv = np.repeat(np.arange(n), deg).astype(np.int32)
+    snd = rng.integers(0, n - 3, size=len(rcv)).astype(np.int32)  # last nodes never send
+    snd[:5] = rcv[:5]  # self loops
+    snd[10:14] = snd[10]  # duplicates
+    e = len(rcv)
+    wl = workloads.Workload(config=2, name="edge", irreps_in=c["irreps_in"], sh_lmax=3, irreps_out=None,
+                            out_lmax=3, n_nodes=n, n_edges=e, senders=snd, receivers=rcv)
+    x = rng.standard_normal((n, plan.d_in, plan.n_channels)).astype(np.float32)
+    y = rng.standard_normal((e, plan.d_sh)).astype(np.float32)
+    w = rng.standard_normal((e, plan.n_paths, plan.n_channels)).astype(np.float32)
+    g = rng.standard_normal((n, plan.d_out, plan.n_channels)).astype(np.float32)
+    worst = run_conv_parity(wl, plan, cp, x, y, w, g)
+    assert max(worst) < 1e-5
+    out = e3j.e3j_conv_fwd(plan, _cuda(x), _cuda(y), _cuda(w), _cuda(snd), _cuda(rcv))
+    assert torch.count_nonzero(out[[0, 7, 8, 40]]) == 0
+
+
+@pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
+def test_empty_graph(flags):
+    plan = e3j.e3j_plan_create("128x0e+128x1o", 3, None, 3, flags)
+    n = 5
+    x = torch.randn((n, plan.d_in, plan.n_channels), device=DEV)
+    empty_i = torch.zeros(0, dtype=torch.int32, device=DEV)
+    out = torch.full((n, plan.d_out, plan.n_channels), 7.0, device=DEV)
+    e3j.e3j_conv_fwd(plan, x, torch.zeros((0, plan.d_sh), device=DEV),
+                     torch.zeros((0, plan.n_paths, plan.n_channels), device=DEV), empty_i, empty_i, out=out)
+    assert torch.count_nonzero(out) == 0
+    gx, gy, gw = e3j.e3j_conv_bwd(plan, x, torch.zeros((0, plan.d_sh), device=DEV),
+                                  torch.zeros((0, plan.n_paths, plan.n_channels), device=DEV), empty_i,
+                                  empty_i, torch.randn_like(out))
+    assert torch.count_nonzero(gx) == 0 and gy.numel() == 0 and gw.numel() == 0
+
+
+@pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
+@pytest.mark.parametrize("rows", [1, 333])
+def test_tensor_product(rows, flags):
+    c = workloads.CONFIGS[4]
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], None, 3, flags)
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], None, 3)
+    x1, x2, w, g = workloads.make_tp_rows(rows, plan.n_paths, plan.d_out)
+    d = [_cuda(a) for a in (x1, x2, w, g)]
+    out = e3j.e3j_tp_fwd(plan, d[0], d[1], d[2])
+    g1, g2, gw = e3j.e3j_tp_bwd(plan, d[0], d[1], d[2], d[3])
+    out_b = e3j.e3j_tp_fwd(plan, d[0], d[1], d[2])
+    g1b, g2b, gwb = e3j.e3j_tp_bwd(plan, d[0], d[1], d[2], d[3])
+    for a, b in ((out, out_b), (g1, g1b), (g2, g2b), (gw, gwb)):
+        assert torch.equal(a, b)
+    ref = oconv.tp_fwd(cp, x1, x2, w)
+    r1, r2, rw = oconv.tp_bwd(cp, x1, x2, w, g)
+    assert_blockwise_close(out.cpu().numpy(), ref, blocks_of_paths(cp.paths, "out"), what="tp out")
+    assert_blockwise_close(g1.cpu().numpy(), r1, blocks_of_paths(cp.paths, "x"), what="tp grad_x1")
+    assert_blockwise_close(g2.cpu().numpy(), r2, blocks_of_paths(cp.paths, "sh"), what="tp grad_x2")
+    assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="tp grad_w")
+
+
+def test_optional_gradients_can_be_skipped():
+    wl, plan, cp, x, y, w, g = make_case(1)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    full = e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, _cuda(g))
+    only_x = e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, _cuda(g), grad_sh=False, grad_w=False)
+    only_w = e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, _cuda(g), grad_x=False, grad_sh=False)
+    assert only_x[1] is None and only_x[2] is None and torch.equal(only_x[0], full[0])
+    assert only_w[0] is None and torch.equal(only_w[2], full[2])
+
+
+def test_graph_prepare_matches_numpy():
+    for config, n_atoms in [(1, None), (2, 192), (5, 3000)]:
+        wl = workloads.make_graph(config, n_atoms)
+        rowptr, perm, colptr = e3j.e3j_graph_prepare(wl.n_nodes, _cuda(wl.senders), _cuda(wl.receivers))
+        n = wl.n_nodes
+        assert np.array_equal(rowptr.cpu().numpy(), np.searchsorted(wl.receivers, np.arange(n + 1), side="left"))
+        assert np.array_equal(perm.cpu().numpy(), np.argsort(wl.senders, kind="stable"))
+        assert np.array_equal(colptr.cpu().numpy(),
+                              np.concatenate([[0], np.cumsum(np.bincount(wl.senders, minlength=n))]))
+    # a hub sender exercises the long-bucket sort
+    rng = np.random.default_rng(3)
+    n, e = 50, 5000
+    rcv = np.sort(rng.integers(0, n, e)).astype(np.int32)
+    snd = np.where(rng.random(e) < 0.5, 7, rng.integers(0, n, e)).astype(np.int32)
+    rowptr, perm, colptr = e3j.e3j_graph_prepare(n, _cuda(snd), _cuda(rcv))
+    assert np.array_equal(perm.cpu().numpy(), np.argsort(snd, kind="stable"))
+
+
+def test_graph_validate_reports_bad_graphs():
+    good_s = torch.tensor([0, 1, 2], dtype=torch.int32, device=DEV)
+    good_r = torch.tensor([0, 0, 2], dtype=torch.int32, device=DEV)
+    assert e3j.e3j_graph_validate(3, good_s, good_r) == 0
+    assert e3j.e3j_graph_validate(3, good_s, torch.tensor([1, 0, 2], dtype=torch.int32, device=DEV)) == -7
+    assert e3j.e3j_graph_validate(2, good_s, good_r) == -7
+
+
+def test_workspace_errors_are_reported():
+    wl, plan, cp, x, y, w, g = make_case(1)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    tiny = torch.empty(16, dtype=torch.uint8, device=DEV)
+    with pytest.raises(ValueError):
+        e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, _cuda(g), workspace=tiny)

@@ -1,0 +1,111 @@
+"""Host logic of libe3j (CPU only): the library loads, exports every declared symbol, and its
+plan builder (ladder-operator coefficients) agrees with the oracle (Racah closed form)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2609_35099_b200 as e3j
+from oracle import cg
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2609_35099_b200 import build
+    build.build()
+
+
+def test_library_exports_every_declared_symbol(repo_root):
+    header = open(os.path.join(repo_root, "include", "e3j.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    names = set(re.findall(r"\b(e3j_[a-z0-9_]+)\s*\(", header))
+    assert {"e3j_plan_create", "e3j_conv_fwd", "e3j_conv_bwd", "e3j_plan_destroy", "e3j_tp_fwd",
+            "e3j_tp_bwd", "e3j_graph_prepare"} <= names
+    lib = ctypes.CDLL(str(e3j.library_path()))
+    for n in sorted(names):
+        assert hasattr(lib, n), f"{n} declared in e3j.h but not exported"
+
+
+SIGNATURES = [
+    ("8x0e+8x1o", 2, "0e+1o+1e+2e+2o", -1),
+    ("128x0e+128x1o", 3, None, 3),
+    ("128x0e+128x1o", 3, "0e+1o+2e+3o", -1),
+    ("64x0e+64x1o+64x2e+64x3o", 3, None, 3),
+    ("128x0e+128x1o+128x2e", 3, None, 3),
+    ("4x0e+4x0o+4x1o+4x1e+4x2e+4x2o", 2, None, 4),
+    ("2x3o+2x4e", 2, None, -1),
+]
+
+
+@pytest.mark.parametrize("sig", SIGNATURES)
+def test_ladder_coefficients_equal_racah_coefficients(sig):
+    irreps_in, lmax, irreps_out, out_lmax = sig
+    plan = e3j.e3j_plan_create(irreps_in, lmax, irreps_out, out_lmax)
+    C, i3, paths, nq = cg.dense_coupling(irreps_in, lmax, irreps_out, None if out_lmax < 0 else out_lmax)
+    info = e3j.e3j_plan_info(plan)
+    assert (info["n_channels"], info["d_in"], info["d_sh"], info["n_paths"], info["d_out"]) == \
+        (nq, C.shape[1], C.shape[2], len(paths), C.shape[0])
+    assert info["nnz"] == np.count_nonzero(C)
+    assert info["n_pairs"] == np.count_nonzero(np.abs(C).sum(axis=2))
+    i0, i1, i2, k, val = e3j.e3j_plan_records(plan)
+    dense = np.zeros_like(C)
+    dense[i0, i1, i2] = val
+    assert np.abs(dense - C).max() < 1e-13
+    assert np.array_equal(k, i3[i0])
+    order = np.lexsort((i2, i1, i0))
+    assert np.array_equal(order, np.arange(len(i0)))  # sorted by (i0, i1, i2)
+    for got, want in zip(e3j.e3j_plan_paths(plan), paths):
+        assert (got["in_index"], got["l1"], got["p1"], got["l2"], got["L"], got["p"], got["x_off"],
+                got["y_off"], got["out_off"]) == \
+            (want.in_index, want.l1, want.p1, want.l2, want.L, want.p, want.x_off, want.y_off, want.out_off)
+
+
+def test_high_degree_ladder_blocks_match_racah():
+    lib = ctypes.CDLL(str(e3j.library_path()))  # noqa: F841  (loads the builder)
+    for l1, l2, outs in [(5, 4, "1e+4e+9e"), (6, 6, "0e+6e+12e"), (8, 3, "5o+8o+11o")]:
+        plan = e3j.e3j_plan_create(f"1x{l1}e", l2, outs, -1)
+        i0, i1, i2, k, val = e3j.e3j_plan_records(plan)
+        for p in e3j.e3j_plan_paths(plan):
+            if p["l2"] != l2:
+                continue
+            blk = cg.real_cg_block(l1, l2, p["L"])
+            sel = k == e3j.e3j_plan_paths(plan).index(p)
+            dense = np.zeros_like(blk)
+            dense[i0[sel] - p["out_off"], i1[sel], i2[sel] - p["y_off"]] = val[sel]
+            assert np.abs(dense - blk).max() < 1e-12
+
+
+@pytest.mark.parametrize("bad,status", [
+    ("", -2), ("8x", -2), ("8x0z", -2), ("8x0e++8x1o", -2), ("8x0e+4x1o", -3), ("1x9e", -4)])
+def test_bad_descriptors_return_status_codes(bad, status):
+    with pytest.raises(e3j.E3JError) as err:
+        e3j.e3j_plan_create(bad, 2)
+    assert err.value.status == status
+
+
+def test_no_coupling_path_is_an_error():
+    with pytest.raises(e3j.E3JError) as err:
+        e3j.e3j_plan_create("4x0e", 1, "3e")
+    assert err.value.status == -4
+
+
+def test_status_strings():
+    assert e3j.e3j_status_string(0) == "ok"
+    assert "workspace" in e3j.e3j_status_string(-5)
+
+
+def test_compute_calls_fail_loudly_without_a_device():
+    torch = pytest.importorskip("torch")
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    plan = e3j.e3j_plan_create("4x0e+4x1o", 1)
+    x = torch.zeros((2, 4, 4))
+    with pytest.raises(TypeError):
+        e3j.e3j_tp_fwd(plan, x, torch.zeros((2, 4)), torch.zeros((2, plan.n_paths, 4)))
+    # straight through the C ABI with non-null dummy pointers: the CUDA error surfaces as a status
+    lib = e3j._load()
+    dummy = ctypes.c_void_p(256)
+    st = lib.e3j_tp_fwd(plan.handle, 1, dummy, dummy, dummy, dummy, None)
+    assert st == -6
