@@ -105,6 +105,13 @@ int e3j_plan_create(e3j_plan** out, const char* irreps_in, int sh_lmax, const ch
                     int out_lmax, unsigned flags);
 int e3j_plan_destroy(e3j_plan* plan);
 int e3j_plan_info(const e3j_plan* plan, e3j_plan_info_t* info);
+/* Canonical text of the plan's signature (multiplicity | input irreps | sh_lmax | paths);
+ * specialised kernels are selected by it.  The string is owned by the plan. */
+const char* e3j_plan_signature(const e3j_plan* plan);
+/* Reads (and clears) the plan's sticky device status word on the current device into the HOST
+ * word *status: 0 = fine, 1 = a bounded wait inside a specialised kernel gave up (the kernel
+ * then returned early and its outputs are invalid).  Synchronises the device. */
+int e3j_plan_device_status(const e3j_plan* plan, int32_t* status);
 /* Copies up to `capacity` path descriptors (host memory); returns P or an error. */
 int e3j_plan_paths(const e3j_plan* plan, e3j_path_info_t* paths, int capacity);
 /* Copies the coefficient records, sorted by (i0,i1,i2), into HOST arrays of

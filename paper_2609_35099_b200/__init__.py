@@ -19,7 +19,7 @@ from pathlib import Path
 
 __all__ = [
     "E3JError", "Plan", "library_path", "e3j_plan_create", "e3j_plan_destroy", "e3j_plan_info",
-    "e3j_plan_paths", "e3j_plan_records", "e3j_graph_prepare", "e3j_graph_validate",
+    "e3j_plan_paths", "e3j_plan_records", "e3j_plan_signature", "e3j_plan_device_status", "e3j_graph_prepare", "e3j_graph_validate",
     "e3j_conv_fwd_workspace_bytes", "e3j_conv_bwd_workspace_bytes", "e3j_conv_fwd", "e3j_conv_bwd",
     "e3j_tp_fwd", "e3j_tp_bwd", "e3j_status_string", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
 ]
@@ -69,6 +69,10 @@ def _load():
     lib.e3j_plan_info.argtypes = [vp, ctypes.POINTER(_PlanInfo)]
     lib.e3j_plan_paths.argtypes = [vp, ctypes.POINTER(_PathInfo), i32]
     lib.e3j_plan_records.argtypes = [vp, vp, vp, vp, vp, vp, i32]
+    lib.e3j_plan_signature.argtypes = [vp]
+    lib.e3j_plan_signature.restype = ctypes.c_char_p
+    lib.e3j_plan_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
+    lib.e3j_plan_device_status.restype = i32
     lib.e3j_graph_prepare.argtypes = [i64, i64, vp, vp, vp, vp, vp, vp]
     lib.e3j_graph_validate.argtypes = [i64, i64, vp, vp, vp, vp]
     lib.e3j_conv_fwd_workspace_bytes.argtypes = [vp, i64, i64]
@@ -131,6 +135,17 @@ def e3j_plan_destroy(plan: Plan) -> None:
 
 def e3j_plan_info(plan: Plan) -> dict:
     return {name: getattr(plan, name) for name, _ in _PlanInfo._fields_}
+
+
+def e3j_plan_signature(plan: Plan) -> str:
+    return _load().e3j_plan_signature(plan.handle).decode()
+
+
+def e3j_plan_device_status(plan: Plan) -> int:
+    """Sticky device status of the plan on the current device (0 = fine); synchronises."""
+    st = ctypes.c_int32(0)
+    _check(_load().e3j_plan_device_status(plan.handle, ctypes.byref(st)), "e3j_plan_device_status")
+    return int(st.value)
 
 
 def e3j_plan_paths(plan: Plan) -> list[dict]:

@@ -65,6 +65,7 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
     const size_t o_r0 = reserve(nb), o_r1 = reserve(nb), o_r2 = reserve(nb);
     const size_t o_s0 = reserve(4 * s0.size()), o_s1 = reserve(4 * s1.size()), o_s2 = reserve(4 * s2.size());
     const size_t o_ip = reserve(4 * i0_path.size()), o_po = reserve(4 * path_off.size());
+    const size_t o_st = reserve(256);
     std::vector<char> host(off, 0);
     std::memcpy(host.data() + o_r0, r0.data(), nb);
     std::memcpy(host.data() + o_r1, r1.data(), nb);
@@ -89,6 +90,7 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
     t.i2_start = (const int32_t*)(b + o_s2);
     t.i0_path = (const int32_t*)(b + o_ip);
     t.path_out_off = (const int32_t*)(b + o_po);
+    t.status = (int32_t*)(b + o_st);
     plan->dev.push_back(t);
     out = t;
     return E3J_OK;
@@ -115,7 +117,8 @@ WorkspaceLayout layout(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, b
     L.perm = off;   if (bwd) off = align_up(off + 4 * (size_t)std::max<int64_t>(n_edges, 1), 256);
     L.scratch = off;
     const FastKernels* fk = fast_lookup(plan);
-    if (fk) off += bwd ? fk->bwd_scratch_bytes(n_nodes, n_edges) : fk->fwd_scratch_bytes(n_nodes, n_edges);
+    if (fk && bwd && fk->bwd_scratch_bytes) off += fk->bwd_scratch_bytes(n_nodes, n_edges);
+    if (fk && !bwd && fk->fwd_scratch_bytes) off += fk->fwd_scratch_bytes(n_nodes, n_edges);
     L.total = align_up(off, 256);
     return L;
 }
@@ -168,6 +171,18 @@ int e3j_plan_info(const e3j_plan* plan, e3j_plan_info_t* info) {
     info->n_channels = plan->nq; info->d_in = plan->d; info->d_sh = plan->dp;
     info->n_paths = plan->P; info->d_out = plan->D; info->nnz = (int)plan->rec.size();
     info->n_pairs = plan->n_pairs; info->specialised = plan->fast_id >= 0 ? 1 : 0;
+    return E3J_OK;
+}
+
+const char* e3j_plan_signature(const e3j_plan* plan) { return plan ? plan->signature.c_str() : nullptr; }
+
+int e3j_plan_device_status(const e3j_plan* plan, int32_t* status) {
+    if (!plan || !status) return E3J_ERR_INVALID_ARG;
+    DeviceTables t;
+    if (int s = get_device_tables(plan, t)) return s;
+    E3J_CUDA_TRY(cudaDeviceSynchronize());
+    E3J_CUDA_TRY(cudaMemcpy(status, t.status, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (*status != 0) E3J_CUDA_TRY(cudaMemset(t.status, 0, sizeof(int32_t)));
     return E3J_OK;
 }
 
@@ -232,11 +247,14 @@ int e3j_conv_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
     char* ws = (char*)workspace;
 
     const FastKernels* fk = fast_lookup(plan);
-    if (fk && n_edges > 0) {
+    if (fk && fk->conv_fwd && n_edges > 0) {
+        DeviceTables t;
+        if (int s = get_device_tables(plan, t)) return s;
         ConvArgs a{};
         a.n_nodes = n_nodes; a.n_edges = n_edges; a.x = x; a.sh = sh; a.w = w;
         a.senders = senders; a.receivers = receivers; a.rowptr = rowptr; a.out = out;
         a.workspace = ws + L.scratch; a.workspace_bytes = workspace_bytes - L.scratch; a.stream = st;
+        a.status = t.status;
         return fk->conv_fwd(a);
     }
     if (!rowptr) {
@@ -273,8 +291,11 @@ int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
         sender_perm = pm; colptr = cp;
     }
     const FastKernels* fk = fast_lookup(plan);
-    if (fk && n_edges > 0) {
+    if (fk && fk->conv_bwd && n_edges > 0) {
+        DeviceTables t;
+        if (int s = get_device_tables(plan, t)) return s;
         ConvArgs a{};
+        a.status = t.status;
         a.n_nodes = n_nodes; a.n_edges = n_edges; a.x = x; a.sh = sh; a.w = w;
         a.senders = senders; a.receivers = receivers; a.rowptr = rowptr;
         a.sender_perm = sender_perm; a.colptr = colptr; a.grad_out = grad_out;

@@ -47,6 +47,7 @@ struct ConvArgs {
     void* workspace;
     size_t workspace_bytes;
     cudaStream_t stream;
+    int32_t* status;  // device status word of the plan on this device
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

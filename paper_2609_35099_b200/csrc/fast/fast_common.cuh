@@ -1,0 +1,123 @@
+// Building blocks of the signature-specialised kernels (sm_100a).
+//
+// Data movement: edge-local operands (weights, harmonics) stream through a ring of
+// shared-memory stages filled by bulk asynchronous copies (cp.async.bulk, completion
+// counted on an mbarrier); sender rows are gathered into the same stage by one bulk
+// copy per edge.  One producer warp issues the copies, the consumer warps wait on the
+// stage's "full" barrier and hand the stage back through its "empty" barrier.
+// No multicast, no tensor maps: every copy is a contiguous, 16-byte aligned range.
+//
+// Every wait is bounded: after kSpinLimit failed polls a warp records an error in the
+// status word, and the CTA drains and returns instead of spinning forever.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace e3j {
+namespace fast {
+
+constexpr uint32_t kSpinLimit = 1u << 22;  // polls of mbarrier.try_wait before giving up
+constexpr int kStatusTimeout = 1;          // value stored in the device status word
+
+// ---------------------------------------------------------------- vector helpers
+__device__ __forceinline__ float4 vmul(const float4 a, const float4 b) {
+    return make_float4(a.x * b.x, a.y * b.y, a.z * b.z, a.w * b.w);
+}
+__device__ __forceinline__ float2 vmul(const float2 a, const float2 b) { return make_float2(a.x * b.x, a.y * b.y); }
+__device__ __forceinline__ void vfma(float4& acc, const float a, const float4 b) {
+    acc.x = fmaf(a, b.x, acc.x); acc.y = fmaf(a, b.y, acc.y); acc.z = fmaf(a, b.z, acc.z); acc.w = fmaf(a, b.w, acc.w);
+}
+__device__ __forceinline__ void vfma(float2& acc, const float a, const float2 b) {
+    acc.x = fmaf(a, b.x, acc.x); acc.y = fmaf(a, b.y, acc.y);
+}
+__device__ __forceinline__ void vfma(float4& acc, const float4 a, const float4 b) {
+    acc.x = fmaf(a.x, b.x, acc.x); acc.y = fmaf(a.y, b.y, acc.y); acc.z = fmaf(a.z, b.z, acc.z); acc.w = fmaf(a.w, b.w, acc.w);
+}
+__device__ __forceinline__ void vfma(float2& acc, const float2 a, const float2 b) {
+    acc.x = fmaf(a.x, b.x, acc.x); acc.y = fmaf(a.y, b.y, acc.y);
+}
+// sum over the lane's channels of a*b, added to t
+__device__ __forceinline__ float vdot_acc(const float4 a, const float4 b, float t) {
+    return fmaf(a.w, b.w, fmaf(a.z, b.z, fmaf(a.y, b.y, fmaf(a.x, b.x, t))));
+}
+__device__ __forceinline__ float vdot_acc(const float2 a, const float2 b, float t) {
+    return fmaf(a.y, b.y, fmaf(a.x, b.x, t));
+}
+__device__ __forceinline__ void vzero(float4& v) { v = make_float4(0.f, 0.f, 0.f, 0.f); }
+__device__ __forceinline__ void vzero(float2& v) { v = make_float2(0.f, 0.f); }
+__device__ __forceinline__ float4 vadd(const float4 a, const float4 b) {
+    return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+}
+__device__ __forceinline__ float2 vadd(const float2 a, const float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
+
+template <int V> struct VecOf;
+template <> struct VecOf<4> { using type = float4; };
+template <> struct VecOf<2> { using type = float2; };
+
+// ---------------------------------------------------------------- mbarrier / bulk copy (PTX)
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and records the failure) if the phase never completes.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1;
+    if (status) atomicExch(status, kStatusTimeout);
+    return false;
+}
+// Contiguous global -> shared copy; both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// ---------------------------------------------------------------- A-matrix tables
+// For every (i0,i1) pair slot: where its records start and how many there are.
+struct PairRec {
+    int16_t start, count;
+};
+
+struct FwdParams {
+    const float* x; const float* sh; const float* w;
+    const int32_t* senders; const int32_t* receivers;
+    float* out;
+    int64_t n_nodes, n_edges, chunk;   // chunk = edges per CTA (multiple of 4)
+    float* partial;                    // [G][2][D*NQ] boundary-row partial sums
+    int32_t* part_recv;                // [G][2] receiver of the head / tail partial, or -1
+    int32_t* status;                   // device status word (0 = fine)
+};
+
+// Sums the pieces of every receiver row that was split between CTAs, in CTA order.
+__global__ void fwd_fixup_kernel(int n_cta, int row_f4, const float4* __restrict__ partial,
+                                 const int32_t* __restrict__ part_recv, float4* __restrict__ out);
+
+}  // namespace fast
+}  // namespace e3j

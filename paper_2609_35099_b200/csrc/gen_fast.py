@@ -1,0 +1,260 @@
+#!/usr/bin/env python
+"""Generator of the signature-specialised kernel sources under csrc/fast/.
+
+    python paper_2609_35099_b200/csrc/gen_fast.py [--check]
+
+For every entry of fast/signatures.json this script asks the library's own plan builder
+(e3j_plan_create / e3j_plan_records of an already built libe3j.so) for the coefficient records of
+that signature and writes fast/sig_<name>.cu: a struct of compile-time constants, the record
+tables, and fully unrolled per-edge bodies in which every (i0,i1) pair is a straight-line FMA on
+registers (the counterpart of the paper's trace-time specialisation of the coefficient loop).
+fast/registry_entries.inc lists the generated entries.  The generated files are committed, so a
+clean checkout builds without running this script; --check verifies that they are current.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+from pathlib import Path
+
+HERE = Path(__file__).resolve().parent
+sys.path.insert(0, str(HERE.parent.parent))
+
+
+def load_records(sig):
+    import paper_2609_35099_b200 as e3j
+    plan = e3j.e3j_plan_create(sig["irreps_in"], sig["sh_lmax"], sig.get("irreps_out"),
+                               sig.get("out_lmax", -1), e3j.E3J_PLAN_GENERIC_ONLY)
+    info = e3j.e3j_plan_info(plan)
+    paths = e3j.e3j_plan_paths(plan)
+    i0, i1, i2, i3, val = e3j.e3j_plan_records(plan)
+    recs = [(int(a), int(b), int(c), int(k), float(v)) for a, b, c, k, v in zip(i0, i1, i2, i3, val)]
+    signature = e3j.e3j_plan_signature(plan)
+    return info, paths, recs, signature
+
+
+def partition_rows(costs, n_groups):
+    """Contiguous partition of rows into n_groups minimising the largest group cost (DP)."""
+    n = len(costs)
+    n_groups = min(n_groups, n)
+    pre = [0]
+    for c in costs:
+        pre.append(pre[-1] + c)
+    INF = float("inf")
+    best = [[INF] * (n + 1) for _ in range(n_groups + 1)]
+    cut = [[0] * (n + 1) for _ in range(n_groups + 1)]
+    best[0][0] = 0
+    for g in range(1, n_groups + 1):
+        for j in range(g, n + 1):
+            for i in range(g - 1, j):
+                v = max(best[g - 1][i], pre[j] - pre[i])
+                if v < best[g][j]:
+                    best[g][j], cut[g][j] = v, i
+    bounds = [n]
+    j = n
+    for g in range(n_groups, 0, -1):
+        j = cut[g][j]
+        bounds.append(j)
+    return list(reversed(bounds))
+
+
+def fmt_float(v: float) -> str:
+    """Shortest decimal literal that round-trips the float32 value."""
+    import numpy as np
+    f = float(np.float32(v))
+    s = f"{f:.9g}"
+    if "." not in s and "e" not in s:
+        s += ".0"
+    return s + "f"
+
+
+class Sig:
+    def __init__(self, sig):
+        self.cfg = sig
+        self.name = sig["name"]
+        self.info, self.paths, self.recs, self.signature = load_records(sig)
+        self.NQ, self.DIN, self.DSH = self.info["n_channels"], self.info["d_in"], self.info["d_sh"]
+        self.P, self.D, self.NNZ = self.info["n_paths"], self.info["d_out"], self.info["nnz"]
+        self.V = sig["V"]
+        assert self.NQ % (32 * self.V) == 0, "channels must fill whole warps"
+        # pairs in (i0, i1) order with their records
+        self.pairs = []  # (i0, i1, k, [(i2, val)])
+        for i0, i1, i2, k, v in self.recs:
+            if self.pairs and self.pairs[-1][0] == i0 and self.pairs[-1][1] == i1:
+                self.pairs[-1][3].append((i2, v))
+            else:
+                self.pairs.append((i0, i1, k, [(i2, v)]))
+        assert len(self.pairs) == self.info["n_pairs"]
+        self.row_path = [None] * self.D
+        for k, p in enumerate(self.paths):
+            for m in range(2 * p["L"] + 1):
+                self.row_path[p["out_off"] + m] = k
+        self.row_pairs = [[] for _ in range(self.D)]
+        for pi, (i0, i1, k, rl) in enumerate(self.pairs):
+            self.row_pairs[i0].append(pi)
+
+    # ---------------------------------------------------------------- forward
+    def fwd_layout(self):
+        FW = self.cfg["FW"]
+        costs = []
+        for row in range(self.D):
+            k = self.row_path[row]
+            l1 = self.paths[k]["l1"]
+            first_row_of_path = row == self.paths[k]["out_off"]
+            costs.append(len(self.row_pairs[row]) * 1.0 + ((2 * l1 + 1) * 1.0 + 0.5 if first_row_of_path else 0.0) + 0.3)
+        bounds = partition_rows(costs, FW)
+        while len(bounds) < FW + 1:
+            bounds.append(bounds[-1])
+        a0, slots = [0], []  # slot -> pair index or None
+        for g in range(FW):
+            for row in range(bounds[g], bounds[g + 1]):
+                slots += self.row_pairs[row]
+            while len(slots) % 4:
+                slots.append(None)
+            a0.append(len(slots))
+        return bounds, a0, slots
+
+    def emit(self) -> str:
+        V, NQ = self.V, self.NQ
+        FW, FT, FS = self.cfg["FW"], self.cfg["FT"], self.cfg["FS"]
+        bounds, a0, slots = self.fwd_layout()
+        slot_of_pair = {pi: s for s, pi in enumerate(slots) if pi is not None}
+        rmax = max(bounds[g + 1] - bounds[g] for g in range(FW))
+        vec = f"float{V}"
+        # record tables in slot order
+        rec_val, rec_i2, pair_tab = [], [], []
+        for pi in slots:
+            if pi is None:
+                pair_tab.append((len(rec_val), 0))
+                continue
+            rl = self.pairs[pi][3]
+            pair_tab.append((len(rec_val), len(rl)))
+            for i2, v in rl:
+                rec_val.append(v); rec_i2.append(i2)
+        assert len(rec_val) == self.NNZ
+        S = f"Sig_{self.name}"
+        o = []
+        o.append(f"// GENERATED by csrc/gen_fast.py from fast/signatures.json -- do not edit.")
+        o.append(f"// signature: {self.signature}")
+        o.append(f"// {self.cfg['irreps_in']} (x) harmonics l<={self.cfg['sh_lmax']}: P={self.P} D={self.D} "
+                 f"nnz={self.NNZ} pairs={len(self.pairs)}")
+        o.append('#include "fast_fwd.cuh"')
+        o.append('#include "fast_launch.cuh"')
+        o.append("")
+        o.append("namespace e3j {\nnamespace fast {\nnamespace {")
+        o.append(f"__device__ const PairRec kPair_{self.name}[{len(pair_tab)}] = {{")
+        o.append("    " + ", ".join(f"{{{s},{c}}}" for s, c in pair_tab) + "};")
+        o.append(f"__device__ const float kVal_{self.name}[{self.NNZ}] = {{")
+        o.append("    " + ", ".join(fmt_float(v) for v in rec_val) + "};")
+        o.append(f"__device__ const unsigned char kI2_{self.name}[{self.NNZ}] = {{")
+        o.append("    " + ", ".join(str(i) for i in rec_i2) + "};")
+        o.append("")
+        o.append(f"struct {S} {{")
+        o.append(f"    static constexpr int NQ = {NQ}, DIN = {self.DIN}, DSH = {self.DSH}, P = {self.P}, D = {self.D};")
+        o.append(f"    static constexpr int NNZ = {self.NNZ}, NPAIR = {len(self.pairs)}, V = {V};")
+        o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, F_RMAX = {rmax}, F_APAD = {len(slots)};")
+        o.append(f"    using Vec = {vec};")
+        o.append(f"    __device__ static __forceinline__ PairRec pair_rec(int i) {{ return kPair_{self.name}[i]; }}")
+        o.append(f"    __device__ static __forceinline__ float rec_val(int i) {{ return kVal_{self.name}[i]; }}")
+        o.append(f"    __device__ static __forceinline__ unsigned char rec_i2(int i) {{ return kI2_{self.name}[i]; }}")
+
+        def table_fn(fname, values):
+            o.append(f"    __device__ static __forceinline__ int {fname}(int g) {{")
+            o.append("        switch (g) {")
+            for i, v in enumerate(values):
+                o.append(f"            case {i}: return {v};")
+            o.append(f"            default: return {values[-1]};")
+            o.append("        }\n    }")
+
+        table_fn("f_row0", bounds)
+        table_fn("f_a0", a0)
+
+        # ---- fwd_edge
+        o.append(f"    __device__ static __forceinline__ void fwd_edge(const int g, Vec (&acc)[F_RMAX], "
+                 f"const Vec* __restrict__ xs, const Vec* __restrict__ ss, const float* __restrict__ As) {{")
+        o.append(f"        constexpr int NQV = NQ / V;")
+        o.append("        switch (g) {")
+        for g in range(FW):
+            o.append(f"        case {g}: {{")
+            rows = range(bounds[g], bounds[g + 1])
+            need_x = sorted({self.pairs[pi][1] for row in rows for pi in self.row_pairs[row]})
+            for i1 in need_x:
+                o.append(f"            const Vec x{i1} = xs[{i1} * NQV];")
+            loaded_a = set()
+            cur_path = None
+            for row in rows:
+                k = self.row_path[row]
+                if k != cur_path:
+                    cur_path = k
+                    p = self.paths[k]
+                    o.append(f"            const Vec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
+                    used = sorted({self.pairs[pi][1] for r2 in rows if self.row_path[r2] == k for pi in self.row_pairs[r2]})
+                    for i1 in used:
+                        o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                for pi in self.row_pairs[row]:
+                    slot = slot_of_pair[pi]
+                    q, lane = slot // 4, "xyzw"[slot % 4]
+                    if q not in loaded_a:
+                        loaded_a.add(q)
+                        o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
+                    i1 = self.pairs[pi][1]
+                    o.append(f"            vfma(acc[{row - bounds[g]}], a{q}.{lane}, sx{k}_{i1});")
+            o.append("        } break;")
+        o.append("        default: break;")
+        o.append("        }\n    }")
+
+        # ---- fwd_store
+        o.append(f"    __device__ static __forceinline__ void fwd_store(const int g, const Vec (&acc)[F_RMAX], Vec* __restrict__ dst) {{")
+        o.append(f"        constexpr int NQV = NQ / V;")
+        o.append("        switch (g) {")
+        for g in range(FW):
+            o.append(f"        case {g}:")
+            for row in range(bounds[g], bounds[g + 1]):
+                o.append(f"            dst[{row} * NQV] = acc[{row - bounds[g]}];")
+            o.append("            break;")
+        o.append("        default: break;")
+        o.append("        }\n    }")
+        o.append("};")
+        o.append("}  // namespace")
+        o.append("}  // namespace fast")
+        o.append("")
+        o.append(f"extern const FastKernels kFast_{self.name};")
+        o.append(f"const FastKernels kFast_{self.name} = {{")
+        o.append(f'    "{self.signature}",')
+        o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, nullptr, &fast::launch_fwd<fast::{S}>, nullptr, nullptr, nullptr}};")
+        o.append("}  // namespace e3j")
+        return "\n".join(o) + "\n"
+
+
+def generate():
+    sigs = json.loads((HERE / "fast" / "signatures.json").read_text())
+    files = {}
+    for sig in sigs:
+        files[f"sig_{sig['name']}.cu"] = Sig(sig).emit()
+    entries = "// GENERATED by csrc/gen_fast.py -- one E3J_FAST_ENTRY(name) per specialised signature\n"
+    entries += "".join(f"E3J_FAST_ENTRY(kFast_{sig['name']})\n" for sig in sigs)
+    files["registry_entries.inc"] = entries
+    return files
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--check", action="store_true", help="exit 1 if a generated file is out of date")
+    args = ap.parse_args()
+    files = generate()
+    stale = []
+    for name, text in files.items():
+        path = HERE / "fast" / name
+        if not path.exists() or path.read_text() != text:
+            stale.append(name)
+            if not args.check:
+                path.write_text(text)
+    if args.check and stale:
+        print("stale generated files:", ", ".join(stale))
+        sys.exit(1)
+    print("generated" if not args.check else "up to date", ", ".join(files))
+
+
+if __name__ == "__main__":
+    main()

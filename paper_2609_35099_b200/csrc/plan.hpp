@@ -37,6 +37,7 @@ struct DeviceTables {
     const PackedRecord* by_i2 = nullptr;
     const int32_t* i2_start = nullptr;  // [d'+1]
     const int32_t* path_out_off = nullptr;  // [P+1]
+    int32_t* status = nullptr;  // sticky device status word (0 = fine), see e3j_plan_device_status
 };
 
 }  // namespace e3j
