@@ -42,7 +42,7 @@ struct FwdSmem {
 };
 
 template <class S>
-__global__ void __launch_bounds__((S::FW * (S::NQ / (32 * S::V)) + 1) * 32, 1)
+__global__ void __launch_bounds__((S::FW * (S::NQ / (32 * S::V)) + 1) * 32, S::FC)
 fast_fwd_kernel(const FwdParams p) {
     using Vec = typename VecOf<S::V>::type;
     using L = FwdSmem<S>;

@@ -6,7 +6,8 @@
 namespace e3j {
 namespace fast {
 
-constexpr int kMaxCtas = 192;  // upper bound on the number of SMs used for scratch sizing
+constexpr int kMaxSms = 192;       // upper bound on the SM count, for scratch sizing
+constexpr size_t kPartRecvBytes = 8192;  // slot of the [n_cta][2] boundary receiver ids
 
 inline int sm_count() {
     static thread_local int cached_dev = -1, cached = 0;
@@ -15,25 +16,25 @@ inline int sm_count() {
     if (dev != cached_dev) {
         int n = 0;
         if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-        cached = n > kMaxCtas ? kMaxCtas : n;
+        cached = n > kMaxSms ? kMaxSms : n;
         cached_dev = dev;
     }
     return cached;
 }
 
-// scratch: [part_recv: 2*kMaxCtas ints, padded to 2048 B][partial rows: 2*kMaxCtas*D*NQ floats]
+// scratch: [part_recv: 2*n_cta ints in an 8 KB slot][partial rows: 2*n_cta*D*NQ floats], n_cta <= kMaxSms*S::FC
 template <class S>
 size_t fwd_scratch_bytes(int64_t, int64_t) {
-    return 2048 + sizeof(float) * 2 * (size_t)kMaxCtas * S::D * S::NQ;
+    return kPartRecvBytes + sizeof(float) * 2 * (size_t)kMaxSms * S::FC * S::D * S::NQ;
 }
 
 template <class S>
 int launch_fwd(const ConvArgs& a) {
     using L = FwdSmem<S>;
-    static_assert(L::total <= 227 * 1024, "forward stage ring does not fit in shared memory");
-    static_assert(2 * kMaxCtas * sizeof(int32_t) <= 2048, "part_recv does not fit its slot");
+    static_assert(L::total * S::FC + 1024 * S::FC <= 228 * 1024, "forward stage ring does not fit in shared memory");
+    static_assert(2 * kMaxSms * S::FC * sizeof(int32_t) <= kPartRecvBytes, "part_recv does not fit its slot");
     if (a.workspace_bytes < fwd_scratch_bytes<S>(a.n_nodes, a.n_edges)) return E3J_ERR_WORKSPACE;
-    const int n_cta = sm_count();
+    const int n_cta = sm_count() * S::FC;
     static thread_local int attr_dev = -1;
     int dev = 0;
     E3J_CUDA_TRY(cudaGetDevice(&dev));
@@ -47,7 +48,7 @@ int launch_fwd(const ConvArgs& a) {
     const int64_t per = (a.n_edges + n_cta - 1) / n_cta;
     p.chunk = (per + 3) / 4 * 4;
     p.part_recv = reinterpret_cast<int32_t*>(a.workspace);
-    p.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(a.workspace) + 2048);
+    p.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(a.workspace) + kPartRecvBytes);
     p.status = a.status;
     constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 1) * 32;
     fast_fwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);

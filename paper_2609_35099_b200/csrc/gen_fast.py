@@ -117,7 +117,7 @@ class Sig:
 
     def emit(self) -> str:
         V, NQ = self.V, self.NQ
-        FW, FT, FS = self.cfg["FW"], self.cfg["FT"], self.cfg["FS"]
+        FW, FT, FS, FC = self.cfg["FW"], self.cfg["FT"], self.cfg["FS"], self.cfg["FC"]
         bounds, a0, slots = self.fwd_layout()
         slot_of_pair = {pi: s for s, pi in enumerate(slots) if pi is not None}
         rmax = max(bounds[g + 1] - bounds[g] for g in range(FW))
@@ -153,7 +153,7 @@ class Sig:
         o.append(f"struct {S} {{")
         o.append(f"    static constexpr int NQ = {NQ}, DIN = {self.DIN}, DSH = {self.DSH}, P = {self.P}, D = {self.D};")
         o.append(f"    static constexpr int NNZ = {self.NNZ}, NPAIR = {len(self.pairs)}, V = {V};")
-        o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, F_RMAX = {rmax}, F_APAD = {len(slots)};")
+        o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, FC = {FC}, F_RMAX = {rmax}, F_APAD = {len(slots)};")
         o.append(f"    using Vec = {vec};")
         o.append(f"    __device__ static __forceinline__ PairRec pair_rec(int i) {{ return kPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float rec_val(int i) {{ return kVal_{self.name}[i]; }}")
