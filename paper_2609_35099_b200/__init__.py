@@ -25,7 +25,10 @@ __all__ = [
 ]
 
 E3J_PLAN_GENERIC_ONLY = 1
-_LIB_PATH = Path(__file__).resolve().parent / "libe3j.so"
+import os as _os
+
+# E3J_LIBRARY selects another build of the same library (e.g. an experimental variant).
+_LIB_PATH = Path(_os.environ.get("E3J_LIBRARY") or (Path(__file__).resolve().parent / "libe3j.so"))
 _lib = None
 
 

@@ -153,14 +153,14 @@ class Sig:
         o.append(f"struct {S} {{")
         o.append(f"    static constexpr int NQ = {NQ}, DIN = {self.DIN}, DSH = {self.DSH}, P = {self.P}, D = {self.D};")
         o.append(f"    static constexpr int NNZ = {self.NNZ}, NPAIR = {len(self.pairs)}, V = {V};")
-        o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, FC = {FC}, F_RMAX = {rmax}, F_APAD = {len(slots)};")
+        o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, FC = {FC}, F_RMAX = {rmax}, F_APAD = {len(slots)}, F_NREC = {max(c for _, c in pair_tab)}, F_MAXREG = {self.cfg.get("F_MAXREG", 255)};")
         o.append(f"    using Vec = {vec};")
         o.append(f"    __device__ static __forceinline__ PairRec pair_rec(int i) {{ return kPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float rec_val(int i) {{ return kVal_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ unsigned char rec_i2(int i) {{ return kI2_{self.name}[i]; }}")
 
         def table_fn(fname, values):
-            o.append(f"    __device__ static __forceinline__ int {fname}(int g) {{")
+            o.append(f"    static constexpr int {fname}(int g) {{")
             o.append("        switch (g) {")
             for i, v in enumerate(values):
                 o.append(f"            case {i}: return {v};")
@@ -171,12 +171,12 @@ class Sig:
         table_fn("f_a0", a0)
 
         # ---- fwd_edge
-        o.append(f"    __device__ static __forceinline__ void fwd_edge(const int g, Vec (&acc)[F_RMAX], "
+        o.append(f"    template <int G>")
+        o.append(f"    __device__ static __forceinline__ void fwd_edge(Vec (&acc)[F_RMAX], "
                  f"const Vec* __restrict__ xs, const Vec* __restrict__ ss, const float* __restrict__ As) {{")
         o.append(f"        constexpr int NQV = NQ / V;")
-        o.append("        switch (g) {")
         for g in range(FW):
-            o.append(f"        case {g}: {{")
+            o.append(f"        if constexpr (G == {g}) {{")
             rows = range(bounds[g], bounds[g + 1])
             need_x = sorted({self.pairs[pi][1] for row in rows for pi in self.row_pairs[row]})
             for i1 in need_x:
@@ -200,21 +200,19 @@ class Sig:
                         o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
                     i1 = self.pairs[pi][1]
                     o.append(f"            vfma(acc[{row - bounds[g]}], a{q}.{lane}, sx{k}_{i1});")
-            o.append("        } break;")
-        o.append("        default: break;")
-        o.append("        }\n    }")
+            o.append("        }")
+        o.append("    }")
 
         # ---- fwd_store
-        o.append(f"    __device__ static __forceinline__ void fwd_store(const int g, const Vec (&acc)[F_RMAX], Vec* __restrict__ dst) {{")
+        o.append(f"    template <int G>")
+        o.append(f"    __device__ static __forceinline__ void fwd_store(const Vec (&acc)[F_RMAX], Vec* __restrict__ dst) {{")
         o.append(f"        constexpr int NQV = NQ / V;")
-        o.append("        switch (g) {")
         for g in range(FW):
-            o.append(f"        case {g}:")
+            o.append(f"        if constexpr (G == {g}) {{")
             for row in range(bounds[g], bounds[g + 1]):
                 o.append(f"            dst[{row} * NQV] = acc[{row - bounds[g]}];")
-            o.append("            break;")
-        o.append("        default: break;")
-        o.append("        }\n    }")
+            o.append("        }")
+        o.append("    }")
         o.append("};")
         o.append("}  // namespace")
         o.append("}  // namespace fast")
