@@ -23,3 +23,4 @@ __global__ void fwd_fixup_kernel(int n_cta, int row_f4, const float4* __restrict
 
 }  // namespace fast
 }  // namespace e3j
+

@@ -2,7 +2,7 @@
 //
 // Work split: the receiver-sorted edge list is cut into one contiguous range per CTA
 // (equal edge counts, so every SM streams the same number of bytes).  A CTA walks its
-// range in tiles of S::FT edges; warp (g, ch) owns output rows
+// range in tiles of S::FT edges; consumer warp (g, ch) owns output rows
 // [S::f_row0(g), S::f_row0(g+1)) and channels [ch*32*V, (ch+1)*32*V) and keeps their
 // running sum for the current receiver in registers.  When the receiver changes the
 // sum is stored (paper, forward algorithm: accumulate over the receiver's edges, store
@@ -13,55 +13,68 @@
 // A[i0,i1] = sum_{i2} C[i0,i1,i2] y[i2] (warp-uniform, kept in shared memory); the
 // per-channel work is then acc[i0] += A[i0,i1] * (s[k] * x[i1]) with s factored out of
 // the path sum (paper, "Factoring out the edge scalar").
+//
+// Warps g, g+FW, ... land on the same SM sub-partition and run the same specialised
+// body, so each sub-partition's instruction stream is one compact loop.  The last warp
+// of the CTA is the producer: it issues the bulk copies of a tile and stages the tile's
+// harmonics and receiver ids.  The warps of a row group compute the group's A entries of
+// the next tile right after finishing the current one.
 #pragma once
 #include "fast_common.cuh"
 
 namespace e3j {
 namespace fast {
 
+#ifdef E3J_PROF
+// Cycle accounting for tuning (debug builds only): [cta][warp][phase] clock ticks.
+__device__ long long g_fwd_prof[1024 * 16 * 8];
+#define E3J_TICK(slot) { const long long _now = clock64(); prof_acc[slot] += _now - prof_t; prof_t = _now; }
+#else
+#define E3J_TICK(slot)
+#endif
+
+// Per A slot: up to two records, A = c0 * y[i2_0] + c1 * y[i2_1].
+struct ASlot {
+    float c0, c1;
+    int i2_0, i2_1;
+};
+
 template <class S>
 struct FwdSmem {
     static constexpr int T = S::FT, NS = S::FS;
     static constexpr int CH = S::NQ / (32 * S::V);
+    static constexpr int NCONS = S::FW * CH;       // consumer warps
     static constexpr int S_EDGE = S::P * S::NQ;    // floats of weights per edge
     static constexpr int X_EDGE = S::DIN * S::NQ;  // floats of one sender row
-    static constexpr int A_WARP = T * S::F_APAD + 32;  // A floats per channel chunk (+ dummy slots)
     static constexpr size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
     static constexpr size_t off_bar = 0;                                  // full[NS], empty[NS]
     static constexpr size_t off_abort = off_bar + 16 * NS;
-    static constexpr size_t off_A = up(off_abort + 4, 16);                // float[CH][A_WARP]
-    static constexpr size_t off_stage = up(off_A + 4 * CH * A_WARP, 128);
+    static constexpr int FL_WARP = S::F_RMAX * 32 * S::V;                 // floats of one warp's store buffer
+    static constexpr size_t off_flush = up(off_abort + 4, 128);           // float[warps][FL_WARP]
+    static constexpr size_t off_stage = up(off_flush + (S::F_BULK_STORE ? 4 * (size_t)NCONS * FL_WARP : 0), 128);
     static constexpr size_t st_s = 0;
     static constexpr size_t st_x = st_s + 4 * (size_t)T * S_EDGE;
-    static constexpr size_t st_y = st_x + 4 * (size_t)T * X_EDGE;
+    static constexpr size_t st_A = st_x + 4 * (size_t)T * X_EDGE;         // A[T][APAD]: scalars, or duplicated pairs when S::PK
+    static constexpr size_t st_y = st_A + (S::PK ? 8 : 4) * (size_t)T * S::F_APAD;
     static constexpr size_t st_r = st_y + 4 * (size_t)T * S::DSH;         // recv[T], change mask
     static constexpr size_t stage_bytes = up(st_r + 4 * (T + 1), 128);
     static constexpr size_t total = off_stage + NS * stage_bytes;
 };
 
-// One warp: row group G, channel chunk ch.  Warps g, g+FW, ... land on the same SM
-// sub-partition and run the same code, which keeps the instruction stream of a
-// sub-partition to one specialised body.
-//
-// There is no dedicated producer warp: the warp whose index equals (tile mod warps)
-// refills a stage (after every warp has released it) with the tile NS steps ahead.
+// ------------------------------------------------------------------------ consumer
 template <class S, int G>
-__device__ __forceinline__ void fwd_warp(const FwdParams& p, unsigned char* smem, const int ch, const int warp,
-                                         const int lane, const int64_t e_begin, const int64_t e_end,
-                                         const int n_tiles) {
-    using Vec = typename VecOf<S::V>::type;
+__device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* smem, const int ch, const int warp,
+                                             const int lane, const int64_t e_begin, const int64_t e_end,
+                                             const int n_tiles) {
+    using Vec = typename VecOf<S::V, S::PK>::type;
+    using AT = typename AOf<S::PK>::type;
     using L = FwdSmem<S>;
-    constexpr int T = L::T, NS = L::NS, NW = S::FW * L::CH;
+    constexpr int T = L::T, NS = L::NS;
     constexpr int NQV = S::NQ / S::V;
-    constexpr int A0 = S::f_a0(G), NP = S::f_a0(G + 1) - A0;
     constexpr int ROW0 = S::f_row0(G), ROW1 = S::f_row0(G + 1);
-    constexpr int NI = (T * NP + 31) / 32;   // A entries computed per lane and tile
-    constexpr int NR = S::F_NREC;            // records per (i0,i1) pair, at most
-    constexpr int YPL = (T * S::DSH + 31) / 32;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
     uint64_t* empty = full + NS;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
-    float* A_w = reinterpret_cast<float*>(smem + L::off_A) + (size_t)ch * L::A_WARP;
     const int cta = blockIdx.x;
     const int vlane = ch * 32 + lane;
     const int64_t row_elems = (int64_t)S::D * S::NQ;
@@ -69,67 +82,38 @@ __device__ __forceinline__ void fwd_warp(const FwdParams& p, unsigned char* smem
     const int next_recv = (e_end < p.n_edges) ? p.receivers[e_end] : -2;
     if (warp == 0 && lane == 0) { p.part_recv[2 * cta] = -1; p.part_recv[2 * cta + 1] = -1; }
 
-    // ---- refill duty: metadata of the next tile this warp will issue, prefetched in registers
-    int duty = warp, m_snd = 0, m_rcv = -1, m_before = -1;
-    float m_y[YPL];
-    auto load_meta = [&](int u) {
-        if (u >= n_tiles) return;
-        const int64_t e0 = e_begin + (int64_t)u * T;
-        const int n_e = (int)min((int64_t)T, e_end - e0);
-        if (lane < n_e) { m_snd = p.senders[e0 + lane]; m_rcv = p.receivers[e0 + lane]; }
-        m_before = (u > 0) ? p.receivers[e0 - 1] : -1;
+    // The CH warps of row group G share the group's A entries of a tile: each lane of the
+    // CH*32 computes entries idx = pl, pl + CH*32, ... (entry idx -> edge idx / NP, slot idx % NP).
+    constexpr int A0 = S::f_a0(G), NP = S::f_a0(G + 1) - A0;
+    constexpr int NI = (T * NP + L::CH * 32 - 1) / (L::CH * 32);
+    ASlot a_tab[NI];
+    int a_dst[NI];
+    {
+        const int pl = ch * 32 + lane;
 #pragma unroll
-        for (int i = 0; i < YPL; ++i) {
-            const int idx = i * 32 + lane;
-            if (idx < n_e * S::DSH) m_y[i] = p.sh[e0 * S::DSH + idx];
-        }
-    };
-    auto issue = [&](int u) {
-        const int stage = u % NS;
-        unsigned char* st = smem + L::off_stage + (size_t)stage * L::stage_bytes;
-        const int64_t e0 = e_begin + (int64_t)u * T;
-        const int n_e = (int)min((int64_t)T, e_end - e0);
-        int* recv_t = reinterpret_cast<int*>(st + L::st_r);
-        float* y_t = reinterpret_cast<float*>(st + L::st_y);
-        int before = __shfl_up_sync(0xffffffffu, m_rcv, 1);
-        if (lane == 0) before = m_before;
-        const unsigned mask = __ballot_sync(0xffffffffu, lane < n_e && m_rcv != before);
-        if (lane < n_e) recv_t[lane] = m_rcv;
-        if (lane == 0) recv_t[T] = (int)mask;
-#pragma unroll
-        for (int i = 0; i < YPL; ++i) {
-            const int idx = i * 32 + lane;
-            if (idx < n_e * S::DSH) y_t[idx] = m_y[i];
-        }
-        __syncwarp();
-        if (lane == 0) {
-            mbar_arrive_expect_tx(&full[stage], (uint32_t)n_e * (uint32_t)(4 * (L::S_EDGE + L::X_EDGE)));
-            bulk_g2s(st + L::st_s, p.w + (size_t)e0 * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE, &full[stage]);
-        }
-        if (lane < n_e)
-            bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE, p.x + (size_t)m_snd * L::X_EDGE, 4u * L::X_EDGE,
-                     &full[stage]);
-    };
-    load_meta(duty);
-    if (duty < NS && duty < n_tiles) { issue(duty); duty += NW; load_meta(duty); }
-
-    // ---- this lane's share of the tile's A entries: A[dst] = sum_r coef[r] * y_tile[src[r]]
-    float a_coef[NI][NR];
-    int a_src[NI][NR], a_dst[NI];
-#pragma unroll
-    for (int i = 0; i < NI; ++i) {
-        const int idx = lane + 32 * i;
-        const bool valid = idx < T * NP;
-        const int e_i = valid ? idx / NP : 0, slot = A0 + (valid ? idx % NP : 0);
-        const PairRec pr = S::pair_rec(slot);
-        a_dst[i] = valid ? e_i * S::F_APAD + slot : T * S::F_APAD + lane;
-#pragma unroll
-        for (int r = 0; r < NR; ++r) {
-            const bool on = valid && r < pr.count;
-            a_coef[i][r] = on ? S::rec_val(pr.start + r) : 0.f;
-            a_src[i][r] = on ? e_i * S::DSH + S::rec_i2(pr.start + r) : 0;
+        for (int i = 0; i < NI; ++i) {
+            const int idx = pl + L::CH * 32 * i;
+            const bool valid = idx < T * NP;
+            const int e_i = valid ? idx / NP : 0, slot = A0 + (valid ? idx % NP : 0);
+            const PairRec pr = S::pair_rec(slot);
+            ASlot a{0.f, 0.f, 0, 0};
+            if (valid && pr.count > 0) { a.c0 = S::rec_val(pr.start); a.i2_0 = e_i * S::DSH + S::rec_i2(pr.start); }
+            if (valid && pr.count > 1) { a.c1 = S::rec_val(pr.start + 1); a.i2_1 = e_i * S::DSH + S::rec_i2(pr.start + 1); }
+            a_tab[i] = a;
+            a_dst[i] = valid ? e_i * S::F_APAD + slot : -1;
         }
     }
+    // A[e][slot] = sum over the slot's records of c * y[e][i2] for one landed tile
+    // (entries of edges beyond the tile's length are computed from stale data and never read)
+    auto make_A = [&](unsigned char* st) {
+        const float* y_t = reinterpret_cast<const float*>(st + L::st_y);
+        AT* A_t = reinterpret_cast<AT*>(st + L::st_A);
+#pragma unroll
+        for (int i = 0; i < NI; ++i)
+            if (a_dst[i] >= 0)
+                a_store(A_t + a_dst[i], fmaf(a_tab[i].c1, y_t[a_tab[i].i2_1], a_tab[i].c0 * y_t[a_tab[i].i2_0]));
+        if constexpr (L::CH > 1) named_barrier_sync(1 + G, L::CH * 32); else __syncwarp();
+    };
 
     Vec acc[S::F_RMAX];
 #pragma unroll
@@ -145,6 +129,9 @@ __device__ __forceinline__ void fwd_warp(const FwdParams& p, unsigned char* smem
             for (int row = ROW0; row < ROW1; ++row) dst[(size_t)row * NQV] = zero;
         }
     };
+    // Finished rows are either stored directly or (S::F_BULK_STORE) staged in shared memory
+    // and written by a bulk asynchronous store, which frees the accumulator registers at once.
+    Vec* fl = reinterpret_cast<Vec*>(smem + L::off_flush) + (size_t)warp * (L::FL_WARP / S::V);
     auto flush = [&](bool at_end) {
         const bool head = seg_first && cur == prev_recv;
         const bool tail = at_end && cur == next_recv;
@@ -158,60 +145,84 @@ __device__ __forceinline__ void fwd_warp(const FwdParams& p, unsigned char* smem
         } else {
             base = p.out + (size_t)cur * row_elems;
         }
-        S::template fwd_store<G>(acc, reinterpret_cast<Vec*>(base) + vlane);
+        if constexpr (S::F_BULK_STORE) {
+            if (lane < ROW1 - ROW0) bulk_wait_read();  // the previous use of the buffer has been read out
+            __syncwarp();
+            S::template fwd_store<G>(acc, fl + lane, 32);
+            fence_async_shared();
+            __syncwarp();
+            if (lane < ROW1 - ROW0) {
+                bulk_s2g(base + (size_t)(ROW0 + lane) * S::NQ + ch * 32 * S::V, fl + lane * 32, 32 * S::V * 4);
+                bulk_commit();
+            }
+        } else {
+            S::template fwd_store<G>(acc, reinterpret_cast<Vec*>(base) + (size_t)ROW0 * NQV + vlane, NQV);
+        }
+    };
+    auto new_receiver = [&](const int r) {
+        if (cur >= 0) { flush(false); seg_first = false; }
+        zero_rows((cur >= 0 ? cur : prev_recv) + 1, r);
+        cur = r;
+#pragma unroll
+        for (int q = 0; q < S::F_RMAX; ++q) vzero(acc[q]);
     };
 
-    for (int t = 0; t < n_tiles; ++t) {
-        const int stage = t % NS, use = t / NS;
-        if (!mbar_wait(&full[stage], use & 1, abort_flag, p.status)) break;
-        const unsigned char* st = smem + L::off_stage + (size_t)stage * L::stage_bytes;
-        const int n_e = (int)min((int64_t)T, e_end - (e_begin + (int64_t)t * T));
+#ifdef E3J_PROF
+    long long prof_acc[6] = {0, 0, 0, 0, 0, 0};
+    long long prof_t = clock64();
+#endif
+    int stage = 0, phase = 0;                 // ring slot of tile t and the parity of its use
+    int left = (int)(e_end - e_begin);        // edges of this CTA not yet consumed
+    bool ok = n_tiles > 0 && mbar_wait(&full[0], 0, abort_flag, p.status);
+    if (ok) make_A(smem + L::off_stage);
+    for (int t = 0; ok && t < n_tiles; ++t) {
+        E3J_TICK(5)
+        const unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
+        const int n_e = min(T, left);
+        left -= T;
         const int* recv_t = reinterpret_cast<const int*>(st + L::st_r);
-        const float* y_t = reinterpret_cast<const float*>(st + L::st_y);
-        // entries of edges beyond n_e are computed from stale data and never read
-#pragma unroll
-        for (int i = 0; i < NI; ++i) {
-            float a = 0.f;
-#pragma unroll
-            for (int r = 0; r < NR; ++r) a = fmaf(a_coef[i][r], y_t[a_src[i][r]], a);
-            A_w[a_dst[i]] = a;
-        }
-        const int mask = recv_t[T];  // bit i: edge i starts a new receiver
-        __syncwarp();
+        unsigned mask = (unsigned)recv_t[T];  // bit i: edge i starts a new receiver
         const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + vlane;
         const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + vlane;
-        const float* As = A_w;
-#pragma unroll 1  // the body is long straight-line code; unrolling it overflows the instruction cache
-        for (int e_i = 0; e_i < n_e; ++e_i) {
-            if ((mask >> e_i) & 1) {
-                const int r = recv_t[e_i];
-                if (cur >= 0) { flush(false); seg_first = false; }
-                zero_rows((cur >= 0 ? cur : prev_recv) + 1, r);
-                cur = r;
-#pragma unroll
-                for (int q = 0; q < S::F_RMAX; ++q) vzero(acc[q]);
+        const AT* As = reinterpret_cast<const AT*>(st + L::st_A);
+        int e_i = 0;
+#pragma unroll 1
+        while (e_i < n_e) {
+            if (e_i + 2 <= n_e && (mask & 3u) == 0u) {
+                // two edges of the current receiver: straight-line, constant offsets
+                S::template fwd_edge<G>(acc, xs, ss, As);
+                S::template fwd_edge<G>(acc, xs + L::X_EDGE / S::V, ss + L::S_EDGE / S::V, As + S::F_APAD);
+                xs += 2 * (L::X_EDGE / S::V); ss += 2 * (L::S_EDGE / S::V); As += 2 * S::F_APAD;
+                e_i += 2; mask >>= 2;
+            } else {
+                if (mask & 1u) new_receiver(recv_t[e_i]);
+                S::template fwd_edge<G>(acc, xs, ss, As);
+                xs += L::X_EDGE / S::V; ss += L::S_EDGE / S::V; As += S::F_APAD;
+                e_i += 1; mask >>= 1;
             }
-            S::template fwd_edge<G>(acc, xs, ss, As);
-            xs += L::X_EDGE / S::V; ss += L::S_EDGE / S::V; As += S::F_APAD;
         }
+        E3J_TICK(2)
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[stage]);
-        if (t + NS == duty && duty < n_tiles) {
-            // every warp has released this stage once empty's phase `use` completes
-            if (!mbar_wait(&empty[stage], use & 1, abort_flag, p.status)) break;
-            issue(duty);
-            duty += NW;
-            load_meta(duty);
+        if (++stage == NS) { stage = 0; phase ^= 1; }
+        if (t + 1 < n_tiles) {
+            // next tile: wait for its data, then this warp's share of its A entries
+            ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
+            E3J_TICK(0)
+            if (ok) make_A(smem + L::off_stage + stage * (int)L::stage_bytes);
+            E3J_TICK(1)
         }
     }
+#ifdef E3J_PROF
+    if (lane == 0 && blockIdx.x < 1024)
+        for (int i = 0; i < 6; ++i) g_fwd_prof[(blockIdx.x * 16 + warp) * 8 + i] = prof_acc[i];
+#endif
     if (!*abort_flag) {
         if (cur >= 0) {
             flush(true);
             if (e_end == p.n_edges) zero_rows(cur + 1, (int)p.n_nodes);
         }
-    } else {
-        // give copies that are still in flight time to land before shared memory is released
-        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        if constexpr (S::F_BULK_STORE) bulk_wait_all();
     }
 }
 
@@ -219,7 +230,7 @@ template <class S, int G>
 struct FwdDispatch {
     template <class... Args>
     __device__ static __forceinline__ void run(const int g, Args&&... args) {
-        if (g == G) fwd_warp<S, G>(args...);
+        if (g == G) fwd_consumer<S, G>(args...);
         else FwdDispatch<S, G + 1>::run(g, args...);
     }
 };
@@ -229,13 +240,94 @@ struct FwdDispatch<S, S::FW> {
     __device__ static __forceinline__ void run(const int, Args&&...) {}
 };
 
+// ------------------------------------------------------------------------ producer
 template <class S>
-__global__ void __launch_bounds__(S::FW * (S::NQ / (32 * S::V)) * 32, S::FC)
+__device__ __forceinline__ void fwd_producer(const FwdParams& p, unsigned char* smem, const int warp, const int lane,
+                                             const int64_t e_begin, const int64_t e_end, const int n_tiles) {
+    using L = FwdSmem<S>;
+    using AT = typename AOf<S::PK>::type;
+    constexpr int T = L::T, NS = L::NS;
+    constexpr int YPL = (T * S::DSH + 31) / 32;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
+    uint64_t* empty = full + NS;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
+    int snd_a = 0, rcv_a = -1, snd_b = 0, rcv_b = -1;
+    float y_a[YPL], y_b[YPL];
+    auto load_meta = [&](int t, int& snd, int& rcv, float (&yv)[YPL]) {
+        if (t >= n_tiles) return;
+        const int64_t e0 = e_begin + (int64_t)t * T;
+        const int n_e = (int)min((int64_t)T, e_end - e0);
+        if (lane < n_e) { snd = p.senders[e0 + lane]; rcv = p.receivers[e0 + lane]; }
+#pragma unroll
+        for (int i = 0; i < YPL; ++i) {
+            const int idx = i * 32 + lane;
+            if (idx < n_e * S::DSH) yv[i] = p.sh[e0 * S::DSH + idx];
+        }
+    };
+    load_meta(0, snd_a, rcv_a, y_a);
+    load_meta(1, snd_b, rcv_b, y_b);
+#ifdef E3J_PROF
+    long long prof_acc[6] = {0, 0, 0, 0, 0, 0};
+    long long prof_t = clock64();
+#endif
+    int armed = 0, last_rcv = -1, stage = 0, phase = 0;
+    for (int t = 0; t < n_tiles; ++t) {
+        // phase of `empty` that ends the previous use of this ring slot
+        if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
+        E3J_TICK(0)
+        unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
+        const int64_t e0 = e_begin + (int64_t)t * T;
+        const int n_e = (int)min((int64_t)T, e_end - e0);
+        int* recv_t = reinterpret_cast<int*>(st + L::st_r);
+        float* y_t = reinterpret_cast<float*>(st + L::st_y);
+        // copies first: they are the long pole
+        if (lane == 0) {
+            mbar_expect_tx(&full[stage], (uint32_t)n_e * (uint32_t)(4 * (L::S_EDGE + L::X_EDGE)));
+            bulk_g2s(st + L::st_s, p.w + (size_t)e0 * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE, &full[stage]);
+        }
+        if (lane < n_e)
+            bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE, p.x + (size_t)snd_a * L::X_EDGE, 4u * L::X_EDGE,
+                     &full[stage]);
+        armed = t + 1;
+        int before = __shfl_up_sync(0xffffffffu, rcv_a, 1);
+        if (lane == 0) before = last_rcv;
+        const unsigned mask = __ballot_sync(0xffffffffu, lane < n_e && rcv_a != before);
+        last_rcv = __shfl_sync(0xffffffffu, rcv_a, n_e - 1);
+        if (lane < n_e) recv_t[lane] = rcv_a;
+        if (lane == 0) recv_t[T] = (int)mask;
+#pragma unroll
+        for (int i = 0; i < YPL; ++i) {
+            const int idx = i * 32 + lane;
+            if (idx < n_e * S::DSH) y_t[idx] = y_a[i];
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[stage]);  // the staged harmonics / receiver ids are in place
+        E3J_TICK(1)
+        snd_a = snd_b; rcv_a = rcv_b;
+#pragma unroll
+        for (int i = 0; i < YPL; ++i) y_a[i] = y_b[i];
+        load_meta(t + 2, snd_b, rcv_b, y_b);
+        if (++stage == NS) { stage = 0; phase ^= 1; }
+    }
+#ifdef E3J_PROF
+    if (lane == 0 && blockIdx.x < 1024)
+        for (int i = 0; i < 6; ++i) g_fwd_prof[(blockIdx.x * 16 + warp) * 8 + i] = prof_acc[i];
+#endif
+    if (*abort_flag) {
+        // let copies already in flight land before the CTA's shared memory is released
+        for (int t = max(0, armed - NS); t < armed; ++t)
+            for (uint32_t it = 0; it < kSpinLimit; ++it)
+                if (mbar_try_wait(&full[t % NS], (t / NS) & 1)) break;
+    }
+}
+
+template <class S>
+__global__ void __launch_bounds__((S::FW * (S::NQ / (32 * S::V)) + 1) * 32, S::FC)
 fast_fwd_kernel(const FwdParams p) {
     using L = FwdSmem<S>;
-    constexpr int T = L::T, NS = L::NS, NW = S::FW * L::CH;
+    constexpr int T = L::T, NS = L::NS, NCONS = L::NCONS;
     static_assert(T <= 31, "the change mask is one 32-bit word");
-    static_assert(NS <= NW, "one warp refills one stage at a time");
+    static_assert(S::F_NREC <= 2, "an A slot holds at most two records");
 
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
@@ -248,12 +340,13 @@ fast_fwd_kernel(const FwdParams p) {
     const int n_tiles = (int)((e_end - e_begin + T - 1) / T);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NW); }
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NCONS); }
         *abort_flag = 0;
         mbar_fence_init();
     }
     __syncthreads();
-    FwdDispatch<S, 0>::run(warp % S::FW, p, smem, warp / S::FW, warp, lane, e_begin, e_end, n_tiles);
+    if (warp == NCONS) fwd_producer<S>(p, smem, warp, lane, e_begin, e_end, n_tiles);
+    else FwdDispatch<S, 0>::run(warp % S::FW, p, smem, warp / S::FW, warp, lane, e_begin, e_end, n_tiles);
 }
 
 }  // namespace fast

@@ -50,7 +50,7 @@ int launch_fwd(const ConvArgs& a) {
     p.part_recv = reinterpret_cast<int32_t*>(a.workspace);
     p.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(a.workspace) + kPartRecvBytes);
     p.status = a.status;
-    constexpr int threads = S::FW * (S::NQ / (32 * S::V)) * 32;
+    constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 1) * 32;  // consumers + one producer warp
     fast_fwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
     fwd_fixup_kernel<<<n_cta, 256, 0, a.stream>>>(n_cta, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),
@@ -60,3 +60,10 @@ int launch_fwd(const ConvArgs& a) {
 
 }  // namespace fast
 }  // namespace e3j
+
+#ifdef E3J_PROF
+// debug builds only: copies the forward kernel's cycle counters to the host
+extern "C" __attribute__((weak)) int e3j_debug_fwd_prof(long long* host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, e3j::fast::g_fwd_prof, sizeof(long long) * n);
+}
+#endif

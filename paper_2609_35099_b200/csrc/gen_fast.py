@@ -110,7 +110,7 @@ class Sig:
         for g in range(FW):
             for row in range(bounds[g], bounds[g + 1]):
                 slots += self.row_pairs[row]
-            while len(slots) % 4:
+            while len(slots) % (2 if self.cfg.get('PK', 0) else 4):
                 slots.append(None)
             a0.append(len(slots))
         return bounds, a0, slots
@@ -121,7 +121,8 @@ class Sig:
         bounds, a0, slots = self.fwd_layout()
         slot_of_pair = {pi: s for s, pi in enumerate(slots) if pi is not None}
         rmax = max(bounds[g + 1] - bounds[g] for g in range(FW))
-        vec = f"float{V}"
+        PK = bool(self.cfg.get("PK", 0))
+        vec = ({2: "u64", 4: "ulonglong2"} if PK else {2: "float2", 4: "float4"})[V]
         # record tables in slot order
         rec_val, rec_i2, pair_tab = [], [], []
         for pi in slots:
@@ -153,7 +154,10 @@ class Sig:
         o.append(f"struct {S} {{")
         o.append(f"    static constexpr int NQ = {NQ}, DIN = {self.DIN}, DSH = {self.DSH}, P = {self.P}, D = {self.D};")
         o.append(f"    static constexpr int NNZ = {self.NNZ}, NPAIR = {len(self.pairs)}, V = {V};")
+        o.append(f"    static constexpr bool PK = {str(PK).lower()};  // packed fp32 pairs (fma.rn.f32x2) or plain fp32")
+        o.append(f"    using AT = {'u64' if PK else 'float'};")
         o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, FC = {FC}, F_RMAX = {rmax}, F_APAD = {len(slots)}, F_NREC = {max(c for _, c in pair_tab)}, F_MAXREG = {self.cfg.get("F_MAXREG", 255)};")
+        o.append(f"    static constexpr bool F_BULK_STORE = {str(bool(self.cfg.get('F_BULK_STORE', 0))).lower()};")
         o.append(f"    using Vec = {vec};")
         o.append(f"    __device__ static __forceinline__ PairRec pair_rec(int i) {{ return kPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float rec_val(int i) {{ return kVal_{self.name}[i]; }}")
@@ -173,7 +177,7 @@ class Sig:
         # ---- fwd_edge
         o.append(f"    template <int G>")
         o.append(f"    __device__ static __forceinline__ void fwd_edge(Vec (&acc)[F_RMAX], "
-                 f"const Vec* __restrict__ xs, const Vec* __restrict__ ss, const float* __restrict__ As) {{")
+                 f"const Vec* __restrict__ xs, const Vec* __restrict__ ss, const AT* __restrict__ As) {{")
         o.append(f"        constexpr int NQV = NQ / V;")
         for g in range(FW):
             o.append(f"        if constexpr (G == {g}) {{")
@@ -182,35 +186,48 @@ class Sig:
             for i1 in need_x:
                 o.append(f"            const Vec x{i1} = xs[{i1} * NQV];")
             loaded_a = set()
-            cur_path = None
+            paths_here = []
             for row in rows:
-                k = self.row_path[row]
-                if k != cur_path:
-                    cur_path = k
-                    p = self.paths[k]
-                    o.append(f"            const Vec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
-                    used = sorted({self.pairs[pi][1] for r2 in rows if self.row_path[r2] == k for pi in self.row_pairs[r2]})
-                    for i1 in used:
-                        o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
-                for pi in self.row_pairs[row]:
-                    slot = slot_of_pair[pi]
-                    q, lane = slot // 4, "xyzw"[slot % 4]
-                    if q not in loaded_a:
-                        loaded_a.add(q)
-                        o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
-                    i1 = self.pairs[pi][1]
-                    o.append(f"            vfma(acc[{row - bounds[g]}], a{q}.{lane}, sx{k}_{i1});")
+                if self.row_path[row] not in paths_here:
+                    paths_here.append(self.row_path[row])
+            for k in paths_here:
+                p = self.paths[k]
+                prow = [r2 for r2 in rows if self.row_path[r2] == k]
+                o.append(f"            const Vec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
+                used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.row_pairs[r2]})
+                for i1 in used:
+                    o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                # round-robin over the rows of the path so that consecutive FMAs hit different accumulators
+                depth = max(len(self.row_pairs[r2]) for r2 in prow)
+                for j in range(depth):
+                    for row in prow:
+                        if j >= len(self.row_pairs[row]):
+                            continue
+                        pi = self.row_pairs[row][j]
+                        slot = slot_of_pair[pi]
+                        if PK:
+                            q, lane = slot // 2, "xy"[slot % 2]
+                            if q not in loaded_a:
+                                loaded_a.add(q)
+                                o.append(f"            const ulonglong2 a{q} = *reinterpret_cast<const ulonglong2*>(As + {2 * q});")
+                        else:
+                            q, lane = slot // 4, "xyzw"[slot % 4]
+                            if q not in loaded_a:
+                                loaded_a.add(q)
+                                o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
+                        i1 = self.pairs[pi][1]
+                        o.append(f"            vfma(acc[{row - bounds[g]}], a{q}.{lane}, sx{k}_{i1});")
             o.append("        }")
         o.append("    }")
 
         # ---- fwd_store
         o.append(f"    template <int G>")
-        o.append(f"    __device__ static __forceinline__ void fwd_store(const Vec (&acc)[F_RMAX], Vec* __restrict__ dst) {{")
-        o.append(f"        constexpr int NQV = NQ / V;")
+        o.append(f"    // writes the group's rows to dst[r * stride] (dst already offset by the lane and the first row)")
+        o.append(f"    __device__ static __forceinline__ void fwd_store(const Vec (&acc)[F_RMAX], Vec* __restrict__ dst, const int stride) {{")
         for g in range(FW):
             o.append(f"        if constexpr (G == {g}) {{")
             for row in range(bounds[g], bounds[g + 1]):
-                o.append(f"            dst[{row} * NQV] = acc[{row - bounds[g]}];")
+                o.append(f"            dst[{row - bounds[g]} * stride] = acc[{row - bounds[g]}];")
             o.append("        }")
         o.append("    }")
         o.append("};")
