@@ -291,7 +291,8 @@ int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
         sender_perm = pm; colptr = cp;
     }
     const FastKernels* fk = fast_lookup(plan);
-    if (fk && fk->conv_bwd && n_edges > 0) {
+    // the specialised sweep produces all three cotangents at once; partial requests use the generic kernels
+    if (fk && fk->conv_bwd && n_edges > 0 && grad_x && grad_sh && grad_w) {
         DeviceTables t;
         if (int s = get_device_tables(plan, t)) return s;
         ConvArgs a{};

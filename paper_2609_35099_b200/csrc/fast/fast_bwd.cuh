@@ -1,0 +1,319 @@
+// Signature-specialised backward convolution, pass 1 (template over a generated struct S).
+//
+// One sweep over the receiver-sorted edges computes the three cotangents of the paper's
+// message-passing-backward equation in the factored form of its "Backward sweep of one
+// edge tile":  with A[i0,i1] = sum_{i2} C y[i2] and k the path (irreducible block) of i0,
+//   u[k,i1]     = sum_{i0 in k} A[i0,i1] * dm[b,i0]            (per channel)
+//   grad_w[e,k] = sum_{i1} x[a,i1] * u[k,i1]
+//   dx_e[i1]    = sum_k s[e,k] * u[k,i1]                       (this edge's share of grad_x[a])
+//   grad_sh[e,i2] = sum_q sum_{pairs} C[i0,i1,i2] * (s[e,k] x[a,i1]) * dm[b,i0]
+// grad_w and grad_sh are edge-local and final.  dx_e is written to a scratch array
+// [E,d,N_q]; pass 2 (bwd_dx_reduce_kernel) adds the rows of every sender in edge order, so no
+// floating-point atomics are needed and the result is bit-reproducible.
+//
+// Work split: equal contiguous edge ranges per CTA; consumer warp (g, ch) owns the paths of
+// group g (whole paths, so grad_w[e,k] is complete inside one warp) and channels
+// [ch*32*V, (ch+1)*32*V).  The rows of dm that a warp needs stay in registers while the receiver
+// does not change.  Per edge the warps exchange their dx_e and grad_sh partial sums through
+// shared memory and add them in a fixed order.  The last warp is the producer: bulk copies of
+// the edge-local operands and the sender rows, staging of harmonics / ids, and the A entries.
+#pragma once
+#include "fast_common.cuh"
+#include "fast_fwd.cuh"  // ASlot
+
+namespace e3j {
+namespace fast {
+
+struct BwdParams {
+    const float* x; const float* sh; const float* w;
+    const int32_t* senders; const int32_t* receivers;
+    const float* grad_out;
+    float* grad_sh; float* grad_w;
+    float* dx_edge;                    // scratch [E][d][N_q]
+    int64_t n_nodes, n_edges, chunk;   // chunk = edges per CTA
+    int32_t* status;
+};
+
+template <class S>
+struct BwdSmem {
+    static constexpr int T = S::BT, NS = S::BS;
+    static constexpr int CH = S::NQ / (32 * S::V);
+    static constexpr int NCONS = S::BW * CH;
+    static constexpr int S_EDGE = S::P * S::NQ;
+    static constexpr int X_EDGE = S::DIN * S::NQ;
+    static constexpr int DYP = 16;                 // grad_sh partial sums per warp (d' padded)
+    static_assert(S::DSH <= DYP, "harmonics beyond l = 3 need a wider reduction");
+    static constexpr size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+    static constexpr size_t off_bar = 0;
+    static constexpr size_t off_xch = off_bar + 16 * NS;                               // exchange barrier
+    static constexpr size_t off_abort = off_xch + 8;
+    static constexpr size_t off_dxs = up(off_abort + 4, 128);                        // float[2][BW][DIN][NQ]
+    static constexpr size_t off_dyp = off_dxs + 4 * 2 * (size_t)S::BW * X_EDGE;      // float[2][NCONS][DYP]
+    static constexpr size_t off_stage = up(off_dyp + 4 * 2 * (size_t)NCONS * DYP, 128);
+    static constexpr size_t st_s = 0;
+    static constexpr size_t st_x = st_s + 4 * (size_t)T * S_EDGE;
+    static constexpr size_t st_A = st_x + 4 * (size_t)T * X_EDGE;
+    static constexpr size_t st_y = st_A + 4 * (size_t)T * S::B_APAD;
+    static constexpr size_t st_r = st_y + 4 * (size_t)T * S::DSH;                    // recv[T], change mask
+    static constexpr size_t stage_bytes = up(st_r + 4 * (T + 1), 128);
+    static constexpr size_t total = off_stage + NS * stage_bytes;
+};
+
+// Sum of v[0..15] over the 32 lanes.  On return lane L holds (in the return value) the total
+// of entry ((L >> 1) & 15) with bit order (b4 b3 b2 b1) -> entry index b4*8 + b3*4 + b2*2 + b1.
+__device__ __forceinline__ float reduce16_over_lanes(float (&v)[16], const int lane) {
+    const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4, b1 = lane & 2;
+    float w8[8], w4[4], w2[2];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const float send = b4 ? v[j] : v[j + 8], keep = b4 ? v[j + 8] : v[j];
+        w8[j] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float send = b3 ? w8[j] : w8[j + 4], keep = b3 ? w8[j + 4] : w8[j];
+        w4[j] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const float send = b2 ? w4[j] : w4[j + 2], keep = b2 ? w4[j + 2] : w4[j];
+        w2[j] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+    const float send = b1 ? w2[0] : w2[1], keep = b1 ? w2[1] : w2[0];
+    float r = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+    r += __shfl_xor_sync(0xffffffffu, r, 1);
+    return r;
+}
+
+template <class S, int G>
+__device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* smem, const int ch, const int warp,
+                                             const int lane, const int64_t e_begin, const int64_t e_end,
+                                             const int n_tiles) {
+    using Vec = typename VecOf<S::V, false>::type;
+    using L = BwdSmem<S>;
+    constexpr int T = L::T, NS = L::NS, NCONS = L::NCONS;
+    constexpr int NQV = S::NQ / S::V;
+    constexpr int ROW0 = S::b_row0(G), NROW = S::b_row0(G + 1) - ROW0;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
+    uint64_t* empty = full + NS;
+    uint64_t* xch = reinterpret_cast<uint64_t*>(smem + L::off_xch);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
+    float* dxs = reinterpret_cast<float*>(smem + L::off_dxs);
+    float* dyp = reinterpret_cast<float*>(smem + L::off_dyp);
+    const int vlane = ch * 32 + lane;
+    const int64_t row_elems = (int64_t)S::D * S::NQ;
+
+    Vec dm[S::B_RMAX];   // this warp's rows of grad_out[receiver]
+#pragma unroll
+    for (int r = 0; r < S::B_RMAX; ++r) vzero(dm[r]);
+
+    int stage = 0, phase = 0, buf = 0, xphase = 0;
+    bool alive = true;
+    int left = (int)(e_end - e_begin);
+    int64_t e = e_begin;
+    for (int t = 0; alive && t < n_tiles; ++t) {
+        if (!mbar_wait(&full[stage], phase, abort_flag, p.status)) break;
+        const unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
+        const int n_e = min(T, left);
+        left -= T;
+        const int* recv_t = reinterpret_cast<const int*>(st + L::st_r);
+        unsigned mask = (unsigned)recv_t[T];
+        const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + vlane;
+        const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + vlane;
+        const float* As = reinterpret_cast<const float*>(st + L::st_A);
+#pragma unroll 1
+        for (int e_i = 0; alive && e_i < n_e; ++e_i, ++e) {
+            if (mask & 1u) {
+                const Vec* g = reinterpret_cast<const Vec*>(p.grad_out + (size_t)recv_t[e_i] * row_elems) +
+                               (size_t)ROW0 * NQV + vlane;
+#pragma unroll
+                for (int r = 0; r < NROW; ++r) dm[r] = g[(size_t)r * NQV];
+            }
+            mask >>= 1;
+            Vec dxp[S::DIN];
+            float dyl[16];
+#pragma unroll
+            for (int i = 0; i < S::DIN; ++i) vzero(dxp[i]);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) dyl[i] = 0.f;
+            Vec* gw = reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + vlane;
+            S::template bwd_edge<G>(dm, xs, ss, As, dxp, dyl, gw);
+            xs += L::X_EDGE / S::V; ss += L::S_EDGE / S::V; As += S::B_APAD;
+
+            // this warp's partial sums -> shared memory
+            const float dy_tot = reduce16_over_lanes(dyl, lane);
+            if ((lane & 1) == 0) {
+                const int idx = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+                dyp[(buf * NCONS + warp) * L::DYP + idx] = dy_tot;
+            }
+            Vec* my = reinterpret_cast<Vec*>(dxs + (size_t)(buf * S::BW + G) * L::X_EDGE) + vlane;
+#pragma unroll
+            for (int i = 0; i < S::DIN; ++i) my[i * NQV] = dxp[i];
+            // every consumer warp has deposited its partial sums (bounded wait, like every other wait here)
+            __syncwarp();
+            if (lane == 0) mbar_arrive(xch);
+            alive = mbar_wait(xch, xphase, abort_flag, p.status);
+            xphase ^= 1;
+            if (!alive) break;
+            // fixed-order sums over the path groups / warps; rows and entries are dealt out to the warps
+            for (int i1 = G; i1 < S::DIN; i1 += S::BW) {
+                Vec sum; vzero(sum);
+#pragma unroll
+                for (int g2 = 0; g2 < S::BW; ++g2)
+                    sum = vadd(sum, reinterpret_cast<const Vec*>(dxs + (size_t)(buf * S::BW + g2) * L::X_EDGE)[i1 * NQV + vlane]);
+                reinterpret_cast<Vec*>(p.dx_edge + (size_t)e * L::X_EDGE)[i1 * NQV + vlane] = sum;
+            }
+            if (warp == 0 && lane < S::DSH) {
+                float sum = 0.f;
+#pragma unroll
+                for (int w2 = 0; w2 < NCONS; ++w2) sum += dyp[(buf * NCONS + w2) * L::DYP + lane];
+                p.grad_sh[(size_t)e * S::DSH + lane] = sum;
+            }
+            buf ^= 1;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[stage]);
+        if (++stage == NS) { stage = 0; phase ^= 1; }
+    }
+}
+
+template <class S, int G>
+struct BwdDispatch {
+    template <class... Args>
+    __device__ static __forceinline__ void run(const int g, Args&&... args) {
+        if (g == G) bwd_consumer<S, G>(args...);
+        else BwdDispatch<S, G + 1>::run(g, args...);
+    }
+};
+template <class S>
+struct BwdDispatch<S, S::BW> {
+    template <class... Args>
+    __device__ static __forceinline__ void run(const int, Args&&...) {}
+};
+
+template <class S>
+__device__ __forceinline__ void bwd_producer(const BwdParams& p, unsigned char* smem, const int lane,
+                                             const int64_t e_begin, const int64_t e_end, const int n_tiles) {
+    using L = BwdSmem<S>;
+    constexpr int T = L::T, NS = L::NS;
+    constexpr int YPL = (T * S::DSH + 31) / 32;
+    constexpr int NA = (S::B_APAD + 31) / 32;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
+    uint64_t* empty = full + NS;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
+
+    ASlot tab[NA];  // this lane's A slots (lane, lane + 32, ...)
+#pragma unroll
+    for (int i = 0; i < NA; ++i) {
+        const int slot = lane + 32 * i;
+        ASlot a{0.f, 0.f, 0, 0};
+        if (slot < S::B_APAD) {
+            const PairRec pr = S::b_pair_rec(slot);
+            if (pr.count > 0) { a.c0 = S::b_rec_val(pr.start); a.i2_0 = S::b_rec_i2(pr.start); }
+            if (pr.count > 1) { a.c1 = S::b_rec_val(pr.start + 1); a.i2_1 = S::b_rec_i2(pr.start + 1); }
+        }
+        tab[i] = a;
+    }
+    int snd_a = 0, rcv_a = -1, snd_b = 0, rcv_b = -1;
+    float y_a[YPL], y_b[YPL];
+    auto load_meta = [&](int t, int& snd, int& rcv, float (&yv)[YPL]) {
+        if (t >= n_tiles) return;
+        const int64_t e0 = e_begin + (int64_t)t * T;
+        const int n_e = (int)min((int64_t)T, e_end - e0);
+        if (lane < n_e) { snd = p.senders[e0 + lane]; rcv = p.receivers[e0 + lane]; }
+#pragma unroll
+        for (int i = 0; i < YPL; ++i) {
+            const int idx = i * 32 + lane;
+            if (idx < n_e * S::DSH) yv[i] = p.sh[e0 * S::DSH + idx];
+        }
+    };
+    load_meta(0, snd_a, rcv_a, y_a);
+    load_meta(1, snd_b, rcv_b, y_b);
+    int armed = 0, last_rcv = -1, stage = 0, phase = 0;
+    for (int t = 0; t < n_tiles; ++t) {
+        if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
+        unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
+        const int64_t e0 = e_begin + (int64_t)t * T;
+        const int n_e = (int)min((int64_t)T, e_end - e0);
+        int* recv_t = reinterpret_cast<int*>(st + L::st_r);
+        float* y_t = reinterpret_cast<float*>(st + L::st_y);
+        float* A_t = reinterpret_cast<float*>(st + L::st_A);
+        if (lane == 0) {
+            mbar_expect_tx(&full[stage], (uint32_t)n_e * (uint32_t)(4 * (L::S_EDGE + L::X_EDGE)));
+            bulk_g2s(st + L::st_s, p.w + (size_t)e0 * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE, &full[stage]);
+        }
+        if (lane < n_e)
+            bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE, p.x + (size_t)snd_a * L::X_EDGE, 4u * L::X_EDGE,
+                     &full[stage]);
+        armed = t + 1;
+        int before = __shfl_up_sync(0xffffffffu, rcv_a, 1);
+        if (lane == 0) before = last_rcv;
+        const unsigned mask = __ballot_sync(0xffffffffu, lane < n_e && rcv_a != before);
+        last_rcv = __shfl_sync(0xffffffffu, rcv_a, n_e - 1);
+        if (lane < n_e) recv_t[lane] = rcv_a;
+        if (lane == 0) recv_t[T] = (int)mask;
+#pragma unroll
+        for (int i = 0; i < YPL; ++i) {
+            const int idx = i * 32 + lane;
+            if (idx < n_e * S::DSH) y_t[idx] = y_a[i];
+        }
+        __syncwarp();
+        // A[e][slot] = sum over the slot's records of c * y[e][i2]
+        // (entries of edges beyond n_e are computed from stale data and never read)
+#pragma unroll
+        for (int i = 0; i < NA; ++i) {
+            const int slot = lane + 32 * i;
+            if (slot < S::B_APAD) {
+#pragma unroll
+                for (int e_i = 0; e_i < T; ++e_i) {
+                    const float* ye = y_t + e_i * S::DSH;
+                    A_t[e_i * S::B_APAD + slot] = fmaf(tab[i].c1, ye[tab[i].i2_1], tab[i].c0 * ye[tab[i].i2_0]);
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[stage]);
+        snd_a = snd_b; rcv_a = rcv_b;
+#pragma unroll
+        for (int i = 0; i < YPL; ++i) y_a[i] = y_b[i];
+        load_meta(t + 2, snd_b, rcv_b, y_b);
+        if (++stage == NS) { stage = 0; phase ^= 1; }
+    }
+    if (*abort_flag) {
+        for (int t = max(0, armed - NS); t < armed; ++t)
+            for (uint32_t it = 0; it < kSpinLimit; ++it)
+                if (mbar_try_wait(&full[t % NS], (t / NS) & 1)) break;
+    }
+}
+
+template <class S>
+__global__ void __launch_bounds__((S::BW * (S::NQ / (32 * S::V)) + 1) * 32, S::BC)
+fast_bwd_kernel(const BwdParams p) {
+    using L = BwdSmem<S>;
+    constexpr int T = L::T, NS = L::NS, NCONS = L::NCONS;
+    static_assert(T <= 31, "the change mask is one 32-bit word");
+    static_assert(S::B_NREC <= 2, "an A slot holds at most two records");
+
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
+    uint64_t* empty = full + NS;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t e_begin = min(p.n_edges, (int64_t)blockIdx.x * p.chunk);
+    const int64_t e_end = min(p.n_edges, e_begin + p.chunk);
+    const int n_tiles = (int)((e_end - e_begin + T - 1) / T);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NCONS); }
+        mbar_init(reinterpret_cast<uint64_t*>(smem + L::off_xch), NCONS);
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    if (warp == NCONS) bwd_producer<S>(p, smem, lane, e_begin, e_end, n_tiles);
+    else BwdDispatch<S, 0>::run(warp % S::BW, p, smem, warp / S::BW, warp, lane, e_begin, e_end, n_tiles);
+}
+
+}  // namespace fast
+}  // namespace e3j

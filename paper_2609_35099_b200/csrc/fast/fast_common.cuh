@@ -65,6 +65,21 @@ __device__ __forceinline__ void vfma(float4& acc, const float a, const float4 b)
 __device__ __forceinline__ void vfma(float2& acc, const float a, const float2 b) {
     acc.x = fmaf(a, b.x, acc.x); acc.y = fmaf(a, b.y, acc.y);
 }
+__device__ __forceinline__ void vfma(float4& acc, const float4 a, const float4 b) {
+    acc.x = fmaf(a.x, b.x, acc.x); acc.y = fmaf(a.y, b.y, acc.y); acc.z = fmaf(a.z, b.z, acc.z); acc.w = fmaf(a.w, b.w, acc.w);
+}
+__device__ __forceinline__ void vfma(float2& acc, const float2 a, const float2 b) {
+    acc.x = fmaf(a.x, b.x, acc.x); acc.y = fmaf(a.y, b.y, acc.y);
+}
+// sum over the lane's channels of a * b
+__device__ __forceinline__ float vdot(const float4 a, const float4 b) {
+    return fmaf(a.w, b.w, fmaf(a.z, b.z, fmaf(a.y, b.y, a.x * b.x)));
+}
+__device__ __forceinline__ float vdot(const float2 a, const float2 b) { return fmaf(a.y, b.y, a.x * b.x); }
+__device__ __forceinline__ float4 vadd(const float4 a, const float4 b) {
+    return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+}
+__device__ __forceinline__ float2 vadd(const float2 a, const float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
 __device__ __forceinline__ void vzero(float4& v) { v = make_float4(0.f, 0.f, 0.f, 0.f); }
 __device__ __forceinline__ void vzero(float2& v) { v = make_float2(0.f, 0.f); }
 
@@ -160,6 +175,11 @@ struct FwdParams {
 // Sums the pieces of every receiver row that was split between CTAs, in CTA order.
 __global__ void fwd_fixup_kernel(int n_cta, int row_f4, const float4* __restrict__ partial,
                                  const int32_t* __restrict__ part_recv, float4* __restrict__ out);
+
+// Backward pass 2: grad_x[a] = sum of the per-edge shares of the edges sent by a, in edge order.
+__global__ void bwd_dx_reduce_kernel(int64_t n_nodes, int row_f4, const float4* __restrict__ dx_edge,
+                                     const int32_t* __restrict__ sender_perm, const int32_t* __restrict__ colptr,
+                                     float4* __restrict__ grad_x);
 
 }  // namespace fast
 }  // namespace e3j

@@ -1,6 +1,9 @@
 // Host-side launchers of the signature-specialised kernels.
 #pragma once
+#include <algorithm>
+
 #include "../fast_registry.hpp"
+#include "fast_bwd.cuh"
 #include "fast_fwd.cuh"
 
 namespace e3j {
@@ -55,6 +58,41 @@ int launch_fwd(const ConvArgs& a) {
     if (int s = after_launch()) return s;
     fwd_fixup_kernel<<<n_cta, 256, 0, a.stream>>>(n_cta, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),
                                                  p.part_recv, reinterpret_cast<float4*>(a.out));
+    return after_launch();
+}
+
+// scratch of the backward: this edge's share of grad_x, [E][d][N_q]
+template <class S>
+size_t bwd_scratch_bytes(int64_t, int64_t n_edges) {
+    return align_up(sizeof(float) * (size_t)(n_edges > 0 ? n_edges : 1) * S::DIN * S::NQ, 256);
+}
+
+template <class S>
+int launch_bwd(const ConvArgs& a) {
+    using L = BwdSmem<S>;
+    static_assert(L::total * S::BC + 1024 * S::BC <= 228 * 1024, "backward stage ring does not fit in shared memory");
+    if (a.workspace_bytes < bwd_scratch_bytes<S>(a.n_nodes, a.n_edges)) return E3J_ERR_WORKSPACE;
+    const int n_cta = sm_count() * S::BC;
+    static thread_local int attr_dev = -1;
+    int dev = 0;
+    E3J_CUDA_TRY(cudaGetDevice(&dev));
+    if (attr_dev != dev) {
+        E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));
+        attr_dev = dev;
+    }
+    BwdParams p{};
+    p.x = a.x; p.sh = a.sh; p.w = a.w; p.senders = a.senders; p.receivers = a.receivers;
+    p.grad_out = a.grad_out; p.grad_sh = a.grad_sh; p.grad_w = a.grad_w;
+    p.dx_edge = reinterpret_cast<float*>(a.workspace);
+    p.n_nodes = a.n_nodes; p.n_edges = a.n_edges;
+    p.chunk = (a.n_edges + n_cta - 1) / n_cta;
+    p.status = a.status;
+    constexpr int threads = (S::BW * (S::NQ / (32 * S::V)) + 1) * 32;
+    fast_bwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
+    if (int s = after_launch()) return s;
+    const int64_t blocks = std::min<int64_t>(a.n_nodes, 148 * 16);
+    bwd_dx_reduce_kernel<<<(int)blocks, S::DIN * S::NQ / 4, 0, a.stream>>>(a.n_nodes, S::DIN * S::NQ / 4,
+        reinterpret_cast<const float4*>(p.dx_edge), a.sender_perm, a.colptr, reinterpret_cast<float4*>(a.grad_x));
     return after_launch();
 }
 

@@ -115,6 +115,109 @@ class Sig:
             a0.append(len(slots))
         return bounds, a0, slots
 
+    # ---------------------------------------------------------------- backward
+    def bwd_layout(self):
+        """Contiguous groups of whole paths, balanced by estimated instruction count."""
+        BW = self.cfg["BW"]
+        costs = []
+        for k, p in enumerate(self.paths):
+            rows = range(p["out_off"], p["out_off"] + 2 * p["L"] + 1)
+            npairs = sum(len(self.row_pairs[r]) for r in rows)
+            nrec = sum(len(self.pairs[pi][3]) for r in rows for pi in self.row_pairs[r])
+            combos = len({self.pairs[pi][1] for r in rows for pi in self.row_pairs[r]})
+            costs.append(4.0 * npairs + nrec + 6.0 * combos + 3.0)
+        pb = partition_rows(costs, BW)
+        while len(pb) < BW + 1:
+            pb.append(pb[-1])
+        row0 = [self.paths[pb[g]]["out_off"] if pb[g] < self.P else self.D for g in range(BW + 1)]
+        a0, slots = [0], []
+        for g in range(BW):
+            for row in range(row0[g], row0[g + 1]):
+                slots += self.row_pairs[row]
+            while len(slots) % 4:
+                slots.append(None)
+            a0.append(len(slots))
+        return pb, row0, a0, slots
+
+    def emit_bwd(self):
+        if "BW" not in self.cfg:
+            return []
+        V, NQ = self.V, self.NQ
+        BW, BT, BS, BC = self.cfg["BW"], self.cfg["BT"], self.cfg["BS"], self.cfg["BC"]
+        pb, row0, a0, slots = self.bwd_layout()
+        slot_of_pair = {pi: s for s, pi in enumerate(slots) if pi is not None}
+        rmax = max(row0[g + 1] - row0[g] for g in range(BW))
+        rec_val, rec_i2, pair_tab = [], [], []
+        for pi in slots:
+            if pi is None:
+                pair_tab.append((len(rec_val), 0)); continue
+            rl = self.pairs[pi][3]
+            pair_tab.append((len(rec_val), len(rl)))
+            for i2, v in rl:
+                rec_val.append(v); rec_i2.append(i2)
+        self.bwd_tables = (pair_tab, rec_val, rec_i2)
+        o = []
+        o.append(f"    // ---- backward: path groups {pb}")
+        o.append(f"    static constexpr int BW = {BW}, BT = {BT}, BS = {BS}, BC = {BC}, B_RMAX = {rmax}, B_APAD = {len(slots)}, "
+                 f"B_NREC = {max(c for _, c in pair_tab)};")
+        o.append(f"    __device__ static __forceinline__ PairRec b_pair_rec(int i) {{ return kBPair_{self.name}[i]; }}")
+        o.append(f"    __device__ static __forceinline__ float b_rec_val(int i) {{ return kBVal_{self.name}[i]; }}")
+        o.append(f"    __device__ static __forceinline__ unsigned char b_rec_i2(int i) {{ return kBI2_{self.name}[i]; }}")
+        o.append(f"    static constexpr int b_row0(int g) {{")
+        o.append("        switch (g) {")
+        for i, v in enumerate(row0):
+            o.append(f"            case {i}: return {v};")
+        o.append(f"            default: return {row0[-1]};")
+        o.append("        }\n    }")
+        o.append(f"    template <int G>")
+        o.append(f"    __device__ static __forceinline__ void bwd_edge(const Vec (&dm)[B_RMAX], const Vec* __restrict__ xs, "
+                 f"const Vec* __restrict__ ss, const float* __restrict__ As, Vec (&dxp)[DIN], float (&dyl)[16], "
+                 f"Vec* __restrict__ gw) {{")
+        o.append(f"        constexpr int NQV = NQ / V;")
+        for g in range(BW):
+            o.append(f"        if constexpr (G == {g}) {{")
+            rows = range(row0[g], row0[g + 1])
+            need_x = sorted({self.pairs[pi][1] for row in rows for pi in self.row_pairs[row]})
+            for i1 in need_x:
+                o.append(f"            const Vec x{i1} = xs[{i1} * NQV];")
+            loaded_a = set()
+            for k in range(pb[g], pb[g + 1]):
+                p = self.paths[k]
+                prow = list(range(p["out_off"], p["out_off"] + 2 * p["L"] + 1))
+                used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.row_pairs[r2]})
+                o.append(f"            const Vec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
+                for i1 in used:
+                    o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                    o.append(f"            Vec u{k}_{i1}; vzero(u{k}_{i1});")
+                depth = max(len(self.row_pairs[r2]) for r2 in prow)
+                for j in range(depth):
+                    for row in prow:
+                        if j >= len(self.row_pairs[row]):
+                            continue
+                        pi = self.row_pairs[row][j]
+                        slot = slot_of_pair[pi]
+                        q, lane = slot // 4, "xyzw"[slot % 4]
+                        if q not in loaded_a:
+                            loaded_a.add(q)
+                            o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
+                        i1 = self.pairs[pi][1]
+                        r = row - row0[g]
+                        o.append(f"            vfma(u{k}_{i1}, a{q}.{lane}, dm[{r}]);")
+                        o.append(f"            {{ const float t = vdot(sx{k}_{i1}, dm[{r}]);")
+                        for i2, c in self.pairs[pi][3]:
+                            o.append(f"              dyl[{i2}] = fmaf({fmt_float(c)}, t, dyl[{i2}]);")
+                        o.append("            }")
+                first = used[0]
+                o.append(f"            Vec ds{k} = vmul(x{first}, u{k}_{first});")
+                for i1 in used[1:]:
+                    o.append(f"            vfma(ds{k}, x{i1}, u{k}_{i1});")
+                o.append(f"            gw[{k} * NQV] = ds{k};")
+                for i1 in used:
+                    o.append(f"            vfma(dxp[{i1}], s{k}, u{k}_{i1});")
+            o.append("        }")
+        o.append("    }")
+        return o
+
     def emit(self) -> str:
         V, NQ = self.V, self.NQ
         FW, FT, FS, FC = self.cfg["FW"], self.cfg["FT"], self.cfg["FS"], self.cfg["FC"]
@@ -141,6 +244,7 @@ class Sig:
         o.append(f"// {self.cfg['irreps_in']} (x) harmonics l<={self.cfg['sh_lmax']}: P={self.P} D={self.D} "
                  f"nnz={self.NNZ} pairs={len(self.pairs)}")
         o.append('#include "fast_fwd.cuh"')
+        o.append('#include "fast_bwd.cuh"')
         o.append('#include "fast_launch.cuh"')
         o.append("")
         o.append("namespace e3j {\nnamespace fast {\nnamespace {")
@@ -150,6 +254,15 @@ class Sig:
         o.append("    " + ", ".join(fmt_float(v) for v in rec_val) + "};")
         o.append(f"__device__ const unsigned char kI2_{self.name}[{self.NNZ}] = {{")
         o.append("    " + ", ".join(str(i) for i in rec_i2) + "};")
+        bwd_lines = self.emit_bwd()
+        if bwd_lines:
+            bpair, bval, bi2 = self.bwd_tables
+            o.append(f"__device__ const PairRec kBPair_{self.name}[{len(bpair)}] = {{")
+            o.append("    " + ", ".join(f"{{{s_},{c_}}}" for s_, c_ in bpair) + "};")
+            o.append(f"__device__ const float kBVal_{self.name}[{len(bval)}] = {{")
+            o.append("    " + ", ".join(fmt_float(v) for v in bval) + "};")
+            o.append(f"__device__ const unsigned char kBI2_{self.name}[{len(bi2)}] = {{")
+            o.append("    " + ", ".join(str(i) for i in bi2) + "};")
         o.append("")
         o.append(f"struct {S} {{")
         o.append(f"    static constexpr int NQ = {NQ}, DIN = {self.DIN}, DSH = {self.DSH}, P = {self.P}, D = {self.D};")
@@ -230,6 +343,7 @@ class Sig:
                 o.append(f"            dst[{row - bounds[g]} * stride] = acc[{row - bounds[g]}];")
             o.append("        }")
         o.append("    }")
+        o += bwd_lines
         o.append("};")
         o.append("}  // namespace")
         o.append("}  // namespace fast")
@@ -237,7 +351,11 @@ class Sig:
         o.append(f"extern const FastKernels kFast_{self.name};")
         o.append(f"const FastKernels kFast_{self.name} = {{")
         o.append(f'    "{self.signature}",')
-        o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, nullptr, &fast::launch_fwd<fast::{S}>, nullptr, nullptr, nullptr}};")
+        if bwd_lines:
+            o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, &fast::bwd_scratch_bytes<fast::{S}>, "
+                     f"&fast::launch_fwd<fast::{S}>, &fast::launch_bwd<fast::{S}>, nullptr, nullptr}};")
+        else:
+            o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, nullptr, &fast::launch_fwd<fast::{S}>, nullptr, nullptr, nullptr}};")
         o.append("}  // namespace e3j")
         return "\n".join(o) + "\n"
 
