@@ -203,15 +203,19 @@ class Sig:
                         i1 = self.pairs[pi][1]
                         r = row - row0[g]
                         o.append(f"            vfma(u{k}_{i1}, a{q}.{lane}, dm[{r}]);")
-                        o.append(f"            {{ const float t = vdot(sx{k}_{i1}, dm[{r}]);")
-                        for i2, c in self.pairs[pi][3]:
-                            o.append(f"              dyl[{i2}] = fmaf({fmt_float(c)}, t, dyl[{i2}]);")
-                        o.append("            }")
+                        if not self.cfg.get("DBG_NODY"):
+                            o.append(f"            {{ const float t = vdot(sx{k}_{i1}, dm[{r}]);")
+                            for i2, c in self.pairs[pi][3]:
+                                o.append(f"              dyl[{i2}] = fmaf({fmt_float(c)}, t, dyl[{i2}]);")
+                            o.append("            }")
                 first = used[0]
                 o.append(f"            Vec ds{k} = vmul(x{first}, u{k}_{first});")
                 for i1 in used[1:]:
                     o.append(f"            vfma(ds{k}, x{i1}, u{k}_{i1});")
-                o.append(f"            gw[{k} * NQV] = ds{k};")
+                if self.cfg.get("DBG_NODS"):
+                    o.append(f"            if (ds{k}.x == 1.2345f) gw[{k} * NQV] = ds{k};")
+                else:
+                    o.append(f"            gw[{k} * NQV] = ds{k};")
                 for i1 in used:
                     o.append(f"            vfma(dxp[{i1}], s{k}, u{k}_{i1});")
             o.append("        }")
