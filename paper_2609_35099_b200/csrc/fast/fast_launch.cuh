@@ -25,10 +25,15 @@ inline int sm_count() {
     return cached;
 }
 
-// scratch: [part_recv: 2*n_cta ints in an 8 KB slot][partial rows: 2*n_cta*D*NQ floats], n_cta <= kMaxSms*S::FC
+// scratch: [part_recv: 2*n_cta ints in an 8 KB slot][partial rows: 2*n_cta*D*NQ floats],
+// n_cta = (SMs of the current device) * S::FC
+template <class S>
+size_t fwd_scratch_need(int n_cta) {
+    return kPartRecvBytes + sizeof(float) * 2 * (size_t)n_cta * S::D * S::NQ;
+}
 template <class S>
 size_t fwd_scratch_bytes(int64_t, int64_t) {
-    return kPartRecvBytes + sizeof(float) * 2 * (size_t)kMaxSms * S::FC * S::D * S::NQ;
+    return fwd_scratch_need<S>(sm_count() * S::FC);
 }
 
 template <class S>
@@ -36,8 +41,8 @@ int launch_fwd(const ConvArgs& a) {
     using L = FwdSmem<S>;
     static_assert(L::total * S::FC + 1024 * S::FC <= 228 * 1024, "forward stage ring does not fit in shared memory");
     static_assert(2 * kMaxSms * S::FC * sizeof(int32_t) <= kPartRecvBytes, "part_recv does not fit its slot");
-    if (a.workspace_bytes < fwd_scratch_bytes<S>(a.n_nodes, a.n_edges)) return E3J_ERR_WORKSPACE;
     const int n_cta = sm_count() * S::FC;
+    if (a.workspace_bytes < fwd_scratch_need<S>(n_cta)) return E3J_ERR_WORKSPACE;
     static thread_local int attr_dev = -1;
     int dev = 0;
     E3J_CUDA_TRY(cudaGetDevice(&dev));

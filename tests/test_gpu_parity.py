@@ -18,6 +18,16 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
+@pytest.fixture(autouse=True)
+def _release_device_memory():
+    """The full-size cases hold tens of GB; hand cached blocks back between tests."""
+    yield
+    import gc
+    gc.collect()
+    if torch.cuda.is_available():
+        torch.cuda.empty_cache()
+
+
 def _cuda(a):
     return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
 
@@ -192,3 +202,112 @@ def test_workspace_errors_are_reported():
     tiny = torch.empty(16, dtype=torch.uint8, device=DEV)
     with pytest.raises(ValueError):
         e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, _cuda(g), workspace=tiny)
+
+
+# ------------------------------------------------------------------ full-size configurations, sampled
+def _seeded_normal(shape, seed):
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(seed)
+    return torch.randn(shape, generator=gen, device=DEV, dtype=torch.float32)
+
+
+def _checksum(t):
+    """Order-independent exact fingerprint of a float tensor (wrapping integer sum of its bit patterns)."""
+    return int(t.view(torch.int32).to(torch.int64).sum().item())
+
+
+def test_config5_full_size_sampled():
+    """100k atoms, 4.77 M edges, skewed degrees (26..106): the bench launch configuration at scale.
+    Outputs are checked on sampled receivers / edges / senders that the oracle recomputes one by one."""
+    c = workloads.CONFIGS[5]
+    wl = workloads.make_graph(5)
+    n, e = wl.n_nodes, wl.n_edges
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], None, c["out_lmax"])
+    assert plan.specialised == 1
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], None, c["out_lmax"])
+    rng = np.random.Generator(np.random.PCG64([5, 1]))
+    x = rng.standard_normal((n, plan.d_in, plan.n_channels), dtype=np.float32)
+    y = workloads.edge_harmonics(wl)
+    dx_, dy_ = _cuda(x), _cuda(y)
+    dw_ = _seeded_normal((e, plan.n_paths, plan.n_channels), 51)
+    dg_ = _seeded_normal((n, plan.d_out, plan.n_channels), 52)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    rowptr, perm, colptr = e3j.e3j_graph_prepare(n, snd, rcv)
+    assert e3j.e3j_graph_validate(n, snd, rcv) == 0
+    out = e3j.e3j_conv_fwd(plan, dx_, dy_, dw_, snd, rcv, rowptr)
+    gx, gy, gw = e3j.e3j_conv_bwd(plan, dx_, dy_, dw_, snd, rcv, dg_, rowptr, perm, colptr)
+    torch.cuda.synchronize()
+    assert e3j.e3j_plan_device_status(plan) == 0
+    sums = [_checksum(t) for t in (out, gx, gy, gw)]
+    out.zero_(); gx.zero_(); gy.zero_()
+    e3j.e3j_conv_fwd(plan, dx_, dy_, dw_, snd, rcv, rowptr, out=out)
+    e3j.e3j_conv_bwd(plan, dx_, dy_, dw_, snd, rcv, dg_, rowptr, perm, colptr, grad_x=gx, grad_sh=gy, grad_w=gw)
+    torch.cuda.synchronize()
+    assert sums == [_checksum(t) for t in (out, gx, gy, gw)], "results differ between two runs"
+
+    deg = np.bincount(wl.receivers, minlength=n)
+    rp = rowptr.cpu().numpy()
+    pick = np.unique(np.concatenate([rng.choice(n, 40, replace=False), np.argsort(deg)[-8:], np.argsort(deg)[:4],
+                                     [0, n - 1]]))
+    out_blocks, w_blocks = blocks_of_paths(cp.paths, "out"), blocks_of_paths(cp.paths, "w")
+    for b in pick:
+        e0, e1 = int(rp[b]), int(rp[b + 1])
+        s_ids = wl.senders[e0:e1]
+        nodes, local = np.unique(np.concatenate([s_ids, [b]]), return_inverse=True)
+        lb = int(local[-1])
+        order = np.arange(e1 - e0)
+        xs = x[nodes]
+        ws = dw_[e0:e1].cpu().numpy()
+        gs = np.zeros((len(nodes), plan.d_out, plan.n_channels), np.float32)
+        gs[lb] = dg_[b].cpu().numpy()
+        l_snd = local[:-1].astype(np.int32)
+        l_rcv = np.full(e1 - e0, lb, np.int32)
+        ref = oconv.conv_fwd(cp, xs, y[e0:e1], ws, l_snd[order], l_rcv)
+        assert_blockwise_close(out[b].cpu().numpy()[None], ref[lb][None], out_blocks, what=f"out[{b}]")
+        _, ry, rw = oconv.conv_bwd(cp, xs, y[e0:e1], ws, l_snd, l_rcv, gs)
+        if e1 > e0:
+            assert_blockwise_close(gw[e0:e1].cpu().numpy(), rw, w_blocks, what=f"grad_w[{b}]")
+            assert_blockwise_close(gy[e0:e1].cpu().numpy(), ry, blocks_of_paths(cp.paths, "sh"), what=f"grad_sh[{b}]")
+    # grad_x of sampled senders: all edges they send (scattered over the edge list)
+    senders_sorted = perm.cpu().numpy()
+    cptr = colptr.cpu().numpy()
+    for a in rng.choice(n, 24, replace=False):
+        ids = np.sort(senders_sorted[cptr[a]:cptr[a + 1]])
+        rc = wl.receivers[ids]
+        nodes, l_rcv = np.unique(rc, return_inverse=True)
+        xs = np.zeros((len(nodes) + 1, plan.d_in, plan.n_channels), np.float32)
+        xs[-1] = x[a]
+        gs = np.concatenate([dg_[torch.from_numpy(nodes).to(DEV)].cpu().numpy(),
+                             np.zeros((1, plan.d_out, plan.n_channels), np.float32)])
+        ws = dw_[torch.from_numpy(ids).to(DEV)].cpu().numpy()
+        l_snd = np.full(len(ids), len(nodes), np.int32)
+        rx, _, _ = oconv.conv_bwd(cp, xs, y[ids], ws, l_snd, l_rcv.astype(np.int32), gs)
+        assert_blockwise_close(gx[a].cpu().numpy()[None], rx[-1][None], blocks_of_paths(cp.paths, "x"), what=f"grad_x[{a}]")
+
+
+def test_tensor_product_full_size_sampled():
+    """Config 4 at 2^20 rows (75 GB of forward I/O); sampled rows against the oracle."""
+    c = workloads.CONFIGS[4]
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], None, 3)
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], None, 3)
+    rows = 1 << 20
+    free, _ = torch.cuda.mem_get_info()
+    need = 4 * rows * (2 * plan.d_in * plan.n_channels + 2 * plan.d_sh + 2 * plan.n_paths * plan.n_channels
+                       + plan.d_out * plan.n_channels)
+    if free < need * 1.1:
+        pytest.skip("not enough free device memory for 2^20 rows")
+    x1 = _seeded_normal((rows, plan.d_in, plan.n_channels), 41)
+    x2 = _seeded_normal((rows, plan.d_sh), 42)
+    w = _seeded_normal((rows, plan.n_paths, plan.n_channels), 43)
+    out = e3j.e3j_tp_fwd(plan, x1, x2, w)
+    pick = np.unique(np.concatenate([np.random.default_rng(4).choice(rows, 40, replace=False), [0, rows - 1]]))
+    idx = torch.from_numpy(pick).to(DEV)
+    h = lambda t: t[idx].cpu().numpy()
+    ref = oconv.tp_fwd(cp, h(x1), h(x2), h(w))
+    assert_blockwise_close(h(out), ref, blocks_of_paths(cp.paths, "out"), what="tp out")
+    # the output buffer doubles as the cotangent of the backward (as a training step would feed it back)
+    g1, g2, gw = e3j.e3j_tp_bwd(plan, x1, x2, w, out)
+    r1, r2, rw = oconv.tp_bwd(cp, h(x1), h(x2), h(w), h(out))
+    assert_blockwise_close(h(g1), r1, blocks_of_paths(cp.paths, "x"), what="tp grad_x1")
+    assert_blockwise_close(h(g2), r2, blocks_of_paths(cp.paths, "sh"), what="tp grad_x2")
+    assert_blockwise_close(h(gw), rw, blocks_of_paths(cp.paths, "w"), what="tp grad_w")
