@@ -45,6 +45,15 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback (6650 GB/s, earlier pool measurement)"
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per call from the ncu captures summarised in
+# profiles/fast_fwd_kernel_water3000.txt, profiles/fast_bwd_kernel_water3000.txt and the launch-list run
+# (specialised kernels, workload water3000).  Other workloads / the generic kernels report null.
+NCU_TRAFFIC = {
+    ("water3000", "fwd"): 1.110510e9 + 0.082842e9 + 0.016341e9,          # fast_fwd_kernel + fwd_fixup_kernel
+    ("water3000", "bwd"): 1.259801e9 + 1.363752e9 + 0.330465e9 + 0.0020e9,  # fast_bwd_kernel + bwd_dx_reduce_kernel
+}
+
+
 def algorithmic_bytes(n, e, d, dp, P, D, nq):
     """Minimal bytes with the paper's accounting (inputs + outputs, no scratch, no residuals)."""
     x, y, s, idx = n * d * nq * 4, e * dp * 4, e * P * nq * 4, 2 * e * 4
@@ -285,13 +294,18 @@ def main():
         fb, bb = algorithmic_bytes(n, e, plan.d_in, plan.d_sh, plan.n_paths, plan.d_out, plan.n_channels)
         f_ms, b_ms = statistics.mean(fwd_ms), statistics.mean(bwd_ms)
 
-        def roof(nbytes, ms, kernel):
+        def roof(nbytes, ms, kernel, key):
             ach = nbytes / (ms * 1e-3) / 1e9
+            traffic = NCU_TRAFFIC.get((wl.name, key)) if plan.specialised else None
             return {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s",
                     "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "peak_source": peak_src,
-                    "algorithmic_bytes_per_launch": nbytes, "avg_ms": ms, "traffic": None}
+                    "algorithmic_bytes_per_launch": nbytes, "avg_ms": ms, "traffic": traffic}
 
-        roofs = {"fwd": roof(fb, f_ms, "e3j_conv_fwd call"), "bwd": roof(bb, b_ms, "e3j_conv_bwd call")}
+        spec = bool(plan.specialised)
+        roofs = {"fwd": roof(fb, f_ms, "e3j_conv_fwd call: fast_fwd_kernel (96 %) + fwd_fixup_kernel" if spec
+                             else "e3j_conv_fwd call: generic conv_fwd_kernel", "fwd"),
+                 "bwd": roof(bb, b_ms, "e3j_conv_bwd call: fast_bwd_kernel (93 %) + bwd_dx_reduce_kernel" if spec
+                             else "e3j_conv_bwd call: generic edge + node kernels", "bwd")}
         dominant = roofs["bwd"] if b_ms >= f_ms else roofs["fwd"]
         line = {
             "metric": "conv_fwd_bwd_edges_per_s", "value": e * world / (ms_per_step * 1e-3), "unit": "edges/s",
