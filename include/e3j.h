@@ -148,6 +148,31 @@ int e3j_conv_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
                  const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
                  size_t workspace_bytes, void* stream);
 
+/* Forward convolution without any device allocation or workspace (no counterpart in the paper;
+ * added for hosts that cannot allocate).  Some users of this library run where device memory
+ * cannot be obtained at call time: a molecular-dynamics engine or an inference server that
+ * reserves all of its device memory at start-up and forbids cudaMalloc inside the time-step /
+ * request loop, or a plug-in that is handed tensors but has no allocator to make a workspace
+ * from.  For them the scratch of the specialised forward kernel lives in a 24 MiB file-scope
+ * __device__ array inside the library (every GPU that loads the library holds it until the process
+ * exits); the caller passes inputs and the output only.  This function and everything it calls
+ * perform no cudaMalloc / cudaFree and no allocating library call.
+ *   - Works only for plans with specialised kernels (e3j_plan_info().specialised == 1); other
+ *     plans return E3J_ERR_UNSUPPORTED.  A plan whose scratch need on the current device (it
+ *     depends on D * N_q and the SM count, not on the graph) exceeds 24 MiB returns
+ *     E3J_ERR_WORKSPACE.
+ *   - The first call on each device looks the array's address up (cudaGetSymbolAddress, with that
+ *     device current) and caches it; make that first call before any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents.
+ *     Nothing in it has to be zero at entry (the kernel writes every word before reading it), but
+ *     two calls that overlap on the GPU (different streams) race on it: serialise them.
+ *   - Results are the same as e3j_conv_fwd's.  Bounded-wait failures are not reported through
+ *     e3j_plan_device_status here.
+ * Arguments as for e3j_conv_fwd (receivers non-decreasing; rowptr is not needed). */
+int e3j_conv_fwd_noalloc(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                         const float* sh, const float* w, const int32_t* senders,
+                         const int32_t* receivers, float* out, void* stream);
+
 /* Convolution backward.  grad_out [n_nodes,D,N_q]; grad_x [n_nodes,d,N_q],
  * grad_sh [n_edges,d'], grad_w [n_edges,P,N_q]; any of the three may be NULL (not
  * computed).  rowptr, sender_perm, colptr as produced by e3j_graph_prepare, or NULL

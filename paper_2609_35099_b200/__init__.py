@@ -20,7 +20,8 @@ from pathlib import Path
 __all__ = [
     "E3JError", "Plan", "library_path", "e3j_plan_create", "e3j_plan_destroy", "e3j_plan_info",
     "e3j_plan_paths", "e3j_plan_records", "e3j_plan_signature", "e3j_plan_device_status", "e3j_graph_prepare", "e3j_graph_validate",
-    "e3j_conv_fwd_workspace_bytes", "e3j_conv_bwd_workspace_bytes", "e3j_conv_fwd", "e3j_conv_bwd",
+    "e3j_conv_fwd_workspace_bytes", "e3j_conv_bwd_workspace_bytes", "e3j_conv_fwd", "e3j_conv_fwd_noalloc",
+    "e3j_conv_bwd",
     "e3j_tp_fwd", "e3j_tp_bwd", "e3j_status_string", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
 ]
 
@@ -84,6 +85,8 @@ def _load():
     lib.e3j_conv_bwd_workspace_bytes.restype = sz
     lib.e3j_conv_fwd.argtypes = [vp, i64, i64] + [vp] * 8 + [sz, vp]
     lib.e3j_conv_bwd.argtypes = [vp, i64, i64] + [vp] * 13 + [sz, vp]
+    lib.e3j_conv_fwd_noalloc.argtypes = [vp, i64, i64] + [vp] * 7
+    lib.e3j_conv_fwd_noalloc.restype = i32
     lib.e3j_tp_fwd.argtypes = [vp, i64] + [vp] * 5
     lib.e3j_tp_bwd.argtypes = [vp, i64] + [vp] * 8
     lib.e3j_status_string.argtypes = [i32]
@@ -258,6 +261,26 @@ def e3j_conv_fwd(plan: Plan, x, sh, w, senders, receivers, rowptr=None, out=None
         _dev_ptr(rowptr, i32, (n + 1,), "rowptr"),
         _dev_ptr(out, f32, (n, plan.d_out, plan.n_channels), "out"),
         ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_fwd")
+    return out
+
+
+def e3j_conv_fwd_noalloc(plan: Plan, x, sh, w, senders, receivers, out, stream=None):
+    """Forward convolution through the allocation-free entry point.
+
+    For callers that must not allocate device memory at call time (engines that reserve everything at
+    start-up, plug-ins without an allocator): the kernel's scratch lives inside the library, and this
+    wrapper allocates nothing either, so `out` must be passed in.  Calls on one device share that scratch and
+    must not overlap on the GPU."""
+    torch = _torch()
+    n, e = x.shape[0], senders.numel()
+    f32, i32 = torch.float32, torch.int32
+    _check(_load().e3j_conv_fwd_noalloc(
+        plan.handle, n, e,
+        _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"),
+        _dev_ptr(sh, f32, (e, plan.d_sh), "sh"),
+        _dev_ptr(w, f32, (e, plan.n_paths, plan.n_channels), "w"),
+        _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
+        _dev_ptr(out, f32, (n, plan.d_out, plan.n_channels), "out"), _stream(stream)), "e3j_conv_fwd_noalloc")
     return out
 
 
