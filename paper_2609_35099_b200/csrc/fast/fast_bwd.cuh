@@ -37,7 +37,7 @@ struct BwdParams {
 template <class S>
 struct BwdSmem {
     static constexpr int T = S::BT, NS = S::BS;
-    static constexpr int CH = S::NQ / (32 * S::V);
+    static constexpr int CH = S::NQ / (32 * S::BV);
     static constexpr int NCONS = S::BW * CH;
     static constexpr int S_EDGE = S::P * S::NQ;
     static constexpr int X_EDGE = S::DIN * S::NQ;
@@ -85,15 +85,18 @@ __device__ __forceinline__ float reduce16_over_lanes(float (&v)[16], const int l
     return r;
 }
 
-template <class S, int G>
-__device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* smem, const int ch, const int warp,
-                                             const int lane, const int64_t e_begin, const int64_t e_end,
-                                             const int n_tiles) {
-    using Vec = typename VecOf<S::V, false>::type;
+// The loop, the exchange and the reductions below are the same instructions for every path group; only
+// S::bwd_edge's body differs (chosen by a switch on g), which keeps the kernel's hot code small enough
+// for the SM's instruction cache.
+template <class S>
+__device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* smem, const int G, const int ch,
+                                             const int warp, const int lane, const int64_t e_begin,
+                                             const int64_t e_end, const int n_tiles) {
+    using Vec = typename S::BVec;
     using L = BwdSmem<S>;
     constexpr int T = L::T, NS = L::NS, NCONS = L::NCONS;
-    constexpr int NQV = S::NQ / S::V;
-    constexpr int ROW0 = S::b_row0(G), NROW = S::b_row0(G + 1) - ROW0;
+    constexpr int NQV = S::NQ / S::BV;
+    const int ROW0 = S::b_row0(G), NROW = S::b_row0(G + 1) - ROW0;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
     uint64_t* empty = full + NS;
     uint64_t* xch = reinterpret_cast<uint64_t*>(smem + L::off_xch);
@@ -127,7 +130,8 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
                 const Vec* g = reinterpret_cast<const Vec*>(p.grad_out + (size_t)recv_t[e_i] * row_elems) +
                                (size_t)ROW0 * NQV + vlane;
 #pragma unroll
-                for (int r = 0; r < NROW; ++r) dm[r] = g[(size_t)r * NQV];
+                for (int r = 0; r < S::B_RMAX; ++r)
+                    if (r < NROW) dm[r] = g[(size_t)r * NQV];
             }
             mask >>= 1;
             Vec dxp[S::DIN];
@@ -137,8 +141,8 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
 #pragma unroll
             for (int i = 0; i < 16; ++i) dyl[i] = 0.f;
             Vec* gw = reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + vlane;
-            S::template bwd_edge<G>(dm, xs, ss, As, dxp, dyl, gw);
-            xs += L::X_EDGE / S::V; ss += L::S_EDGE / S::V; As += S::B_APAD;
+            S::bwd_edge(G, dm, xs, ss, As, dxp, dyl, gw);
+            xs += L::X_EDGE / S::BV; ss += L::S_EDGE / S::BV; As += S::B_APAD;
 
             // this warp's partial sums -> shared memory
 #ifdef E3J_DBG_NOBFLY
@@ -186,20 +190,6 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
         if (++stage == NS) { stage = 0; phase ^= 1; }
     }
 }
-
-template <class S, int G>
-struct BwdDispatch {
-    template <class... Args>
-    __device__ static __forceinline__ void run(const int g, Args&&... args) {
-        if (g == G) bwd_consumer<S, G>(args...);
-        else BwdDispatch<S, G + 1>::run(g, args...);
-    }
-};
-template <class S>
-struct BwdDispatch<S, S::BW> {
-    template <class... Args>
-    __device__ static __forceinline__ void run(const int, Args&&...) {}
-};
 
 template <class S>
 __device__ __forceinline__ void bwd_producer(const BwdParams& p, unsigned char* smem, const int lane,
@@ -297,7 +287,7 @@ __device__ __forceinline__ void bwd_producer(const BwdParams& p, unsigned char* 
 }
 
 template <class S>
-__global__ void __launch_bounds__((S::BW * (S::NQ / (32 * S::V)) + 1) * 32, S::BC)
+__global__ void __launch_bounds__((S::BW * (S::NQ / (32 * S::BV)) + 1) * 32, S::BC)
 fast_bwd_kernel(const BwdParams p) {
     using L = BwdSmem<S>;
     constexpr int T = L::T, NS = L::NS, NCONS = L::NCONS;
@@ -322,7 +312,7 @@ fast_bwd_kernel(const BwdParams p) {
     }
     __syncthreads();
     if (warp == NCONS) bwd_producer<S>(p, smem, lane, e_begin, e_end, n_tiles);
-    else BwdDispatch<S, 0>::run(warp % S::BW, p, smem, warp / S::BW, warp, lane, e_begin, e_end, n_tiles);
+    else bwd_consumer<S>(p, smem, warp % S::BW, warp / S::BW, warp, lane, e_begin, e_end, n_tiles);
 }
 
 }  // namespace fast

@@ -92,7 +92,7 @@ int launch_bwd(const ConvArgs& a) {
     p.n_nodes = a.n_nodes; p.n_edges = a.n_edges;
     p.chunk = (a.n_edges + n_cta - 1) / n_cta;
     p.status = a.status;
-    constexpr int threads = (S::BW * (S::NQ / (32 * S::V)) + 1) * 32;
+    constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;
     fast_bwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
     const int64_t blocks = std::min<int64_t>(a.n_nodes, 148 * 16);

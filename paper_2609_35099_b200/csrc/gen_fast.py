@@ -142,7 +142,9 @@ class Sig:
     def emit_bwd(self):
         if "BW" not in self.cfg:
             return []
-        V, NQ = self.V, self.NQ
+        V, NQ = self.cfg.get("BV", self.V), self.NQ
+        assert NQ % (32 * V) == 0
+        bvec = {2: "float2", 4: "float4"}[V]
         BW, BT, BS, BC = self.cfg["BW"], self.cfg["BT"], self.cfg["BS"], self.cfg["BC"]
         pb, row0, a0, slots = self.bwd_layout()
         slot_of_pair = {pi: s for s, pi in enumerate(slots) if pi is not None}
@@ -158,6 +160,8 @@ class Sig:
         self.bwd_tables = (pair_tab, rec_val, rec_i2)
         o = []
         o.append(f"    // ---- backward: path groups {pb}")
+        o.append(f"    static constexpr int BV = {V};  // channels per lane in the backward")
+        o.append(f"    using BVec = {bvec};")
         o.append(f"    static constexpr int BW = {BW}, BT = {BT}, BS = {BS}, BC = {BC}, B_RMAX = {rmax}, B_APAD = {len(slots)}, "
                  f"B_NREC = {max(c for _, c in pair_tab)};")
         o.append(f"    __device__ static __forceinline__ PairRec b_pair_rec(int i) {{ return kBPair_{self.name}[i]; }}")
@@ -169,26 +173,26 @@ class Sig:
             o.append(f"            case {i}: return {v};")
         o.append(f"            default: return {row0[-1]};")
         o.append("        }\n    }")
-        o.append(f"    template <int G>")
-        o.append(f"    __device__ static __forceinline__ void bwd_edge(const Vec (&dm)[B_RMAX], const Vec* __restrict__ xs, "
-                 f"const Vec* __restrict__ ss, const float* __restrict__ As, Vec (&dxp)[DIN], float (&dyl)[16], "
-                 f"Vec* __restrict__ gw) {{")
-        o.append(f"        constexpr int NQV = NQ / V;")
+        o.append(f"    __device__ static __forceinline__ void bwd_edge(const int G, const BVec (&dm)[B_RMAX], const BVec* __restrict__ xs, "
+                 f"const BVec* __restrict__ ss, const float* __restrict__ As, BVec (&dxp)[DIN], float (&dyl)[16], "
+                 f"BVec* __restrict__ gw) {{")
+        o.append(f"        constexpr int NQV = NQ / BV;")
+        o.append("        switch (G) {")
         for g in range(BW):
-            o.append(f"        if constexpr (G == {g}) {{")
+            o.append(f"        case {g}: {{")
             rows = range(row0[g], row0[g + 1])
             need_x = sorted({self.pairs[pi][1] for row in rows for pi in self.row_pairs[row]})
             for i1 in need_x:
-                o.append(f"            const Vec x{i1} = xs[{i1} * NQV];")
+                o.append(f"            const BVec x{i1} = xs[{i1} * NQV];")
             loaded_a = set()
             for k in range(pb[g], pb[g + 1]):
                 p = self.paths[k]
                 prow = list(range(p["out_off"], p["out_off"] + 2 * p["L"] + 1))
                 used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.row_pairs[r2]})
-                o.append(f"            const Vec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
+                o.append(f"            const BVec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
                 for i1 in used:
-                    o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
-                    o.append(f"            Vec u{k}_{i1}; vzero(u{k}_{i1});")
+                    o.append(f"            const BVec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                    o.append(f"            BVec u{k}_{i1}; vzero(u{k}_{i1});")
                 depth = max(len(self.row_pairs[r2]) for r2 in prow)
                 for j in range(depth):
                     for row in prow:
@@ -209,7 +213,7 @@ class Sig:
                                 o.append(f"              dyl[{i2}] = fmaf({fmt_float(c)}, t, dyl[{i2}]);")
                             o.append("            }")
                 first = used[0]
-                o.append(f"            Vec ds{k} = vmul(x{first}, u{k}_{first});")
+                o.append(f"            BVec ds{k} = vmul(x{first}, u{k}_{first});")
                 for i1 in used[1:]:
                     o.append(f"            vfma(ds{k}, x{i1}, u{k}_{i1});")
                 if self.cfg.get("DBG_NODS"):
@@ -218,7 +222,9 @@ class Sig:
                     o.append(f"            gw[{k} * NQV] = ds{k};")
                 for i1 in used:
                     o.append(f"            vfma(dxp[{i1}], s{k}, u{k}_{i1});")
-            o.append("        }")
+            o.append("        } break;")
+        o.append("        default: break;")
+        o.append("        }")
         o.append("    }")
         return o
 
@@ -273,7 +279,7 @@ class Sig:
         o.append(f"    static constexpr int NNZ = {self.NNZ}, NPAIR = {len(self.pairs)}, V = {V};")
         o.append(f"    static constexpr bool PK = {str(PK).lower()};  // packed fp32 pairs (fma.rn.f32x2) or plain fp32")
         o.append(f"    using AT = {'u64' if PK else 'float'};")
-        o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, FC = {FC}, F_RMAX = {rmax}, F_APAD = {len(slots)}, F_NREC = {max(c for _, c in pair_tab)}, F_MAXREG = {self.cfg.get("F_MAXREG", 255)};")
+        o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, FC = {FC}, F_RMAX = {rmax}, F_APAD = {len(slots)}, F_NREC = {max(c for _, c in pair_tab)}, F_NPMAX = {max(a0[g + 1] - a0[g] for g in range(FW))}, F_MAXREG = {self.cfg.get("F_MAXREG", 255)};")
         o.append(f"    static constexpr bool F_BULK_STORE = {str(bool(self.cfg.get('F_BULK_STORE', 0))).lower()};")
         o.append(f"    using Vec = {vec};")
         o.append(f"    __device__ static __forceinline__ PairRec pair_rec(int i) {{ return kPair_{self.name}[i]; }}")
@@ -338,8 +344,8 @@ class Sig:
         o.append("    }")
 
         # ---- fwd_store
-        o.append(f"    template <int G>")
         o.append(f"    // writes the group's rows to dst[r * stride] (dst already offset by the lane and the first row)")
+        o.append(f"    template <int G>")
         o.append(f"    __device__ static __forceinline__ void fwd_store(const Vec (&acc)[F_RMAX], Vec* __restrict__ dst, const int stride) {{")
         for g in range(FW):
             o.append(f"        if constexpr (G == {g}) {{")
