@@ -343,7 +343,8 @@ int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
     if (!x1 || !x2 || !w || !grad_out) return E3J_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const FastKernels* fk = fast_lookup(plan);
-    if (fk && fk->tp_bwd) return fk->tp_bwd(rows, x1, x2, w, grad_out, grad_x1, grad_x2, grad_w, st);
+    if (fk && fk->tp_bwd && grad_x1 && grad_x2 && grad_w)
+        return fk->tp_bwd(rows, x1, x2, w, grad_out, grad_x1, grad_x2, grad_w, st);
     DeviceTables t;
     if (int s = get_device_tables(plan, t)) return s;
     const Dims dm = dims_of(plan);

@@ -32,6 +32,7 @@ struct BwdParams {
     float* dx_edge;                    // scratch [E][d][N_q]
     int64_t n_nodes, n_edges, chunk;   // chunk = edges per CTA
     int32_t* status;
+    int identity;                      // 1: every edge is its own sender and receiver; dx_edge is then grad_x itself
 };
 
 template <class S>
@@ -220,7 +221,10 @@ __device__ __forceinline__ void bwd_producer(const BwdParams& p, unsigned char* 
         if (t >= n_tiles) return;
         const int64_t e0 = e_begin + (int64_t)t * T;
         const int n_e = (int)min((int64_t)T, e_end - e0);
-        if (lane < n_e) { snd = p.senders[e0 + lane]; rcv = p.receivers[e0 + lane]; }
+        if (lane < n_e) {
+            if (p.identity) { snd = rcv = (int)(e0 + lane); }
+            else { snd = p.senders[e0 + lane]; rcv = p.receivers[e0 + lane]; }
+        }
 #pragma unroll
         for (int i = 0; i < YPL; ++i) {
             const int idx = i * 32 + lane;

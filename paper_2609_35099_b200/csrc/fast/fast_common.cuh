@@ -170,6 +170,7 @@ struct FwdParams {
     float* partial;                    // [G][2][D*NQ] boundary-row partial sums
     int32_t* part_recv;                // [G][2] receiver of the head / tail partial, or -1
     int32_t* status;                   // device status word (0 = fine)
+    int identity;                      // 1: every edge is its own sender and receiver (standalone tensor product)
 };
 
 // Sums the pieces of every receiver row that was split between CTAs, in CTA order.

@@ -78,9 +78,11 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
     const int cta = blockIdx.x;
     const int vlane = ch * 32 + lane;
     const int64_t row_elems = (int64_t)S::D * S::NQ;
-    const int prev_recv = (e_begin > 0 && e_begin < e_end) ? p.receivers[e_begin - 1] : -1;
-    const int next_recv = (e_end < p.n_edges) ? p.receivers[e_end] : -2;
-    if (warp == 0 && lane == 0) { p.part_recv[2 * cta] = -1; p.part_recv[2 * cta + 1] = -1; }
+    // identity mode: receiver of edge e is e, so no row ever straddles a CTA boundary
+    const int prev_recv = p.identity ? (int)e_begin - 1
+                                     : ((e_begin > 0 && e_begin < e_end) ? p.receivers[e_begin - 1] : -1);
+    const int next_recv = p.identity ? (int)e_end : ((e_end < p.n_edges) ? p.receivers[e_end] : -2);
+    if (!p.identity && warp == 0 && lane == 0) { p.part_recv[2 * cta] = -1; p.part_recv[2 * cta + 1] = -1; }
 
     // The CH warps of row group G share the group's A entries of a tile: each lane of the
     // CH*32 computes entries idx = pl, pl + CH*32, ... (entry idx -> edge idx / NP, slot idx % NP).
@@ -212,7 +214,7 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
     if (!*abort_flag) {
         if (cur >= 0) {
             flush(true);
-            if (e_end == p.n_edges) zero_rows(cur + 1, (int)p.n_nodes);
+            if (e_end == p.n_edges && !p.identity) zero_rows(cur + 1, (int)p.n_nodes);
         }
         if constexpr (S::F_BULK_STORE) bulk_wait_all();
     }
@@ -249,7 +251,10 @@ __device__ __forceinline__ void fwd_producer(const FwdParams& p, unsigned char* 
         if (t >= n_tiles) return;
         const int64_t e0 = e_begin + (int64_t)t * T;
         const int n_e = (int)min((int64_t)T, e_end - e0);
-        if (lane < n_e) { snd = p.senders[e0 + lane]; rcv = p.receivers[e0 + lane]; }
+        if (lane < n_e) {
+            if (p.identity) { snd = rcv = (int)(e0 + lane); }
+            else { snd = p.senders[e0 + lane]; rcv = p.receivers[e0 + lane]; }
+        }
 #pragma unroll
         for (int i = 0; i < YPL; ++i) {
             const int idx = i * 32 + lane;

@@ -66,6 +66,51 @@ int launch_fwd(const ConvArgs& a) {
     return after_launch();
 }
 
+// Standalone tensor product = the forward kernel with every row its own sender and receiver: no row
+// straddles a CTA boundary, so there is no scratch and no fix-up launch.
+template <class S>
+int launch_tp_fwd(int64_t rows, const float* x1, const float* x2, const float* w, float* out, cudaStream_t st) {
+    using L = FwdSmem<S>;
+    const int n_cta = sm_count() * S::FC;
+    static thread_local int attr_dev = -1;
+    int dev = 0;
+    E3J_CUDA_TRY(cudaGetDevice(&dev));
+    if (attr_dev != dev) {
+        E3J_CUDA_TRY(cudaFuncSetAttribute(fast_fwd_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));
+        attr_dev = dev;
+    }
+    FwdParams p{};
+    p.x = x1; p.sh = x2; p.w = w; p.out = out; p.n_nodes = rows; p.n_edges = rows; p.identity = 1;
+    const int64_t per = (rows + n_cta - 1) / n_cta;
+    p.chunk = (per + 3) / 4 * 4;
+    constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 1) * 32;
+    fast_fwd_kernel<S><<<n_cta, threads, L::total, st>>>(p);
+    return after_launch();
+}
+
+template <class S>
+int launch_tp_bwd(int64_t rows, const float* x1, const float* x2, const float* w, const float* g, float* gx1,
+                  float* gx2, float* gw, cudaStream_t st) {
+    using L = BwdSmem<S>;
+    if (!gx1 || !gx2 || !gw) return E3J_ERR_UNSUPPORTED;  // caller falls back to the generic kernels
+    const int n_cta = sm_count() * S::BC;
+    static thread_local int attr_dev = -1;
+    int dev = 0;
+    E3J_CUDA_TRY(cudaGetDevice(&dev));
+    if (attr_dev != dev) {
+        E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));
+        attr_dev = dev;
+    }
+    BwdParams p{};
+    p.x = x1; p.sh = x2; p.w = w; p.grad_out = g; p.grad_sh = gx2; p.grad_w = gw;
+    p.dx_edge = gx1;  // each row is its own sender: the per-edge share is the gradient
+    p.n_nodes = rows; p.n_edges = rows; p.identity = 1;
+    p.chunk = (rows + n_cta - 1) / n_cta;
+    constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;
+    fast_bwd_kernel<S><<<n_cta, threads, L::total, st>>>(p);
+    return after_launch();
+}
+
 // scratch of the backward: this edge's share of grad_x, [E][d][N_q]
 template <class S>
 size_t bwd_scratch_bytes(int64_t, int64_t n_edges) {

@@ -363,7 +363,8 @@ class Sig:
         o.append(f'    "{self.signature}",')
         if bwd_lines:
             o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, &fast::bwd_scratch_bytes<fast::{S}>, "
-                     f"&fast::launch_fwd<fast::{S}>, &fast::launch_bwd<fast::{S}>, nullptr, nullptr}};")
+                     f"&fast::launch_fwd<fast::{S}>, &fast::launch_bwd<fast::{S}>, &fast::launch_tp_fwd<fast::{S}>, "
+                     f"&fast::launch_tp_bwd<fast::{S}>}};")
         else:
             o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, nullptr, &fast::launch_fwd<fast::{S}>, nullptr, nullptr, nullptr}};")
         o.append("}  // namespace e3j")
