@@ -48,7 +48,8 @@ struct FwdSmem {
     static constexpr int X_EDGE = S::DIN * S::NQ;  // floats of one sender row
     static constexpr size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
     static constexpr size_t off_bar = 0;                                  // full[NS], empty[NS]
-    static constexpr size_t off_abort = off_bar + 16 * NS;
+    static constexpr size_t off_pair = off_bar + 16 * NS;                 // pair[FW]: a row group's warps have written their A shares
+    static constexpr size_t off_abort = off_pair + 8 * S::FW;
     static constexpr int FL_WARP = S::F_RMAX * 32 * S::V;                 // floats of one warp's store buffer
     static constexpr size_t off_flush = up(off_abort + 4, 128);           // float[warps][FL_WARP]
     static constexpr size_t off_stage = up(off_flush + (S::F_BULK_STORE ? 4 * (size_t)NCONS * FL_WARP : 0), 128);
@@ -107,14 +108,24 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
     }
     // A[e][slot] = sum over the slot's records of c * y[e][i2] for one landed tile
     // (entries of edges beyond the tile's length are computed from stale data and never read)
-    auto make_A = [&](unsigned char* st) {
+    uint64_t* pair = reinterpret_cast<uint64_t*>(smem + L::off_pair) + G;
+    int pair_phase = 0;
+    auto make_A = [&](unsigned char* st) -> bool {
         const float* y_t = reinterpret_cast<const float*>(st + L::st_y);
         AT* A_t = reinterpret_cast<AT*>(st + L::st_A);
 #pragma unroll
         for (int i = 0; i < NI; ++i)
             if (a_dst[i] >= 0)
                 a_store(A_t + a_dst[i], fmaf(a_tab[i].c1, y_t[a_tab[i].i2_1], a_tab[i].c0 * y_t[a_tab[i].i2_0]));
-        if constexpr (L::CH > 1) named_barrier_sync(1 + G, L::CH * 32); else __syncwarp();
+        __syncwarp();
+        if constexpr (L::CH > 1) {
+            // the group's other warps hold the rest of the entries (bounded wait, like every wait here)
+            if (lane == 0) mbar_arrive(pair);
+            const bool ok = mbar_wait(pair, pair_phase, abort_flag, p.status);
+            pair_phase ^= 1;
+            return ok;
+        }
+        return true;
     };
 
     Vec acc[S::F_RMAX];
@@ -176,7 +187,7 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
     int stage = 0, phase = 0;                 // ring slot of tile t and the parity of its use
     int left = (int)(e_end - e_begin);        // edges of this CTA not yet consumed
     bool ok = n_tiles > 0 && mbar_wait(&full[0], 0, abort_flag, p.status);
-    if (ok) make_A(smem + L::off_stage);
+    if (ok) ok = make_A(smem + L::off_stage);
     for (int t = 0; ok && t < n_tiles; ++t) {
         E3J_TICK(5)
         const unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
@@ -203,7 +214,7 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
             // next tile: wait for its data, then this warp's share of its A entries
             ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
             E3J_TICK(0)
-            if (ok) make_A(smem + L::off_stage + stage * (int)L::stage_bytes);
+            if (ok) ok = make_A(smem + L::off_stage + stage * (int)L::stage_bytes);
             E3J_TICK(1)
         }
     }
@@ -338,6 +349,7 @@ fast_fwd_kernel(const FwdParams p) {
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NCONS); }
+        for (int g = 0; g < S::FW; ++g) mbar_init(reinterpret_cast<uint64_t*>(smem + L::off_pair) + g, L::CH);
         *abort_flag = 0;
         mbar_fence_init();
     }
