@@ -146,11 +146,7 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
             xs += L::X_EDGE / S::BV; ss += L::S_EDGE / S::BV; As += S::B_APAD;
 
             // this warp's partial sums -> shared memory
-#ifdef E3J_DBG_NOBFLY
-            const float dy_tot = dyl[lane & 15];
-#else
             const float dy_tot = reduce16_over_lanes(dyl, lane);
-#endif
             if ((lane & 1) == 0) {
                 const int idx = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
                 dyp[(buf * NCONS + warp) * L::DYP + idx] = dy_tot;
@@ -159,24 +155,18 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
 #pragma unroll
             for (int i = 0; i < S::DIN; ++i) my[i * NQV] = dxp[i];
             // every consumer warp has deposited its partial sums (bounded wait, like every other wait here)
-#ifndef E3J_DBG_NOXCH
             __syncwarp();
             if (lane == 0) mbar_arrive(xch);
             alive = mbar_wait(xch, xphase, abort_flag, p.status);
             xphase ^= 1;
             if (!alive) break;
-#endif
             // fixed-order sums over the path groups / warps; rows and entries are dealt out to the warps
             for (int i1 = G; i1 < S::DIN; i1 += S::BW) {
                 Vec sum; vzero(sum);
 #pragma unroll
                 for (int g2 = 0; g2 < S::BW; ++g2)
                     sum = vadd(sum, reinterpret_cast<const Vec*>(dxs + (size_t)(buf * S::BW + g2) * L::X_EDGE)[i1 * NQV + vlane]);
-#ifndef E3J_DBG_NODXST
                 reinterpret_cast<Vec*>(p.dx_edge + (size_t)e * L::X_EDGE)[i1 * NQV + vlane] = sum;
-#else
-                if (sum.x == 1.2345f) reinterpret_cast<Vec*>(p.dx_edge + (size_t)e * L::X_EDGE)[i1 * NQV + vlane] = sum;
-#endif
             }
             if (warp == 0 && lane < S::DSH) {
                 float sum = 0.f;

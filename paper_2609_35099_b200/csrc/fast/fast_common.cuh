@@ -20,41 +20,9 @@ namespace fast {
 constexpr uint32_t kSpinLimit = 1u << 22;  // polls of mbarrier.try_wait before giving up
 constexpr int kStatusTimeout = 1;          // value stored in the device status word
 
-// ---------------------------------------------------------------- packed fp32 pairs
-// sm_100 executes two fp32 operations per lane in one instruction on a 64-bit register
-// pair (fma.rn.f32x2 / mul.rn.f32x2).  The per-channel arithmetic below is issue-bound,
-// so every channel vector is kept as packed pairs: u64 = 2 channels, ulonglong2 = 4.
-typedef unsigned long long u64;
-
-__device__ __forceinline__ u64 pk_fma(const u64 a, const u64 b, const u64 c) {
-    u64 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ u64 pk_mul(const u64 a, const u64 b) {
-    u64 d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ u64 pk_dup(const float a) {  // (a, a)
-    u64 d;
-    asm("mov.b64 %0, {%1, %1};" : "=l"(d) : "f"(a));
-    return d;
-}
-__device__ __forceinline__ u64 vmul(const u64 a, const u64 b) { return pk_mul(a, b); }
-__device__ __forceinline__ ulonglong2 vmul(const ulonglong2 a, const ulonglong2 b) {
-    return make_ulonglong2(pk_mul(a.x, b.x), pk_mul(a.y, b.y));
-}
-// acc += a * b with a = (A, A) a duplicated scalar
-__device__ __forceinline__ void vfma(u64& acc, const u64 a, const u64 b) { acc = pk_fma(a, b, acc); }
-__device__ __forceinline__ void vfma(ulonglong2& acc, const u64 a, const ulonglong2 b) {
-    acc.x = pk_fma(a, b.x, acc.x);
-    acc.y = pk_fma(a, b.y, acc.y);
-}
-__device__ __forceinline__ void vzero(u64& v) { v = 0ull; }
-__device__ __forceinline__ void vzero(ulonglong2& v) { v = make_ulonglong2(0ull, 0ull); }
-
-// plain fp32 vectors (one instruction per channel)
+// ---------------------------------------------------------------- channel vectors
+// A lane owns V consecutive channels (float2 or float4): one 8- or 16-byte shared-memory
+// load feeds V FMAs.
 __device__ __forceinline__ float4 vmul(const float4 a, const float4 b) {
     return make_float4(a.x * b.x, a.y * b.y, a.z * b.z, a.w * b.w);
 }
@@ -83,17 +51,9 @@ __device__ __forceinline__ float2 vadd(const float2 a, const float2 b) { return 
 __device__ __forceinline__ void vzero(float4& v) { v = make_float4(0.f, 0.f, 0.f, 0.f); }
 __device__ __forceinline__ void vzero(float2& v) { v = make_float2(0.f, 0.f); }
 
-// channel vector type: V channels per lane, packed pairs (PK) or plain floats
-template <int V, bool PK> struct VecOf;
-template <> struct VecOf<4, true> { using type = ulonglong2; };
-template <> struct VecOf<2, true> { using type = u64; };
-template <> struct VecOf<4, false> { using type = float4; };
-template <> struct VecOf<2, false> { using type = float2; };
-// element type of the A table in shared memory: the pair (A, A) or the scalar A
-template <bool PK> struct AOf { using type = float; };
-template <> struct AOf<true> { using type = u64; };
-__device__ __forceinline__ void a_store(u64* dst, const float a) { *dst = pk_dup(a); }
-__device__ __forceinline__ void a_store(float* dst, const float a) { *dst = a; }
+template <int V> struct VecOf;
+template <> struct VecOf<4> { using type = float4; };
+template <> struct VecOf<2> { using type = float2; };
 
 // ---------------------------------------------------------------- mbarrier / bulk copy (PTX)
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -139,19 +99,6 @@ __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, u
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
         ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
-// Contiguous shared -> global copy (asynchronous proxy); completion is tracked per issuing thread
-// with bulk_commit / bulk_wait_read.  Both addresses 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_s2g(void* dst_gmem, const void* src_smem, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                 ::"l"(dst_gmem), "r"(smem_u32(src_smem)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// all bulk stores committed by this thread have finished READING shared memory
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-// ... and have been written
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-// generic-proxy writes to shared memory become visible to the asynchronous proxy
-__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---------------------------------------------------------------- A-matrix tables
 // For every (i0,i1) pair slot: where its records start and how many there are.

@@ -25,13 +25,6 @@
 namespace e3j {
 namespace fast {
 
-#ifdef E3J_PROF
-// Cycle accounting for tuning (debug builds only): [cta][warp][phase] clock ticks.
-__device__ long long g_fwd_prof[1024 * 16 * 8];
-#define E3J_TICK(slot) { const long long _now = clock64(); prof_acc[slot] += _now - prof_t; prof_t = _now; }
-#else
-#define E3J_TICK(slot)
-#endif
 
 // Per A slot: up to two records, A = c0 * y[i2_0] + c1 * y[i2_1].
 struct ASlot {
@@ -50,13 +43,11 @@ struct FwdSmem {
     static constexpr size_t off_bar = 0;                                  // full[NS], empty[NS]
     static constexpr size_t off_pair = off_bar + 16 * NS;                 // pair[FW]: a row group's warps have written their A shares
     static constexpr size_t off_abort = off_pair + 8 * S::FW;
-    static constexpr int FL_WARP = S::F_RMAX * 32 * S::V;                 // floats of one warp's store buffer
-    static constexpr size_t off_flush = up(off_abort + 4, 128);           // float[warps][FL_WARP]
-    static constexpr size_t off_stage = up(off_flush + (S::F_BULK_STORE ? 4 * (size_t)NCONS * FL_WARP : 0), 128);
+    static constexpr size_t off_stage = up(off_abort + 4, 128);
     static constexpr size_t st_s = 0;
     static constexpr size_t st_x = st_s + 4 * (size_t)T * S_EDGE;
-    static constexpr size_t st_A = st_x + 4 * (size_t)T * X_EDGE;         // A[T][APAD]: scalars, or duplicated pairs when S::PK
-    static constexpr size_t st_y = st_A + (S::PK ? 8 : 4) * (size_t)T * S::F_APAD;
+    static constexpr size_t st_A = st_x + 4 * (size_t)T * X_EDGE;         // float A[T][APAD]
+    static constexpr size_t st_y = st_A + 4 * (size_t)T * S::F_APAD;
     static constexpr size_t st_r = st_y + 4 * (size_t)T * S::DSH;         // recv[T], change mask
     static constexpr size_t stage_bytes = up(st_r + 4 * (T + 1), 128);
     static constexpr size_t total = off_stage + NS * stage_bytes;
@@ -67,8 +58,7 @@ template <class S, int G>
 __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* smem, const int ch, const int warp,
                                              const int lane, const int64_t e_begin, const int64_t e_end,
                                              const int n_tiles) {
-    using Vec = typename VecOf<S::V, S::PK>::type;
-    using AT = typename AOf<S::PK>::type;
+    using Vec = typename VecOf<S::V>::type;
     using L = FwdSmem<S>;
     constexpr int T = L::T, NS = L::NS;
     constexpr int NQV = S::NQ / S::V;
@@ -112,11 +102,11 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
     int pair_phase = 0;
     auto make_A = [&](unsigned char* st) -> bool {
         const float* y_t = reinterpret_cast<const float*>(st + L::st_y);
-        AT* A_t = reinterpret_cast<AT*>(st + L::st_A);
+        float* A_t = reinterpret_cast<float*>(st + L::st_A);
 #pragma unroll
         for (int i = 0; i < NI; ++i)
             if (a_dst[i] >= 0)
-                a_store(A_t + a_dst[i], fmaf(a_tab[i].c1, y_t[a_tab[i].i2_1], a_tab[i].c0 * y_t[a_tab[i].i2_0]));
+                A_t[a_dst[i]] = (fmaf(a_tab[i].c1, y_t[a_tab[i].i2_1], a_tab[i].c0 * y_t[a_tab[i].i2_0]));
         __syncwarp();
         if constexpr (L::CH > 1) {
             // the group's other warps hold the rest of the entries (bounded wait, like every wait here)
@@ -142,9 +132,7 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
             for (int row = ROW0; row < ROW1; ++row) dst[(size_t)row * NQV] = zero;
         }
     };
-    // Finished rows are either stored directly or (S::F_BULK_STORE) staged in shared memory
-    // and written by a bulk asynchronous store, which frees the accumulator registers at once.
-    Vec* fl = reinterpret_cast<Vec*>(smem + L::off_flush) + (size_t)warp * (L::FL_WARP / S::V);
+    // A finished row goes straight to global memory (its final place, or this CTA's partial-row slot).
     auto flush = [&](bool at_end) {
         const bool head = seg_first && cur == prev_recv;
         const bool tail = at_end && cur == next_recv;
@@ -158,19 +146,7 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
         } else {
             base = p.out + (size_t)cur * row_elems;
         }
-        if constexpr (S::F_BULK_STORE) {
-            if (lane < ROW1 - ROW0) bulk_wait_read();  // the previous use of the buffer has been read out
-            __syncwarp();
-            S::template fwd_store<G>(acc, fl + lane, 32);
-            fence_async_shared();
-            __syncwarp();
-            if (lane < ROW1 - ROW0) {
-                bulk_s2g(base + (size_t)(ROW0 + lane) * S::NQ + ch * 32 * S::V, fl + lane * 32, 32 * S::V * 4);
-                bulk_commit();
-            }
-        } else {
-            S::template fwd_store<G>(acc, reinterpret_cast<Vec*>(base) + (size_t)ROW0 * NQV + vlane, NQV);
-        }
+        S::template fwd_store<G>(acc, reinterpret_cast<Vec*>(base) + (size_t)ROW0 * NQV + vlane, NQV);
     };
     auto new_receiver = [&](const int r) {
         if (cur >= 0) { flush(false); seg_first = false; }
@@ -180,16 +156,11 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
         for (int q = 0; q < S::F_RMAX; ++q) vzero(acc[q]);
     };
 
-#ifdef E3J_PROF
-    long long prof_acc[6] = {0, 0, 0, 0, 0, 0};
-    long long prof_t = clock64();
-#endif
     int stage = 0, phase = 0;                 // ring slot of tile t and the parity of its use
     int left = (int)(e_end - e_begin);        // edges of this CTA not yet consumed
     bool ok = n_tiles > 0 && mbar_wait(&full[0], 0, abort_flag, p.status);
     if (ok) ok = make_A(smem + L::off_stage);
     for (int t = 0; ok && t < n_tiles; ++t) {
-        E3J_TICK(5)
         const unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
         const int n_e = min(T, left);
         left -= T;
@@ -197,7 +168,7 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
         unsigned mask = (unsigned)recv_t[T];  // bit i: edge i starts a new receiver
         const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + vlane;
         const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + vlane;
-        const AT* As = reinterpret_cast<const AT*>(st + L::st_A);
+        const float* As = reinterpret_cast<const float*>(st + L::st_A);
         // one compact body per edge: a longer (unrolled) loop costs more in instruction fetch than it saves
 #pragma unroll 1
         for (int e_i = 0; e_i < n_e; ++e_i) {
@@ -206,28 +177,20 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
             S::template fwd_edge<G>(acc, xs, ss, As);
             xs += L::X_EDGE / S::V; ss += L::S_EDGE / S::V; As += S::F_APAD;
         }
-        E3J_TICK(2)
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[stage]);
         if (++stage == NS) { stage = 0; phase ^= 1; }
         if (t + 1 < n_tiles) {
             // next tile: wait for its data, then this warp's share of its A entries
             ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
-            E3J_TICK(0)
             if (ok) ok = make_A(smem + L::off_stage + stage * (int)L::stage_bytes);
-            E3J_TICK(1)
         }
     }
-#ifdef E3J_PROF
-    if (lane == 0 && blockIdx.x < 1024)
-        for (int i = 0; i < 6; ++i) g_fwd_prof[(blockIdx.x * 16 + warp) * 8 + i] = prof_acc[i];
-#endif
     if (!*abort_flag) {
         if (cur >= 0) {
             flush(true);
             if (e_end == p.n_edges && !p.identity) zero_rows(cur + 1, (int)p.n_nodes);
         }
-        if constexpr (S::F_BULK_STORE) bulk_wait_all();
     }
 }
 
@@ -250,7 +213,6 @@ template <class S>
 __device__ __forceinline__ void fwd_producer(const FwdParams& p, unsigned char* smem, const int warp, const int lane,
                                              const int64_t e_begin, const int64_t e_end, const int n_tiles) {
     using L = FwdSmem<S>;
-    using AT = typename AOf<S::PK>::type;
     constexpr int T = L::T, NS = L::NS;
     constexpr int YPL = (T * S::DSH + 31) / 32;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
@@ -274,15 +236,10 @@ __device__ __forceinline__ void fwd_producer(const FwdParams& p, unsigned char* 
     };
     load_meta(0, snd_a, rcv_a, y_a);
     load_meta(1, snd_b, rcv_b, y_b);
-#ifdef E3J_PROF
-    long long prof_acc[6] = {0, 0, 0, 0, 0, 0};
-    long long prof_t = clock64();
-#endif
     int armed = 0, last_rcv = -1, stage = 0, phase = 0;
     for (int t = 0; t < n_tiles; ++t) {
         // phase of `empty` that ends the previous use of this ring slot
         if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
-        E3J_TICK(0)
         unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
         const int64_t e0 = e_begin + (int64_t)t * T;
         const int n_e = (int)min((int64_t)T, e_end - e0);
@@ -310,17 +267,12 @@ __device__ __forceinline__ void fwd_producer(const FwdParams& p, unsigned char* 
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&full[stage]);  // the staged harmonics / receiver ids are in place
-        E3J_TICK(1)
         snd_a = snd_b; rcv_a = rcv_b;
 #pragma unroll
         for (int i = 0; i < YPL; ++i) y_a[i] = y_b[i];
         load_meta(t + 2, snd_b, rcv_b, y_b);
         if (++stage == NS) { stage = 0; phase ^= 1; }
     }
-#ifdef E3J_PROF
-    if (lane == 0 && blockIdx.x < 1024)
-        for (int i = 0; i < 6; ++i) g_fwd_prof[(blockIdx.x * 16 + warp) * 8 + i] = prof_acc[i];
-#endif
     if (*abort_flag) {
         // let copies already in flight land before the CTA's shared memory is released
         for (int t = max(0, armed - NS); t < armed; ++t)

@@ -148,10 +148,3 @@ int launch_bwd(const ConvArgs& a) {
 
 }  // namespace fast
 }  // namespace e3j
-
-#ifdef E3J_PROF
-// debug builds only: copies the forward kernel's cycle counters to the host
-extern "C" __attribute__((weak)) int e3j_debug_fwd_prof(long long* host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, e3j::fast::g_fwd_prof, sizeof(long long) * n);
-}
-#endif

@@ -110,7 +110,7 @@ class Sig:
         for g in range(FW):
             for row in range(bounds[g], bounds[g + 1]):
                 slots += self.row_pairs[row]
-            while len(slots) % (2 if self.cfg.get('PK', 0) else 4):
+            while len(slots) % 4:
                 slots.append(None)
             a0.append(len(slots))
         return bounds, a0, slots
@@ -207,19 +207,15 @@ class Sig:
                         i1 = self.pairs[pi][1]
                         r = row - row0[g]
                         o.append(f"            vfma(u{k}_{i1}, a{q}.{lane}, dm[{r}]);")
-                        if not self.cfg.get("DBG_NODY"):
-                            o.append(f"            {{ const float t = vdot(sx{k}_{i1}, dm[{r}]);")
-                            for i2, c in self.pairs[pi][3]:
-                                o.append(f"              dyl[{i2}] = fmaf({fmt_float(c)}, t, dyl[{i2}]);")
-                            o.append("            }")
+                        o.append(f"            {{ const float t = vdot(sx{k}_{i1}, dm[{r}]);")
+                        for i2, c in self.pairs[pi][3]:
+                            o.append(f"              dyl[{i2}] = fmaf({fmt_float(c)}, t, dyl[{i2}]);")
+                        o.append("            }")
                 first = used[0]
                 o.append(f"            BVec ds{k} = vmul(x{first}, u{k}_{first});")
                 for i1 in used[1:]:
                     o.append(f"            vfma(ds{k}, x{i1}, u{k}_{i1});")
-                if self.cfg.get("DBG_NODS"):
-                    o.append(f"            if (ds{k}.x == 1.2345f) gw[{k} * NQV] = ds{k};")
-                else:
-                    o.append(f"            gw[{k} * NQV] = ds{k};")
+                o.append(f"            gw[{k} * NQV] = ds{k};")
                 for i1 in used:
                     o.append(f"            vfma(dxp[{i1}], s{k}, u{k}_{i1});")
             o.append("        } break;")
@@ -234,8 +230,7 @@ class Sig:
         bounds, a0, slots = self.fwd_layout()
         slot_of_pair = {pi: s for s, pi in enumerate(slots) if pi is not None}
         rmax = max(bounds[g + 1] - bounds[g] for g in range(FW))
-        PK = bool(self.cfg.get("PK", 0))
-        vec = ({2: "u64", 4: "ulonglong2"} if PK else {2: "float2", 4: "float4"})[V]
+        vec = {2: "float2", 4: "float4"}[V]
         # record tables in slot order
         rec_val, rec_i2, pair_tab = [], [], []
         for pi in slots:
@@ -277,10 +272,7 @@ class Sig:
         o.append(f"struct {S} {{")
         o.append(f"    static constexpr int NQ = {NQ}, DIN = {self.DIN}, DSH = {self.DSH}, P = {self.P}, D = {self.D};")
         o.append(f"    static constexpr int NNZ = {self.NNZ}, NPAIR = {len(self.pairs)}, V = {V};")
-        o.append(f"    static constexpr bool PK = {str(PK).lower()};  // packed fp32 pairs (fma.rn.f32x2) or plain fp32")
-        o.append(f"    using AT = {'u64' if PK else 'float'};")
         o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, FC = {FC}, F_RMAX = {rmax}, F_APAD = {len(slots)}, F_NREC = {max(c for _, c in pair_tab)}, F_NPMAX = {max(a0[g + 1] - a0[g] for g in range(FW))}, F_MAXREG = {self.cfg.get("F_MAXREG", 255)};")
-        o.append(f"    static constexpr bool F_BULK_STORE = {str(bool(self.cfg.get('F_BULK_STORE', 0))).lower()};")
         o.append(f"    using Vec = {vec};")
         o.append(f"    __device__ static __forceinline__ PairRec pair_rec(int i) {{ return kPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float rec_val(int i) {{ return kVal_{self.name}[i]; }}")
@@ -300,7 +292,7 @@ class Sig:
         # ---- fwd_edge
         o.append(f"    template <int G>")
         o.append(f"    __device__ static __forceinline__ void fwd_edge(Vec (&acc)[F_RMAX], "
-                 f"const Vec* __restrict__ xs, const Vec* __restrict__ ss, const AT* __restrict__ As) {{")
+                 f"const Vec* __restrict__ xs, const Vec* __restrict__ ss, const float* __restrict__ As) {{")
         o.append(f"        constexpr int NQV = NQ / V;")
         for g in range(FW):
             o.append(f"        if constexpr (G == {g}) {{")
@@ -328,16 +320,10 @@ class Sig:
                             continue
                         pi = self.row_pairs[row][j]
                         slot = slot_of_pair[pi]
-                        if PK:
-                            q, lane = slot // 2, "xy"[slot % 2]
-                            if q not in loaded_a:
-                                loaded_a.add(q)
-                                o.append(f"            const ulonglong2 a{q} = *reinterpret_cast<const ulonglong2*>(As + {2 * q});")
-                        else:
-                            q, lane = slot // 4, "xyzw"[slot % 4]
-                            if q not in loaded_a:
-                                loaded_a.add(q)
-                                o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
+                        q, lane = slot // 4, "xyzw"[slot % 4]
+                        if q not in loaded_a:
+                            loaded_a.add(q)
+                            o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
                         i1 = self.pairs[pi][1]
                         o.append(f"            vfma(acc[{row - bounds[g]}], a{q}.{lane}, sx{k}_{i1});")
             o.append("        }")
