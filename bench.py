@@ -49,8 +49,8 @@ def measured_peak():
 # profiles/fast_fwd_kernel_water3000.txt, profiles/fast_bwd_kernel_water3000.txt and the launch-list run
 # (specialised kernels, workload water3000).  Other workloads / the generic kernels report null.
 NCU_TRAFFIC = {
-    ("water3000", "fwd"): 1.110510e9 + 0.082842e9 + 0.016341e9,          # fast_fwd_kernel + fwd_fixup_kernel
-    ("water3000", "bwd"): 1.259801e9 + 1.363752e9 + 0.330465e9 + 0.0020e9,  # fast_bwd_kernel + bwd_dx_reduce_kernel
+    ("water3000", "fwd"): 1.110601e9 + 0.086230e9 + 0.016343e9,          # fast_fwd_kernel + fwd_fixup_kernel
+    ("water3000", "bwd"): 1.260743e9 + 1.361455e9 + 0.330491e9 + 0.0018e9,  # fast_bwd_kernel + bwd_dx_reduce_kernel
 }
 
 
@@ -168,13 +168,84 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_tp(args, e3j, workloads, torch, dev, rank, world, barrier):
+    """Secondary workload: the standalone tensor product (rows are their own senders and receivers).
+
+    The arrays are tens of GB at 2^20 rows, so they are drawn on the device with a seeded generator; there is
+    no end-to-end or CPU leg for this workload (the headline workload carries those).
+    """
+    import torch.distributed as dist
+    c = workloads.CONFIGS[4]
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"],
+                               e3j.E3J_PLAN_GENERIC_ONLY if args.generic else 0)
+    rows, nq = args.rows, plan.n_channels
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4 + rank)
+    x1 = torch.randn((rows, plan.d_in, nq), device=dev, generator=gen)
+    x2 = torch.randn((rows, plan.d_sh), device=dev, generator=gen)
+    w = torch.randn((rows, plan.n_paths, nq), device=dev, generator=gen)
+    g = torch.randn((rows, plan.d_out, nq), device=dev, generator=gen)
+    out = torch.empty_like(g)
+    g1, g2, gw = torch.empty_like(x1), torch.empty_like(x2), torch.empty_like(w)
+    stream = torch.cuda.current_stream()
+    fwd = lambda: e3j.e3j_tp_fwd(plan, x1, x2, w, out=out)
+    bwd = lambda: e3j.e3j_tp_bwd(plan, x1, x2, w, g, grad_x1=g1, grad_x2=g2, grad_w=gw)
+    for _ in range(args.warmup):
+        fwd(); bwd()
+    torch.cuda.synchronize()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    marks = [(ev(), ev(), ev()) for _ in range(args.steps)]
+    sampler = ClockSampler(dev.index) if rank == 0 else None
+    launches0 = e3j.e3j_launch_count()
+    barrier(); torch.cuda.synchronize()
+    for a, b, cc in marks:
+        a.record(stream); fwd(); b.record(stream); bwd(); cc.record(stream)
+    torch.cuda.synchronize(); barrier()
+    launches = e3j.e3j_launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    total_ms = marks[0][0].elapsed_time(marks[-1][2])
+    if world > 1:
+        tm = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        total_ms = float(tm.item())
+    if rank != 0:
+        return
+    f_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in marks)
+    b_ms = statistics.mean(b.elapsed_time(cc) for _, b, cc in marks)
+    peak, peak_src = measured_peak()
+    prim = 4 * rows * (plan.d_in * nq + plan.d_sh + plan.n_paths * nq)
+    fb = prim + 4 * rows * plan.d_out * nq
+    bb = fb + prim
+
+    def roof(nbytes, ms, kernel):
+        ach = nbytes / (ms * 1e-3) / 1e9
+        return {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "peak_source": peak_src,
+                "algorithmic_bytes_per_launch": nbytes, "avg_ms": ms, "traffic": None}
+
+    roofs = {"fwd": roof(fb, f_ms, "e3j_tp_fwd call"), "bwd": roof(bb, b_ms, "e3j_tp_bwd call")}
+    ms_per_step = total_ms / args.steps
+    print(json.dumps({
+        "metric": "tp_fwd_bwd_rows_per_s", "value": rows * world / (ms_per_step * 1e-3), "unit": "rows/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic (seeded device generator)",
+        "config": {"workload": f"tp rows={rows} {c['irreps_in']} (x) l<={c['sh_lmax']}", "rows_per_gpu": rows,
+                   "specialised_kernels": bool(plan.specialised), "l2": "inputs larger than L2"},
+        "clocks": clocks, "e2e": None, "gpu_launches": launches, "fwd_ms": f_ms, "bwd_ms": b_ms,
+        "roofline": roofs["bwd"] if b_ms >= f_ms else roofs["fwd"], "roofline_fwd": roofs["fwd"],
+        "roofline_bwd": roofs["bwd"], "cpu_baseline": None}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 5])
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5],
+                    help="2 = headline workload; 3 / 5 = other convolution workloads; 4 = standalone tensor product rows")
+    ap.add_argument("--rows", type=int, default=1 << 20, help="rows of the tensor-product workload (--config 4)")
     ap.add_argument("--generic", action="store_true", help="force the table-driven generic kernels")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -206,6 +277,10 @@ def main():
     def barrier():
         if world > 1:
             dist.barrier()
+
+    if args.config == 4:
+        run_tp(args, e3j, workloads, torch, dev, rank, world, barrier)
+        return
 
     c, wl = build_workload(args.config)
     plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"],
@@ -306,7 +381,7 @@ def main():
         spec = bool(plan.specialised)
         roofs = {"fwd": roof(fb, f_ms, "e3j_conv_fwd call: fast_fwd_kernel (96 %) + fwd_fixup_kernel" if spec
                              else "e3j_conv_fwd call: generic conv_fwd_kernel", "fwd"),
-                 "bwd": roof(bb, b_ms, "e3j_conv_bwd call: fast_bwd_kernel (93 %) + bwd_dx_reduce_kernel" if spec
+                 "bwd": roof(bb, b_ms, "e3j_conv_bwd call: fast_bwd_kernel (91 %) + bwd_dx_reduce_kernel" if spec
                              else "e3j_conv_bwd call: generic edge + node kernels", "bwd")}
         dominant = roofs["bwd"] if b_ms >= f_ms else roofs["fwd"]
         line = {
