@@ -275,6 +275,7 @@ __device__ __forceinline__ void bwd_producer(const BwdParams& p, unsigned char* 
     }
     if (*abort_flag) {
         for (int t = max(0, armed - NS); t < armed; ++t)
+#pragma unroll 1
             for (uint32_t it = 0; it < kSpinLimit; ++it)
                 if (mbar_try_wait(&full[t % NS], (t / NS) & 1)) break;
     }

@@ -15,10 +15,10 @@
 // the path sum (paper, "Factoring out the edge scalar").
 //
 // Warps g, g+FW, ... land on the same SM sub-partition and run the same specialised
-// body, so each sub-partition's instruction stream is one compact loop.  The last warp
-// of the CTA is the producer: it issues the bulk copies of a tile and stages the tile's
-// harmonics and receiver ids.  The warps of a row group compute the group's A entries of
-// the next tile right after finishing the current one.
+// body, so each sub-partition's instruction stream is one compact loop.  The last two
+// warps of the CTA are producers: one issues the copies of a tile, the other stages the
+// tile's receiver ids and computes its A entries, so the consumers' instruction stream
+// is the per-edge body and nothing else.
 #pragma once
 #include "fast_common.cuh"
 
@@ -41,8 +41,7 @@ struct FwdSmem {
     static constexpr int X_EDGE = S::DIN * S::NQ;  // floats of one sender row
     static constexpr size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
     static constexpr size_t off_bar = 0;                                  // full[NS], empty[NS]
-    static constexpr size_t off_pair = off_bar + 16 * NS;                 // pair[FW]: a row group's warps have written their A shares
-    static constexpr size_t off_abort = off_pair + 8 * S::FW;
+    static constexpr size_t off_abort = off_bar + 16 * NS;
     static constexpr size_t off_stage = up(off_abort + 4, 128);
     static constexpr size_t st_s = 0;
     static constexpr size_t st_x = st_s + 4 * (size_t)T * S_EDGE;
@@ -74,49 +73,6 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
                                      : ((e_begin > 0 && e_begin < e_end) ? p.receivers[e_begin - 1] : -1);
     const int next_recv = p.identity ? (int)e_end : ((e_end < p.n_edges) ? p.receivers[e_end] : -2);
     if (!p.identity && warp == 0 && lane == 0) { p.part_recv[2 * cta] = -1; p.part_recv[2 * cta + 1] = -1; }
-
-    // The CH warps of row group G share the group's A entries of a tile: each lane of the
-    // CH*32 computes entries idx = pl, pl + CH*32, ... (entry idx -> edge idx / NP, slot idx % NP).
-    constexpr int A0 = S::f_a0(G), NP = S::f_a0(G + 1) - A0;
-    constexpr int NI = (T * NP + L::CH * 32 - 1) / (L::CH * 32);
-    ASlot a_tab[NI];
-    int a_dst[NI];
-    {
-        const int pl = ch * 32 + lane;
-#pragma unroll
-        for (int i = 0; i < NI; ++i) {
-            const int idx = pl + L::CH * 32 * i;
-            const bool valid = idx < T * NP;
-            const int e_i = valid ? idx / NP : 0, slot = A0 + (valid ? idx % NP : 0);
-            const PairRec pr = S::pair_rec(slot);
-            ASlot a{0.f, 0.f, 0, 0};
-            if (valid && pr.count > 0) { a.c0 = S::rec_val(pr.start); a.i2_0 = e_i * S::DSH + S::rec_i2(pr.start); }
-            if (valid && pr.count > 1) { a.c1 = S::rec_val(pr.start + 1); a.i2_1 = e_i * S::DSH + S::rec_i2(pr.start + 1); }
-            a_tab[i] = a;
-            a_dst[i] = valid ? e_i * S::F_APAD + slot : -1;
-        }
-    }
-    // A[e][slot] = sum over the slot's records of c * y[e][i2] for one landed tile
-    // (entries of edges beyond the tile's length are computed from stale data and never read)
-    uint64_t* pair = reinterpret_cast<uint64_t*>(smem + L::off_pair) + G;
-    int pair_phase = 0;
-    auto make_A = [&](unsigned char* st) -> bool {
-        const float* y_t = reinterpret_cast<const float*>(st + L::st_y);
-        float* A_t = reinterpret_cast<float*>(st + L::st_A);
-#pragma unroll
-        for (int i = 0; i < NI; ++i)
-            if (a_dst[i] >= 0)
-                A_t[a_dst[i]] = (fmaf(a_tab[i].c1, y_t[a_tab[i].i2_1], a_tab[i].c0 * y_t[a_tab[i].i2_0]));
-        __syncwarp();
-        if constexpr (L::CH > 1) {
-            // the group's other warps hold the rest of the entries (bounded wait, like every wait here)
-            if (lane == 0) mbar_arrive(pair);
-            const bool ok = mbar_wait(pair, pair_phase, abort_flag, p.status);
-            pair_phase ^= 1;
-            return ok;
-        }
-        return true;
-    };
 
     Vec acc[S::F_RMAX];
 #pragma unroll
@@ -159,7 +115,6 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
     int stage = 0, phase = 0;                 // ring slot of tile t and the parity of its use
     int left = (int)(e_end - e_begin);        // edges of this CTA not yet consumed
     bool ok = n_tiles > 0 && mbar_wait(&full[0], 0, abort_flag, p.status);
-    if (ok) ok = make_A(smem + L::off_stage);
     for (int t = 0; ok && t < n_tiles; ++t) {
         const unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
         const int n_e = min(T, left);
@@ -169,22 +124,26 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
         const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + vlane;
         const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + vlane;
         const float* As = reinterpret_cast<const float*>(st + L::st_A);
-        // one compact body per edge: a longer (unrolled) loop costs more in instruction fetch than it saves
-#pragma unroll 1
-        for (int e_i = 0; e_i < n_e; ++e_i) {
+        // Runs of edges with the same receiver: the inner loop is the bare per-edge body with no receiver
+        // test in it (with the test inside, the same body ran 40 % slower), and it is not unrolled (a longer
+        // loop costs more in instruction fetch than it saves).
+        int e_i = 0;
+        while (e_i < n_e) {
             if (mask & 1u) new_receiver(recv_t[e_i]);
-            mask >>= 1;
-            S::template fwd_edge<G>(acc, xs, ss, As);
-            xs += L::X_EDGE / S::V; ss += L::S_EDGE / S::V; As += S::F_APAD;
+            mask >>= 1;                                        // bit 0 now belongs to edge e_i + 1
+            const int run = min(mask ? __ffs((int)mask) : T, n_e - e_i);
+            mask >>= run - 1;
+            e_i += run;
+#pragma unroll 1
+            for (int j = 0; j < run; ++j) {
+                S::template fwd_edge<G>(acc, xs, ss, As);
+                xs += L::X_EDGE / S::V; ss += L::S_EDGE / S::V; As += S::F_APAD;
+            }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[stage]);
         if (++stage == NS) { stage = 0; phase ^= 1; }
-        if (t + 1 < n_tiles) {
-            // next tile: wait for its data, then this warp's share of its A entries
-            ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
-            if (ok) ok = make_A(smem + L::off_stage + stage * (int)L::stage_bytes);
-        }
+        if (t + 1 < n_tiles) ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
     }
     if (!*abort_flag) {
         if (cur >= 0) {
@@ -208,52 +167,114 @@ struct FwdDispatch<S, S::FW> {
     __device__ static __forceinline__ void run(const int, Args&&...) {}
 };
 
-// ------------------------------------------------------------------------ producer
+// ------------------------------------------------------------------------ producers
+// Two warps feed the ring.  The copy warp waits for a free slot and issues the tile's copies at once;
+// the table warp stages the tile's receiver ids and computes its A entries.  A tile is "full" when the
+// bulk copy's bytes, the 32 deferred arrivals of the sender-row copies and the table warp's arrival are in.
 template <class S>
-__device__ __forceinline__ void fwd_producer(const FwdParams& p, unsigned char* smem, const int warp, const int lane,
-                                             const int64_t e_begin, const int64_t e_end, const int n_tiles) {
+__device__ __forceinline__ void fwd_copy_producer(const FwdParams& p, unsigned char* smem, const int lane,
+                                                  const int64_t e_begin, const int64_t e_end, const int n_tiles) {
     using L = FwdSmem<S>;
     constexpr int T = L::T, NS = L::NS;
-    constexpr int YPL = (T * S::DSH + 31) / 32;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
     uint64_t* empty = full + NS;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
-    int snd_a = 0, rcv_a = -1, snd_b = 0, rcv_b = -1;
-    float y_a[YPL], y_b[YPL];
-    auto load_meta = [&](int t, int& snd, int& rcv, float (&yv)[YPL]) {
+    int snd_a = 0, snd_b = 0;
+    auto load_snd = [&](int t, int& snd) {  // sender ids two tiles ahead of their use
         if (t >= n_tiles) return;
         const int64_t e0 = e_begin + (int64_t)t * T;
         const int n_e = (int)min((int64_t)T, e_end - e0);
-        if (lane < n_e) {
-            if (p.identity) { snd = rcv = (int)(e0 + lane); }
-            else { snd = p.senders[e0 + lane]; rcv = p.receivers[e0 + lane]; }
-        }
-#pragma unroll
-        for (int i = 0; i < YPL; ++i) {
-            const int idx = i * 32 + lane;
-            if (idx < n_e * S::DSH) yv[i] = p.sh[e0 * S::DSH + idx];
-        }
+        if (lane < n_e) snd = p.identity ? (int)(e0 + lane) : p.senders[e0 + lane];
     };
-    load_meta(0, snd_a, rcv_a, y_a);
-    load_meta(1, snd_b, rcv_b, y_b);
-    int armed = 0, last_rcv = -1, stage = 0, phase = 0;
+    load_snd(0, snd_a);
+    load_snd(1, snd_b);
+    int armed = 0, stage = 0, phase = 0;
+#pragma unroll 1
     for (int t = 0; t < n_tiles; ++t) {
         // phase of `empty` that ends the previous use of this ring slot
         if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
         unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
         const int64_t e0 = e_begin + (int64_t)t * T;
         const int n_e = (int)min((int64_t)T, e_end - e0);
-        int* recv_t = reinterpret_cast<int*>(st + L::st_r);
-        float* y_t = reinterpret_cast<float*>(st + L::st_y);
-        // copies first: they are the long pole
+        // The tile's weights are one bulk copy; the gathered sender rows go as 16-byte asynchronous copies
+        // from all lanes (a bulk copy per row holds the issuing lane for ~150 cycles each), counted on the
+        // same barrier by one deferred arrival per lane.
         if (lane == 0) {
-            mbar_expect_tx(&full[stage], (uint32_t)n_e * (uint32_t)(4 * (L::S_EDGE + L::X_EDGE)));
+            mbar_expect_tx(&full[stage], (uint32_t)n_e * 4u * L::S_EDGE);
             bulk_g2s(st + L::st_s, p.w + (size_t)e0 * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE, &full[stage]);
         }
-        if (lane < n_e)
-            bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE, p.x + (size_t)snd_a * L::X_EDGE, 4u * L::X_EDGE,
-                     &full[stage]);
+#pragma unroll
+        for (int e_i = 0; e_i < T; ++e_i) {
+            const int snd = __shfl_sync(0xffffffffu, snd_a, e_i);
+            if (e_i < n_e) {
+                const char* src = reinterpret_cast<const char*>(p.x + (size_t)snd * L::X_EDGE);
+                unsigned char* dst = st + L::st_x + (size_t)e_i * 4 * L::X_EDGE;
+#pragma unroll
+                for (int c = 0; c < (4 * L::X_EDGE) / (16 * 32); ++c)
+                    cp_async16(dst + 16 * (c * 32 + lane), src + 16 * (c * 32 + lane));
+            }
+        }
+        cp_async_arrive_noinc(&full[stage]);
         armed = t + 1;
+        snd_a = snd_b;
+        load_snd(t + 2, snd_b);
+        if (++stage == NS) { stage = 0; phase ^= 1; }
+    }
+    if (*abort_flag) {
+        // let copies already in flight land before the CTA's shared memory is released
+        for (int t = max(0, armed - NS); t < armed; ++t)
+#pragma unroll 1
+            for (uint32_t it = 0; it < kSpinLimit; ++it)
+                if (mbar_try_wait(&full[t % NS], (t / NS) & 1)) break;
+    }
+}
+
+template <class S>
+__device__ __forceinline__ void fwd_table_producer(const FwdParams& p, unsigned char* smem, const int lane,
+                                                   const int64_t e_begin, const int64_t e_end, const int n_tiles) {
+    using L = FwdSmem<S>;
+    constexpr int T = L::T, NS = L::NS;
+    constexpr int YPL = (T * S::DSH + 31) / 32;
+    constexpr int NA = (S::F_APAD + 31) / 32;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
+    uint64_t* empty = full + NS;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
+    ASlot tab[NA];  // this lane's A slots (lane, lane + 32, ...)
+#pragma unroll
+    for (int i = 0; i < NA; ++i) {
+        const int slot = lane + 32 * i;
+        ASlot a{0.f, 0.f, 0, 0};
+        if (slot < S::F_APAD) {
+            const PairRec pr = S::pair_rec(slot);
+            if (pr.count > 0) { a.c0 = S::rec_val(pr.start); a.i2_0 = S::rec_i2(pr.start); }
+            if (pr.count > 1) { a.c1 = S::rec_val(pr.start + 1); a.i2_1 = S::rec_i2(pr.start + 1); }
+        }
+        tab[i] = a;
+    }
+    int rcv_a = -1, rcv_b = -1;
+    float y_a[YPL], y_b[YPL];
+    auto load_meta = [&](int t, int& rcv, float (&yv)[YPL]) {
+        if (t >= n_tiles) return;
+        const int64_t e0 = e_begin + (int64_t)t * T;
+        const int n_e = (int)min((int64_t)T, e_end - e0);
+        if (lane < n_e) rcv = p.identity ? (int)(e0 + lane) : p.receivers[e0 + lane];
+#pragma unroll
+        for (int i = 0; i < YPL; ++i) {
+            const int idx = i * 32 + lane;
+            if (idx < n_e * S::DSH) yv[i] = p.sh[e0 * S::DSH + idx];
+        }
+    };
+    load_meta(0, rcv_a, y_a);
+    load_meta(1, rcv_b, y_b);
+    int last_rcv = -1, stage = 0, phase = 0;
+#pragma unroll 1
+    for (int t = 0; t < n_tiles; ++t) {
+        if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
+        unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
+        const int64_t e0 = e_begin + (int64_t)t * T;
+        const int n_e = (int)min((int64_t)T, e_end - e0);
+        int* recv_t = reinterpret_cast<int*>(st + L::st_r);
+        float* y_t = reinterpret_cast<float*>(st + L::st_y);
         int before = __shfl_up_sync(0xffffffffu, rcv_a, 1);
         if (lane == 0) before = last_rcv;
         const unsigned mask = __ballot_sync(0xffffffffu, lane < n_e && rcv_a != before);
@@ -266,27 +287,44 @@ __device__ __forceinline__ void fwd_producer(const FwdParams& p, unsigned char* 
             if (idx < n_e * S::DSH) y_t[idx] = y_a[i];
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&full[stage]);  // the staged harmonics / receiver ids are in place
-        snd_a = snd_b; rcv_a = rcv_b;
+        // A[e][slot] = sum over the slot's records of c * y[e][i2]: contracted once per edge here, so that
+        // the consumers' per-channel loop never touches a coefficient.  All loads come before the first
+        // store, so that they are in flight together.
+        // (entries of edges beyond n_e are computed from stale data and never read)
+        float* A_t = reinterpret_cast<float*>(st + L::st_A);
+        float a_val[NA][T];
+#pragma unroll
+        for (int i = 0; i < NA; ++i)
+#pragma unroll
+            for (int e_i = 0; e_i < T; ++e_i) {
+                const float* ye = y_t + e_i * S::DSH;
+                a_val[i][e_i] = fmaf(tab[i].c1, ye[tab[i].i2_1], tab[i].c0 * ye[tab[i].i2_0]);
+            }
+#pragma unroll
+        for (int i = 0; i < NA; ++i) {
+            const int slot = lane + 32 * i;
+            if (slot < S::F_APAD) {
+#pragma unroll
+                for (int e_i = 0; e_i < T; ++e_i) A_t[e_i * S::F_APAD + slot] = a_val[i][e_i];
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[stage]);  // the staged A entries and receiver ids are in place
+        rcv_a = rcv_b;
 #pragma unroll
         for (int i = 0; i < YPL; ++i) y_a[i] = y_b[i];
-        load_meta(t + 2, snd_b, rcv_b, y_b);
+        load_meta(t + 2, rcv_b, y_b);
         if (++stage == NS) { stage = 0; phase ^= 1; }
-    }
-    if (*abort_flag) {
-        // let copies already in flight land before the CTA's shared memory is released
-        for (int t = max(0, armed - NS); t < armed; ++t)
-            for (uint32_t it = 0; it < kSpinLimit; ++it)
-                if (mbar_try_wait(&full[t % NS], (t / NS) & 1)) break;
     }
 }
 
 template <class S>
-__global__ void __launch_bounds__((S::FW * (S::NQ / (32 * S::V)) + 1) * 32, S::FC)
+__global__ void __launch_bounds__((S::FW * (S::NQ / (32 * S::V)) + 2) * 32, S::FC)
 fast_fwd_kernel(const FwdParams p) {
     using L = FwdSmem<S>;
     constexpr int T = L::T, NS = L::NS, NCONS = L::NCONS;
     static_assert(T <= 31, "the change mask is one 32-bit word");
+    static_assert((4 * L::X_EDGE) % (16 * 32) == 0, "a sender row is a whole number of 16-byte chunks per lane");
     static_assert(S::F_NREC <= 2, "an A slot holds at most two records");
 
     extern __shared__ __align__(128) unsigned char smem[];
@@ -300,13 +338,14 @@ fast_fwd_kernel(const FwdParams p) {
     const int n_tiles = (int)((e_end - e_begin + T - 1) / T);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NCONS); }
-        for (int g = 0; g < S::FW; ++g) mbar_init(reinterpret_cast<uint64_t*>(smem + L::off_pair) + g, L::CH);
+        // full: the table warp's arrival + one deferred arrival per lane of the copy warp (sender-row copies)
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1 + 32); mbar_init(&empty[s], NCONS); }
         *abort_flag = 0;
         mbar_fence_init();
     }
     __syncthreads();
-    if (warp == NCONS) fwd_producer<S>(p, smem, warp, lane, e_begin, e_end, n_tiles);
+    if (warp == NCONS) fwd_copy_producer<S>(p, smem, lane, e_begin, e_end, n_tiles);
+    else if (warp == NCONS + 1) fwd_table_producer<S>(p, smem, lane, e_begin, e_end, n_tiles);
     else FwdDispatch<S, 0>::run(warp % S::FW, p, smem, warp / S::FW, warp, lane, e_begin, e_end, n_tiles);
 }
 

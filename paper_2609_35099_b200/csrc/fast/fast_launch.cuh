@@ -58,7 +58,7 @@ int launch_fwd(const ConvArgs& a) {
     p.part_recv = reinterpret_cast<int32_t*>(a.workspace);
     p.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(a.workspace) + kPartRecvBytes);
     p.status = a.status;
-    constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 1) * 32;  // consumers + one producer warp
+    constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 2) * 32;  // consumers + two producer warps
     fast_fwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
     fwd_fixup_kernel<<<n_cta, 256, 0, a.stream>>>(n_cta, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),
@@ -83,7 +83,7 @@ int launch_tp_fwd(int64_t rows, const float* x1, const float* x2, const float* w
     p.x = x1; p.sh = x2; p.w = w; p.out = out; p.n_nodes = rows; p.n_edges = rows; p.identity = 1;
     const int64_t per = (rows + n_cta - 1) / n_cta;
     p.chunk = (per + 3) / 4 * 4;
-    constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 1) * 32;
+    constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 2) * 32;
     fast_fwd_kernel<S><<<n_cta, threads, L::total, st>>>(p);
     return after_launch();
 }
