@@ -97,7 +97,7 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
     using L = BwdSmem<S>;
     constexpr int T = L::T, NS = L::NS, NCONS = L::NCONS;
     constexpr int NQV = S::NQ / S::BV;
-    const int ROW0 = S::b_row0(G), NROW = S::b_row0(G + 1) - ROW0;
+    const int NROW = S::b_nrow(G);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
     uint64_t* empty = full + NS;
     uint64_t* xch = reinterpret_cast<uint64_t*>(smem + L::off_xch);
@@ -128,11 +128,10 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
 #pragma unroll 1
         for (int e_i = 0; alive && e_i < n_e; ++e_i, ++e) {
             if (mask & 1u) {
-                const Vec* g = reinterpret_cast<const Vec*>(p.grad_out + (size_t)recv_t[e_i] * row_elems) +
-                               (size_t)ROW0 * NQV + vlane;
+                const Vec* g = reinterpret_cast<const Vec*>(p.grad_out + (size_t)recv_t[e_i] * row_elems) + vlane;
 #pragma unroll
                 for (int r = 0; r < S::B_RMAX; ++r)
-                    if (r < NROW) dm[r] = g[(size_t)r * NQV];
+                    if (r < NROW) dm[r] = g[(size_t)S::b_row(G, r) * NQV];  // rows of this warp's path group
             }
             mask >>= 1;
             Vec dxp[S::DIN];

@@ -117,27 +117,73 @@ class Sig:
 
     # ---------------------------------------------------------------- backward
     def bwd_layout(self):
-        """Contiguous groups of whole paths, balanced by estimated instruction count."""
+        """Groups of whole paths (any subset, not only contiguous ones), balanced by estimated
+        instruction count: longest-processing-time assignment, paths inside a group in path order."""
         BW = self.cfg["BW"]
+        V = self.cfg.get("BV", self.V)
         costs = []
         for k, p in enumerate(self.paths):
             rows = range(p["out_off"], p["out_off"] + 2 * p["L"] + 1)
             npairs = sum(len(self.row_pairs[r]) for r in rows)
             nrec = sum(len(self.pairs[pi][3]) for r in rows for pi in self.row_pairs[r])
             combos = len({self.pairs[pi][1] for r in rows for pi in self.row_pairs[r]})
-            costs.append(4.0 * npairs + nrec + 6.0 * combos + 3.0)
-        pb = partition_rows(costs, BW)
-        while len(pb) < BW + 1:
-            pb.append(pb[-1])
-        row0 = [self.paths[pb[g]]["out_off"] if pb[g] < self.P else self.D for g in range(BW + 1)]
+            # per pair: u += A dm and the lane dot product; per record one scalar FMA; per (path, i1): s*x,
+            # the grad_w and grad_x FMAs; per path the weight load and the grad_w store
+            costs.append(2.0 * V * npairs + nrec + 3.0 * V * combos + npairs / 4.0 + 2.0)
+        nrows = [2 * p["L"] + 1 for p in self.paths]
+
+        def assign(cap, order):
+            bins = [[0.0, 0, []] for _ in range(BW)]
+            for k in order:
+                ok = [i for i in range(BW) if bins[i][1] + nrows[k] <= cap]
+                if not ok:
+                    return None
+                tgt = min(ok, key=lambda i: (bins[i][0], i))
+                bins[tgt][0] += costs[k]
+                bins[tgt][1] += nrows[k]
+                bins[tgt][2].append(k)
+            return bins
+
+        # The rows of a group live in registers, so the largest group's row count is capped: take the
+        # smallest cap whose best assignment found is within 3 % of the best over all caps.
+        import random
+        rng = random.Random(1234)
+        lpt = sorted(range(self.P), key=lambda k: (-costs[k], k))
+        found = {}
+        for cap in range(-(-self.D // BW), self.D + 1):
+            best = None
+            for trial in range(400):
+                order = list(lpt)
+                if trial:
+                    for _ in range(1 + trial % 4):  # a few swaps of neighbours in the LPT order
+                        i = rng.randrange(len(order) - 1)
+                        order[i], order[i + 1] = order[i + 1], order[i]
+                bins = assign(cap, order)
+                if bins is not None and (best is None or max(b[0] for b in bins) < max(b[0] for b in best)):
+                    best = bins
+            if best is not None:
+                found[cap] = best
+            if len(found) >= 6:
+                break
+        floor_cost = min(max(b[0] for b in bins) for bins in found.values())
+        cap = min(c for c, bins in found.items() if max(b[0] for b in bins) <= 1.03 * floor_cost)
+        bins = [[b[0], b[2]] for b in found[cap]]
+        groups = sorted((sorted(b[1]) for b in bins), key=lambda g: (g[0] if g else self.P))
+        rows_of = []
+        for g in groups:
+            rows = []
+            for k in g:
+                p = self.paths[k]
+                rows += list(range(p["out_off"], p["out_off"] + 2 * p["L"] + 1))
+            rows_of.append(rows)
         a0, slots = [0], []
-        for g in range(BW):
-            for row in range(row0[g], row0[g + 1]):
+        for rows in rows_of:
+            for row in rows:
                 slots += self.row_pairs[row]
             while len(slots) % 4:
                 slots.append(None)
             a0.append(len(slots))
-        return pb, row0, a0, slots
+        return groups, rows_of, a0, slots
 
     def emit_bwd(self):
         if "BW" not in self.cfg:
@@ -146,9 +192,9 @@ class Sig:
         assert NQ % (32 * V) == 0
         bvec = {2: "float2", 4: "float4"}[V]
         BW, BT, BS, BC = self.cfg["BW"], self.cfg["BT"], self.cfg["BS"], self.cfg["BC"]
-        pb, row0, a0, slots = self.bwd_layout()
+        groups, rows_of, a0, slots = self.bwd_layout()
         slot_of_pair = {pi: s for s, pi in enumerate(slots) if pi is not None}
-        rmax = max(row0[g + 1] - row0[g] for g in range(BW))
+        rmax = max(len(r) for r in rows_of)
         rec_val, rec_i2, pair_tab = [], [], []
         for pi in slots:
             if pi is None:
@@ -157,9 +203,10 @@ class Sig:
             pair_tab.append((len(rec_val), len(rl)))
             for i2, v in rl:
                 rec_val.append(v); rec_i2.append(i2)
-        self.bwd_tables = (pair_tab, rec_val, rec_i2)
+        row_tab = [rows + [rows[-1] if rows else 0] * (rmax - len(rows)) for rows in rows_of]
+        self.bwd_tables = (pair_tab, rec_val, rec_i2, row_tab)
         o = []
-        o.append(f"    // ---- backward: path groups {pb}")
+        o.append(f"    // ---- backward: path groups {groups}")
         o.append(f"    static constexpr int BV = {V};  // channels per lane in the backward")
         o.append(f"    using BVec = {bvec};")
         o.append(f"    static constexpr int BW = {BW}, BT = {BT}, BS = {BS}, BC = {BC}, B_RMAX = {rmax}, B_APAD = {len(slots)}, "
@@ -167,11 +214,13 @@ class Sig:
         o.append(f"    __device__ static __forceinline__ PairRec b_pair_rec(int i) {{ return kBPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float b_rec_val(int i) {{ return kBVal_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ unsigned char b_rec_i2(int i) {{ return kBI2_{self.name}[i]; }}")
-        o.append(f"    static constexpr int b_row0(int g) {{")
+        o.append(f"    // output rows of path group g: b_nrow(g) of them, the r-th is b_row(g, r)")
+        o.append(f"    __device__ static __forceinline__ int b_row(int g, int r) {{ return kBRow_{self.name}[g * B_RMAX + r]; }}")
+        o.append(f"    static constexpr int b_nrow(int g) {{")
         o.append("        switch (g) {")
-        for i, v in enumerate(row0):
-            o.append(f"            case {i}: return {v};")
-        o.append(f"            default: return {row0[-1]};")
+        for i, rows in enumerate(rows_of):
+            o.append(f"            case {i}: return {len(rows)};")
+        o.append(f"            default: return 0;")
         o.append("        }\n    }")
         o.append(f"    __device__ static __forceinline__ void bwd_edge(const int G, const BVec (&dm)[B_RMAX], const BVec* __restrict__ xs, "
                  f"const BVec* __restrict__ ss, const float* __restrict__ As, BVec (&dxp)[DIN], float (&dyl)[16], "
@@ -180,12 +229,13 @@ class Sig:
         o.append("        switch (G) {")
         for g in range(BW):
             o.append(f"        case {g}: {{")
-            rows = range(row0[g], row0[g + 1])
+            rows = rows_of[g]
+            local = {row: i for i, row in enumerate(rows)}
             need_x = sorted({self.pairs[pi][1] for row in rows for pi in self.row_pairs[row]})
             for i1 in need_x:
                 o.append(f"            const BVec x{i1} = xs[{i1} * NQV];")
             loaded_a = set()
-            for k in range(pb[g], pb[g + 1]):
+            for k in groups[g]:
                 p = self.paths[k]
                 prow = list(range(p["out_off"], p["out_off"] + 2 * p["L"] + 1))
                 used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.row_pairs[r2]})
@@ -205,7 +255,7 @@ class Sig:
                             loaded_a.add(q)
                             o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
                         i1 = self.pairs[pi][1]
-                        r = row - row0[g]
+                        r = local[row]
                         o.append(f"            vfma(u{k}_{i1}, a{q}.{lane}, dm[{r}]);")
                         o.append(f"            {{ const float t = vdot(sx{k}_{i1}, dm[{r}]);")
                         for i2, c in self.pairs[pi][3]:
@@ -261,13 +311,15 @@ class Sig:
         o.append("    " + ", ".join(str(i) for i in rec_i2) + "};")
         bwd_lines = self.emit_bwd()
         if bwd_lines:
-            bpair, bval, bi2 = self.bwd_tables
+            bpair, bval, bi2, brow = self.bwd_tables
             o.append(f"__device__ const PairRec kBPair_{self.name}[{len(bpair)}] = {{")
             o.append("    " + ", ".join(f"{{{s_},{c_}}}" for s_, c_ in bpair) + "};")
             o.append(f"__device__ const float kBVal_{self.name}[{len(bval)}] = {{")
             o.append("    " + ", ".join(fmt_float(v) for v in bval) + "};")
             o.append(f"__device__ const unsigned char kBI2_{self.name}[{len(bi2)}] = {{")
             o.append("    " + ", ".join(str(i) for i in bi2) + "};")
+            o.append(f"__device__ const unsigned char kBRow_{self.name}[{len(brow) * len(brow[0])}] = {{")
+            o.append("    " + ", ".join(str(i) for rows in brow for i in rows) + "};")
         o.append("")
         o.append(f"struct {S} {{")
         o.append(f"    static constexpr int NQ = {NQ}, DIN = {self.DIN}, DSH = {self.DSH}, P = {self.P}, D = {self.D};")
