@@ -15,11 +15,11 @@
 // group g (whole paths, so grad_w[e,k] is complete inside one warp) and channels
 // [ch*32*V, (ch+1)*32*V).  The rows of dm that a warp needs stay in registers while the receiver
 // does not change.  Per edge the warps exchange their dx_e and grad_sh partial sums through
-// shared memory and add them in a fixed order.  The last warp is the producer: bulk copies of
-// the edge-local operands and the sender rows, staging of harmonics / ids, and the A entries.
+// shared memory and add them in a fixed order.  The last warp is the producer (the code shared with the
+// forward kernel, run by one warp here): a tile's copies, then its receiver ids and A entries.
 #pragma once
 #include "fast_common.cuh"
-#include "fast_fwd.cuh"  // ASlot
+#include "fast_producer.cuh"
 
 namespace e3j {
 namespace fast {
@@ -182,103 +182,12 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
 }
 
 template <class S>
-__device__ __forceinline__ void bwd_producer(const BwdParams& p, unsigned char* smem, const int lane,
-                                             const int64_t e_begin, const int64_t e_end, const int n_tiles) {
-    using L = BwdSmem<S>;
-    constexpr int T = L::T, NS = L::NS;
-    constexpr int YPL = (T * S::DSH + 31) / 32;
-    constexpr int NA = (S::B_APAD + 31) / 32;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
-    uint64_t* empty = full + NS;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
-
-    ASlot tab[NA];  // this lane's A slots (lane, lane + 32, ...)
-#pragma unroll
-    for (int i = 0; i < NA; ++i) {
-        const int slot = lane + 32 * i;
-        ASlot a{0.f, 0.f, 0, 0};
-        if (slot < S::B_APAD) {
-            const PairRec pr = S::b_pair_rec(slot);
-            if (pr.count > 0) { a.c0 = S::b_rec_val(pr.start); a.i2_0 = S::b_rec_i2(pr.start); }
-            if (pr.count > 1) { a.c1 = S::b_rec_val(pr.start + 1); a.i2_1 = S::b_rec_i2(pr.start + 1); }
-        }
-        tab[i] = a;
-    }
-    int snd_a = 0, rcv_a = -1, snd_b = 0, rcv_b = -1;
-    float y_a[YPL], y_b[YPL];
-    auto load_meta = [&](int t, int& snd, int& rcv, float (&yv)[YPL]) {
-        if (t >= n_tiles) return;
-        const int64_t e0 = e_begin + (int64_t)t * T;
-        const int n_e = (int)min((int64_t)T, e_end - e0);
-        if (lane < n_e) {
-            if (p.identity) { snd = rcv = (int)(e0 + lane); }
-            else { snd = p.senders[e0 + lane]; rcv = p.receivers[e0 + lane]; }
-        }
-#pragma unroll
-        for (int i = 0; i < YPL; ++i) {
-            const int idx = i * 32 + lane;
-            if (idx < n_e * S::DSH) yv[i] = p.sh[e0 * S::DSH + idx];
-        }
-    };
-    load_meta(0, snd_a, rcv_a, y_a);
-    load_meta(1, snd_b, rcv_b, y_b);
-    int armed = 0, last_rcv = -1, stage = 0, phase = 0;
-    for (int t = 0; t < n_tiles; ++t) {
-        if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
-        unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
-        const int64_t e0 = e_begin + (int64_t)t * T;
-        const int n_e = (int)min((int64_t)T, e_end - e0);
-        int* recv_t = reinterpret_cast<int*>(st + L::st_r);
-        float* y_t = reinterpret_cast<float*>(st + L::st_y);
-        float* A_t = reinterpret_cast<float*>(st + L::st_A);
-        if (lane == 0) {
-            mbar_expect_tx(&full[stage], (uint32_t)n_e * (uint32_t)(4 * (L::S_EDGE + L::X_EDGE)));
-            bulk_g2s(st + L::st_s, p.w + (size_t)e0 * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE, &full[stage]);
-        }
-        if (lane < n_e)
-            bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE, p.x + (size_t)snd_a * L::X_EDGE, 4u * L::X_EDGE,
-                     &full[stage]);
-        armed = t + 1;
-        int before = __shfl_up_sync(0xffffffffu, rcv_a, 1);
-        if (lane == 0) before = last_rcv;
-        const unsigned mask = __ballot_sync(0xffffffffu, lane < n_e && rcv_a != before);
-        last_rcv = __shfl_sync(0xffffffffu, rcv_a, n_e - 1);
-        if (lane < n_e) recv_t[lane] = rcv_a;
-        if (lane == 0) recv_t[T] = (int)mask;
-#pragma unroll
-        for (int i = 0; i < YPL; ++i) {
-            const int idx = i * 32 + lane;
-            if (idx < n_e * S::DSH) y_t[idx] = y_a[i];
-        }
-        __syncwarp();
-        // A[e][slot] = sum over the slot's records of c * y[e][i2]
-        // (entries of edges beyond n_e are computed from stale data and never read)
-#pragma unroll
-        for (int i = 0; i < NA; ++i) {
-            const int slot = lane + 32 * i;
-            if (slot < S::B_APAD) {
-#pragma unroll
-                for (int e_i = 0; e_i < T; ++e_i) {
-                    const float* ye = y_t + e_i * S::DSH;
-                    A_t[e_i * S::B_APAD + slot] = fmaf(tab[i].c1, ye[tab[i].i2_1], tab[i].c0 * ye[tab[i].i2_0]);
-                }
-            }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&full[stage]);
-        snd_a = snd_b; rcv_a = rcv_b;
-#pragma unroll
-        for (int i = 0; i < YPL; ++i) y_a[i] = y_b[i];
-        load_meta(t + 2, snd_b, rcv_b, y_b);
-        if (++stage == NS) { stage = 0; phase ^= 1; }
-    }
-    if (*abort_flag) {
-        for (int t = max(0, armed - NS); t < armed; ++t)
-#pragma unroll 1
-            for (uint32_t it = 0; it < kSpinLimit; ++it)
-                if (mbar_try_wait(&full[t % NS], (t / NS) & 1)) break;
-    }
-}
+struct BwdTab {
+    static constexpr int APAD = S::B_APAD, DSH = S::DSH;
+    __device__ static __forceinline__ PairRec pair_rec(int i) { return S::b_pair_rec(i); }
+    __device__ static __forceinline__ float rec_val(int i) { return S::b_rec_val(i); }
+    __device__ static __forceinline__ unsigned char rec_i2(int i) { return S::b_rec_i2(i); }
+};
 
 template <class S>
 __global__ void __launch_bounds__((S::BW * (S::NQ / (32 * S::BV)) + 1) * 32, S::BC)
@@ -299,13 +208,14 @@ fast_bwd_kernel(const BwdParams p) {
     const int n_tiles = (int)((e_end - e_begin + T - 1) / T);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NCONS); }
+        // full: the producer's arrival with the copies' byte count and its arrival after the tables
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], NCONS); }
         mbar_init(reinterpret_cast<uint64_t*>(smem + L::off_xch), NCONS);
         *abort_flag = 0;
         mbar_fence_init();
     }
     __syncthreads();
-    if (warp == NCONS) bwd_producer<S>(p, smem, lane, e_begin, e_end, n_tiles);
+    if (warp == NCONS) producer_loop<L, BwdTab<S>, 2>(p, smem, lane, e_begin, e_end, n_tiles);
     else bwd_consumer<S>(p, smem, warp % S::BW, warp / S::BW, warp, lane, e_begin, e_end, n_tiles);
 }
 

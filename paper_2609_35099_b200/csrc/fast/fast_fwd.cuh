@@ -21,16 +21,11 @@
 // is the per-edge body and nothing else.
 #pragma once
 #include "fast_common.cuh"
+#include "fast_producer.cuh"
 
 namespace e3j {
 namespace fast {
 
-
-// Per A slot: up to two records, A = c0 * y[i2_0] + c1 * y[i2_1].
-struct ASlot {
-    float c0, c1;
-    int i2_0, i2_1;
-};
 
 template <class S>
 struct FwdSmem {
@@ -167,156 +162,13 @@ struct FwdDispatch<S, S::FW> {
     __device__ static __forceinline__ void run(const int, Args&&...) {}
 };
 
-// ------------------------------------------------------------------------ producers
-// Two warps feed the ring.  The copy warp waits for a free slot and issues the tile's copies at once;
-// the table warp stages the tile's receiver ids and computes its A entries.  A tile is "full" when the
-// bulk copy's bytes, the 32 deferred arrivals of the sender-row copies and the table warp's arrival are in.
 template <class S>
-__device__ __forceinline__ void fwd_copy_producer(const FwdParams& p, unsigned char* smem, const int lane,
-                                                  const int64_t e_begin, const int64_t e_end, const int n_tiles) {
-    using L = FwdSmem<S>;
-    constexpr int T = L::T, NS = L::NS;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
-    uint64_t* empty = full + NS;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
-    int snd_a = 0, snd_b = 0;
-    auto load_snd = [&](int t, int& snd) {  // sender ids two tiles ahead of their use
-        if (t >= n_tiles) return;
-        const int64_t e0 = e_begin + (int64_t)t * T;
-        const int n_e = (int)min((int64_t)T, e_end - e0);
-        if (lane < n_e) snd = p.identity ? (int)(e0 + lane) : p.senders[e0 + lane];
-    };
-    load_snd(0, snd_a);
-    load_snd(1, snd_b);
-    int armed = 0, stage = 0, phase = 0;
-#pragma unroll 1
-    for (int t = 0; t < n_tiles; ++t) {
-        // phase of `empty` that ends the previous use of this ring slot
-        if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
-        unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
-        const int64_t e0 = e_begin + (int64_t)t * T;
-        const int n_e = (int)min((int64_t)T, e_end - e0);
-        // The tile's weights are one bulk copy; the gathered sender rows go as 16-byte asynchronous copies
-        // from all lanes (a bulk copy per row holds the issuing lane for ~150 cycles each), counted on the
-        // same barrier by one deferred arrival per lane.
-        if (lane == 0) {
-            mbar_expect_tx(&full[stage], (uint32_t)n_e * 4u * L::S_EDGE);
-            bulk_g2s(st + L::st_s, p.w + (size_t)e0 * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE, &full[stage]);
-        }
-#pragma unroll
-        for (int e_i = 0; e_i < T; ++e_i) {
-            const int snd = __shfl_sync(0xffffffffu, snd_a, e_i);
-            if (e_i < n_e) {
-                const char* src = reinterpret_cast<const char*>(p.x + (size_t)snd * L::X_EDGE);
-                unsigned char* dst = st + L::st_x + (size_t)e_i * 4 * L::X_EDGE;
-#pragma unroll
-                for (int c = 0; c < (4 * L::X_EDGE) / (16 * 32); ++c)
-                    cp_async16(dst + 16 * (c * 32 + lane), src + 16 * (c * 32 + lane));
-            }
-        }
-        cp_async_arrive_noinc(&full[stage]);
-        armed = t + 1;
-        snd_a = snd_b;
-        load_snd(t + 2, snd_b);
-        if (++stage == NS) { stage = 0; phase ^= 1; }
-    }
-    if (*abort_flag) {
-        // let copies already in flight land before the CTA's shared memory is released
-        for (int t = max(0, armed - NS); t < armed; ++t)
-#pragma unroll 1
-            for (uint32_t it = 0; it < kSpinLimit; ++it)
-                if (mbar_try_wait(&full[t % NS], (t / NS) & 1)) break;
-    }
-}
-
-template <class S>
-__device__ __forceinline__ void fwd_table_producer(const FwdParams& p, unsigned char* smem, const int lane,
-                                                   const int64_t e_begin, const int64_t e_end, const int n_tiles) {
-    using L = FwdSmem<S>;
-    constexpr int T = L::T, NS = L::NS;
-    constexpr int YPL = (T * S::DSH + 31) / 32;
-    constexpr int NA = (S::F_APAD + 31) / 32;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
-    uint64_t* empty = full + NS;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
-    ASlot tab[NA];  // this lane's A slots (lane, lane + 32, ...)
-#pragma unroll
-    for (int i = 0; i < NA; ++i) {
-        const int slot = lane + 32 * i;
-        ASlot a{0.f, 0.f, 0, 0};
-        if (slot < S::F_APAD) {
-            const PairRec pr = S::pair_rec(slot);
-            if (pr.count > 0) { a.c0 = S::rec_val(pr.start); a.i2_0 = S::rec_i2(pr.start); }
-            if (pr.count > 1) { a.c1 = S::rec_val(pr.start + 1); a.i2_1 = S::rec_i2(pr.start + 1); }
-        }
-        tab[i] = a;
-    }
-    int rcv_a = -1, rcv_b = -1;
-    float y_a[YPL], y_b[YPL];
-    auto load_meta = [&](int t, int& rcv, float (&yv)[YPL]) {
-        if (t >= n_tiles) return;
-        const int64_t e0 = e_begin + (int64_t)t * T;
-        const int n_e = (int)min((int64_t)T, e_end - e0);
-        if (lane < n_e) rcv = p.identity ? (int)(e0 + lane) : p.receivers[e0 + lane];
-#pragma unroll
-        for (int i = 0; i < YPL; ++i) {
-            const int idx = i * 32 + lane;
-            if (idx < n_e * S::DSH) yv[i] = p.sh[e0 * S::DSH + idx];
-        }
-    };
-    load_meta(0, rcv_a, y_a);
-    load_meta(1, rcv_b, y_b);
-    int last_rcv = -1, stage = 0, phase = 0;
-#pragma unroll 1
-    for (int t = 0; t < n_tiles; ++t) {
-        if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
-        unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
-        const int64_t e0 = e_begin + (int64_t)t * T;
-        const int n_e = (int)min((int64_t)T, e_end - e0);
-        int* recv_t = reinterpret_cast<int*>(st + L::st_r);
-        float* y_t = reinterpret_cast<float*>(st + L::st_y);
-        int before = __shfl_up_sync(0xffffffffu, rcv_a, 1);
-        if (lane == 0) before = last_rcv;
-        const unsigned mask = __ballot_sync(0xffffffffu, lane < n_e && rcv_a != before);
-        last_rcv = __shfl_sync(0xffffffffu, rcv_a, n_e - 1);
-        if (lane < n_e) recv_t[lane] = rcv_a;
-        if (lane == 0) recv_t[T] = (int)mask;
-#pragma unroll
-        for (int i = 0; i < YPL; ++i) {
-            const int idx = i * 32 + lane;
-            if (idx < n_e * S::DSH) y_t[idx] = y_a[i];
-        }
-        __syncwarp();
-        // A[e][slot] = sum over the slot's records of c * y[e][i2]: contracted once per edge here, so that
-        // the consumers' per-channel loop never touches a coefficient.  All loads come before the first
-        // store, so that they are in flight together.
-        // (entries of edges beyond n_e are computed from stale data and never read)
-        float* A_t = reinterpret_cast<float*>(st + L::st_A);
-        float a_val[NA][T];
-#pragma unroll
-        for (int i = 0; i < NA; ++i)
-#pragma unroll
-            for (int e_i = 0; e_i < T; ++e_i) {
-                const float* ye = y_t + e_i * S::DSH;
-                a_val[i][e_i] = fmaf(tab[i].c1, ye[tab[i].i2_1], tab[i].c0 * ye[tab[i].i2_0]);
-            }
-#pragma unroll
-        for (int i = 0; i < NA; ++i) {
-            const int slot = lane + 32 * i;
-            if (slot < S::F_APAD) {
-#pragma unroll
-                for (int e_i = 0; e_i < T; ++e_i) A_t[e_i * S::F_APAD + slot] = a_val[i][e_i];
-            }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&full[stage]);  // the staged A entries and receiver ids are in place
-        rcv_a = rcv_b;
-#pragma unroll
-        for (int i = 0; i < YPL; ++i) y_a[i] = y_b[i];
-        load_meta(t + 2, rcv_b, y_b);
-        if (++stage == NS) { stage = 0; phase ^= 1; }
-    }
-}
+struct FwdTab {
+    static constexpr int APAD = S::F_APAD, DSH = S::DSH;
+    __device__ static __forceinline__ PairRec pair_rec(int i) { return S::pair_rec(i); }
+    __device__ static __forceinline__ float rec_val(int i) { return S::rec_val(i); }
+    __device__ static __forceinline__ unsigned char rec_i2(int i) { return S::rec_i2(i); }
+};
 
 template <class S>
 __global__ void __launch_bounds__((S::FW * (S::NQ / (32 * S::V)) + 2) * 32, S::FC)
@@ -324,7 +176,6 @@ fast_fwd_kernel(const FwdParams p) {
     using L = FwdSmem<S>;
     constexpr int T = L::T, NS = L::NS, NCONS = L::NCONS;
     static_assert(T <= 31, "the change mask is one 32-bit word");
-    static_assert((4 * L::X_EDGE) % (16 * 32) == 0, "a sender row is a whole number of 16-byte chunks per lane");
     static_assert(S::F_NREC <= 2, "an A slot holds at most two records");
 
     extern __shared__ __align__(128) unsigned char smem[];
@@ -338,14 +189,14 @@ fast_fwd_kernel(const FwdParams p) {
     const int n_tiles = (int)((e_end - e_begin + T - 1) / T);
 
     if (threadIdx.x == 0) {
-        // full: the table warp's arrival + one deferred arrival per lane of the copy warp (sender-row copies)
-        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1 + 32); mbar_init(&empty[s], NCONS); }
+        // full: the copy warp's arrival (with the byte count) and the table warp's arrival
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], NCONS); }
         *abort_flag = 0;
         mbar_fence_init();
     }
     __syncthreads();
-    if (warp == NCONS) fwd_copy_producer<S>(p, smem, lane, e_begin, e_end, n_tiles);
-    else if (warp == NCONS + 1) fwd_table_producer<S>(p, smem, lane, e_begin, e_end, n_tiles);
+    if (warp == NCONS) producer_loop<L, FwdTab<S>, 0>(p, smem, lane, e_begin, e_end, n_tiles);
+    else if (warp == NCONS + 1) producer_loop<L, FwdTab<S>, 1>(p, smem, lane, e_begin, e_end, n_tiles);
     else FwdDispatch<S, 0>::run(warp % S::FW, p, smem, warp / S::FW, warp, lane, e_begin, e_end, n_tiles);
 }
 

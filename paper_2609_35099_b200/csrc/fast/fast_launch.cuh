@@ -106,7 +106,7 @@ int launch_tp_bwd(int64_t rows, const float* x1, const float* x2, const float* w
     p.dx_edge = gx1;  // each row is its own sender: the per-edge share is the gradient
     p.n_nodes = rows; p.n_edges = rows; p.identity = 1;
     p.chunk = (rows + n_cta - 1) / n_cta;
-    constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;
+    constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;  // consumers + one producer warp
     fast_bwd_kernel<S><<<n_cta, threads, L::total, st>>>(p);
     return after_launch();
 }
@@ -137,7 +137,7 @@ int launch_bwd(const ConvArgs& a) {
     p.n_nodes = a.n_nodes; p.n_edges = a.n_edges;
     p.chunk = (a.n_edges + n_cta - 1) / n_cta;
     p.status = a.status;
-    constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;
+    constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;  // consumers + one producer warp
     fast_bwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
     const int64_t blocks = std::min<int64_t>(a.n_nodes, 148 * 16);
