@@ -134,12 +134,8 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
                     if (r < NROW) dm[r] = g[(size_t)S::b_row(G, r) * NQV];  // rows of this warp's path group
             }
             mask >>= 1;
-            Vec dxp[S::DIN];
+            Vec dxp[S::DIN];   // both are assigned (not accumulated into) by bwd_edge
             float dyl[16];
-#pragma unroll
-            for (int i = 0; i < S::DIN; ++i) vzero(dxp[i]);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) dyl[i] = 0.f;
             Vec* gw = reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + vlane;
             S::bwd_edge(G, dm, xs, ss, As, dxp, dyl, gw);
             xs += L::X_EDGE / S::BV; ss += L::S_EDGE / S::BV; As += S::B_APAD;

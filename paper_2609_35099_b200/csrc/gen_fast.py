@@ -235,6 +235,7 @@ class Sig:
             for i1 in need_x:
                 o.append(f"            const BVec x{i1} = xs[{i1} * NQV];")
             loaded_a = set()
+            dx_touched, dy_touched = set(), set()   # first contribution assigns, later ones accumulate
             for k in groups[g]:
                 p = self.paths[k]
                 prow = list(range(p["out_off"], p["out_off"] + 2 * p["L"] + 1))
@@ -259,7 +260,11 @@ class Sig:
                         o.append(f"            vfma(u{k}_{i1}, a{q}.{lane}, dm[{r}]);")
                         o.append(f"            {{ const float t = vdot(sx{k}_{i1}, dm[{r}]);")
                         for i2, c in self.pairs[pi][3]:
-                            o.append(f"              dyl[{i2}] = fmaf({fmt_float(c)}, t, dyl[{i2}]);")
+                            if i2 in dy_touched:
+                                o.append(f"              dyl[{i2}] = fmaf({fmt_float(c)}, t, dyl[{i2}]);")
+                            else:
+                                dy_touched.add(i2)
+                                o.append(f"              dyl[{i2}] = {fmt_float(c)} * t;")
                         o.append("            }")
                 first = used[0]
                 o.append(f"            BVec ds{k} = vmul(x{first}, u{k}_{first});")
@@ -267,9 +272,25 @@ class Sig:
                     o.append(f"            vfma(ds{k}, x{i1}, u{k}_{i1});")
                 o.append(f"            gw[{k} * NQV] = ds{k};")
                 for i1 in used:
-                    o.append(f"            vfma(dxp[{i1}], s{k}, u{k}_{i1});")
+                    if i1 in dx_touched:
+                        o.append(f"            vfma(dxp[{i1}], s{k}, u{k}_{i1});")
+                    else:
+                        dx_touched.add(i1)
+                        o.append(f"            dxp[{i1}] = vmul(s{k}, u{k}_{i1});")
+            # entries this group never touches
+            for i1 in range(self.DIN):
+                if i1 not in dx_touched:
+                    o.append(f"            vzero(dxp[{i1}]);")
+            for i2 in range(16):
+                if i2 not in dy_touched:
+                    o.append(f"            dyl[{i2}] = 0.f;")
             o.append("        } break;")
-        o.append("        default: break;")
+        o.append("        default: {")
+        o.append("#pragma unroll")
+        o.append("            for (int i = 0; i < DIN; ++i) vzero(dxp[i]);")
+        o.append("#pragma unroll")
+        o.append("            for (int i = 0; i < 16; ++i) dyl[i] = 0.f;")
+        o.append("        } break;")
         o.append("        }")
         o.append("    }")
         return o
