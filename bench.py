@@ -49,8 +49,8 @@ def measured_peak():
 # profiles/fast_fwd_kernel_water3000.txt, profiles/fast_bwd_kernel_water3000.txt and the launch-list run
 # (specialised kernels, workload water3000).  Other workloads / the generic kernels report null.
 NCU_TRAFFIC = {
-    ("water3000", "fwd"): 1.110601e9 + 0.086230e9 + 0.016343e9,          # fast_fwd_kernel + fwd_fixup_kernel
-    ("water3000", "bwd"): 1.260743e9 + 1.361455e9 + 0.330491e9 + 0.0018e9,  # fast_bwd_kernel + bwd_dx_reduce_kernel
+    ("water3000", "fwd"): 1.109178e9 + 0.082058e9 + 0.016342e9,          # fast_fwd_kernel + fwd_fixup_kernel
+    ("water3000", "bwd"): 1.259555e9 + 1.361636e9 + 0.330508e9 + 0.0017e9,  # fast_bwd_kernel + bwd_dx_reduce_kernel
 }
 
 
@@ -379,9 +379,9 @@ def main():
                     "algorithmic_bytes_per_launch": nbytes, "avg_ms": ms, "traffic": traffic}
 
         spec = bool(plan.specialised)
-        roofs = {"fwd": roof(fb, f_ms, "e3j_conv_fwd call: fast_fwd_kernel (96 %) + fwd_fixup_kernel" if spec
+        roofs = {"fwd": roof(fb, f_ms, "e3j_conv_fwd call: fast_fwd_kernel (97 %) + fwd_fixup_kernel" if spec
                              else "e3j_conv_fwd call: generic conv_fwd_kernel", "fwd"),
-                 "bwd": roof(bb, b_ms, "e3j_conv_bwd call: fast_bwd_kernel (91 %) + bwd_dx_reduce_kernel" if spec
+                 "bwd": roof(bb, b_ms, "e3j_conv_bwd call: fast_bwd_kernel (90 %) + bwd_dx_reduce_kernel" if spec
                              else "e3j_conv_bwd call: generic edge + node kernels", "bwd")}
         dominant = roofs["bwd"] if b_ms >= f_ms else roofs["fwd"]
         line = {
