@@ -29,16 +29,13 @@ __global__ void bwd_dx_reduce_kernel(int64_t n_nodes, int row_f4, const float4* 
         for (int i = threadIdx.x; i < row_f4; i += blockDim.x) {
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             int j = j0;
-            // four independent loads in flight; the additions stay in edge order
-            for (; j + 4 <= j1; j += 4) {
-                const float4 v0 = dx_edge[(size_t)sender_perm[j] * row_f4 + i];
-                const float4 v1 = dx_edge[(size_t)sender_perm[j + 1] * row_f4 + i];
-                const float4 v2 = dx_edge[(size_t)sender_perm[j + 2] * row_f4 + i];
-                const float4 v3 = dx_edge[(size_t)sender_perm[j + 3] * row_f4 + i];
-                acc.x += v0.x; acc.y += v0.y; acc.z += v0.z; acc.w += v0.w;
-                acc.x += v1.x; acc.y += v1.y; acc.z += v1.z; acc.w += v1.w;
-                acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w;
-                acc.x += v3.x; acc.y += v3.y; acc.z += v3.z; acc.w += v3.w;
+            // eight independent loads in flight; the additions stay in edge order
+            for (; j + 8 <= j1; j += 8) {
+                float4 v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = dx_edge[(size_t)sender_perm[j + u] * row_f4 + i];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
             }
             for (; j < j1; ++j) {
                 const float4 v = dx_edge[(size_t)sender_perm[j] * row_f4 + i];

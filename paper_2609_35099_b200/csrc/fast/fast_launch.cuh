@@ -140,7 +140,8 @@ int launch_bwd(const ConvArgs& a) {
     constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;  // consumers + one producer warp
     fast_bwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
-    const int64_t blocks = std::min<int64_t>(a.n_nodes, 148 * 16);
+    // one CTA per sender: the hardware hands them out as CTAs finish, so uneven degrees do not leave a tail
+    const int64_t blocks = std::min<int64_t>(a.n_nodes, (int64_t)1 << 30);
     bwd_dx_reduce_kernel<<<(int)blocks, S::DIN * S::NQ / 4, 0, a.stream>>>(a.n_nodes, S::DIN * S::NQ / 4,
         reinterpret_cast<const float4*>(p.dx_edge), a.sender_perm, a.colptr, reinterpret_cast<float4*>(a.grad_x));
     return after_launch();
