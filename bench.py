@@ -105,6 +105,13 @@ class ClockSampler:
                 "power_w_max": max(power), "samples": len(sm)}
 
 
+def call_stats(ms):
+    srt = sorted(ms)
+    k = max(1, len(srt) // 5)
+    return {"median": statistics.median(srt), "mean_fastest_20pct": statistics.mean(srt[:k]), "min": srt[0],
+            "max": srt[-1], "mean": statistics.mean(srt)}
+
+
 def oracle_sample(wl, cp, x, y, w, g, n_rows):
     """Sub-problem made of the first n_rows receivers (their edges are a prefix of the edge list)."""
     n_rows = min(n_rows, wl.n_nodes)
@@ -395,6 +402,9 @@ def main():
                        "parallelism": "independent systems per rank, no collective"},
             "fwd_edges_per_s": e * world / (f_ms * 1e-3), "fwd_ms": f_ms, "bwd_ms": b_ms,
             "fwd_plus_bwd_frac_of_nominal_8TBs": (fb + bb) / ((f_ms + b_ms) * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+            # per-call statistics over the timed steps: median, the paper's statistic (mean of the fastest
+            # 20 % of the runs, as in its efficiency-comparison section), minimum and maximum
+            "call_stats_ms": {"fwd": call_stats(fwd_ms), "bwd": call_stats(bwd_ms)},
             "roofline": dominant, "roofline_fwd": roofs["fwd"], "roofline_bwd": roofs["bwd"],
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         }
