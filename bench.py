@@ -254,6 +254,8 @@ def main():
                     help="2 = headline workload; 3 / 5 = other convolution workloads; 4 = standalone tensor product rows")
     ap.add_argument("--rows", type=int, default=1 << 20, help="rows of the tensor-product workload (--config 4)")
     ap.add_argument("--generic", action="store_true", help="force the table-driven generic kernels")
+    ap.add_argument("--pad", type=float, default=0.0,
+                    help="append this fraction of padding edges and call the padded entry points (rates count real edges)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -294,23 +296,35 @@ def main():
                                e3j.E3J_PLAN_GENERIC_ONLY if args.generic else 0)
     n, e = wl.n_nodes, wl.n_edges
     x, y, w, g = workloads.make_features(wl, plan.n_paths, plan.d_out)
-    host = dict(x=x, y=y, w=w, g=g, snd=wl.senders, rcv=wl.receivers)
+    snd_h, rcv_h = wl.senders, wl.receivers
+    n_pad = int(round(args.pad * e))
+    if n_pad:
+        # padding entries: receiver id = n_nodes (the padding mark), the rest arbitrary
+        y = np.concatenate([y, np.zeros((n_pad, y.shape[1]), np.float32)])
+        w = np.concatenate([w, np.zeros((n_pad,) + w.shape[1:], np.float32)])
+        snd_h = np.concatenate([snd_h, np.zeros(n_pad, np.int32)])
+        rcv_h = np.concatenate([rcv_h, np.full(n_pad, n, np.int32)])
+    e_buf = e + n_pad
+    host = dict(x=x, y=y, w=w, g=g, snd=snd_h, rcv=rcv_h)
     pinned = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in host.items()}
     d = {k: v.to(dev) for k, v in pinned.items()}
     stream = torch.cuda.current_stream()
-    rowptr, perm, colptr = e3j.e3j_graph_prepare(n, d["snd"], d["rcv"])
+    prepare = e3j.e3j_graph_prepare_padded if n_pad else e3j.e3j_graph_prepare
+    conv_fwd = e3j.e3j_conv_fwd_padded if n_pad else e3j.e3j_conv_fwd
+    conv_bwd = e3j.e3j_conv_bwd_padded if n_pad else e3j.e3j_conv_bwd
+    rowptr, perm, colptr = prepare(n, d["snd"], d["rcv"])
     out = torch.empty((n, plan.d_out, plan.n_channels), device=dev)
     gx = torch.empty((n, plan.d_in, plan.n_channels), device=dev)
-    gy = torch.empty((e, plan.d_sh), device=dev)
-    gw = torch.empty((e, plan.n_paths, plan.n_channels), device=dev)
-    ws_f = torch.empty(max(e3j.e3j_conv_fwd_workspace_bytes(plan, n, e), 256), dtype=torch.uint8, device=dev)
-    ws_b = torch.empty(max(e3j.e3j_conv_bwd_workspace_bytes(plan, n, e), 256), dtype=torch.uint8, device=dev)
+    gy = torch.empty((e_buf, plan.d_sh), device=dev)
+    gw = torch.empty((e_buf, plan.n_paths, plan.n_channels), device=dev)
+    ws_f = torch.empty(max(e3j.e3j_conv_fwd_workspace_bytes(plan, n, e_buf), 256), dtype=torch.uint8, device=dev)
+    ws_b = torch.empty(max(e3j.e3j_conv_bwd_workspace_bytes(plan, n, e_buf), 256), dtype=torch.uint8, device=dev)
 
     def fwd(t):
-        e3j.e3j_conv_fwd(plan, t["x"], t["y"], t["w"], t["snd"], t["rcv"], rowptr, out=out, workspace=ws_f)
+        conv_fwd(plan, t["x"], t["y"], t["w"], t["snd"], t["rcv"], rowptr, out=out, workspace=ws_f)
 
     def bwd(t):
-        e3j.e3j_conv_bwd(plan, t["x"], t["y"], t["w"], t["snd"], t["rcv"], t["g"], rowptr, perm, colptr,
+        conv_bwd(plan, t["x"], t["y"], t["w"], t["snd"], t["rcv"], t["g"], rowptr, perm, colptr,
                          grad_x=gx, grad_sh=gy, grad_w=gw, workspace=ws_b)
 
     for _ in range(args.warmup):
@@ -395,7 +409,7 @@ def main():
             "metric": "conv_fwd_bwd_edges_per_s", "value": e * world / (ms_per_step * 1e-3), "unit": "edges/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "n_nodes": n, "n_edges": e, "irreps_in": c["irreps_in"],
+            "config": {"workload": wl.name, "n_nodes": n, "n_edges": e, "padding_edges": n_pad, "irreps_in": c["irreps_in"],
                        "sh_lmax": c["sh_lmax"], "n_paths": plan.n_paths, "d_out": plan.d_out,
                        "channels": plan.n_channels, "specialised_kernels": bool(plan.specialised),
                        "l2": "inputs (>1 GB per step) exceed the 126 MB L2; no explicit flush",

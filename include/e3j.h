@@ -185,6 +185,35 @@ int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
                  const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
                  float* grad_w, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Padded edge lists (paper: the neighbour list of the molecular-dynamics runs is kept
+ * at a fixed padded size and padding edges are flagged; the paper does not give the
+ * mechanism, the convention here is): an edge whose receiver id is >= n_nodes is
+ * padding.  With receivers non-decreasing the padding edges are the last ones, and the
+ * number of real edges is rowptr[n_nodes], which the kernels read on the device - the
+ * host never needs it, so a buffer of n_edges_padded entries can be reused while the
+ * real count changes.  Nothing of a padding edge is read (its sender, harmonics and
+ * weights may hold anything); out and grad_x are those of the real edges; the grad_sh
+ * and grad_w rows of padding edges are set to zero.
+ * e3j_graph_prepare_padded: as e3j_graph_prepare; sender_perm receives rowptr[n_nodes]
+ * entries (the rest is not written), colptr[n_nodes] equals that count.
+ * e3j_conv_fwd_padded / e3j_conv_bwd_padded: as e3j_conv_fwd / e3j_conv_bwd with
+ * n_edges_padded the length of the edge arrays; rowptr is required (E3J_ERR_INVALID_ARG
+ * if NULL) and must come from e3j_graph_prepare_padded (or hold the same values);
+ * sender_perm / colptr as produced by it, or NULL (derived into the workspace).
+ * Workspace sizes: the e3j_conv_*_workspace_bytes functions with n_edges_padded. */
+int e3j_graph_prepare_padded(int64_t n_nodes, int64_t n_edges_padded, const int32_t* senders,
+                             const int32_t* receivers, int32_t* rowptr, int32_t* sender_perm,
+                             int32_t* colptr, void* stream);
+int e3j_conv_fwd_padded(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges_padded, const float* x,
+                        const float* sh, const float* w, const int32_t* senders,
+                        const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                        size_t workspace_bytes, void* stream);
+int e3j_conv_bwd_padded(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges_padded, const float* x,
+                        const float* sh, const float* w, const int32_t* senders,
+                        const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                        const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
+                        float* grad_w, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Standalone channelwise tensor product with per-row, per-path weights (paper:
  * tensor-product formula followed by the edge-scalar weighting; backward: the
  * tensor-product backward rule, one streaming pass).  Rows are their own receivers:

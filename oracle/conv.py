@@ -135,3 +135,26 @@ def tp_bwd(cp: Coupling, x1, x2, w, dz):
     dw = np.zeros_like(w)
     np.add.at(dw, (slice(None), cp.i3, slice(None)), z * dz)
     return dx1, dx2, dw
+
+
+# ---------------------------------------------------------------------------------------------
+# Padded edge lists.  The paper keeps the neighbour list of its molecular-dynamics runs at a fixed
+# padded size and flags the padding edges, without saying how; the reading taken here: an edge
+# whose receiver id is >= the number of nodes is padding.  A padding edge takes no part in any
+# sum, nothing of it is looked at, and its rows of the edge-local cotangents are zero.
+def conv_fwd_padded(cp: Coupling, x, y, s, senders, receivers) -> np.ndarray:
+    """The forward sum over the real edges only."""
+    real = np.asarray(receivers) < x.shape[0]
+    return conv_fwd(cp, x, np.asarray(y)[real], np.asarray(s)[real], np.asarray(senders)[real],
+                    np.asarray(receivers)[real])
+
+
+def conv_bwd_padded(cp: Coupling, x, y, s, senders, receivers, dm):
+    """(dx, dy, ds): dx from the real edges; dy, ds rows of padding edges are zero."""
+    real = np.asarray(receivers) < x.shape[0]
+    dx, dy_r, ds_r = conv_bwd(cp, x, np.asarray(y)[real], np.asarray(s)[real], np.asarray(senders)[real],
+                              np.asarray(receivers)[real], dm)
+    e = len(receivers)
+    dy = np.zeros((e, cp.dp)); ds = np.zeros((e, cp.P, cp.nq))
+    dy[real] = dy_r; ds[real] = ds_r
+    return dx, dy, ds

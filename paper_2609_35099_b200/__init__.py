@@ -79,12 +79,15 @@ def _load():
     lib.e3j_plan_device_status.restype = i32
     lib.e3j_graph_prepare.argtypes = [i64, i64, vp, vp, vp, vp, vp, vp]
     lib.e3j_graph_validate.argtypes = [i64, i64, vp, vp, vp, vp]
+    lib.e3j_graph_prepare_padded.argtypes = [i64, i64, vp, vp, vp, vp, vp, vp]
     lib.e3j_conv_fwd_workspace_bytes.argtypes = [vp, i64, i64]
     lib.e3j_conv_fwd_workspace_bytes.restype = sz
     lib.e3j_conv_bwd_workspace_bytes.argtypes = [vp, i64, i64]
     lib.e3j_conv_bwd_workspace_bytes.restype = sz
     lib.e3j_conv_fwd.argtypes = [vp, i64, i64] + [vp] * 8 + [sz, vp]
     lib.e3j_conv_bwd.argtypes = [vp, i64, i64] + [vp] * 13 + [sz, vp]
+    lib.e3j_conv_fwd_padded.argtypes = [vp, i64, i64] + [vp] * 8 + [sz, vp]
+    lib.e3j_conv_bwd_padded.argtypes = [vp, i64, i64] + [vp] * 13 + [sz, vp]
     lib.e3j_conv_fwd_noalloc.argtypes = [vp, i64, i64] + [vp] * 7
     lib.e3j_conv_fwd_noalloc.restype = i32
     lib.e3j_tp_fwd.argtypes = [vp, i64] + [vp] * 5
@@ -205,22 +208,29 @@ def _workspace(nbytes: int, like, workspace):
     return workspace
 
 
-def e3j_graph_prepare(n_nodes: int, senders, receivers, want_transpose: bool = True, stream=None):
+def e3j_graph_prepare(n_nodes: int, senders, receivers, want_transpose: bool = True, stream=None,
+                      _entry: str = "e3j_graph_prepare"):
     """(rowptr, sender_perm, colptr) int32 CUDA tensors; the last two are None unless want_transpose."""
     torch = _torch()
     e = senders.numel()
     rowptr = torch.empty(n_nodes + 1, dtype=torch.int32, device=senders.device)
     perm = torch.empty(max(e, 1), dtype=torch.int32, device=senders.device) if want_transpose else None
     colptr = torch.empty(n_nodes + 1, dtype=torch.int32, device=senders.device) if want_transpose else None
-    _check(_load().e3j_graph_prepare(n_nodes, e, _dev_ptr(senders, torch.int32, (e,), "senders"),
-                                     _dev_ptr(receivers, torch.int32, (e,), "receivers"),
-                                     _dev_ptr(rowptr, torch.int32, None, "rowptr"),
-                                     _dev_ptr(perm, torch.int32, None, "sender_perm"),
-                                     _dev_ptr(colptr, torch.int32, None, "colptr"), _stream(stream)),
-           "e3j_graph_prepare")
+    _check(getattr(_load(), _entry)(n_nodes, e, _dev_ptr(senders, torch.int32, (e,), "senders"),
+                                    _dev_ptr(receivers, torch.int32, (e,), "receivers"),
+                                    _dev_ptr(rowptr, torch.int32, None, "rowptr"),
+                                    _dev_ptr(perm, torch.int32, None, "sender_perm"),
+                                    _dev_ptr(colptr, torch.int32, None, "colptr"), _stream(stream)),
+           _entry)
     if perm is not None:
         perm = perm[:e]
     return rowptr, perm, colptr
+
+
+def e3j_graph_prepare_padded(n_nodes: int, senders, receivers, want_transpose: bool = True, stream=None):
+    """As e3j_graph_prepare for a padded edge list (edges with receiver >= n_nodes are padding and come last):
+    rowptr[n_nodes] is the number of real edges, of sender_perm only that many entries are written."""
+    return e3j_graph_prepare(n_nodes, senders, receivers, want_transpose, stream, "e3j_graph_prepare_padded")
 
 
 def e3j_graph_validate(n_nodes: int, senders, receivers, stream=None) -> int:
@@ -244,7 +254,7 @@ def e3j_conv_bwd_workspace_bytes(plan: Plan, n_nodes: int, n_edges: int) -> int:
 
 
 def e3j_conv_fwd(plan: Plan, x, sh, w, senders, receivers, rowptr=None, out=None, workspace=None,
-                 stream=None):
+                 stream=None, _entry: str = "e3j_conv_fwd"):
     torch = _torch()
     n, e = x.shape[0], senders.numel()
     f32, i32 = torch.float32, torch.int32
@@ -252,7 +262,7 @@ def e3j_conv_fwd(plan: Plan, x, sh, w, senders, receivers, rowptr=None, out=None
         out = torch.empty((n, plan.d_out, plan.n_channels), dtype=f32, device=x.device)
     nbytes = e3j_conv_fwd_workspace_bytes(plan, n, e)
     workspace = _workspace(nbytes, x, workspace)
-    _check(_load().e3j_conv_fwd(
+    _check(getattr(_load(), _entry)(
         plan.handle, n, e,
         _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"),
         _dev_ptr(sh, f32, (e, plan.d_sh), "sh"),
@@ -260,8 +270,13 @@ def e3j_conv_fwd(plan: Plan, x, sh, w, senders, receivers, rowptr=None, out=None
         _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
         _dev_ptr(rowptr, i32, (n + 1,), "rowptr"),
         _dev_ptr(out, f32, (n, plan.d_out, plan.n_channels), "out"),
-        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_fwd")
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), _entry)
     return out
+
+
+def e3j_conv_fwd_padded(plan: Plan, x, sh, w, senders, receivers, rowptr, out=None, workspace=None, stream=None):
+    """Forward convolution over a padded edge list; rowptr (from e3j_graph_prepare_padded) is required."""
+    return e3j_conv_fwd(plan, x, sh, w, senders, receivers, rowptr, out, workspace, stream, "e3j_conv_fwd_padded")
 
 
 def e3j_conv_fwd_noalloc(plan: Plan, x, sh, w, senders, receivers, out, stream=None):
@@ -285,7 +300,8 @@ def e3j_conv_fwd_noalloc(plan: Plan, x, sh, w, senders, receivers, out, stream=N
 
 
 def e3j_conv_bwd(plan: Plan, x, sh, w, senders, receivers, grad_out, rowptr=None, sender_perm=None,
-                 colptr=None, grad_x=True, grad_sh=True, grad_w=True, workspace=None, stream=None):
+                 colptr=None, grad_x=True, grad_sh=True, grad_w=True, workspace=None, stream=None,
+                 _entry: str = "e3j_conv_bwd"):
     """Returns (grad_x, grad_sh, grad_w).  Each grad_* argument is True (allocate), False/None
     (not wanted) or a preallocated tensor."""
     torch = _torch()
@@ -302,7 +318,7 @@ def e3j_conv_bwd(plan: Plan, x, sh, w, senders, receivers, grad_out, rowptr=None
     grad_w = alloc(grad_w, (e, plan.n_paths, plan.n_channels))
     nbytes = e3j_conv_bwd_workspace_bytes(plan, n, e)
     workspace = _workspace(nbytes, x, workspace)
-    _check(_load().e3j_conv_bwd(
+    _check(getattr(_load(), _entry)(
         plan.handle, n, e,
         _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"),
         _dev_ptr(sh, f32, (e, plan.d_sh), "sh"),
@@ -314,8 +330,16 @@ def e3j_conv_bwd(plan: Plan, x, sh, w, senders, receivers, grad_out, rowptr=None
         _dev_ptr(grad_x, f32, (n, plan.d_in, plan.n_channels), "grad_x"),
         _dev_ptr(grad_sh, f32, (e, plan.d_sh), "grad_sh"),
         _dev_ptr(grad_w, f32, (e, plan.n_paths, plan.n_channels), "grad_w"),
-        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_bwd")
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), _entry)
     return grad_x, grad_sh, grad_w
+
+
+def e3j_conv_bwd_padded(plan: Plan, x, sh, w, senders, receivers, grad_out, rowptr, sender_perm=None,
+                        colptr=None, grad_x=True, grad_sh=True, grad_w=True, workspace=None, stream=None):
+    """Backward convolution over a padded edge list; rowptr (from e3j_graph_prepare_padded) is required.
+    The grad_sh / grad_w rows of padding edges come back as zeros."""
+    return e3j_conv_bwd(plan, x, sh, w, senders, receivers, grad_out, rowptr, sender_perm, colptr, grad_x,
+                        grad_sh, grad_w, workspace, stream, "e3j_conv_bwd_padded")
 
 
 def e3j_tp_fwd(plan: Plan, x1, x2, w, out=None, stream=None):

@@ -13,7 +13,7 @@ thread_local int g_last_cuda_error = 0;
 std::atomic<int64_t> g_launch_count{0};
 
 int graph_prepare(int64_t, int64_t, const int32_t*, const int32_t*, int32_t*, int32_t*, int32_t*,
-                  cudaStream_t);
+                  cudaStream_t, bool padded = false);
 int graph_validate(int64_t, int64_t, const int32_t*, const int32_t*, int32_t*, cudaStream_t);
 
 namespace {
@@ -215,6 +215,17 @@ int e3j_graph_prepare(int64_t n_nodes, int64_t n_edges, const int32_t* senders,
                          (cudaStream_t)stream);
 }
 
+int e3j_graph_prepare_padded(int64_t n_nodes, int64_t n_edges, const int32_t* senders,
+                             const int32_t* receivers, int32_t* rowptr, int32_t* sender_perm,
+                             int32_t* colptr, void* stream) {
+    if (n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
+        return E3J_ERR_INVALID_ARG;
+    if (n_edges > 0 && (!senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    if ((sender_perm == nullptr) != (colptr == nullptr)) return E3J_ERR_INVALID_ARG;
+    return graph_prepare(n_nodes, n_edges, senders, receivers, rowptr, sender_perm, colptr,
+                         (cudaStream_t)stream, true);
+}
+
 int e3j_graph_validate(int64_t n_nodes, int64_t n_edges, const int32_t* senders,
                        const int32_t* receivers, int32_t* status, void* stream) {
     if (n_nodes < 0 || n_edges < 0 || !status) return E3J_ERR_INVALID_ARG;
@@ -232,15 +243,17 @@ size_t e3j_conv_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64
     return layout(plan, n_nodes, n_edges, true).total;
 }
 
-int e3j_conv_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
-                 const float* sh, const float* w, const int32_t* senders,
-                 const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
-                 size_t workspace_bytes, void* stream) {
+static int conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                         const float* sh, const float* w, const int32_t* senders,
+                         const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                         size_t workspace_bytes, void* stream, bool padded) {
     if (!plan || n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
         return E3J_ERR_INVALID_ARG;
     if (n_nodes == 0) return E3J_OK;
     if (!out || !x) return E3J_ERR_INVALID_ARG;
     if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    if (padded && !rowptr) return E3J_ERR_INVALID_ARG;  // rowptr[n_nodes] is where the kernels learn the edge count
+    const int32_t* n_real = padded ? rowptr + n_nodes : nullptr;
     cudaStream_t st = (cudaStream_t)stream;
     const WorkspaceLayout L = layout(plan, n_nodes, n_edges, false);
     if (int s = check_workspace(workspace, workspace_bytes, L.total)) return s;
@@ -255,6 +268,7 @@ int e3j_conv_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
         a.senders = senders; a.receivers = receivers; a.rowptr = rowptr; a.out = out;
         a.workspace = ws + L.scratch; a.workspace_bytes = workspace_bytes - L.scratch; a.stream = st;
         a.status = t.status;
+        a.n_real = n_real;
         return fk->conv_fwd(a);
     }
     if (!rowptr) {
@@ -269,17 +283,35 @@ int e3j_conv_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
     return after_launch();
 }
 
-int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+int e3j_conv_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
                  const float* sh, const float* w, const int32_t* senders,
-                 const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
-                 const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
-                 float* grad_w, void* workspace, size_t workspace_bytes, void* stream) {
+                 const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                 size_t workspace_bytes, void* stream) {
+    return conv_fwd_impl(plan, n_nodes, n_edges, x, sh, w, senders, receivers, rowptr, out, workspace,
+                         workspace_bytes, stream, false);
+}
+
+int e3j_conv_fwd_padded(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges_padded, const float* x,
+                        const float* sh, const float* w, const int32_t* senders,
+                        const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    return conv_fwd_impl(plan, n_nodes, n_edges_padded, x, sh, w, senders, receivers, rowptr, out, workspace,
+                         workspace_bytes, stream, true);
+}
+
+static int conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                         const float* sh, const float* w, const int32_t* senders,
+                         const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                         const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
+                         float* grad_w, void* workspace, size_t workspace_bytes, void* stream, bool padded) {
     if (!plan || n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
         return E3J_ERR_INVALID_ARG;
     if (n_nodes == 0) return E3J_OK;
     if (!x || !grad_out) return E3J_ERR_INVALID_ARG;
     if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
     if ((sender_perm == nullptr) != (colptr == nullptr)) return E3J_ERR_INVALID_ARG;
+    if (padded && !rowptr) return E3J_ERR_INVALID_ARG;  // rowptr[n_nodes] is where the kernels learn the edge count
+    const int32_t* n_real = padded ? rowptr + n_nodes : nullptr;
     cudaStream_t st = (cudaStream_t)stream;
     const WorkspaceLayout L = layout(plan, n_nodes, n_edges, true);
     if (int s = check_workspace(workspace, workspace_bytes, L.total)) return s;
@@ -287,7 +319,7 @@ int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
     if (grad_x && !sender_perm) {
         int32_t* cp = (int32_t*)(ws + L.colptr);
         int32_t* pm = (int32_t*)(ws + L.perm);
-        if (int s = graph_prepare(n_nodes, n_edges, senders, receivers, nullptr, pm, cp, st)) return s;
+        if (int s = graph_prepare(n_nodes, n_edges, senders, receivers, nullptr, pm, cp, st, padded)) return s;
         sender_perm = pm; colptr = cp;
     }
     const FastKernels* fk = fast_lookup(plan);
@@ -302,6 +334,7 @@ int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
         a.sender_perm = sender_perm; a.colptr = colptr; a.grad_out = grad_out;
         a.grad_x = grad_x; a.grad_sh = grad_sh; a.grad_w = grad_w;
         a.workspace = ws + L.scratch; a.workspace_bytes = workspace_bytes - L.scratch; a.stream = st;
+        a.n_real = n_real;
         return fk->conv_bwd(a);
     }
     DeviceTables t;
@@ -309,7 +342,7 @@ int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
     const Dims dm = dims_of(plan);
     if ((grad_w || grad_sh) && n_edges > 0) {
         generic::conv_bwd_edge_kernel<false><<<grid_for(n_edges), 256, 0, st>>>(
-            t, dm, n_edges, x, sh, w, senders, receivers, grad_out, grad_w, grad_sh);
+            t, dm, n_edges, x, sh, w, senders, receivers, grad_out, grad_w, grad_sh, n_real);
         if (int s = after_launch()) return s;
     }
     if (grad_x) {
@@ -318,6 +351,24 @@ int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
         if (int s = after_launch()) return s;
     }
     return E3J_OK;
+}
+
+int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                 const float* sh, const float* w, const int32_t* senders,
+                 const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                 const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
+                 float* grad_w, void* workspace, size_t workspace_bytes, void* stream) {
+    return conv_bwd_impl(plan, n_nodes, n_edges, x, sh, w, senders, receivers, rowptr, sender_perm, colptr,
+                         grad_out, grad_x, grad_sh, grad_w, workspace, workspace_bytes, stream, false);
+}
+
+int e3j_conv_bwd_padded(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges_padded, const float* x,
+                        const float* sh, const float* w, const int32_t* senders,
+                        const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                        const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
+                        float* grad_w, void* workspace, size_t workspace_bytes, void* stream) {
+    return conv_bwd_impl(plan, n_nodes, n_edges_padded, x, sh, w, senders, receivers, rowptr, sender_perm,
+                         colptr, grad_out, grad_x, grad_sh, grad_w, workspace, workspace_bytes, stream, true);
 }
 
 int e3j_tp_fwd(const e3j_plan* plan, int64_t rows, const float* x1, const float* x2,
@@ -350,7 +401,7 @@ int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
     const Dims dm = dims_of(plan);
     if (grad_w || grad_x2) {
         generic::conv_bwd_edge_kernel<true><<<grid_for(rows), 256, 0, st>>>(t, dm, rows, x1, x2, w, nullptr,
-                                                                           nullptr, grad_out, grad_w, grad_x2);
+                                                                           nullptr, grad_out, grad_w, grad_x2, nullptr);
         if (int s = after_launch()) return s;
     }
     if (grad_x1) {

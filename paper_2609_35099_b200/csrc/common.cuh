@@ -48,6 +48,7 @@ struct ConvArgs {
     size_t workspace_bytes;
     cudaStream_t stream;
     int32_t* status;  // device status word of the plan on this device
+    const int32_t* n_real;  // padded call: device word with the number of real edges (rowptr[n_nodes]); else null
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

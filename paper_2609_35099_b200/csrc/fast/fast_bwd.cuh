@@ -33,6 +33,7 @@ struct BwdParams {
     int64_t n_nodes, n_edges, chunk;   // chunk = edges per CTA
     int32_t* status;
     int identity;                      // 1: every edge is its own sender and receiver; dx_edge is then grad_x itself
+    const int32_t* n_real;             // padded call: device word holding the number of real edges (else null)
 };
 
 template <class S>
@@ -199,8 +200,8 @@ fast_bwd_kernel(const BwdParams p) {
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t e_begin = min(p.n_edges, (int64_t)blockIdx.x * p.chunk);
-    const int64_t e_end = min(p.n_edges, e_begin + p.chunk);
+    int64_t n_edges, chunk, e_begin, e_end;   // n_edges: the real edges (a padded call learns their number here)
+    cta_edge_range(p.n_edges, p.chunk, p.n_real, n_edges, chunk, e_begin, e_end);
     const int n_tiles = (int)((e_end - e_begin + T - 1) / T);
 
     if (threadIdx.x == 0) {

@@ -21,6 +21,16 @@ __global__ void fwd_fixup_kernel(int n_cta, int row_f4, const float4* __restrict
     }
 }
 
+__global__ void bwd_zero_padding_kernel(const int32_t* __restrict__ n_real, int64_t n_edges, int w_row_f4,
+                                        int sh_row, float4* __restrict__ grad_w, float* __restrict__ grad_sh) {
+    const int64_t first = min((int64_t)*n_real, n_edges);
+    const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t e = first + blockIdx.x; e < n_edges; e += gridDim.x) {
+        for (int i = threadIdx.x; i < w_row_f4; i += blockDim.x) grad_w[(size_t)e * w_row_f4 + i] = z;
+        for (int i = threadIdx.x; i < sh_row; i += blockDim.x) grad_sh[(size_t)e * sh_row + i] = 0.f;
+    }
+}
+
 __global__ void bwd_dx_reduce_kernel(int64_t n_nodes, int row_f4, const float4* __restrict__ dx_edge,
                                      const int32_t* __restrict__ sender_perm, const int32_t* __restrict__ colptr,
                                      float4* __restrict__ grad_x) {

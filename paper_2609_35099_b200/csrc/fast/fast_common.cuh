@@ -116,11 +116,32 @@ struct FwdParams {
     int32_t* part_recv;                // [G][2] receiver of the head / tail partial, or -1
     int32_t* status;                   // device status word (0 = fine)
     int identity;                      // 1: every edge is its own sender and receiver (standalone tensor product)
+    const int32_t* n_real;             // padded call: device word holding the number of real edges (else null)
 };
 
 // Sums the pieces of every receiver row that was split between CTAs, in CTA order.
 __global__ void fwd_fixup_kernel(int n_cta, int row_f4, const float4* __restrict__ partial,
                                  const int32_t* __restrict__ part_recv, float4* __restrict__ out);
+
+// The edges this CTA works on.  Plain call: the host's split (n_edges, chunk).  Padded call: the number of real
+// edges is only known on the device, so the equal split is formed here from *n_real.
+__device__ __forceinline__ void cta_edge_range(const int64_t n_edges_host, const int64_t chunk_host,
+                                               const int32_t* n_real, int64_t& n_edges, int64_t& chunk,
+                                               int64_t& e_begin, int64_t& e_end) {
+    n_edges = n_edges_host;
+    chunk = chunk_host;
+    if (n_real) {
+        n_edges = min((int64_t)*n_real, n_edges_host);
+        const int64_t per = (n_edges + gridDim.x - 1) / gridDim.x;
+        chunk = max((int64_t)4, (per + 3) / 4 * 4);
+    }
+    e_begin = min(n_edges, (int64_t)blockIdx.x * chunk);
+    e_end = min(n_edges, e_begin + chunk);
+}
+
+// Backward of a padded call: zero rows of grad_w and grad_sh for the padding edges [*n_real, n_edges).
+__global__ void bwd_zero_padding_kernel(const int32_t* __restrict__ n_real, int64_t n_edges, int w_row_f4,
+                                        int sh_row, float4* __restrict__ grad_w, float* __restrict__ grad_sh);
 
 // Backward pass 2: grad_x[a] = sum of the per-edge shares of the edges sent by a, in edge order.
 __global__ void bwd_dx_reduce_kernel(int64_t n_nodes, int row_f4, const float4* __restrict__ dx_edge,

@@ -51,7 +51,7 @@ struct FwdSmem {
 template <class S, int G>
 __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* smem, const int ch, const int warp,
                                              const int lane, const int64_t e_begin, const int64_t e_end,
-                                             const int n_tiles) {
+                                             const int n_tiles, const int64_t n_edges) {
     using Vec = typename VecOf<S::V>::type;
     using L = FwdSmem<S>;
     constexpr int T = L::T, NS = L::NS;
@@ -66,7 +66,7 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
     // identity mode: receiver of edge e is e, so no row ever straddles a CTA boundary
     const int prev_recv = p.identity ? (int)e_begin - 1
                                      : ((e_begin > 0 && e_begin < e_end) ? p.receivers[e_begin - 1] : -1);
-    const int next_recv = p.identity ? (int)e_end : ((e_end < p.n_edges) ? p.receivers[e_end] : -2);
+    const int next_recv = p.identity ? (int)e_end : ((e_end < n_edges) ? p.receivers[e_end] : -2);
     if (!p.identity && warp == 0 && lane == 0) { p.part_recv[2 * cta] = -1; p.part_recv[2 * cta + 1] = -1; }
 
     Vec acc[S::F_RMAX];
@@ -143,8 +143,10 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
     if (!*abort_flag) {
         if (cur >= 0) {
             flush(true);
-            if (e_end == p.n_edges && !p.identity) zero_rows(cur + 1, (int)p.n_nodes);
+            if (e_end == n_edges && !p.identity) zero_rows(cur + 1, (int)p.n_nodes);
         }
+        // a padded call without a single real edge: nobody saw a receiver, the first CTA writes the zero rows
+        if (n_edges == 0 && cta == 0 && !p.identity) zero_rows(0, (int)p.n_nodes);
     }
 }
 
@@ -184,8 +186,8 @@ fast_fwd_kernel(const FwdParams p) {
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t e_begin = min(p.n_edges, (int64_t)blockIdx.x * p.chunk);
-    const int64_t e_end = min(p.n_edges, e_begin + p.chunk);
+    int64_t n_edges, chunk, e_begin, e_end;   // n_edges: the real edges (a padded call learns their number here)
+    cta_edge_range(p.n_edges, p.chunk, p.n_real, n_edges, chunk, e_begin, e_end);
     const int n_tiles = (int)((e_end - e_begin + T - 1) / T);
 
     if (threadIdx.x == 0) {
@@ -197,7 +199,7 @@ fast_fwd_kernel(const FwdParams p) {
     __syncthreads();
     if (warp == NCONS) producer_loop<L, FwdTab<S>, 0>(p, smem, lane, e_begin, e_end, n_tiles);
     else if (warp == NCONS + 1) producer_loop<L, FwdTab<S>, 1>(p, smem, lane, e_begin, e_end, n_tiles);
-    else FwdDispatch<S, 0>::run(warp % S::FW, p, smem, warp / S::FW, warp, lane, e_begin, e_end, n_tiles);
+    else FwdDispatch<S, 0>::run(warp % S::FW, p, smem, warp / S::FW, warp, lane, e_begin, e_end, n_tiles, n_edges);
 }
 
 }  // namespace fast

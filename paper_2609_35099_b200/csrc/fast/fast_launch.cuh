@@ -58,6 +58,7 @@ int launch_fwd(const ConvArgs& a) {
     p.part_recv = reinterpret_cast<int32_t*>(a.workspace);
     p.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(a.workspace) + kPartRecvBytes);
     p.status = a.status;
+    p.n_real = a.n_real;
     constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 2) * 32;  // consumers + two producer warps
     fast_fwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
@@ -137,9 +138,15 @@ int launch_bwd(const ConvArgs& a) {
     p.n_nodes = a.n_nodes; p.n_edges = a.n_edges;
     p.chunk = (a.n_edges + n_cta - 1) / n_cta;
     p.status = a.status;
+    p.n_real = a.n_real;
     constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;  // consumers + one producer warp
     fast_bwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
+    if (a.n_real) {
+        bwd_zero_padding_kernel<<<148 * 8, 256, 0, a.stream>>>(a.n_real, a.n_edges, S::P * S::NQ / 4, S::DSH,
+                                                              reinterpret_cast<float4*>(a.grad_w), a.grad_sh);
+        if (int s = after_launch()) return s;
+    }
     // one CTA per sender: the hardware hands them out as CTAs finish, so uneven degrees do not leave a tail
     const int64_t blocks = std::min<int64_t>(a.n_nodes, (int64_t)1 << 30);
     bwd_dx_reduce_kernel<<<(int)blocks, S::DIN * S::NQ / 4, 0, a.stream>>>(a.n_nodes, S::DIN * S::NQ / 4,

@@ -53,9 +53,18 @@ conv_bwd_edge_kernel(DeviceTables t, Dims dm, int64_t n_edges, const float* __re
                      const float* __restrict__ sh, const float* __restrict__ w,
                      const int32_t* __restrict__ senders, const int32_t* __restrict__ receivers,
                      const float* __restrict__ g, float* __restrict__ grad_w,
-                     float* __restrict__ grad_sh) {
+                     float* __restrict__ grad_sh, const int32_t* __restrict__ n_real) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    // padded call: edges from *n_real on are padding; their gradient rows are zero and nothing of them is read
+    const int64_t n_live = n_real ? min((int64_t)*n_real, n_edges) : n_edges;
     for (int64_t e = blockIdx.x; e < n_edges; e += gridDim.x) {
+        if (e >= n_live) {
+            if (grad_w)
+                for (int idx = threadIdx.x; idx < dm.P * dm.nq; idx += blockDim.x)
+                    grad_w[(size_t)e * dm.P * dm.nq + idx] = 0.f;
+            if (grad_sh && threadIdx.x < dm.dp) grad_sh[(size_t)e * dm.dp + threadIdx.x] = 0.f;
+            continue;
+        }
         const int64_t a = IDENT ? e : (int64_t)senders[e];
         const int64_t b = IDENT ? e : (int64_t)receivers[e];
         const float* xa = x + (size_t)a * dm.d * dm.nq;

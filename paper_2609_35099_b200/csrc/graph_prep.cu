@@ -20,11 +20,14 @@ __global__ void rowptr_kernel(int64_t n_nodes, int64_t n_edges, const int32_t* _
     }
 }
 
-__global__ void count_senders_kernel(int64_t n_edges, const int32_t* __restrict__ senders,
-                                     int32_t* __restrict__ colptr) {
+// `pad_recv`: when not null, edges whose receiver id is >= n_nodes are padding and are left out.
+__global__ void count_senders_kernel(int64_t n_nodes, int64_t n_edges, const int32_t* __restrict__ senders,
+                                     const int32_t* __restrict__ pad_recv, int32_t* __restrict__ colptr) {
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < n_edges;
-         e += (int64_t)gridDim.x * blockDim.x)
+         e += (int64_t)gridDim.x * blockDim.x) {
+        if (pad_recv && pad_recv[e] >= n_nodes) continue;
         atomicAdd(&colptr[senders[e]], 1);
+    }
 }
 
 // In-place exclusive scan of v[0..n) by one block; v[n] receives the total.
@@ -66,10 +69,12 @@ __global__ void __launch_bounds__(1024) exclusive_scan_kernel(int64_t n, int32_t
 }
 
 // Claims a slot for every edge; afterwards colptr[a] is the END of bucket a.
-__global__ void fill_kernel(int64_t n_edges, const int32_t* __restrict__ senders,
-                            int32_t* __restrict__ colptr, int32_t* __restrict__ perm) {
+__global__ void fill_kernel(int64_t n_nodes, int64_t n_edges, const int32_t* __restrict__ senders,
+                            const int32_t* __restrict__ pad_recv, int32_t* __restrict__ colptr,
+                            int32_t* __restrict__ perm) {
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < n_edges;
          e += (int64_t)gridDim.x * blockDim.x) {
+        if (pad_recv && pad_recv[e] >= n_nodes) continue;
         const int32_t pos = atomicAdd(&colptr[senders[e]], 1);
         perm[pos] = (int32_t)e;
     }
@@ -144,7 +149,8 @@ inline int blocks_for(int64_t n, int threads) {
 }  // namespace
 
 int graph_prepare(int64_t n_nodes, int64_t n_edges, const int32_t* senders, const int32_t* receivers,
-                  int32_t* rowptr, int32_t* sender_perm, int32_t* colptr, cudaStream_t st) {
+                  int32_t* rowptr, int32_t* sender_perm, int32_t* colptr, cudaStream_t st, bool padded) {
+    const int32_t* pad_recv = padded ? receivers : nullptr;
     if (rowptr) {
         rowptr_kernel<<<blocks_for(n_nodes + 1, 256), 256, 0, st>>>(n_nodes, n_edges, receivers, rowptr);
         if (int s = after_launch()) return s;
@@ -152,13 +158,14 @@ int graph_prepare(int64_t n_nodes, int64_t n_edges, const int32_t* senders, cons
     if (sender_perm && colptr) {
         E3J_CUDA_TRY(cudaMemsetAsync(colptr, 0, sizeof(int32_t) * (size_t)(n_nodes + 1), st));
         if (n_edges > 0) {
-            count_senders_kernel<<<blocks_for(n_edges, 256), 256, 0, st>>>(n_edges, senders, colptr);
+            count_senders_kernel<<<blocks_for(n_edges, 256), 256, 0, st>>>(n_nodes, n_edges, senders, pad_recv, colptr);
             if (int s = after_launch()) return s;
         }
         exclusive_scan_kernel<<<1, 1024, 0, st>>>(n_nodes, colptr);
         if (int s = after_launch()) return s;
         if (n_edges > 0) {
-            fill_kernel<<<blocks_for(n_edges, 256), 256, 0, st>>>(n_edges, senders, colptr, sender_perm);
+            fill_kernel<<<blocks_for(n_edges, 256), 256, 0, st>>>(n_nodes, n_edges, senders, pad_recv, colptr,
+                                                               sender_perm);
             if (int s = after_launch()) return s;
             sort_buckets_kernel<<<blocks_for(n_nodes, 128), 128, 0, st>>>(n_nodes, colptr, sender_perm);
             if (int s = after_launch()) return s;

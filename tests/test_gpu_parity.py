@@ -160,6 +160,60 @@ def test_tensor_product(rows, flags):
     assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="tp grad_w")
 
 
+@pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
+@pytest.mark.parametrize("config,n_atoms,pad", [(1, None, 37), (2, 192, 1500), (2, 192, 0)])
+def test_padded_edge_lists(config, n_atoms, pad, flags):
+    """Padded calls: the real edges give bit for bit what the plain call gives on the unpadded list, whatever
+    the padding entries hold (NaN weights, wild sender ids); padding rows of grad_sh / grad_w are zero; the
+    number of real edges is never passed from the host."""
+    wl, plan, cp, x, y, w, g = make_case(config, n_atoms, flags=flags)
+    n, e = wl.n_nodes, wl.n_edges
+    rng = np.random.default_rng(5)
+    yp = np.concatenate([y, np.full((pad, y.shape[1]), np.nan, np.float32)])
+    wp = np.concatenate([w, np.full((pad,) + w.shape[1:], np.nan, np.float32)])
+    sndp = np.concatenate([wl.senders, rng.integers(-2 ** 30, 2 ** 30, pad).astype(np.int32)])
+    rcvp = np.concatenate([wl.receivers, np.sort(rng.integers(n, 2 ** 30, pad)).astype(np.int32)])
+    dx, dg = _cuda(x), _cuda(g)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    rowptr, perm, colptr = e3j.e3j_graph_prepare(n, snd, rcv)
+    out = e3j.e3j_conv_fwd(plan, dx, _cuda(y), _cuda(w), snd, rcv, rowptr)
+    gx, gy, gw = e3j.e3j_conv_bwd(plan, dx, _cuda(y), _cuda(w), snd, rcv, dg, rowptr, perm, colptr)
+    psnd, prcv, py, pw = _cuda(sndp), _cuda(rcvp), _cuda(yp), _cuda(wp)
+    prow, pperm, pcol = e3j.e3j_graph_prepare_padded(n, psnd, prcv)
+    assert int(prow[n]) == e and int(pcol[n]) == e
+    assert torch.equal(prow, rowptr) and torch.equal(pcol, colptr) and torch.equal(pperm[:e], perm[:e])
+    pout = e3j.e3j_conv_fwd_padded(plan, dx, py, pw, psnd, prcv, prow)
+    for prepared in (True, False):
+        pgx, pgy, pgw = e3j.e3j_conv_bwd_padded(plan, dx, py, pw, psnd, prcv, dg, prow,
+                                                pperm if prepared else None, pcol if prepared else None)
+        torch.cuda.synchronize()
+        assert torch.equal(pout, out) and torch.equal(pgx, gx)
+        assert torch.equal(pgy[:e], gy) and torch.equal(pgw[:e], gw)
+        assert torch.count_nonzero(pgy[e:]) == 0 and torch.count_nonzero(pgw[e:]) == 0
+    ref = oconv.conv_fwd_padded(cp, x, yp, wp, sndp, rcvp)
+    assert_blockwise_close(pout.cpu().numpy(), ref, blocks_of_paths(cp.paths, "out"), what="out")
+    with pytest.raises(e3j.E3JError):
+        e3j.e3j_conv_fwd_padded(plan, dx, py, pw, psnd, prcv, None)
+
+
+@pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
+def test_padded_list_without_real_edges(flags):
+    wl, plan, cp, x, y, w, g = make_case(2, 192, flags=flags)
+    n, pad = wl.n_nodes, 64
+    rng = np.random.default_rng(6)
+    py = _cuda(np.full((pad, y.shape[1]), np.nan, np.float32))
+    pw = _cuda(np.full((pad,) + w.shape[1:], np.nan, np.float32))
+    psnd = _cuda(rng.integers(0, n, pad).astype(np.int32))
+    prcv = _cuda(np.full(pad, n, np.int32))
+    prow, pperm, pcol = e3j.e3j_graph_prepare_padded(n, psnd, prcv)
+    out = torch.full((n, plan.d_out, plan.n_channels), 7.0, device=DEV)
+    e3j.e3j_conv_fwd_padded(plan, _cuda(x), py, pw, psnd, prcv, prow, out=out)
+    gx, gy, gw = e3j.e3j_conv_bwd_padded(plan, _cuda(x), py, pw, psnd, prcv, _cuda(g), prow, pperm, pcol)
+    torch.cuda.synchronize()
+    for t in (out, gx, gy, gw):
+        assert torch.count_nonzero(t) == 0
+
+
 def test_optional_gradients_can_be_skipped():
     wl, plan, cp, x, y, w, g = make_case(1)
     snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)

@@ -200,3 +200,27 @@ def test_empty_receivers_give_zero_rows_and_silent_senders_zero_gradients():
     assert np.all(out[[0, 1, 3, 5]] == 0) and np.abs(out[2]).max() > 0
     dx, dy, ds = conv.conv_bwd(cp, x, y, s, snd, rcv, rng.standard_normal(out.shape).astype(np.float32))
     assert np.all(dx[2:] == 0) and np.abs(dx[0]).max() > 0
+
+
+def test_padding_edges_take_no_part():
+    """Padded edge list (receiver id >= number of nodes marks padding): the real edges give exactly the
+    unpadded result whatever the padding entries hold, padding rows of the edge-local cotangents are zero."""
+    rng = np.random.default_rng(13)
+    cp = conv.Coupling("2x0e+2x1o", 1)
+    n, e, pad = 5, 7, 4
+    snd = rng.integers(0, n, e).astype(np.int32); rcv = np.sort(rng.integers(0, n, e)).astype(np.int32)
+    x, y, s = _random_inputs(rng, cp, n, e)
+    dm = rng.standard_normal((n, cp.D, cp.nq)).astype(np.float32)
+    ref = conv.conv_fwd(cp, x, y, s, snd, rcv)
+    rx, ry, rs = conv.conv_bwd(cp, x, y, s, snd, rcv, dm)
+    yp = np.concatenate([y, np.full((pad, cp.dp), np.nan, np.float32)])
+    sp = np.concatenate([s, np.full((pad, cp.P, cp.nq), np.inf, np.float32)])
+    sndp = np.concatenate([snd, np.full(pad, -5, np.int32)])
+    rcvp = np.concatenate([rcv, np.array([n, n, n + 3, 2 ** 30], np.int32)])
+    assert np.array_equal(conv.conv_fwd_padded(cp, x, yp, sp, sndp, rcvp), ref)
+    dx, dy, ds = conv.conv_bwd_padded(cp, x, yp, sp, sndp, rcvp, dm)
+    assert np.array_equal(dx, rx) and np.array_equal(dy[:e], ry) and np.array_equal(ds[:e], rs)
+    assert np.all(dy[e:] == 0) and np.all(ds[e:] == 0)
+    # nothing but padding: zero output, zero gradients
+    out0 = conv.conv_fwd_padded(cp, x, yp[e:], sp[e:], sndp[e:], rcvp[e:])
+    assert out0.shape == ref.shape and np.all(out0 == 0)
