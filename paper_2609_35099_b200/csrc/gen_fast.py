@@ -163,10 +163,11 @@ class Sig:
                     best = bins
             if best is not None:
                 found[cap] = best
-            if len(found) >= 6:
+            if len(found) >= self.cfg.get("B_CAPS", 6):
                 break
         floor_cost = min(max(b[0] for b in bins) for bins in found.values())
-        cap = min(c for c, bins in found.items() if max(b[0] for b in bins) <= 1.03 * floor_cost)
+        slack = 1.0 + self.cfg.get("B_SLACK_PCT", 3) / 100.0
+        cap = min(c for c, bins in found.items() if max(b[0] for b in bins) <= slack * floor_cost)
         bins = [[b[0], b[2]] for b in found[cap]]
         groups = sorted((sorted(b[1]) for b in bins), key=lambda g: (g[0] if g else self.P))
         rows_of = []
