@@ -51,7 +51,14 @@ __device__ __forceinline__ float2 vadd(const float2 a, const float2 b) { return 
 __device__ __forceinline__ void vzero(float4& v) { v = make_float4(0.f, 0.f, 0.f, 0.f); }
 __device__ __forceinline__ void vzero(float2& v) { v = make_float2(0.f, 0.f); }
 
+// one channel per lane
+__device__ __forceinline__ float vmul(const float a, const float b) { return a * b; }
+__device__ __forceinline__ void vfma(float& acc, const float a, const float b) { acc = fmaf(a, b, acc); }
+__device__ __forceinline__ float vdot(const float a, const float b) { return a * b; }
+__device__ __forceinline__ float vadd(const float a, const float b) { return a + b; }
+__device__ __forceinline__ void vzero(float& v) { v = 0.f; }
 template <int V> struct VecOf;
+template <> struct VecOf<1> { using type = float; };
 template <> struct VecOf<4> { using type = float4; };
 template <> struct VecOf<2> { using type = float2; };
 

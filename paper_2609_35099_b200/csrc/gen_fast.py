@@ -191,7 +191,7 @@ class Sig:
             return []
         V, NQ = self.cfg.get("BV", self.V), self.NQ
         assert NQ % (32 * V) == 0
-        bvec = {2: "float2", 4: "float4"}[V]
+        bvec = {1: "float", 2: "float2", 4: "float4"}[V]
         BW, BT, BS, BC = self.cfg["BW"], self.cfg["BT"], self.cfg["BS"], self.cfg["BC"]
         groups, rows_of, a0, slots = self.bwd_layout()
         slot_of_pair = {pi: s for s, pi in enumerate(slots) if pi is not None}
@@ -302,7 +302,7 @@ class Sig:
         bounds, a0, slots = self.fwd_layout()
         slot_of_pair = {pi: s for s, pi in enumerate(slots) if pi is not None}
         rmax = max(bounds[g + 1] - bounds[g] for g in range(FW))
-        vec = {2: "float2", 4: "float4"}[V]
+        vec = {1: "float", 2: "float2", 4: "float4"}[V]
         # record tables in slot order
         rec_val, rec_i2, pair_tab = [], [], []
         for pi in slots:
