@@ -88,6 +88,18 @@ def test_conv_natural_parity_outputs():
     assert max(worst) < 1e-5
 
 
+def test_scalar_input_signature():
+    """First-layer signature: scalar node features only (128x0e), every output up to l = 3."""
+    import dataclasses
+    wl = dataclasses.replace(workloads.make_graph(2, 300), irreps_in="128x0e")
+    plan = e3j.e3j_plan_create("128x0e", 3, None, 3)
+    assert plan.specialised and plan.n_paths == 4 and plan.d_out == 16
+    cp = oconv.Coupling("128x0e", 3, None, 3)
+    x, y, w, g = workloads.make_features(wl, plan.n_paths, plan.d_out)
+    worst = run_conv_parity(wl, plan, cp, x, y, w, g)
+    assert max(worst) < 1e-5
+
+
 def test_conv_without_prepared_graph():
     worst = run_conv_parity(*make_case(1), prepared=False)
     assert max(worst) < 1e-5
