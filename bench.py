@@ -292,8 +292,10 @@ def main():
         return
 
     c, wl = build_workload(args.config)
+    t_plan = time.perf_counter()
     plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"],
                                e3j.E3J_PLAN_GENERIC_ONLY if args.generic else 0)
+    plan_build_ms = 1e3 * (time.perf_counter() - t_plan)   # host: paths, ladder-operator CG, record tables
     n, e = wl.n_nodes, wl.n_edges
     x, y, w, g = workloads.make_features(wl, plan.n_paths, plan.d_out)
     snd_h, rcv_h = wl.senders, wl.receivers
@@ -313,6 +315,15 @@ def main():
     conv_fwd = e3j.e3j_conv_fwd_padded if n_pad else e3j.e3j_conv_fwd
     conv_bwd = e3j.e3j_conv_bwd_padded if n_pad else e3j.e3j_conv_bwd
     rowptr, perm, colptr = prepare(n, d["snd"], d["rcv"])
+    # graph preparation is once per neighbour list and not part of the step; timed on its own
+    torch.cuda.synchronize()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record(stream)
+    for _ in range(5):
+        prepare(n, d["snd"], d["rcv"])
+    g1.record(stream)
+    torch.cuda.synchronize()
+    graph_prepare_ms = g0.elapsed_time(g1) / 5
     out = torch.empty((n, plan.d_out, plan.n_channels), device=dev)
     gx = torch.empty((n, plan.d_in, plan.n_channels), device=dev)
     gy = torch.empty((e_buf, plan.d_sh), device=dev)
@@ -419,6 +430,7 @@ def main():
             # per-call statistics over the timed steps: median, the paper's statistic (mean of the fastest
             # 20 % of the runs, as in its efficiency-comparison section), minimum and maximum
             "call_stats_ms": {"fwd": call_stats(fwd_ms), "bwd": call_stats(bwd_ms)},
+            "outside_the_step_ms": {"plan_build_host": plan_build_ms, "graph_prepare_device": graph_prepare_ms},
             "roofline": dominant, "roofline_fwd": roofs["fwd"], "roofline_bwd": roofs["bwd"],
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         }
