@@ -60,7 +60,8 @@ enum {
     E3J_ERR_INVALID_ARG = -1,   /* NULL pointer, negative size, capacity too small        */
     E3J_ERR_BAD_IRREPS = -2,    /* descriptor string does not parse                         */
     E3J_ERR_MUL_NOT_UNIFORM = -3, /* input irreps must share one multiplicity (= N_q)       */
-    E3J_ERR_UNSUPPORTED = -4,   /* a dimension exceeds 255, l > 8, or nothing couples        */
+    E3J_ERR_UNSUPPORTED = -4,   /* a dimension exceeds 255, l > 8, nothing couples; compute
+                                   calls: channel count N_q not a multiple of 4              */
     E3J_ERR_WORKSPACE = -5,     /* workspace NULL, misaligned (256 B) or too small            */
     E3J_ERR_CUDA = -6,          /* a CUDA runtime call failed; see e3j_last_cuda_error()      */
     E3J_ERR_GRAPH = -7          /* written by e3j_graph_validate into its device status word */

@@ -249,6 +249,7 @@ static int conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges,
                          size_t workspace_bytes, void* stream, bool padded) {
     if (!plan || n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
         return E3J_ERR_INVALID_ARG;
+    if (plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;  // the kernels work on groups of four channels
     if (n_nodes == 0) return E3J_OK;
     if (!out || !x) return E3J_ERR_INVALID_ARG;
     if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
@@ -306,6 +307,7 @@ static int conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges,
                          float* grad_w, void* workspace, size_t workspace_bytes, void* stream, bool padded) {
     if (!plan || n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
         return E3J_ERR_INVALID_ARG;
+    if (plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;  // the kernels work on groups of four channels
     if (n_nodes == 0) return E3J_OK;
     if (!x || !grad_out) return E3J_ERR_INVALID_ARG;
     if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
@@ -374,6 +376,7 @@ int e3j_conv_bwd_padded(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges_p
 int e3j_tp_fwd(const e3j_plan* plan, int64_t rows, const float* x1, const float* x2,
                const float* w, float* out, void* stream) {
     if (!plan || rows < 0) return E3J_ERR_INVALID_ARG;
+    if (plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;  // the kernels work on groups of four channels
     if (rows == 0) return E3J_OK;
     if (!x1 || !x2 || !w || !out) return E3J_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
@@ -390,6 +393,7 @@ int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
                const float* w, const float* grad_out, float* grad_x1, float* grad_x2,
                float* grad_w, void* stream) {
     if (!plan || rows < 0) return E3J_ERR_INVALID_ARG;
+    if (plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;  // the kernels work on groups of four channels
     if (rows == 0) return E3J_OK;
     if (!x1 || !x2 || !w || !grad_out) return E3J_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
@@ -418,7 +422,7 @@ const char* e3j_status_string(int status) {
         case E3J_ERR_INVALID_ARG: return "invalid argument";
         case E3J_ERR_BAD_IRREPS: return "irreps descriptor does not parse";
         case E3J_ERR_MUL_NOT_UNIFORM: return "input irreps must share one multiplicity";
-        case E3J_ERR_UNSUPPORTED: return "unsupported plan (a dimension exceeds 255, l > 8, or no path couples)";
+        case E3J_ERR_UNSUPPORTED: return "unsupported plan (a dimension exceeds 255, l > 8, no path couples, or channels not a multiple of 4)";
         case E3J_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case E3J_ERR_CUDA: return "CUDA runtime error";
         case E3J_ERR_GRAPH: return "graph invalid (receivers not sorted or index out of range)";
