@@ -257,6 +257,17 @@ def test_one_plan_on_two_streams():
     assert e3j.e3j_plan_device_status(plan) == 0
 
 
+def test_channel_counts_must_be_multiples_of_four():
+    plan = e3j.e3j_plan_create("6x0e+6x1o", 1)
+    x = torch.zeros((2, plan.d_in, 6), device=DEV)
+    sh = torch.zeros((1, plan.d_sh), device=DEV)
+    w = torch.zeros((1, plan.n_paths, 6), device=DEV)
+    idx = torch.zeros(1, dtype=torch.int32, device=DEV)
+    with pytest.raises(e3j.E3JError) as err:
+        e3j.e3j_conv_fwd(plan, x, sh, w, idx, idx)
+    assert err.value.status == e3j.E3J_ERR_UNSUPPORTED
+
+
 def test_optional_gradients_can_be_skipped():
     wl, plan, cp, x, y, w, g = make_case(1)
     snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
