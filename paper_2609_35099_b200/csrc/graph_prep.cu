@@ -92,20 +92,32 @@ __device__ inline void sift_down(int32_t* v, int64_t root, int64_t n) {
 }
 
 // Sorts every bucket ascending by edge id.  colptr holds bucket ENDS here.
-__global__ void sort_buckets_kernel(int64_t n_nodes, const int32_t* __restrict__ colptr,
-                                    int32_t* __restrict__ perm) {
-    for (int64_t a = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; a < n_nodes;
-         a += (int64_t)gridDim.x * blockDim.x) {
+// One warp per bucket.  Edge ids are distinct, so an element's place is the number of smaller ones: buckets
+// of up to kRankMax entries are staged in shared memory and every lane counts the ranks of its elements;
+// a longer bucket (a hub sender) is heap-sorted in place by one lane.
+constexpr int kRankMax = 1024;
+constexpr int kSortWarps = 4;
+
+__global__ void __launch_bounds__(32 * kSortWarps)
+sort_buckets_kernel(int64_t n_nodes, const int32_t* __restrict__ colptr, int32_t* __restrict__ perm) {
+    __shared__ int32_t stage[kSortWarps][kRankMax];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int32_t* mine = stage[warp];
+    for (int64_t a = (int64_t)blockIdx.x * kSortWarps + warp; a < n_nodes; a += (int64_t)gridDim.x * kSortWarps) {
         const int64_t begin = a ? colptr[a - 1] : 0, n = colptr[a] - begin;
         int32_t* v = perm + begin;
-        if (n <= 32) {
-            for (int64_t i = 1; i < n; ++i) {
-                const int32_t key = v[i];
-                int64_t j = i - 1;
-                while (j >= 0 && v[j] > key) { v[j + 1] = v[j]; --j; }
-                v[j + 1] = key;
+        if (n <= 1) continue;
+        if (n <= kRankMax) {
+            for (int i = lane; i < n; i += 32) mine[i] = v[i];
+            __syncwarp();
+            for (int i = lane; i < n; i += 32) {
+                const int32_t key = mine[i];
+                int rank = 0;
+                for (int j = 0; j < n; ++j) rank += mine[j] < key;
+                v[rank] = key;
             }
-        } else {
+            __syncwarp();
+        } else if (lane == 0) {
             for (int64_t i = n / 2 - 1; i >= 0; --i) sift_down(v, i, n);
             for (int64_t end = n - 1; end > 0; --end) {
                 const int32_t tmp = v[0]; v[0] = v[end]; v[end] = tmp;
@@ -167,7 +179,7 @@ int graph_prepare(int64_t n_nodes, int64_t n_edges, const int32_t* senders, cons
             fill_kernel<<<blocks_for(n_edges, 256), 256, 0, st>>>(n_nodes, n_edges, senders, pad_recv, colptr,
                                                                sender_perm);
             if (int s = after_launch()) return s;
-            sort_buckets_kernel<<<blocks_for(n_nodes, 128), 128, 0, st>>>(n_nodes, colptr, sender_perm);
+            sort_buckets_kernel<<<blocks_for(n_nodes, kSortWarps), 32 * kSortWarps, 0, st>>>(n_nodes, colptr, sender_perm);
             if (int s = after_launch()) return s;
             shift_up_kernel<<<1, 1024, 0, st>>>(n_nodes, colptr);
             if (int s = after_launch()) return s;
