@@ -254,6 +254,8 @@ def main():
                     help="2 = headline workload; 3 / 5 = other convolution workloads; 4 = standalone tensor product rows")
     ap.add_argument("--rows", type=int, default=1 << 20, help="rows of the tensor-product workload (--config 4)")
     ap.add_argument("--generic", action="store_true", help="force the table-driven generic kernels")
+    ap.add_argument("--collapse", action="store_true",
+                    help="plan with collapsed output multiplicities (table-driven kernels; no CPU leg)")
     ap.add_argument("--pad", type=float, default=0.0,
                     help="append this fraction of padding edges and call the padded entry points (rates count real edges)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -294,7 +296,10 @@ def main():
     c, wl = build_workload(args.config)
     t_plan = time.perf_counter()
     plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"],
-                               e3j.E3J_PLAN_GENERIC_ONLY if args.generic else 0)
+                               (e3j.E3J_PLAN_GENERIC_ONLY if args.generic else 0) |
+                               (e3j.E3J_PLAN_COLLAPSE_OUTPUTS if args.collapse else 0))
+    if args.collapse:
+        args.no_cpu_baseline = True
     plan_build_ms = 1e3 * (time.perf_counter() - t_plan)   # host: paths, ladder-operator CG, record tables
     n, e = wl.n_nodes, wl.n_edges
     x, y, w, g = workloads.make_features(wl, plan.n_paths, plan.d_out)
@@ -420,7 +425,7 @@ def main():
             "metric": "conv_fwd_bwd_edges_per_s", "value": e * world / (ms_per_step * 1e-3), "unit": "edges/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "n_nodes": n, "n_edges": e, "padding_edges": n_pad, "irreps_in": c["irreps_in"],
+            "config": {"workload": wl.name, "n_nodes": n, "n_edges": e, "padding_edges": n_pad, "collapsed_outputs": bool(args.collapse), "irreps_in": c["irreps_in"],
                        "sh_lmax": c["sh_lmax"], "n_paths": plan.n_paths, "d_out": plan.d_out,
                        "channels": plan.n_channels, "specialised_kernels": bool(plan.specialised),
                        "l2": "inputs (>1 GB per step) exceed the 126 MB L2; no explicit flush",

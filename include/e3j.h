@@ -69,6 +69,13 @@ enum {
 
 /* plan flags */
 #define E3J_PLAN_GENERIC_ONLY 1u /* never pick a signature-specialised kernel */
+/* Collapsed output multiplicities (paper: the coefficient set used for the comparison with the SO(2)
+ * convolution, which "sums all isomorphic copies of a given irreducible output space together"): all paths
+ * that land on the same (L, p) share one output block, out[b, block(L,p) + M, q] = sum over those paths of
+ * w[e, path, q] * (...), so D = sum over distinct (L, p) of (2L + 1) while the weights stay one block per
+ * path.  out_off of e3j_path_info_t is then the same for the paths of a block.  Such plans run on the
+ * table-driven kernels. */
+#define E3J_PLAN_COLLAPSE_OUTPUTS 2u
 
 typedef struct e3j_plan e3j_plan; /* opaque; immutable after creation; usable from several streams */
 

@@ -158,3 +158,37 @@ def conv_bwd_padded(cp: Coupling, x, y, s, senders, receivers, dm):
     dy = np.zeros((e, cp.dp)); ds = np.zeros((e, cp.P, cp.nq))
     dy[real] = dy_r; ds[real] = ds_r
     return dx, dy, ds
+
+
+# ---------------------------------------------------------------------------------------------
+# Collapsed output multiplicities.  The paper evaluates its kernels also with a coefficient set
+# that "sums all isomorphic copies of a given irreducible output space together": every path
+# that lands on the same (L, parity) adds into one shared output block.  Written out here from
+# the uncollapsed definition: out_c = R out, with R the 0/1 matrix that maps row M of every
+# path's block to row M of the shared block of its (L, parity); the backward is the chain rule
+# through that sum (dm = R^T dm_c).  Blocks are ordered as their first path is.
+def collapse_matrix(cp: Coupling) -> np.ndarray:
+    """(R [D_collapsed, D], block offset of every path)."""
+    block_off, offsets, d_c = {}, [], 0
+    for p in cp.paths:
+        key = (p.L, p.p)
+        if key not in block_off:
+            block_off[key] = d_c
+            d_c += 2 * p.L + 1
+        offsets.append(block_off[key])
+    R = np.zeros((d_c, cp.D))
+    for p, off in zip(cp.paths, offsets):
+        for m in range(2 * p.L + 1):
+            R[off + m, p.out_off + m] = 1.0
+    return R, offsets
+
+
+def conv_fwd_collapsed(cp: Coupling, x, y, s, senders, receivers) -> np.ndarray:
+    R, _ = collapse_matrix(cp)
+    return np.einsum("ci,niq->ncq", R, conv_fwd(cp, x, y, s, senders, receivers))
+
+
+def conv_bwd_collapsed(cp: Coupling, x, y, s, senders, receivers, dm_c):
+    R, _ = collapse_matrix(cp)
+    dm = np.einsum("ci,ncq->niq", R, np.asarray(dm_c, dtype=np.float64)).astype(np.float32)
+    return conv_bwd(cp, x, y, s, senders, receivers, dm)

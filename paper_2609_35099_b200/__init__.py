@@ -26,6 +26,7 @@ __all__ = [
 ]
 
 E3J_PLAN_GENERIC_ONLY = 1
+E3J_PLAN_COLLAPSE_OUTPUTS = 2
 # status codes of include/e3j.h
 E3J_OK, E3J_ERR_INVALID_ARG, E3J_ERR_BAD_IRREPS, E3J_ERR_MUL_NOT_UNIFORM = 0, -1, -2, -3
 E3J_ERR_UNSUPPORTED, E3J_ERR_WORKSPACE, E3J_ERR_CUDA, E3J_ERR_GRAPH = -4, -5, -6, -7

@@ -48,12 +48,13 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
         if (t.device == device) { out = t; return E3J_OK; }
 
     std::vector<PackedRecord> r0, r1, r2;
-    std::vector<int32_t> s0, s1, s2, i0_path(plan->D), path_off(plan->P + 1);
+    std::vector<int32_t> s0, s1, s2, i0_path(plan->D), path_off(plan->P + 1), path_rows(plan->P);
     pack_sorted(plan->rec, plan->D, [](const Record& r) { return r.i0; }, r0, s0, 0);
     pack_sorted(plan->rec, plan->d, [](const Record& r) { return r.i1; }, r1, s1, 1);
     pack_sorted(plan->rec, plan->dp, [](const Record& r) { return r.i2; }, r2, s2, 2);
     for (int k = 0; k < plan->P; ++k) {
         path_off[k] = plan->paths[k].out_off;
+        path_rows[k] = 2 * plan->paths[k].L + 1;
         for (int m = 0; m < 2 * plan->paths[k].L + 1; ++m) i0_path[plan->paths[k].out_off + m] = k;
     }
     path_off[plan->P] = plan->D;
@@ -65,6 +66,7 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
     const size_t o_r0 = reserve(nb), o_r1 = reserve(nb), o_r2 = reserve(nb);
     const size_t o_s0 = reserve(4 * s0.size()), o_s1 = reserve(4 * s1.size()), o_s2 = reserve(4 * s2.size());
     const size_t o_ip = reserve(4 * i0_path.size()), o_po = reserve(4 * path_off.size());
+    const size_t o_pr = reserve(4 * path_rows.size());
     const size_t o_st = reserve(256);
     std::vector<char> host(off, 0);
     std::memcpy(host.data() + o_r0, r0.data(), nb);
@@ -75,6 +77,7 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
     std::memcpy(host.data() + o_s2, s2.data(), 4 * s2.size());
     std::memcpy(host.data() + o_ip, i0_path.data(), 4 * i0_path.size());
     std::memcpy(host.data() + o_po, path_off.data(), 4 * path_off.size());
+    std::memcpy(host.data() + o_pr, path_rows.data(), 4 * path_rows.size());
 
     DeviceTables t;
     t.device = device;
@@ -90,6 +93,7 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
     t.i2_start = (const int32_t*)(b + o_s2);
     t.i0_path = (const int32_t*)(b + o_ip);
     t.path_out_off = (const int32_t*)(b + o_po);
+    t.path_rows = (const int32_t*)(b + o_pr);
     t.status = (int32_t*)(b + o_st);
     plan->dev.push_back(t);
     out = t;
@@ -103,7 +107,9 @@ inline int grid_for(int64_t n) {
     return (int)g;
 }
 
-inline Dims dims_of(const e3j_plan* p) { return Dims{p->nq, p->d, p->dp, p->P, p->D}; }
+inline Dims dims_of(const e3j_plan* p) {
+    return Dims{p->nq, p->d, p->dp, p->P, p->D, (p->flags & E3J_PLAN_COLLAPSE_OUTPUTS) ? 1 : 0};
+}
 
 // workspace layout shared by fwd and bwd: [rowptr | colptr | sender_perm | kernel scratch]
 struct WorkspaceLayout {

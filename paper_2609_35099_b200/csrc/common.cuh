@@ -35,6 +35,7 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out);
 
 struct Dims {
     int nq, d, dp, P, D;
+    int collapsed;  // several paths may share an output row (E3J_PLAN_COLLAPSE_OUTPUTS)
 };
 
 // Scalar description of a graph launch shared by the generic and specialised paths.

@@ -48,6 +48,23 @@ conv_fwd_kernel(DeviceTables t, Dims dm, int64_t n_nodes, const float* __restric
             const int r0 = t.i0_start[i0], r1 = t.i0_start[i0 + 1];
             float4 acc = f4_zero();
             int64_t e = e0;
+            if (dm.collapsed) {
+                // several paths land on this output row: the weight belongs to the record, not to the row
+                for (; e < e1; ++e) {
+                    const int64_t a = IDENT ? e : (int64_t)senders[e];
+                    const float4* xa = x4 + (size_t)a * dm.d * nq4 + q;
+                    const float* ye = sh + (size_t)e * dm.dp;
+                    const float4* we = w4 + (size_t)e * dm.P * nq4 + q;
+                    float4 z = f4_zero();
+                    for (int r = r0; r < r1; ++r) {
+                        const PackedRecord rc = t.by_i0[r];
+                        f4_fma(z, rc.val * ye[rc.b], f4_mul(we[(size_t)rc.c * nq4], xa[(size_t)rc.a * nq4]));
+                    }
+                    acc.x += z.x; acc.y += z.y; acc.z += z.z; acc.w += z.w;
+                }
+                out4[((size_t)b * dm.D + i0) * nq4 + q] = acc;
+                continue;
+            }
             // four edges at a time: their loads are independent and in flight together; the additions stay
             // in edge order
             for (; e + 4 <= e1; e += 4) {
@@ -115,10 +132,12 @@ conv_bwd_edge_kernel(DeviceTables t, Dims dm, int64_t n_edges, const float* __re
             for (int idx = threadIdx.x; idx < dm.P * nq4; idx += blockDim.x) {
                 const int k = idx / nq4, q = idx - k * nq4;
                 float4 sum = f4_zero();
-                for (int i0 = t.path_out_off[k]; i0 < t.path_out_off[k + 1]; ++i0) {
+                const int row0 = t.path_out_off[k];
+                for (int i0 = row0; i0 < row0 + t.path_rows[k]; ++i0) {
                     float4 z = f4_zero();
                     for (int r = t.i0_start[i0]; r < t.i0_start[i0 + 1]; ++r) {
                         const PackedRecord rc = t.by_i0[r];
+                        if (rc.c != k) continue;  // (a collapsed plan has other paths' records on this row)
                         f4_fma(z, rc.val * ye[rc.b], xa[(size_t)rc.a * nq4 + q]);
                     }
                     f4_fma(sum, gb[(size_t)i0 * nq4 + q], z);

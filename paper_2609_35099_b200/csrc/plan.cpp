@@ -231,9 +231,14 @@ int build_plan(e3j_plan& plan, const char* irreps_in, int sh_lmax, const char* i
     plan.flags = flags;
     plan.paths.clear();
     plan.rec.clear();
-    int out_off = 0;
+    // Output blocks: one per path, or (E3J_PLAN_COLLAPSE_OUTPUTS) one per distinct (L, p), shared by all
+    // the paths that land on it.  The paths are sorted by output irrep, so those paths are neighbours.
+    const bool collapse = (flags & E3J_PLAN_COLLAPSE_OUTPUTS) != 0;
+    int out_off = 0, next_off = 0;
     for (int k = 0; k < plan.P; ++k) {
         const Raw& r = raw[k];
+        const bool same_block = collapse && k > 0 && raw[k - 1].L == r.L && raw[k - 1].p == r.p;
+        if (!same_block) out_off = next_off;
         e3j_path_info_t pi{r.in_index, r.l1, r.p1, r.l2, r.L, r.p, r.x_off, r.l2 * r.l2, out_off};
         plan.paths.push_back(pi);
         const std::vector<double> T = real_cg_ladder(r.l1, r.l2, r.L);
@@ -244,18 +249,20 @@ int build_plan(e3j_plan& plan, const char* irreps_in, int sh_lmax, const char* i
                     const double v = T[((size_t)M * n1 + a) * n2 + b];
                     if (v != 0.0) plan.rec.push_back({out_off + M, r.x_off + a, pi.y_off + b, k, v});
                 }
-        out_off += nL;
+        if (!same_block) next_off = out_off + nL;
     }
-    plan.D = out_off;
+    plan.D = next_off;
     if (plan.D > 255 || plan.d > 255 || plan.dp > 255 || plan.P > 255) return E3J_ERR_UNSUPPORTED;
     std::sort(plan.rec.begin(), plan.rec.end(), [](const Record& a, const Record& b) {
         if (a.i0 != b.i0) return a.i0 < b.i0;
+        if (a.i3 != b.i3) return a.i3 < b.i3;   // (only collapsed plans have several paths per output row)
         if (a.i1 != b.i1) return a.i1 < b.i1;
         return a.i2 < b.i2;
     });
     plan.n_pairs = 0;
     for (size_t i = 0; i < plan.rec.size(); ++i)
-        if (i == 0 || plan.rec[i].i0 != plan.rec[i - 1].i0 || plan.rec[i].i1 != plan.rec[i - 1].i1)
+        if (i == 0 || plan.rec[i].i0 != plan.rec[i - 1].i0 || plan.rec[i].i1 != plan.rec[i - 1].i1 ||
+            plan.rec[i].i3 != plan.rec[i - 1].i3)
             ++plan.n_pairs;
 
     // canonical signature: multiplicity, input irreps, harmonic degree, output blocks
@@ -267,6 +274,7 @@ int build_plan(e3j_plan& plan, const char* irreps_in, int sh_lmax, const char* i
         const e3j_path_info_t& p = plan.paths[k];
         sig << (k ? "," : "") << p.in_index << ":" << p.l2 << ":" << p.L;
     }
+    if (collapse) sig << "|collapsed";
     plan.signature = sig.str();
     return E3J_OK;
 }

@@ -36,7 +36,8 @@ struct DeviceTables {
     // sorted by i2: (a,b,c) = (i0,i1,path)
     const PackedRecord* by_i2 = nullptr;
     const int32_t* i2_start = nullptr;  // [d'+1]
-    const int32_t* path_out_off = nullptr;  // [P+1]
+    const int32_t* path_out_off = nullptr;  // [P+1] first output row of every path (last entry: D)
+    const int32_t* path_rows = nullptr;     // [P] rows of every path, 2L+1
     int32_t* status = nullptr;  // sticky device status word (0 = fine), see e3j_plan_device_status
 };
 
@@ -46,7 +47,7 @@ struct e3j_plan {
     int nq = 0, d = 0, dp = 0, P = 0, D = 0, n_pairs = 0;
     unsigned flags = 0;
     std::vector<e3j_path_info_t> paths;
-    std::vector<e3j::Record> rec;  // sorted by (i0,i1,i2)
+    std::vector<e3j::Record> rec;  // sorted by (i0,i3,i1,i2)
     std::string signature;         // canonical text of (irreps_in | sh_lmax | output blocks)
     int fast_id = -1;              // index into the specialised-kernel registry, or -1
     mutable std::mutex mu;

@@ -268,6 +268,32 @@ def test_channel_counts_must_be_multiples_of_four():
     assert err.value.status == e3j.E3J_ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("config,n_atoms", [(1, None), (2, 192), (3, 200)])
+def test_collapsed_output_multiplicities(config, n_atoms):
+    """Plans with E3J_PLAN_COLLAPSE_OUTPUTS: paths landing on one (L, parity) share an output block."""
+    c = workloads.CONFIGS[config]
+    wl = workloads.make_graph(config, n_atoms)
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"],
+                               e3j.E3J_PLAN_COLLAPSE_OUTPUTS)
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"])
+    R, offs = oconv.collapse_matrix(cp)
+    assert plan.d_out == R.shape[0] < cp.D
+    x, y, w, _ = workloads.make_features(wl, plan.n_paths, plan.d_out)
+    g = np.random.default_rng(9).standard_normal((wl.n_nodes, plan.d_out, plan.n_channels)).astype(np.float32)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    rowptr, perm, colptr = e3j.e3j_graph_prepare(wl.n_nodes, snd, rcv)
+    out = e3j.e3j_conv_fwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, rowptr)
+    gx, gy, gw = e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, _cuda(g), rowptr, perm, colptr)
+    torch.cuda.synchronize()
+    ref = oconv.conv_fwd_collapsed(cp, x, y, w, wl.senders, wl.receivers)
+    rx, ry, rw = oconv.conv_bwd_collapsed(cp, x, y, w, wl.senders, wl.receivers, g)
+    blocks = sorted({(off, off + 2 * p.L + 1) for p, off in zip(cp.paths, offs)})
+    assert_blockwise_close(out.cpu().numpy(), ref, blocks, what="out")
+    assert_blockwise_close(gx.cpu().numpy(), rx, blocks_of_paths(cp.paths, "x"), what="grad_x")
+    assert_blockwise_close(gy.cpu().numpy(), ry, blocks_of_paths(cp.paths, "sh"), what="grad_sh")
+    assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="grad_w")
+
+
 def test_optional_gradients_can_be_skipped():
     wl, plan, cp, x, y, w, g = make_case(1)
     snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)

@@ -224,3 +224,37 @@ def test_padding_edges_take_no_part():
     # nothing but padding: zero output, zero gradients
     out0 = conv.conv_fwd_padded(cp, x, yp[e:], sp[e:], sndp[e:], rcvp[e:])
     assert out0.shape == ref.shape and np.all(out0 == 0)
+
+
+def test_collapsed_outputs_against_a_direct_sum_over_paths():
+    """Collapsed multiplicities: paths landing on the same (L, parity) add into one block.  Checked against
+    the sum written path by path (one dense contraction per path, added into the block of its irrep), against
+    the uncollapsed result when no two paths share an irrep, and through the adjoint identity."""
+    rng = np.random.default_rng(21)
+    cp = conv.Coupling("2x0e+2x1o", 2)
+    n, e = 5, 9
+    snd = rng.integers(0, n, e).astype(np.int32); rcv = np.sort(rng.integers(0, n, e)).astype(np.int32)
+    x, y, s = _random_inputs(rng, cp, n, e)
+    R, offs = conv.collapse_matrix(cp)
+    keys = sorted({(p.L, p.p) for p in cp.paths})
+    assert R.shape == (sum(2 * L + 1 for L, _ in keys), cp.D) and len(keys) < cp.P
+    got = conv.conv_fwd_collapsed(cp, x, y, s, snd, rcv)
+    want = np.zeros_like(got)
+    x64, y64, s64 = x.astype(np.float64), y.astype(np.float64), s.astype(np.float64)
+    for p, off in zip(cp.paths, offs):
+        Ck = cp.C[p.out_off:p.out_off + 2 * p.L + 1]          # [2L+1, d, d'] of this path alone
+        for ed in range(e):
+            m = np.einsum("mij,iq,j->mq", Ck, x64[snd[ed]], y64[ed]) * s64[ed, p.k][None, :]
+            want[rcv[ed], off:off + 2 * p.L + 1] += m
+    assert np.abs(got - want).max() < 1e-12
+    # adjoint identity through the collapsed map
+    dm = rng.standard_normal(got.shape).astype(np.float32)
+    dx, dy, ds = conv.conv_bwd_collapsed(cp, x, y, s, snd, rcv, dm)
+    lhs = float((dm.astype(np.float64) * got).sum())
+    assert abs(lhs - float((dx * x64).sum())) < 1e-10 * abs(lhs)
+    assert abs(lhs - float((dy * y64).sum())) < 1e-10 * abs(lhs)
+    assert abs(lhs - float((ds * s64).sum())) < 1e-10 * abs(lhs)
+    # one path per irrep: nothing to collapse
+    cp1 = conv.Coupling("2x0e", 2)
+    R1, _ = conv.collapse_matrix(cp1)
+    assert np.array_equal(R1, np.eye(cp1.D))

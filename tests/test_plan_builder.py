@@ -109,3 +109,25 @@ def test_compute_calls_fail_loudly_without_a_device():
     dummy = ctypes.c_void_p(256)
     st = lib.e3j_tp_fwd(plan.handle, 1, dummy, dummy, dummy, dummy, None)
     assert st == -6
+
+
+@pytest.mark.parametrize("sig", [("8x0e+8x1o", 2, "0e+1o+1e+2e+2o", -1), ("128x0e+128x1o", 3, None, 3),
+                                 ("64x0e+64x1o+64x2e+64x3o", 3, None, 3)])
+def test_collapsed_plan_tables(sig):
+    """E3J_PLAN_COLLAPSE_OUTPUTS: same paths, records and weights, output rows shared per (L, parity)."""
+    from oracle import conv as oconv
+    irreps_in, lmax, irreps_out, out_lmax = sig
+    full = e3j.e3j_plan_create(irreps_in, lmax, irreps_out, out_lmax)
+    plan = e3j.e3j_plan_create(irreps_in, lmax, irreps_out, out_lmax, e3j.E3J_PLAN_COLLAPSE_OUTPUTS)
+    cp = oconv.Coupling(irreps_in, lmax, irreps_out, None if out_lmax < 0 else out_lmax)
+    R, offs = oconv.collapse_matrix(cp)
+    assert not plan.specialised and plan.n_paths == full.n_paths and plan.d_out == R.shape[0]
+    assert [p["out_off"] for p in e3j.e3j_plan_paths(plan)] == offs
+    i0, i1, i2, k, val = e3j.e3j_plan_records(plan)
+    dense = np.zeros((R.shape[0], cp.d, cp.dp, cp.P))
+    dense[i0, i1, i2, k] = val
+    want = np.zeros_like(dense)
+    for p, off in zip(cp.paths, offs):
+        want[off:off + 2 * p.L + 1, :, :, p.k] = cp.C[p.out_off:p.out_off + 2 * p.L + 1]
+    assert np.abs(dense - want).max() < 1e-13
+    assert e3j.e3j_plan_signature(plan) != e3j.e3j_plan_signature(full)
