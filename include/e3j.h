@@ -222,6 +222,26 @@ int e3j_conv_bwd_padded(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges_p
                         const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
                         float* grad_w, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Double backward (paper: "Differentiation", the double-backward rule needed when the loss contains
+ * forces, i.e. gradients of the first backward).  The backward maps (x, sh, w, grad_out) to
+ * (grad_x, grad_sh, grad_w).  Given cotangents ct_x, ct_sh, ct_w of those three results (shapes of
+ * x, sh, w; any may be NULL = zero) this call returns the cotangents of the backward's four inputs:
+ *   gg_out = F(ct_x, sh, w) + F(x, ct_sh, w) + F(x, sh, ct_w)            [n_nodes,D,N_q]   (F = forward map)
+ *   g_x    = grad_x of the backward taken at (sh <- ct_sh)  +  at (w <- ct_w)              [n_nodes,d,N_q]
+ *   g_sh   = grad_sh at (x <- ct_x)  +  at (w <- ct_w)                                      [n_edges,d']
+ *   g_w    = grad_w at (x <- ct_x)   +  at (sh <- ct_sh)                                    [n_edges,P,N_q]
+ * all with the same grad_out; any output may be NULL.  This is the composition the paper describes (three
+ * forward and three backward passes of this library plus the sums); the single fused sweep the paper leaves
+ * as future work is not built.  rowptr, sender_perm and colptr are required (e3j_graph_prepare); the
+ * workspace (e3j_conv_bwd_bwd_workspace_bytes) also holds one scratch tensor of each output's size. */
+size_t e3j_conv_bwd_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges);
+int e3j_conv_bwd_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                     const float* sh, const float* w, const int32_t* senders,
+                     const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                     const int32_t* colptr, const float* grad_out, const float* ct_x,
+                     const float* ct_sh, const float* ct_w, float* gg_out, float* g_x, float* g_sh,
+                     float* g_w, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Standalone channelwise tensor product with per-row, per-path weights (paper:
  * tensor-product formula followed by the edge-scalar weighting; backward: the
  * tensor-product backward rule, one streaming pass).  Rows are their own receivers:

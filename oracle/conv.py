@@ -192,3 +192,18 @@ def conv_bwd_collapsed(cp: Coupling, x, y, s, senders, receivers, dm_c):
     R, _ = collapse_matrix(cp)
     dm = np.einsum("ci,ncq->niq", R, np.asarray(dm_c, dtype=np.float64)).astype(np.float32)
     return conv_bwd(cp, x, y, s, senders, receivers, dm)
+
+
+# ---------------------------------------------------------------------------------------------
+# Double backward (paper, "Differentiation", message-passing double backward): with (ux, uy, us) the
+# cotangents of the backward's results (dx, dy, ds), the cotangents of the backward's inputs are
+#   d(dm) = conv(ux, y, s) + conv(x, uy, s) + conv(x, y, us)
+#   dx = dx[conv_bwd(x, uy, s, dm)] + dx[conv_bwd(x, y, us, dm)]         and cyclically for y and s.
+def conv_bwd_bwd(cp: Coupling, x, y, s, senders, receivers, dm, ux, uy, us):
+    """(g_dm, g_x, g_y, g_s) in float64."""
+    g_dm = (conv_fwd(cp, ux, y, s, senders, receivers) + conv_fwd(cp, x, uy, s, senders, receivers) +
+            conv_fwd(cp, x, y, us, senders, receivers))
+    _, y_from_x, s_from_x = conv_bwd(cp, ux, y, s, senders, receivers, dm)
+    x_from_y, _, s_from_y = conv_bwd(cp, x, uy, s, senders, receivers, dm)
+    x_from_s, y_from_s, _ = conv_bwd(cp, x, y, us, senders, receivers, dm)
+    return g_dm, x_from_y + x_from_s, y_from_x + y_from_s, s_from_x + s_from_y

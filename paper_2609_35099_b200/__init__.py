@@ -91,6 +91,9 @@ def _load():
     lib.e3j_conv_fwd.argtypes = [vp, i64, i64] + [vp] * 8 + [sz, vp]
     lib.e3j_conv_bwd.argtypes = [vp, i64, i64] + [vp] * 13 + [sz, vp]
     lib.e3j_conv_fwd_padded.argtypes = [vp, i64, i64] + [vp] * 8 + [sz, vp]
+    lib.e3j_conv_bwd_bwd_workspace_bytes.argtypes = [vp, i64, i64]
+    lib.e3j_conv_bwd_bwd_workspace_bytes.restype = sz
+    lib.e3j_conv_bwd_bwd.argtypes = [vp, i64, i64] + [vp] * 17 + [sz, vp]
     lib.e3j_conv_bwd_padded.argtypes = [vp, i64, i64] + [vp] * 13 + [sz, vp]
     lib.e3j_conv_fwd_noalloc.argtypes = [vp, i64, i64] + [vp] * 7
     lib.e3j_conv_fwd_noalloc.restype = i32
@@ -344,6 +347,41 @@ def e3j_conv_bwd_padded(plan: Plan, x, sh, w, senders, receivers, grad_out, rowp
     The grad_sh / grad_w rows of padding edges come back as zeros."""
     return e3j_conv_bwd(plan, x, sh, w, senders, receivers, grad_out, rowptr, sender_perm, colptr, grad_x,
                         grad_sh, grad_w, workspace, stream, "e3j_conv_bwd_padded")
+
+
+def e3j_conv_bwd_bwd_workspace_bytes(plan: Plan, n_nodes: int, n_edges: int) -> int:
+    return int(_load().e3j_conv_bwd_bwd_workspace_bytes(plan.handle, n_nodes, n_edges))
+
+
+def e3j_conv_bwd_bwd(plan: Plan, x, sh, w, senders, receivers, grad_out, rowptr, sender_perm, colptr,
+                     ct_x=None, ct_sh=None, ct_w=None, gg_out=True, g_x=True, g_sh=True, g_w=True,
+                     workspace=None, stream=None):
+    """Double backward: cotangents (ct_x, ct_sh, ct_w) of the backward's results -> cotangents
+    (gg_out, g_x, g_sh, g_w) of the backward's inputs (grad_out, x, sh, w).  A missing ct_* is zero; each
+    output argument is True (allocate), False/None (not wanted) or a preallocated tensor."""
+    torch = _torch()
+    n, e = x.shape[0], senders.numel()
+    f32, i32 = torch.float32, torch.int32
+
+    def alloc(flag, shape):
+        if flag is True:
+            return torch.empty(shape, dtype=f32, device=x.device)
+        return flag if isinstance(flag, torch.Tensor) else None
+
+    s_x, s_sh = (n, plan.d_in, plan.n_channels), (e, plan.d_sh)
+    s_w, s_out = (e, plan.n_paths, plan.n_channels), (n, plan.d_out, plan.n_channels)
+    gg_out, g_x, g_sh, g_w = alloc(gg_out, s_out), alloc(g_x, s_x), alloc(g_sh, s_sh), alloc(g_w, s_w)
+    workspace = _workspace(e3j_conv_bwd_bwd_workspace_bytes(plan, n, e), x, workspace)
+    _check(_load().e3j_conv_bwd_bwd(
+        plan.handle, n, e, _dev_ptr(x, f32, s_x, "x"), _dev_ptr(sh, f32, s_sh, "sh"), _dev_ptr(w, f32, s_w, "w"),
+        _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
+        _dev_ptr(rowptr, i32, (n + 1,), "rowptr"), _dev_ptr(sender_perm, i32, (e,), "sender_perm"),
+        _dev_ptr(colptr, i32, (n + 1,), "colptr"), _dev_ptr(grad_out, f32, s_out, "grad_out"),
+        _dev_ptr(ct_x, f32, s_x, "ct_x"), _dev_ptr(ct_sh, f32, s_sh, "ct_sh"), _dev_ptr(ct_w, f32, s_w, "ct_w"),
+        _dev_ptr(gg_out, f32, s_out, "gg_out"), _dev_ptr(g_x, f32, s_x, "g_x"), _dev_ptr(g_sh, f32, s_sh, "g_sh"),
+        _dev_ptr(g_w, f32, s_w, "g_w"),
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_bwd_bwd")
+    return gg_out, g_x, g_sh, g_w
 
 
 def e3j_tp_fwd(plan: Plan, x1, x2, w, out=None, stream=None):

@@ -129,6 +129,46 @@ WorkspaceLayout layout(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, b
     return L;
 }
 
+// dst[i] += src[i]
+__global__ void add_into_kernel(int64_t n, float* __restrict__ dst, const float* __restrict__ src, int vec_ok) {
+    const int64_t tid = blockIdx.x * (int64_t)blockDim.x + threadIdx.x, stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t n4 = vec_ok ? n / 4 : 0;
+    float4* d4 = reinterpret_cast<float4*>(dst);
+    const float4* s4 = reinterpret_cast<const float4*>(src);
+    for (int64_t i = tid; i < n4; i += stride) {
+        float4 a = d4[i];
+        const float4 b = s4[i];
+        a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        d4[i] = a;
+    }
+    for (int64_t i = 4 * n4 + tid; i < n; i += stride) dst[i] += src[i];
+}
+int add_into(float* dst, const float* src, size_t n, cudaStream_t st) {
+    if (n == 0) return E3J_OK;
+    const int vec_ok = (((uintptr_t)dst | (uintptr_t)src) & 15u) == 0;
+    add_into_kernel<<<148 * 16, 256, 0, st>>>((int64_t)n, dst, src, vec_ok);
+    return after_launch();
+}
+
+// workspace of the double backward: [forward ws | backward ws | out-sized | x-sized | sh-sized | w-sized]
+struct DoubleBwdLayout {
+    size_t fwd, bwd, t_out, t_x, t_sh, t_w, total, fwd_bytes, bwd_bytes;
+};
+DoubleBwdLayout dbl_layout(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges) {
+    DoubleBwdLayout L{};
+    L.fwd_bytes = layout(plan, n_nodes, n_edges, false).total;
+    L.bwd_bytes = layout(plan, n_nodes, n_edges, true).total;
+    size_t off = 0;
+    L.fwd = off; off = align_up(off + L.fwd_bytes, 256);
+    L.bwd = off; off = align_up(off + L.bwd_bytes, 256);
+    L.t_out = off; off = align_up(off + 4 * (size_t)n_nodes * plan->D * plan->nq, 256);
+    L.t_x = off; off = align_up(off + 4 * (size_t)n_nodes * plan->d * plan->nq, 256);
+    L.t_sh = off; off = align_up(off + 4 * (size_t)n_edges * ((plan->dp + 3) / 4 * 4), 256);
+    L.t_w = off; off = align_up(off + 4 * (size_t)n_edges * plan->P * plan->nq, 256);
+    L.total = off;
+    return L;
+}
+
 int check_workspace(const void* ws, size_t have, size_t need) {
     if (need == 0) return E3J_OK;
     if (!ws || ((uintptr_t)ws & 255u) || have < need) return E3J_ERR_WORKSPACE;
@@ -377,6 +417,93 @@ int e3j_conv_bwd_padded(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges_p
                         float* grad_w, void* workspace, size_t workspace_bytes, void* stream) {
     return conv_bwd_impl(plan, n_nodes, n_edges_padded, x, sh, w, senders, receivers, rowptr, sender_perm,
                          colptr, grad_out, grad_x, grad_sh, grad_w, workspace, workspace_bytes, stream, true);
+}
+
+size_t e3j_conv_bwd_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges) {
+    if (!plan || n_nodes < 0 || n_edges < 0) return 0;
+    return dbl_layout(plan, n_nodes, n_edges).total;
+}
+
+int e3j_conv_bwd_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                     const float* sh, const float* w, const int32_t* senders,
+                     const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                     const int32_t* colptr, const float* grad_out, const float* ct_x,
+                     const float* ct_sh, const float* ct_w, float* gg_out, float* g_x, float* g_sh,
+                     float* g_w, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!plan || n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
+        return E3J_ERR_INVALID_ARG;
+    if (plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;
+    if (n_nodes == 0) return E3J_OK;
+    if (!x || !grad_out) return E3J_ERR_INVALID_ARG;
+    if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    if (!rowptr || !sender_perm || !colptr) return E3J_ERR_INVALID_ARG;  // six passes: prepare the graph once
+    cudaStream_t st = (cudaStream_t)stream;
+    const DoubleBwdLayout L = dbl_layout(plan, n_nodes, n_edges);
+    if (int s = check_workspace(workspace, workspace_bytes, L.total)) return s;
+    char* ws = (char*)workspace;
+    float* t_out = (float*)(ws + L.t_out);
+    float* t_x = (float*)(ws + L.t_x);
+    float* t_sh = (float*)(ws + L.t_sh);
+    float* t_w = (float*)(ws + L.t_w);
+    const size_t n_out = (size_t)n_nodes * plan->D * plan->nq, n_x = (size_t)n_nodes * plan->d * plan->nq;
+    const size_t n_sh = (size_t)n_edges * plan->dp, n_w = (size_t)n_edges * plan->P * plan->nq;
+
+    // cotangent of grad_out: the forward map with one argument replaced by its cotangent, three times
+    if (gg_out) {
+        bool first = true;
+        const float* xs[3] = {ct_x, x, x};
+        const float* ys[3] = {sh, ct_sh, sh};
+        const float* wsrc[3] = {w, w, ct_w};
+        const float* cts[3] = {ct_x, ct_sh, ct_w};
+        for (int term = 0; term < 3; ++term) {
+            if (!cts[term]) continue;
+            float* dst = first ? gg_out : t_out;
+            if (int s = conv_fwd_impl(plan, n_nodes, n_edges, xs[term], ys[term], wsrc[term], senders, receivers,
+                                      rowptr, dst, ws + L.fwd, L.fwd_bytes, stream, false)) return s;
+            if (!first)
+                if (int s = add_into(gg_out, t_out, n_out, st)) return s;
+            first = false;
+        }
+        if (first) E3J_CUDA_TRY(cudaMemsetAsync(gg_out, 0, 4 * n_out, st));
+    }
+    // cotangents of x, sh, w: the backward map with one primal replaced by its cotangent; each pass yields the
+    // two cotangents that are not the replaced argument's own (all three are computed so that the specialised
+    // sweep can be used; the third goes to scratch)
+    bool have_x = false, have_sh = false, have_w = false;
+    auto put = [&](float* dst, float* tmp, bool& have, size_t n) -> int {
+        // result of this pass is in `have ? tmp : dst`; fold it into dst
+        if (!dst) return E3J_OK;
+        if (have) return add_into(dst, tmp, n, st);
+        have = true;
+        return E3J_OK;
+    };
+    if ((g_sh || g_w) && ct_x) {   // x <- ct_x: contributes to sh and w
+        float* o_sh = g_sh ? g_sh : t_sh;
+        float* o_w = g_w ? g_w : t_w;
+        if (int s = conv_bwd_impl(plan, n_nodes, n_edges, ct_x, sh, w, senders, receivers, rowptr, sender_perm, colptr,
+                                  grad_out, t_x, o_sh, o_w, ws + L.bwd, L.bwd_bytes, stream, false)) return s;
+        have_sh = g_sh != nullptr; have_w = g_w != nullptr;
+    }
+    if ((g_x || g_w) && ct_sh) {   // sh <- ct_sh: contributes to x and w
+        float* o_x = g_x ? g_x : t_x;
+        float* o_w = (g_w && !have_w) ? g_w : t_w;
+        if (int s = conv_bwd_impl(plan, n_nodes, n_edges, x, ct_sh, w, senders, receivers, rowptr, sender_perm, colptr,
+                                  grad_out, o_x, t_sh, o_w, ws + L.bwd, L.bwd_bytes, stream, false)) return s;
+        have_x = g_x != nullptr;
+        if (int s = put(g_w, t_w, have_w, n_w)) return s;
+    }
+    if ((g_x || g_sh) && ct_w) {   // w <- ct_w: contributes to x and sh
+        float* o_x = (g_x && !have_x) ? g_x : t_x;
+        float* o_sh = (g_sh && !have_sh) ? g_sh : t_sh;
+        if (int s = conv_bwd_impl(plan, n_nodes, n_edges, x, sh, ct_w, senders, receivers, rowptr, sender_perm, colptr,
+                                  grad_out, o_x, o_sh, t_w, ws + L.bwd, L.bwd_bytes, stream, false)) return s;
+        if (int s = put(g_x, t_x, have_x, n_x)) return s;
+        if (int s = put(g_sh, t_sh, have_sh, n_sh)) return s;
+    }
+    if (g_x && !have_x) E3J_CUDA_TRY(cudaMemsetAsync(g_x, 0, 4 * n_x, st));
+    if (g_sh && !have_sh) E3J_CUDA_TRY(cudaMemsetAsync(g_sh, 0, 4 * n_sh, st));
+    if (g_w && !have_w) E3J_CUDA_TRY(cudaMemsetAsync(g_w, 0, 4 * n_w, st));
+    return E3J_OK;
 }
 
 int e3j_tp_fwd(const e3j_plan* plan, int64_t rows, const float* x1, const float* x2,

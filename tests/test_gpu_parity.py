@@ -294,6 +294,43 @@ def test_collapsed_output_multiplicities(config, n_atoms):
     assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="grad_w")
 
 
+@pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
+@pytest.mark.parametrize("config,n_atoms", [(1, None), (2, 192)])
+def test_double_backward(config, n_atoms, flags):
+    """Cotangents of the backward's inputs against the oracle; a missing cotangent is zero; outputs that are
+    not wanted are skipped; two runs give the same bits."""
+    wl, plan, cp, x, y, w, g = make_case(config, n_atoms, flags=flags)
+    n, e = wl.n_nodes, wl.n_edges
+    rng = np.random.default_rng(77)
+    ux = rng.standard_normal(x.shape).astype(np.float32)
+    uy = rng.standard_normal(y.shape).astype(np.float32)
+    uw = rng.standard_normal(w.shape).astype(np.float32)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    rowptr, perm, colptr = e3j.e3j_graph_prepare(n, snd, rcv)
+    dev = [_cuda(a) for a in (x, y, w)]
+    run = lambda cx, cy, cw, **kw: e3j.e3j_conv_bwd_bwd(plan, dev[0], dev[1], dev[2], snd, rcv, _cuda(g), rowptr, perm,
+                                                        colptr, cx, cy, cw, **kw)
+    got = run(_cuda(ux), _cuda(uy), _cuda(uw))
+    again = run(_cuda(ux), _cuda(uy), _cuda(uw))
+    torch.cuda.synchronize()
+    for a, b in zip(got, again):
+        assert torch.equal(a, b)
+    ref = oconv.conv_bwd_bwd(cp, x, y, w, wl.senders, wl.receivers, g, ux, uy, uw)
+    kinds = ("out", "x", "sh", "w")
+    for a, r, kind in zip(got, ref, kinds):
+        assert_blockwise_close(a.cpu().numpy(), r, blocks_of_paths(cp.paths, kind), what="double backward " + kind)
+    # only the harmonics' cotangent given, only two outputs wanted
+    gg, gx, gsh, gw = run(None, _cuda(uy), None, g_sh=False, g_w=None)
+    assert gsh is None and gw is None
+    zero_x, zero_w = np.zeros_like(x), np.zeros_like(w)
+    ref1 = oconv.conv_bwd_bwd(cp, x, y, w, wl.senders, wl.receivers, g, zero_x, uy, zero_w)
+    assert_blockwise_close(gg.cpu().numpy(), ref1[0], blocks_of_paths(cp.paths, "out"), what="gg_out (ct_sh only)")
+    assert_blockwise_close(gx.cpu().numpy(), ref1[1], blocks_of_paths(cp.paths, "x"), what="g_x (ct_sh only)")
+    # no cotangent at all: zeros
+    for t in run(None, None, None):
+        assert torch.count_nonzero(t) == 0
+
+
 def test_optional_gradients_can_be_skipped():
     wl, plan, cp, x, y, w, g = make_case(1)
     snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)

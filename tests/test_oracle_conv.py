@@ -258,3 +258,36 @@ def test_collapsed_outputs_against_a_direct_sum_over_paths():
     cp1 = conv.Coupling("2x0e", 2)
     R1, _ = conv.collapse_matrix(cp1)
     assert np.array_equal(R1, np.eye(cp1.D))
+
+
+def test_double_backward_is_the_derivative_of_the_backward():
+    """Phi = <ux, dx> + <uy, dy> + <us, ds> with (dx, dy, ds) = conv_bwd(x, y, s, dm) is linear in each of
+    x, y, s, dm, so central differences of Phi give its gradient up to rounding; the double backward must
+    return exactly that gradient."""
+    rng = np.random.default_rng(31)
+    cp = conv.Coupling("2x0e+2x1o", 2)
+    n, e = 4, 7
+    snd = rng.integers(0, n, e).astype(np.int32); rcv = np.sort(rng.integers(0, n, e)).astype(np.int32)
+    x, y, s = _random_inputs(rng, cp, n, e)
+    dm = rng.standard_normal((n, cp.D, cp.nq)).astype(np.float32)
+    ux, uy, us = _random_inputs(rng, cp, n, e)
+    # inputs on a binary grid, so that adding the step is exact in float32 (the oracle takes float32 inputs)
+    x, y, s, dm = [np.round(a * 256.0) / 256.0 for a in (x, y, s, dm)]
+    x, y, s, dm = [a.astype(np.float32) for a in (x, y, s, dm)]
+    got = conv.conv_bwd_bwd(cp, x, y, s, snd, rcv, dm, ux, uy, us)
+
+    def phi(x_, y_, s_, dm_):
+        dx, dy, ds = conv.conv_bwd(cp, x_, y_, s_, snd, rcv, dm_)
+        return float((ux * dx).sum() + (uy * dy).sum() + (us * ds).sum())
+
+    args = [x, y, s, dm]
+    h = 0.25   # exactly representable; Phi is linear in every argument
+    for which, grad in zip((3, 0, 1, 2), got):
+        base = args[which]
+        flat_idx = rng.choice(base.size, size=min(12, base.size), replace=False)
+        for fi in flat_idx:
+            idx = np.unravel_index(fi, base.shape)
+            plus = [a.copy() for a in args]; minus = [a.copy() for a in args]
+            plus[which][idx] += h; minus[which][idx] -= h
+            fd = (phi(*plus) - phi(*minus)) / (2 * h)
+            assert abs(fd - grad[idx]) <= 1e-9 * max(1.0, abs(fd)), (which, idx, fd, grad[idx])
