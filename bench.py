@@ -49,8 +49,8 @@ def measured_peak():
 # profiles/fast_fwd_kernel_water3000.txt, profiles/fast_bwd_kernel_water3000.txt and the launch-list run
 # (specialised kernels, workload water3000).  Other workloads / the generic kernels report null.
 NCU_TRAFFIC = {
-    ("water3000", "fwd"): 1.109178e9 + 0.082058e9 + 0.016342e9,          # fast_fwd_kernel + fwd_fixup_kernel
-    ("water3000", "bwd"): 1.259555e9 + 1.361636e9 + 0.330508e9 + 0.0017e9,  # fast_bwd_kernel + bwd_dx_reduce_kernel
+    ("water3000", "fwd"): 1.110542e9 + 0.081376e9 + 0.016343e9,          # fast_fwd_kernel + fwd_fixup_kernel
+    ("water3000", "bwd"): 1.261115e9 + 1.362131e9 + 0.330463e9 + 0.0018e9,  # fast_bwd_kernel + bwd_dx_reduce_kernel
 }
 
 
