@@ -118,7 +118,9 @@ class Sig:
     # ---------------------------------------------------------------- backward
     def bwd_layout(self):
         """Groups of whole paths (any subset, not only contiguous ones), balanced by estimated
-        instruction count: longest-processing-time assignment, paths inside a group in path order."""
+        instruction count: longest-processing-time assignment, paths inside a group in path order.
+        Optional signature keys: B_SLACK_PCT (how far above the best balance a smaller row cap may be,
+        default 3) and B_CAPS (how many row caps are tried, default 6)."""
         BW = self.cfg["BW"]
         V = self.cfg.get("BV", self.V)
         costs = []
