@@ -24,8 +24,9 @@ sys.path.insert(0, str(HERE.parent.parent))
 
 def load_records(sig):
     import paper_2609_35099_b200 as e3j
+    flags = e3j.E3J_PLAN_GENERIC_ONLY | (e3j.E3J_PLAN_COLLAPSE_OUTPUTS if sig.get("collapse") else 0)
     plan = e3j.e3j_plan_create(sig["irreps_in"], sig["sh_lmax"], sig.get("irreps_out"),
-                               sig.get("out_lmax", -1), e3j.E3J_PLAN_GENERIC_ONLY)
+                               sig.get("out_lmax", -1), flags)
     info = e3j.e3j_plan_info(plan)
     paths = e3j.e3j_plan_paths(plan)
     i0, i1, i2, i3, val = e3j.e3j_plan_records(plan)
@@ -78,31 +79,38 @@ class Sig:
         self.P, self.D, self.NNZ = self.info["n_paths"], self.info["d_out"], self.info["nnz"]
         self.V = sig["V"]
         assert self.NQ % (32 * self.V) == 0, "channels must fill whole warps"
-        # pairs in (i0, i1) order with their records
+        # pairs in (i0, path, i1) order with their records (a collapsed plan has several paths per output row)
         self.pairs = []  # (i0, i1, k, [(i2, val)])
         for i0, i1, i2, k, v in self.recs:
-            if self.pairs and self.pairs[-1][0] == i0 and self.pairs[-1][1] == i1:
+            if self.pairs and self.pairs[-1][0] == i0 and self.pairs[-1][1] == i1 and self.pairs[-1][2] == k:
                 self.pairs[-1][3].append((i2, v))
             else:
                 self.pairs.append((i0, i1, k, [(i2, v)]))
         assert len(self.pairs) == self.info["n_pairs"]
-        self.row_path = [None] * self.D
-        for k, p in enumerate(self.paths):
-            for m in range(2 * p["L"] + 1):
-                self.row_path[p["out_off"] + m] = k
-        self.row_pairs = [[] for _ in range(self.D)]
+        self.row_pairs = [[] for _ in range(self.D)]   # all pairs of an output row
+        self.rp = {}                                   # (row, path) -> pairs
+        self.row_paths = [[] for _ in range(self.D)]   # paths that reach an output row, in path order
         for pi, (i0, i1, k, rl) in enumerate(self.pairs):
             self.row_pairs[i0].append(pi)
+            self.rp.setdefault((i0, k), []).append(pi)
+            if k not in self.row_paths[i0]:
+                self.row_paths[i0].append(k)
+
+    def path_rows(self, k):
+        p = self.paths[k]
+        return range(p["out_off"], p["out_off"] + 2 * p["L"] + 1)
+
+    def pairs_of(self, row, k):
+        return self.rp.get((row, k), [])
 
     # ---------------------------------------------------------------- forward
     def fwd_layout(self):
         FW = self.cfg["FW"]
         costs = []
         for row in range(self.D):
-            k = self.row_path[row]
-            l1 = self.paths[k]["l1"]
-            first_row_of_path = row == self.paths[k]["out_off"]
-            costs.append(len(self.row_pairs[row]) * 1.0 + ((2 * l1 + 1) * 1.0 + 0.5 if first_row_of_path else 0.0) + 0.3)
+            starts = sum((2 * self.paths[k]["l1"] + 1) * 1.0 + 0.5 for k in self.row_paths[row]
+                         if row == self.paths[k]["out_off"])
+            costs.append(len(self.row_pairs[row]) * 1.0 + starts + 0.3)
         bounds = partition_rows(costs, FW)
         while len(bounds) < FW + 1:
             bounds.append(bounds[-1])
@@ -125,10 +133,10 @@ class Sig:
         V = self.cfg.get("BV", self.V)
         costs = []
         for k, p in enumerate(self.paths):
-            rows = range(p["out_off"], p["out_off"] + 2 * p["L"] + 1)
-            npairs = sum(len(self.row_pairs[r]) for r in rows)
-            nrec = sum(len(self.pairs[pi][3]) for r in rows for pi in self.row_pairs[r])
-            combos = len({self.pairs[pi][1] for r in rows for pi in self.row_pairs[r]})
+            rows = self.path_rows(k)
+            npairs = sum(len(self.pairs_of(r, k)) for r in rows)
+            nrec = sum(len(self.pairs[pi][3]) for r in rows for pi in self.pairs_of(r, k))
+            combos = len({self.pairs[pi][1] for r in rows for pi in self.pairs_of(r, k)})
             # per pair: u += A dm and the lane dot product; per record one scalar FMA; per (path, i1): s*x,
             # the grad_w and grad_x FMAs; per path the weight load and the grad_w store
             costs.append(2.0 * V * npairs + nrec + 3.0 * V * combos + npairs / 4.0 + 2.0)
@@ -172,17 +180,17 @@ class Sig:
         cap = min(c for c, bins in found.items() if max(b[0] for b in bins) <= slack * floor_cost)
         bins = [[b[0], b[2]] for b in found[cap]]
         groups = sorted((sorted(b[1]) for b in bins), key=lambda g: (g[0] if g else self.P))
-        rows_of = []
+        rows_of = []   # distinct output rows of every group (paths of a collapsed plan may share rows)
         for g in groups:
             rows = []
             for k in g:
-                p = self.paths[k]
-                rows += list(range(p["out_off"], p["out_off"] + 2 * p["L"] + 1))
+                rows += [r for r in self.path_rows(k) if r not in rows]
             rows_of.append(rows)
         a0, slots = [0], []
-        for rows in rows_of:
-            for row in rows:
-                slots += self.row_pairs[row]
+        for g in groups:
+            for k in g:
+                for row in self.path_rows(k):
+                    slots += self.pairs_of(row, k)
             while len(slots) % 4:
                 slots.append(None)
             a0.append(len(slots))
@@ -234,25 +242,26 @@ class Sig:
             o.append(f"        case {g}: {{")
             rows = rows_of[g]
             local = {row: i for i, row in enumerate(rows)}
-            need_x = sorted({self.pairs[pi][1] for row in rows for pi in self.row_pairs[row]})
+            need_x = sorted({self.pairs[pi][1] for k in groups[g] for row in self.path_rows(k)
+                             for pi in self.pairs_of(row, k)})
             for i1 in need_x:
                 o.append(f"            const BVec x{i1} = xs[{i1} * NQV];")
             loaded_a = set()
             dx_touched, dy_touched = set(), set()   # first contribution assigns, later ones accumulate
             for k in groups[g]:
                 p = self.paths[k]
-                prow = list(range(p["out_off"], p["out_off"] + 2 * p["L"] + 1))
-                used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.row_pairs[r2]})
+                prow = list(self.path_rows(k))
+                used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
                 o.append(f"            const BVec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
                 for i1 in used:
                     o.append(f"            const BVec sx{k}_{i1} = vmul(s{k}, x{i1});")
                     o.append(f"            BVec u{k}_{i1}; vzero(u{k}_{i1});")
-                depth = max(len(self.row_pairs[r2]) for r2 in prow)
+                depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
                 for j in range(depth):
                     for row in prow:
-                        if j >= len(self.row_pairs[row]):
+                        if j >= len(self.pairs_of(row, k)):
                             continue
-                        pi = self.row_pairs[row][j]
+                        pi = self.pairs_of(row, k)[j]
                         slot = slot_of_pair[pi]
                         q, lane = slot // 4, "xyzw"[slot % 4]
                         if q not in loaded_a:
@@ -379,22 +388,23 @@ class Sig:
             loaded_a = set()
             paths_here = []
             for row in rows:
-                if self.row_path[row] not in paths_here:
-                    paths_here.append(self.row_path[row])
+                for k in self.row_paths[row]:
+                    if k not in paths_here:
+                        paths_here.append(k)
             for k in paths_here:
                 p = self.paths[k]
-                prow = [r2 for r2 in rows if self.row_path[r2] == k]
+                prow = [r2 for r2 in rows if self.pairs_of(r2, k)]
                 o.append(f"            const Vec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
-                used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.row_pairs[r2]})
+                used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
                 for i1 in used:
                     o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
                 # round-robin over the rows of the path so that consecutive FMAs hit different accumulators
-                depth = max(len(self.row_pairs[r2]) for r2 in prow)
+                depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
                 for j in range(depth):
                     for row in prow:
-                        if j >= len(self.row_pairs[row]):
+                        if j >= len(self.pairs_of(row, k)):
                             continue
-                        pi = self.row_pairs[row][j]
+                        pi = self.pairs_of(row, k)[j]
                         slot = slot_of_pair[pi]
                         q, lane = slot // 4, "xyzw"[slot % 4]
                         if q not in loaded_a:
