@@ -100,6 +100,20 @@ def test_scalar_input_signature():
     assert max(worst) < 1e-5
 
 
+@pytest.mark.parametrize("channels", [64, 256])
+def test_other_channel_counts_of_the_water_box_signature(channels):
+    """The water-box signature with 64 and 256 channels (generated kernels exist for both)."""
+    import dataclasses
+    irreps = f"{channels}x0e+{channels}x1o"
+    wl = dataclasses.replace(workloads.make_graph(2, 240), irreps_in=irreps)
+    plan = e3j.e3j_plan_create(irreps, 3, None, 3)
+    assert plan.specialised and plan.n_channels == channels
+    cp = oconv.Coupling(irreps, 3, None, 3)
+    x, y, w, g = workloads.make_features(wl, plan.n_paths, plan.d_out)
+    worst = run_conv_parity(wl, plan, cp, x, y, w, g)
+    assert max(worst) < 1e-5
+
+
 def test_conv_without_prepared_graph():
     worst = run_conv_parity(*make_case(1), prepared=False)
     assert max(worst) < 1e-5
