@@ -1,0 +1,253 @@
+// Edge-wise backward pass 1: one consumer warp computes the whole backward of one edge.
+//
+// The path-group kernel of fast_bwd.cuh keeps each warp's rows of grad_out[receiver] in registers and pays for
+// it with an exchange of partial sums between the warps after every edge.  Here the receiver's row block is
+// staged once in shared memory and every warp reads the rows where its body needs them: a warp owns an edge
+// from the first load to the last store, nothing is exchanged, the lane reduction of grad_sh happens once per
+// edge instead of once per edge and path group, and all warps of an SM run the same instructions.
+//
+// Ring: NS tiles of up to T edges (T = number of consumer warps, warp j takes edge j of the tile).  A tile
+// never spans a receiver change, so it needs one staged row block of grad_out; the NS blocks form a ring of
+// their own that advances only when the receiver changes (the tiles in flight use at most NS - 1 of them).
+// The producer warp cuts the tiles, issues the bulk copies (weights, sender rows, the receiver's block when
+// it is new) and contracts the A entries; the metadata it needs (receiver and sender ids, harmonics) arrives
+// two 32-edge windows ahead through 4-byte asynchronous copies.
+//
+// Only for signatures whose channels fit one warp (N_q = 32 * BV) and for graph calls (not the standalone
+// tensor product, where every row has its own grad_out block).
+#pragma once
+#include "fast_bwd.cuh"
+#include "fast_producer.cuh"
+
+namespace e3j {
+namespace fast {
+
+__device__ __forceinline__ void cp_async4(void* dst_smem, const void* src_gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst_smem)), "l"(src_gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <class S>
+struct Bwd1Smem {
+    static constexpr int T = S::ET, NS = S::ES;
+    static constexpr int S_EDGE = S::P * S::NQ;
+    static constexpr int X_EDGE = S::DIN * S::NQ;
+    static constexpr int DM_ROW = S::D * S::NQ;     // grad_out[receiver]
+    static constexpr int WIN = 32;                  // edges per metadata window; the ring holds two windows
+    static constexpr size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+    static constexpr size_t off_bar = 0;                                   // full[NS], empty[NS]
+    static constexpr size_t off_abort = off_bar + 16 * NS;
+    static constexpr size_t off_meta = up(off_abort + 4, 16);              // int[NS][4]: first edge, n_e | last << 8, block
+    static constexpr size_t off_rcv = off_meta + 16 * NS;                  // int[2 * WIN]
+    static constexpr size_t off_snd = off_rcv + 4 * 2 * WIN;               // int[2 * WIN]
+    static constexpr size_t off_y = off_snd + 4 * 2 * WIN;                 // float[2 * WIN][DSH]
+    static constexpr size_t off_dm = up(off_y + 4 * 2 * WIN * S::DSH, 128);  // float[NS][D][NQ]
+    static constexpr size_t off_stage = up(off_dm + 4 * (size_t)NS * DM_ROW, 128);
+    static constexpr size_t st_s = 0;
+    static constexpr size_t st_x = st_s + 4 * (size_t)T * S_EDGE;
+    static constexpr size_t st_A = st_x + 4 * (size_t)T * X_EDGE;
+    static constexpr size_t stage_bytes = up(st_A + 4 * (size_t)T * S::B_APAD, 128);
+    static constexpr size_t total = off_stage + NS * stage_bytes;
+};
+
+// ------------------------------------------------------------------------ consumer: one edge per tile
+template <class S>
+__device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char* smem, const int warp, const int lane,
+                                              const int64_t e_begin) {
+    using Vec = typename S::BVec;
+    using L = Bwd1Smem<S>;
+    constexpr int NS = L::NS;
+    constexpr int NQV = S::NQ / S::BV;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
+    uint64_t* empty = full + NS;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
+    int stage = 0, phase = 0;
+    for (;;) {
+        if (!mbar_wait(&full[stage], phase, abort_flag, p.status)) break;
+        const int* meta = reinterpret_cast<const int*>(smem + L::off_meta) + 4 * stage;
+        const int first = meta[0], n_e = meta[1] & 0xff, last = meta[1] >> 8, block = meta[2];
+        if (warp < n_e) {
+            const unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
+            const int64_t e = e_begin + first + warp;
+            const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + warp * (L::X_EDGE / S::BV) + lane;
+            const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + warp * (L::S_EDGE / S::BV) + lane;
+            const float* As = reinterpret_cast<const float*>(st + L::st_A) + warp * S::B_APAD;
+            const Vec* dms = reinterpret_cast<const Vec*>(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW) + lane;
+            Vec dxp[S::DIN];   // both are assigned (not accumulated into) by bwd_edge_all
+            float dyl[16];
+            Vec* gw = reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + lane;
+            S::bwd_edge_all(dms, xs, ss, As, dxp, dyl, gw);
+            Vec* dxo = reinterpret_cast<Vec*>(p.dx_edge + (size_t)e * L::X_EDGE) + lane;
+#pragma unroll
+            for (int i = 0; i < S::DIN; ++i) dxo[i * NQV] = dxp[i];
+            // sum over the channels: even lanes end up with one entry each
+            const float dy_tot = reduce16_over_lanes(dyl, lane);
+            const int idx = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+            if ((lane & 1) == 0 && idx < S::DSH) p.grad_sh[(size_t)e * S::DSH + idx] = dy_tot;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[stage]);
+        if (++stage == NS) { stage = 0; phase ^= 1; }
+        if (last) break;
+    }
+}
+
+// ------------------------------------------------------------------------ producer
+template <class S>
+__device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char* smem, const int lane,
+                                              const int64_t e_begin, const int64_t e_end) {
+    using L = Bwd1Smem<S>;
+    using Tab = BwdTab<S>;
+    constexpr int T = L::T, NS = L::NS, WIN = L::WIN, DSH = S::DSH;
+    constexpr int NA = (Tab::APAD + 31) / 32;
+    static_assert(T < 32 && WIN == 32, "a tile is cut with one ballot; windows are one warp wide");
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
+    uint64_t* empty = full + NS;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
+    int* rcv_ring = reinterpret_cast<int*>(smem + L::off_rcv);
+    int* snd_ring = reinterpret_cast<int*>(smem + L::off_snd);
+    float* y_ring = reinterpret_cast<float*>(smem + L::off_y);
+    const int n_tot = (int)(e_end - e_begin);
+
+    ASlot tab[NA];   // this lane's A slots (lane, lane + 32, ...)
+#pragma unroll
+    for (int i = 0; i < NA; ++i) {
+        const int slot = lane + 32 * i;
+        ASlot a{0.f, 0.f, 0, 0};
+        if (slot < Tab::APAD) {
+            const PairRec pr = Tab::pair_rec(slot);
+            if (pr.count > 0) { a.c0 = Tab::rec_val(pr.start); a.i2_0 = Tab::rec_i2(pr.start); }
+            if (pr.count > 1) { a.c1 = Tab::rec_val(pr.start + 1); a.i2_1 = Tab::rec_i2(pr.start + 1); }
+        }
+        tab[i] = a;
+    }
+
+    // window w = edges [32 w, 32 w + 32) of this CTA's range, kept in ring half (w & 1); one copy group each
+    auto issue_window = [&](const int w) {
+        const int i = WIN * w + lane;
+        const int half = (w & 1) * WIN;
+        if (i < n_tot) {
+            cp_async4(&rcv_ring[half + lane], p.receivers + e_begin + i);
+            cp_async4(&snd_ring[half + lane], p.senders + e_begin + i);
+        }
+#pragma unroll
+        for (int j = 0; j < DSH; ++j) {
+            const int idx = j * 32 + lane;   // entry of the window's [32][DSH] block
+            if (WIN * w + idx / DSH < n_tot)
+                cp_async4(&y_ring[half * DSH + idx], p.sh + (e_begin + (int64_t)WIN * w) * DSH + idx);
+        }
+        cp_async_commit();
+    };
+    issue_window(0);
+    issue_window(1);
+
+    int wbase = 0;               // windows wbase and wbase + 1 are in the ring or on their way
+    int done = 0;                // edges handed out so far
+    int block = NS - 1;          // ring position of the current receiver's grad_out block
+    int last_rcv = -1;
+    int stage = 0, phase = 0, armed = 0;
+#pragma unroll 1
+    for (int t = 0;; ++t) {
+        if ((done >> 5) > wbase) {   // the half that held window wbase - 1 is free
+            wbase = done >> 5;
+            issue_window(wbase + 1);
+        }
+        // the newest group may stay in flight unless this tile reaches into it
+        if ((done & 31) + T > WIN) cp_async_wait<0>(); else cp_async_wait<1>();
+        __syncwarp();
+        // the tile: edges done .. done + n_e - 1, all of one receiver
+        const int i = done + lane;
+        const int r = (lane < T && i < n_tot) ? rcv_ring[i & (2 * WIN - 1)] : -2;
+        const int r0 = __shfl_sync(0xffffffffu, r, 0);
+        const unsigned differs = __ballot_sync(0xffffffffu, r != r0);   // lane T always differs
+        const int n_e = n_tot > 0 ? __ffs((int)differs) - 1 : 0;
+        const int last = done + n_e >= n_tot;
+        // phase of `empty` that ends the previous use of this ring slot
+        if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
+        const bool new_block = n_e > 0 && r0 != last_rcv;
+        if (new_block) {
+            block = block + 1 == NS ? 0 : block + 1;
+            last_rcv = r0;
+        }
+        unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
+        if (lane == 0) {
+            int* meta = reinterpret_cast<int*>(smem + L::off_meta) + 4 * stage;
+            meta[0] = done; meta[1] = n_e | (last << 8); meta[2] = block;
+            // arrival and byte count in one step: the phase cannot complete before the bytes are expected
+            mbar_arrive_expect_tx(&full[stage], (uint32_t)n_e * 4u * (L::S_EDGE + L::X_EDGE) +
+                                                    (new_block ? 4u * L::DM_ROW : 0u));
+            if (n_e > 0)
+                bulk_g2s(st + L::st_s, p.w + (size_t)(e_begin + done) * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE,
+                         &full[stage]);
+        }
+        if (lane < n_e)
+            bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE,
+                     p.x + (size_t)snd_ring[i & (2 * WIN - 1)] * L::X_EDGE, 4u * L::X_EDGE, &full[stage]);
+        if (lane == 31 && new_block)
+            bulk_g2s(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW, p.grad_out + (size_t)r0 * L::DM_ROW,
+                     4u * L::DM_ROW, &full[stage]);
+        armed = t + 1;
+        // A[e][slot] = sum over the slot's records of c * y[e][i2]; all loads before the first store
+        // (entries of edges beyond n_e are computed from stale data and never read)
+        float* A_t = reinterpret_cast<float*>(st + L::st_A);
+        float a_val[NA][T];
+#pragma unroll
+        for (int k = 0; k < NA; ++k)
+#pragma unroll
+            for (int e_i = 0; e_i < T; ++e_i) {
+                const float* ye = y_ring + ((done + e_i) & (2 * WIN - 1)) * DSH;
+                a_val[k][e_i] = fmaf(tab[k].c1, ye[tab[k].i2_1], tab[k].c0 * ye[tab[k].i2_0]);
+            }
+#pragma unroll
+        for (int k = 0; k < NA; ++k) {
+            const int slot = lane + 32 * k;
+            if (slot < Tab::APAD) {
+#pragma unroll
+                for (int e_i = 0; e_i < T; ++e_i) A_t[e_i * Tab::APAD + slot] = a_val[k][e_i];
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[stage]);   // the staged A entries and the tile's metadata are in place
+        if (++stage == NS) { stage = 0; phase ^= 1; }
+        done += n_e;
+        if (last) break;
+    }
+    cp_async_wait<0>();
+    if (*abort_flag) drain_copies<L>(smem, armed);
+}
+
+template <class S>
+__global__ void __launch_bounds__((S::ET + 1) * 32, 1)
+fast_bwd1_kernel(const BwdParams p) {
+    using L = Bwd1Smem<S>;
+    constexpr int T = L::T, NS = L::NS;
+    static_assert(S::NQ == 32 * S::BV, "one warp holds all channels of an edge");
+    static_assert(S::B_NREC <= 2, "an A slot holds at most two records");
+    static_assert(S::DSH <= 16, "harmonics beyond l = 3 need a wider reduction");
+
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
+    uint64_t* empty = full + NS;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int64_t n_edges, chunk, e_begin, e_end;   // n_edges: the real edges (a padded call learns their number here)
+    cta_edge_range(p.n_edges, p.chunk, p.n_real, n_edges, chunk, e_begin, e_end);
+
+    if (threadIdx.x == 0) {
+        // full: the producer's arrival with the copies' byte count and its arrival after the tables
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], T); }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    if (warp == T) bwd1_producer<S>(p, smem, lane, e_begin, e_end);
+    else bwd1_consumer<S>(p, smem, warp, lane, e_begin);
+}
+
+}  // namespace fast
+}  // namespace e3j

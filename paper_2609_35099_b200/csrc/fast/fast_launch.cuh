@@ -4,6 +4,7 @@
 
 #include "../fast_registry.hpp"
 #include "fast_bwd.cuh"
+#include "fast_bwd1.cuh"
 #include "fast_fwd.cuh"
 
 namespace e3j {
@@ -123,14 +124,8 @@ int launch_bwd(const ConvArgs& a) {
     using L = BwdSmem<S>;
     static_assert(L::total * S::BC + 1024 * S::BC <= 228 * 1024, "backward stage ring does not fit in shared memory");
     if (a.workspace_bytes < bwd_scratch_bytes<S>(a.n_nodes, a.n_edges)) return E3J_ERR_WORKSPACE;
-    const int n_cta = sm_count() * S::BC;
-    static thread_local int attr_dev = -1;
-    int dev = 0;
-    E3J_CUDA_TRY(cudaGetDevice(&dev));
-    if (attr_dev != dev) {
-        E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));
-        attr_dev = dev;
-    }
+    constexpr bool kEdgewise = S::ET > 0;   // one warp per edge, one CTA per SM (fast_bwd1.cuh)
+    const int n_cta = sm_count() * (kEdgewise ? 1 : S::BC);
     BwdParams p{};
     p.x = a.x; p.sh = a.sh; p.w = a.w; p.senders = a.senders; p.receivers = a.receivers;
     p.grad_out = a.grad_out; p.grad_sh = a.grad_sh; p.grad_w = a.grad_w;
@@ -139,8 +134,25 @@ int launch_bwd(const ConvArgs& a) {
     p.chunk = (a.n_edges + n_cta - 1) / n_cta;
     p.status = a.status;
     p.n_real = a.n_real;
-    constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;  // consumers + one producer warp
-    fast_bwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
+    static thread_local int attr_dev = -1;
+    int dev = 0;
+    E3J_CUDA_TRY(cudaGetDevice(&dev));
+    if constexpr (kEdgewise) {
+        using L1 = Bwd1Smem<S>;
+        static_assert(L1::total + 1024 <= 228 * 1024, "edge-wise backward ring does not fit in shared memory");
+        if (attr_dev != dev) {
+            E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd1_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L1::total));
+            attr_dev = dev;
+        }
+        fast_bwd1_kernel<S><<<n_cta, (S::ET + 1) * 32, L1::total, a.stream>>>(p);  // consumers + one producer warp
+    } else {
+        if (attr_dev != dev) {
+            E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));
+            attr_dev = dev;
+        }
+        constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;  // consumers + one producer warp
+        fast_bwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
+    }
     if (int s = after_launch()) return s;
     if (a.n_real) {
         bwd_zero_padding_kernel<<<148 * 8, 256, 0, a.stream>>>(a.n_real, a.n_edges, S::P * S::NQ / 4, S::DSH,

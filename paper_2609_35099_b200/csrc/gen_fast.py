@@ -222,6 +222,9 @@ class Sig:
         o.append(f"    using BVec = {bvec};")
         o.append(f"    static constexpr int BW = {BW}, BT = {BT}, BS = {BS}, BC = {BC}, B_RMAX = {rmax}, B_APAD = {len(slots)}, "
                  f"B_NREC = {max(c for _, c in pair_tab)};")
+        o.append(f"    // edge-wise backward (one warp per edge, grad_out rows read from shared memory): edges per tile "
+                 f"(0 = not generated), ring stages")
+        o.append(f"    static constexpr int ET = {self.cfg.get('ET', 0)}, ES = {self.cfg.get('ES', 2)};")
         o.append(f"    __device__ static __forceinline__ PairRec b_pair_rec(int i) {{ return kBPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float b_rec_val(int i) {{ return kBVal_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ unsigned char b_rec_i2(int i) {{ return kBI2_{self.name}[i]; }}")
@@ -304,6 +307,72 @@ class Sig:
         o.append("            for (int i = 0; i < 16; ++i) dyl[i] = 0.f;")
         o.append("        } break;")
         o.append("        }")
+        o.append("    }")
+        if self.cfg.get("ET", 0):
+            o += self.emit_bwd_edgewise(slot_of_pair)
+        return o
+
+    def emit_bwd_edgewise(self, slot_of_pair):
+        """The whole backward of one edge in one warp: every path in turn, the rows of grad_out[receiver]
+        loaded from shared memory (dms) where they are used, no partial sums to exchange."""
+        o = []
+        o.append(f"    __device__ static __forceinline__ void bwd_edge_all(const BVec* __restrict__ dms, const BVec* __restrict__ xs, "
+                 f"const BVec* __restrict__ ss, const float* __restrict__ As, BVec (&dxp)[DIN], float (&dyl)[16], "
+                 f"BVec* __restrict__ gw) {{")
+        o.append(f"        constexpr int NQV = NQ / BV;")
+        for i1 in range(self.DIN):
+            o.append(f"        const BVec x{i1} = xs[{i1} * NQV];")
+        loaded_a, dx_touched, dy_touched = set(), set(), set()
+        for k in range(self.P):
+            p = self.paths[k]
+            prow = list(self.path_rows(k))
+            used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
+            o.append(f"        const BVec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
+            for i1 in used:
+                o.append(f"        const BVec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                o.append(f"        BVec u{k}_{i1}; vzero(u{k}_{i1});")
+            depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
+            have = set()
+            for j in range(depth):
+                for row in prow:
+                    if j >= len(self.pairs_of(row, k)):
+                        continue
+                    if row not in have:
+                        have.add(row)
+                        o.append(f"        const BVec d{k}_{row} = dms[{row} * NQV];")
+                    pi = self.pairs_of(row, k)[j]
+                    slot = slot_of_pair[pi]
+                    q, lane = slot // 4, "xyzw"[slot % 4]
+                    if q not in loaded_a:
+                        loaded_a.add(q)
+                        o.append(f"        const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
+                    i1 = self.pairs[pi][1]
+                    o.append(f"        vfma(u{k}_{i1}, a{q}.{lane}, d{k}_{row});")
+                    o.append(f"        {{ const float t = vdot(sx{k}_{i1}, d{k}_{row});")
+                    for i2, c in self.pairs[pi][3]:
+                        if i2 in dy_touched:
+                            o.append(f"          dyl[{i2}] = fmaf({fmt_float(c)}, t, dyl[{i2}]);")
+                        else:
+                            dy_touched.add(i2)
+                            o.append(f"          dyl[{i2}] = {fmt_float(c)} * t;")
+                    o.append("        }")
+            first = used[0]
+            o.append(f"        BVec ds{k} = vmul(x{first}, u{k}_{first});")
+            for i1 in used[1:]:
+                o.append(f"        vfma(ds{k}, x{i1}, u{k}_{i1});")
+            o.append(f"        gw[{k} * NQV] = ds{k};")
+            for i1 in used:
+                if i1 in dx_touched:
+                    o.append(f"        vfma(dxp[{i1}], s{k}, u{k}_{i1});")
+                else:
+                    dx_touched.add(i1)
+                    o.append(f"        dxp[{i1}] = vmul(s{k}, u{k}_{i1});")
+        for i1 in range(self.DIN):
+            if i1 not in dx_touched:
+                o.append(f"        vzero(dxp[{i1}]);")
+        for i2 in range(16):
+            if i2 not in dy_touched:
+                o.append(f"        dyl[{i2}] = 0.f;")
         o.append("    }")
         return o
 
