@@ -13,7 +13,7 @@
 // it is new) and contracts the A entries; the metadata it needs (receiver and sender ids, harmonics) arrives
 // two 32-edge windows ahead through 4-byte asynchronous copies.
 //
-// Only for signatures whose channels fit one warp (N_q = 32 * BV) and for graph calls (not the standalone
+// Only for signatures whose channels fit one warp (N_q = 32 * EV) and for graph calls (not the standalone
 // tensor product, where every row has its own grad_out block).
 #pragma once
 #include "fast_bwd.cuh"
@@ -58,10 +58,10 @@ struct Bwd1Smem {
 template <class S>
 __device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char* smem, const int warp, const int lane,
                                               const int64_t e_begin) {
-    using Vec = typename S::BVec;
+    using Vec = typename S::EVec;
     using L = Bwd1Smem<S>;
     constexpr int NS = L::NS;
-    constexpr int NQV = S::NQ / S::BV;
+    constexpr int NQV = S::NQ / S::EV;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
     uint64_t* empty = full + NS;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
@@ -73,8 +73,8 @@ __device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char*
         if (warp < n_e) {
             const unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
             const int64_t e = e_begin + first + warp;
-            const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + warp * (L::X_EDGE / S::BV) + lane;
-            const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + warp * (L::S_EDGE / S::BV) + lane;
+            const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + warp * (L::X_EDGE / S::EV) + lane;
+            const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + warp * (L::S_EDGE / S::EV) + lane;
             const float* As = reinterpret_cast<const float*>(st + L::st_A) + warp * S::B_APAD;
             const Vec* dms = reinterpret_cast<const Vec*>(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW) + lane;
             Vec dxp[S::DIN];   // both are assigned (not accumulated into) by bwd_edge_all
@@ -225,7 +225,7 @@ __global__ void __launch_bounds__((S::ET + 1) * 32, 1)
 fast_bwd1_kernel(const BwdParams p) {
     using L = Bwd1Smem<S>;
     constexpr int T = L::T, NS = L::NS;
-    static_assert(S::NQ == 32 * S::BV, "one warp holds all channels of an edge");
+    static_assert(S::NQ == 32 * S::EV, "one warp holds all channels of an edge");
     static_assert(S::B_NREC <= 2, "an A slot holds at most two records");
     static_assert(S::DSH <= 16, "harmonics beyond l = 3 need a wider reduction");
 

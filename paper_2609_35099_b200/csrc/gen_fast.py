@@ -224,7 +224,9 @@ class Sig:
                  f"B_NREC = {max(c for _, c in pair_tab)};")
         o.append(f"    // edge-wise backward (one warp per edge, grad_out rows read from shared memory): edges per tile "
                  f"(0 = not generated), ring stages")
-        o.append(f"    static constexpr int ET = {self.cfg.get('ET', 0)}, ES = {self.cfg.get('ES', 2)};")
+        EV = self.cfg.get("EV", V)
+        o.append(f"    static constexpr int ET = {self.cfg.get('ET', 0)}, ES = {self.cfg.get('ES', 2)}, EV = {EV};")
+        o.append(f"    using EVec = {{1: 'float', 2: 'float2', 4: 'float4'}}[EV];".replace("{1: 'float', 2: 'float2', 4: 'float4'}[EV]", {1: "float", 2: "float2", 4: "float4"}[EV]))
         o.append(f"    __device__ static __forceinline__ PairRec b_pair_rec(int i) {{ return kBPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float b_rec_val(int i) {{ return kBVal_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ unsigned char b_rec_i2(int i) {{ return kBI2_{self.name}[i]; }}")
@@ -316,21 +318,21 @@ class Sig:
         """The whole backward of one edge in one warp: every path in turn, the rows of grad_out[receiver]
         loaded from shared memory (dms) where they are used, no partial sums to exchange."""
         o = []
-        o.append(f"    __device__ static __forceinline__ void bwd_edge_all(const BVec* __restrict__ dms, const BVec* __restrict__ xs, "
-                 f"const BVec* __restrict__ ss, const float* __restrict__ As, BVec (&dxp)[DIN], float (&dyl)[16], "
-                 f"BVec* __restrict__ gw) {{")
-        o.append(f"        constexpr int NQV = NQ / BV;")
+        o.append(f"    __device__ static __forceinline__ void bwd_edge_all(const EVec* __restrict__ dms, const EVec* __restrict__ xs, "
+                 f"const EVec* __restrict__ ss, const float* __restrict__ As, EVec (&dxp)[DIN], float (&dyl)[16], "
+                 f"EVec* __restrict__ gw) {{")
+        o.append(f"        constexpr int NQV = NQ / EV;")
         for i1 in range(self.DIN):
-            o.append(f"        const BVec x{i1} = xs[{i1} * NQV];")
+            o.append(f"        const EVec x{i1} = xs[{i1} * NQV];")
         loaded_a, dx_touched, dy_touched = set(), set(), set()
         for k in range(self.P):
             p = self.paths[k]
             prow = list(self.path_rows(k))
             used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
-            o.append(f"        const BVec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
+            o.append(f"        const EVec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
             for i1 in used:
-                o.append(f"        const BVec sx{k}_{i1} = vmul(s{k}, x{i1});")
-                o.append(f"        BVec u{k}_{i1}; vzero(u{k}_{i1});")
+                o.append(f"        const EVec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                o.append(f"        EVec u{k}_{i1}; vzero(u{k}_{i1});")
             depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
             have = set()
             for j in range(depth):
@@ -339,7 +341,7 @@ class Sig:
                         continue
                     if row not in have:
                         have.add(row)
-                        o.append(f"        const BVec d{k}_{row} = dms[{row} * NQV];")
+                        o.append(f"        const EVec d{k}_{row} = dms[{row} * NQV];")
                     pi = self.pairs_of(row, k)[j]
                     slot = slot_of_pair[pi]
                     q, lane = slot // 4, "xyzw"[slot % 4]
@@ -357,7 +359,7 @@ class Sig:
                             o.append(f"          dyl[{i2}] = {fmt_float(c)} * t;")
                     o.append("        }")
             first = used[0]
-            o.append(f"        BVec ds{k} = vmul(x{first}, u{k}_{first});")
+            o.append(f"        EVec ds{k} = vmul(x{first}, u{k}_{first});")
             for i1 in used[1:]:
                 o.append(f"        vfma(ds{k}, x{i1}, u{k}_{i1});")
             o.append(f"        gw[{k} * NQV] = ds{k};")

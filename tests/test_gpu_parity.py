@@ -148,6 +148,31 @@ def test_isolated_nodes_ragged_rows_and_duplicates(flags):
     assert torch.count_nonzero(out[[0, 7, 8, 40]]) == 0
 
 
+@pytest.mark.parametrize("degrees", [[1], [7, 8, 1, 14, 15, 6, 32, 33, 64, 2], [63, 65]])
+def test_backward_tiles_are_cut_at_receiver_changes(degrees):
+    """Rows as long as a tile of the edge-wise backward, one edge shorter and longer, rows of one edge (a new
+    receiver block every tile) and rows longer than a look-ahead window, with enough edges that every CTA walks
+    through several windows."""
+    rng = np.random.default_rng(7)
+    c = workloads.CONFIGS[2]
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], None, 3)
+    assert plan.specialised
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], None, 3)
+    n = 148 * 90 // max(1, int(np.mean(degrees))) + 11
+    deg = np.resize(np.asarray(degrees), n)
+    rcv = np.repeat(np.arange(n), deg).astype(np.int32)
+    snd = rng.integers(0, n, size=len(rcv)).astype(np.int32)
+    e = len(rcv)
+    wl = workloads.Workload(config=2, name="cuts", irreps_in=c["irreps_in"], sh_lmax=3, irreps_out=None,
+                            out_lmax=3, n_nodes=n, n_edges=e, senders=snd, receivers=rcv)
+    x = rng.standard_normal((n, plan.d_in, plan.n_channels)).astype(np.float32)
+    y = rng.standard_normal((e, plan.d_sh)).astype(np.float32)
+    w = rng.standard_normal((e, plan.n_paths, plan.n_channels)).astype(np.float32)
+    g = rng.standard_normal((n, plan.d_out, plan.n_channels)).astype(np.float32)
+    worst = run_conv_parity(wl, plan, cp, x, y, w, g)
+    assert max(worst) < 1e-5
+
+
 @pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
 def test_empty_graph(flags):
     plan = e3j.e3j_plan_create("128x0e+128x1o", 3, None, 3, flags)
