@@ -13,8 +13,14 @@
 // it is new) and contracts the A entries; the metadata it needs (receiver and sender ids, harmonics) arrives
 // two 32-edge windows ahead through 4-byte asynchronous copies.
 //
-// Only for signatures whose channels fit one warp (N_q = 32 * EV) and for graph calls (not the standalone
-// tensor product, where every row has its own grad_out block).
+// Standalone tensor product (ROWS = true): every row is its own sender and receiver, so its grad_out block
+// travels with it in the ring slot, tiles are fixed runs of T rows, and each ring slot has its own T consumer
+// warps (a slot of a 100-row signature is 70 KB: three of them, one warp each, keep more bytes in flight than
+// a double-buffered pair would).
+//
+// Channels beyond one warp's (CH = N_q / (32 EV) > 1): CH warps share an edge, each with its own channels.
+// Only the channel sum of grad_sh joins them: every warp leaves its 16 partial sums in the slot, and the first
+// warp of the edge adds them in warp order once all have arrived (bounded wait on a barrier of their own).
 #pragma once
 #include "fast_bwd.cuh"
 #include "fast_producer.cuh"
@@ -31,76 +37,112 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-template <class S>
+template <class S, bool ROWS>
 struct Bwd1Smem {
-    static constexpr int T = S::ET, NS = S::ES;
+    static constexpr int T = ROWS ? S::ETR : S::ET, NS = ROWS ? S::ESR : S::ES;
+    static constexpr int CH = S::NQ / (32 * S::EV); // warps per edge
+    static constexpr int NG = ROWS ? NS : 1;        // groups of T * CH consumer warps (ROWS: one per ring slot)
     static constexpr int S_EDGE = S::P * S::NQ;
     static constexpr int X_EDGE = S::DIN * S::NQ;
     static constexpr int DM_ROW = S::D * S::NQ;     // grad_out[receiver]
     static constexpr int WIN = 32;                  // edges per metadata window; the ring holds two windows
     static constexpr size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
     static constexpr size_t off_bar = 0;                                   // full[NS], empty[NS]
-    static constexpr size_t off_abort = off_bar + 16 * NS;
+    static constexpr size_t off_join = off_bar + 16 * NS;                  // join[NS][T]: the CH warps of an edge
+    static constexpr size_t off_abort = off_join + 8 * NS * T;
     static constexpr size_t off_meta = up(off_abort + 4, 16);              // int[NS][4]: first edge, n_e | last << 8, block
     static constexpr size_t off_rcv = off_meta + 16 * NS;                  // int[2 * WIN]
     static constexpr size_t off_snd = off_rcv + 4 * 2 * WIN;               // int[2 * WIN]
     static constexpr size_t off_y = off_snd + 4 * 2 * WIN;                 // float[2 * WIN][DSH]
-    static constexpr size_t off_dm = up(off_y + 4 * 2 * WIN * S::DSH, 128);  // float[NS][D][NQ]
-    static constexpr size_t off_stage = up(off_dm + 4 * (size_t)NS * DM_ROW, 128);
+    static constexpr size_t off_dm = up(off_y + 4 * 2 * WIN * S::DSH, 128);  // float[NS][D][NQ] (graph calls)
+    static constexpr size_t off_stage = up(off_dm + (ROWS ? 0 : 4 * (size_t)NS * DM_ROW), 128);
     static constexpr size_t st_s = 0;
     static constexpr size_t st_x = st_s + 4 * (size_t)T * S_EDGE;
     static constexpr size_t st_A = st_x + 4 * (size_t)T * X_EDGE;
-    static constexpr size_t stage_bytes = up(st_A + 4 * (size_t)T * S::B_APAD, 128);
+    static constexpr size_t st_dy = st_A + 4 * (size_t)T * S::B_APAD;            // float[T][CH][16] (CH > 1)
+    static constexpr size_t st_dm = up(st_dy + (CH > 1 ? 4 * (size_t)T * CH * 16 : 0), 128);   // float[T][D][NQ] (ROWS)
+    static constexpr size_t stage_bytes = up(st_dm + (ROWS ? 4 * (size_t)T * DM_ROW : 0), 128);
     static constexpr size_t total = off_stage + NS * stage_bytes;
 };
 
 // ------------------------------------------------------------------------ consumer: one edge per tile
-template <class S>
+template <class S, bool ROWS>
 __device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char* smem, const int warp, const int lane,
-                                              const int64_t e_begin) {
+                                              const int64_t e_begin, const int64_t e_end) {
     using Vec = typename S::EVec;
-    using L = Bwd1Smem<S>;
+    using L = Bwd1Smem<S, ROWS>;
     constexpr int NS = L::NS;
     constexpr int NQV = S::NQ / S::EV;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
     uint64_t* empty = full + NS;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
-    int stage = 0, phase = 0;
-    for (;;) {
+    constexpr int CH = L::CH;
+    const int j = (warp / CH) % L::T;            // this warp's edge of a tile
+    const int c = warp % CH;                     // and its share of the channels
+    const int vlane = c * 32 + lane;
+    uint64_t* join = reinterpret_cast<uint64_t*>(smem + L::off_join);
+    int stage = ROWS ? warp / (L::T * CH) : 0, phase = 0;
+    unsigned join_phase = 0;   // bit s: parity of the next use of this edge slot's join barrier in ring slot s
+    // ROWS: tiles are fixed runs of T rows and this warp's group takes every NS-th of them
+    int my_tiles = ROWS ? ((int)((e_end - e_begin + L::T - 1) / L::T) - stage + NS - 1) / NS : 1;
+    while (my_tiles > 0) {
         if (!mbar_wait(&full[stage], phase, abort_flag, p.status)) break;
         const int* meta = reinterpret_cast<const int*>(smem + L::off_meta) + 4 * stage;
         const int first = meta[0], n_e = meta[1] & 0xff, last = meta[1] >> 8, block = meta[2];
-        if (warp < n_e) {
+        if (j < n_e) {
             const unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
-            const int64_t e = e_begin + first + warp;
-            const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + warp * (L::X_EDGE / S::EV) + lane;
-            const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + warp * (L::S_EDGE / S::EV) + lane;
-            const float* As = reinterpret_cast<const float*>(st + L::st_A) + warp * S::B_APAD;
-            const Vec* dms = reinterpret_cast<const Vec*>(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW) + lane;
+            const int64_t e = e_begin + first + j;
+            const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + j * (L::X_EDGE / S::EV) + vlane;
+            const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + j * (L::S_EDGE / S::EV) + vlane;
+            const float* As = reinterpret_cast<const float*>(st + L::st_A) + j * S::B_APAD;
+            const Vec* dms = (ROWS ? reinterpret_cast<const Vec*>(st + L::st_dm) + j * (L::DM_ROW / S::EV)
+                                   : reinterpret_cast<const Vec*>(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW)) + vlane;
             Vec dxp[S::DIN];   // both are assigned (not accumulated into) by bwd_edge_all
             float dyl[16];
-            Vec* gw = reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + lane;
+            Vec* gw = reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + vlane;
             S::bwd_edge_all(dms, xs, ss, As, dxp, dyl, gw);
-            Vec* dxo = reinterpret_cast<Vec*>(p.dx_edge + (size_t)e * L::X_EDGE) + lane;
+            Vec* dxo = reinterpret_cast<Vec*>(p.dx_edge + (size_t)e * L::X_EDGE) + vlane;
 #pragma unroll
             for (int i = 0; i < S::DIN; ++i) dxo[i * NQV] = dxp[i];
             // sum over the channels: even lanes end up with one entry each
             const float dy_tot = reduce16_over_lanes(dyl, lane);
             const int idx = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
-            if ((lane & 1) == 0 && idx < S::DSH) p.grad_sh[(size_t)e * S::DSH + idx] = dy_tot;
+            if constexpr (CH == 1) {
+                if ((lane & 1) == 0 && idx < S::DSH) p.grad_sh[(size_t)e * S::DSH + idx] = dy_tot;
+            } else {
+                float* dyx = const_cast<float*>(reinterpret_cast<const float*>(st + L::st_dy)) + j * CH * 16;
+                if ((lane & 1) == 0) dyx[c * 16 + idx] = dy_tot;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&join[stage * L::T + j]);
+                if (c == 0) {   // fixed-order sum over the edge's warps
+                    if (!mbar_wait(&join[stage * L::T + j], (join_phase >> stage) & 1u, abort_flag, p.status)) break;
+                    if (lane < S::DSH) {
+                        float sum = 0.f;
+#pragma unroll
+                        for (int c2 = 0; c2 < CH; ++c2) sum += dyx[c2 * 16 + lane];
+                        p.grad_sh[(size_t)e * S::DSH + lane] = sum;
+                    }
+                }
+                join_phase ^= 1u << stage;   // (a short tile leaves the barriers of its unused edge slots alone)
+            }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[stage]);
-        if (++stage == NS) { stage = 0; phase ^= 1; }
-        if (last) break;
+        if (ROWS) {
+            phase ^= 1;   // this group's slot again, one trip round the ring later
+            --my_tiles;
+        } else {
+            if (++stage == NS) { stage = 0; phase ^= 1; }
+            if (last) break;
+        }
     }
 }
 
 // ------------------------------------------------------------------------ producer
-template <class S>
+template <class S, bool ROWS>
 __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char* smem, const int lane,
                                               const int64_t e_begin, const int64_t e_end) {
-    using L = Bwd1Smem<S>;
+    using L = Bwd1Smem<S, ROWS>;
     using Tab = BwdTab<S>;
     constexpr int T = L::T, NS = L::NS, WIN = L::WIN, DSH = S::DSH;
     constexpr int NA = (Tab::APAD + 31) / 32;
@@ -130,7 +172,7 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
     auto issue_window = [&](const int w) {
         const int i = WIN * w + lane;
         const int half = (w & 1) * WIN;
-        if (i < n_tot) {
+        if (!ROWS && i < n_tot) {
             cp_async4(&rcv_ring[half + lane], p.receivers + e_begin + i);
             cp_async4(&snd_ring[half + lane], p.senders + e_begin + i);
         }
@@ -145,6 +187,10 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
     issue_window(0);
     issue_window(1);
 
+    if (ROWS && n_tot == 0) {    // the consumers of a call without rows expect no tile
+        cp_async_wait<0>();
+        return;
+    }
     int wbase = 0;               // windows wbase and wbase + 1 are in the ring or on their way
     int done = 0;                // edges handed out so far
     int block = NS - 1;          // ring position of the current receiver's grad_out block
@@ -159,16 +205,21 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
         // the newest group may stay in flight unless this tile reaches into it
         if ((done & 31) + T > WIN) cp_async_wait<0>(); else cp_async_wait<1>();
         __syncwarp();
-        // the tile: edges done .. done + n_e - 1, all of one receiver
+        // the tile: edges done .. done + n_e - 1, all of one receiver (ROWS: the next T rows)
         const int i = done + lane;
-        const int r = (lane < T && i < n_tot) ? rcv_ring[i & (2 * WIN - 1)] : -2;
-        const int r0 = __shfl_sync(0xffffffffu, r, 0);
-        const unsigned differs = __ballot_sync(0xffffffffu, r != r0);   // lane T always differs
-        const int n_e = n_tot > 0 ? __ffs((int)differs) - 1 : 0;
+        int r0 = -1, n_e;
+        if (ROWS) {
+            n_e = min(T, n_tot - done);
+        } else {
+            const int r = (lane < T && i < n_tot) ? rcv_ring[i & (2 * WIN - 1)] : -2;
+            r0 = __shfl_sync(0xffffffffu, r, 0);
+            const unsigned differs = __ballot_sync(0xffffffffu, r != r0);   // lane T always differs
+            n_e = n_tot > 0 ? __ffs((int)differs) - 1 : 0;
+        }
         const int last = done + n_e >= n_tot;
         // phase of `empty` that ends the previous use of this ring slot
         if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
-        const bool new_block = n_e > 0 && r0 != last_rcv;
+        const bool new_block = !ROWS && n_e > 0 && r0 != last_rcv;
         if (new_block) {
             block = block + 1 == NS ? 0 : block + 1;
             last_rcv = r0;
@@ -178,18 +229,27 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
             int* meta = reinterpret_cast<int*>(smem + L::off_meta) + 4 * stage;
             meta[0] = done; meta[1] = n_e | (last << 8); meta[2] = block;
             // arrival and byte count in one step: the phase cannot complete before the bytes are expected
-            mbar_arrive_expect_tx(&full[stage], (uint32_t)n_e * 4u * (L::S_EDGE + L::X_EDGE) +
+            mbar_arrive_expect_tx(&full[stage], (uint32_t)n_e * 4u * (L::S_EDGE + L::X_EDGE + (ROWS ? L::DM_ROW : 0)) +
                                                     (new_block ? 4u * L::DM_ROW : 0u));
             if (n_e > 0)
                 bulk_g2s(st + L::st_s, p.w + (size_t)(e_begin + done) * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE,
                          &full[stage]);
         }
-        if (lane < n_e)
-            bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE,
-                     p.x + (size_t)snd_ring[i & (2 * WIN - 1)] * L::X_EDGE, 4u * L::X_EDGE, &full[stage]);
-        if (lane == 31 && new_block)
-            bulk_g2s(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW, p.grad_out + (size_t)r0 * L::DM_ROW,
-                     4u * L::DM_ROW, &full[stage]);
+        if (ROWS) {   // the rows' inputs and grad_out blocks are contiguous
+            if (lane == 1)
+                bulk_g2s(st + L::st_x, p.x + (size_t)(e_begin + done) * L::X_EDGE, (uint32_t)n_e * 4u * L::X_EDGE,
+                         &full[stage]);
+            if (lane == 2)
+                bulk_g2s(st + L::st_dm, p.grad_out + (size_t)(e_begin + done) * L::DM_ROW,
+                         (uint32_t)n_e * 4u * L::DM_ROW, &full[stage]);
+        } else {
+            if (lane < n_e)
+                bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE,
+                         p.x + (size_t)snd_ring[i & (2 * WIN - 1)] * L::X_EDGE, 4u * L::X_EDGE, &full[stage]);
+            if (lane == 31 && new_block)
+                bulk_g2s(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW, p.grad_out + (size_t)r0 * L::DM_ROW,
+                         4u * L::DM_ROW, &full[stage]);
+        }
         armed = t + 1;
         // A[e][slot] = sum over the slot's records of c * y[e][i2]; all loads before the first store
         // (entries of edges beyond n_e are computed from stale data and never read)
@@ -220,12 +280,12 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
     if (*abort_flag) drain_copies<L>(smem, armed);
 }
 
-template <class S>
-__global__ void __launch_bounds__((S::ET + 1) * 32, 1)
+template <class S, bool ROWS>
+__global__ void __launch_bounds__((Bwd1Smem<S, ROWS>::T * Bwd1Smem<S, ROWS>::CH * Bwd1Smem<S, ROWS>::NG + 1) * 32, 1)
 fast_bwd1_kernel(const BwdParams p) {
-    using L = Bwd1Smem<S>;
-    constexpr int T = L::T, NS = L::NS;
-    static_assert(S::NQ == 32 * S::EV, "one warp holds all channels of an edge");
+    using L = Bwd1Smem<S, ROWS>;
+    constexpr int T = L::T, NS = L::NS, NCONS = L::T * L::CH * L::NG;
+    static_assert(S::NQ == 32 * S::EV * L::CH, "the channels are dealt out to whole warps");
     static_assert(S::B_NREC <= 2, "an A slot holds at most two records");
     static_assert(S::DSH <= 16, "harmonics beyond l = 3 need a wider reduction");
 
@@ -239,14 +299,16 @@ fast_bwd1_kernel(const BwdParams p) {
     cta_edge_range(p.n_edges, p.chunk, p.n_real, n_edges, chunk, e_begin, e_end);
 
     if (threadIdx.x == 0) {
-        // full: the producer's arrival with the copies' byte count and its arrival after the tables
-        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], T); }
+        // full: the producer's arrival with the copies' byte count and its arrival after the tables;
+        // empty: the T warps that work on the slot
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], T * L::CH); }
+        for (int s = 0; s < NS * T; ++s) mbar_init(reinterpret_cast<uint64_t*>(smem + L::off_join) + s, L::CH);
         *abort_flag = 0;
         mbar_fence_init();
     }
     __syncthreads();
-    if (warp == T) bwd1_producer<S>(p, smem, lane, e_begin, e_end);
-    else bwd1_consumer<S>(p, smem, warp, lane, e_begin);
+    if (warp == NCONS) bwd1_producer<S, ROWS>(p, smem, lane, e_begin, e_end);
+    else bwd1_consumer<S, ROWS>(p, smem, warp, lane, e_begin, e_end);
 }
 
 }  // namespace fast

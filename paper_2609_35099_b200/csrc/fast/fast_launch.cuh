@@ -95,21 +95,32 @@ int launch_tp_bwd(int64_t rows, const float* x1, const float* x2, const float* w
                   float* gx2, float* gw, cudaStream_t st) {
     using L = BwdSmem<S>;
     if (!gx1 || !gx2 || !gw) return E3J_ERR_UNSUPPORTED;  // caller falls back to the generic kernels
-    const int n_cta = sm_count() * S::BC;
-    static thread_local int attr_dev = -1;
-    int dev = 0;
-    E3J_CUDA_TRY(cudaGetDevice(&dev));
-    if (attr_dev != dev) {
-        E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));
-        attr_dev = dev;
-    }
+    constexpr bool kRowwise = S::ETR > 0;   // one warp per row, one CTA per SM (fast_bwd1.cuh)
+    const int n_cta = sm_count() * (kRowwise ? 1 : S::BC);
     BwdParams p{};
     p.x = x1; p.sh = x2; p.w = w; p.grad_out = g; p.grad_sh = gx2; p.grad_w = gw;
     p.dx_edge = gx1;  // each row is its own sender: the per-edge share is the gradient
     p.n_nodes = rows; p.n_edges = rows; p.identity = 1;
     p.chunk = (rows + n_cta - 1) / n_cta;
-    constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;  // consumers + one producer warp
-    fast_bwd_kernel<S><<<n_cta, threads, L::total, st>>>(p);
+    static thread_local int attr_dev = -1;
+    int dev = 0;
+    E3J_CUDA_TRY(cudaGetDevice(&dev));
+    if constexpr (kRowwise) {
+        using L1 = Bwd1Smem<S, true>;
+        static_assert(L1::total + 1024 <= 228 * 1024, "row-wise backward ring does not fit in shared memory");
+        if (attr_dev != dev) {
+            E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd1_kernel<S, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L1::total));
+            attr_dev = dev;
+        }
+        fast_bwd1_kernel<S, true><<<n_cta, (L1::T * L1::CH * L1::NG + 1) * 32, L1::total, st>>>(p);
+    } else {
+        if (attr_dev != dev) {
+            E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));
+            attr_dev = dev;
+        }
+        constexpr int threads = (S::BW * (S::NQ / (32 * S::BV)) + 1) * 32;  // consumers + one producer warp
+        fast_bwd_kernel<S><<<n_cta, threads, L::total, st>>>(p);
+    }
     return after_launch();
 }
 
@@ -138,13 +149,13 @@ int launch_bwd(const ConvArgs& a) {
     int dev = 0;
     E3J_CUDA_TRY(cudaGetDevice(&dev));
     if constexpr (kEdgewise) {
-        using L1 = Bwd1Smem<S>;
+        using L1 = Bwd1Smem<S, false>;
         static_assert(L1::total + 1024 <= 228 * 1024, "edge-wise backward ring does not fit in shared memory");
         if (attr_dev != dev) {
-            E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd1_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L1::total));
+            E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd1_kernel<S, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L1::total));
             attr_dev = dev;
         }
-        fast_bwd1_kernel<S><<<n_cta, (S::ET + 1) * 32, L1::total, a.stream>>>(p);  // consumers + one producer warp
+        fast_bwd1_kernel<S, false><<<n_cta, (L1::T * L1::CH + 1) * 32, L1::total, a.stream>>>(p);  // consumers + one producer warp
     } else {
         if (attr_dev != dev) {
             E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));

@@ -226,6 +226,8 @@ class Sig:
                  f"(0 = not generated), ring stages")
         EV = self.cfg.get("EV", V)
         o.append(f"    static constexpr int ET = {self.cfg.get('ET', 0)}, ES = {self.cfg.get('ES', 2)}, EV = {EV};")
+        o.append(f"    // the same for the standalone tensor product: rows per ring slot (0 = not generated), ring slots")
+        o.append(f"    static constexpr int ETR = {self.cfg.get('ETR', 0)}, ESR = {self.cfg.get('ESR', 3)};")
         o.append(f"    using EVec = {{1: 'float', 2: 'float2', 4: 'float4'}}[EV];".replace("{1: 'float', 2: 'float2', 4: 'float4'}[EV]", {1: "float", 2: "float2", 4: "float4"}[EV]))
         o.append(f"    __device__ static __forceinline__ PairRec b_pair_rec(int i) {{ return kBPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float b_rec_val(int i) {{ return kBVal_{self.name}[i]; }}")
@@ -310,7 +312,7 @@ class Sig:
         o.append("        } break;")
         o.append("        }")
         o.append("    }")
-        if self.cfg.get("ET", 0):
+        if self.cfg.get("ET", 0) or self.cfg.get("ETR", 0):
             o += self.emit_bwd_edgewise(slot_of_pair)
         return o
 
