@@ -46,11 +46,11 @@ def measured_peak():
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per call from the ncu captures summarised in
-# profiles/fast_fwd_kernel_water3000.txt, profiles/fast_bwd_kernel_water3000.txt and the launch-list run
+# profiles/fast_fwd_kernel_water3000.txt, profiles/fast_bwd1_kernel_water3000.txt and the launch-list run
 # (specialised kernels, workload water3000).  Other workloads / the generic kernels report null.
 NCU_TRAFFIC = {
     ("water3000", "fwd"): 1.110542e9 + 0.081376e9 + 0.016343e9,          # fast_fwd_kernel + fwd_fixup_kernel
-    ("water3000", "bwd"): 1.261115e9 + 1.362131e9 + 0.330463e9 + 0.0018e9,  # fast_bwd_kernel + bwd_dx_reduce_kernel
+    ("water3000", "bwd"): 1.257002e9 + 1.362881e9 + 0.330463e9 + 0.0018e9,  # fast_bwd1_kernel + bwd_dx_reduce_kernel
 }
 
 
@@ -418,7 +418,7 @@ def main():
         spec = bool(plan.specialised)
         roofs = {"fwd": roof(fb, f_ms, "e3j_conv_fwd call: fast_fwd_kernel (97 %) + fwd_fixup_kernel" if spec
                              else "e3j_conv_fwd call: generic conv_fwd_kernel", "fwd"),
-                 "bwd": roof(bb, b_ms, "e3j_conv_bwd call: fast_bwd_kernel (90 %) + bwd_dx_reduce_kernel" if spec
+                 "bwd": roof(bb, b_ms, "e3j_conv_bwd call: fast_bwd1_kernel (89 %) + bwd_dx_reduce_kernel" if spec
                              else "e3j_conv_bwd call: generic edge + node kernels", "bwd")}
         dominant = roofs["bwd"] if b_ms >= f_ms else roofs["fwd"]
         line = {
