@@ -230,9 +230,12 @@ int e3j_conv_bwd_padded(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges_p
  *   g_x    = grad_x of the backward taken at (sh <- ct_sh)  +  at (w <- ct_w)              [n_nodes,d,N_q]
  *   g_sh   = grad_sh at (x <- ct_x)  +  at (w <- ct_w)                                      [n_edges,d']
  *   g_w    = grad_w at (x <- ct_x)   +  at (sh <- ct_sh)                                    [n_edges,P,N_q]
- * all with the same grad_out; any output may be NULL.  This is the composition the paper describes (three
- * forward and three backward passes of this library plus the sums); the single fused sweep the paper leaves
- * as future work is not built.  rowptr, sender_perm and colptr are required (e3j_graph_prepare); the
+ * all with the same grad_out; any output may be NULL.  In general this is the composition the paper describes
+ * (three forward and three backward passes of this library plus the sums).  For signatures with generated
+ * double-backward kernels, when all three cotangents are given, it is the fused form the paper leaves as future
+ * work: one forward-shaped sweep for gg_out (two terms per coefficient pair) and, if g_x, g_sh and g_w are all
+ * wanted, one edge sweep for them (each reads x, sh, w and their cotangents once).  The results of the two forms
+ * differ by rounding only.  rowptr, sender_perm and colptr are required (e3j_graph_prepare); the
  * workspace (e3j_conv_bwd_bwd_workspace_bytes) also holds one scratch tensor of each output's size. */
 size_t e3j_conv_bwd_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges);
 int e3j_conv_bwd_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,

@@ -448,8 +448,20 @@ int e3j_conv_bwd_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, con
     const size_t n_out = (size_t)n_nodes * plan->D * plan->nq, n_x = (size_t)n_nodes * plan->d * plan->nq;
     const size_t n_sh = (size_t)n_edges * plan->dp, n_w = (size_t)n_edges * plan->P * plan->nq;
 
+    const FastKernels* fk = fast_lookup(plan);
     // cotangent of grad_out: the forward map with one argument replaced by its cotangent, three times
-    if (gg_out) {
+    // (or the fused sweep of a specialised signature)
+    if (gg_out && fk && fk->dbl_out && n_edges > 0 && ct_x && ct_sh && ct_w) {
+        DeviceTables t;
+        if (int s = get_device_tables(plan, t)) return s;
+        const WorkspaceLayout W = layout(plan, n_nodes, n_edges, false);
+        ConvArgs a{};
+        a.status = t.status;
+        a.n_nodes = n_nodes; a.n_edges = n_edges; a.x = x; a.sh = sh; a.w = w;
+        a.senders = senders; a.receivers = receivers; a.rowptr = rowptr; a.out = gg_out;
+        a.workspace = ws + L.fwd + W.scratch; a.workspace_bytes = L.fwd_bytes - W.scratch; a.stream = st;
+        if (int s = fk->dbl_out(a, ct_x, ct_sh, ct_w)) return s;
+    } else if (gg_out) {
         bool first = true;
         const float* xs[3] = {ct_x, x, x};
         const float* ys[3] = {sh, ct_sh, sh};
@@ -469,6 +481,20 @@ int e3j_conv_bwd_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, con
     // cotangents of x, sh, w: the backward map with one primal replaced by its cotangent; each pass yields the
     // two cotangents that are not the replaced argument's own (all three are computed so that the specialised
     // sweep can be used; the third goes to scratch)
+    if (fk && fk->dbl_edges && n_edges > 0 && ct_x && ct_sh && ct_w && g_x && g_sh && g_w) {
+        // one fused sweep instead of the three backward passes below
+        DeviceTables t;
+        if (int s = get_device_tables(plan, t)) return s;
+        const WorkspaceLayout W = layout(plan, n_nodes, n_edges, true);
+        ConvArgs a{};
+        a.status = t.status;
+        a.n_nodes = n_nodes; a.n_edges = n_edges; a.x = x; a.sh = sh; a.w = w;
+        a.senders = senders; a.receivers = receivers; a.rowptr = rowptr;
+        a.sender_perm = sender_perm; a.colptr = colptr; a.grad_out = grad_out;
+        a.grad_x = g_x; a.grad_sh = g_sh; a.grad_w = g_w;
+        a.workspace = ws + L.bwd + W.scratch; a.workspace_bytes = L.bwd_bytes - W.scratch; a.stream = st;
+        return fk->dbl_edges(a, ct_x, ct_sh, ct_w);
+    }
     bool have_x = false, have_sh = false, have_w = false;
     auto put = [&](float* dst, float* tmp, bool& have, size_t n) -> int {
         // result of this pass is in `have ? tmp : dst`; fold it into dst

@@ -34,10 +34,13 @@ struct BwdParams {
     int32_t* status;
     int identity;                      // 1: every edge is its own sender and receiver; dx_edge is then grad_x itself
     const int32_t* n_real;             // padded call: device word holding the number of real edges (else null)
+    // fused double backward only: cotangents of grad_x, grad_sh, grad_w (laid out like x, sh, w)
+    const float* ct_x; const float* ct_sh; const float* ct_w;
 };
 
 template <class S>
 struct BwdSmem {
+    static constexpr bool DBL = false;             // (the producer code is shared with the double-backward forward)
     static constexpr int T = S::BT, NS = S::BS;
     static constexpr int CH = S::NQ / (32 * S::BV);
     static constexpr int NCONS = S::BW * CH;

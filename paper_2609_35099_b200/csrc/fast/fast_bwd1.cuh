@@ -18,6 +18,12 @@
 // warps (a slot of a 100-row signature is 70 KB: three of them, one warp each, keep more bytes in flight than
 // a double-buffered pair would).
 //
+// Fused double backward (DBL = true, graph calls): the same sweep with the cotangents (ux, uy, us) of
+// (grad_x, grad_sh, grad_w) staged beside (x, y, s) -- two sender rows, two weight rows and two A tables per
+// edge -- and the body S::bwd2_edge_all, which yields the cotangents of s and y and this edge's share of the
+// cotangent of x (the message-passing double backward of the paper, its three edge outputs; the cotangent of
+// grad_out is a forward-shaped sum and has its own kernel).
+//
 // Channels beyond one warp's (CH = N_q / (32 EV) > 1): CH warps share an edge, each with its own channels.
 // Only the channel sum of grad_sh joins them: every warp leaves its 16 partial sums in the slot, and the first
 // warp of the edge adds them in warp order once all have arrived (bounded wait on a barrier of their own).
@@ -37,10 +43,13 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-template <class S, bool ROWS>
+template <class S, bool ROWS, bool DBL = false>
 struct Bwd1Smem {
-    static constexpr int T = ROWS ? S::ETR : S::ET, NS = ROWS ? S::ESR : S::ES;
-    static constexpr int CH = S::NQ / (32 * S::EV); // warps per edge
+    static_assert(!(ROWS && DBL), "the fused double backward exists for graph calls only");
+    static constexpr int T = DBL ? S::DT : ROWS ? S::ETR : S::ET, NS = DBL ? S::DS : ROWS ? S::ESR : S::ES;
+    static constexpr int VW = DBL ? S::DV : S::EV;  // channels per lane
+    using Vec = typename VecOf<VW>::type;
+    static constexpr int CH = S::NQ / (32 * VW);    // warps per edge
     static constexpr int NG = ROWS ? NS : 1;        // groups of T * CH consumer warps (ROWS: one per ring slot)
     static constexpr int S_EDGE = S::P * S::NQ;
     static constexpr int X_EDGE = S::DIN * S::NQ;
@@ -54,25 +63,30 @@ struct Bwd1Smem {
     static constexpr size_t off_rcv = off_meta + 16 * NS;                  // int[2 * WIN]
     static constexpr size_t off_snd = off_rcv + 4 * 2 * WIN;               // int[2 * WIN]
     static constexpr size_t off_y = off_snd + 4 * 2 * WIN;                 // float[2 * WIN][DSH]
-    static constexpr size_t off_dm = up(off_y + 4 * 2 * WIN * S::DSH, 128);  // float[NS][D][NQ] (graph calls)
+    static constexpr size_t off_uy = off_y + 4 * 2 * WIN * S::DSH;         // float[2 * WIN][DSH] (DBL)
+    static constexpr size_t off_dm = up(off_uy + (DBL ? 4 * 2 * WIN * S::DSH : 0), 128);  // float[NS][D][NQ] (graph calls)
     static constexpr size_t off_stage = up(off_dm + (ROWS ? 0 : 4 * (size_t)NS * DM_ROW), 128);
+    static constexpr int NIN = DBL ? 2 : 1;         // copies of every per-edge input (DBL: primal and cotangent)
     static constexpr size_t st_s = 0;
-    static constexpr size_t st_x = st_s + 4 * (size_t)T * S_EDGE;
-    static constexpr size_t st_A = st_x + 4 * (size_t)T * X_EDGE;
-    static constexpr size_t st_dy = st_A + 4 * (size_t)T * S::B_APAD;            // float[T][CH][16] (CH > 1)
+    static constexpr size_t st_us = st_s + 4 * (size_t)T * S_EDGE;               // (DBL)
+    static constexpr size_t st_x = st_s + 4 * (size_t)NIN * T * S_EDGE;
+    static constexpr size_t st_ux = st_x + 4 * (size_t)T * X_EDGE;               // (DBL)
+    static constexpr size_t st_A = st_x + 4 * (size_t)NIN * T * X_EDGE;
+    static constexpr size_t st_B = st_A + 4 * (size_t)T * S::B_APAD;             // (DBL)
+    static constexpr size_t st_dy = st_A + 4 * (size_t)NIN * T * S::B_APAD;      // float[T][CH][16] (CH > 1)
     static constexpr size_t st_dm = up(st_dy + (CH > 1 ? 4 * (size_t)T * CH * 16 : 0), 128);   // float[T][D][NQ] (ROWS)
     static constexpr size_t stage_bytes = up(st_dm + (ROWS ? 4 * (size_t)T * DM_ROW : 0), 128);
     static constexpr size_t total = off_stage + NS * stage_bytes;
 };
 
 // ------------------------------------------------------------------------ consumer: one edge per tile
-template <class S, bool ROWS>
+template <class S, bool ROWS, bool DBL>
 __device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char* smem, const int warp, const int lane,
                                               const int64_t e_begin, const int64_t e_end) {
-    using Vec = typename S::EVec;
-    using L = Bwd1Smem<S, ROWS>;
-    constexpr int NS = L::NS;
-    constexpr int NQV = S::NQ / S::EV;
+    using L = Bwd1Smem<S, ROWS, DBL>;
+    using Vec = typename L::Vec;
+    constexpr int NS = L::NS, VW = L::VW;
+    constexpr int NQV = S::NQ / VW;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
     uint64_t* empty = full + NS;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
@@ -92,15 +106,22 @@ __device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char*
         if (j < n_e) {
             const unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
             const int64_t e = e_begin + first + j;
-            const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + j * (L::X_EDGE / S::EV) + vlane;
-            const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + j * (L::S_EDGE / S::EV) + vlane;
+            const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + j * (L::X_EDGE / VW) + vlane;
+            const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + j * (L::S_EDGE / VW) + vlane;
             const float* As = reinterpret_cast<const float*>(st + L::st_A) + j * S::B_APAD;
-            const Vec* dms = (ROWS ? reinterpret_cast<const Vec*>(st + L::st_dm) + j * (L::DM_ROW / S::EV)
+            const Vec* dms = (ROWS ? reinterpret_cast<const Vec*>(st + L::st_dm) + j * (L::DM_ROW / VW)
                                    : reinterpret_cast<const Vec*>(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW)) + vlane;
             Vec dxp[S::DIN];   // both are assigned (not accumulated into) by bwd_edge_all
             float dyl[16];
             Vec* gw = reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + vlane;
-            S::bwd_edge_all(dms, xs, ss, As, dxp, dyl, gw);
+            if constexpr (DBL) {
+                const Vec* uxs = reinterpret_cast<const Vec*>(st + L::st_ux) + j * (L::X_EDGE / VW) + vlane;
+                const Vec* uss = reinterpret_cast<const Vec*>(st + L::st_us) + j * (L::S_EDGE / VW) + vlane;
+                const float* Bs = reinterpret_cast<const float*>(st + L::st_B) + j * S::B_APAD;
+                S::bwd2_edge_all(dms, xs, uxs, ss, uss, As, Bs, dxp, dyl, gw);
+            } else {
+                S::bwd_edge_all(dms, xs, ss, As, dxp, dyl, gw);
+            }
             Vec* dxo = reinterpret_cast<Vec*>(p.dx_edge + (size_t)e * L::X_EDGE) + vlane;
 #pragma unroll
             for (int i = 0; i < S::DIN; ++i) dxo[i * NQV] = dxp[i];
@@ -139,10 +160,10 @@ __device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char*
 }
 
 // ------------------------------------------------------------------------ producer
-template <class S, bool ROWS>
+template <class S, bool ROWS, bool DBL>
 __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char* smem, const int lane,
                                               const int64_t e_begin, const int64_t e_end) {
-    using L = Bwd1Smem<S, ROWS>;
+    using L = Bwd1Smem<S, ROWS, DBL>;
     using Tab = BwdTab<S>;
     constexpr int T = L::T, NS = L::NS, WIN = L::WIN, DSH = S::DSH;
     constexpr int NA = (Tab::APAD + 31) / 32;
@@ -153,6 +174,7 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
     int* rcv_ring = reinterpret_cast<int*>(smem + L::off_rcv);
     int* snd_ring = reinterpret_cast<int*>(smem + L::off_snd);
     float* y_ring = reinterpret_cast<float*>(smem + L::off_y);
+    float* uy_ring = reinterpret_cast<float*>(smem + L::off_uy);
     const int n_tot = (int)(e_end - e_begin);
 
     ASlot tab[NA];   // this lane's A slots (lane, lane + 32, ...)
@@ -179,8 +201,10 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
 #pragma unroll
         for (int j = 0; j < DSH; ++j) {
             const int idx = j * 32 + lane;   // entry of the window's [32][DSH] block
-            if (WIN * w + idx / DSH < n_tot)
+            if (WIN * w + idx / DSH < n_tot) {
                 cp_async4(&y_ring[half * DSH + idx], p.sh + (e_begin + (int64_t)WIN * w) * DSH + idx);
+                if (DBL) cp_async4(&uy_ring[half * DSH + idx], p.ct_sh + (e_begin + (int64_t)WIN * w) * DSH + idx);
+            }
         }
         cp_async_commit();
     };
@@ -229,7 +253,7 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
             int* meta = reinterpret_cast<int*>(smem + L::off_meta) + 4 * stage;
             meta[0] = done; meta[1] = n_e | (last << 8); meta[2] = block;
             // arrival and byte count in one step: the phase cannot complete before the bytes are expected
-            mbar_arrive_expect_tx(&full[stage], (uint32_t)n_e * 4u * (L::S_EDGE + L::X_EDGE + (ROWS ? L::DM_ROW : 0)) +
+            mbar_arrive_expect_tx(&full[stage], (uint32_t)n_e * 4u * (L::NIN * (L::S_EDGE + L::X_EDGE) + (ROWS ? L::DM_ROW : 0)) +
                                                     (new_block ? 4u * L::DM_ROW : 0u));
             if (n_e > 0)
                 bulk_g2s(st + L::st_s, p.w + (size_t)(e_begin + done) * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE,
@@ -243,9 +267,16 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
                 bulk_g2s(st + L::st_dm, p.grad_out + (size_t)(e_begin + done) * L::DM_ROW,
                          (uint32_t)n_e * 4u * L::DM_ROW, &full[stage]);
         } else {
-            if (lane < n_e)
-                bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE,
-                         p.x + (size_t)snd_ring[i & (2 * WIN - 1)] * L::X_EDGE, 4u * L::X_EDGE, &full[stage]);
+            if (lane < n_e) {
+                const size_t snd = (size_t)snd_ring[i & (2 * WIN - 1)];
+                bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE, p.x + snd * L::X_EDGE, 4u * L::X_EDGE, &full[stage]);
+                if (DBL)
+                    bulk_g2s(st + L::st_ux + (size_t)lane * 4 * L::X_EDGE, p.ct_x + snd * L::X_EDGE, 4u * L::X_EDGE,
+                             &full[stage]);
+            }
+            if (DBL && lane == 30 && n_e > 0)
+                bulk_g2s(st + L::st_us, p.ct_w + (size_t)(e_begin + done) * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE,
+                         &full[stage]);
             if (lane == 31 && new_block)
                 bulk_g2s(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW, p.grad_out + (size_t)r0 * L::DM_ROW,
                          4u * L::DM_ROW, &full[stage]);
@@ -253,21 +284,25 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
         armed = t + 1;
         // A[e][slot] = sum over the slot's records of c * y[e][i2]; all loads before the first store
         // (entries of edges beyond n_e are computed from stale data and never read)
-        float* A_t = reinterpret_cast<float*>(st + L::st_A);
-        float a_val[NA][T];
 #pragma unroll
-        for (int k = 0; k < NA; ++k)
+        for (int tbl = 0; tbl < L::NIN; ++tbl) {   // A from the harmonics; DBL: B from their cotangent as well
+            float* A_t = reinterpret_cast<float*>(st + (tbl ? L::st_B : L::st_A));
+            const float* ring = tbl ? uy_ring : y_ring;
+            float a_val[NA][T];
 #pragma unroll
-            for (int e_i = 0; e_i < T; ++e_i) {
-                const float* ye = y_ring + ((done + e_i) & (2 * WIN - 1)) * DSH;
-                a_val[k][e_i] = fmaf(tab[k].c1, ye[tab[k].i2_1], tab[k].c0 * ye[tab[k].i2_0]);
-            }
+            for (int k = 0; k < NA; ++k)
 #pragma unroll
-        for (int k = 0; k < NA; ++k) {
-            const int slot = lane + 32 * k;
-            if (slot < Tab::APAD) {
+                for (int e_i = 0; e_i < T; ++e_i) {
+                    const float* ye = ring + ((done + e_i) & (2 * WIN - 1)) * DSH;
+                    a_val[k][e_i] = fmaf(tab[k].c1, ye[tab[k].i2_1], tab[k].c0 * ye[tab[k].i2_0]);
+                }
 #pragma unroll
-                for (int e_i = 0; e_i < T; ++e_i) A_t[e_i * Tab::APAD + slot] = a_val[k][e_i];
+            for (int k = 0; k < NA; ++k) {
+                const int slot = lane + 32 * k;
+                if (slot < Tab::APAD) {
+#pragma unroll
+                    for (int e_i = 0; e_i < T; ++e_i) A_t[e_i * Tab::APAD + slot] = a_val[k][e_i];
+                }
             }
         }
         __syncwarp();
@@ -280,12 +315,12 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
     if (*abort_flag) drain_copies<L>(smem, armed);
 }
 
-template <class S, bool ROWS>
-__global__ void __launch_bounds__((Bwd1Smem<S, ROWS>::T * Bwd1Smem<S, ROWS>::CH * Bwd1Smem<S, ROWS>::NG + 1) * 32, 1)
+template <class S, bool ROWS, bool DBL = false>
+__global__ void __launch_bounds__((Bwd1Smem<S, ROWS, DBL>::T * Bwd1Smem<S, ROWS, DBL>::CH * Bwd1Smem<S, ROWS, DBL>::NG + 1) * 32, 1)
 fast_bwd1_kernel(const BwdParams p) {
-    using L = Bwd1Smem<S, ROWS>;
+    using L = Bwd1Smem<S, ROWS, DBL>;
     constexpr int T = L::T, NS = L::NS, NCONS = L::T * L::CH * L::NG;
-    static_assert(S::NQ == 32 * S::EV * L::CH, "the channels are dealt out to whole warps");
+    static_assert(S::NQ == 32 * L::VW * L::CH, "the channels are dealt out to whole warps");
     static_assert(S::B_NREC <= 2, "an A slot holds at most two records");
     static_assert(S::DSH <= 16, "harmonics beyond l = 3 need a wider reduction");
 
@@ -307,8 +342,8 @@ fast_bwd1_kernel(const BwdParams p) {
         mbar_fence_init();
     }
     __syncthreads();
-    if (warp == NCONS) bwd1_producer<S, ROWS>(p, smem, lane, e_begin, e_end);
-    else bwd1_consumer<S, ROWS>(p, smem, warp, lane, e_begin, e_end);
+    if (warp == NCONS) bwd1_producer<S, ROWS, DBL>(p, smem, lane, e_begin, e_end);
+    else bwd1_consumer<S, ROWS, DBL>(p, smem, warp, lane, e_begin, e_end);
 }
 
 }  // namespace fast

@@ -124,6 +124,8 @@ struct FwdParams {
     int32_t* status;                   // device status word (0 = fine)
     int identity;                      // 1: every edge is its own sender and receiver (standalone tensor product)
     const int32_t* n_real;             // padded call: device word holding the number of real edges (else null)
+    // fused double backward only: cotangents of grad_x, grad_sh, grad_w (laid out like x, sh, w)
+    const float* ct_x; const float* ct_sh; const float* ct_w;
 };
 
 // Sums the pieces of every receiver row that was split between CTAs, in CTA order.

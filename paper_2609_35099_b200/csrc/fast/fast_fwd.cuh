@@ -27,9 +27,13 @@ namespace e3j {
 namespace fast {
 
 
-template <class S>
+// DBL: the cotangent of grad_out in the double backward, a forward-shaped sum with two terms per coefficient
+// pair (S::fwd2_edge); the ring then holds the cotangents (ux, uy -> B, us) beside (x, y -> A, s).
+template <class S, bool DBL_ = false>
 struct FwdSmem {
-    static constexpr int T = S::FT, NS = S::FS;
+    static constexpr bool DBL = DBL_;
+    static constexpr int NIN = DBL ? 2 : 1;
+    static constexpr int T = DBL ? S::DFT : S::FT, NS = DBL ? S::DFS : S::FS;
     static constexpr int CH = S::NQ / (32 * S::V);
     static constexpr int NCONS = S::FW * CH;       // consumer warps
     static constexpr int S_EDGE = S::P * S::NQ;    // floats of weights per edge
@@ -39,21 +43,25 @@ struct FwdSmem {
     static constexpr size_t off_abort = off_bar + 16 * NS;
     static constexpr size_t off_stage = up(off_abort + 4, 128);
     static constexpr size_t st_s = 0;
-    static constexpr size_t st_x = st_s + 4 * (size_t)T * S_EDGE;
-    static constexpr size_t st_A = st_x + 4 * (size_t)T * X_EDGE;         // float A[T][APAD]
-    static constexpr size_t st_y = st_A + 4 * (size_t)T * S::F_APAD;
-    static constexpr size_t st_r = st_y + 4 * (size_t)T * S::DSH;         // recv[T], change mask
+    static constexpr size_t st_us = st_s + 4 * (size_t)T * S_EDGE;        // (DBL)
+    static constexpr size_t st_x = st_s + 4 * (size_t)NIN * T * S_EDGE;
+    static constexpr size_t st_ux = st_x + 4 * (size_t)T * X_EDGE;        // (DBL)
+    static constexpr size_t st_A = st_x + 4 * (size_t)NIN * T * X_EDGE;   // float A[T][APAD]
+    static constexpr size_t st_B = st_A + 4 * (size_t)T * S::F_APAD;      // (DBL)
+    static constexpr size_t st_y = st_A + 4 * (size_t)NIN * T * S::F_APAD;
+    static constexpr size_t st_uy = st_y + 4 * (size_t)T * S::DSH;        // (DBL)
+    static constexpr size_t st_r = st_y + 4 * (size_t)NIN * T * S::DSH;   // recv[T], change mask
     static constexpr size_t stage_bytes = up(st_r + 4 * (T + 1), 128);
     static constexpr size_t total = off_stage + NS * stage_bytes;
 };
 
 // ------------------------------------------------------------------------ consumer
-template <class S, int G>
+template <class S, int G, bool DBL>
 __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* smem, const int ch, const int warp,
                                              const int lane, const int64_t e_begin, const int64_t e_end,
                                              const int n_tiles, const int64_t n_edges) {
     using Vec = typename VecOf<S::V>::type;
-    using L = FwdSmem<S>;
+    using L = FwdSmem<S, DBL>;
     constexpr int T = L::T, NS = L::NS;
     constexpr int NQV = S::NQ / S::V;
     constexpr int ROW0 = S::f_row0(G), ROW1 = S::f_row0(G + 1);
@@ -119,6 +127,9 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
         const Vec* xs = reinterpret_cast<const Vec*>(st + L::st_x) + vlane;
         const Vec* ss = reinterpret_cast<const Vec*>(st + L::st_s) + vlane;
         const float* As = reinterpret_cast<const float*>(st + L::st_A);
+        const Vec* uxs = reinterpret_cast<const Vec*>(st + L::st_ux) + vlane;   // (DBL)
+        const Vec* uss = reinterpret_cast<const Vec*>(st + L::st_us) + vlane;
+        const float* Bs = reinterpret_cast<const float*>(st + L::st_B);
         // Runs of edges with the same receiver: the inner loop is the bare per-edge body with no receiver
         // test in it (with the test inside, the same body ran 40 % slower), and it is not unrolled (a longer
         // loop costs more in instruction fetch than it saves).
@@ -131,7 +142,12 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
             e_i += run;
 #pragma unroll 1
             for (int j = 0; j < run; ++j) {
-                S::template fwd_edge<G>(acc, xs, ss, As);
+                if constexpr (DBL) {
+                    S::template fwd2_edge<G>(acc, xs, uxs, ss, uss, As, Bs);
+                    uxs += L::X_EDGE / S::V; uss += L::S_EDGE / S::V; Bs += S::F_APAD;
+                } else {
+                    S::template fwd_edge<G>(acc, xs, ss, As);
+                }
                 xs += L::X_EDGE / S::V; ss += L::S_EDGE / S::V; As += S::F_APAD;
             }
         }
@@ -150,16 +166,16 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
     }
 }
 
-template <class S, int G>
+template <class S, int G, bool DBL>
 struct FwdDispatch {
     template <class... Args>
     __device__ static __forceinline__ void run(const int g, Args&&... args) {
-        if (g == G) fwd_consumer<S, G>(args...);
-        else FwdDispatch<S, G + 1>::run(g, args...);
+        if (g == G) fwd_consumer<S, G, DBL>(args...);
+        else FwdDispatch<S, G + 1, DBL>::run(g, args...);
     }
 };
-template <class S>
-struct FwdDispatch<S, S::FW> {
+template <class S, bool DBL>
+struct FwdDispatch<S, S::FW, DBL> {
     template <class... Args>
     __device__ static __forceinline__ void run(const int, Args&&...) {}
 };
@@ -172,10 +188,10 @@ struct FwdTab {
     __device__ static __forceinline__ unsigned char rec_i2(int i) { return S::rec_i2(i); }
 };
 
-template <class S>
-__global__ void __launch_bounds__((S::FW * (S::NQ / (32 * S::V)) + 2) * 32, S::FC)
+template <class S, bool DBL = false>
+__global__ void __launch_bounds__((S::FW * (S::NQ / (32 * S::V)) + 2) * 32, DBL ? S::DFC : S::FC)
 fast_fwd_kernel(const FwdParams p) {
-    using L = FwdSmem<S>;
+    using L = FwdSmem<S, DBL>;
     constexpr int T = L::T, NS = L::NS, NCONS = L::NCONS;
     static_assert(T <= 31, "the change mask is one 32-bit word");
     static_assert(S::F_NREC <= 2, "an A slot holds at most two records");
@@ -199,7 +215,7 @@ fast_fwd_kernel(const FwdParams p) {
     __syncthreads();
     if (warp == NCONS) producer_loop<L, FwdTab<S>, 0>(p, smem, lane, e_begin, e_end, n_tiles);
     else if (warp == NCONS + 1) producer_loop<L, FwdTab<S>, 1>(p, smem, lane, e_begin, e_end, n_tiles);
-    else FwdDispatch<S, 0>::run(warp % S::FW, p, smem, warp / S::FW, warp, lane, e_begin, e_end, n_tiles, n_edges);
+    else FwdDispatch<S, 0, DBL>::run(warp % S::FW, p, smem, warp / S::FW, warp, lane, e_begin, e_end, n_tiles, n_edges);
 }
 
 }  // namespace fast

@@ -177,5 +177,71 @@ int launch_bwd(const ConvArgs& a) {
     return after_launch();
 }
 
+// Fused double backward, edge outputs: the edge-wise sweep over (x, sh, w) and their cotangents, then the
+// sender-ordered sum of the per-edge shares (the scratch is that of launch_bwd).
+template <class S>
+int launch_dbl_edges(const ConvArgs& a, const float* ct_x, const float* ct_sh, const float* ct_w) {
+    using L1 = Bwd1Smem<S, false, true>;
+    static_assert(L1::total + 1024 <= 228 * 1024, "double-backward ring does not fit in shared memory");
+    static_assert(L1::T < 30, "lanes 30 and 31 of the producer issue the tile's shared copies");
+    if (a.workspace_bytes < bwd_scratch_bytes<S>(a.n_nodes, a.n_edges)) return E3J_ERR_WORKSPACE;
+    const int n_cta = sm_count();
+    BwdParams p{};
+    p.x = a.x; p.sh = a.sh; p.w = a.w; p.senders = a.senders; p.receivers = a.receivers;
+    p.ct_x = ct_x; p.ct_sh = ct_sh; p.ct_w = ct_w;
+    p.grad_out = a.grad_out; p.grad_sh = a.grad_sh; p.grad_w = a.grad_w;
+    p.dx_edge = reinterpret_cast<float*>(a.workspace);
+    p.n_nodes = a.n_nodes; p.n_edges = a.n_edges;
+    p.chunk = (a.n_edges + n_cta - 1) / n_cta;
+    p.status = a.status;
+    static thread_local int attr_dev = -1;
+    int dev = 0;
+    E3J_CUDA_TRY(cudaGetDevice(&dev));
+    if (attr_dev != dev) {
+        E3J_CUDA_TRY(cudaFuncSetAttribute(fast_bwd1_kernel<S, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L1::total));
+        attr_dev = dev;
+    }
+    fast_bwd1_kernel<S, false, true><<<n_cta, (L1::T * L1::CH + 1) * 32, L1::total, a.stream>>>(p);
+    if (int s = after_launch()) return s;
+    const int64_t blocks = std::min<int64_t>(a.n_nodes, (int64_t)1 << 30);
+    bwd_dx_reduce_kernel<<<(int)blocks, S::DIN * S::NQ / 4, 0, a.stream>>>(a.n_nodes, S::DIN * S::NQ / 4,
+        reinterpret_cast<const float4*>(p.dx_edge), a.sender_perm, a.colptr, reinterpret_cast<float4*>(a.grad_x));
+    return after_launch();
+}
+
+// Fused double backward, cotangent of grad_out: the forward sweep with two terms per coefficient pair, written
+// to a.out (scratch and fix-up as in launch_fwd).
+template <class S>
+int launch_dbl_out(const ConvArgs& a, const float* ct_x, const float* ct_sh, const float* ct_w) {
+    using L = FwdSmem<S, true>;
+    static_assert(L::total * S::DFC + 1024 * S::DFC <= 228 * 1024, "double-backward forward ring does not fit in shared memory");
+    static_assert(S::DFC <= S::FC, "the scratch is sized for the forward's CTA count");
+    static_assert(L::T < 31, "lane 31 of the copy warp issues the tile's second weight copy");
+    const int n_cta = sm_count() * S::DFC;
+    if (a.workspace_bytes < fwd_scratch_need<S>(n_cta)) return E3J_ERR_WORKSPACE;
+    static thread_local int attr_dev = -1;
+    int dev = 0;
+    E3J_CUDA_TRY(cudaGetDevice(&dev));
+    if (attr_dev != dev) {
+        E3J_CUDA_TRY(cudaFuncSetAttribute(fast_fwd_kernel<S, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));
+        attr_dev = dev;
+    }
+    FwdParams p{};
+    p.x = a.x; p.sh = a.sh; p.w = a.w; p.senders = a.senders; p.receivers = a.receivers; p.out = a.out;
+    p.ct_x = ct_x; p.ct_sh = ct_sh; p.ct_w = ct_w;
+    p.n_nodes = a.n_nodes; p.n_edges = a.n_edges;
+    const int64_t per = (a.n_edges + n_cta - 1) / n_cta;
+    p.chunk = (per + 3) / 4 * 4;
+    p.part_recv = reinterpret_cast<int32_t*>(a.workspace);
+    p.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(a.workspace) + kPartRecvBytes);
+    p.status = a.status;
+    constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 2) * 32;  // consumers + two producer warps
+    fast_fwd_kernel<S, true><<<n_cta, threads, L::total, a.stream>>>(p);
+    if (int s = after_launch()) return s;
+    fwd_fixup_kernel<<<n_cta, 256, 0, a.stream>>>(n_cta, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),
+                                                 p.part_recv, reinterpret_cast<float4*>(a.out));
+    return after_launch();
+}
+
 }  // namespace fast
 }  // namespace e3j

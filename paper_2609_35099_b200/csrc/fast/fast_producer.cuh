@@ -7,7 +7,8 @@
 // (combined_producer: less hot code, one warp fewer).
 //
 // L describes the shared-memory ring (T, NS, S_EDGE, X_EDGE, off_bar, off_abort, off_stage, stage_bytes and the
-// offsets st_s / st_x / st_A / st_y / st_r inside a stage); Tab gives the A-slot tables of the kernel
+// offsets st_s / st_x / st_A / st_y / st_r inside a stage; with L::DBL also st_us / st_ux / st_B / st_uy for the
+// cotangents that the fused double backward stages beside the primal inputs); Tab gives the A-slot tables of the kernel
 // (APAD, DSH, pair_rec, rec_val, rec_i2); P is the kernel's parameter struct (x, sh, w, senders, receivers,
 // identity, status).
 #pragma once
@@ -51,12 +52,19 @@ struct CopyPart {
         const int n_e = (int)min((int64_t)T, e_end - e0);
         if (lane == 0) {
             // arrival and byte count in one step: the phase cannot complete before the bytes are expected
-            mbar_arrive_expect_tx(full_bar, (uint32_t)n_e * 4u * (L::S_EDGE + L::X_EDGE));
+            mbar_arrive_expect_tx(full_bar, (uint32_t)n_e * 4u * (L::DBL ? 2u : 1u) * (L::S_EDGE + L::X_EDGE));
             bulk_g2s(st + L::st_s, p.w + (size_t)e0 * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE, full_bar);
         }
         if (lane < n_e)
             bulk_g2s(st + L::st_x + (size_t)lane * 4 * L::X_EDGE, p.x + (size_t)snd_a * L::X_EDGE, 4u * L::X_EDGE,
                      full_bar);
+        if constexpr (L::DBL) {
+            if (lane == 31)
+                bulk_g2s(st + L::st_us, p.ct_w + (size_t)e0 * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE, full_bar);
+            if (lane < n_e)
+                bulk_g2s(st + L::st_ux + (size_t)lane * 4 * L::X_EDGE, p.ct_x + (size_t)snd_a * L::X_EDGE,
+                         4u * L::X_EDGE, full_bar);
+        }
         snd_a = snd_b;
         load(t + 2, snd_b);   // two tiles ahead of its use
     }
@@ -75,6 +83,7 @@ struct TablePart {
     ASlot tab[NA];              // this lane's A slots (lane, lane + 32, ...)
     int rcv_a = -1, rcv_b = -1; // receiver ids of the next two tiles
     float y_a[YPL], y_b[YPL];   // harmonics of the next two tiles
+    float uy_a[L::DBL ? YPL : 1], uy_b[L::DBL ? YPL : 1];   // and their cotangents (double backward)
     int last_rcv = -1;
 
     __device__ __forceinline__ TablePart(const P& p_, int lane_, int64_t b, int64_t e, int n)
@@ -92,6 +101,17 @@ struct TablePart {
         }
         load(0, rcv_a, y_a);
         load(1, rcv_b, y_b);
+        if constexpr (L::DBL) { load_ct(0, uy_a); load_ct(1, uy_b); }
+    }
+    __device__ __forceinline__ void load_ct(int t, float (&yv)[L::DBL ? YPL : 1]) {
+        if (t >= n_tiles) return;
+        const int64_t e0 = e_begin + (int64_t)t * T;
+        const int n_e = (int)min((int64_t)T, e_end - e0);
+#pragma unroll
+        for (int i = 0; i < (L::DBL ? YPL : 0); ++i) {
+            const int idx = i * 32 + lane;
+            if (idx < n_e * Tab::DSH) yv[i] = p.ct_sh[e0 * Tab::DSH + idx];
+        }
     }
     __device__ __forceinline__ void load(int t, int& rcv, float (&yv)[YPL]) {
         if (t >= n_tiles) return;
@@ -121,6 +141,14 @@ struct TablePart {
             const int idx = i * 32 + lane;
             if (idx < n_e * Tab::DSH) y_t[idx] = y_a[i];
         }
+        if constexpr (L::DBL) {
+            float* uy_t = reinterpret_cast<float*>(st + L::st_uy);
+#pragma unroll
+            for (int i = 0; i < YPL; ++i) {
+                const int idx = i * 32 + lane;
+                if (idx < n_e * Tab::DSH) uy_t[idx] = uy_a[i];
+            }
+        }
         __syncwarp();
         // A[e][slot] = sum over the slot's records of c * y[e][i2]: contracted once per edge here, so that
         // the consumers' per-channel loop never touches a coefficient.  All loads come before the first
@@ -143,11 +171,35 @@ struct TablePart {
                 for (int e_i = 0; e_i < T; ++e_i) A_t[e_i * Tab::APAD + slot] = a_val[i][e_i];
             }
         }
+        if constexpr (L::DBL) {   // the same contraction with the cotangent of the harmonics: B
+            float* B_t = reinterpret_cast<float*>(st + L::st_B);
+            const float* uy_t = reinterpret_cast<const float*>(st + L::st_uy);
+#pragma unroll
+            for (int i = 0; i < NA; ++i)
+#pragma unroll
+                for (int e_i = 0; e_i < T; ++e_i) {
+                    const float* ye = uy_t + e_i * Tab::DSH;
+                    a_val[i][e_i] = fmaf(tab[i].c1, ye[tab[i].i2_1], tab[i].c0 * ye[tab[i].i2_0]);
+                }
+#pragma unroll
+            for (int i = 0; i < NA; ++i) {
+                const int slot = lane + 32 * i;
+                if (slot < Tab::APAD) {
+#pragma unroll
+                    for (int e_i = 0; e_i < T; ++e_i) B_t[e_i * Tab::APAD + slot] = a_val[i][e_i];
+                }
+            }
+        }
         __syncwarp();
         rcv_a = rcv_b;
 #pragma unroll
         for (int i = 0; i < YPL; ++i) y_a[i] = y_b[i];
         load(t + 2, rcv_b, y_b);
+        if constexpr (L::DBL) {
+#pragma unroll
+            for (int i = 0; i < YPL; ++i) uy_a[i] = uy_b[i];
+            load_ct(t + 2, uy_b);
+        }
     }
 };
 

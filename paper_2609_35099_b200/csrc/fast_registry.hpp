@@ -16,6 +16,12 @@ struct FastKernels {
     int (*tp_fwd)(int64_t rows, const float* x1, const float* x2, const float* w, float* out, cudaStream_t);
     int (*tp_bwd)(int64_t rows, const float* x1, const float* x2, const float* w, const float* g,
                   float* gx1, float* gx2, float* gw, cudaStream_t);
+    // fused double backward (null: the caller composes it from conv_fwd and conv_bwd).  Cotangents of
+    // (grad_x, grad_sh, grad_w) in, both need the scratch of conv_bwd / conv_fwd respectively:
+    // dbl_edges writes the cotangents of x, sh, w into args.grad_x / grad_sh / grad_w,
+    // dbl_out the cotangent of grad_out into args.out.
+    int (*dbl_edges)(const ConvArgs&, const float* ct_x, const float* ct_sh, const float* ct_w);
+    int (*dbl_out)(const ConvArgs&, const float* ct_x, const float* ct_sh, const float* ct_w);
 };
 
 // Index of the entry generated for `signature`, or -1.

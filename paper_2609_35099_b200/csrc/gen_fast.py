@@ -228,6 +228,10 @@ class Sig:
         o.append(f"    static constexpr int ET = {self.cfg.get('ET', 0)}, ES = {self.cfg.get('ES', 2)}, EV = {EV};")
         o.append(f"    // the same for the standalone tensor product: rows per ring slot (0 = not generated), ring slots")
         o.append(f"    static constexpr int ETR = {self.cfg.get('ETR', 0)}, ESR = {self.cfg.get('ESR', 3)};")
+        o.append(f"    // fused double backward (edge outputs): edges per tile (0 = not generated), ring stages")
+        DV = self.cfg.get("DV", EV)
+        o.append(f"    static constexpr int DT = {self.cfg.get('DT', 0)}, DS = {self.cfg.get('DS', 2)}, DV = {DV};")
+        o.append(f"    using DVec = {{1: 'float', 2: 'float2', 4: 'float4'}}[DV];".replace("{1: 'float', 2: 'float2', 4: 'float4'}[DV]", {1: "float", 2: "float2", 4: "float4"}[DV]))
         o.append(f"    using EVec = {{1: 'float', 2: 'float2', 4: 'float4'}}[EV];".replace("{1: 'float', 2: 'float2', 4: 'float4'}[EV]", {1: "float", 2: "float2", 4: "float4"}[EV]))
         o.append(f"    __device__ static __forceinline__ PairRec b_pair_rec(int i) {{ return kBPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float b_rec_val(int i) {{ return kBVal_{self.name}[i]; }}")
@@ -314,6 +318,8 @@ class Sig:
         o.append("    }")
         if self.cfg.get("ET", 0) or self.cfg.get("ETR", 0):
             o += self.emit_bwd_edgewise(slot_of_pair)
+        if self.cfg.get("DT", 0):
+            o += self.emit_bwd2_edgewise(slot_of_pair)
         return o
 
     def emit_bwd_edgewise(self, slot_of_pair):
@@ -380,6 +386,79 @@ class Sig:
         o.append("    }")
         return o
 
+    def emit_bwd2_edgewise(self, slot_of_pair):
+        """Edge outputs of the double backward in one sweep, one warp per edge.  With the cotangents (ux, uy, us)
+        of (grad_x, grad_sh, grad_w), A = C y, B = C uy, g = grad_out[receiver]:
+          v[k,i1] = sum_i0 A g[i0],  v2[k,i1] = sum_i0 B g[i0],  sxu[k,i1] = s[k] ux[i1] + us[k] x[i1]
+          d_s[k]  = sum_i1 ux[i1] v + x[i1] v2;   d_x[i1] = sum_k us[k] v + s[k] v2;
+          d_y[i2] = sum C g[i0] sxu[k,i1]."""
+        o = []
+        o.append(f"    __device__ static __forceinline__ void bwd2_edge_all(const DVec* __restrict__ dms, const DVec* __restrict__ xs, "
+                 f"const DVec* __restrict__ uxs, const DVec* __restrict__ ss, const DVec* __restrict__ uss, "
+                 f"const float* __restrict__ As, const float* __restrict__ Bs, DVec (&dxp)[DIN], float (&dyl)[16], "
+                 f"DVec* __restrict__ gw) {{")
+        o.append(f"        constexpr int NQV = NQ / DV;")
+        for i1 in range(self.DIN):
+            o.append(f"        const DVec x{i1} = xs[{i1} * NQV];")
+            o.append(f"        const DVec ux{i1} = uxs[{i1} * NQV];")
+        loaded_a, dx_touched, dy_touched = set(), set(), set()
+        for k in range(self.P):
+            p = self.paths[k]
+            prow = list(self.path_rows(k))
+            used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
+            o.append(f"        const DVec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
+            o.append(f"        const DVec us{k} = uss[{k} * NQV];")
+            for i1 in used:
+                o.append(f"        DVec sxu{k}_{i1} = vmul(s{k}, ux{i1}); vfma(sxu{k}_{i1}, us{k}, x{i1});")
+                o.append(f"        DVec v{k}_{i1}; vzero(v{k}_{i1});")
+                o.append(f"        DVec w{k}_{i1}; vzero(w{k}_{i1});")
+            depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
+            have = set()
+            for j in range(depth):
+                for row in prow:
+                    if j >= len(self.pairs_of(row, k)):
+                        continue
+                    if row not in have:
+                        have.add(row)
+                        o.append(f"        const DVec d{k}_{row} = dms[{row} * NQV];")
+                    pi = self.pairs_of(row, k)[j]
+                    slot = slot_of_pair[pi]
+                    q, lane = slot // 4, "xyzw"[slot % 4]
+                    if q not in loaded_a:
+                        loaded_a.add(q)
+                        o.append(f"        const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
+                        o.append(f"        const float4 b{q} = *reinterpret_cast<const float4*>(Bs + {4 * q});")
+                    i1 = self.pairs[pi][1]
+                    o.append(f"        vfma(v{k}_{i1}, a{q}.{lane}, d{k}_{row});")
+                    o.append(f"        vfma(w{k}_{i1}, b{q}.{lane}, d{k}_{row});")
+                    o.append(f"        {{ const float t = vdot(sxu{k}_{i1}, d{k}_{row});")
+                    for i2, c in self.pairs[pi][3]:
+                        if i2 in dy_touched:
+                            o.append(f"          dyl[{i2}] = fmaf({fmt_float(c)}, t, dyl[{i2}]);")
+                        else:
+                            dy_touched.add(i2)
+                            o.append(f"          dyl[{i2}] = {fmt_float(c)} * t;")
+                    o.append("        }")
+            first = used[0]
+            o.append(f"        DVec ds{k} = vmul(ux{first}, v{k}_{first}); vfma(ds{k}, x{first}, w{k}_{first});")
+            for i1 in used[1:]:
+                o.append(f"        vfma(ds{k}, ux{i1}, v{k}_{i1}); vfma(ds{k}, x{i1}, w{k}_{i1});")
+            o.append(f"        gw[{k} * NQV] = ds{k};")
+            for i1 in used:
+                if i1 in dx_touched:
+                    o.append(f"        vfma(dxp[{i1}], us{k}, v{k}_{i1}); vfma(dxp[{i1}], s{k}, w{k}_{i1});")
+                else:
+                    dx_touched.add(i1)
+                    o.append(f"        dxp[{i1}] = vmul(us{k}, v{k}_{i1}); vfma(dxp[{i1}], s{k}, w{k}_{i1});")
+        for i1 in range(self.DIN):
+            if i1 not in dx_touched:
+                o.append(f"        vzero(dxp[{i1}]);")
+        for i2 in range(16):
+            if i2 not in dy_touched:
+                o.append(f"        dyl[{i2}] = 0.f;")
+        o.append("    }")
+        return o
+
     def emit(self) -> str:
         V, NQ = self.V, self.NQ
         FW, FT, FS, FC = self.cfg["FW"], self.cfg["FT"], self.cfg["FS"], self.cfg["FC"]
@@ -431,6 +510,8 @@ class Sig:
         o.append(f"    static constexpr int NQ = {NQ}, DIN = {self.DIN}, DSH = {self.DSH}, P = {self.P}, D = {self.D};")
         o.append(f"    static constexpr int NNZ = {self.NNZ}, NPAIR = {len(self.pairs)}, V = {V};")
         o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, FC = {FC}, F_RMAX = {rmax}, F_APAD = {len(slots)}, F_NREC = {max(c for _, c in pair_tab)}, F_NPMAX = {max(a0[g + 1] - a0[g] for g in range(FW))}, F_MAXREG = {self.cfg.get("F_MAXREG", 255)};")
+        o.append(f"    // fused double backward (cotangent of grad_out): tile, stages, CTAs per SM (DFT = 0: not generated)")
+        o.append(f"    static constexpr int DFT = {self.cfg.get('DFT', 0)}, DFS = {self.cfg.get('DFS', 2)}, DFC = {self.cfg.get('DFC', 1)};")
         o.append(f"    using Vec = {vec};")
         o.append(f"    __device__ static __forceinline__ PairRec pair_rec(int i) {{ return kPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float rec_val(int i) {{ return kVal_{self.name}[i]; }}")
@@ -488,6 +569,53 @@ class Sig:
             o.append("        }")
         o.append("    }")
 
+        # ---- fwd2_edge: cotangent of grad_out in the double backward,
+        # acc[i0] += A[i0,i1] (s ux[i1] + us x[i1]) + B[i0,i1] (s x[i1]),  A = C y, B = C uy
+        if self.cfg.get("DFT", 0):
+            o.append(f"    template <int G>")
+            o.append(f"    __device__ static __forceinline__ void fwd2_edge(Vec (&acc)[F_RMAX], "
+                     f"const Vec* __restrict__ xs, const Vec* __restrict__ uxs, const Vec* __restrict__ ss, "
+                     f"const Vec* __restrict__ uss, const float* __restrict__ As, const float* __restrict__ Bs) {{")
+            o.append(f"        constexpr int NQV = NQ / V;")
+            for g in range(FW):
+                o.append(f"        if constexpr (G == {g}) {{")
+                rows = range(bounds[g], bounds[g + 1])
+                need_x = sorted({self.pairs[pi][1] for row in rows for pi in self.row_pairs[row]})
+                for i1 in need_x:
+                    o.append(f"            const Vec x{i1} = xs[{i1} * NQV];")
+                    o.append(f"            const Vec ux{i1} = uxs[{i1} * NQV];")
+                loaded_a = set()
+                paths_here = []
+                for row in rows:
+                    for k in self.row_paths[row]:
+                        if k not in paths_here:
+                            paths_here.append(k)
+                for k in paths_here:
+                    prow = [r2 for r2 in rows if self.pairs_of(r2, k)]
+                    o.append(f"            const Vec s{k} = ss[{k} * NQV];")
+                    o.append(f"            const Vec us{k} = uss[{k} * NQV];")
+                    used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
+                    for i1 in used:
+                        o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                        o.append(f"            Vec sxu{k}_{i1} = vmul(s{k}, ux{i1}); vfma(sxu{k}_{i1}, us{k}, x{i1});")
+                    depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
+                    for j in range(depth):
+                        for row in prow:
+                            if j >= len(self.pairs_of(row, k)):
+                                continue
+                            pi = self.pairs_of(row, k)[j]
+                            slot = slot_of_pair[pi]
+                            q, lane = slot // 4, "xyzw"[slot % 4]
+                            if q not in loaded_a:
+                                loaded_a.add(q)
+                                o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
+                                o.append(f"            const float4 b{q} = *reinterpret_cast<const float4*>(Bs + {4 * q});")
+                            i1 = self.pairs[pi][1]
+                            o.append(f"            vfma(acc[{row - bounds[g]}], a{q}.{lane}, sxu{k}_{i1});")
+                            o.append(f"            vfma(acc[{row - bounds[g]}], b{q}.{lane}, sx{k}_{i1});")
+                o.append("        }")
+            o.append("    }")
+
         # ---- fwd_store
         o.append(f"    // writes the group's rows to dst[r * stride] (dst already offset by the lane and the first row)")
         o.append(f"    template <int G>")
@@ -509,9 +637,13 @@ class Sig:
         if bwd_lines:
             o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, &fast::bwd_scratch_bytes<fast::{S}>, "
                      f"&fast::launch_fwd<fast::{S}>, &fast::launch_bwd<fast::{S}>, &fast::launch_tp_fwd<fast::{S}>, "
-                     f"&fast::launch_tp_bwd<fast::{S}>}};")
+                     f"&fast::launch_tp_bwd<fast::{S}>,")
+            dbl_e = f"&fast::launch_dbl_edges<fast::{S}>" if self.cfg.get("DT", 0) else "nullptr"
+            dbl_o = f"&fast::launch_dbl_out<fast::{S}>" if self.cfg.get("DFT", 0) else "nullptr"
+            o.append(f"    {dbl_e}, {dbl_o}}};")
         else:
-            o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, nullptr, &fast::launch_fwd<fast::{S}>, nullptr, nullptr, nullptr}};")
+            o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, nullptr, &fast::launch_fwd<fast::{S}>, nullptr, nullptr, nullptr, "
+                     f"nullptr, nullptr}};")
         o.append("}  // namespace e3j")
         return "\n".join(o) + "\n"
 

@@ -334,7 +334,7 @@ def test_collapsed_output_multiplicities(config, n_atoms):
 
 
 @pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
-@pytest.mark.parametrize("config,n_atoms", [(1, None), (2, 192)])
+@pytest.mark.parametrize("config,n_atoms", [(1, None), (2, 192), (2, 1200)])
 def test_double_backward(config, n_atoms, flags):
     """Cotangents of the backward's inputs against the oracle; a missing cotangent is zero; outputs that are
     not wanted are skipped; two runs give the same bits."""
