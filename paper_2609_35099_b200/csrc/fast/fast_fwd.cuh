@@ -34,7 +34,8 @@ struct FwdSmem {
     static constexpr bool DBL = DBL_;
     static constexpr int NIN = DBL ? 2 : 1;
     static constexpr int T = DBL ? S::DFT : S::FT, NS = DBL ? S::DFS : S::FS;
-    static constexpr int CH = S::NQ / (32 * S::V);
+    static constexpr int VW = DBL ? S::DFV : S::V;   // channels per lane
+    static constexpr int CH = S::NQ / (32 * VW);
     static constexpr int NCONS = S::FW * CH;       // consumer warps
     static constexpr int S_EDGE = S::P * S::NQ;    // floats of weights per edge
     static constexpr int X_EDGE = S::DIN * S::NQ;  // floats of one sender row
@@ -60,10 +61,10 @@ template <class S, int G, bool DBL>
 __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* smem, const int ch, const int warp,
                                              const int lane, const int64_t e_begin, const int64_t e_end,
                                              const int n_tiles, const int64_t n_edges) {
-    using Vec = typename VecOf<S::V>::type;
     using L = FwdSmem<S, DBL>;
+    using Vec = typename VecOf<L::VW>::type;
     constexpr int T = L::T, NS = L::NS;
-    constexpr int NQV = S::NQ / S::V;
+    constexpr int NQV = S::NQ / L::VW;
     constexpr int ROW0 = S::f_row0(G), ROW1 = S::f_row0(G + 1);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
     uint64_t* empty = full + NS;
@@ -144,11 +145,11 @@ __device__ __forceinline__ void fwd_consumer(const FwdParams& p, unsigned char* 
             for (int j = 0; j < run; ++j) {
                 if constexpr (DBL) {
                     S::template fwd2_edge<G>(acc, xs, uxs, ss, uss, As, Bs);
-                    uxs += L::X_EDGE / S::V; uss += L::S_EDGE / S::V; Bs += S::F_APAD;
+                    uxs += L::X_EDGE / L::VW; uss += L::S_EDGE / L::VW; Bs += S::F_APAD;
                 } else {
                     S::template fwd_edge<G>(acc, xs, ss, As);
                 }
-                xs += L::X_EDGE / S::V; ss += L::S_EDGE / S::V; As += S::F_APAD;
+                xs += L::X_EDGE / L::VW; ss += L::S_EDGE / L::VW; As += S::F_APAD;
             }
         }
         __syncwarp();
@@ -189,7 +190,7 @@ struct FwdTab {
 };
 
 template <class S, bool DBL = false>
-__global__ void __launch_bounds__((S::FW * (S::NQ / (32 * S::V)) + 2) * 32, DBL ? S::DFC : S::FC)
+__global__ void __launch_bounds__((FwdSmem<S, DBL>::NCONS + 2) * 32, DBL ? S::DFC : S::FC)
 fast_fwd_kernel(const FwdParams p) {
     using L = FwdSmem<S, DBL>;
     constexpr int T = L::T, NS = L::NS, NCONS = L::NCONS;

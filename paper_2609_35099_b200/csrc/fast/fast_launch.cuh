@@ -235,7 +235,7 @@ int launch_dbl_out(const ConvArgs& a, const float* ct_x, const float* ct_sh, con
     p.part_recv = reinterpret_cast<int32_t*>(a.workspace);
     p.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(a.workspace) + kPartRecvBytes);
     p.status = a.status;
-    constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 2) * 32;  // consumers + two producer warps
+    constexpr int threads = (L::NCONS + 2) * 32;  // consumers + two producer warps
     fast_fwd_kernel<S, true><<<n_cta, threads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
     fwd_fixup_kernel<<<n_cta, 256, 0, a.stream>>>(n_cta, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),

@@ -511,7 +511,10 @@ class Sig:
         o.append(f"    static constexpr int NNZ = {self.NNZ}, NPAIR = {len(self.pairs)}, V = {V};")
         o.append(f"    static constexpr int FW = {FW}, FT = {FT}, FS = {FS}, FC = {FC}, F_RMAX = {rmax}, F_APAD = {len(slots)}, F_NREC = {max(c for _, c in pair_tab)}, F_NPMAX = {max(a0[g + 1] - a0[g] for g in range(FW))}, F_MAXREG = {self.cfg.get("F_MAXREG", 255)};")
         o.append(f"    // fused double backward (cotangent of grad_out): tile, stages, CTAs per SM (DFT = 0: not generated)")
-        o.append(f"    static constexpr int DFT = {self.cfg.get('DFT', 0)}, DFS = {self.cfg.get('DFS', 2)}, DFC = {self.cfg.get('DFC', 1)};")
+        DFV = self.cfg.get("DFV", V)
+        dfvec = {1: "float", 2: "float2", 4: "float4"}[DFV]
+        o.append(f"    static constexpr int DFT = {self.cfg.get('DFT', 0)}, DFS = {self.cfg.get('DFS', 2)}, DFC = {self.cfg.get('DFC', 1)}, DFV = {DFV};")
+        o.append(f"    using DFVec = {dfvec};")
         o.append(f"    using Vec = {vec};")
         o.append(f"    __device__ static __forceinline__ PairRec pair_rec(int i) {{ return kPair_{self.name}[i]; }}")
         o.append(f"    __device__ static __forceinline__ float rec_val(int i) {{ return kVal_{self.name}[i]; }}")
@@ -573,17 +576,17 @@ class Sig:
         # acc[i0] += A[i0,i1] (s ux[i1] + us x[i1]) + B[i0,i1] (s x[i1]),  A = C y, B = C uy
         if self.cfg.get("DFT", 0):
             o.append(f"    template <int G>")
-            o.append(f"    __device__ static __forceinline__ void fwd2_edge(Vec (&acc)[F_RMAX], "
-                     f"const Vec* __restrict__ xs, const Vec* __restrict__ uxs, const Vec* __restrict__ ss, "
-                     f"const Vec* __restrict__ uss, const float* __restrict__ As, const float* __restrict__ Bs) {{")
-            o.append(f"        constexpr int NQV = NQ / V;")
+            o.append(f"    __device__ static __forceinline__ void fwd2_edge(DFVec (&acc)[F_RMAX], "
+                     f"const DFVec* __restrict__ xs, const DFVec* __restrict__ uxs, const DFVec* __restrict__ ss, "
+                     f"const DFVec* __restrict__ uss, const float* __restrict__ As, const float* __restrict__ Bs) {{")
+            o.append(f"        constexpr int NQV = NQ / DFV;")
             for g in range(FW):
                 o.append(f"        if constexpr (G == {g}) {{")
                 rows = range(bounds[g], bounds[g + 1])
                 need_x = sorted({self.pairs[pi][1] for row in rows for pi in self.row_pairs[row]})
                 for i1 in need_x:
-                    o.append(f"            const Vec x{i1} = xs[{i1} * NQV];")
-                    o.append(f"            const Vec ux{i1} = uxs[{i1} * NQV];")
+                    o.append(f"            const DFVec x{i1} = xs[{i1} * NQV];")
+                    o.append(f"            const DFVec ux{i1} = uxs[{i1} * NQV];")
                 loaded_a = set()
                 paths_here = []
                 for row in rows:
@@ -592,12 +595,12 @@ class Sig:
                             paths_here.append(k)
                 for k in paths_here:
                     prow = [r2 for r2 in rows if self.pairs_of(r2, k)]
-                    o.append(f"            const Vec s{k} = ss[{k} * NQV];")
-                    o.append(f"            const Vec us{k} = uss[{k} * NQV];")
+                    o.append(f"            const DFVec s{k} = ss[{k} * NQV];")
+                    o.append(f"            const DFVec us{k} = uss[{k} * NQV];")
                     used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
                     for i1 in used:
-                        o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
-                        o.append(f"            Vec sxu{k}_{i1} = vmul(s{k}, ux{i1}); vfma(sxu{k}_{i1}, us{k}, x{i1});")
+                        o.append(f"            const DFVec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                        o.append(f"            DFVec sxu{k}_{i1} = vmul(s{k}, ux{i1}); vfma(sxu{k}_{i1}, us{k}, x{i1});")
                     depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
                     for j in range(depth):
                         for row in prow:
@@ -618,8 +621,8 @@ class Sig:
 
         # ---- fwd_store
         o.append(f"    // writes the group's rows to dst[r * stride] (dst already offset by the lane and the first row)")
-        o.append(f"    template <int G>")
-        o.append(f"    __device__ static __forceinline__ void fwd_store(const Vec (&acc)[F_RMAX], Vec* __restrict__ dst, const int stride) {{")
+        o.append(f"    template <int G, class VecT>")
+        o.append(f"    __device__ static __forceinline__ void fwd_store(const VecT (&acc)[F_RMAX], VecT* __restrict__ dst, const int stride) {{")
         for g in range(FW):
             o.append(f"        if constexpr (G == {g}) {{")
             for row in range(bounds[g], bounds[g + 1]):
