@@ -40,6 +40,12 @@
  *   - There is no CPU fallback.  Without a usable CUDA device every compute call
  *     returns E3J_ERR_CUDA.
  *
+ * Alignment: arrays with a channel axis (x, w, out, grad_out and their gradients
+ * and cotangents) are read and written as 128-bit vectors and by 16-byte bulk
+ * copies, so they must start on a 16-byte boundary; a compute call given a
+ * misaligned one returns E3J_ERR_INVALID_ARG without launching anything.  The
+ * harmonics (sh) and the index arrays need only their natural 4-byte alignment.
+ *
  * Errors: every function returns an int status (0 = E3J_OK, negative = error);
  * nothing throws across this boundary.  e3j_status_string() names a status,
  * e3j_last_cuda_error() returns the cudaError_t behind the last E3J_ERR_CUDA
@@ -57,7 +63,8 @@ extern "C" {
 
 enum {
     E3J_OK = 0,
-    E3J_ERR_INVALID_ARG = -1,   /* NULL pointer, negative size, capacity too small        */
+    E3J_ERR_INVALID_ARG = -1,   /* NULL pointer, negative size, capacity too small; compute
+                                   calls: a per-channel array not 16-byte aligned            */
     E3J_ERR_BAD_IRREPS = -2,    /* descriptor string does not parse                         */
     E3J_ERR_MUL_NOT_UNIFORM = -3, /* input irreps must share one multiplicity (= N_q)       */
     E3J_ERR_UNSUPPORTED = -4,   /* a dimension exceeds 255, l > 8, nothing couples; compute

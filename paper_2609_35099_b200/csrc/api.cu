@@ -1,6 +1,7 @@
 // C ABI of libe3j: argument checking, device-table upload, kernel dispatch.
 #include <algorithm>
 #include <cstring>
+#include <initializer_list>
 #include <new>
 
 #include "common.cuh"
@@ -169,6 +170,14 @@ DoubleBwdLayout dbl_layout(const e3j_plan* plan, int64_t n_nodes, int64_t n_edge
     return L;
 }
 
+// Channel rows are read and written as 128-bit vectors and by 16-byte bulk copies: every per-channel array
+// must start on a 16-byte boundary (NULL = absent is fine).  A misaligned pointer is refused on the host.
+bool aligned16(std::initializer_list<const void*> ptrs) {
+    for (const void* q : ptrs)
+        if ((uintptr_t)q & 15u) return false;
+    return true;
+}
+
 int check_workspace(const void* ws, size_t have, size_t need) {
     if (need == 0) return E3J_OK;
     if (!ws || ((uintptr_t)ws & 255u) || have < need) return E3J_ERR_WORKSPACE;
@@ -299,6 +308,7 @@ static int conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges,
     if (n_nodes == 0) return E3J_OK;
     if (!out || !x) return E3J_ERR_INVALID_ARG;
     if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    if (!aligned16({x, w, out})) return E3J_ERR_INVALID_ARG;
     if (padded && !rowptr) return E3J_ERR_INVALID_ARG;  // rowptr[n_nodes] is where the kernels learn the edge count
     const int32_t* n_real = padded ? rowptr + n_nodes : nullptr;
     cudaStream_t st = (cudaStream_t)stream;
@@ -358,6 +368,7 @@ static int conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges,
     if (!x || !grad_out) return E3J_ERR_INVALID_ARG;
     if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
     if ((sender_perm == nullptr) != (colptr == nullptr)) return E3J_ERR_INVALID_ARG;
+    if (!aligned16({x, w, grad_out, grad_x, grad_w})) return E3J_ERR_INVALID_ARG;
     if (padded && !rowptr) return E3J_ERR_INVALID_ARG;  // rowptr[n_nodes] is where the kernels learn the edge count
     const int32_t* n_real = padded ? rowptr + n_nodes : nullptr;
     cudaStream_t st = (cudaStream_t)stream;
@@ -437,6 +448,7 @@ int e3j_conv_bwd_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, con
     if (!x || !grad_out) return E3J_ERR_INVALID_ARG;
     if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
     if (!rowptr || !sender_perm || !colptr) return E3J_ERR_INVALID_ARG;  // six passes: prepare the graph once
+    if (!aligned16({x, w, grad_out, ct_x, ct_w, gg_out, g_x, g_w})) return E3J_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const DoubleBwdLayout L = dbl_layout(plan, n_nodes, n_edges);
     if (int s = check_workspace(workspace, workspace_bytes, L.total)) return s;
@@ -538,6 +550,7 @@ int e3j_tp_fwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
     if (plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;  // the kernels work on groups of four channels
     if (rows == 0) return E3J_OK;
     if (!x1 || !x2 || !w || !out) return E3J_ERR_INVALID_ARG;
+    if (!aligned16({x1, w, out})) return E3J_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const FastKernels* fk = fast_lookup(plan);
     if (fk && fk->tp_fwd) return fk->tp_fwd(rows, x1, x2, w, out, st);
@@ -555,6 +568,7 @@ int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
     if (plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;  // the kernels work on groups of four channels
     if (rows == 0) return E3J_OK;
     if (!x1 || !x2 || !w || !grad_out) return E3J_ERR_INVALID_ARG;
+    if (!aligned16({x1, w, grad_out, grad_x1, grad_w})) return E3J_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const FastKernels* fk = fast_lookup(plan);
     if (fk && fk->tp_bwd && grad_x1 && grad_x2 && grad_w)

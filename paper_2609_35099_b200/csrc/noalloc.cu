@@ -48,6 +48,7 @@ extern "C" int e3j_conv_fwd_noalloc(const e3j_plan* plan, int64_t n_nodes, int64
     if (n_nodes == 0) return E3J_OK;
     if (!out || !x) return E3J_ERR_INVALID_ARG;
     if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    if (((uintptr_t)x | (uintptr_t)w | (uintptr_t)out) & 15u) return E3J_ERR_INVALID_ARG;  // 128-bit rows
     const FastKernels* fk = fast_lookup(plan);
     if (!fk || !fk->conv_fwd || !fk->fwd_scratch_bytes) return E3J_ERR_UNSUPPORTED;  // no specialised kernel
     cudaStream_t st = (cudaStream_t)stream;

@@ -414,6 +414,45 @@ def test_workspace_errors_are_reported():
         e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, _cuda(g), workspace=tiny)
 
 
+@pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
+def test_misaligned_channel_arrays_are_refused(flags):
+    """Rows are moved as 128-bit vectors and 16-byte bulk copies: a per-channel array that starts 4 bytes off a
+    16-byte boundary must be refused on the host (no launch), whichever argument it is."""
+    wl, plan, cp, x, y, w, g = make_case(2, 192, flags=flags)
+    n, e = wl.n_nodes, wl.n_edges
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+
+    def shifted(a):   # same values, storage offset by one float
+        buf = torch.empty(a.size + 1, dtype=torch.float32, device=DEV)
+        view = buf[1:].view(a.shape)
+        view.copy_(torch.from_numpy(a))
+        assert view.data_ptr() % 16 == 4
+        return view
+
+    good = dict(x=_cuda(x), sh=_cuda(y), w=_cuda(w), g=_cuda(g))
+    for bad in ("x", "w"):
+        args = dict(good)
+        args[bad] = shifted({"x": x, "w": w}[bad])
+        with pytest.raises(e3j.E3JError, match="status -1"):
+            e3j.e3j_conv_fwd(plan, args["x"], args["sh"], args["w"], snd, rcv)
+    for bad in ("x", "w", "g"):
+        args = dict(good)
+        args[bad] = shifted({"x": x, "w": w, "g": g}[bad])
+        with pytest.raises(e3j.E3JError, match="status -1"):
+            e3j.e3j_conv_bwd(plan, args["x"], args["sh"], args["w"], snd, rcv, args["g"])
+    with pytest.raises(e3j.E3JError, match="status -1"):
+        e3j.e3j_conv_fwd(plan, good["x"], good["sh"], good["w"], snd, rcv, out=shifted(g))
+    # the harmonics may sit anywhere a float can
+    out = e3j.e3j_conv_fwd(plan, good["x"], shifted(y), good["w"], snd, rcv)
+    ref = e3j.e3j_conv_fwd(plan, good["x"], good["sh"], good["w"], snd, rcv)
+    assert torch.equal(out, ref)
+    gx, gy, gw = e3j.e3j_conv_bwd(plan, good["x"], shifted(y), good["w"], snd, rcv, good["g"])
+    rx, ry, rw = e3j.e3j_conv_bwd(plan, good["x"], good["sh"], good["w"], snd, rcv, good["g"])
+    assert torch.equal(gx, rx) and torch.equal(gy, ry) and torch.equal(gw, rw)
+    torch.cuda.synchronize()
+    assert e3j.e3j_plan_device_status(plan) == 0
+
+
 # ------------------------------------------------------------------ full-size configurations, sampled
 def _seeded_normal(shape, seed):
     gen = torch.Generator(device=DEV)
