@@ -258,6 +258,8 @@ def main():
                     help="plan with collapsed output multiplicities (table-driven kernels; no CPU leg)")
     ap.add_argument("--pad", type=float, default=0.0,
                     help="append this fraction of padding edges and call the padded entry points (rates count real edges)")
+    ap.add_argument("--double-backward", action="store_true",
+                    help="also time e3j_conv_bwd_bwd (after the steps, reported beside them; plain lists only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -370,6 +372,35 @@ def main():
         total_ms = float(tm.item())
     ms_per_step = total_ms / args.steps
 
+    # ---- the double backward of the same workload (not part of the step)
+    dbl = None
+    if args.double_backward and not args.pad:
+        gen = torch.Generator(device=dev); gen.manual_seed(11)
+        cts = [torch.randn(d[k].shape, generator=gen, device=dev) for k in ("x", "y", "w")]
+        ws_d = torch.empty(max(e3j.e3j_conv_bwd_bwd_workspace_bytes(plan, n, e), 256), dtype=torch.uint8, device=dev)
+        gg = torch.empty_like(out)
+
+        def dbl_call():
+            e3j.e3j_conv_bwd_bwd(plan, d["x"], d["y"], d["w"], d["snd"], d["rcv"], d["g"], rowptr, perm, colptr,
+                                 cts[0], cts[1], cts[2], gg_out=gg, g_x=gx, g_sh=gy, g_w=gw, workspace=ws_d)
+
+        for _ in range(3):
+            dbl_call()
+        k_dbl = max(3, min(args.steps, 50))
+        l0 = e3j.e3j_launch_count()
+        d0, d1 = ev(), ev()
+        torch.cuda.synchronize()
+        d0.record(stream)
+        for _ in range(k_dbl):
+            dbl_call()
+        d1.record(stream)
+        torch.cuda.synchronize()
+        dbl = {"ms": d0.elapsed_time(d1) / k_dbl, "calls": k_dbl,
+               "launches_per_call": (e3j.e3j_launch_count() - l0) // k_dbl,
+               "note": "4 launches = fused sweeps (forward-shaped + fix-up, edge-wise + sender sum); "
+                       "more = composition of forward and backward passes"}
+        del ws_d, cts, gg
+
     # ---- end to end: pinned host buffers in, results out, inside the timed region
     e2e = None
     if not args.no_e2e:
@@ -436,6 +467,7 @@ def main():
             # 20 % of the runs, as in its efficiency-comparison section), minimum and maximum
             "call_stats_ms": {"fwd": call_stats(fwd_ms), "bwd": call_stats(bwd_ms)},
             "outside_the_step_ms": {"plan_build_host": plan_build_ms, "graph_prepare_device": graph_prepare_ms},
+            "double_backward": dbl,
             "roofline": dominant, "roofline_fwd": roofs["fwd"], "roofline_bwd": roofs["bwd"],
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         }
