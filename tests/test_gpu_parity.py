@@ -414,6 +414,42 @@ def test_workspace_errors_are_reported():
         e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, _cuda(g), workspace=tiny)
 
 
+def test_calls_can_be_captured_in_a_cuda_graph():
+    """With a prepared graph and caller-owned outputs and workspaces the calls only enqueue kernels: a stream
+    capture of forward + backward + double backward replays to the same bits as the eager calls."""
+    wl, plan, cp, x, y, w, g = make_case(2, 192)
+    n, e = wl.n_nodes, wl.n_edges
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    dx, dy, dw, dg = _cuda(x), _cuda(y), _cuda(w), _cuda(g)
+    rowptr, perm, colptr = e3j.e3j_graph_prepare(n, snd, rcv)
+    u8 = lambda nbytes: torch.empty(max(nbytes, 256), dtype=torch.uint8, device=DEV)
+    ws_f, ws_b = u8(e3j.e3j_conv_fwd_workspace_bytes(plan, n, e)), u8(e3j.e3j_conv_bwd_workspace_bytes(plan, n, e))
+    ws_d = u8(e3j.e3j_conv_bwd_bwd_workspace_bytes(plan, n, e))
+    out, gx, gy, gw = torch.empty_like(dg), torch.empty_like(dx), torch.empty_like(dy), torch.empty_like(dw)
+    dd = [torch.empty_like(t) for t in (dg, dx, dy, dw)]
+
+    def step():
+        e3j.e3j_conv_fwd(plan, dx, dy, dw, snd, rcv, rowptr, out=out, workspace=ws_f)
+        e3j.e3j_conv_bwd(plan, dx, dy, dw, snd, rcv, dg, rowptr, perm, colptr, grad_x=gx, grad_sh=gy, grad_w=gw,
+                         workspace=ws_b)
+        e3j.e3j_conv_bwd_bwd(plan, dx, dy, dw, snd, rcv, dg, rowptr, perm, colptr, gx, gy, gw, gg_out=dd[0],
+                             g_x=dd[1], g_sh=dd[2], g_w=dd[3], workspace=ws_d)
+
+    step()   # eager: first use sets the kernels' attributes and uploads the plan's tables
+    torch.cuda.synchronize()
+    eager = [t.clone() for t in (out, gx, gy, gw, *dd)]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for t in (out, gx, gy, gw, *dd):
+        t.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    for a, b in zip(eager, (out, gx, gy, gw, *dd)):
+        assert torch.equal(a, b)
+    assert e3j.e3j_plan_device_status(plan) == 0
+
+
 @pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
 def test_misaligned_channel_arrays_are_refused(flags):
     """Rows are moved as 128-bit vectors and 16-byte bulk copies: a per-channel array that starts 4 bytes off a
