@@ -334,11 +334,14 @@ def test_collapsed_output_multiplicities(config, n_atoms):
 
 
 @pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
-@pytest.mark.parametrize("config,n_atoms", [(1, None), (2, 192), (2, 1200)])
-def test_double_backward(config, n_atoms, flags):
+@pytest.mark.parametrize("config,n_atoms,natural", [(1, None, False), (2, 192, False), (2, 1200, False),
+                                                    (2, 192, True), (3, 200, False)])
+def test_double_backward(config, n_atoms, natural, flags):
     """Cotangents of the backward's inputs against the oracle; a missing cotangent is zero; outputs that are
-    not wanted are skipped; two runs give the same bits."""
-    wl, plan, cp, x, y, w, g = make_case(config, n_atoms, flags=flags)
+    not wanted are skipped; two runs give the same bits.  (Configs 2 and 3 have fused kernels, config 1 and the
+    generic plans take the composition.)"""
+    wl, plan, cp, x, y, w, g = make_case(config, n_atoms, flags=flags,
+                                         **({"irreps_out": workloads.NATURAL_PARITY_OUT} if natural else {}))
     n, e = wl.n_nodes, wl.n_edges
     rng = np.random.default_rng(77)
     ux = rng.standard_normal(x.shape).astype(np.float32)
