@@ -472,10 +472,15 @@ def main():
 
         def roof(nbytes, ms, kernel, key):
             ach = nbytes / (ms * 1e-3) / 1e9
-            traffic = NCU_TRAFFIC.get((wl.name, key)) if plan.specialised else None
-            return {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s",
-                    "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "peak_source": peak_src,
-                    "algorithmic_bytes_per_launch": nbytes, "avg_ms": ms, "traffic": traffic}
+            plain = plan.specialised and not args.pad and not args.collapse
+            traffic = NCU_TRAFFIC.get((wl.name, key)) if plain else None
+            r = {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s",
+                 "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "peak_source": peak_src,
+                 "algorithmic_bytes_per_launch": nbytes, "avg_ms": ms, "traffic": traffic}
+            if traffic:   # what the memory system actually moved (ncu), at the measured duration
+                r["traffic_GBs"] = traffic / (ms * 1e-3) / 1e9
+                r["traffic_frac_of_peak"] = r["traffic_GBs"] / peak
+            return r
 
         spec = bool(plan.specialised)
         roofs = {"fwd": roof(fb, f_ms, "e3j_conv_fwd call: fast_fwd_kernel (97 %) + fwd_fixup_kernel" if spec
