@@ -417,6 +417,67 @@ def test_workspace_errors_are_reported():
         e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, _cuda(g), workspace=tiny)
 
 
+@pytest.mark.parametrize("seed", [1, 2])
+def test_specialised_and_generic_kernels_agree_on_random_graphs(seed):
+    """A cross-check beside the oracle parity tests: on random graphs (sparse rows, rows of tens of edges, hubs of
+    up to 2000 edges, padded lists) and for every generated signature the specialised kernels and the
+    table-driven ones give the same forward, backward, double backward and tensor products to rounding, the
+    specialised backward twice the same bits."""
+    rng = np.random.default_rng(seed)
+    sigs = [("128x0e+128x1o", None, 3), ("64x0e+64x1o", None, 3), ("256x0e+256x1o", None, 3), ("128x0e", None, 3),
+            ("64x0e+64x1o+64x2e+64x3o", None, 3), ("128x0e+128x1o", workloads.NATURAL_PARITY_OUT, -1)]
+
+    def rel(a, b):
+        return (a - b).abs().max().item() / max(b.abs().max().item(), 1e-30)
+
+    for it in range(12):
+        irr, iro, olm = sigs[it % len(sigs)]
+        pf = e3j.e3j_plan_create(irr, 3, iro, olm)
+        pg = e3j.e3j_plan_create(irr, 3, iro, olm, e3j.E3J_PLAN_GENERIC_ONLY)
+        assert pf.specialised and not pg.specialised
+        n = int(rng.integers(2, 300))
+        deg = [rng.integers(0, 12, size=n), rng.integers(0, 3, size=n), rng.integers(20, 90, size=n),
+               rng.integers(0, 5, size=n)][it % 4]
+        if it % 4 == 3:
+            deg[rng.integers(0, n)] = int(rng.integers(100, 2000))
+        rcv = np.repeat(np.arange(n), deg).astype(np.int32)
+        e, pad = len(rcv), int(rng.integers(0, 150)) if it % 2 else 0
+        snd = rng.integers(0, n, size=e).astype(np.int32)
+        if e + pad == 0:
+            continue
+        s = _cuda(np.concatenate([snd, np.zeros(pad, np.int32)]))
+        r = _cuda(np.concatenate([rcv, np.full(pad, n, np.int32)]))
+        x = torch.randn((n, pf.d_in, pf.n_channels), device=DEV)
+        y = torch.randn((e + pad, pf.d_sh), device=DEV)
+        w = torch.randn((e + pad, pf.n_paths, pf.n_channels), device=DEV)
+        g = torch.randn((n, pf.d_out, pf.n_channels), device=DEV)
+        if pad:
+            rowptr, perm, colptr = e3j.e3j_graph_prepare_padded(n, s, r)
+            fwd, bwd = e3j.e3j_conv_fwd_padded, e3j.e3j_conv_bwd_padded
+        else:
+            rowptr, perm, colptr = e3j.e3j_graph_prepare(n, s, r)
+            fwd, bwd = e3j.e3j_conv_fwd, e3j.e3j_conv_bwd
+        errs = [rel(fwd(pf, x, y, w, s, r, rowptr), fwd(pg, x, y, w, s, r, rowptr))]
+        bf, bg = bwd(pf, x, y, w, s, r, g, rowptr, perm, colptr), bwd(pg, x, y, w, s, r, g, rowptr, perm, colptr)
+        again = bwd(pf, x, y, w, s, r, g, rowptr, perm, colptr)
+        assert all(torch.equal(a, b) for a, b in zip(bf, again))
+        errs += [rel(a, b) for a, b in zip(bf, bg)]
+        if not pad and e:
+            cts = [torch.randn_like(t) for t in (x, y, w)]
+            errs += [rel(a, b) for a, b in zip(
+                e3j.e3j_conv_bwd_bwd(pf, x, y, w, s, r, g, rowptr, perm, colptr, *cts),
+                e3j.e3j_conv_bwd_bwd(pg, x, y, w, s, r, g, rowptr, perm, colptr, *cts))]
+        rows = int(rng.integers(1, 500))
+        x1, x2 = torch.randn((rows, pf.d_in, pf.n_channels), device=DEV), torch.randn((rows, pf.d_sh), device=DEV)
+        wt = torch.randn((rows, pf.n_paths, pf.n_channels), device=DEV)
+        gt = torch.randn((rows, pf.d_out, pf.n_channels), device=DEV)
+        errs.append(rel(e3j.e3j_tp_fwd(pf, x1, x2, wt), e3j.e3j_tp_fwd(pg, x1, x2, wt)))
+        errs += [rel(a, b) for a, b in zip(e3j.e3j_tp_bwd(pf, x1, x2, wt, gt), e3j.e3j_tp_bwd(pg, x1, x2, wt, gt))]
+        torch.cuda.synchronize()
+        assert e3j.e3j_plan_device_status(pf) == 0
+        assert max(errs) < 1e-5, (it, irr, n, e, pad, errs)
+
+
 def test_calls_can_be_captured_in_a_cuda_graph():
     """With a prepared graph and caller-owned outputs and workspaces the calls only enqueue kernels: a stream
     capture of forward + backward + double backward replays to the same bits as the eager calls."""
