@@ -100,6 +100,30 @@ def test_scalar_input_signature():
     assert max(worst) < 1e-5
 
 
+def test_lmax2_signature():
+    """The water-box inputs with harmonics and outputs up to l = 2 (9 harmonics per edge: rows of the harmonics
+    array are 36 bytes, only 4-byte aligned), forward, backward and standalone tensor product."""
+    import dataclasses
+    wl = dataclasses.replace(workloads.make_graph(2, 300), sh_lmax=2, out_lmax=2)
+    plan = e3j.e3j_plan_create("128x0e+128x1o", 2, None, 2)
+    assert plan.specialised and plan.n_paths == 9 and plan.d_out == 29 and plan.d_sh == 9
+    cp = oconv.Coupling("128x0e+128x1o", 2, None, 2)
+    x, y, w, g = workloads.make_features(wl, plan.n_paths, plan.d_out)
+    assert y.shape[1] == 9
+    worst = run_conv_parity(wl, plan, cp, x, y, w, g)
+    assert max(worst) < 1e-5
+    rows = 333
+    out = e3j.e3j_tp_fwd(plan, _cuda(x[:rows]), _cuda(y[:rows]), _cuda(w[:rows]))
+    gx1, gx2, gw = e3j.e3j_tp_bwd(plan, _cuda(x[:rows]), _cuda(y[:rows]), _cuda(w[:rows]), _cuda(g[:rows]))
+    ident = np.arange(rows, dtype=np.int32)
+    ref = oconv.conv_fwd(cp, x[:rows], y[:rows], w[:rows], ident, ident)
+    rx, ry, rw = oconv.conv_bwd(cp, x[:rows], y[:rows], w[:rows], ident, ident, g[:rows])
+    assert_blockwise_close(out.cpu().numpy(), ref, blocks_of_paths(cp.paths, "out"), what="tp out")
+    assert_blockwise_close(gx1.cpu().numpy(), rx, blocks_of_paths(cp.paths, "x"), what="tp grad_x1")
+    assert_blockwise_close(gx2.cpu().numpy(), ry, blocks_of_paths(cp.paths, "sh"), what="tp grad_x2")
+    assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="tp grad_w")
+
+
 @pytest.mark.parametrize("channels", [64, 256])
 def test_other_channel_counts_of_the_water_box_signature(channels):
     """The water-box signature with 64 and 256 channels (generated kernels exist for both)."""
