@@ -133,3 +133,26 @@ def test_collapsed_plan_tables(sig):
         want[off:off + 2 * p.L + 1, :, :, p.k] = cp.C[p.out_off:p.out_off + 2 * p.L + 1]
     assert np.abs(dense - want).max() < 1e-13
     assert e3j.e3j_plan_signature(plan) != e3j.e3j_plan_signature(full)
+
+
+def test_generated_kernel_sources_are_up_to_date(repo_root):
+    """The specialised kernels are generated from signatures.json and the plan builder's records; the files in
+    the tree must be what the generator writes today (a stale file would be compiled silently)."""
+    import subprocess
+    import sys
+    gen = os.path.join(repo_root, "paper_2609_35099_b200", "csrc", "gen_fast.py")
+    done = subprocess.run([sys.executable, gen, "--check"], capture_output=True, text=True, cwd=repo_root)
+    assert done.returncode == 0, done.stdout + done.stderr
+
+
+def test_every_generated_signature_is_picked_up_by_its_plan(repo_root):
+    """A plan created from the descriptors of a signature in signatures.json selects the generated kernels."""
+    import json
+    path = os.path.join(repo_root, "paper_2609_35099_b200", "csrc", "fast", "signatures.json")
+    for sig in json.load(open(path)):
+        flags = e3j.E3J_PLAN_COLLAPSE_OUTPUTS if sig.get("collapse") else 0
+        plan = e3j.e3j_plan_create(sig["irreps_in"], sig["sh_lmax"], sig["irreps_out"], sig["out_lmax"], flags)
+        assert plan.specialised, sig["name"]
+        generic = e3j.e3j_plan_create(sig["irreps_in"], sig["sh_lmax"], sig["irreps_out"], sig["out_lmax"],
+                                      flags | e3j.E3J_PLAN_GENERIC_ONLY)
+        assert not generic.specialised
