@@ -448,16 +448,18 @@ def test_specialised_and_generic_kernels_agree_on_random_graphs(seed):
     table-driven ones give the same forward, backward, double backward and tensor products to rounding, the
     specialised backward twice the same bits."""
     rng = np.random.default_rng(seed)
-    sigs = [("128x0e+128x1o", None, 3), ("64x0e+64x1o", None, 3), ("256x0e+256x1o", None, 3), ("128x0e", None, 3),
-            ("64x0e+64x1o+64x2e+64x3o", None, 3), ("128x0e+128x1o", workloads.NATURAL_PARITY_OUT, -1)]
+    sigs = [("128x0e+128x1o", 3, None, 3), ("64x0e+64x1o", 3, None, 3), ("256x0e+256x1o", 3, None, 3),
+            ("128x0e", 3, None, 3), ("64x0e+64x1o+64x2e+64x3o", 3, None, 3),
+            ("128x0e+128x1o", 3, workloads.NATURAL_PARITY_OUT, -1), ("128x0e+128x1o", 2, None, 2),
+            ("128x0e+128x1o+128x2e", 3, None, 3)]
 
     def rel(a, b):
         return (a - b).abs().max().item() / max(b.abs().max().item(), 1e-30)
 
-    for it in range(12):
-        irr, iro, olm = sigs[it % len(sigs)]
-        pf = e3j.e3j_plan_create(irr, 3, iro, olm)
-        pg = e3j.e3j_plan_create(irr, 3, iro, olm, e3j.E3J_PLAN_GENERIC_ONLY)
+    for it in range(16):
+        irr, lmax, iro, olm = sigs[it % len(sigs)]
+        pf = e3j.e3j_plan_create(irr, lmax, iro, olm)
+        pg = e3j.e3j_plan_create(irr, lmax, iro, olm, e3j.E3J_PLAN_GENERIC_ONLY)
         assert pf.specialised and not pg.specialised
         n = int(rng.integers(2, 300))
         deg = [rng.integers(0, 12, size=n), rng.integers(0, 3, size=n), rng.integers(20, 90, size=n),
