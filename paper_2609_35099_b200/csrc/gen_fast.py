@@ -35,10 +35,12 @@ def load_records(sig):
     return info, paths, recs, signature
 
 
-def partition_rows(costs, n_groups):
-    """Contiguous partition of rows into n_groups minimising the largest group cost (DP)."""
+def partition_rows(costs, n_groups, weights=None):
+    """Contiguous partition of rows into n_groups minimising the largest group cost (DP); weights[g] scales
+    the cost of group g (a group whose warp shares its scheduler with a producer warp should get less)."""
     n = len(costs)
     n_groups = min(n_groups, n)
+    weights = list(weights or []) + [1.0] * n_groups
     pre = [0]
     for c in costs:
         pre.append(pre[-1] + c)
@@ -49,7 +51,7 @@ def partition_rows(costs, n_groups):
     for g in range(1, n_groups + 1):
         for j in range(g, n + 1):
             for i in range(g - 1, j):
-                v = max(best[g - 1][i], pre[j] - pre[i])
+                v = max(best[g - 1][i], (pre[j] - pre[i]) * weights[g - 1])
                 if v < best[g][j]:
                     best[g][j], cut[g][j] = v, i
     bounds = [n]
@@ -111,7 +113,14 @@ class Sig:
             starts = sum((2 * self.paths[k]["l1"] + 1) * 1.0 + 0.5 for k in self.row_paths[row]
                          if row == self.paths[k]["out_off"])
             costs.append(len(self.row_pairs[row]) * 1.0 + starts + 0.3)
-        bounds = partition_rows(costs, FW)
+        bounds = partition_rows(costs, FW, self.cfg.get("F_BIAS"))
+        # Measured group sizes override the estimate: consumer warp 1 shares its scheduler with the table
+        # producer warp (and warp 0 with the copy warp), so an even split leaves the other two waiting for it.
+        if self.cfg.get("F_ROWS"):
+            bounds = [0]
+            for r in self.cfg["F_ROWS"]:
+                bounds.append(bounds[-1] + r)
+            assert bounds[-1] == self.D and len(bounds) == FW + 1
         while len(bounds) < FW + 1:
             bounds.append(bounds[-1])
         a0, slots = [0], []  # slot -> pair index or None
