@@ -46,6 +46,10 @@ def _load():
         lib.e3j_oracle_conv_fwd.restype = i32
         lib.e3j_oracle_conv_bwd.argtypes = [i64, i64, i32, i32, i32, i32, i32] + [ptr] * 11
         lib.e3j_oracle_conv_bwd.restype = i32
+        lib.e3j_oracle_conv_fwd_sd.argtypes = lib.e3j_oracle_conv_fwd.argtypes
+        lib.e3j_oracle_conv_fwd_sd.restype = i32
+        lib.e3j_oracle_conv_bwd_sd.argtypes = lib.e3j_oracle_conv_bwd.argtypes
+        lib.e3j_oracle_conv_bwd_sd.restype = i32
         lib.e3j_oracle_threads.restype = i32
         _lib = lib
     return _lib
@@ -207,3 +211,62 @@ def conv_bwd_bwd(cp: Coupling, x, y, s, senders, receivers, dm, ux, uy, us):
     x_from_y, _, s_from_y = conv_bwd(cp, x, uy, s, senders, receivers, dm)
     x_from_s, y_from_s, _ = conv_bwd(cp, x, y, us, senders, receivers, dm)
     return g_dm, x_from_y + x_from_s, y_from_x + y_from_s, s_from_x + s_from_y
+
+
+# ---------------------------------------------------------------------------------------------
+# Edge scalars from the radial network (paper, "Key operations in scope": the scalars s_ab of the
+# message-passing layer depend on the interatomic distance through a radial-basis embedding followed by a
+# multi-layer perceptron, and such scalar mixings are named as candidates for fusion into the message
+# passing).  What is taken inside the convolution here is the perceptron's last, purely linear layer:
+#   s[e, k, q] = sum_j h[e, j] * W[j, k * N_q + q]
+# with h [E, H] the last hidden activations of the edge and W [H, P * N_q] the layer's matrix (no bias;
+# the paper does not state the layer sizes, H is free).  The product is formed in float64 and is never
+# rounded to float32; the convolution is then the defining sum.  Backward: the chain rule through the
+# product, dh = ds W^T and dW = h^T ds, with ds the edge-scalar cotangent of the convolution.
+def radial_weights(h, W, n_paths: int, nq: int) -> np.ndarray:
+    """s[E, P, N_q] = h W in float64."""
+    h = np.asarray(h, dtype=np.float64); W = np.asarray(W, dtype=np.float64)
+    assert h.ndim == 2 and W.shape == (h.shape[1], n_paths * nq), (h.shape, W.shape)
+    return (h @ W).reshape(h.shape[0], n_paths, nq)
+
+
+def _conv_fwd_sd(cp: Coupling, x, y, s, senders, receivers) -> np.ndarray:
+    n, e = x.shape[0], len(senders)
+    x = _f32(x, (n, cp.d, cp.nq)); y = _f32(y, (e, cp.dp))
+    s = np.ascontiguousarray(s, dtype=np.float64); assert s.shape == (e, cp.P, cp.nq)
+    senders, receivers = _i32(senders, e), _i32(receivers, e)
+    out = np.zeros((n, cp.D, cp.nq))
+    rc = _load().e3j_oracle_conv_fwd_sd(n, e, cp.d, cp.dp, cp.P, cp.D, cp.nq, _p(cp.C), _p(cp.i3),
+                                        _p(x), _p(y), _p(s), _p(senders), _p(receivers), _p(out))
+    if rc != 0:
+        raise ValueError("oracle: receivers not sorted or index out of range")
+    return out
+
+
+def _conv_bwd_sd(cp: Coupling, x, y, s, senders, receivers, dm):
+    n, e = x.shape[0], len(senders)
+    x = _f32(x, (n, cp.d, cp.nq)); y = _f32(y, (e, cp.dp)); dm = _f32(dm, (n, cp.D, cp.nq))
+    s = np.ascontiguousarray(s, dtype=np.float64); assert s.shape == (e, cp.P, cp.nq)
+    senders, receivers = _i32(senders, e), _i32(receivers, e)
+    dx = np.zeros((n, cp.d, cp.nq)); dy = np.zeros((e, cp.dp)); ds = np.zeros((e, cp.P, cp.nq))
+    rc = _load().e3j_oracle_conv_bwd_sd(n, e, cp.d, cp.dp, cp.P, cp.D, cp.nq, _p(cp.C), _p(cp.i3),
+                                        _p(x), _p(y), _p(s), _p(senders), _p(receivers), _p(dm),
+                                        _p(dx), _p(dy), _p(ds))
+    if rc != 0:
+        raise ValueError("oracle: receivers not sorted or index out of range")
+    return dx, dy, ds
+
+
+def conv_radial_fwd(cp: Coupling, x, y, h, W, senders, receivers) -> np.ndarray:
+    """m[N, D, N_q] with the edge scalars s = h W formed in float64."""
+    return _conv_fwd_sd(cp, x, y, radial_weights(h, W, cp.P, cp.nq), senders, receivers)
+
+
+def conv_radial_bwd(cp: Coupling, x, y, h, W, senders, receivers, dm):
+    """(dx[N,d,N_q], dy[E,d'], dh[E,H], dW[H,P*N_q]) in float64."""
+    s = radial_weights(h, W, cp.P, cp.nq)
+    dx, dy, ds = _conv_bwd_sd(cp, x, y, s, senders, receivers, dm)
+    ds2 = ds.reshape(ds.shape[0], cp.P * cp.nq)
+    dh = ds2 @ np.asarray(W, dtype=np.float64).T
+    dW = np.asarray(h, dtype=np.float64).T @ ds2
+    return dx, dy, dh, dW

@@ -57,10 +57,12 @@ static int64_t* build_rowptr(int64_t n_nodes, int64_t n_edges, const int32_t* re
     return rowptr;
 }
 
-int e3j_oracle_conv_fwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, int D, int nq,
-                        const double* C, const int32_t* i3, const float* x, const float* y,
-                        const float* s, const int32_t* senders, const int32_t* receivers,
-                        double* out) {
+/* The edge scalars come in as doubles: the float32 entry point promotes them first (exactly), the
+ * radial entry points of conv.py pass s = h W formed in float64. */
+static int conv_fwd_sums(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, int D, int nq,
+                         const double* C, const int32_t* i3, const float* x, const float* y,
+                         const double* s, const int32_t* senders, const int32_t* receivers,
+                         double* out) {
     if (check_graph(n_nodes, n_edges, senders, receivers)) return -1;
     int64_t* rowptr = build_rowptr(n_nodes, n_edges, receivers);
     memset(out, 0, sizeof(double) * (size_t)n_nodes * D * nq);
@@ -70,7 +72,7 @@ int e3j_oracle_conv_fwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, 
         for (int64_t e = rowptr[b]; e < rowptr[b + 1]; ++e) {
             const float* xa = x + (size_t)senders[e] * d * nq;
             const float* ye = y + (size_t)e * dp;
-            const float* se = s + (size_t)e * P * nq;
+            const double* se = s + (size_t)e * P * nq;
             for (int i0 = 0; i0 < D; ++i0) {
                 const int k = i3[i0];
                 for (int i1 = 0; i1 < d; ++i1)
@@ -79,7 +81,7 @@ int e3j_oracle_conv_fwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, 
                         if (c == 0.0) continue;
                         for (int q = 0; q < nq; ++q)
                             mb[(size_t)i0 * nq + q] += c * (double)xa[(size_t)i1 * nq + q] *
-                                                       (double)ye[i2] * (double)se[(size_t)k * nq + q];
+                                                       (double)ye[i2] * se[(size_t)k * nq + q];
                     }
             }
         }
@@ -88,10 +90,34 @@ int e3j_oracle_conv_fwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, 
     return 0;
 }
 
-int e3j_oracle_conv_bwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, int D, int nq,
+static double* promote(const float* s, size_t n) {
+    double* out = (double*)malloc(sizeof(double) * (n > 0 ? n : 1));
+    for (size_t i = 0; i < n; ++i) out[i] = (double)s[i];
+    return out;
+}
+
+int e3j_oracle_conv_fwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, int D, int nq,
                         const double* C, const int32_t* i3, const float* x, const float* y,
                         const float* s, const int32_t* senders, const int32_t* receivers,
-                        const float* dm, double* dx, double* dy, double* ds) {
+                        double* out) {
+    double* sd = promote(s, (size_t)n_edges * P * nq);
+    const int rc = conv_fwd_sums(n_nodes, n_edges, d, dp, P, D, nq, C, i3, x, y, sd, senders, receivers, out);
+    free(sd);
+    return rc;
+}
+
+/* the same sums with the edge scalars given in float64 */
+int e3j_oracle_conv_fwd_sd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, int D, int nq,
+                           const double* C, const int32_t* i3, const float* x, const float* y,
+                           const double* s, const int32_t* senders, const int32_t* receivers,
+                           double* out) {
+    return conv_fwd_sums(n_nodes, n_edges, d, dp, P, D, nq, C, i3, x, y, s, senders, receivers, out);
+}
+
+static int conv_bwd_sums(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, int D, int nq,
+                         const double* C, const int32_t* i3, const float* x, const float* y,
+                         const double* s, const int32_t* senders, const int32_t* receivers,
+                         const float* dm, double* dx, double* dy, double* ds) {
     if (check_graph(n_nodes, n_edges, senders, receivers)) return -1;
     memset(dx, 0, sizeof(double) * (size_t)n_nodes * d * nq);
     memset(dy, 0, sizeof(double) * (size_t)n_edges * dp);
@@ -102,7 +128,7 @@ int e3j_oracle_conv_bwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, 
     for (int64_t e = 0; e < n_edges; ++e) {
         const float* xa = x + (size_t)senders[e] * d * nq;
         const float* ye = y + (size_t)e * dp;
-        const float* se = s + (size_t)e * P * nq;
+        const double* se = s + (size_t)e * P * nq;
         const float* dmb = dm + (size_t)receivers[e] * D * nq;
         for (int i0 = 0; i0 < D; ++i0) {
             const int k = i3[i0];
@@ -134,7 +160,7 @@ int e3j_oracle_conv_bwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, 
         for (int64_t j = colptr[a]; j < colptr[a + 1]; ++j) {
             const int64_t e = perm[j];
             const float* ye = y + (size_t)e * dp;
-            const float* se = s + (size_t)e * P * nq;
+            const double* se = s + (size_t)e * P * nq;
             const float* dmb = dm + (size_t)receivers[e] * D * nq;
             for (int i0 = 0; i0 < D; ++i0) {
                 const int k = i3[i0];
@@ -144,7 +170,7 @@ int e3j_oracle_conv_bwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, 
                         if (c == 0.0) continue;
                         for (int q = 0; q < nq; ++q)
                             dxa[(size_t)i1 * nq + q] += c * (double)ye[i2] *
-                                                        (double)se[(size_t)k * nq + q] *
+                                                        se[(size_t)k * nq + q] *
                                                         (double)dmb[(size_t)i0 * nq + q];
                     }
             }
@@ -154,4 +180,22 @@ int e3j_oracle_conv_bwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, 
     free(perm);
     free(fill);
     return 0;
+}
+
+int e3j_oracle_conv_bwd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, int D, int nq,
+                        const double* C, const int32_t* i3, const float* x, const float* y,
+                        const float* s, const int32_t* senders, const int32_t* receivers,
+                        const float* dm, double* dx, double* dy, double* ds) {
+    double* sd = promote(s, (size_t)n_edges * P * nq);
+    const int rc = conv_bwd_sums(n_nodes, n_edges, d, dp, P, D, nq, C, i3, x, y, sd, senders, receivers, dm,
+                                 dx, dy, ds);
+    free(sd);
+    return rc;
+}
+
+int e3j_oracle_conv_bwd_sd(int64_t n_nodes, int64_t n_edges, int d, int dp, int P, int D, int nq,
+                           const double* C, const int32_t* i3, const float* x, const float* y,
+                           const double* s, const int32_t* senders, const int32_t* receivers,
+                           const float* dm, double* dx, double* dy, double* ds) {
+    return conv_bwd_sums(n_nodes, n_edges, d, dp, P, D, nq, C, i3, x, y, s, senders, receivers, dm, dx, dy, ds);
 }
