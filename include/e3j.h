@@ -76,12 +76,13 @@ enum {
 
 /* plan flags */
 #define E3J_PLAN_GENERIC_ONLY 1u /* never pick a signature-specialised kernel */
-/* Collapsed output multiplicities (paper: the coefficient set used for the comparison with the SO(2)
- * convolution, which "sums all isomorphic copies of a given irreducible output space together"): all paths
+/* Collapsed output multiplicities (paper: the coefficient set of the comparison with the SO(2) convolution, in
+ * which the copies of one irreducible output space that different paths produce are added together): all paths
  * that land on the same (L, p) share one output block, out[b, block(L,p) + M, q] = sum over those paths of
  * w[e, path, q] * (...), so D = sum over distinct (L, p) of (2L + 1) while the weights stay one block per
- * path.  out_off of e3j_path_info_t is then the same for the paths of a block.  Such plans run on the
- * table-driven kernels. */
+ * path.  out_off of e3j_path_info_t is then the same for the paths of a block.  Such plans use generated
+ * kernels where a collapsed signature has been generated (the water-box signature), the table-driven kernels
+ * otherwise. */
 #define E3J_PLAN_COLLAPSE_OUTPUTS 2u
 
 typedef struct e3j_plan e3j_plan; /* opaque; immutable after creation; usable from several streams */
@@ -129,9 +130,10 @@ const char* e3j_plan_signature(const e3j_plan* plan);
 int e3j_plan_device_status(const e3j_plan* plan, int32_t* status);
 /* Copies up to `capacity` path descriptors (host memory); returns P or an error. */
 int e3j_plan_paths(const e3j_plan* plan, e3j_path_info_t* paths, int capacity);
-/* Copies the coefficient records, sorted by (i0,i1,i2), into HOST arrays of
+/* Copies the coefficient records, sorted by (i0, path, i1, i2), into HOST arrays of
  * `capacity` entries each (val in float64 as built, before rounding to float32);
- * returns nnz or an error. */
+ * returns nnz or an error.  For uncollapsed plans every output row belongs to one path and
+ * the order equals (i0, i1, i2). */
 int e3j_plan_records(const e3j_plan* plan, int32_t* i0, int32_t* i1, int32_t* i2, int32_t* i3,
                      double* val, int capacity);
 
@@ -251,6 +253,40 @@ int e3j_conv_bwd_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, con
                      const int32_t* colptr, const float* grad_out, const float* ct_x,
                      const float* ct_sh, const float* ct_w, float* gg_out, float* g_x, float* g_sh,
                      float* g_w, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Edge scalars from the radial network (paper, "Key operations in scope": the scalars of the message-passing
+ * layer come from a radial-basis embedding of the interatomic distance followed by a multi-layer perceptron,
+ * and scalar mixings are named as candidates for fusion into the message passing; appendix "Mathematical
+ * Details", edge scalars).  The last layer of that perceptron is linear, so the per-edge weights are
+ *     w[e, k, q] = sum_j h[e, j] * W[j, k * N_q + q]
+ * with h [n_edges, hidden] the edge's last hidden activations and W [hidden, P * N_q] the layer's matrix (no
+ * bias).  The calls below take (h, W) in place of w, so the [n_edges, P, N_q] weight array, nine tenths of the
+ * convolution's minimal memory traffic, is never an input or an output of the call:
+ *     out     = conv_fwd(x, sh, h W)
+ *     grad_x, grad_sh as in e3j_conv_bwd;  grad_h = grad_w W^T;  grad_W = h^T grad_w   (grad_w internal)
+ * The product runs on the tensor cores with every float32 operand split into two TF32 terms (three tensor-core
+ * products per float32 product), which keeps float32-level accuracy: results agree with the float64 definition
+ * to the same 1e-5 per irreducible block as the other calls, and are bit-identical from run to run (grad_W is
+ * summed over fixed edge ranges in a fixed order).
+ *   hidden must be a multiple of 4; h, W, grad_h, grad_W 16-byte aligned; rowptr / sender_perm / colptr as for
+ *   e3j_conv_fwd / e3j_conv_bwd; any of grad_x, grad_sh, grad_h, grad_W may be NULL.
+ *   Workspace: 256-byte aligned, at least e3j_conv_radial_*_workspace_bytes(); calls that overlap on the GPU
+ *   must not share it.
+ * e3j_radial_weights writes the product itself, w_out [n_edges, P, N_q] (for callers that want the weights, and
+ * as the unfused baseline in measurements). */
+int e3j_radial_weights(const e3j_plan* plan, int64_t n_edges, int hidden, const float* h, const float* W,
+                       float* w_out, void* stream);
+size_t e3j_conv_radial_fwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden);
+int e3j_conv_radial_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
+                        const float* sh, const float* h, const float* W, const int32_t* senders,
+                        const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                        size_t workspace_bytes, void* stream);
+size_t e3j_conv_radial_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden);
+int e3j_conv_radial_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
+                        const float* sh, const float* h, const float* W, const int32_t* senders,
+                        const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                        const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
+                        float* grad_h, float* grad_W, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Standalone channelwise tensor product with per-row, per-path weights (paper:
  * tensor-product formula followed by the edge-scalar weighting; backward: the

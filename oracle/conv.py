@@ -166,8 +166,9 @@ def conv_bwd_padded(cp: Coupling, x, y, s, senders, receivers, dm):
 
 # ---------------------------------------------------------------------------------------------
 # Collapsed output multiplicities.  The paper evaluates its kernels also with a coefficient set
-# that "sums all isomorphic copies of a given irreducible output space together": every path
-# that lands on the same (L, parity) adds into one shared output block.  Written out here from
+# (appendix on the comparison with the SO(2) convolution) in which the copies of one irreducible
+# output space produced by different paths are added: every path that lands on the same
+# (L, parity) adds into one shared output block.  Written out here from
 # the uncollapsed definition: out_c = R out, with R the 0/1 matrix that maps row M of every
 # path's block to row M of the shared block of its (L, parity); the backward is the chain rule
 # through that sum (dm = R^T dm_c).  Blocks are ordered as their first path is.

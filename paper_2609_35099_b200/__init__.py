@@ -21,8 +21,12 @@ __all__ = [
     "E3JError", "Plan", "library_path", "e3j_plan_create", "e3j_plan_destroy", "e3j_plan_info",
     "e3j_plan_paths", "e3j_plan_records", "e3j_plan_signature", "e3j_plan_device_status", "e3j_graph_prepare", "e3j_graph_validate",
     "e3j_conv_fwd_workspace_bytes", "e3j_conv_bwd_workspace_bytes", "e3j_conv_fwd", "e3j_conv_fwd_noalloc",
-    "e3j_conv_bwd",
+    "e3j_conv_bwd", "e3j_graph_prepare_padded", "e3j_conv_fwd_padded", "e3j_conv_bwd_padded",
+    "e3j_conv_bwd_bwd_workspace_bytes", "e3j_conv_bwd_bwd",
+    "e3j_radial_weights", "e3j_conv_radial_fwd_workspace_bytes", "e3j_conv_radial_bwd_workspace_bytes",
+    "e3j_conv_radial_fwd", "e3j_conv_radial_bwd",
     "e3j_tp_fwd", "e3j_tp_bwd", "e3j_status_string", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
+    "E3J_PLAN_COLLAPSE_OUTPUTS",
 ]
 
 E3J_PLAN_GENERIC_ONLY = 1
@@ -30,10 +34,7 @@ E3J_PLAN_COLLAPSE_OUTPUTS = 2
 # status codes of include/e3j.h
 E3J_OK, E3J_ERR_INVALID_ARG, E3J_ERR_BAD_IRREPS, E3J_ERR_MUL_NOT_UNIFORM = 0, -1, -2, -3
 E3J_ERR_UNSUPPORTED, E3J_ERR_WORKSPACE, E3J_ERR_CUDA, E3J_ERR_GRAPH = -4, -5, -6, -7
-import os as _os
-
-# E3J_LIBRARY selects another build of the same library (e.g. an experimental variant).
-_LIB_PATH = Path(_os.environ.get("E3J_LIBRARY") or (Path(__file__).resolve().parent / "libe3j.so"))
+_LIB_PATH = Path(__file__).resolve().parent / "libe3j.so"
 _lib = None
 
 
@@ -97,6 +98,16 @@ def _load():
     lib.e3j_conv_bwd_padded.argtypes = [vp, i64, i64] + [vp] * 13 + [sz, vp]
     lib.e3j_conv_fwd_noalloc.argtypes = [vp, i64, i64] + [vp] * 7
     lib.e3j_conv_fwd_noalloc.restype = i32
+    lib.e3j_radial_weights.argtypes = [vp, i64, i32] + [vp] * 4
+    lib.e3j_radial_weights.restype = i32
+    lib.e3j_conv_radial_fwd_workspace_bytes.argtypes = [vp, i64, i64, i32]
+    lib.e3j_conv_radial_fwd_workspace_bytes.restype = sz
+    lib.e3j_conv_radial_bwd_workspace_bytes.argtypes = [vp, i64, i64, i32]
+    lib.e3j_conv_radial_bwd_workspace_bytes.restype = sz
+    lib.e3j_conv_radial_fwd.argtypes = [vp, i64, i64, i32] + [vp] * 9 + [sz, vp]
+    lib.e3j_conv_radial_fwd.restype = i32
+    lib.e3j_conv_radial_bwd.argtypes = [vp, i64, i64, i32] + [vp] * 15 + [sz, vp]
+    lib.e3j_conv_radial_bwd.restype = i32
     lib.e3j_tp_fwd.argtypes = [vp, i64] + [vp] * 5
     lib.e3j_tp_bwd.argtypes = [vp, i64] + [vp] * 8
     lib.e3j_status_string.argtypes = [i32]
@@ -382,6 +393,83 @@ def e3j_conv_bwd_bwd(plan: Plan, x, sh, w, senders, receivers, grad_out, rowptr,
         _dev_ptr(g_w, f32, s_w, "g_w"),
         ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_bwd_bwd")
     return gg_out, g_x, g_sh, g_w
+
+
+def e3j_radial_weights(plan: Plan, h, W, out=None, stream=None):
+    """w[E, P, N_q] = h W (the radial network's last layer), materialised."""
+    torch = _torch()
+    e, hidden = h.shape
+    f32 = torch.float32
+    if out is None:
+        out = torch.empty((e, plan.n_paths, plan.n_channels), dtype=f32, device=h.device)
+    _check(_load().e3j_radial_weights(
+        plan.handle, e, hidden, _dev_ptr(h, f32, (e, hidden), "h"),
+        _dev_ptr(W, f32, (hidden, plan.n_paths * plan.n_channels), "W"),
+        _dev_ptr(out, f32, (e, plan.n_paths, plan.n_channels), "out"), _stream(stream)), "e3j_radial_weights")
+    return out
+
+
+def e3j_conv_radial_fwd_workspace_bytes(plan: Plan, n_nodes: int, n_edges: int, hidden: int) -> int:
+    return int(_load().e3j_conv_radial_fwd_workspace_bytes(plan.handle, n_nodes, n_edges, hidden))
+
+
+def e3j_conv_radial_bwd_workspace_bytes(plan: Plan, n_nodes: int, n_edges: int, hidden: int) -> int:
+    return int(_load().e3j_conv_radial_bwd_workspace_bytes(plan.handle, n_nodes, n_edges, hidden))
+
+
+def e3j_conv_radial_fwd(plan: Plan, x, sh, h, W, senders, receivers, rowptr=None, out=None, workspace=None,
+                        stream=None):
+    """Forward convolution with the edge weights given as (h [E, hidden], W [hidden, P * N_q])."""
+    torch = _torch()
+    n, e, hidden = x.shape[0], senders.numel(), W.shape[0]
+    f32, i32 = torch.float32, torch.int32
+    if out is None:
+        out = torch.empty((n, plan.d_out, plan.n_channels), dtype=f32, device=x.device)
+    workspace = _workspace(e3j_conv_radial_fwd_workspace_bytes(plan, n, e, hidden), x, workspace)
+    _check(_load().e3j_conv_radial_fwd(
+        plan.handle, n, e, hidden,
+        _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"), _dev_ptr(sh, f32, (e, plan.d_sh), "sh"),
+        _dev_ptr(h, f32, (e, hidden), "h"), _dev_ptr(W, f32, (hidden, plan.n_paths * plan.n_channels), "W"),
+        _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
+        _dev_ptr(rowptr, i32, (n + 1,), "rowptr"),
+        _dev_ptr(out, f32, (n, plan.d_out, plan.n_channels), "out"),
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_radial_fwd")
+    return out
+
+
+def e3j_conv_radial_bwd(plan: Plan, x, sh, h, W, senders, receivers, grad_out, rowptr=None, sender_perm=None,
+                        colptr=None, grad_x=True, grad_sh=True, grad_h=True, grad_W=True, workspace=None,
+                        stream=None):
+    """Returns (grad_x, grad_sh, grad_h, grad_W); each grad_* argument is True (allocate), False/None (not
+    wanted) or a preallocated tensor."""
+    torch = _torch()
+    n, e, hidden = x.shape[0], senders.numel(), W.shape[0]
+    f32, i32 = torch.float32, torch.int32
+
+    def alloc(flag, shape):
+        if flag is True:
+            return torch.empty(shape, dtype=f32, device=x.device)
+        return flag if isinstance(flag, torch.Tensor) else None
+
+    s_w = (hidden, plan.n_paths * plan.n_channels)
+    grad_x = alloc(grad_x, (n, plan.d_in, plan.n_channels))
+    grad_sh = alloc(grad_sh, (e, plan.d_sh))
+    grad_h = alloc(grad_h, (e, hidden))
+    grad_W = alloc(grad_W, s_w)
+    workspace = _workspace(e3j_conv_radial_bwd_workspace_bytes(plan, n, e, hidden), x, workspace)
+    _check(_load().e3j_conv_radial_bwd(
+        plan.handle, n, e, hidden,
+        _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"), _dev_ptr(sh, f32, (e, plan.d_sh), "sh"),
+        _dev_ptr(h, f32, (e, hidden), "h"), _dev_ptr(W, f32, s_w, "W"),
+        _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
+        _dev_ptr(rowptr, i32, (n + 1,), "rowptr"),
+        _dev_ptr(sender_perm, i32, (e,), "sender_perm"), _dev_ptr(colptr, i32, (n + 1,), "colptr"),
+        _dev_ptr(grad_out, f32, (n, plan.d_out, plan.n_channels), "grad_out"),
+        _dev_ptr(grad_x, f32, (n, plan.d_in, plan.n_channels), "grad_x"),
+        _dev_ptr(grad_sh, f32, (e, plan.d_sh), "grad_sh"),
+        _dev_ptr(grad_h, f32, (e, hidden), "grad_h"), _dev_ptr(grad_W, f32, s_w, "grad_W"),
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_radial_bwd")
+    return grad_x, grad_sh, grad_h, grad_W
 
 
 def e3j_tp_fwd(plan: Plan, x1, x2, w, out=None, stream=None):

@@ -298,10 +298,12 @@ size_t e3j_conv_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64
     return layout(plan, n_nodes, n_edges, true).total;
 }
 
-static int conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
-                         const float* sh, const float* w, const int32_t* senders,
-                         const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
-                         size_t workspace_bytes, void* stream, bool padded) {
+}  // extern "C"
+
+int e3j::conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                       const float* sh, const float* w, const int32_t* senders,
+                       const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                       size_t workspace_bytes, void* stream, bool padded) {
     if (!plan || n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
         return E3J_ERR_INVALID_ARG;
     if (plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;  // the kernels work on groups of four channels
@@ -340,6 +342,8 @@ static int conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges,
     return after_launch();
 }
 
+extern "C" {
+
 int e3j_conv_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
                  const float* sh, const float* w, const int32_t* senders,
                  const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
@@ -356,11 +360,13 @@ int e3j_conv_fwd_padded(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges_p
                          workspace_bytes, stream, true);
 }
 
-static int conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
-                         const float* sh, const float* w, const int32_t* senders,
-                         const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
-                         const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
-                         float* grad_w, void* workspace, size_t workspace_bytes, void* stream, bool padded) {
+}  // extern "C"
+
+int e3j::conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
+                       const float* sh, const float* w, const int32_t* senders,
+                       const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                       const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
+                       float* grad_w, void* workspace, size_t workspace_bytes, void* stream, bool padded) {
     if (!plan || n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
         return E3J_ERR_INVALID_ARG;
     if (plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;  // the kernels work on groups of four channels
@@ -411,6 +417,8 @@ static int conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges,
     }
     return E3J_OK;
 }
+
+extern "C" {
 
 int e3j_conv_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
                  const float* sh, const float* w, const int32_t* senders,

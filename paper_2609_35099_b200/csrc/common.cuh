@@ -54,4 +54,13 @@ struct ConvArgs {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// The bodies of e3j_conv_fwd / e3j_conv_bwd (and their padded forms), for entry points that compose them.
+int conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x, const float* sh,
+                  const float* w, const int32_t* senders, const int32_t* receivers, const int32_t* rowptr,
+                  float* out, void* workspace, size_t workspace_bytes, void* stream, bool padded);
+int conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x, const float* sh,
+                  const float* w, const int32_t* senders, const int32_t* receivers, const int32_t* rowptr,
+                  const int32_t* sender_perm, const int32_t* colptr, const float* grad_out, float* grad_x,
+                  float* grad_sh, float* grad_w, void* workspace, size_t workspace_bytes, void* stream, bool padded);
+
 }  // namespace e3j

@@ -1,0 +1,200 @@
+// Convolution with the edge scalars taken from the radial network's last linear layer: s = h W.
+//
+// This file holds the tensor-core products around that layer (radial_gemm.cuh), the entry point that
+// materialises s, and the entry points that run the convolution on (h, W) instead of w.
+#include <algorithm>
+
+#include "common.cuh"
+#include "fast/fast_launch.cuh"
+#include "radial_gemm.cuh"
+
+namespace e3j {
+namespace radial {
+
+__global__ void layer_sum_kernel(int n_ranges, int64_t n_elems, const float* __restrict__ partial,
+                                 float* __restrict__ grad_W) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n_elems; i += stride) {
+        float acc = partial[i];
+        for (int r = 1; r < n_ranges; ++r) acc += partial[(size_t)r * n_elems + i];   // fixed order
+        grad_W[i] = acc;
+    }
+}
+
+namespace {
+
+template <class Prob>
+int launch_gemm(const Prob& prob, dim3 grid, cudaStream_t st) {
+    using L = GemmSmem<Prob::N>;
+    static_assert(L::total <= 227 * 1024, "stage ring does not fit in shared memory");
+    static thread_local int attr_dev = -1;
+    int dev = 0;
+    E3J_CUDA_TRY(cudaGetDevice(&dev));
+    if (attr_dev != dev) {
+        E3J_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32x3_kernel<Prob>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));
+        attr_dev = dev;
+    }
+    gemm_tf32x3_kernel<Prob><<<grid, kGemmThreads, L::total, st>>>(prob);
+    return after_launch();
+}
+
+inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+
+}  // namespace
+
+// number of edge ranges of the layer-gradient product on the current device
+int layer_ranges(int C) {
+    const int n_cb = (C + 127) / 128;
+    return std::max(1, fast::sm_count() / n_cb);
+}
+
+int radial_weights(int64_t n_edges, int H, int C, const float* h, const float* W, float* s, int32_t* status,
+                   cudaStream_t st) {
+    if (n_edges == 0) return E3J_OK;
+    const int n_cb = (C + 127) / 128;
+    const int n_ranges = std::max(1, fast::sm_count() / n_cb);
+    RadialWeights p{};
+    p.h = h; p.W = W; p.s = s; p.n_edges = n_edges; p.H = H; p.C = C; p.status = status;
+    p.chunk = round_up((n_edges + n_ranges - 1) / n_ranges, 128);
+    return launch_gemm(p, dim3(n_cb, n_ranges), st);
+}
+
+int grad_hidden(int64_t n_edges, int H, int C, const float* gs, const float* W, float* gh, int32_t* status,
+                cudaStream_t st) {
+    if (n_edges == 0) return E3J_OK;
+    const int n_cta = fast::sm_count();
+    GradHidden p{};
+    p.gs = gs; p.W = W; p.gh = gh; p.n_edges = n_edges; p.H = H; p.C = C; p.status = status;
+    p.chunk = round_up((n_edges + n_cta - 1) / n_cta, 128);
+    return launch_gemm(p, dim3(n_cta, (H + 63) / 64), st);
+}
+
+// partial: [layer_ranges(C)][H][C] floats of scratch
+int grad_layer(int64_t n_edges, int H, int C, const float* gs, const float* h, float* partial, float* gW,
+               int32_t* status, cudaStream_t st) {
+    const int64_t n_elems = (int64_t)H * C;
+    if (n_edges == 0) {
+        E3J_CUDA_TRY(cudaMemsetAsync(gW, 0, sizeof(float) * (size_t)n_elems, st));
+        return E3J_OK;
+    }
+    const int n_cb = (C + 127) / 128, n_ranges = layer_ranges(C);
+    GradLayer p{};
+    p.gs = gs; p.h = h; p.partial = partial; p.n_edges = n_edges; p.H = H; p.C = C; p.status = status;
+    p.chunk = round_up((n_edges + n_ranges - 1) / n_ranges, kChunkK);
+    if (int s = launch_gemm(p, dim3(n_cb, n_ranges, (H + 63) / 64), st)) return s;
+    const int blocks = (int)std::min<int64_t>((n_elems + 255) / 256, 4 * fast::sm_count());
+    layer_sum_kernel<<<blocks, 256, 0, st>>>(n_ranges, n_elems, partial, gW);
+    return after_launch();
+}
+
+namespace {
+
+// workspace of the composed calls: [conv workspace | s | grad_s | layer partials]
+struct RadialLayout {
+    size_t conv, s, gs, partial, total, conv_bytes;
+};
+RadialLayout radial_layout(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int H, bool bwd) {
+    RadialLayout L{};
+    const size_t C = (size_t)plan->P * plan->nq;
+    L.conv_bytes = bwd ? e3j_conv_bwd_workspace_bytes(plan, n_nodes, n_edges)
+                       : e3j_conv_fwd_workspace_bytes(plan, n_nodes, n_edges);
+    size_t off = 0;
+    L.conv = off; off = align_up(off + L.conv_bytes, 256);
+    L.s = off; off = align_up(off + 4 * (size_t)std::max<int64_t>(n_edges, 1) * C, 256);
+    L.gs = off; if (bwd) off = align_up(off + 4 * (size_t)std::max<int64_t>(n_edges, 1) * C, 256);
+    L.partial = off; if (bwd) off = align_up(off + 4 * (size_t)(fast::kMaxSms) * H * C, 256);
+    L.total = off;
+    return L;
+}
+
+bool radial_args_ok(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int H) {
+    return plan && n_nodes >= 0 && n_edges >= 0 && n_nodes < (1ll << 31) - 1 && n_edges < (1ll << 31) - 1 && H > 0;
+}
+
+}  // namespace
+}  // namespace radial
+}  // namespace e3j
+
+using namespace e3j;
+
+extern "C" {
+
+int e3j_radial_weights(const e3j_plan* plan, int64_t n_edges, int hidden, const float* h, const float* W,
+                       float* w_out, void* stream) {
+    if (!radial::radial_args_ok(plan, 0, n_edges, hidden)) return E3J_ERR_INVALID_ARG;
+    if (hidden % 4 != 0 || plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;
+    if (n_edges == 0) return E3J_OK;
+    if (!h || !W || !w_out) return E3J_ERR_INVALID_ARG;
+    if (((uintptr_t)h | (uintptr_t)W | (uintptr_t)w_out) & 15u) return E3J_ERR_INVALID_ARG;
+    DeviceTables t;
+    if (int s = get_device_tables(plan, t)) return s;
+    return radial::radial_weights(n_edges, hidden, plan->P * plan->nq, h, W, w_out, t.status, (cudaStream_t)stream);
+}
+
+size_t e3j_conv_radial_fwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden) {
+    if (!radial::radial_args_ok(plan, n_nodes, n_edges, hidden)) return 0;
+    return radial::radial_layout(plan, n_nodes, n_edges, hidden, false).total;
+}
+
+size_t e3j_conv_radial_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden) {
+    if (!radial::radial_args_ok(plan, n_nodes, n_edges, hidden)) return 0;
+    return radial::radial_layout(plan, n_nodes, n_edges, hidden, true).total;
+}
+
+int e3j_conv_radial_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
+                        const float* sh, const float* h, const float* W, const int32_t* senders,
+                        const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    if (!radial::radial_args_ok(plan, n_nodes, n_edges, hidden)) return E3J_ERR_INVALID_ARG;
+    if (hidden % 4 != 0 || plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;
+    if (n_nodes == 0) return E3J_OK;
+    if (n_edges > 0 && (!h || !W)) return E3J_ERR_INVALID_ARG;
+    if (((uintptr_t)h | (uintptr_t)W) & 15u) return E3J_ERR_INVALID_ARG;
+    const radial::RadialLayout L = radial::radial_layout(plan, n_nodes, n_edges, hidden, false);
+    if (!workspace || ((uintptr_t)workspace & 255u) || workspace_bytes < L.total) return E3J_ERR_WORKSPACE;
+    char* ws = (char*)workspace;
+    float* s = (float*)(ws + L.s);
+    if (n_edges > 0) {
+        DeviceTables t;
+        if (int st = get_device_tables(plan, t)) return st;
+        if (int st = radial::radial_weights(n_edges, hidden, plan->P * plan->nq, h, W, s, t.status, (cudaStream_t)stream))
+            return st;
+    }
+    return conv_fwd_impl(plan, n_nodes, n_edges, x, sh, s, senders, receivers, rowptr, out, ws + L.conv, L.conv_bytes,
+                         stream, false);
+}
+
+int e3j_conv_radial_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
+                        const float* sh, const float* h, const float* W, const int32_t* senders,
+                        const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                        const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_sh,
+                        float* grad_h, float* grad_W, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!radial::radial_args_ok(plan, n_nodes, n_edges, hidden)) return E3J_ERR_INVALID_ARG;
+    if (hidden % 4 != 0 || plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;
+    if (n_nodes == 0) return E3J_OK;
+    if (!W || (n_edges > 0 && !h)) return E3J_ERR_INVALID_ARG;
+    if (((uintptr_t)h | (uintptr_t)W | (uintptr_t)grad_h | (uintptr_t)grad_W) & 15u) return E3J_ERR_INVALID_ARG;
+    const radial::RadialLayout L = radial::radial_layout(plan, n_nodes, n_edges, hidden, true);
+    if (!workspace || ((uintptr_t)workspace & 255u) || workspace_bytes < L.total) return E3J_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* ws = (char*)workspace;
+    float* s = (float*)(ws + L.s);
+    float* gs = (float*)(ws + L.gs);
+    const int C = plan->P * plan->nq;
+    DeviceTables t;
+    if (int rc = get_device_tables(plan, t)) return rc;
+    if (int rc = radial::radial_weights(n_edges, hidden, C, h, W, s, t.status, st)) return rc;
+    // the convolution's own backward, with the edge-scalar cotangent kept as scratch
+    const bool want_gs = grad_h || grad_W;
+    if (int rc = conv_bwd_impl(plan, n_nodes, n_edges, x, sh, s, senders, receivers, rowptr, sender_perm, colptr,
+                               grad_out, grad_x, grad_sh, want_gs ? gs : nullptr, ws + L.conv, L.conv_bytes, stream,
+                               false)) return rc;
+    // chain rule through s = h W
+    if (grad_h)
+        if (int rc = radial::grad_hidden(n_edges, hidden, C, gs, W, grad_h, t.status, st)) return rc;
+    if (grad_W)
+        if (int rc = radial::grad_layer(n_edges, hidden, C, gs, h, (float*)(ws + L.partial), grad_W, t.status, st)) return rc;
+    return E3J_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,339 @@
+// Dense products around the radial network's last layer, on the fifth-generation tensor cores (sm_100a).
+//
+// One kernel template computes C[m, n] = sum_k A[m, k] * B[n, k] for float32 operands with the three-term TF32
+// split of umma.cuh.  Output tiles are 128 (m) x N (n = 64 or 128) and live in tensor memory while the K loop
+// runs; operands pass through a ring of shared-memory stages of 32 k each, written by converter warps that read
+// float32 from global memory, split every value into its (hi, lo) TF32 pair and store both in the K-major
+// core-matrix layout that the tensor cores read.  Roles: warps 0-3 read finished tiles out of tensor memory
+// and store them, warps 4-7 convert, warp 8 issues the tcgen05.mma instructions (one lane).
+//
+// A Problem type describes one product: which output tiles a CTA owns, how many K chunks a tile has, where
+// operand values come from (zero outside the matrices) and where results go.  Three instances are used:
+//   s^T      = W^T h^T      edge scalars from the hidden activations            (RadialWeights)
+//   grad_h   = grad_s W^T   cotangent of the hidden activations                 (GradHidden)
+//   grad_W^T = grad_s^T h   cotangent of the layer, per edge range of a CTA     (GradLayer, then an ordered sum)
+//
+// Accumulation: the tensor cores add into their float32 accumulators with truncation, so a long chain of
+// products drifts (measured: 2e-5 relative after 1200 accumulation steps).  A tile of the pipeline therefore
+// covers at most kGroupChunks K chunks (96 steps); where a sum is longer, the epilogue warps add the finished
+// partial tiles in float32 registers (round to nearest) and store once the last group has arrived
+// (Prob::ACCUMULATE, Prob::flush).
+//
+// Every wait is bounded (fast::mbar_wait): on a time-out the CTA records the failure in the status word,
+// stops issuing work, lets the tensor cores drain, frees its tensor memory and returns.
+#pragma once
+#include "fast/fast_common.cuh"
+#include "umma.cuh"
+
+namespace e3j {
+namespace radial {
+
+constexpr int kTileM = 128;      // rows of an output tile = tensor-memory lanes
+constexpr int kChunkK = 32;      // k per shared-memory stage (four tcgen05.mma steps of 8)
+constexpr int kStages = 3;
+constexpr int kGroupChunks = 8;  // K chunks accumulated inside tensor memory before the tile is read out
+constexpr int kGemmThreads = 9 * 32;
+
+template <int N>
+struct GemmSmem {
+    static constexpr size_t a_bytes = (size_t)kTileM * kChunkK * 4;   // one of hi / lo
+    static constexpr size_t b_bytes = (size_t)N * kChunkK * 4;
+    static constexpr size_t stage_bytes = 2 * a_bytes + 2 * b_bytes;  // A_hi, A_lo, B_hi, B_lo
+    static constexpr size_t off_bar = 0;       // stage_full[kStages], stage_empty[kStages], d_full[2], d_empty[2], drain
+    static constexpr size_t off_tmem = 8 * (2 * kStages + 5);
+    static constexpr size_t off_abort = off_tmem + 4;
+    static constexpr size_t off_stage = 1024;
+    static constexpr size_t total = off_stage + kStages * stage_bytes;
+};
+
+// Converter: fills rows [0, ROWS) x k [0, 32) of one operand of one stage.  LANE_ROWS = 8: a warp item is
+// 8 rows x 4 k-quads (sources with k contiguous); LANE_ROWS = 32: 32 rows x 1 k-quad (sources with rows
+// contiguous).  Either way 8 consecutive lanes write 128 contiguous bytes of shared memory.
+template <int ROWS, int LANE_ROWS, class Load>
+__device__ __forceinline__ void convert_operand(unsigned char* hi, unsigned char* lo, const int cwarp, const int lane,
+                                                const Load& load) {
+    constexpr int QUADS = kChunkK / 4;
+    constexpr int LANE_QUADS = 32 / LANE_ROWS;
+    constexpr int ITEMS = (ROWS / LANE_ROWS) * (QUADS / LANE_QUADS);   // warp items of the operand
+    static_assert(ROWS % LANE_ROWS == 0 && QUADS % LANE_QUADS == 0, "operand does not tile");
+#pragma unroll 2
+    for (int item = cwarp; item < ITEMS; item += 4) {
+        const int rg = item / (QUADS / LANE_QUADS), qg = item % (QUADS / LANE_QUADS);
+        const int row = rg * LANE_ROWS + lane % LANE_ROWS;
+        const int quad = qg * LANE_QUADS + lane / LANE_ROWS;
+        const float4 v = load(row, quad * 4);
+        float4 h, l;
+        umma::split_tf32(v, h, l);
+        const uint32_t off = umma::tile_offset(row, quad * 4, kChunkK);
+        *reinterpret_cast<float4*>(hi + off) = h;
+        *reinterpret_cast<float4*>(lo + off) = l;
+    }
+}
+
+template <class Prob>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob prob) {
+    constexpr int N = Prob::N;
+    using L = GemmSmem<N>;
+    constexpr uint32_t kTmemCols = 2 * N;   // two accumulator tiles
+    static_assert(kTmemCols == 128 || kTmemCols == 256, "tensor-memory allocation must be a power of two");
+    extern __shared__ __align__(1024) unsigned char smem[];
+    uint64_t* stage_full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
+    uint64_t* stage_empty = stage_full + kStages;
+    uint64_t* d_full = stage_empty + kStages;
+    uint64_t* d_empty = d_full + 2;
+    uint64_t* drain = d_empty + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::off_tmem);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { fast::mbar_init(&stage_full[s], 4); fast::mbar_init(&stage_empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { fast::mbar_init(&d_full[b], 1); fast::mbar_init(&d_empty[b], 4); }
+        fast::mbar_init(drain, 1);
+        *abort_flag = 0;
+        fast::mbar_fence_init();
+    }
+    if (warp == 8) umma::tmem_alloc(tmem_slot, kTmemCols);
+    umma::fence_before_sync();
+    __syncthreads();
+    umma::fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int n_tiles = prob.n_tiles();
+    if (warp < 4) {
+        // ------------------------------------------------ epilogue: tensor memory -> registers -> global
+        float acc[Prob::ACCUMULATE ? N : 1];
+#pragma unroll
+        for (int i = 0; i < (Prob::ACCUMULATE ? N : 1); ++i) acc[i] = 0.f;
+        for (int t = 0; t < n_tiles; ++t) {
+            const int db = t & 1;
+            if (!fast::mbar_wait(&d_full[db], (t >> 1) & 1, abort_flag, prob.status)) break;
+            umma::fence_after_sync();
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(db * N);
+            const bool flush = prob.flush(t);
+#pragma unroll
+            for (int c0 = 0; c0 < N; c0 += 32) {
+                float v[32];
+                umma::tmem_ld32(taddr + c0, v);
+                umma::tmem_ld_wait();
+                if (c0 + 32 == N) {   // the tile has left tensor memory: the next product may overwrite it
+                    umma::fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) fast::mbar_arrive(&d_empty[db]);
+                }
+                if constexpr (Prob::ACCUMULATE) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) { v[i] += acc[c0 + i]; acc[c0 + i] = flush ? 0.f : v[i]; }
+                }
+                if (flush) prob.store(t, warp * 32 + lane, c0, v);
+            }
+        }
+    } else if (warp < 8) {
+        // ------------------------------------------------ converters: global float32 -> (hi, lo) TF32 stages
+        const int cwarp = warp - 4;
+        int it = 0;
+        bool ok = true;
+        for (int t = 0; ok && t < n_tiles; ++t) {
+            const int n_chunks = prob.n_chunks(t);
+            for (int kc = 0; kc < n_chunks; ++kc, ++it) {
+                const int s = it % kStages;
+                if (it >= kStages && !fast::mbar_wait(&stage_empty[s], ((it / kStages) + 1) & 1, abort_flag, prob.status)) { ok = false; break; }
+                unsigned char* st = smem + L::off_stage + (size_t)s * L::stage_bytes;
+                convert_operand<kTileM, Prob::A_LANE_ROWS>(st, st + L::a_bytes, cwarp, lane,
+                    [&](int row, int k) { return prob.load_a(t, kc, row, k); });
+                convert_operand<N, Prob::B_LANE_ROWS>(st + 2 * L::a_bytes, st + 2 * L::a_bytes + L::b_bytes, cwarp, lane,
+                    [&](int row, int k) { return prob.load_b(t, kc, row, k); });
+                umma::fence_smem_to_async();
+                __syncwarp();
+                if (lane == 0) fast::mbar_arrive(&stage_full[s]);
+            }
+        }
+    } else {
+        // ------------------------------------------------ tensor-core issue (lane 0 of warp 8)
+        constexpr uint32_t idesc = umma::idesc_tf32(kTileM, N);
+        const uint32_t sbo = umma::sbo_bytes(kChunkK);
+        int it = 0;
+        bool ok = true;
+        for (int t = 0; ok && t < n_tiles; ++t) {
+            const int db = t & 1;
+            const int n_chunks = prob.n_chunks(t);
+            if (t >= 2 && !fast::mbar_wait(&d_empty[db], ((t >> 1) + 1) & 1, abort_flag, prob.status)) break;
+            for (int kc = 0; kc < n_chunks; ++kc, ++it) {
+                const int s = it % kStages;
+                if (!fast::mbar_wait(&stage_full[s], (it / kStages) & 1, abort_flag, prob.status)) { ok = false; break; }
+                umma::fence_after_sync();
+                if (lane == 0) {
+                    const uint32_t a_hi = umma::smem_addr(smem + L::off_stage + (size_t)s * L::stage_bytes);
+                    const uint32_t a_lo = a_hi + (uint32_t)L::a_bytes;
+                    const uint32_t b_hi = a_hi + 2 * (uint32_t)L::a_bytes, b_lo = b_hi + (uint32_t)L::b_bytes;
+                    const uint32_t d = tmem_base + (uint32_t)(db * N);
+                    // small terms first: a_lo b_hi, a_hi b_lo, then a_hi b_hi
+                    const uint32_t pa[3] = {a_lo, a_hi, a_hi}, pb[3] = {b_hi, b_lo, b_hi};
+#pragma unroll
+                    for (int pass = 0; pass < 3; ++pass)
+#pragma unroll
+                        for (int ks = 0; ks < kChunkK / 8; ++ks)
+                            umma::mma_tf32(d, umma::make_desc(pa[pass] + ks * 2 * umma::kLbo, umma::kLbo, sbo),
+                                           umma::make_desc(pb[pass] + ks * 2 * umma::kLbo, umma::kLbo, sbo), idesc,
+                                           (kc > 0 || pass > 0 || ks > 0) ? 1u : 0u);
+                    umma::commit(&stage_empty[s]);                       // the stage may be refilled
+                    if (kc == n_chunks - 1) umma::commit(&d_full[db]);   // the tile is complete
+                }
+                __syncwarp();
+            }
+        }
+        // abort path only: let the products still in flight finish before tensor memory is freed
+        if (*abort_flag) {
+            if (lane == 0) umma::commit(drain);
+            __syncwarp();
+#pragma unroll 1
+            for (uint32_t spin = 0; spin < fast::kSpinLimit; ++spin)
+                if (fast::mbar_try_wait(drain, 0)) break;
+        }
+    }
+    umma::fence_before_sync();
+    __syncthreads();
+    if (warp == 8) umma::tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ------------------------------------------------------------------------------------------------ problems
+// s[e, c] = sum_j h[e, j] W[j, c]: tile (column block cb of 128 c) x (128 edges); m = c, n = edge, k = j.
+struct RadialWeights {
+    static constexpr int N = 128, A_LANE_ROWS = 32, B_LANE_ROWS = 8;
+    static constexpr bool ACCUMULATE = false;   // k = hidden is short: one chain per tile
+    __device__ __forceinline__ bool flush(int) const { return true; }
+    const float* h; const float* W; float* s;
+    int64_t n_edges, chunk;   // chunk: edges per CTA row of the grid (multiple of 128)
+    int H, C;
+    int32_t* status;
+    __device__ __forceinline__ int64_t e_begin() const { return min(n_edges, (int64_t)blockIdx.y * chunk); }
+    __device__ __forceinline__ int n_tiles() const {
+        const int64_t e0 = e_begin(), e1 = min(n_edges, e0 + chunk);
+        return (int)((e1 - e0 + 127) / 128);
+    }
+    __device__ __forceinline__ int n_chunks(int) const { return (H + kChunkK - 1) / kChunkK; }
+    __device__ __forceinline__ float4 load_a(int, int kc, int row, int k) const {   // W^T: row = c, k = j
+        const int c = blockIdx.x * 128 + row, j = kc * kChunkK + k;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < C) {
+            if (j + 0 < H) v.x = W[(size_t)(j + 0) * C + c];
+            if (j + 1 < H) v.y = W[(size_t)(j + 1) * C + c];
+            if (j + 2 < H) v.z = W[(size_t)(j + 2) * C + c];
+            if (j + 3 < H) v.w = W[(size_t)(j + 3) * C + c];
+        }
+        return v;
+    }
+    __device__ __forceinline__ float4 load_b(int t, int kc, int row, int k) const {   // h: row = edge, k = j
+        const int64_t e = e_begin() + (int64_t)t * 128 + row;
+        const int j = kc * kChunkK + k;
+        if (e >= n_edges || e >= e_begin() + chunk || j >= H) return make_float4(0.f, 0.f, 0.f, 0.f);
+        return *reinterpret_cast<const float4*>(h + (size_t)e * H + j);   // H % 4 == 0
+    }
+    __device__ __forceinline__ void store(int t, int m, int n0, const float (&v)[32]) const {
+        const int c = blockIdx.x * 128 + m;
+        if (c >= C) return;
+        const int64_t e0 = e_begin() + (int64_t)t * 128 + n0;
+        const int64_t e_end = min(n_edges, e_begin() + chunk);
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (e0 + i < e_end) s[(size_t)(e0 + i) * C + c] = v[i];   // lanes: consecutive c
+    }
+};
+
+// grad_h[e, j] = sum_c grad_s[e, c] W[j, c]: tile = 128 edges x (64 j, block blockIdx.y); m = edge, n = j, k = c.
+struct GradHidden {
+    static constexpr int N = 64, A_LANE_ROWS = 8, B_LANE_ROWS = 8;
+    static constexpr bool ACCUMULATE = true;
+    const float* gs; const float* W; float* gh;
+    int64_t n_edges, chunk;   // chunk: edges per CTA (multiple of 128)
+    int H, C;
+    int32_t* status;
+    // pipeline tile t = (edge tile t / groups, group t % groups of kGroupChunks chunks of c)
+    __device__ __forceinline__ int total_chunks() const { return (C + kChunkK - 1) / kChunkK; }
+    __device__ __forceinline__ int groups() const { return (total_chunks() + kGroupChunks - 1) / kGroupChunks; }
+    __device__ __forceinline__ int64_t e_begin() const { return min(n_edges, (int64_t)blockIdx.x * chunk); }
+    __device__ __forceinline__ int n_tiles() const {
+        const int64_t e0 = e_begin(), e1 = min(n_edges, e0 + chunk);
+        return (int)((e1 - e0 + 127) / 128) * groups();
+    }
+    __device__ __forceinline__ int n_chunks(int t) const {
+        return min(kGroupChunks, total_chunks() - (t % groups()) * kGroupChunks);
+    }
+    __device__ __forceinline__ bool flush(int t) const { return t % groups() == groups() - 1; }
+    __device__ __forceinline__ float4 load_a(int t, int kc, int row, int k) const {   // grad_s: row = edge, k = c
+        const int g = groups();
+        const int64_t e = e_begin() + (int64_t)(t / g) * 128 + row;
+        const int c = ((t % g) * kGroupChunks + kc) * kChunkK + k;
+        if (e >= n_edges || e >= e_begin() + chunk || c >= C) return make_float4(0.f, 0.f, 0.f, 0.f);
+        return *reinterpret_cast<const float4*>(gs + (size_t)e * C + c);   // C % 4 == 0
+    }
+    __device__ __forceinline__ float4 load_b(int t, int kc, int row, int k) const {   // W: row = j, k = c
+        const int c = ((t % groups()) * kGroupChunks + kc) * kChunkK + k, j = blockIdx.y * 64 + row;
+        if (j >= H || c >= C) return make_float4(0.f, 0.f, 0.f, 0.f);
+        return *reinterpret_cast<const float4*>(W + (size_t)j * C + c);
+    }
+    __device__ __forceinline__ void store(int t, int m, int n0, const float (&v)[32]) const {
+        const int64_t e = e_begin() + (int64_t)(t / groups()) * 128 + m;
+        if (e >= n_edges || e >= e_begin() + chunk) return;
+        const int j0 = blockIdx.y * 64 + n0;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+            if (j0 + i < H)   // H % 4 == 0
+                *reinterpret_cast<float4*>(gh + (size_t)e * H + j0 + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+    }
+};
+
+// partial[r, j, c] = sum over the edges of range r of h[e, j] grad_s[e, c]: one tile per CTA,
+// m = c (column block of 128), n = j (block blockIdx.z of 64), k = edge.  grad_W = sum_r partial[r] in range
+// order (layer_sum_kernel).
+struct GradLayer {
+    static constexpr int N = 64, A_LANE_ROWS = 32, B_LANE_ROWS = 32;
+    static constexpr bool ACCUMULATE = true;
+    const float* gs; const float* h; float* partial;
+    int64_t n_edges, chunk;   // chunk: edges per range (multiple of 32)
+    int H, C;
+    int32_t* status;
+    __device__ __forceinline__ int64_t e_begin() const { return min(n_edges, (int64_t)blockIdx.y * chunk); }
+    // pipeline tile t = group t of kGroupChunks chunks of the range's edges; one output tile per CTA
+    __device__ __forceinline__ int total_chunks() const {
+        const int64_t e0 = e_begin(), e1 = min(n_edges, e0 + chunk);
+        return (int)max((int64_t)1, (e1 - e0 + kChunkK - 1) / kChunkK);   // an empty range still writes a zero tile
+    }
+    __device__ __forceinline__ int n_tiles() const { return (total_chunks() + kGroupChunks - 1) / kGroupChunks; }
+    __device__ __forceinline__ int n_chunks(int t) const { return min(kGroupChunks, total_chunks() - t * kGroupChunks); }
+    __device__ __forceinline__ bool flush(int t) const { return t == n_tiles() - 1; }
+    __device__ __forceinline__ float4 column(const float* base, int ld, int col, bool col_ok, int kc, int k) const {
+        const int64_t e = e_begin() + (int64_t)kc * kChunkK + k, e_end = min(n_edges, e_begin() + chunk);
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (col_ok) {
+            if (e + 0 < e_end) v.x = base[(size_t)(e + 0) * ld + col];
+            if (e + 1 < e_end) v.y = base[(size_t)(e + 1) * ld + col];
+            if (e + 2 < e_end) v.z = base[(size_t)(e + 2) * ld + col];
+            if (e + 3 < e_end) v.w = base[(size_t)(e + 3) * ld + col];
+        }
+        return v;
+    }
+    __device__ __forceinline__ float4 load_a(int t, int kc, int row, int k) const {   // grad_s^T: row = c, k = edge
+        const int c = blockIdx.x * 128 + row;
+        return column(gs, C, c, c < C, t * kGroupChunks + kc, k);
+    }
+    __device__ __forceinline__ float4 load_b(int t, int kc, int row, int k) const {   // h^T: row = j, k = edge
+        const int j = blockIdx.z * 64 + row;
+        return column(h, H, j, j < H, t * kGroupChunks + kc, k);
+    }
+    __device__ __forceinline__ void store(int, int m, int n0, const float (&v)[32]) const {
+        const int c = blockIdx.x * 128 + m;
+        if (c >= C) return;
+        float* dst = partial + (size_t)blockIdx.y * H * C;
+        const int j0 = blockIdx.z * 64 + n0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (j0 + i < H) dst[(size_t)(j0 + i) * C + c] = v[i];   // lanes: consecutive c
+    }
+};
+
+// grad_W[j, c] = sum_r partial[r, j, c], r ascending.
+__global__ void layer_sum_kernel(int n_ranges, int64_t n_elems, const float* __restrict__ partial, float* __restrict__ grad_W);
+
+}  // namespace radial
+}  // namespace e3j

@@ -1,0 +1,116 @@
+// Fifth-generation tensor-core building blocks (sm_100a): tensor-memory allocation, shared-memory matrix
+// descriptors, tcgen05.mma issue / commit, tensor-memory loads, and the split of float32 operands into two
+// TF32 terms.  Used by the kernels that form the edge scalars s = h W (the radial network's last layer) on the
+// tensor cores, standalone or inside the convolution.
+//
+// Operand layout used everywhere in this library: K-major, no swizzle.  A tile of R rows by K columns of
+// 32-bit elements is stored as core matrices of 8 rows x 16 bytes (four elements of one row are contiguous,
+// the 8 rows of a core matrix follow each other at 16 bytes); core matrices that are neighbours along K sit
+// kLbo bytes apart, neighbours along the rows kSbo(K) bytes apart:
+//     byte(r, k) = (r / 8) * sbo + (k / 4) * 128 + (r % 8) * 16 + (k % 4) * 4,        sbo = (K / 4) * 128
+// One tcgen05.mma of kind::tf32 consumes K = 8 (two core matrices along K); the descriptor of step j starts
+// 256 bytes after that of step j - 1.
+//
+// Accuracy: the tensor cores multiply TF32 values (10 explicit mantissa bits).  Every float32 operand v is
+// therefore split into hi = tf32(v) and lo = tf32(v - hi), and a product a b is accumulated as
+// a_lo b_hi + a_hi b_lo + a_hi b_hi (the term a_lo b_lo, below 2^-22 of the product, is dropped), which keeps
+// the float32 accumulators within a few float32 roundings of the exact product.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace e3j {
+namespace umma {
+
+constexpr uint32_t kLbo = 128;   // bytes between core matrices that are neighbours along K
+__host__ __device__ constexpr uint32_t sbo_bytes(int k_elems) { return (uint32_t)(k_elems / 4) * 128u; }
+// byte offset of element (r, k) of a K-major tile with K = k_elems
+__host__ __device__ constexpr uint32_t tile_offset(int r, int k, int k_elems) {
+    return (uint32_t)(r / 8) * sbo_bytes(k_elems) + (uint32_t)(k / 4) * 128u + (uint32_t)(r % 8) * 16u + (uint32_t)(k % 4) * 4u;
+}
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// 64-bit shared-memory matrix descriptor: start address, leading (K) and stride (row) byte offsets in units
+// of 16 bytes, descriptor version 1 (sm_100), no swizzle, base offset 0.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+    const uint32_t lo = ((saddr >> 4) & 0x3FFFu) | (((lbo >> 4) & 0x3FFFu) << 16);
+    const uint32_t hi = ((sbo >> 4) & 0x3FFFu) | (1u << 14);
+    return ((uint64_t)hi << 32) | lo;
+}
+
+// 32-bit instruction descriptor of kind::tf32: float32 accumulators, TF32 A and B, both K-major, dense.
+__host__ __device__ constexpr uint32_t idesc_tf32(int m, int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// D[tmem] (+)= A[smem] * B[smem]; issued by ONE thread.  accumulate = 0 overwrites D.
+__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier receives one arrival when every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// makes this thread's shared-memory writes visible to the tensor cores (asynchronous proxy)
+__device__ __forceinline__ void fence_smem_to_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Tensor memory: allocation by one whole warp; the base address (lane 0, first column) lands in *slot.
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t columns) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_addr(slot)), "r"(columns) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t base, uint32_t columns) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(columns) : "memory");
+}
+
+// A warp reads its 32 lanes of tensor memory (lanes 32 * (warp % 4) ...): thread t gets lane t, columns
+// [col, col + N).  taddr = base + (lane0 << 16) + col.
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// float32 -> (hi, lo) TF32 pair, both rounded to nearest; v = hi + lo up to 2^-22 |v|.
+__device__ __forceinline__ void split_tf32(float v, float& hi, float& lo) {
+    uint32_t h, l;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(v));
+    hi = __uint_as_float(h);
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(l) : "f"(v - hi));
+    lo = __uint_as_float(l);
+}
+__device__ __forceinline__ void split_tf32(const float4 v, float4& hi, float4& lo) {
+    split_tf32(v.x, hi.x, lo.x); split_tf32(v.y, hi.y, lo.y); split_tf32(v.z, hi.z, lo.z); split_tf32(v.w, hi.w, lo.w);
+}
+
+}  // namespace umma
+}  // namespace e3j

@@ -287,6 +287,19 @@ def make_features(wl: Workload, n_paths: int, n_out: int, with_weights: bool = T
     return x, y, w, grad_out
 
 
+def make_radial(wl: Workload, n_paths: int, hidden: int = 64):
+    """Stand-ins for the radial network's last layer: hidden activations h[E, hidden] ~ N(0,1) and the layer
+    matrix W[hidden, P * N_q] ~ N(0, 1/hidden), float32 (so that h W has the unit scale of the stand-in weights
+    of make_features).  The paper gives num_rbf = 8 and no layer sizes; 64 is the usual width of MACE's radial
+    perceptron."""
+    c = CONFIGS[wl.config]
+    rng = np.random.Generator(np.random.PCG64([c["seed"], 2]))
+    nq, _, _ = feature_dims(wl.irreps_in, wl.sh_lmax)
+    h = rng.standard_normal((wl.n_edges, hidden), dtype=np.float32)
+    W = rng.standard_normal((hidden, n_paths * nq), dtype=np.float32) * np.float32(1.0 / np.sqrt(hidden))
+    return h, W
+
+
 def make_tp_rows(rows: int, n_paths: int, n_out: int, seed: int = 4):
     """Config 4: x1[B,9,128], x2[B,16], w[B,P,128], grad_out[B,D,128], N(0,1) float32."""
     c = CONFIGS[4]
