@@ -7,6 +7,18 @@
 
 namespace e3j {
 
+// The radial network's last layer and the slot tables of the graph (device pointers).
+struct RadialArgs {
+    const float* h;            // [n_edges, hidden]
+    const float* W;            // [hidden, P * N_q]
+    int hidden;
+    const int32_t* slotptr;    // [n_nodes + 1] first slot of every receiver; slotptr[n_nodes] = number of slots
+    const int32_t* slot_edge;  // [slots] edge of the slot, or -1 (padding to a multiple of 8 per receiver)
+    const int32_t* group_recv; // [slots / 8] receiver of every group of 8 slots
+    void* scratch;             // boundary rows: as for conv_fwd, sized by radial_fwd_scratch_bytes
+    size_t scratch_bytes;
+};
+
 struct FastKernels {
     const char* signature;  // plan signature this entry was generated for
     size_t (*fwd_scratch_bytes)(int64_t n_nodes, int64_t n_edges);
@@ -22,6 +34,9 @@ struct FastKernels {
     // dbl_out the cotangent of grad_out into args.out.
     int (*dbl_edges)(const ConvArgs&, const float* ct_x, const float* ct_sh, const float* ct_w);
     int (*dbl_out)(const ConvArgs&, const float* ct_x, const float* ct_sh, const float* ct_w);
+    // forward with the edge scalars formed in the kernel from the radial layer (null: the caller materialises
+    // them first); see fast/fast_radial.cuh
+    int (*radial_fwd)(const ConvArgs&, const RadialArgs&);
 };
 
 // Index of the entry generated for `signature`, or -1.

@@ -495,6 +495,8 @@ class Sig:
         o.append('#include "fast_fwd.cuh"')
         o.append('#include "fast_bwd.cuh"')
         o.append('#include "fast_launch.cuh"')
+        if self.cfg.get("RF", 0):
+            o.append('#include "fast_radial.cuh"')
         o.append("")
         o.append("namespace e3j {\nnamespace fast {\nnamespace {")
         o.append(f"__device__ const PairRec kPair_{self.name}[{len(pair_tab)}] = {{")
@@ -638,6 +640,22 @@ class Sig:
                 o.append(f"            dst[{row - bounds[g]} * stride] = acc[{row - bounds[g]}];")
             o.append("        }")
         o.append("    }")
+        if self.cfg.get("RF", 0):
+            # forward A entries of one edge from harmonics held in registers (the convolution that forms its
+            # edge scalars from the radial layer computes them with one lane per edge)
+            assert len(slots) % 4 == 0
+            o.append(f"    // A[slot] = sum over the slot's records of c * y[i2], four slots per store")
+            o.append(f"    __device__ static __forceinline__ void a_entries(const float (&y)[DSH], float4* __restrict__ dst) {{")
+            for q in range(len(slots) // 4):
+                terms = []
+                for s_i in range(4 * q, 4 * q + 4):
+                    pi = slots[s_i]
+                    if pi is None:
+                        terms.append("0.f")
+                    else:
+                        terms.append(" + ".join(f"{fmt_float(v)} * y[{i2}]" for i2, v in self.pairs[pi][3]))
+                o.append(f"        dst[{q}] = make_float4({', '.join(terms)});")
+            o.append("    }")
         o += bwd_lines
         o.append("};")
         o.append("}  // namespace")
@@ -652,7 +670,8 @@ class Sig:
                      f"&fast::launch_tp_bwd<fast::{S}>,")
             dbl_e = f"&fast::launch_dbl_edges<fast::{S}>" if self.cfg.get("DT", 0) else "nullptr"
             dbl_o = f"&fast::launch_dbl_out<fast::{S}>" if self.cfg.get("DFT", 0) else "nullptr"
-            o.append(f"    {dbl_e}, {dbl_o}}};")
+            rf = f", &fast::launch_radial_fwd<fast::{S}>" if self.cfg.get("RF", 0) else ""
+            o.append(f"    {dbl_e}, {dbl_o}{rf}}};")
         else:
             o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, nullptr, &fast::launch_fwd<fast::{S}>, nullptr, nullptr, nullptr, "
                      f"nullptr, nullptr}};")

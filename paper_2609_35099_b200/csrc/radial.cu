@@ -6,9 +6,15 @@
 
 #include "common.cuh"
 #include "fast/fast_launch.cuh"
+#include "fast/fast_radial.cuh"
+#include "fast_registry.hpp"
 #include "radial_gemm.cuh"
 
 namespace e3j {
+
+int graph_prepare(int64_t, int64_t, const int32_t*, const int32_t*, int32_t*, int32_t*, int32_t*, cudaStream_t,
+                  bool padded = false);
+
 namespace radial {
 
 __global__ void layer_sum_kernel(int n_ranges, int64_t n_elems, const float* __restrict__ partial,
@@ -89,16 +95,38 @@ int grad_layer(int64_t n_edges, int H, int C, const float* gs, const float* h, f
 
 namespace {
 
-// workspace of the composed calls: [conv workspace | s | grad_s | layer partials]
+// Does the plan have a kernel that forms the edge scalars itself, for this hidden width?
+const FastKernels* fused_forward(const e3j_plan* plan, int H) {
+    const FastKernels* fk = fast_lookup(plan);
+    return (fk && fk->radial_fwd && fk->fwd_scratch_bytes && H % 8 == 0 && H <= fast::kMaxHidden) ? fk : nullptr;
+}
+
+// workspace of the composed calls: [conv workspace | s | grad_s | layer partials]; of the forward with in-kernel
+// edge scalars: [rowptr | slotptr | slot_edge | group_recv | boundary-row scratch]
 struct RadialLayout {
     size_t conv, s, gs, partial, total, conv_bytes;
+    size_t rowptr, slotptr, slot_edge, group_recv, scratch, scratch_bytes;
+    bool fused;
 };
 RadialLayout radial_layout(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int H, bool bwd) {
     RadialLayout L{};
     const size_t C = (size_t)plan->P * plan->nq;
+    size_t off = 0;
+    const FastKernels* fk = bwd ? nullptr : fused_forward(plan, H);
+    if (fk) {
+        L.fused = true;
+        const size_t cap = (size_t)fast::radial_slot_capacity(n_nodes, n_edges);
+        L.rowptr = off; off = align_up(off + 4 * (size_t)(n_nodes + 1), 256);
+        L.slotptr = off; off = align_up(off + 4 * (size_t)(n_nodes + 1), 256);
+        L.slot_edge = off; off = align_up(off + 4 * cap, 256);
+        L.group_recv = off; off = align_up(off + 4 * (cap / fast::kGroup), 256);
+        L.scratch_bytes = fk->fwd_scratch_bytes(n_nodes, n_edges);   // sized for more CTAs than there are ranges
+        L.scratch = off; off = align_up(off + L.scratch_bytes, 256);
+        L.total = off;
+        return L;
+    }
     L.conv_bytes = bwd ? e3j_conv_bwd_workspace_bytes(plan, n_nodes, n_edges)
                        : e3j_conv_fwd_workspace_bytes(plan, n_nodes, n_edges);
-    size_t off = 0;
     L.conv = off; off = align_up(off + L.conv_bytes, 256);
     L.s = off; off = align_up(off + 4 * (size_t)std::max<int64_t>(n_edges, 1) * C, 256);
     L.gs = off; if (bwd) off = align_up(off + 4 * (size_t)std::max<int64_t>(n_edges, 1) * C, 256);
@@ -153,6 +181,35 @@ int e3j_conv_radial_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, 
     const radial::RadialLayout L = radial::radial_layout(plan, n_nodes, n_edges, hidden, false);
     if (!workspace || ((uintptr_t)workspace & 255u) || workspace_bytes < L.total) return E3J_ERR_WORKSPACE;
     char* ws = (char*)workspace;
+    if (L.fused && n_edges > 0) {
+        // edge scalars formed inside the kernel: slot tables of the graph, then one sweep
+        if (!x || !out || !sh || !senders || !receivers) return E3J_ERR_INVALID_ARG;
+        if (((uintptr_t)x | (uintptr_t)out) & 15u) return E3J_ERR_INVALID_ARG;
+        cudaStream_t st = (cudaStream_t)stream;
+        if (!rowptr) {
+            int32_t* rp = (int32_t*)(ws + L.rowptr);
+            if (int rc = graph_prepare(n_nodes, n_edges, senders, receivers, rp, nullptr, nullptr, st)) return rc;
+            rowptr = rp;
+        }
+        int32_t* slotptr = (int32_t*)(ws + L.slotptr);
+        int32_t* slot_edge = (int32_t*)(ws + L.slot_edge);
+        int32_t* group_recv = (int32_t*)(ws + L.group_recv);
+        if (int rc = fast::build_slot_tables(n_nodes, n_edges, rowptr, slotptr, slot_edge, group_recv, st)) return rc;
+        DeviceTables t;
+        if (int rc = get_device_tables(plan, t)) return rc;
+        ConvArgs a{};
+        a.n_nodes = n_nodes; a.n_edges = n_edges; a.x = x; a.sh = sh; a.senders = senders; a.receivers = receivers;
+        a.rowptr = rowptr; a.out = out; a.stream = st; a.status = t.status;
+        RadialArgs r{};
+        r.h = h; r.W = W; r.hidden = hidden; r.slotptr = slotptr; r.slot_edge = slot_edge; r.group_recv = group_recv;
+        r.scratch = ws + L.scratch; r.scratch_bytes = L.scratch_bytes;
+        return radial::fused_forward(plan, hidden)->radial_fwd(a, r);
+    }
+    if (L.fused) {   // no edges: every receiver row is empty
+        if (!out) return E3J_ERR_INVALID_ARG;
+        E3J_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(float) * (size_t)n_nodes * plan->D * plan->nq, (cudaStream_t)stream));
+        return E3J_OK;
+    }
     float* s = (float*)(ws + L.s);
     if (n_edges > 0) {
         DeviceTables t;
