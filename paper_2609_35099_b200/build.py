@@ -25,7 +25,7 @@ BUILD = CSRC / "build"
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xptxas", "-v", "--expt-relaxed-constexpr",
-]
+] + os.environ.get("E3J_NVCC_EXTRA", "").split()   # e.g. -DE3J_RADIAL_PROF (role cycle counters of fast_radial.cuh)
 
 
 def sources() -> list[Path]:

@@ -65,3 +65,4 @@ int build_slot_tables(int64_t n_nodes, int64_t n_edges, const int32_t* rowptr, i
 
 }  // namespace fast
 }  // namespace e3j
+

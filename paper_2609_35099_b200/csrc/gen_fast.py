@@ -106,17 +106,20 @@ class Sig:
         return self.rp.get((row, k), [])
 
     # ---------------------------------------------------------------- forward
-    def fwd_layout(self):
-        FW = self.cfg["FW"]
+    def fwd_layout(self, FW=None):
+        """Row groups of the forward bodies.  FW given: the layout of the forward that forms its edge scalars in
+        the kernel (its own number of row groups, balanced by the estimate alone)."""
+        radial = FW is not None
+        FW = FW or self.cfg["FW"]
         costs = []
         for row in range(self.D):
             starts = sum((2 * self.paths[k]["l1"] + 1) * 1.0 + 0.5 for k in self.row_paths[row]
                          if row == self.paths[k]["out_off"])
             costs.append(len(self.row_pairs[row]) * 1.0 + starts + 0.3)
-        bounds = partition_rows(costs, FW, self.cfg.get("F_BIAS"))
+        bounds = partition_rows(costs, FW, None if radial else self.cfg.get("F_BIAS"))
         # Measured group sizes override the estimate: consumer warp 1 shares its scheduler with the table
         # producer warp (and warp 0 with the copy warp), so an even split leaves the other two waiting for it.
-        if self.cfg.get("F_ROWS"):
+        if self.cfg.get("F_ROWS") and not radial:
             bounds = [0]
             for r in self.cfg["F_ROWS"]:
                 bounds.append(bounds[-1] + r)
@@ -468,6 +471,82 @@ class Sig:
         o.append("    }")
         return o
 
+    def emit_radial(self):
+        """Bodies of the forward that forms its edge scalars in the kernel: RF row groups (one consumer warp each),
+        their own A-slot order, and the A entries of one edge computed from harmonics held in registers."""
+        RW = self.cfg["RF"]
+        bounds, a0, slots = self.fwd_layout(RW)
+        slot_of_pair = {pi: s for s, pi in enumerate(slots) if pi is not None}
+        rmax = max(bounds[g + 1] - bounds[g] for g in range(RW))
+        o = []
+        o.append(f"    // ---- forward with in-kernel edge scalars (fast_radial.cuh): {RW} row groups")
+        o.append(f"    static constexpr int R_FW = {RW}, R_RMAX = {rmax}, R_APAD = {len(slots)};")
+        o.append(f"    static constexpr int r_row0(int g) {{")
+        o.append("        switch (g) {")
+        for i, v in enumerate(bounds):
+            o.append(f"            case {i}: return {v};")
+        o.append(f"            default: return {bounds[-1]};")
+        o.append("        }\n    }")
+        o.append(f"    template <int G>")
+        o.append(f"    __device__ static __forceinline__ void rfwd_edge(Vec (&acc)[R_RMAX], "
+                 f"const Vec* __restrict__ xs, const Vec* __restrict__ ss, const float* __restrict__ As) {{")
+        o.append(f"        constexpr int NQV = NQ / V;")
+        for g in range(RW):
+            o.append(f"        if constexpr (G == {g}) {{")
+            rows = range(bounds[g], bounds[g + 1])
+            need_x = sorted({self.pairs[pi][1] for row in rows for pi in self.row_pairs[row]})
+            for i1 in need_x:
+                o.append(f"            const Vec x{i1} = xs[{i1} * NQV];")
+            loaded_a = set()
+            paths_here = []
+            for row in rows:
+                for k in self.row_paths[row]:
+                    if k not in paths_here:
+                        paths_here.append(k)
+            for k in paths_here:
+                prow = [r2 for r2 in rows if self.pairs_of(r2, k)]
+                o.append(f"            const Vec s{k} = ss[{k} * NQV];")
+                used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
+                for i1 in used:
+                    o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
+                for j in range(depth):
+                    for row in prow:
+                        if j >= len(self.pairs_of(row, k)):
+                            continue
+                        pi = self.pairs_of(row, k)[j]
+                        slot = slot_of_pair[pi]
+                        q, lane = slot // 4, "xyzw"[slot % 4]
+                        if q not in loaded_a:
+                            loaded_a.add(q)
+                            o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
+                        i1 = self.pairs[pi][1]
+                        o.append(f"            vfma(acc[{row - bounds[g]}], a{q}.{lane}, sx{k}_{i1});")
+            o.append("        }")
+        o.append("    }")
+        o.append(f"    template <int G, class VecT>")
+        o.append(f"    __device__ static __forceinline__ void rfwd_store(const VecT (&acc)[R_RMAX], VecT* __restrict__ dst, const int stride) {{")
+        for g in range(RW):
+            o.append(f"        if constexpr (G == {g}) {{")
+            for row in range(bounds[g], bounds[g + 1]):
+                o.append(f"            dst[{row - bounds[g]} * stride] = acc[{row - bounds[g]}];")
+            o.append("        }")
+        o.append("    }")
+        assert len(slots) % 4 == 0
+        o.append(f"    // A[slot] = sum over the slot's records of c * y[i2], four slots per store")
+        o.append(f"    __device__ static __forceinline__ void a_entries(const float (&y)[DSH], float4* __restrict__ dst) {{")
+        for q in range(len(slots) // 4):
+            terms = []
+            for s_i in range(4 * q, 4 * q + 4):
+                pi = slots[s_i]
+                if pi is None:
+                    terms.append("0.f")
+                else:
+                    terms.append(" + ".join(f"{fmt_float(v)} * y[{i2}]" for i2, v in self.pairs[pi][3]))
+            o.append(f"        dst[{q}] = make_float4({', '.join(terms)});")
+        o.append("    }")
+        return o
+
     def emit(self) -> str:
         V, NQ = self.V, self.NQ
         FW, FT, FS, FC = self.cfg["FW"], self.cfg["FT"], self.cfg["FS"], self.cfg["FC"]
@@ -641,21 +720,7 @@ class Sig:
             o.append("        }")
         o.append("    }")
         if self.cfg.get("RF", 0):
-            # forward A entries of one edge from harmonics held in registers (the convolution that forms its
-            # edge scalars from the radial layer computes them with one lane per edge)
-            assert len(slots) % 4 == 0
-            o.append(f"    // A[slot] = sum over the slot's records of c * y[i2], four slots per store")
-            o.append(f"    __device__ static __forceinline__ void a_entries(const float (&y)[DSH], float4* __restrict__ dst) {{")
-            for q in range(len(slots) // 4):
-                terms = []
-                for s_i in range(4 * q, 4 * q + 4):
-                    pi = slots[s_i]
-                    if pi is None:
-                        terms.append("0.f")
-                    else:
-                        terms.append(" + ".join(f"{fmt_float(v)} * y[{i2}]" for i2, v in self.pairs[pi][3]))
-                o.append(f"        dst[{q}] = make_float4({', '.join(terms)});")
-            o.append("    }")
+            o += self.emit_radial()
         o += bwd_lines
         o.append("};")
         o.append("}  // namespace")

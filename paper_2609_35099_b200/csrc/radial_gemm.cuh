@@ -56,14 +56,24 @@ __device__ __forceinline__ void convert_operand(unsigned char* hi, unsigned char
     constexpr int LANE_QUADS = 32 / LANE_ROWS;
     constexpr int ITEMS = (ROWS / LANE_ROWS) * (QUADS / LANE_QUADS);   // warp items of the operand
     static_assert(ROWS % LANE_ROWS == 0 && QUADS % LANE_QUADS == 0, "operand does not tile");
-#pragma unroll 2
-    for (int item = cwarp; item < ITEMS; item += 4) {
+    static_assert(ITEMS % 4 == 0, "four converter warps share the items");
+    constexpr int NI = ITEMS / 4;
+    float4 v[NI];
+    // every load of the operand is issued before the first conversion, so that they are in flight together
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        const int item = cwarp + 4 * i;
+        const int rg = item / (QUADS / LANE_QUADS), qg = item % (QUADS / LANE_QUADS);
+        v[i] = load(rg * LANE_ROWS + lane % LANE_ROWS, (qg * LANE_QUADS + lane / LANE_ROWS) * 4);
+    }
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        const int item = cwarp + 4 * i;
         const int rg = item / (QUADS / LANE_QUADS), qg = item % (QUADS / LANE_QUADS);
         const int row = rg * LANE_ROWS + lane % LANE_ROWS;
         const int quad = qg * LANE_QUADS + lane / LANE_ROWS;
-        const float4 v = load(row, quad * 4);
         float4 h, l;
-        umma::split_tf32(v, h, l);
+        umma::split_tf32(v[i], h, l);
         const uint32_t off = umma::tile_offset(row, quad * 4, kChunkK);
         *reinterpret_cast<float4*>(hi + off) = h;
         *reinterpret_cast<float4*>(lo + off) = l;
