@@ -260,6 +260,10 @@ def main():
                     help="append this fraction of padding edges and call the padded entry points (rates count real edges)")
     ap.add_argument("--double-backward", action="store_true",
                     help="also time e3j_conv_bwd_bwd (after the steps, reported beside them; plain lists only)")
+    ap.add_argument("--fused-radial", action="store_true",
+                    help="also time the convolution that takes the radial network's last layer (h, W) instead of the "
+                         "weights (after the steps, reported beside them)")
+    ap.add_argument("--hidden", type=int, default=64, help="width of the radial network's last hidden layer")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -401,6 +405,68 @@ def main():
                        "more = composition of forward and backward passes"}
         del ws_d, cts, gg
 
+    # ---- the same convolution with the edge weights given as the radial network's last layer (h, W) instead of w:
+    # the forward that forms them inside the kernel, beside the unfused form (tensor-core product into memory, then
+    # the plain forward), and the backward (composed: product, convolution backward, two more products)
+    radial = None
+    if args.fused_radial and not args.pad and not args.collapse and not args.generic:
+        H = args.hidden
+        gen = torch.Generator(device=dev); gen.manual_seed(12)
+        hh = torch.randn((e, H), generator=gen, device=dev)
+        WW = torch.randn((H, plan.n_paths * plan.n_channels), generator=gen, device=dev) / (H ** 0.5)
+        ws_rf = torch.empty(max(e3j.e3j_conv_radial_fwd_workspace_bytes(plan, n, e, H), 256), dtype=torch.uint8, device=dev)
+        ws_rb = torch.empty(max(e3j.e3j_conv_radial_bwd_workspace_bytes(plan, n, e, H), 256), dtype=torch.uint8, device=dev)
+        w_mat = torch.empty((e, plan.n_paths, plan.n_channels), device=dev)
+        gh, gW = torch.empty_like(hh), torch.empty_like(WW)
+
+        def timed(fn, k):
+            for _ in range(3):
+                fn()
+            l0 = e3j.e3j_launch_count()
+            a, b = ev(), ev()
+            torch.cuda.synchronize()
+            a.record(stream)
+            for _ in range(k):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / k, (e3j.e3j_launch_count() - l0) // k
+
+        k_r = max(3, min(args.steps, 50))
+        rf_ms, rf_launches = timed(lambda: e3j.e3j_conv_radial_fwd(plan, d["x"], d["y"], hh, WW, d["snd"], d["rcv"], rowptr,
+                                                                    out=out, workspace=ws_rf), k_r)
+        gemm_ms, _ = timed(lambda: e3j.e3j_radial_weights(plan, hh, WW, out=w_mat), k_r)
+        plain_ms, _ = timed(lambda: conv_fwd(plan, d["x"], d["y"], w_mat, d["snd"], d["rcv"], rowptr, out=out, workspace=ws_f), k_r)
+        rb_ms, rb_launches = timed(lambda: e3j.e3j_conv_radial_bwd(plan, d["x"], d["y"], hh, WW, d["snd"], d["rcv"], d["g"], rowptr,
+                                                                    perm, colptr, grad_x=gx, grad_sh=gy, grad_h=gh, grad_W=gW,
+                                                                    workspace=ws_rb), max(3, k_r // 3))
+        nq_, P_, D_ = plan.n_channels, plan.n_paths, plan.d_out
+        bytes_fwd = 4 * (n * plan.d_in * nq_ + e * plan.d_sh + e * H + H * P_ * nq_ + 2 * e + n * D_ * nq_)
+        fma_conv = e * (plan.n_pairs + sum(2 * p["l1"] + 1 for p in e3j.e3j_plan_paths(plan))) * nq_   # FP32 issue slots x 32 lanes
+        flop_tensor = 3 * 2.0 * e * H * P_ * nq_                                                      # three TF32 products
+        peak_hbm, _src = measured_peak()
+        try:
+            with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+                bf16_peak = float(json.load(f)["bf16_tflops"])
+        except Exception:
+            bf16_peak = 1590.0
+        fp32_peak = 148 * 128 * 1.965e9   # FMA lanes x max SM clock (nominal unit counts)
+        radial = {
+            "hidden": H, "fused_fwd_ms": rf_ms, "fused_fwd_launches": rf_launches,
+            "unfused_fwd_ms": gemm_ms + plain_ms, "unfused_parts_ms": {"radial_weights": gemm_ms, "conv_fwd": plain_ms},
+            "bwd_ms": rb_ms, "bwd_launches": rb_launches, "bwd_form": "composed (weights and their cotangent materialised)",
+            "fwd_edges_per_s": e / (rf_ms * 1e-3),
+            "roofline_fwd": {
+                "minimal_bytes": bytes_fwd, "hbm_GBs": bytes_fwd / (rf_ms * 1e-3) / 1e9,
+                "hbm_frac_of_measured": bytes_fwd / (rf_ms * 1e-3) / 1e9 / peak_hbm,
+                "bound": "alu", "fp32_fma_per_s": fma_conv / (rf_ms * 1e-3), "fp32_peak_fma_per_s": fp32_peak,
+                "fp32_issue_frac": fma_conv / (rf_ms * 1e-3) / fp32_peak,
+                "tensor_tf32_TFLOPs": flop_tensor / (rf_ms * 1e-3) / 1e12,
+                "tensor_frac_of_tf32_peak": flop_tensor / (rf_ms * 1e-3) / 1e12 / (0.5 * bf16_peak),
+                "tensor_peak_note": "TF32 peak taken as half the measured bf16 peak (nominal ratio)"},
+        }
+        del ws_rf, ws_rb, w_mat, hh, WW, gh, gW
+
     # ---- end to end: pinned host buffers in, results out, inside the timed region.  Every step copies its inputs
     # from pinned host memory and its four results back; the copies run on streams of their own with two sets
     # of device buffers, so that the transfers of neighbouring steps overlap each other and the kernels.
@@ -503,7 +569,7 @@ def main():
             # 20 % of the runs, as in its efficiency-comparison section), minimum and maximum
             "call_stats_ms": {"fwd": call_stats(fwd_ms), "bwd": call_stats(bwd_ms)},
             "outside_the_step_ms": {"plan_build_host": plan_build_ms, "graph_prepare_device": graph_prepare_ms},
-            "double_backward": dbl,
+            "double_backward": dbl, "radial": radial,
             "roofline": dominant, "roofline_fwd": roofs["fwd"], "roofline_bwd": roofs["bwd"],
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         }

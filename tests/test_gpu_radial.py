@@ -145,3 +145,92 @@ def test_conv_radial_empty_graph_and_bad_arguments():
     with pytest.raises(e3j.E3JError) as err:
         e3j.e3j_radial_weights(plan, torch.zeros((3, 6), device=DEV), W6)
     assert err.value.status == e3j.E3J_ERR_UNSUPPORTED
+
+
+def _seeded_normal(shape, seed):
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(seed)
+    return torch.randn(shape, generator=gen, device=DEV, dtype=torch.float32)
+
+
+def _range_boundary_receivers(rowptr, n_ranges):
+    """Receivers whose slot groups are cut by a CTA range boundary of the forward that forms its edge scalars in
+    the kernel (host restatement of its split: 8 slots per group, tiles of 16 groups, equal tile counts)."""
+    deg = np.diff(rowptr)
+    groups = (deg + 7) // 8
+    first_group = np.concatenate([[0], np.cumsum(groups)])
+    n_groups = int(first_group[-1])
+    tiles_total = (n_groups + 15) // 16
+    tiles_per = (tiles_total + n_ranges - 1) // n_ranges
+    cuts = [16 * tiles_per * r for r in range(1, n_ranges) if 16 * tiles_per * r < n_groups]
+    rec = np.searchsorted(first_group, cuts, side="right") - 1
+    return np.unique(np.concatenate([rec, np.maximum(rec - 1, 0)]))
+
+
+def test_conv_radial_config5_full_size_sampled():
+    """100k atoms, 4.77 M edges: the weights (31 GB as an array) exist only inside the forward kernel.  Sampled
+    receivers, every receiver cut by a CTA range boundary included, are recomputed by the oracle; the backward is
+    checked on the sampled receivers' edges (grad_sh, grad_h), on sampled senders (grad_x) and, for grad_W and the
+    whole of grad_h, by the adjoint identities <grad_W, W> = <grad_h, h> = <grad_out, out>."""
+    c = workloads.CONFIGS[5]
+    wl = workloads.make_graph(5)
+    n, e, H = wl.n_nodes, wl.n_edges, 64
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], None, c["out_lmax"])
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], None, c["out_lmax"])
+    rng = np.random.Generator(np.random.PCG64([5, 3]))
+    x = rng.standard_normal((n, plan.d_in, plan.n_channels), dtype=np.float32)
+    y = workloads.edge_harmonics(wl)
+    W = (rng.standard_normal((H, plan.n_paths * plan.n_channels), dtype=np.float32) / np.float32(8.0))
+    dx_, dy_, dW_ = _cuda(x), _cuda(y), _cuda(W)
+    dh_ = _seeded_normal((e, H), 53)
+    dg_ = _seeded_normal((n, plan.d_out, plan.n_channels), 54)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    rowptr, perm, colptr = e3j.e3j_graph_prepare(n, snd, rcv)
+    out = e3j.e3j_conv_radial_fwd(plan, dx_, dy_, dh_, dW_, snd, rcv, rowptr)
+    out2 = e3j.e3j_conv_radial_fwd(plan, dx_, dy_, dh_, dW_, snd, rcv, rowptr)
+    torch.cuda.synchronize()
+    assert e3j.e3j_plan_device_status(plan) == 0
+    assert torch.equal(out, out2), "forward differs between two runs"
+    del out2
+    gx, gy, gh, gW = e3j.e3j_conv_radial_bwd(plan, dx_, dy_, dh_, dW_, snd, rcv, dg_, rowptr, perm, colptr)
+    torch.cuda.synchronize()
+    assert e3j.e3j_plan_device_status(plan) == 0
+
+    rp = rowptr.cpu().numpy()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    deg = np.diff(rp)
+    pick = np.unique(np.concatenate([rng.choice(n, 30, replace=False), np.argsort(deg)[-4:], np.argsort(deg)[:4], [0, n - 1],
+                                     _range_boundary_receivers(rp, max(1, sms // 8))]))
+    out_blocks = blocks_of_paths(cp.paths, "out")
+    for b in pick:
+        e0, e1 = int(rp[b]), int(rp[b + 1])
+        nodes, local = np.unique(np.concatenate([wl.senders[e0:e1], [b]]), return_inverse=True)
+        lb = int(local[-1])
+        hs = dh_[e0:e1].cpu().numpy()
+        l_snd, l_rcv = local[:-1].astype(np.int32), np.full(e1 - e0, lb, np.int32)
+        ref = oconv.conv_radial_fwd(cp, x[nodes], y[e0:e1], hs, W, l_snd, l_rcv)
+        assert_blockwise_close(out[b].cpu().numpy()[None], ref[lb][None], out_blocks, what=f"out[{b}]")
+        gs = np.zeros((len(nodes), plan.d_out, plan.n_channels), np.float32)
+        gs[lb] = dg_[b].cpu().numpy()
+        _, ry, rh, _ = oconv.conv_radial_bwd(cp, x[nodes], y[e0:e1], hs, W, l_snd, l_rcv, gs)
+        if e1 > e0:
+            assert_blockwise_close(gy[e0:e1].cpu().numpy(), ry, blocks_of_paths(cp.paths, "sh"), what=f"grad_sh[{b}]")
+            assert_blockwise_close(gh[e0:e1].cpu().numpy(), rh, [(0, H)], what=f"grad_h[{b}]")
+    senders_sorted, cptr = perm.cpu().numpy(), colptr.cpu().numpy()
+    for a in rng.choice(n, 12, replace=False):
+        ids = np.sort(senders_sorted[cptr[a]:cptr[a + 1]])
+        nodes, l_rcv = np.unique(wl.receivers[ids], return_inverse=True)
+        xs = np.zeros((len(nodes) + 1, plan.d_in, plan.n_channels), np.float32)
+        xs[-1] = x[a]
+        gs = np.concatenate([dg_[torch.from_numpy(nodes).to(DEV)].cpu().numpy(),
+                             np.zeros((1, plan.d_out, plan.n_channels), np.float32)])
+        hs = dh_[torch.from_numpy(ids).to(DEV)].cpu().numpy()
+        rx, _, _, _ = oconv.conv_radial_bwd(cp, xs, y[ids], hs, W, np.full(len(ids), len(nodes), np.int32),
+                                            l_rcv.astype(np.int32), gs)
+        assert_blockwise_close(gx[a].cpu().numpy()[None], rx[-1][None], blocks_of_paths(cp.paths, "x"), what=f"grad_x[{a}]")
+    # the map is linear in W and in h: <grad_W, W> = <grad_h, h> = <grad_out, out>, sums in float64
+    ref = float((dg_.double() * out.double()).sum().item())
+    via_W = float((gW.double() * dW_.double()).sum().item())
+    via_h = float((gh.double() * dh_.double()).sum().item())
+    scale = float((dg_.double() * out.double()).abs().sum().item())
+    assert abs(via_W - ref) <= 1e-6 * scale and abs(via_h - ref) <= 1e-6 * scale, (ref, via_W, via_h, scale)
