@@ -52,6 +52,15 @@ NCU_TRAFFIC = {
     ("water3000", "fwd"): 1.109031e9 + 0.083995e9 + 0.016343e9,          # fast_fwd_kernel + fwd_fixup_kernel
     ("water3000", "bwd"): 1.257002e9 + 1.362881e9 + 0.330463e9 + 0.0018e9,  # fast_bwd1_kernel + bwd_dx_reduce_kernel
 }
+# Where each term above is printed (file under profiles/, kernel, metric): tests/test_bench_traffic.py checks them.
+NCU_TRAFFIC_SOURCE = {
+    ("water3000", "fwd"): [("fast_fwd_kernel_water3000.txt", "fast_fwd_kernel", "dram__bytes_read.sum", 1.109031e9),
+                           ("fast_fwd_kernel_water3000.txt", "fast_fwd_kernel", "dram__bytes_write.sum", 0.083995e9),
+                           ("small_kernels_traffic_water3000.txt", "fwd_fixup_kernel", "total", 0.016343e9)],
+    ("water3000", "bwd"): [("fast_bwd1_kernel_water3000.txt", "fast_bwd1_kernel", "dram__bytes_read.sum", 1.257002e9),
+                           ("fast_bwd1_kernel_water3000.txt", "fast_bwd1_kernel", "dram__bytes_write.sum", 1.362881e9),
+                           ("small_kernels_traffic_water3000.txt", "bwd_dx_reduce_kernel", "total", 0.330463e9 + 0.0018e9)],
+}
 
 
 def algorithmic_bytes(n, e, d, dp, P, D, nq):
@@ -258,8 +267,11 @@ def main():
                     help="plan with collapsed output multiplicities (table-driven kernels; no CPU leg)")
     ap.add_argument("--pad", type=float, default=0.0,
                     help="append this fraction of padding edges and call the padded entry points (rates count real edges)")
-    ap.add_argument("--double-backward", action="store_true",
-                    help="also time e3j_conv_bwd_bwd (after the steps, reported beside them; plain lists only)")
+    ap.add_argument("--double-backward", action="store_true", help="(default for configs 2 and 3; kept for old command lines)")
+    ap.add_argument("--no-double-backward", action="store_true",
+                    help="skip the timing of e3j_conv_bwd_bwd (after the steps, reported beside them; plain lists only)")
+    ap.add_argument("--sustained-s", type=float, default=2.0,
+                    help="length of the extra back-to-back loop whose means and clocks go into `sustained` (0 = skip)")
     ap.add_argument("--fused-radial", action="store_true",
                     help="also time the convolution that takes the radial network's last layer (h, W) instead of the "
                          "weights (after the steps, reported beside them)")
@@ -376,9 +388,31 @@ def main():
         total_ms = float(tm.item())
     ms_per_step = total_ms / args.steps
 
+    # ---- the same step back to back for at least two seconds: the forward is bound by instruction issue and follows
+    # the SM clock, which the power cap lowers in long runs, so the clock dependence goes on the record whatever
+    # --steps is
+    sustained = None
+    if args.sustained_s > 0 and world == 1:
+        k_s = max(args.steps, int(args.sustained_s * 1e3 / max(ms_per_step, 1e-3)) + 1)
+        marks_s = [(ev(), ev(), ev()) for _ in range(k_s)]
+        samp = ClockSampler(local_rank)
+        torch.cuda.synchronize()
+        for a, b, cc in marks_s:
+            a.record(stream); fwd(d); b.record(stream); bwd(d); cc.record(stream)
+        torch.cuda.synchronize()
+        clk = samp.stop()
+        f_s = statistics.mean(a.elapsed_time(b) for a, b, _ in marks_s)
+        b_s = statistics.mean(b.elapsed_time(cc) for _, b, cc in marks_s)
+        mhz, mx = clk.get("sm_mhz"), clk.get("sm_max_mhz")
+        sustained = {"steps": k_s, "seconds": marks_s[0][0].elapsed_time(marks_s[-1][2]) * 1e-3, "fwd_ms": f_s, "bwd_ms": b_s,
+                     "clocks": clk,
+                     "fwd_ms_at_max_clock": f_s * mhz / mx if mhz and mx else None,
+                     "bwd_ms_at_max_clock": b_s * mhz / mx if mhz and mx else None}
+        del marks_s
+
     # ---- the double backward of the same workload (not part of the step)
     dbl = None
-    if args.double_backward and not args.pad:
+    if not args.no_double_backward and not args.pad and not args.generic and not args.collapse and args.config in (2, 3):
         gen = torch.Generator(device=dev); gen.manual_seed(11)
         cts = [torch.randn(d[k].shape, generator=gen, device=dev) for k in ("x", "y", "w")]
         ws_d = torch.empty(max(e3j.e3j_conv_bwd_bwd_workspace_bytes(plan, n, e), 256), dtype=torch.uint8, device=dev)
@@ -543,9 +577,11 @@ def main():
             r = {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s",
                  "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "peak_source": peak_src,
                  "algorithmic_bytes_per_launch": nbytes, "avg_ms": ms, "traffic": traffic}
-            if traffic:   # what the memory system actually moved (ncu), at the measured duration
+            if traffic:   # what the memory system moved in the committed ncu capture, at this run's duration
                 r["traffic_GBs"] = traffic / (ms * 1e-3) / 1e9
                 r["traffic_frac_of_peak"] = r["traffic_GBs"] / peak
+                r["traffic_source"] = ("committed ncu captures (not measured in this run): " +
+                                       ", ".join(sorted({"profiles/" + f for f, _, _, _ in NCU_TRAFFIC_SOURCE[(wl.name, key)]})))
             return r
 
         spec = bool(plan.specialised)
@@ -569,7 +605,7 @@ def main():
             # 20 % of the runs, as in its efficiency-comparison section), minimum and maximum
             "call_stats_ms": {"fwd": call_stats(fwd_ms), "bwd": call_stats(bwd_ms)},
             "outside_the_step_ms": {"plan_build_host": plan_build_ms, "graph_prepare_device": graph_prepare_ms},
-            "double_backward": dbl, "radial": radial,
+            "double_backward": dbl, "radial": radial, "sustained": sustained,
             "roofline": dominant, "roofline_fwd": roofs["fwd"], "roofline_bwd": roofs["bwd"],
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         }

@@ -183,12 +183,15 @@ int e3j_conv_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const f
  *   - All calls on a device share the one array, which keeps the previous call's contents.
  *     Nothing in it has to be zero at entry (the kernel writes every word before reading it), but
  *     two calls that overlap on the GPU (different streams) race on it: serialise them.
- *   - Results are the same as e3j_conv_fwd's.  Bounded-wait failures are not reported through
- *     e3j_plan_device_status here.
+ *   - Results are the same as e3j_conv_fwd's.  A bounded wait that gives up inside the kernel is not
+ *     reported through e3j_plan_device_status (that word lives in allocated memory) but through a
+ *     status word that is static like the scratch: e3j_noalloc_status reads it into the HOST word
+ *     *status and clears it (0 = fine; synchronises the device; allocates nothing).
  * Arguments as for e3j_conv_fwd (receivers non-decreasing; rowptr is not needed). */
 int e3j_conv_fwd_noalloc(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
                          const float* sh, const float* w, const int32_t* senders,
                          const int32_t* receivers, float* out, void* stream);
+int e3j_noalloc_status(int32_t* status);
 
 /* Convolution backward.  grad_out [n_nodes,D,N_q]; grad_x [n_nodes,d,N_q],
  * grad_sh [n_edges,d'], grad_w [n_edges,P,N_q]; any of the three may be NULL (not
@@ -299,6 +302,14 @@ int e3j_tp_fwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
 int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float* x2,
                const float* w, const float* grad_out, float* grad_x1, float* grad_x2,
                float* grad_w, void* stream);
+
+/* Self-test of the kernels' bounded waits (no counterpart in the paper).  Every wait inside the specialised
+ * kernels gives up after a fixed number of polls, records the failure in the plan's device status word and
+ * lets the kernel drain instead of hanging the GPU.  This call exercises that path on purpose, without any
+ * risk of a hang: one warp waits, for at most spin_limit polls (1 .. 2^20), on a barrier that nothing will
+ * complete.  On return *returned is what the wait returned (0 = gave up), *abort_flag the kernel's abort flag
+ * (1), both HOST words, and e3j_plan_device_status(plan) reads 1 once and 0 afterwards.  Synchronises. */
+int e3j_selftest_bounded_wait(const e3j_plan* plan, uint32_t spin_limit, int32_t* returned, int32_t* abort_flag);
 
 const char* e3j_status_string(int status);
 int e3j_last_cuda_error(void);

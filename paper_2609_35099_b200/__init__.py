@@ -20,12 +20,12 @@ from pathlib import Path
 __all__ = [
     "E3JError", "Plan", "library_path", "e3j_plan_create", "e3j_plan_destroy", "e3j_plan_info",
     "e3j_plan_paths", "e3j_plan_records", "e3j_plan_signature", "e3j_plan_device_status", "e3j_graph_prepare", "e3j_graph_validate",
-    "e3j_conv_fwd_workspace_bytes", "e3j_conv_bwd_workspace_bytes", "e3j_conv_fwd", "e3j_conv_fwd_noalloc",
+    "e3j_conv_fwd_workspace_bytes", "e3j_conv_bwd_workspace_bytes", "e3j_conv_fwd", "e3j_conv_fwd_noalloc", "e3j_noalloc_status",
     "e3j_conv_bwd", "e3j_graph_prepare_padded", "e3j_conv_fwd_padded", "e3j_conv_bwd_padded",
     "e3j_conv_bwd_bwd_workspace_bytes", "e3j_conv_bwd_bwd",
     "e3j_radial_weights", "e3j_conv_radial_fwd_workspace_bytes", "e3j_conv_radial_bwd_workspace_bytes",
     "e3j_conv_radial_fwd", "e3j_conv_radial_bwd",
-    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_status_string", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
+    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
     "E3J_PLAN_COLLAPSE_OUTPUTS",
 ]
 
@@ -98,6 +98,8 @@ def _load():
     lib.e3j_conv_bwd_padded.argtypes = [vp, i64, i64] + [vp] * 13 + [sz, vp]
     lib.e3j_conv_fwd_noalloc.argtypes = [vp, i64, i64] + [vp] * 7
     lib.e3j_conv_fwd_noalloc.restype = i32
+    lib.e3j_noalloc_status.argtypes = [ctypes.POINTER(ctypes.c_int32)]
+    lib.e3j_noalloc_status.restype = i32
     lib.e3j_radial_weights.argtypes = [vp, i64, i32] + [vp] * 4
     lib.e3j_radial_weights.restype = i32
     lib.e3j_conv_radial_fwd_workspace_bytes.argtypes = [vp, i64, i64, i32]
@@ -110,6 +112,8 @@ def _load():
     lib.e3j_conv_radial_bwd.restype = i32
     lib.e3j_tp_fwd.argtypes = [vp, i64] + [vp] * 5
     lib.e3j_tp_bwd.argtypes = [vp, i64] + [vp] * 8
+    lib.e3j_selftest_bounded_wait.argtypes = [vp, u32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+    lib.e3j_selftest_bounded_wait.restype = i32
     lib.e3j_status_string.argtypes = [i32]
     lib.e3j_status_string.restype = ctypes.c_char_p
     lib.e3j_last_cuda_error.restype = i32
@@ -317,6 +321,14 @@ def e3j_conv_fwd_noalloc(plan: Plan, x, sh, w, senders, receivers, out, stream=N
     return out
 
 
+def e3j_noalloc_status() -> int:
+    """Status word of the allocation-free entry point on the current device (0 = fine; non-zero: a bounded wait
+    inside its kernel gave up and the output of that call is invalid).  Reads and clears; synchronises."""
+    st = ctypes.c_int32(0)
+    _check(_load().e3j_noalloc_status(ctypes.byref(st)), "e3j_noalloc_status")
+    return int(st.value)
+
+
 def e3j_conv_bwd(plan: Plan, x, sh, w, senders, receivers, grad_out, rowptr=None, sender_perm=None,
                  colptr=None, grad_x=True, grad_sh=True, grad_w=True, workspace=None, stream=None,
                  _entry: str = "e3j_conv_bwd"):
@@ -505,6 +517,14 @@ def e3j_tp_bwd(plan: Plan, x1, x2, w, grad_out, grad_x1=True, grad_x2=True, grad
         _dev_ptr(grad_x1, f32, None, "grad_x1"), _dev_ptr(grad_x2, f32, None, "grad_x2"),
         _dev_ptr(grad_w, f32, None, "grad_w"), _stream(stream)), "e3j_tp_bwd")
     return grad_x1, grad_x2, grad_w
+
+
+def e3j_selftest_bounded_wait(plan: Plan, spin_limit: int = 1000):
+    """(returned, abort_flag) of a wait that is made to run out after spin_limit polls; sets the plan's status word."""
+    a, b = ctypes.c_int32(-1), ctypes.c_int32(-1)
+    _check(_load().e3j_selftest_bounded_wait(plan.handle, spin_limit, ctypes.byref(a), ctypes.byref(b)),
+           "e3j_selftest_bounded_wait")
+    return int(a.value), int(b.value)
 
 
 def e3j_status_string(status: int) -> str:

@@ -6,6 +6,7 @@
 
 #include "common.cuh"
 #include "fast_registry.hpp"
+#include "fast/fast_common.cuh"
 #include "generic_kernels.cuh"
 
 namespace e3j {
@@ -104,7 +105,7 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
 namespace {
 
 inline int grid_for(int64_t n) {
-    int64_t g = std::min<int64_t>(std::max<int64_t>(n, 1), 148 * 32);
+    int64_t g = std::min<int64_t>(std::max<int64_t>(n, 1), (int64_t)sm_count() * 32);
     return (int)g;
 }
 
@@ -147,7 +148,7 @@ __global__ void add_into_kernel(int64_t n, float* __restrict__ dst, const float*
 int add_into(float* dst, const float* src, size_t n, cudaStream_t st) {
     if (n == 0) return E3J_OK;
     const int vec_ok = (((uintptr_t)dst | (uintptr_t)src) & 15u) == 0;
-    add_into_kernel<<<148 * 16, 256, 0, st>>>((int64_t)n, dst, src, vec_ok);
+    add_into_kernel<<<sm_count() * 16, 256, 0, st>>>((int64_t)n, dst, src, vec_ok);
     return after_launch();
 }
 
@@ -594,6 +595,21 @@ int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
                                                                            nullptr, grad_out, grad_x1);
         if (int s = after_launch()) return s;
     }
+    return E3J_OK;
+}
+
+int e3j_selftest_bounded_wait(const e3j_plan* plan, uint32_t spin_limit, int32_t* returned, int32_t* abort_flag) {
+    if (!plan || !returned || !abort_flag || spin_limit == 0 || spin_limit > (1u << 20)) return E3J_ERR_INVALID_ARG;
+    DeviceTables t;
+    if (int s = get_device_tables(plan, t)) return s;
+    // two result words behind the status word, in the plan's own device allocation (its last 256-byte section)
+    int32_t* result = t.status + 8;
+    fast::bounded_wait_selftest_kernel<<<1, 32>>>(spin_limit, t.status, result);
+    if (int s = after_launch()) return s;
+    E3J_CUDA_TRY(cudaDeviceSynchronize());
+    int32_t host[2] = {0, 0};
+    E3J_CUDA_TRY(cudaMemcpy(host, result, sizeof(host), cudaMemcpyDeviceToHost));
+    *returned = host[0]; *abort_flag = host[1];
     return E3J_OK;
 }
 

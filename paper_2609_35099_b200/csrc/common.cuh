@@ -54,6 +54,22 @@ struct ConvArgs {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// SM count of the current device (cached per thread; grids are sized in multiples of it), capped at kMaxSms,
+// the bound that scratch sizes are computed with.  148 (B200) if the device cannot be queried.
+constexpr int kMaxSms = 192;
+inline int sm_count() {
+    static thread_local int cached_dev = -1, cached = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (dev != cached_dev) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached = n > kMaxSms ? kMaxSms : n;
+        cached_dev = dev;
+    }
+    return cached;
+}
+
 // The bodies of e3j_conv_fwd / e3j_conv_bwd (and their padded forms), for entry points that compose them.
 int conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x, const float* sh,
                   const float* w, const int32_t* senders, const int32_t* receivers, const int32_t* rowptr,

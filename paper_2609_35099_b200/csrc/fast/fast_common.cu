@@ -21,6 +21,19 @@ __global__ void fwd_fixup_kernel(int n_cta, int row_f4, const float4* __restrict
     }
 }
 
+// One warp, one barrier with one expected arrival that never comes, no copy in flight: the wait runs out after
+// `limit` polls, records the time-out in *status and returns false; result[0] = what the wait returned,
+// result[1] = the CTA's abort flag afterwards.  Nothing here can hang: the loop is bounded by `limit`.
+__global__ void bounded_wait_selftest_kernel(uint32_t limit, int32_t* status, int32_t* result) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) { mbar_init(&bar, 1); abort_flag = 0; mbar_fence_init(); }
+    __syncthreads();
+    const bool ok = mbar_wait_limit(&bar, 0, &abort_flag, status, limit);
+    __syncthreads();
+    if (threadIdx.x == 0) { result[0] = ok ? 1 : 0; result[1] = abort_flag; }
+}
+
 __global__ void bwd_zero_padding_kernel(const int32_t* __restrict__ n_real, int64_t n_edges, int w_row_f4,
                                         int sh_row, float4* __restrict__ grad_w, float* __restrict__ grad_sh) {
     const int64_t first = min((int64_t)*n_real, n_edges);

@@ -90,16 +90,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false (and records the failure) if the phase never completes.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+// Bounded wait.  Returns false (and records the failure) if the phase does not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                const uint32_t limit) {
 #pragma unroll 1  // an unrolled spin loop only bloats the kernel text
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }
     *abort_flag = 1;
     if (status) atomicExch(status, kStatusTimeout);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    return mbar_wait_limit(bar, parity, abort_flag, status, kSpinLimit);
 }
 // Contiguous global -> shared copy; both addresses 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
@@ -151,6 +155,9 @@ __device__ __forceinline__ void cta_edge_range(const int64_t n_edges_host, const
 // Backward of a padded call: zero rows of grad_w and grad_sh for the padding edges [*n_real, n_edges).
 __global__ void bwd_zero_padding_kernel(const int32_t* __restrict__ n_real, int64_t n_edges, int w_row_f4,
                                         int sh_row, float4* __restrict__ grad_w, float* __restrict__ grad_sh);
+
+// Self-test of the bounded wait (e3j_selftest_bounded_wait): one warp waits on a barrier that nobody arrives on.
+__global__ void bounded_wait_selftest_kernel(uint32_t limit, int32_t* status, int32_t* result);
 
 // Backward pass 2: grad_x[a] = sum of the per-edge shares of the edges sent by a, in edge order.
 __global__ void bwd_dx_reduce_kernel(int64_t n_nodes, int row_f4, const float4* __restrict__ dx_edge,

@@ -10,21 +10,9 @@
 namespace e3j {
 namespace fast {
 
-constexpr int kMaxSms = 192;       // upper bound on the SM count, for scratch sizing
+using e3j::kMaxSms;   // upper bound on the SM count, for scratch sizing
+using e3j::sm_count;
 constexpr size_t kPartRecvBytes = 8192;  // slot of the [n_cta][2] boundary receiver ids
-
-inline int sm_count() {
-    static thread_local int cached_dev = -1, cached = 0;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (dev != cached_dev) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-        cached = n > kMaxSms ? kMaxSms : n;
-        cached_dev = dev;
-    }
-    return cached;
-}
 
 // scratch: [part_recv: 2*n_cta ints in an 8 KB slot][partial rows: 2*n_cta*D*NQ floats],
 // n_cta = (SMs of the current device) * S::FC
@@ -166,7 +154,7 @@ int launch_bwd(const ConvArgs& a) {
     }
     if (int s = after_launch()) return s;
     if (a.n_real) {
-        bwd_zero_padding_kernel<<<148 * 8, 256, 0, a.stream>>>(a.n_real, a.n_edges, S::P * S::NQ / 4, S::DSH,
+        bwd_zero_padding_kernel<<<sm_count() * 8, 256, 0, a.stream>>>(a.n_real, a.n_edges, S::P * S::NQ / 4, S::DSH,
                                                               reinterpret_cast<float4*>(a.grad_w), a.grad_sh);
         if (int s = after_launch()) return s;
     }

@@ -154,7 +154,7 @@ __global__ void validate_kernel(int64_t n_nodes, int64_t n_edges, const int32_t*
 inline int blocks_for(int64_t n, int threads) {
     int64_t b = (n + threads - 1) / threads;
     if (b < 1) b = 1;
-    if (b > 148 * 16) b = 148 * 16;
+    if (b > sm_count() * 16) b = sm_count() * 16;
     return (int)b;
 }
 

@@ -364,8 +364,32 @@ def test_double_backward(config, n_atoms, natural, flags):
     """Cotangents of the backward's inputs against the oracle; a missing cotangent is zero; outputs that are
     not wanted are skipped; two runs give the same bits.  (Configs 2 and 3 have fused kernels, config 1 and the
     generic plans take the composition.)"""
-    wl, plan, cp, x, y, w, g = make_case(config, n_atoms, flags=flags,
-                                         **({"irreps_out": workloads.NATURAL_PARITY_OUT} if natural else {}))
+    _check_double_backward(*make_case(config, n_atoms, flags=flags,
+                                      **({"irreps_out": workloads.NATURAL_PARITY_OUT} if natural else {})))
+
+
+@pytest.mark.parametrize("irreps,lmax,n_atoms", [
+    ("128x0e+128x1o", 2, 300),             # l <= 2
+    ("256x0e+256x1o", 3, 192),             # 256 channels: two warps per edge
+    ("64x0e+64x1o", 3, 300),
+    ("128x0e", 3, 300),                    # scalar inputs
+    ("128x0e+128x1o+128x2e", 3, 192),      # the tensor-product signature as a graph call
+])
+def test_double_backward_of_the_other_generated_signatures(irreps, lmax, n_atoms):
+    """Every generated signature except the collapsed one has the fused double-backward kernels."""
+    import dataclasses
+    wl = dataclasses.replace(workloads.make_graph(2, n_atoms), irreps_in=irreps, sh_lmax=lmax, out_lmax=lmax)
+    plan = e3j.e3j_plan_create(irreps, lmax, None, lmax)
+    assert plan.specialised
+    cp = oconv.Coupling(irreps, lmax, None, lmax)
+    x, y, w, g = workloads.make_features(wl, plan.n_paths, plan.d_out)
+    before = e3j.e3j_launch_count()
+    _check_double_backward(wl, plan, cp, x, y, w, g, partial=False)
+    # two calls, each the two fused sweeps with their follow-up kernels (4 launches), plus graph preparation
+    assert e3j.e3j_launch_count() - before <= 20   # the composition would take more than forty
+
+
+def _check_double_backward(wl, plan, cp, x, y, w, g, partial=True):
     n, e = wl.n_nodes, wl.n_edges
     rng = np.random.default_rng(77)
     ux = rng.standard_normal(x.shape).astype(np.float32)
@@ -385,6 +409,8 @@ def test_double_backward(config, n_atoms, natural, flags):
     kinds = ("out", "x", "sh", "w")
     for a, r, kind in zip(got, ref, kinds):
         assert_blockwise_close(a.cpu().numpy(), r, blocks_of_paths(cp.paths, kind), what="double backward " + kind)
+    if not partial:
+        return
     # only the harmonics' cotangent given, only two outputs wanted
     gg, gx, gsh, gw = run(None, _cuda(uy), None, g_sh=False, g_w=None)
     assert gsh is None and gw is None
@@ -395,6 +421,20 @@ def test_double_backward(config, n_atoms, natural, flags):
     # no cotangent at all: zeros
     for t in run(None, None, None):
         assert torch.count_nonzero(t) == 0
+
+
+def test_a_bounded_wait_that_runs_out_is_reported():
+    """Every wait in the specialised kernels gives up after a fixed number of polls.  The self-test makes one run
+    out on purpose (a barrier that nothing completes, 1000 polls): the wait returns, the kernel ends, the plan's
+    status word reads 1 once, and the plan keeps working."""
+    wl, plan, cp, x, y, w, g = make_case(2, 192)
+    assert e3j.e3j_plan_device_status(plan) == 0
+    returned, abort_flag = e3j.e3j_selftest_bounded_wait(plan, 1000)
+    assert (returned, abort_flag) == (0, 1)
+    assert e3j.e3j_plan_device_status(plan) == 1
+    assert e3j.e3j_plan_device_status(plan) == 0      # reading clears it
+    run_conv_parity(wl, plan, cp, x, y, w, g)         # the context and the plan are still usable
+    assert e3j.e3j_plan_device_status(plan) == 0
 
 
 def test_optional_gradients_can_be_skipped():
@@ -622,8 +662,15 @@ def test_config5_full_size_sampled():
 
     deg = np.bincount(wl.receivers, minlength=n)
     rp = rowptr.cpu().numpy()
+    # every receiver whose edges are cut by a CTA's edge-range boundary of the forward (their rows go through the
+    # partial-row scratch and the fix-up kernel): ranges of ceil4(ceil(E / CTAs)) edges, 2 CTAs per SM
+    n_cta = 2 * torch.cuda.get_device_properties(0).multi_processor_count
+    chunk = (-(-e // n_cta) + 3) // 4 * 4
+    cuts = np.arange(chunk, e, chunk)
+    straddled = np.unique(wl.receivers[cuts][wl.receivers[cuts] == wl.receivers[cuts - 1]])
+    assert len(straddled) > 100
     pick = np.unique(np.concatenate([rng.choice(n, 40, replace=False), np.argsort(deg)[-8:], np.argsort(deg)[:4],
-                                     [0, n - 1]]))
+                                     [0, n - 1], straddled]))
     out_blocks, w_blocks = blocks_of_paths(cp.paths, "out"), blocks_of_paths(cp.paths, "w")
     for b in pick:
         e0, e1 = int(rp[b]), int(rp[b + 1])

@@ -126,6 +126,8 @@ def test_collapsed_plan_tables(sig):
     assert plan.specialised == (irreps_in == "128x0e+128x1o" and irreps_out is None)
     assert [p["out_off"] for p in e3j.e3j_plan_paths(plan)] == offs
     i0, i1, i2, k, val = e3j.e3j_plan_records(plan)
+    keys = list(zip(i0.tolist(), k.tolist(), i1.tolist(), i2.tolist()))
+    assert keys == sorted(keys)   # sorted by (i0, path, i1, i2): the order the kernel generator relies on
     dense = np.zeros((R.shape[0], cp.d, cp.dp, cp.P))
     dense[i0, i1, i2, k] = val
     want = np.zeros_like(dense)
@@ -156,3 +158,19 @@ def test_every_generated_signature_is_picked_up_by_its_plan(repo_root):
         generic = e3j.e3j_plan_create(sig["irreps_in"], sig["sh_lmax"], sig["irreps_out"], sig["out_lmax"],
                                       flags | e3j.E3J_PLAN_GENERIC_ONLY)
         assert not generic.specialised
+
+
+def test_every_generated_signature_fits_the_allocation_free_scratch(repo_root):
+    """e3j_conv_fwd_noalloc keeps the forward's boundary-row scratch in a 24 MiB static array: 8 KB of receiver ids
+    plus two partial rows (D x N_q floats) per CTA, FC CTAs per SM.  Every signature in signatures.json must fit
+    on a 148-SM device (the one closest to the limit is the 156-row config-3 signature)."""
+    import json
+    sigs = json.load(open(os.path.join(repo_root, "paper_2609_35099_b200", "csrc", "fast", "signatures.json")))
+    worst = 0
+    for s in sigs:
+        flags = e3j.E3J_PLAN_COLLAPSE_OUTPUTS if s.get("collapse") else 0
+        plan = e3j.e3j_plan_create(s["irreps_in"], s["sh_lmax"], s["irreps_out"], s["out_lmax"], flags)
+        need = 8192 + 4 * 2 * (148 * s["FC"]) * plan.d_out * plan.n_channels
+        worst = max(worst, need)
+        assert need <= 24 << 20, (s["name"], need)
+    assert worst > 20 << 20   # the bound is tight: a new, larger signature must raise the array, not pass by luck

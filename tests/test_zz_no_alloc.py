@@ -37,6 +37,7 @@ def test_noalloc_forward_matches_workspace_forward_twice():
         torch.cuda.synchronize()
         assert_blockwise_close(out.cpu().numpy(), want.cpu().numpy().astype(np.float64), blocks,
                                what=f"noalloc call {call}")
+    assert e3j.e3j_noalloc_status() == 0   # no bounded wait gave up (the word is static, like the scratch)
     # and the reference entry point itself agrees with the oracle on this graph
     ref = oconv.conv_fwd(cp, x, y, w, wl.senders, wl.receivers)
     assert_blockwise_close(want.cpu().numpy(), ref, blocks, what="workspace forward")
@@ -48,6 +49,26 @@ def test_noalloc_forward_matches_workspace_forward_twice():
     out2 = torch.full_like(want2, float("nan"))
     e3j.e3j_conv_fwd_noalloc(plan, *a2, out2)
     assert_blockwise_close(out2.cpu().numpy(), want2.cpu().numpy().astype(np.float64), blocks, what="noalloc second graph")
+
+
+def test_noalloc_forward_on_the_signature_closest_to_the_scratch_limit():
+    """64x(0e+1o+2e+3o): 156 output rows, the largest need of the generated signatures (23.7 of the 24 MiB on
+    148 SMs) and the one-channel-per-lane consumer layout."""
+    c = workloads.CONFIGS[3]
+    wl = workloads.make_graph(3, n_atoms=250)
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], None, c["out_lmax"])
+    assert plan.specialised == 1
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], None, c["out_lmax"])
+    x, y, w, _ = workloads.make_features(wl, plan.n_paths, plan.d_out)
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+    args = [t(v) for v in (x, y, w, wl.senders, wl.receivers)]
+    want = e3j.e3j_conv_fwd(plan, *args)
+    blocks = blocks_of_paths(cp.paths, "out")
+    for call in range(2):
+        out = torch.full_like(want, float("nan"))
+        e3j.e3j_conv_fwd_noalloc(plan, *args, out)
+        assert_blockwise_close(out.cpu().numpy(), want.cpu().numpy().astype(np.float64), blocks, what=f"noalloc call {call}")
+    assert e3j.e3j_noalloc_status() == 0
 
 
 def test_noalloc_rejects_plans_without_specialised_kernels_and_handles_empty_graphs():
