@@ -1,18 +1,23 @@
 // Registry of signature-specialised kernels.  Entries are appended by the generated
-// translation units listed in fast/registry_entries.inc.
+// translation units listed in fast/registry_entries.inc (a build with overlay signatures, see build.py,
+// points E3J_REGISTRY_INC at its own list).
 #include "fast_registry.hpp"
 
 #include <cstring>
 
 namespace e3j {
 
+#ifndef E3J_REGISTRY_INC
+#define E3J_REGISTRY_INC "fast/registry_entries.inc"
+#endif
+
 #define E3J_FAST_ENTRY(name) extern const FastKernels name;
-#include "fast/registry_entries.inc"
+#include E3J_REGISTRY_INC
 #undef E3J_FAST_ENTRY
 
 static const FastKernels* const kEntries[] = {
 #define E3J_FAST_ENTRY(name) &name,
-#include "fast/registry_entries.inc"
+#include E3J_REGISTRY_INC
 #undef E3J_FAST_ENTRY
     nullptr};
 

@@ -72,11 +72,70 @@ def fmt_float(v: float) -> str:
     return s + "f"
 
 
+def auto_params(sig, info):
+    """Tile parameters for a signature that gives none ("auto": 1, or an overlay entry): channels per lane from the
+    channel count, row groups from the number of coefficient pairs, tile sizes from what fits in shared memory
+    (the formulas of FwdSmem / BwdSmem / Bwd1Smem) and CTAs per SM from the registers the bodies need.  The
+    hand-tuned entries of signatures.json were found by measurement; these are the starting point such a search
+    would begin from."""
+    NQ, DIN, DSH, P, D = info["n_channels"], info["d_in"], info["d_sh"], info["n_paths"], info["d_out"]
+    apad = info["n_pairs"] + 16
+    if NQ % 32:
+        raise ValueError("generated kernels need a multiple of 32 channels")
+    V = 4 if NQ % 128 == 0 else 2 if NQ % 64 == 0 else 1
+    CH = NQ // (32 * V)
+    smem = 227 * 1024
+    up = lambda v, a: (v + a - 1) // a * a
+    need = {4: 168, 2: 104, 1: 72}[V]
+    out = {"V": V, "FW": 4 if info["n_pairs"] <= 300 else 2, "FS": 2, "BV": V, "BW": 4, "BS": 2, "EV": V, "ES": 2}
+    # forward: CTAs per SM by registers, then the largest tile that fits
+    threads = (out["FW"] * CH + 2) * 32
+    FC = 2 if 65536 // (2 * threads) >= need else 1
+    edge = 4 * (P * NQ + DIN * NQ + apad + DSH)
+    while True:
+        T = min(12, ((smem // FC - 1024 - 256) // out["FS"] - 256) // edge)
+        if T >= 3 or FC == 1:
+            break
+        FC = 1
+    if T < 1:
+        raise ValueError("one edge does not fit the forward stage ring")
+    out.update(FT=T, FC=FC)
+    # path-group backward (the fallback; always compiled)
+    fixed = 256 + 4 * 2 * out["BW"] * DIN * NQ + 4 * 2 * out["BW"] * CH * 16
+    BC = FC
+    while True:
+        BT = min(8, ((smem // BC - 1024 - fixed) // out["BS"] - 256) // edge)
+        if BT >= 2 or BC == 1:
+            break
+        BC = 1
+    if BT < 1:
+        raise ValueError("one edge does not fit the backward stage ring")
+    out.update(BT=BT, BC=BC)
+    # edge-wise backward: one CTA per SM, T edges x CH warps per edge.  When shared memory allows only a few edges
+    # per tile, halving the channels per lane doubles the warps (measured on 128x(0e+1o+2e+3o), l <= 2: 4 -> 8
+    # consumer warps, 1.77 -> 1.08 ms)
+    def edgewise(EV):
+        CHe = NQ // (32 * EV)
+        warps = 65536 // (32 * {4: 224, 2: 128, 1: 96}[EV]) - 1
+        fixed = 2048 + 4 * 2 * 32 * DSH + 4 * out["ES"] * D * NQ
+        return min(warps // CHe, 16, ((smem - 1024 - fixed) // out["ES"] - 256) // (edge + 4 * CHe * 16)), CHe
+    EV = V
+    ET, CHe = edgewise(EV)
+    if ET * CHe < 6 and EV > 1:
+        EV //= 2
+        ET, CHe = edgewise(EV)
+    if ET >= 2:
+        out.update(ET=ET, EV=EV)
+    return out
+
+
 class Sig:
     def __init__(self, sig):
-        self.cfg = sig
         self.name = sig["name"]
         self.info, self.paths, self.recs, self.signature = load_records(sig)
+        if "V" not in sig:   # no (or only some) tile parameters given: derive the rest
+            sig = {**auto_params(sig, self.info), **sig}
+        self.cfg = sig
         self.NQ, self.DIN, self.DSH = self.info["n_channels"], self.info["d_in"], self.info["d_sh"]
         self.P, self.D, self.NNZ = self.info["n_paths"], self.info["d_out"], self.info["nnz"]
         self.V = sig["V"]
@@ -744,8 +803,15 @@ class Sig:
         return "\n".join(o) + "\n"
 
 
-def generate():
+def generate(extra=None):
+    """{file name: text} for the committed signatures plus, if given, the entries of an overlay list."""
     sigs = json.loads((HERE / "fast" / "signatures.json").read_text())
+    if extra:
+        have = {s["name"] for s in sigs}
+        for s in extra:
+            if s["name"] in have:
+                raise ValueError(f"overlay signature {s['name']} already exists")
+        sigs = sigs + list(extra)
     files = {}
     for sig in sigs:
         files[f"sig_{sig['name']}.cu"] = Sig(sig).emit()
