@@ -303,6 +303,28 @@ int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
                const float* w, const float* grad_out, float* grad_x1, float* grad_x2,
                float* grad_w, void* stream);
 
+/* Receiver sharding over several GPUs, one process per GPU (paper: the one-line SPMD sharding of its API; the
+ * backward as message passing on the transposed graph).  A rank owns the receivers [node_lo, node_hi) and the
+ * edges into them, a contiguous slice of the receiver-sorted edge list; every edge-local tensor (sh, w, their
+ * gradients) and every output row lives with its receiver and never moves.  What crosses GPUs is node rows only:
+ * forward, the x rows of the halo (senders the rank does not own); backward, the grad_x shares for those
+ * senders, which their owners add in rank order (bit-reproducible).  The exchange itself is the caller's
+ * (torch.distributed / NCCL; paper_2609_35099_b200/sharding.py); remote rows land in local memory before any
+ * kernel of this library reads them.
+ * e3j_shard_prepare: integer kernels.  In: the slice's global sender / receiver ids.  Out: local ids
+ *   (owned node node_lo + i -> i; halo node halo_ids[h] -> (node_hi - node_lo) + h), halo_ids in ascending global
+ *   order (capacity n_nodes) and the DEVICE word *n_halo.  The local problem then has (node_hi - node_lo) + n_halo
+ *   nodes and runs through e3j_graph_prepare / e3j_conv_fwd / e3j_conv_bwd unchanged.
+ * e3j_rows_gather: dst[i, :] = src[ids[i], :].  e3j_rows_add: dst[ids[i], :] += src[i, :]; ids must not repeat
+ *   within a call (the ids of one rank's halo do not).  row_len floats, a multiple of 4; 16-byte aligned rows. */
+size_t e3j_shard_prepare_workspace_bytes(int64_t n_nodes);
+int e3j_shard_prepare(int64_t n_nodes, int64_t n_edges_shard, int32_t node_lo, int32_t node_hi,
+                      const int32_t* senders, const int32_t* receivers, int32_t* local_senders,
+                      int32_t* local_receivers, int32_t* halo_ids, int32_t* n_halo, void* workspace,
+                      size_t workspace_bytes, void* stream);
+int e3j_rows_gather(float* dst, const float* src, const int32_t* ids, int64_t n_ids, int64_t row_len, void* stream);
+int e3j_rows_add(float* dst, const float* src, const int32_t* ids, int64_t n_ids, int64_t row_len, void* stream);
+
 /* Self-test of the kernels' bounded waits (no counterpart in the paper).  Every wait inside the specialised
  * kernels gives up after a fixed number of polls, records the failure in the plan's device status word and
  * lets the kernel drain instead of hanging the GPU.  This call exercises that path on purpose, without any

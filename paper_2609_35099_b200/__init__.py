@@ -25,7 +25,7 @@ __all__ = [
     "e3j_conv_bwd_bwd_workspace_bytes", "e3j_conv_bwd_bwd",
     "e3j_radial_weights", "e3j_conv_radial_fwd_workspace_bytes", "e3j_conv_radial_bwd_workspace_bytes",
     "e3j_conv_radial_fwd", "e3j_conv_radial_bwd",
-    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
+    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_shard_prepare", "e3j_rows_gather", "e3j_rows_add", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
     "E3J_PLAN_COLLAPSE_OUTPUTS",
 ]
 
@@ -112,6 +112,14 @@ def _load():
     lib.e3j_conv_radial_bwd.restype = i32
     lib.e3j_tp_fwd.argtypes = [vp, i64] + [vp] * 5
     lib.e3j_tp_bwd.argtypes = [vp, i64] + [vp] * 8
+    lib.e3j_shard_prepare_workspace_bytes.argtypes = [i64]
+    lib.e3j_shard_prepare_workspace_bytes.restype = sz
+    lib.e3j_shard_prepare.argtypes = [i64, i64, i32, i32] + [vp] * 7 + [sz, vp]
+    lib.e3j_shard_prepare.restype = i32
+    lib.e3j_rows_gather.argtypes = [vp, vp, vp, i64, i64, vp]
+    lib.e3j_rows_gather.restype = i32
+    lib.e3j_rows_add.argtypes = [vp, vp, vp, i64, i64, vp]
+    lib.e3j_rows_add.restype = i32
     lib.e3j_selftest_bounded_wait.argtypes = [vp, u32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
     lib.e3j_selftest_bounded_wait.restype = i32
     lib.e3j_status_string.argtypes = [i32]
@@ -517,6 +525,48 @@ def e3j_tp_bwd(plan: Plan, x1, x2, w, grad_out, grad_x1=True, grad_x2=True, grad
         _dev_ptr(grad_x1, f32, None, "grad_x1"), _dev_ptr(grad_x2, f32, None, "grad_x2"),
         _dev_ptr(grad_w, f32, None, "grad_w"), _stream(stream)), "e3j_tp_bwd")
     return grad_x1, grad_x2, grad_w
+
+
+def e3j_shard_prepare(n_nodes: int, node_lo: int, node_hi: int, senders, receivers, stream=None):
+    """Local problem of the rank that owns receivers [node_lo, node_hi): (local_senders, local_receivers, halo_ids)
+    for its slice of the edge list (global ids in).  halo_ids (ascending global ids) is cut to its length, which
+    costs one device-to-host read of the count."""
+    torch = _torch()
+    e, i32 = senders.numel(), torch.int32
+    dev = senders.device
+    ls = torch.empty(max(e, 1), dtype=i32, device=dev)
+    lr = torch.empty(max(e, 1), dtype=i32, device=dev)
+    halo = torch.empty(max(n_nodes, 1), dtype=i32, device=dev)
+    count = torch.zeros(1, dtype=i32, device=dev)
+    ws = torch.empty(max(int(_load().e3j_shard_prepare_workspace_bytes(n_nodes)), 256), dtype=torch.uint8, device=dev)
+    _check(_load().e3j_shard_prepare(n_nodes, e, node_lo, node_hi, _dev_ptr(senders, i32, (e,), "senders"),
+                                     _dev_ptr(receivers, i32, (e,), "receivers"), _dev_ptr(ls, i32, None, "local_senders"),
+                                     _dev_ptr(lr, i32, None, "local_receivers"), _dev_ptr(halo, i32, None, "halo_ids"),
+                                     _dev_ptr(count, i32, None, "n_halo"), ctypes.c_void_p(ws.data_ptr()), ws.numel(),
+                                     _stream(stream)), "e3j_shard_prepare")
+    return ls[:e], lr[:e], halo[:int(count.item())]
+
+
+def e3j_rows_gather(dst, src, ids, stream=None):
+    """dst[i] = src[ids[i]] for float32 tensors whose trailing dimensions form the row."""
+    torch = _torch()
+    n = ids.numel()
+    row = src[0].numel() if src.shape[0] else 0
+    if n:
+        _check(_load().e3j_rows_gather(_dev_ptr(dst, torch.float32, None, "dst"), _dev_ptr(src, torch.float32, None, "src"),
+                                       _dev_ptr(ids, torch.int32, (n,), "ids"), n, row, _stream(stream)), "e3j_rows_gather")
+    return dst
+
+
+def e3j_rows_add(dst, src, ids, stream=None):
+    """dst[ids[i]] += src[i]; ids must not repeat within the call."""
+    torch = _torch()
+    n = ids.numel()
+    row = dst[0].numel() if dst.shape[0] else 0
+    if n:
+        _check(_load().e3j_rows_add(_dev_ptr(dst, torch.float32, None, "dst"), _dev_ptr(src, torch.float32, None, "src"),
+                                    _dev_ptr(ids, torch.int32, (n,), "ids"), n, row, _stream(stream)), "e3j_rows_add")
+    return dst
 
 
 def e3j_selftest_bounded_wait(plan: Plan, spin_limit: int = 1000):
