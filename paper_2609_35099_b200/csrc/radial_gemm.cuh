@@ -5,7 +5,7 @@
 // runs; operands pass through a ring of shared-memory stages of 32 k each, written by converter warps that read
 // float32 from global memory, split every value into its (hi, lo) TF32 pair and store both in the K-major
 // core-matrix layout that the tensor cores read.  Roles: warps 0-3 read finished tiles out of tensor memory
-// and store them, warps 4-7 convert, warp 8 issues the tcgen05.mma instructions (one lane).
+// and store them, eight warps convert, the last warp issues the tcgen05.mma instructions (one lane).
 //
 // A Problem type describes one product: which output tiles a CTA owns, how many K chunks a tile has, where
 // operand values come from (zero outside the matrices) and where results go.  Three instances are used:
@@ -32,7 +32,9 @@ constexpr int kTileM = 128;      // rows of an output tile = tensor-memory lanes
 constexpr int kChunkK = 32;      // k per shared-memory stage (four tcgen05.mma steps of 8)
 constexpr int kStages = 3;
 constexpr int kGroupChunks = 8;  // K chunks accumulated inside tensor memory before the tile is read out
-constexpr int kGemmThreads = 9 * 32;
+constexpr int kConvWarps = 8;     // converter warps
+constexpr int kPrefetch = 2;      // chunks of loads in flight per converter thread
+constexpr int kGemmThreads = (4 + kConvWarps + 1) * 32;   // epilogue, converters, tensor-core issue
 
 template <int N>
 struct GemmSmem {
@@ -46,39 +48,48 @@ struct GemmSmem {
     static constexpr size_t total = off_stage + kStages * stage_bytes;
 };
 
-// Converter: fills rows [0, ROWS) x k [0, 32) of one operand of one stage.  LANE_ROWS = 8: a warp item is
-// 8 rows x 4 k-quads (sources with k contiguous); LANE_ROWS = 32: 32 rows x 1 k-quad (sources with rows
-// contiguous).  Either way 8 consecutive lanes write 128 contiguous bytes of shared memory.
-template <int ROWS, int LANE_ROWS, class Load>
-__device__ __forceinline__ void convert_operand(unsigned char* hi, unsigned char* lo, const int cwarp, const int lane,
-                                                const Load& load) {
-    constexpr int QUADS = kChunkK / 4;
-    constexpr int LANE_QUADS = 32 / LANE_ROWS;
-    constexpr int ITEMS = (ROWS / LANE_ROWS) * (QUADS / LANE_QUADS);   // warp items of the operand
+// Converters: an operand of a stage is rows [0, ROWS) x k [0, 32).  LANE_ROWS = 8: a warp item is 8 rows x 4 k-quads
+// (sources with k contiguous); LANE_ROWS = 32: 32 rows x 1 k-quad (sources with rows contiguous).  Either way 8
+// consecutive lanes write 128 contiguous bytes of shared memory.  The work is two halves: all loads of a chunk go
+// out first (into registers), the conversion and the stores follow one chunk later, so that the loads of chunk
+// i + 1 are in flight while chunk i is converted.
+template <int ROWS, int LANE_ROWS>
+struct OperandItems {
+    static constexpr int QUADS = kChunkK / 4;
+    static constexpr int LANE_QUADS = 32 / LANE_ROWS;
+    static constexpr int ITEMS = (ROWS / LANE_ROWS) * (QUADS / LANE_QUADS);   // warp items of the operand
     static_assert(ROWS % LANE_ROWS == 0 && QUADS % LANE_QUADS == 0, "operand does not tile");
-    static_assert(ITEMS % 4 == 0, "four converter warps share the items");
-    constexpr int NI = ITEMS / 4;
-    float4 v[NI];
-    // every load of the operand is issued before the first conversion, so that they are in flight together
-#pragma unroll
-    for (int i = 0; i < NI; ++i) {
-        const int item = cwarp + 4 * i;
+    static_assert(ITEMS % kConvWarps == 0, "the converter warps share the items");
+    static constexpr int NI = ITEMS / kConvWarps;
+    __device__ static __forceinline__ void coords(int i, int cwarp, int lane, int& row, int& k) {
+        const int item = cwarp + kConvWarps * i;
         const int rg = item / (QUADS / LANE_QUADS), qg = item % (QUADS / LANE_QUADS);
-        v[i] = load(rg * LANE_ROWS + lane % LANE_ROWS, (qg * LANE_QUADS + lane / LANE_ROWS) * 4);
+        row = rg * LANE_ROWS + lane % LANE_ROWS;
+        k = (qg * LANE_QUADS + lane / LANE_ROWS) * 4;
     }
+    template <class Load>
+    __device__ static __forceinline__ void load(float4 (&v)[NI], int cwarp, int lane, const Load& ld) {
 #pragma unroll
-    for (int i = 0; i < NI; ++i) {
-        const int item = cwarp + 4 * i;
-        const int rg = item / (QUADS / LANE_QUADS), qg = item % (QUADS / LANE_QUADS);
-        const int row = rg * LANE_ROWS + lane % LANE_ROWS;
-        const int quad = qg * LANE_QUADS + lane / LANE_ROWS;
-        float4 h, l;
-        umma::split_tf32(v[i], h, l);
-        const uint32_t off = umma::tile_offset(row, quad * 4, kChunkK);
-        *reinterpret_cast<float4*>(hi + off) = h;
-        *reinterpret_cast<float4*>(lo + off) = l;
+        for (int i = 0; i < NI; ++i) {
+            int row, k;
+            coords(i, cwarp, lane, row, k);
+            v[i] = ld(row, k);
+        }
     }
-}
+    __device__ static __forceinline__ void store(const float4 (&v)[NI], unsigned char* hi, unsigned char* lo, int cwarp,
+                                                 int lane) {
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+            int row, k;
+            coords(i, cwarp, lane, row, k);
+            float4 h, l;
+            umma::split_tf32(v[i], h, l);
+            const uint32_t off = umma::tile_offset(row, k, kChunkK);
+            *reinterpret_cast<float4*>(hi + off) = h;
+            *reinterpret_cast<float4*>(lo + off) = l;
+        }
+    }
+};
 
 template <class Prob>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob prob) {
@@ -97,13 +108,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { fast::mbar_init(&stage_full[s], 4); fast::mbar_init(&stage_empty[s], 1); }
+        for (int s = 0; s < kStages; ++s) { fast::mbar_init(&stage_full[s], kConvWarps); fast::mbar_init(&stage_empty[s], 1); }
         for (int b = 0; b < 2; ++b) { fast::mbar_init(&d_full[b], 1); fast::mbar_init(&d_empty[b], 4); }
         fast::mbar_init(drain, 1);
         *abort_flag = 0;
         fast::mbar_fence_init();
     }
-    if (warp == 8) umma::tmem_alloc(tmem_slot, kTmemCols);
+    if (warp == 4 + kConvWarps) umma::tmem_alloc(tmem_slot, kTmemCols);
     umma::fence_before_sync();
     __syncthreads();
     umma::fence_after_sync();
@@ -138,24 +149,41 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
                 if (flush) prob.store(t, warp * 32 + lane, c0, v);
             }
         }
-    } else if (warp < 8) {
+    } else if (warp < 4 + kConvWarps) {
         // ------------------------------------------------ converters: global float32 -> (hi, lo) TF32 stages
+        using OA = OperandItems<kTileM, Prob::A_LANE_ROWS>;
+        using OB = OperandItems<N, Prob::B_LANE_ROWS>;
         const int cwarp = warp - 4;
-        int it = 0;
+        // kPrefetch chunks of loads are in flight per thread: chunk i is converted while the loads of chunks
+        // i + 1 .. i + kPrefetch - 1 travel (one global-memory latency per chunk would otherwise bound the kernel)
+        float4 va[kPrefetch][OA::NI], vb[kPrefetch][OB::NI];
+        int tf = 0, kf = 0;                      // next chunk to fetch
+        int ts = 0, ks = 0;                      // next chunk to convert and store
+        auto fetch = [&](float4 (&a)[OA::NI], float4 (&b)[OB::NI]) {
+            if (tf >= n_tiles) return;
+            const int tt = tf, kk = kf;
+            OA::load(a, cwarp, lane, [&](int row, int k) { return prob.load_a(tt, kk, row, k); });
+            OB::load(b, cwarp, lane, [&](int row, int k) { return prob.load_b(tt, kk, row, k); });
+            if (++kf == prob.n_chunks(tf)) { kf = 0; ++tf; }
+        };
+#pragma unroll
+        for (int u = 0; u < kPrefetch; ++u) fetch(va[u], vb[u]);
         bool ok = true;
-        for (int t = 0; ok && t < n_tiles; ++t) {
-            const int n_chunks = prob.n_chunks(t);
-            for (int kc = 0; kc < n_chunks; ++kc, ++it) {
-                const int s = it % kStages;
+#pragma unroll 1
+        for (int it0 = 0; ok && ts < n_tiles; it0 += kPrefetch) {
+#pragma unroll
+            for (int u = 0; u < kPrefetch; ++u) {
+                if (!ok || ts >= n_tiles) break;
+                const int it = it0 + u, s = it % kStages;
                 if (it >= kStages && !fast::mbar_wait(&stage_empty[s], ((it / kStages) + 1) & 1, abort_flag, prob.status)) { ok = false; break; }
                 unsigned char* st = smem + L::off_stage + (size_t)s * L::stage_bytes;
-                convert_operand<kTileM, Prob::A_LANE_ROWS>(st, st + L::a_bytes, cwarp, lane,
-                    [&](int row, int k) { return prob.load_a(t, kc, row, k); });
-                convert_operand<N, Prob::B_LANE_ROWS>(st + 2 * L::a_bytes, st + 2 * L::a_bytes + L::b_bytes, cwarp, lane,
-                    [&](int row, int k) { return prob.load_b(t, kc, row, k); });
+                OA::store(va[u], st, st + L::a_bytes, cwarp, lane);
+                OB::store(vb[u], st + 2 * L::a_bytes, st + 2 * L::a_bytes + L::b_bytes, cwarp, lane);
                 umma::fence_smem_to_async();
                 __syncwarp();
                 if (lane == 0) fast::mbar_arrive(&stage_full[s]);
+                if (++ks == prob.n_chunks(ts)) { ks = 0; ++ts; }
+                fetch(va[u], vb[u]);             // refill this register set with the chunk kPrefetch ahead
             }
         }
     } else {
@@ -203,7 +231,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
     }
     umma::fence_before_sync();
     __syncthreads();
-    if (warp == 8) umma::tmem_dealloc(tmem_base, kTmemCols);
+    if (warp == 4 + kConvWarps) umma::tmem_dealloc(tmem_base, kTmemCols);
 }
 
 // ------------------------------------------------------------------------------------------------ problems
@@ -244,9 +272,15 @@ struct RadialWeights {
         if (c >= C) return;
         const int64_t e0 = e_begin() + (int64_t)t * 128 + n0;
         const int64_t e_end = min(n_edges, e_begin() + chunk);
+        float* dst = s + (size_t)e0 * C + c;   // lanes: consecutive c; one row of s further per value
+        if (e0 + 32 <= e_end) {                // whole piece inside the range: no per-store test
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-            if (e0 + i < e_end) s[(size_t)(e0 + i) * C + c] = v[i];   // lanes: consecutive c
+            for (int i = 0; i < 32; ++i) dst[(size_t)i * C] = v[i];
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (e0 + i < e_end) dst[(size_t)i * C] = v[i];
+        }
     }
 };
 
@@ -334,11 +368,16 @@ struct GradLayer {
     __device__ __forceinline__ void store(int, int m, int n0, const float (&v)[32]) const {
         const int c = blockIdx.x * 128 + m;
         if (c >= C) return;
-        float* dst = partial + (size_t)blockIdx.y * H * C;
         const int j0 = blockIdx.z * 64 + n0;
+        float* dst = partial + (size_t)blockIdx.y * H * C + (size_t)j0 * C + c;   // lanes: consecutive c
+        if (j0 + 32 <= H) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-            if (j0 + i < H) dst[(size_t)(j0 + i) * C + c] = v[i];   // lanes: consecutive c
+            for (int i = 0; i < 32; ++i) dst[(size_t)i * C] = v[i];
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (j0 + i < H) dst[(size_t)i * C] = v[i];
+        }
     }
 };
 
