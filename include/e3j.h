@@ -303,6 +303,22 @@ int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
                const float* w, const float* grad_out, float* grad_x1, float* grad_x2,
                float* grad_w, void* stream);
 
+/* Float64 convolution (paper, appendix on the benchmark setup: float64 builds of the kernels are shipped beside
+ * the float32 ones).  Same operation, layouts, graph arguments and conventions as e3j_conv_fwd / e3j_conv_bwd with
+ * every tensor in float64 and the coupling coefficients in float64 as the plan builder computed them.  Table-driven
+ * kernels for every plan (there are no signature-specialised float64 kernels): each output element is one thread's
+ * sum in a fixed order, bit-identical from run to run.  No alignment requirement beyond 8 bytes.  rowptr /
+ * sender_perm / colptr as produced by e3j_graph_prepare, or NULL (then derived into the workspace, 256-byte
+ * aligned, e3j_conv_f64_workspace_bytes()); any of grad_x, grad_sh, grad_w may be NULL. */
+size_t e3j_conv_f64_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges);
+int e3j_conv_fwd_f64(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const double* x, const double* sh,
+                     const double* w, const int32_t* senders, const int32_t* receivers, const int32_t* rowptr,
+                     double* out, void* workspace, size_t workspace_bytes, void* stream);
+int e3j_conv_bwd_f64(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const double* x, const double* sh,
+                     const double* w, const int32_t* senders, const int32_t* receivers, const int32_t* sender_perm,
+                     const int32_t* colptr, const double* grad_out, double* grad_x, double* grad_sh, double* grad_w,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
 /* Receiver sharding over several GPUs, one process per GPU (paper: the one-line SPMD sharding of its API; the
  * backward as message passing on the transposed graph).  A rank owns the receivers [node_lo, node_hi) and the
  * edges into them, a contiguous slice of the receiver-sorted edge list; every edge-local tensor (sh, w, their

@@ -25,7 +25,7 @@ __all__ = [
     "e3j_conv_bwd_bwd_workspace_bytes", "e3j_conv_bwd_bwd",
     "e3j_radial_weights", "e3j_conv_radial_fwd_workspace_bytes", "e3j_conv_radial_bwd_workspace_bytes",
     "e3j_conv_radial_fwd", "e3j_conv_radial_bwd",
-    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_shard_prepare", "e3j_rows_gather", "e3j_rows_add", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
+    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_conv_fwd_f64", "e3j_conv_bwd_f64", "e3j_shard_prepare", "e3j_rows_gather", "e3j_rows_add", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
     "E3J_PLAN_COLLAPSE_OUTPUTS",
 ]
 
@@ -112,6 +112,12 @@ def _load():
     lib.e3j_conv_radial_bwd.restype = i32
     lib.e3j_tp_fwd.argtypes = [vp, i64] + [vp] * 5
     lib.e3j_tp_bwd.argtypes = [vp, i64] + [vp] * 8
+    lib.e3j_conv_f64_workspace_bytes.argtypes = [vp, i64, i64]
+    lib.e3j_conv_f64_workspace_bytes.restype = sz
+    lib.e3j_conv_fwd_f64.argtypes = [vp, i64, i64] + [vp] * 8 + [sz, vp]
+    lib.e3j_conv_fwd_f64.restype = i32
+    lib.e3j_conv_bwd_f64.argtypes = [vp, i64, i64] + [vp] * 12 + [sz, vp]
+    lib.e3j_conv_bwd_f64.restype = i32
     lib.e3j_shard_prepare_workspace_bytes.argtypes = [i64]
     lib.e3j_shard_prepare_workspace_bytes.restype = sz
     lib.e3j_shard_prepare.argtypes = [i64, i64, i32, i32] + [vp] * 7 + [sz, vp]
@@ -525,6 +531,40 @@ def e3j_tp_bwd(plan: Plan, x1, x2, w, grad_out, grad_x1=True, grad_x2=True, grad
         _dev_ptr(grad_x1, f32, None, "grad_x1"), _dev_ptr(grad_x2, f32, None, "grad_x2"),
         _dev_ptr(grad_w, f32, None, "grad_w"), _stream(stream)), "e3j_tp_bwd")
     return grad_x1, grad_x2, grad_w
+
+
+def e3j_conv_fwd_f64(plan: Plan, x, sh, w, senders, receivers, rowptr=None, out=None, stream=None):
+    """Float64 forward convolution (table-driven kernels)."""
+    torch = _torch()
+    n, e, f64, i32 = x.shape[0], senders.numel(), torch.float64, torch.int32
+    if out is None:
+        out = torch.empty((n, plan.d_out, plan.n_channels), dtype=f64, device=x.device)
+    ws = _workspace(int(_load().e3j_conv_f64_workspace_bytes(plan.handle, n, e)), x, None)
+    _check(_load().e3j_conv_fwd_f64(
+        plan.handle, n, e, _dev_ptr(x, f64, (n, plan.d_in, plan.n_channels), "x"), _dev_ptr(sh, f64, (e, plan.d_sh), "sh"),
+        _dev_ptr(w, f64, (e, plan.n_paths, plan.n_channels), "w"), _dev_ptr(senders, i32, (e,), "senders"),
+        _dev_ptr(receivers, i32, (e,), "receivers"), _dev_ptr(rowptr, i32, (n + 1,), "rowptr"),
+        _dev_ptr(out, f64, (n, plan.d_out, plan.n_channels), "out"), ctypes.c_void_p(ws.data_ptr()), ws.numel(),
+        _stream(stream)), "e3j_conv_fwd_f64")
+    return out
+
+
+def e3j_conv_bwd_f64(plan: Plan, x, sh, w, senders, receivers, grad_out, sender_perm=None, colptr=None, stream=None):
+    """Float64 backward convolution: (grad_x, grad_sh, grad_w)."""
+    torch = _torch()
+    n, e, f64, i32 = x.shape[0], senders.numel(), torch.float64, torch.int32
+    gx = torch.empty((n, plan.d_in, plan.n_channels), dtype=f64, device=x.device)
+    gsh = torch.empty((e, plan.d_sh), dtype=f64, device=x.device)
+    gw = torch.empty((e, plan.n_paths, plan.n_channels), dtype=f64, device=x.device)
+    ws = _workspace(int(_load().e3j_conv_f64_workspace_bytes(plan.handle, n, e)), x, None)
+    _check(_load().e3j_conv_bwd_f64(
+        plan.handle, n, e, _dev_ptr(x, f64, (n, plan.d_in, plan.n_channels), "x"), _dev_ptr(sh, f64, (e, plan.d_sh), "sh"),
+        _dev_ptr(w, f64, (e, plan.n_paths, plan.n_channels), "w"), _dev_ptr(senders, i32, (e,), "senders"),
+        _dev_ptr(receivers, i32, (e,), "receivers"), _dev_ptr(sender_perm, i32, (e,), "sender_perm"),
+        _dev_ptr(colptr, i32, (n + 1,), "colptr"), _dev_ptr(grad_out, f64, (n, plan.d_out, plan.n_channels), "grad_out"),
+        _dev_ptr(gx, f64, None, "grad_x"), _dev_ptr(gsh, f64, None, "grad_sh"), _dev_ptr(gw, f64, None, "grad_w"),
+        ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream(stream)), "e3j_conv_bwd_f64")
+    return gx, gsh, gw
 
 
 def e3j_shard_prepare(n_nodes: int, node_lo: int, node_hi: int, senders, receivers, stream=None):

@@ -22,10 +22,12 @@ namespace {
 
 template <class Key>
 void pack_sorted(const std::vector<Record>& rec, int n_keys, Key key, std::vector<PackedRecord>& out,
-                 std::vector<int32_t>& start, int which) {
+                 std::vector<int32_t>& start, int which, std::vector<double>& val64) {
     std::vector<Record> r = rec;
     std::stable_sort(r.begin(), r.end(), [&](const Record& a, const Record& b) { return key(a) < key(b); });
     out.clear();
+    val64.clear();
+    for (const Record& x : r) val64.push_back(x.val);
     start.assign(n_keys + 1, 0);
     for (const Record& x : r) {
         PackedRecord p{};
@@ -51,9 +53,10 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
 
     std::vector<PackedRecord> r0, r1, r2;
     std::vector<int32_t> s0, s1, s2, i0_path(plan->D), path_off(plan->P + 1), path_rows(plan->P);
-    pack_sorted(plan->rec, plan->D, [](const Record& r) { return r.i0; }, r0, s0, 0);
-    pack_sorted(plan->rec, plan->d, [](const Record& r) { return r.i1; }, r1, s1, 1);
-    pack_sorted(plan->rec, plan->dp, [](const Record& r) { return r.i2; }, r2, s2, 2);
+    std::vector<double> v0, v1, v2;
+    pack_sorted(plan->rec, plan->D, [](const Record& r) { return r.i0; }, r0, s0, 0, v0);
+    pack_sorted(plan->rec, plan->d, [](const Record& r) { return r.i1; }, r1, s1, 1, v1);
+    pack_sorted(plan->rec, plan->dp, [](const Record& r) { return r.i2; }, r2, s2, 2, v2);
     for (int k = 0; k < plan->P; ++k) {
         path_off[k] = plan->paths[k].out_off;
         path_rows[k] = 2 * plan->paths[k].L + 1;
@@ -69,6 +72,8 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
     const size_t o_s0 = reserve(4 * s0.size()), o_s1 = reserve(4 * s1.size()), o_s2 = reserve(4 * s2.size());
     const size_t o_ip = reserve(4 * i0_path.size()), o_po = reserve(4 * path_off.size());
     const size_t o_pr = reserve(4 * path_rows.size());
+    const size_t nv = sizeof(double) * plan->rec.size();
+    const size_t o_v0 = reserve(nv), o_v1 = reserve(nv), o_v2 = reserve(nv);
     const size_t o_st = reserve(256);
     std::vector<char> host(off, 0);
     std::memcpy(host.data() + o_r0, r0.data(), nb);
@@ -80,6 +85,9 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
     std::memcpy(host.data() + o_ip, i0_path.data(), 4 * i0_path.size());
     std::memcpy(host.data() + o_po, path_off.data(), 4 * path_off.size());
     std::memcpy(host.data() + o_pr, path_rows.data(), 4 * path_rows.size());
+    std::memcpy(host.data() + o_v0, v0.data(), nv);
+    std::memcpy(host.data() + o_v1, v1.data(), nv);
+    std::memcpy(host.data() + o_v2, v2.data(), nv);
 
     DeviceTables t;
     t.device = device;
@@ -96,6 +104,9 @@ int get_device_tables(const e3j_plan* plan, DeviceTables& out) {
     t.i0_path = (const int32_t*)(b + o_ip);
     t.path_out_off = (const int32_t*)(b + o_po);
     t.path_rows = (const int32_t*)(b + o_pr);
+    t.val64_i0 = (const double*)(b + o_v0);
+    t.val64_i1 = (const double*)(b + o_v1);
+    t.val64_i2 = (const double*)(b + o_v2);
     t.status = (int32_t*)(b + o_st);
     plan->dev.push_back(t);
     out = t;

@@ -38,6 +38,10 @@ struct DeviceTables {
     const int32_t* i2_start = nullptr;  // [d'+1]
     const int32_t* path_out_off = nullptr;  // [P+1] first output row of every path (last entry: D)
     const int32_t* path_rows = nullptr;     // [P] rows of every path, 2L+1
+    // the record values in float64, in the order of by_i0 / by_i1 / by_i2 (float64 entry points)
+    const double* val64_i0 = nullptr;
+    const double* val64_i1 = nullptr;
+    const double* val64_i2 = nullptr;
     int32_t* status = nullptr;  // sticky device status word (0 = fine), see e3j_plan_device_status
 };
 

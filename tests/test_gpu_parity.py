@@ -750,3 +750,36 @@ def test_tensor_product_full_size_sampled():
     assert_blockwise_close(h(g1), r1, blocks_of_paths(cp.paths, "x"), what="tp grad_x1")
     assert_blockwise_close(h(g2), r2, blocks_of_paths(cp.paths, "sh"), what="tp grad_x2")
     assert_blockwise_close(h(gw), rw, blocks_of_paths(cp.paths, "w"), what="tp grad_w")
+
+
+@pytest.mark.parametrize("config,n_atoms,collapse", [(1, None, False), (2, 192, False), (3, 60, False), (2, 192, True)])
+def test_float64_entry_points(config, n_atoms, collapse):
+    """e3j_conv_fwd_f64 / e3j_conv_bwd_f64 against the oracle at float64 accuracy (the oracle promotes the same
+    float32-representable inputs): 1e-12 of each irreducible block's largest value; two runs give the same bits."""
+    flags = e3j.E3J_PLAN_COLLAPSE_OUTPUTS if collapse else 0
+    wl, plan, cp, x, y, w, g = make_case(config, n_atoms, flags=flags)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    if collapse:
+        R, offs = oconv.collapse_matrix(cp)
+        g = g[:, :R.shape[0]].copy()
+        ref = oconv.conv_fwd_collapsed(cp, x, y, w, wl.senders, wl.receivers)
+        rx, ry, rw = oconv.conv_bwd_collapsed(cp, x, y, w, wl.senders, wl.receivers, g)
+        out_blocks = sorted({(off, off + 2 * p.L + 1) for p, off in zip(cp.paths, offs)})
+    else:
+        ref = oconv.conv_fwd(cp, x, y, w, wl.senders, wl.receivers)
+        rx, ry, rw = oconv.conv_bwd(cp, x, y, w, wl.senders, wl.receivers, g)
+        out_blocks = blocks_of_paths(cp.paths, "out")
+    d = [_cuda(a.astype(np.float64)) for a in (x, y, w, g)]
+    runs = []
+    for _ in range(2):
+        out = e3j.e3j_conv_fwd_f64(plan, d[0], d[1], d[2], snd, rcv)
+        runs.append((out, *e3j.e3j_conv_bwd_f64(plan, d[0], d[1], d[2], snd, rcv, d[3])))
+    torch.cuda.synchronize()
+    for a, b in zip(*runs):
+        assert torch.equal(a, b)
+    out, gx, gy, gw = runs[0]
+    assert out.dtype == torch.float64
+    assert_blockwise_close(out.cpu().numpy(), ref, out_blocks, tol=1e-12, what="f64 out")
+    assert_blockwise_close(gx.cpu().numpy(), rx, blocks_of_paths(cp.paths, "x"), tol=1e-12, what="f64 grad_x")
+    assert_blockwise_close(gy.cpu().numpy(), ry, blocks_of_paths(cp.paths, "sh"), tol=1e-12, what="f64 grad_sh")
+    assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), tol=1e-12, what="f64 grad_w")
