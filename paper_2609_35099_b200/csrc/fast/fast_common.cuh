@@ -39,6 +39,29 @@ __device__ __forceinline__ void vfma(float4& acc, const float4 a, const float4 b
 __device__ __forceinline__ void vfma(float2& acc, const float2 a, const float2 b) {
     acc.x = fmaf(a.x, b.x, acc.x); acc.y = fmaf(a.y, b.y, acc.y);
 }
+// Two channels per instruction: the packed single-precision multiply / fused multiply-add of sm_100 (one issue
+// slot for two IEEE operations, bit-identical to the scalar forms).
+__device__ __forceinline__ float2 pmul(const float2 a, const float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float4 pmul(const float4 a, const float4 b) {
+    const float2 lo = __fmul2_rn(make_float2(a.x, a.y), make_float2(b.x, b.y));
+    const float2 hi = __fmul2_rn(make_float2(a.z, a.w), make_float2(b.z, b.w));
+    return make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+__device__ __forceinline__ void pfma(float2& acc, const float2 a, const float2 b) { acc = __ffma2_rn(a, b, acc); }
+__device__ __forceinline__ void pfma(float2& acc, const float a, const float2 b) { acc = __ffma2_rn(make_float2(a, a), b, acc); }
+__device__ __forceinline__ void pfma(float4& acc, const float4 a, const float4 b) {
+    const float2 lo = __ffma2_rn(make_float2(a.x, a.y), make_float2(b.x, b.y), make_float2(acc.x, acc.y));
+    const float2 hi = __ffma2_rn(make_float2(a.z, a.w), make_float2(b.z, b.w), make_float2(acc.z, acc.w));
+    acc = make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+__device__ __forceinline__ void pfma(float4& acc, const float a, const float4 b) {
+    const float2 aa = make_float2(a, a);
+    const float2 lo = __ffma2_rn(aa, make_float2(b.x, b.y), make_float2(acc.x, acc.y));
+    const float2 hi = __ffma2_rn(aa, make_float2(b.z, b.w), make_float2(acc.z, acc.w));
+    acc = make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+__device__ __forceinline__ float pmul(const float a, const float b) { return a * b; }
+__device__ __forceinline__ void pfma(float& acc, const float a, const float b) { acc = fmaf(a, b, acc); }
 // sum over the lane's channels of a * b
 __device__ __forceinline__ float vdot(const float4 a, const float4 b) {
     return fmaf(a.w, b.w, fmaf(a.z, b.z, fmaf(a.y, b.y, a.x * b.x)));

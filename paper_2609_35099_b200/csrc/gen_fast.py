@@ -157,6 +157,16 @@ class Sig:
             if k not in self.row_paths[i0]:
                 self.row_paths[i0].append(k)
 
+    # Bodies whose multiplies and fused multiply-adds are emitted in the packed two-channel form (pfma / pmul of
+    # fast_common.cuh).  Measured on the 128-channel water signature: the forward-shaped bodies and the double
+    # backward gain (fewer issue slots), the first backward's edge body loses (more registers, it is bound by
+    # memory), so it stays scalar unless the signature's "PK" list names it.
+    PACKED_DEFAULT = ("fwd", "fwd2", "rfwd", "bwd2")
+
+    def ops(self, kind):
+        packed = kind in self.cfg.get("PK", self.PACKED_DEFAULT)
+        return ("pfma", "pmul") if packed else ("vfma", "vmul")
+
     def path_rows(self, k):
         p = self.paths[k]
         return range(p["out_off"], p["out_off"] + 2 * p["L"] + 1)
@@ -336,7 +346,7 @@ class Sig:
                 used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
                 o.append(f"            const BVec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
                 for i1 in used:
-                    o.append(f"            const BVec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                    F, M = self.ops("bwd"); o.append(f"            const BVec sx{k}_{i1} = {M}(s{k}, x{i1});")
                     o.append(f"            BVec u{k}_{i1}; vzero(u{k}_{i1});")
                 depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
                 for j in range(depth):
@@ -351,7 +361,7 @@ class Sig:
                             o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
                         i1 = self.pairs[pi][1]
                         r = local[row]
-                        o.append(f"            vfma(u{k}_{i1}, a{q}.{lane}, dm[{r}]);")
+                        F, M = self.ops("bwd"); o.append(f"            {F}(u{k}_{i1}, a{q}.{lane}, dm[{r}]);")
                         o.append(f"            {{ const float t = vdot(sx{k}_{i1}, dm[{r}]);")
                         for i2, c in self.pairs[pi][3]:
                             if i2 in dy_touched:
@@ -361,16 +371,16 @@ class Sig:
                                 o.append(f"              dyl[{i2}] = {fmt_float(c)} * t;")
                         o.append("            }")
                 first = used[0]
-                o.append(f"            BVec ds{k} = vmul(x{first}, u{k}_{first});")
+                F, M = self.ops("bwd"); o.append(f"            BVec ds{k} = {M}(x{first}, u{k}_{first});")
                 for i1 in used[1:]:
-                    o.append(f"            vfma(ds{k}, x{i1}, u{k}_{i1});")
+                    F, M = self.ops("bwd"); o.append(f"            {F}(ds{k}, x{i1}, u{k}_{i1});")
                 o.append(f"            gw[{k} * NQV] = ds{k};")
                 for i1 in used:
                     if i1 in dx_touched:
-                        o.append(f"            vfma(dxp[{i1}], s{k}, u{k}_{i1});")
+                        F, M = self.ops("bwd"); o.append(f"            {F}(dxp[{i1}], s{k}, u{k}_{i1});")
                     else:
                         dx_touched.add(i1)
-                        o.append(f"            dxp[{i1}] = vmul(s{k}, u{k}_{i1});")
+                        F, M = self.ops("bwd"); o.append(f"            dxp[{i1}] = {M}(s{k}, u{k}_{i1});")
             # entries this group never touches
             for i1 in range(self.DIN):
                 if i1 not in dx_touched:
@@ -410,7 +420,7 @@ class Sig:
             used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
             o.append(f"        const EVec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
             for i1 in used:
-                o.append(f"        const EVec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                F, M = self.ops("bwd"); o.append(f"        const EVec sx{k}_{i1} = {M}(s{k}, x{i1});")
                 o.append(f"        EVec u{k}_{i1}; vzero(u{k}_{i1});")
             depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
             have = set()
@@ -428,7 +438,7 @@ class Sig:
                         loaded_a.add(q)
                         o.append(f"        const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
                     i1 = self.pairs[pi][1]
-                    o.append(f"        vfma(u{k}_{i1}, a{q}.{lane}, d{k}_{row});")
+                    F, M = self.ops("bwd"); o.append(f"        {F}(u{k}_{i1}, a{q}.{lane}, d{k}_{row});")
                     o.append(f"        {{ const float t = vdot(sx{k}_{i1}, d{k}_{row});")
                     for i2, c in self.pairs[pi][3]:
                         if i2 in dy_touched:
@@ -438,16 +448,16 @@ class Sig:
                             o.append(f"          dyl[{i2}] = {fmt_float(c)} * t;")
                     o.append("        }")
             first = used[0]
-            o.append(f"        EVec ds{k} = vmul(x{first}, u{k}_{first});")
+            F, M = self.ops("bwd"); o.append(f"        EVec ds{k} = {M}(x{first}, u{k}_{first});")
             for i1 in used[1:]:
-                o.append(f"        vfma(ds{k}, x{i1}, u{k}_{i1});")
+                F, M = self.ops("bwd"); o.append(f"        {F}(ds{k}, x{i1}, u{k}_{i1});")
             o.append(f"        gw[{k} * NQV] = ds{k};")
             for i1 in used:
                 if i1 in dx_touched:
-                    o.append(f"        vfma(dxp[{i1}], s{k}, u{k}_{i1});")
+                    F, M = self.ops("bwd"); o.append(f"        {F}(dxp[{i1}], s{k}, u{k}_{i1});")
                 else:
                     dx_touched.add(i1)
-                    o.append(f"        dxp[{i1}] = vmul(s{k}, u{k}_{i1});")
+                    F, M = self.ops("bwd"); o.append(f"        dxp[{i1}] = {M}(s{k}, u{k}_{i1});")
         for i1 in range(self.DIN):
             if i1 not in dx_touched:
                 o.append(f"        vzero(dxp[{i1}]);")
@@ -480,7 +490,7 @@ class Sig:
             o.append(f"        const DVec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
             o.append(f"        const DVec us{k} = uss[{k} * NQV];")
             for i1 in used:
-                o.append(f"        DVec sxu{k}_{i1} = vmul(s{k}, ux{i1}); vfma(sxu{k}_{i1}, us{k}, x{i1});")
+                F, M = self.ops("bwd2"); o.append(f"        DVec sxu{k}_{i1} = {M}(s{k}, ux{i1}); {F}(sxu{k}_{i1}, us{k}, x{i1});")
                 o.append(f"        DVec v{k}_{i1}; vzero(v{k}_{i1});")
                 o.append(f"        DVec w{k}_{i1}; vzero(w{k}_{i1});")
             depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
@@ -500,8 +510,8 @@ class Sig:
                         o.append(f"        const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
                         o.append(f"        const float4 b{q} = *reinterpret_cast<const float4*>(Bs + {4 * q});")
                     i1 = self.pairs[pi][1]
-                    o.append(f"        vfma(v{k}_{i1}, a{q}.{lane}, d{k}_{row});")
-                    o.append(f"        vfma(w{k}_{i1}, b{q}.{lane}, d{k}_{row});")
+                    F, M = self.ops("bwd2"); o.append(f"        {F}(v{k}_{i1}, a{q}.{lane}, d{k}_{row});")
+                    F, M = self.ops("bwd2"); o.append(f"        {F}(w{k}_{i1}, b{q}.{lane}, d{k}_{row});")
                     o.append(f"        {{ const float t = vdot(sxu{k}_{i1}, d{k}_{row});")
                     for i2, c in self.pairs[pi][3]:
                         if i2 in dy_touched:
@@ -511,16 +521,16 @@ class Sig:
                             o.append(f"          dyl[{i2}] = {fmt_float(c)} * t;")
                     o.append("        }")
             first = used[0]
-            o.append(f"        DVec ds{k} = vmul(ux{first}, v{k}_{first}); vfma(ds{k}, x{first}, w{k}_{first});")
+            F, M = self.ops("bwd2"); o.append(f"        DVec ds{k} = {M}(ux{first}, v{k}_{first}); {F}(ds{k}, x{first}, w{k}_{first});")
             for i1 in used[1:]:
-                o.append(f"        vfma(ds{k}, ux{i1}, v{k}_{i1}); vfma(ds{k}, x{i1}, w{k}_{i1});")
+                F, M = self.ops("bwd2"); o.append(f"        {F}(ds{k}, ux{i1}, v{k}_{i1}); {F}(ds{k}, x{i1}, w{k}_{i1});")
             o.append(f"        gw[{k} * NQV] = ds{k};")
             for i1 in used:
                 if i1 in dx_touched:
-                    o.append(f"        vfma(dxp[{i1}], us{k}, v{k}_{i1}); vfma(dxp[{i1}], s{k}, w{k}_{i1});")
+                    F, M = self.ops("bwd2"); o.append(f"        {F}(dxp[{i1}], us{k}, v{k}_{i1}); {F}(dxp[{i1}], s{k}, w{k}_{i1});")
                 else:
                     dx_touched.add(i1)
-                    o.append(f"        dxp[{i1}] = vmul(us{k}, v{k}_{i1}); vfma(dxp[{i1}], s{k}, w{k}_{i1});")
+                    F, M = self.ops("bwd2"); o.append(f"        dxp[{i1}] = {M}(us{k}, v{k}_{i1}); {F}(dxp[{i1}], s{k}, w{k}_{i1});")
         for i1 in range(self.DIN):
             if i1 not in dx_touched:
                 o.append(f"        vzero(dxp[{i1}]);")
@@ -567,7 +577,7 @@ class Sig:
                 o.append(f"            const Vec s{k} = ss[{k} * NQV];")
                 used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
                 for i1 in used:
-                    o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                    F, M = self.ops("rfwd"); o.append(f"            const Vec sx{k}_{i1} = {M}(s{k}, x{i1});")
                 depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
                 for j in range(depth):
                     for row in prow:
@@ -580,7 +590,7 @@ class Sig:
                             loaded_a.add(q)
                             o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
                         i1 = self.pairs[pi][1]
-                        o.append(f"            vfma(acc[{row - bounds[g]}], a{q}.{lane}, sx{k}_{i1});")
+                        F, M = self.ops("rfwd"); o.append(f"            {F}(acc[{row - bounds[g]}], a{q}.{lane}, sx{k}_{i1});")
             o.append("        }")
         o.append("    }")
         o.append(f"    template <int G, class VecT>")
@@ -703,7 +713,7 @@ class Sig:
                 o.append(f"            const Vec s{k} = ss[{k} * NQV];  // path {k}: l1={p['l1']} l2={p['l2']} -> L={p['L']}")
                 used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
                 for i1 in used:
-                    o.append(f"            const Vec sx{k}_{i1} = vmul(s{k}, x{i1});")
+                    F, M = self.ops("fwd"); o.append(f"            const Vec sx{k}_{i1} = {M}(s{k}, x{i1});")
                 # round-robin over the rows of the path so that consecutive FMAs hit different accumulators
                 depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
                 for j in range(depth):
@@ -717,7 +727,7 @@ class Sig:
                             loaded_a.add(q)
                             o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
                         i1 = self.pairs[pi][1]
-                        o.append(f"            vfma(acc[{row - bounds[g]}], a{q}.{lane}, sx{k}_{i1});")
+                        F, M = self.ops("fwd"); o.append(f"            {F}(acc[{row - bounds[g]}], a{q}.{lane}, sx{k}_{i1});")
             o.append("        }")
         o.append("    }")
 
@@ -748,8 +758,8 @@ class Sig:
                     o.append(f"            const DFVec us{k} = uss[{k} * NQV];")
                     used = sorted({self.pairs[pi][1] for r2 in prow for pi in self.pairs_of(r2, k)})
                     for i1 in used:
-                        o.append(f"            const DFVec sx{k}_{i1} = vmul(s{k}, x{i1});")
-                        o.append(f"            DFVec sxu{k}_{i1} = vmul(s{k}, ux{i1}); vfma(sxu{k}_{i1}, us{k}, x{i1});")
+                        F, M = self.ops("fwd2"); o.append(f"            const DFVec sx{k}_{i1} = {M}(s{k}, x{i1});")
+                        F, M = self.ops("fwd2"); o.append(f"            DFVec sxu{k}_{i1} = {M}(s{k}, ux{i1}); {F}(sxu{k}_{i1}, us{k}, x{i1});")
                     depth = max(len(self.pairs_of(r2, k)) for r2 in prow)
                     for j in range(depth):
                         for row in prow:
@@ -763,8 +773,8 @@ class Sig:
                                 o.append(f"            const float4 a{q} = *reinterpret_cast<const float4*>(As + {4 * q});")
                                 o.append(f"            const float4 b{q} = *reinterpret_cast<const float4*>(Bs + {4 * q});")
                             i1 = self.pairs[pi][1]
-                            o.append(f"            vfma(acc[{row - bounds[g]}], a{q}.{lane}, sxu{k}_{i1});")
-                            o.append(f"            vfma(acc[{row - bounds[g]}], b{q}.{lane}, sx{k}_{i1});")
+                            F, M = self.ops("fwd2"); o.append(f"            {F}(acc[{row - bounds[g]}], a{q}.{lane}, sxu{k}_{i1});")
+                            F, M = self.ops("fwd2"); o.append(f"            {F}(acc[{row - bounds[g]}], b{q}.{lane}, sx{k}_{i1});")
                 o.append("        }")
             o.append("    }")
 

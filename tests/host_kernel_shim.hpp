@@ -36,6 +36,9 @@ inline void vfma(float4& acc, const float4 a, const float4 b) {
 }
 inline void vfma(float2& acc, const float2 a, const float2 b) { acc.x = fmaf(a.x, b.x, acc.x); acc.y = fmaf(a.y, b.y, acc.y); }
 inline void vfma(float& acc, const float a, const float b) { acc = fmaf(a, b, acc); }
+// the packed forms of the device code compute the same IEEE operations
+template <class A, class B> inline auto pmul(const A a, const B b) { return vmul(a, b); }
+template <class V, class A, class B> inline void pfma(V& acc, const A a, const B b) { vfma(acc, a, b); }
 inline float vdot(const float4 a, const float4 b) { return fmaf(a.w, b.w, fmaf(a.z, b.z, fmaf(a.y, b.y, a.x * b.x))); }
 inline float vdot(const float2 a, const float2 b) { return fmaf(a.y, b.y, a.x * b.x); }
 inline float vdot(const float a, const float b) { return a * b; }
