@@ -30,17 +30,21 @@ __global__ void layer_sum_kernel(int n_ranges, int64_t n_elems, const float* __r
 namespace {
 
 template <class Prob>
-int launch_gemm(const Prob& prob, dim3 grid, cudaStream_t st) {
+int launch_gemm(const Prob& prob, dim3 grid, cudaStream_t st, int resident_chunks = 0) {
     using L = GemmSmem<Prob::N>;
     static_assert(L::total <= 227 * 1024, "stage ring does not fit in shared memory");
+    static_assert(L::res_total(kMaxResidentChunks) <= 227 * 1024, "resident operand does not fit in shared memory");
+    constexpr bool kResident = ProbTraits<Prob>::A_RESIDENT;
+    constexpr size_t most = kResident ? L::res_total(kMaxResidentChunks) : L::total;
     static thread_local int attr_dev = -1;
     int dev = 0;
     E3J_CUDA_TRY(cudaGetDevice(&dev));
     if (attr_dev != dev) {
-        E3J_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32x3_kernel<Prob>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::total));
+        E3J_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32x3_kernel<Prob>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most));
         attr_dev = dev;
     }
-    gemm_tf32x3_kernel<Prob><<<grid, kGemmThreads, L::total, st>>>(prob);
+    const size_t bytes = kResident ? L::res_total(resident_chunks) : L::total;
+    gemm_tf32x3_kernel<Prob><<<grid, kGemmThreads, bytes, st>>>(prob);
     return after_launch();
 }
 
@@ -62,7 +66,13 @@ int radial_weights(int64_t n_edges, int H, int C, const float* h, const float* W
     RadialWeights p{};
     p.h = h; p.W = W; p.s = s; p.n_edges = n_edges; p.H = H; p.C = C; p.status = status;
     p.chunk = round_up((n_edges + n_ranges - 1) / n_ranges, 128);
-    return launch_gemm(p, dim3(n_cb, n_ranges), st);
+    const int chunks = (H + kChunkK - 1) / kChunkK;
+    if (chunks > kMaxResidentChunks) {   // a wide hidden layer: W^T converted per tile like the other operand
+        RadialWeightsWide q{};
+        static_cast<RadialWeights&>(q) = p;
+        return launch_gemm(q, dim3(n_cb, n_ranges), st);
+    }
+    return launch_gemm(p, dim3(n_cb, n_ranges), st, chunks);
 }
 
 int grad_hidden(int64_t n_edges, int H, int C, const float* gs, const float* W, float* gh, int32_t* status,

@@ -33,7 +33,8 @@ constexpr int kChunkK = 32;      // k per shared-memory stage (four tcgen05.mma 
 constexpr int kStages = 3;
 constexpr int kGroupChunks = 8;  // K chunks accumulated inside tensor memory before the tile is read out
 constexpr int kConvWarps = 8;     // converter warps
-constexpr int kPrefetch = 2;      // chunks of loads in flight per converter thread
+constexpr int kPrefetch = 2;      // chunks of loads in flight per converter thread (Prob::PREFETCH where given)
+constexpr int kMaxResidentChunks = 4;   // K chunks of a resident A operand (Prob::A_RESIDENT): K <= 128
 constexpr int kGemmThreads = (4 + kConvWarps + 1) * 32;   // epilogue, converters, tensor-core issue
 
 template <int N>
@@ -41,11 +42,23 @@ struct GemmSmem {
     static constexpr size_t a_bytes = (size_t)kTileM * kChunkK * 4;   // one of hi / lo
     static constexpr size_t b_bytes = (size_t)N * kChunkK * 4;
     static constexpr size_t stage_bytes = 2 * a_bytes + 2 * b_bytes;  // A_hi, A_lo, B_hi, B_lo
-    static constexpr size_t off_bar = 0;       // stage_full[kStages], stage_empty[kStages], d_full[2], d_empty[2], drain
-    static constexpr size_t off_tmem = 8 * (2 * kStages + 5);
+    static constexpr size_t off_bar = 0;       // stage_full[kStages], stage_empty[kStages], d_full[2], d_empty[2], drain, a_ready
+    static constexpr size_t off_tmem = 8 * (2 * kStages + 6);
     static constexpr size_t off_abort = off_tmem + 4;
     static constexpr size_t off_stage = 1024;
     static constexpr size_t total = off_stage + kStages * stage_bytes;
+    // A operand resident (converted once per CTA): [chunks][A_hi, A_lo] first, then stages of B alone
+    static constexpr size_t res_stage_bytes = 2 * b_bytes;
+    static constexpr size_t res_total(int chunks) { return off_stage + (size_t)chunks * 2 * a_bytes + kStages * res_stage_bytes; }
+};
+
+template <class P, class = void> struct ProbTraits {
+    static constexpr bool A_RESIDENT = false;
+    static constexpr int PREFETCH = kPrefetch;
+};
+template <class P> struct ProbTraits<P, decltype((void)P::A_RESIDENT)> {
+    static constexpr bool A_RESIDENT = P::A_RESIDENT;
+    static constexpr int PREFETCH = P::PREFETCH;
 };
 
 // Converters: an operand of a stage is rows [0, ROWS) x k [0, 32).  LANE_ROWS = 8: a warp item is 8 rows x 4 k-quads
@@ -103,6 +116,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
     uint64_t* d_full = stage_empty + kStages;
     uint64_t* d_empty = d_full + 2;
     uint64_t* drain = d_empty + 2;
+    uint64_t* a_ready = drain + 1;
+    constexpr bool kResident = ProbTraits<Prob>::A_RESIDENT;   // A does not depend on the tile: converted once
+    constexpr int kPre = ProbTraits<Prob>::PREFETCH;
+    const int res_chunks = kResident ? prob.n_chunks(0) : 0;
+    unsigned char* const stages = smem + L::off_stage + (size_t)res_chunks * 2 * L::a_bytes;
+    constexpr size_t kStageBytes = kResident ? L::res_stage_bytes : L::stage_bytes;
+    constexpr size_t kStageB = kResident ? 0 : 2 * L::a_bytes;   // where B_hi starts inside a stage
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::off_tmem);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -111,6 +131,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
         for (int s = 0; s < kStages; ++s) { fast::mbar_init(&stage_full[s], kConvWarps); fast::mbar_init(&stage_empty[s], 1); }
         for (int b = 0; b < 2; ++b) { fast::mbar_init(&d_full[b], 1); fast::mbar_init(&d_empty[b], 4); }
         fast::mbar_init(drain, 1);
+        fast::mbar_init(a_ready, kConvWarps);
         *abort_flag = 0;
         fast::mbar_fence_init();
     }
@@ -156,34 +177,45 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
         const int cwarp = warp - 4;
         // kPrefetch chunks of loads are in flight per thread: chunk i is converted while the loads of chunks
         // i + 1 .. i + kPrefetch - 1 travel (one global-memory latency per chunk would otherwise bound the kernel)
-        float4 va[kPrefetch][OA::NI], vb[kPrefetch][OB::NI];
+        if constexpr (kResident) {
+            for (int kc = 0; kc < res_chunks; ++kc) {
+                float4 a[OA::NI];
+                OA::load(a, cwarp, lane, [&](int row, int k) { return prob.load_a(0, kc, row, k); });
+                unsigned char* ra = smem + L::off_stage + (size_t)kc * 2 * L::a_bytes;
+                OA::store(a, ra, ra + L::a_bytes, cwarp, lane);
+            }
+            umma::fence_smem_to_async();
+            __syncwarp();
+            if (lane == 0) fast::mbar_arrive(a_ready);
+        }
+        float4 va[kPre][kResident ? 1 : OA::NI], vb[kPre][OB::NI];
         int tf = 0, kf = 0;                      // next chunk to fetch
         int ts = 0, ks = 0;                      // next chunk to convert and store
-        auto fetch = [&](float4 (&a)[OA::NI], float4 (&b)[OB::NI]) {
+        auto fetch = [&](float4 (&a)[kResident ? 1 : OA::NI], float4 (&b)[OB::NI]) {
             if (tf >= n_tiles) return;
             const int tt = tf, kk = kf;
-            OA::load(a, cwarp, lane, [&](int row, int k) { return prob.load_a(tt, kk, row, k); });
+            if constexpr (!kResident) OA::load(a, cwarp, lane, [&](int row, int k) { return prob.load_a(tt, kk, row, k); });
             OB::load(b, cwarp, lane, [&](int row, int k) { return prob.load_b(tt, kk, row, k); });
             if (++kf == prob.n_chunks(tf)) { kf = 0; ++tf; }
         };
 #pragma unroll
-        for (int u = 0; u < kPrefetch; ++u) fetch(va[u], vb[u]);
+        for (int u = 0; u < kPre; ++u) fetch(va[u], vb[u]);
         bool ok = true;
 #pragma unroll 1
-        for (int it0 = 0; ok && ts < n_tiles; it0 += kPrefetch) {
+        for (int it0 = 0; ok && ts < n_tiles; it0 += kPre) {
 #pragma unroll
-            for (int u = 0; u < kPrefetch; ++u) {
+            for (int u = 0; u < kPre; ++u) {
                 if (!ok || ts >= n_tiles) break;
                 const int it = it0 + u, s = it % kStages;
                 if (it >= kStages && !fast::mbar_wait(&stage_empty[s], ((it / kStages) + 1) & 1, abort_flag, prob.status)) { ok = false; break; }
-                unsigned char* st = smem + L::off_stage + (size_t)s * L::stage_bytes;
-                OA::store(va[u], st, st + L::a_bytes, cwarp, lane);
-                OB::store(vb[u], st + 2 * L::a_bytes, st + 2 * L::a_bytes + L::b_bytes, cwarp, lane);
+                unsigned char* st = stages + (size_t)s * kStageBytes;
+                if constexpr (!kResident) OA::store(va[u], st, st + L::a_bytes, cwarp, lane);
+                OB::store(vb[u], st + kStageB, st + kStageB + L::b_bytes, cwarp, lane);
                 umma::fence_smem_to_async();
                 __syncwarp();
                 if (lane == 0) fast::mbar_arrive(&stage_full[s]);
                 if (++ks == prob.n_chunks(ts)) { ks = 0; ++ts; }
-                fetch(va[u], vb[u]);             // refill this register set with the chunk kPrefetch ahead
+                fetch(va[u], vb[u]);             // refill this register set with the chunk kPre ahead
             }
         }
     } else {
@@ -192,6 +224,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
         const uint32_t sbo = umma::sbo_bytes(kChunkK);
         int it = 0;
         bool ok = true;
+        if (kResident && n_tiles > 0 && !fast::mbar_wait(a_ready, 0, abort_flag, prob.status)) ok = false;
         for (int t = 0; ok && t < n_tiles; ++t) {
             const int db = t & 1;
             const int n_chunks = prob.n_chunks(t);
@@ -201,9 +234,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
                 if (!fast::mbar_wait(&stage_full[s], (it / kStages) & 1, abort_flag, prob.status)) { ok = false; break; }
                 umma::fence_after_sync();
                 if (lane == 0) {
-                    const uint32_t a_hi = umma::smem_addr(smem + L::off_stage + (size_t)s * L::stage_bytes);
+                    const uint32_t st = umma::smem_addr(stages + (size_t)s * kStageBytes);
+                    const uint32_t a_hi = kResident ? umma::smem_addr(smem + L::off_stage + (size_t)kc * 2 * L::a_bytes) : st;
                     const uint32_t a_lo = a_hi + (uint32_t)L::a_bytes;
-                    const uint32_t b_hi = a_hi + 2 * (uint32_t)L::a_bytes, b_lo = b_hi + (uint32_t)L::b_bytes;
+                    const uint32_t b_hi = st + (uint32_t)kStageB, b_lo = b_hi + (uint32_t)L::b_bytes;
                     const uint32_t d = tmem_base + (uint32_t)(db * N);
                     // small terms first: a_lo b_hi, a_hi b_lo, then a_hi b_hi
                     const uint32_t pa[3] = {a_lo, a_hi, a_hi}, pb[3] = {b_hi, b_lo, b_hi};
@@ -239,6 +273,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
 struct RadialWeights {
     static constexpr int N = 128, A_LANE_ROWS = 32, B_LANE_ROWS = 8;
     static constexpr bool ACCUMULATE = false;   // k = hidden is short: one chain per tile
+    static constexpr bool A_RESIDENT = true;    // the CTA's block of W^T serves all of its tiles
+    static constexpr int PREFETCH = 4;          // two tiles of h in flight per converter thread
     __device__ __forceinline__ bool flush(int) const { return true; }
     const float* h; const float* W; float* s;
     int64_t n_edges, chunk;   // chunk: edges per CTA row of the grid (multiple of 128)
@@ -282,6 +318,12 @@ struct RadialWeights {
                 if (e0 + i < e_end) dst[(size_t)i * C] = v[i];
         }
     }
+};
+
+// the same product for hidden widths beyond kMaxResidentChunks * 32: both operands converted per tile
+struct RadialWeightsWide : RadialWeights {
+    static constexpr bool A_RESIDENT = false;
+    static constexpr int PREFETCH = kPrefetch;
 };
 
 // grad_h[e, j] = sum_c grad_s[e, c] W[j, c]: tile = 128 edges x (64 j, block blockIdx.y); m = edge, n = j, k = c.
