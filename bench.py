@@ -49,13 +49,13 @@ def measured_peak():
 # profiles/fast_fwd_kernel_water3000.txt, profiles/fast_bwd1_kernel_water3000.txt and the launch-list run
 # (specialised kernels, workload water3000).  Other workloads / the generic kernels report null.
 NCU_TRAFFIC = {
-    ("water3000", "fwd"): 1.109031e9 + 0.083995e9 + 0.016343e9,          # fast_fwd_kernel + fwd_fixup_kernel
+    ("water3000", "fwd"): 1.109735e9 + 0.085159e9 + 0.016343e9,          # fast_fwd_kernel + fwd_fixup_kernel
     ("water3000", "bwd"): 1.257002e9 + 1.362881e9 + 0.330463e9 + 0.0018e9,  # fast_bwd1_kernel + bwd_dx_reduce_kernel
 }
 # Where each term above is printed (file under profiles/, kernel, metric): tests/test_bench_traffic.py checks them.
 NCU_TRAFFIC_SOURCE = {
-    ("water3000", "fwd"): [("fast_fwd_kernel_water3000.txt", "fast_fwd_kernel", "dram__bytes_read.sum", 1.109031e9),
-                           ("fast_fwd_kernel_water3000.txt", "fast_fwd_kernel", "dram__bytes_write.sum", 0.083995e9),
+    ("water3000", "fwd"): [("fast_fwd_kernel_water3000.txt", "fast_fwd_kernel", "dram__bytes_read.sum", 1.109735e9),
+                           ("fast_fwd_kernel_water3000.txt", "fast_fwd_kernel", "dram__bytes_write.sum", 0.085159e9),
                            ("small_kernels_traffic_water3000.txt", "fwd_fixup_kernel", "total", 0.016343e9)],
     ("water3000", "bwd"): [("fast_bwd1_kernel_water3000.txt", "fast_bwd1_kernel", "dram__bytes_read.sum", 1.257002e9),
                            ("fast_bwd1_kernel_water3000.txt", "fast_bwd1_kernel", "dram__bytes_write.sum", 1.362881e9),
@@ -340,7 +340,8 @@ def main():
                     help="length of the extra back-to-back loop whose means and clocks go into `sustained` (0 = skip)")
     ap.add_argument("--fused-radial", action="store_true",
                     help="also time the convolution that takes the radial network's last layer (h, W) instead of the "
-                         "weights (after the steps, reported beside them)")
+                         "weights (after the steps, reported beside them); default for configs 2 and 3")
+    ap.add_argument("--no-radial", action="store_true", help="skip the radial-layer timings")
     ap.add_argument("--hidden", type=int, default=64, help="width of the radial network's last hidden layer")
     ap.add_argument("--shard", action="store_true",
                     help="one system sharded by receiver over the ranks (halo exchange of x and grad_x inside the step) "
@@ -515,7 +516,8 @@ def main():
     # the forward that forms them inside the kernel, beside the unfused form (tensor-core product into memory, then
     # the plain forward), and the backward (composed: product, convolution backward, two more products)
     radial = None
-    if args.fused_radial and not args.pad and not args.collapse and not args.generic:
+    want_radial = (args.fused_radial or args.config in (2, 3)) and not args.no_radial
+    if want_radial and not args.pad and not args.collapse and not args.generic:
         H = args.hidden
         gen = torch.Generator(device=dev); gen.manual_seed(12)
         hh = torch.randn((e, H), generator=gen, device=dev)

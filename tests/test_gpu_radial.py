@@ -37,6 +37,8 @@ def _cuda(a):
     ("128x0e+128x1o", 3, 300, 40),     # ragged second k chunk
     ("8x0e+8x1o", 2, 513, 64),         # 120 columns: one ragged column block
     ("64x0e+64x1o+64x2e+64x3o", 3, 260, 96),   # three k chunks
+    ("128x0e+128x1o", 3, 700, 128),    # four k chunks: the largest resident block of W^T
+    ("128x0e+128x1o", 3, 390, 160),    # five k chunks: W^T converted per tile (wide hidden layer)
     ("128x0e+128x1o", 3, 0, 64),
 ])
 def test_radial_weights_match_the_float64_product(irreps, lmax, edges, hidden):
