@@ -271,3 +271,30 @@ def conv_radial_bwd(cp: Coupling, x, y, h, W, senders, receivers, dm):
     dh = ds2 @ np.asarray(W, dtype=np.float64).T
     dW = np.asarray(h, dtype=np.float64).T @ ds2
     return dx, dy, dh, dW
+
+
+# ---------------------------------------------------------------------------------------------
+# Harmonics taken from the edge vectors.  The paper lists the harmonic embedding Y(r_ab / |r_ab|) of the
+# edge direction among the operations in scope and feeds it to the convolution as y; here the two are
+# composed: y is evaluated in float64 from the float32 vectors and rounded to float32, the precision it has
+# as an input of the convolution, and the backward continues the chain rule into the vectors.
+def _sh_lmax(cp: Coupling) -> int:
+    lmax = int(round(cp.dp ** 0.5)) - 1
+    assert (lmax + 1) ** 2 == cp.dp
+    return lmax
+
+
+def conv_vec_fwd(cp: Coupling, x, vec, s, senders, receivers) -> np.ndarray:
+    from . import sh
+    vec = np.ascontiguousarray(vec, dtype=np.float32)
+    y = sh.real_sh_all_of_vectors(_sh_lmax(cp), vec.astype(np.float64)).astype(np.float32)
+    return conv_fwd(cp, x, y, s, senders, receivers)
+
+
+def conv_vec_bwd(cp: Coupling, x, vec, s, senders, receivers, dm):
+    """(dx[N,d,N_q], dvec[E,3], ds[E,P,N_q]) in float64."""
+    from . import sh
+    vec = np.ascontiguousarray(vec, dtype=np.float32)
+    y = sh.real_sh_all_of_vectors(_sh_lmax(cp), vec.astype(np.float64)).astype(np.float32)
+    dx, dy, ds = conv_bwd(cp, x, y, s, senders, receivers, dm)
+    return dx, sh.real_sh_all_vjp(_sh_lmax(cp), vec.astype(np.float64), dy), ds

@@ -179,3 +179,66 @@ def test_workload_harmonics_match_the_oracle():
     u = _unit(200, 6)
     for lmax in range(4):
         assert np.allclose(workloads.spherical_harmonics(lmax, u), sh.real_sh_all(lmax, u), atol=1e-14)
+
+
+# ------------------------------------------------------------------ harmonics of edge vectors and their gradient
+def _vectors(n, seed):
+    rng = np.random.default_rng(seed)
+    return _unit(n, seed) * rng.uniform(0.7, 5.0, size=(n, 1))
+
+
+def test_sh_of_vectors_ignores_the_length():
+    v = _vectors(50, 7)
+    u = v / np.linalg.norm(v, axis=1, keepdims=True)
+    assert np.allclose(sh.real_sh_all_of_vectors(3, v), sh.real_sh_all(3, u), atol=1e-14)
+    assert np.allclose(sh.real_sh_all_of_vectors(3, 3.7 * v), sh.real_sh_all(3, u), atol=1e-13)
+    with pytest.raises(ValueError):
+        sh.real_sh_all_of_vectors(2, np.zeros((1, 3)))
+
+
+def test_sh_vjp_closed_forms_for_l1_and_l2():
+    """d/dv of sqrt(3) (y, z, x) / r and of sqrt(5)/2 (3 z^2 / r^2 - 1), written out by hand."""
+    v = _vectors(40, 8)
+    x, y, z = v.T
+    r = np.linalg.norm(v, axis=1)
+    g = np.random.default_rng(9).standard_normal((40, 9))
+    got = sh.real_sh_all_vjp(2, v, g)
+    # l = 1: Y = sqrt(3) (y, z, x) / r  ->  dY_a/dv_b = sqrt(3) (delta_ab / r - v_a v_b / r^3)
+    g1 = g[:, 1:4]                         # cotangents of (y, z, x) components
+    gv = np.stack([g1[:, 2], g1[:, 0], g1[:, 1]], axis=1)   # reordered to (x, y, z)
+    want = math.sqrt(3) * (gv / r[:, None] - v * np.einsum("ni,ni->n", gv, v)[:, None] / r[:, None] ** 3)
+    # l = 2, m = 0: Y = sqrt(5)/2 (3 z^2 / r^2 - 1)  ->  grad = sqrt(5)/2 * 3 * (2 z e_z / r^2 - 2 z^2 v / r^4)
+    ez = np.zeros_like(v); ez[:, 2] = 1.0
+    want += (g[:, 6] * math.sqrt(5) / 2 * 3)[:, None] * (2 * z[:, None] * ez / r[:, None] ** 2
+                                                          - 2 * (z ** 2)[:, None] * v / r[:, None] ** 4)
+    only = np.zeros_like(g); only[:, 1:4] = g[:, 1:4]; only[:, 6] = g[:, 6]
+    assert np.allclose(sh.real_sh_all_vjp(2, v, only), want, atol=1e-8)
+    # the other components contribute too: the full product differs from the partial one
+    assert np.abs(got - want).max() > 1e-3
+
+
+def test_sh_vjp_is_tangential_and_scales_inversely_with_the_length():
+    """Y depends on the direction only: v . grad = 0, and grad(c v) = grad(v) / c."""
+    v = _vectors(30, 10)
+    g = np.random.default_rng(11).standard_normal((30, 16))
+    gv = sh.real_sh_all_vjp(3, v, g)
+    assert np.abs(np.einsum("ni,ni->n", gv, v)).max() < 1e-7
+    assert np.allclose(sh.real_sh_all_vjp(3, 2.5 * v, g), gv / 2.5, atol=1e-8)
+    # Y_0 is constant
+    g0 = np.zeros_like(g); g0[:, 0] = 1.0
+    assert np.abs(sh.real_sh_all_vjp(3, v, g0)).max() < 1e-9
+
+
+def test_sh_vjp_agrees_with_the_rotation_generators():
+    """An infinitesimal rotation of v about axis a changes Y_l by the action of the real generator: checked through
+    the invariance of sum_m Y_lm(v) Y_lm(w) under a joint rotation, i.e. grad_v[Y(v).Y(w)] x v + grad_w[...] x w = 0."""
+    v, w = _vectors(20, 12), _vectors(20, 13)
+    for l in (1, 2, 3):
+        sl = slice(l * l, (l + 1) * (l + 1))
+        Yv, Yw = sh.real_sh_all_of_vectors(3, v), sh.real_sh_all_of_vectors(3, w)
+        gv_in, gw_in = np.zeros_like(Yv), np.zeros_like(Yw)
+        gv_in[:, sl], gw_in[:, sl] = Yw[:, sl], Yv[:, sl]
+        gv = sh.real_sh_all_vjp(3, v, gv_in)
+        gw = sh.real_sh_all_vjp(3, w, gw_in)
+        torque = np.cross(v, gv) + np.cross(w, gw)
+        assert np.abs(torque).max() < 1e-6

@@ -291,3 +291,32 @@ def test_double_backward_is_the_derivative_of_the_backward():
             plus[which][idx] += h; minus[which][idx] -= h
             fd = (phi(*plus) - phi(*minus)) / (2 * h)
             assert abs(fd - grad[idx]) <= 1e-9 * max(1.0, abs(fd)), (which, idx, fd, grad[idx])
+
+
+def test_conv_from_edge_vectors_backward_matches_a_directional_difference():
+    """conv_vec_bwd's dvec against central differences of sum(g * conv_vec_fwd) along a random direction; the
+    vectors sit on a binary grid so that vec +- h * delta is exact in float32 (the rounding of y to float32 inside
+    the forward leaves noise of about 1e-4 of the derivative)."""
+    rng = np.random.default_rng(21)
+    cp = conv.Coupling("4x0e+4x1o", 2)
+    n, e = 5, 14
+    snd = rng.integers(0, n, size=e).astype(np.int32)
+    rcv = np.sort(rng.integers(0, n, size=e)).astype(np.int32)
+    x = rng.standard_normal((n, cp.d, cp.nq)).astype(np.float32)
+    s = rng.standard_normal((e, cp.P, cp.nq)).astype(np.float32)
+    g = rng.standard_normal((n, cp.D, cp.nq)).astype(np.float32)
+    vec = (np.round(rng.uniform(-2, 2, size=(e, 3)) * 64) / 64).astype(np.float32)
+    vec[np.abs(vec).sum(axis=1) < 0.5] += 1.0
+    delta = rng.choice([-1.0, 1.0], size=(e, 3)).astype(np.float32)
+    h = 2.0 ** -8
+    phi = lambda v: float(np.sum(g.astype(np.float64) * conv.conv_vec_fwd(cp, x, v, s, snd, rcv)))
+    fd = (phi(vec + h * delta) - phi(vec - h * delta)) / (2 * h)
+    dx, dvec, ds = conv.conv_vec_bwd(cp, x, vec, s, snd, rcv, g)
+    assert abs(fd - float(np.sum(dvec * delta))) < 2e-3 * max(1.0, np.abs(dvec).sum())
+    # the other two cotangents are those of the convolution with the same harmonics
+    y = sh.real_sh_all_of_vectors(2, vec.astype(np.float64)).astype(np.float32)
+    dx2, _, ds2 = conv.conv_bwd(cp, x, y, s, snd, rcv, g)
+    assert np.array_equal(dx, dx2) and np.array_equal(ds, ds2)
+    # a vector's length does not matter to the forward
+    assert np.allclose(conv.conv_vec_fwd(cp, x, 2 * vec, s, snd, rcv), conv.conv_vec_fwd(cp, x, vec, s, snd, rcv),
+                       atol=1e-5)
