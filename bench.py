@@ -575,6 +575,40 @@ def main():
         }
         del ws_rf, ws_rb, w_mat, hh, WW, gh, gW
 
+    # ---- the convolution on edge vectors: harmonics formed in the kernel's table warp, beside the two-step form
+    vec_block = None
+    if want_radial and not args.pad and not args.collapse and not args.generic and plan.d_sh in (1, 4, 9, 16):
+        lmax = int(round(plan.d_sh ** 0.5)) - 1
+        vv = torch.from_numpy(wl.vectors.astype("float32")).to(dev)
+        ws_vf = torch.empty(max(e3j.e3j_conv_vec_fwd_workspace_bytes(plan, n, e), 256), dtype=torch.uint8, device=dev)
+        ws_vb = torch.empty(max(e3j.e3j_conv_vec_bwd_workspace_bytes(plan, n, e), 256), dtype=torch.uint8, device=dev)
+        y_buf, gv = torch.empty((e, plan.d_sh), device=dev), torch.empty((e, 3), device=dev)
+
+        def timed_v(fn, k):
+            for _ in range(3):
+                fn()
+            a, b = ev(), ev()
+            torch.cuda.synchronize()
+            a.record(stream)
+            for _ in range(k):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / k
+
+        k_v = max(3, min(args.steps, 50))
+        vec_block = {
+            "fwd_ms": timed_v(lambda: e3j.e3j_conv_vec_fwd(plan, d["x"], vv, d["w"], d["snd"], d["rcv"], rowptr, out=out,
+                                                           workspace=ws_vf), k_v),
+            "harmonics_fwd_ms": timed_v(lambda: e3j.e3j_harmonics_fwd(lmax, vv, out=y_buf), k_v),
+            "harmonics_bwd_ms": timed_v(lambda: e3j.e3j_harmonics_bwd(lmax, vv, d["y"], out=gv), k_v),
+            "bwd_ms": timed_v(lambda: e3j.e3j_conv_vec_bwd(plan, d["x"], vv, d["w"], d["snd"], d["rcv"], d["g"], rowptr, perm,
+                                                           colptr, grad_x=gx, grad_vec=gv, grad_w=gw, workspace=ws_vb), k_v),
+            "note": "fwd: harmonics formed inside the convolution kernel (specialised signatures); bwd: harmonics kernel, "
+                    "e3j_conv_bwd, harmonics gradient kernel",
+        }
+        del vv, ws_vf, ws_vb, y_buf, gv
+
     # ---- end to end: pinned host buffers in, results out, inside the timed region.  Every step copies its inputs
     # from pinned host memory and its four results back; the copies run on streams of their own with two sets
     # of device buffers, so that the transfers of neighbouring steps overlap each other and the kernels.
@@ -679,7 +713,7 @@ def main():
             # 20 % of the runs, as in its efficiency-comparison section), minimum and maximum
             "call_stats_ms": {"fwd": call_stats(fwd_ms), "bwd": call_stats(bwd_ms)},
             "outside_the_step_ms": {"plan_build_host": plan_build_ms, "graph_prepare_device": graph_prepare_ms},
-            "double_backward": dbl, "radial": radial, "sustained": sustained,
+            "double_backward": dbl, "radial": radial, "edge_vectors": vec_block, "sustained": sustained,
             "roofline": dominant, "roofline_fwd": roofs["fwd"], "roofline_bwd": roofs["bwd"],
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         }

@@ -303,6 +303,34 @@ int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
                const float* w, const float* grad_out, float* grad_x1, float* grad_x2,
                float* grad_w, void* stream);
 
+/* Harmonics of the edge vectors (paper, "Key Operations in Scope": the harmonic embedding Y(r_ab / |r_ab|) of the edge
+ * direction is what the convolution takes as sh).  Component normalisation (the squares of the 2l+1 components of a
+ * degree sum to 2l+1, Y_0 = 1), degrees stacked l = 0..lmax, m = -l..l inside a degree (l = 1: sqrt(3) (y, z, x)),
+ * lmax <= 3.  Device pointers: edge_vec [n_edges, 3] (r_receiver - r_sender, any length), sh / grad_sh
+ * [n_edges, (lmax+1)^2] (16-byte aligned), grad_vec [n_edges, 3]; outputs fully overwritten.  The gradient is that of the direction:
+ * orthogonal to the vector and proportional to 1 / |vec|.  A zero vector has no direction: its harmonics are the
+ * polynomials' values at the origin and its gradient is zero; callers should not pass one. */
+int e3j_harmonics_fwd(int lmax, int64_t n_edges, const float* edge_vec, float* sh, void* stream);
+int e3j_harmonics_bwd(int lmax, int64_t n_edges, const float* edge_vec, const float* grad_sh, float* grad_vec,
+                      void* stream);
+
+/* The convolution on edge vectors instead of harmonics: out = conv_fwd(x, Y(edge_vec), w), and the backward with the
+ * chain rule continued into the vectors (grad_vec [n_edges, 3] in place of grad_sh).  The plan's harmonics must be
+ * the full set l = 0..lmax, lmax <= 3 (else E3J_ERR_UNSUPPORTED).  Forward: plans with signature-specialised kernels
+ * form the harmonics inside the convolution kernel (no [n_edges, d'] array is read or written); other plans run
+ * e3j_harmonics_fwd into the workspace first.  Backward: composed (harmonics into the workspace, e3j_conv_bwd,
+ * e3j_harmonics_bwd).  Other arguments, alignment and determinism as for e3j_conv_fwd / e3j_conv_bwd; any of
+ * grad_x, grad_vec, grad_w may be NULL.  Workspace: 256-byte aligned, e3j_conv_vec_*_workspace_bytes(). */
+size_t e3j_conv_vec_fwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges);
+size_t e3j_conv_vec_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges);
+int e3j_conv_vec_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x, const float* edge_vec,
+                     const float* w, const int32_t* senders, const int32_t* receivers, const int32_t* rowptr,
+                     float* out, void* workspace, size_t workspace_bytes, void* stream);
+int e3j_conv_vec_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x, const float* edge_vec,
+                     const float* w, const int32_t* senders, const int32_t* receivers, const int32_t* rowptr,
+                     const int32_t* sender_perm, const int32_t* colptr, const float* grad_out, float* grad_x,
+                     float* grad_vec, float* grad_w, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Float64 convolution (paper, appendix on the benchmark setup: float64 builds of the kernels are shipped beside
  * the float32 ones).  Same operation, layouts, graph arguments and conventions as e3j_conv_fwd / e3j_conv_bwd with
  * every tensor in float64 and the coupling coefficients in float64 as the plan builder computed them.  Table-driven

@@ -25,7 +25,8 @@ __all__ = [
     "e3j_conv_bwd_bwd_workspace_bytes", "e3j_conv_bwd_bwd",
     "e3j_radial_weights", "e3j_conv_radial_fwd_workspace_bytes", "e3j_conv_radial_bwd_workspace_bytes",
     "e3j_conv_radial_fwd", "e3j_conv_radial_bwd",
-    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_conv_fwd_f64", "e3j_conv_bwd_f64", "e3j_shard_prepare", "e3j_rows_gather", "e3j_rows_add", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
+    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_harmonics_fwd", "e3j_harmonics_bwd", "e3j_conv_vec_fwd", "e3j_conv_vec_bwd",
+    "e3j_conv_vec_fwd_workspace_bytes", "e3j_conv_vec_bwd_workspace_bytes", "e3j_conv_fwd_f64", "e3j_conv_bwd_f64", "e3j_shard_prepare", "e3j_rows_gather", "e3j_rows_add", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
     "E3J_PLAN_COLLAPSE_OUTPUTS",
 ]
 
@@ -112,6 +113,17 @@ def _load():
     lib.e3j_conv_radial_bwd.restype = i32
     lib.e3j_tp_fwd.argtypes = [vp, i64] + [vp] * 5
     lib.e3j_tp_bwd.argtypes = [vp, i64] + [vp] * 8
+    lib.e3j_harmonics_fwd.argtypes = [i32, i64, vp, vp, vp]
+    lib.e3j_harmonics_fwd.restype = i32
+    lib.e3j_harmonics_bwd.argtypes = [i32, i64, vp, vp, vp, vp]
+    lib.e3j_harmonics_bwd.restype = i32
+    for name in ("e3j_conv_vec_fwd_workspace_bytes", "e3j_conv_vec_bwd_workspace_bytes"):
+        getattr(lib, name).argtypes = [vp, i64, i64]
+        getattr(lib, name).restype = sz
+    lib.e3j_conv_vec_fwd.argtypes = [vp, i64, i64] + [vp] * 8 + [sz, vp]
+    lib.e3j_conv_vec_fwd.restype = i32
+    lib.e3j_conv_vec_bwd.argtypes = [vp, i64, i64] + [vp] * 13 + [sz, vp]
+    lib.e3j_conv_vec_bwd.restype = i32
     lib.e3j_conv_f64_workspace_bytes.argtypes = [vp, i64, i64]
     lib.e3j_conv_f64_workspace_bytes.restype = sz
     lib.e3j_conv_fwd_f64.argtypes = [vp, i64, i64] + [vp] * 8 + [sz, vp]
@@ -531,6 +543,84 @@ def e3j_tp_bwd(plan: Plan, x1, x2, w, grad_out, grad_x1=True, grad_x2=True, grad
         _dev_ptr(grad_x1, f32, None, "grad_x1"), _dev_ptr(grad_x2, f32, None, "grad_x2"),
         _dev_ptr(grad_w, f32, None, "grad_w"), _stream(stream)), "e3j_tp_bwd")
     return grad_x1, grad_x2, grad_w
+
+
+def e3j_harmonics_fwd(lmax: int, edge_vec, out=None, stream=None):
+    """sh[E, (lmax+1)^2] = Y(edge_vec / |edge_vec|), component-normalised real harmonics."""
+    torch = _torch()
+    e, f32 = edge_vec.shape[0], torch.float32
+    if out is None:
+        out = torch.empty((e, (lmax + 1) ** 2), dtype=f32, device=edge_vec.device)
+    _check(_load().e3j_harmonics_fwd(lmax, e, _dev_ptr(edge_vec, f32, (e, 3), "edge_vec"),
+                                     _dev_ptr(out, f32, (e, (lmax + 1) ** 2), "sh"), _stream(stream)), "e3j_harmonics_fwd")
+    return out
+
+
+def e3j_harmonics_bwd(lmax: int, edge_vec, grad_sh, out=None, stream=None):
+    """grad_vec[E, 3] of e3j_harmonics_fwd."""
+    torch = _torch()
+    e, f32 = edge_vec.shape[0], torch.float32
+    if out is None:
+        out = torch.empty((e, 3), dtype=f32, device=edge_vec.device)
+    _check(_load().e3j_harmonics_bwd(lmax, e, _dev_ptr(edge_vec, f32, (e, 3), "edge_vec"),
+                                     _dev_ptr(grad_sh, f32, (e, (lmax + 1) ** 2), "grad_sh"),
+                                     _dev_ptr(out, f32, (e, 3), "grad_vec"), _stream(stream)), "e3j_harmonics_bwd")
+    return out
+
+
+def e3j_conv_vec_fwd_workspace_bytes(plan: Plan, n_nodes: int, n_edges: int) -> int:
+    return int(_load().e3j_conv_vec_fwd_workspace_bytes(plan.handle, n_nodes, n_edges))
+
+
+def e3j_conv_vec_bwd_workspace_bytes(plan: Plan, n_nodes: int, n_edges: int) -> int:
+    return int(_load().e3j_conv_vec_bwd_workspace_bytes(plan.handle, n_nodes, n_edges))
+
+
+def e3j_conv_vec_fwd(plan: Plan, x, edge_vec, w, senders, receivers, rowptr=None, out=None, workspace=None,
+                     stream=None):
+    """Forward convolution with the harmonics formed from the edge vectors [E, 3]."""
+    torch = _torch()
+    n, e = x.shape[0], senders.numel()
+    f32, i32 = torch.float32, torch.int32
+    if out is None:
+        out = torch.empty((n, plan.d_out, plan.n_channels), dtype=f32, device=x.device)
+    workspace = _workspace(e3j_conv_vec_fwd_workspace_bytes(plan, n, e), x, workspace)
+    _check(_load().e3j_conv_vec_fwd(
+        plan.handle, n, e, _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"),
+        _dev_ptr(edge_vec, f32, (e, 3), "edge_vec"), _dev_ptr(w, f32, (e, plan.n_paths, plan.n_channels), "w"),
+        _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
+        _dev_ptr(rowptr, i32, (n + 1,), "rowptr"), _dev_ptr(out, f32, (n, plan.d_out, plan.n_channels), "out"),
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_vec_fwd")
+    return out
+
+
+def e3j_conv_vec_bwd(plan: Plan, x, edge_vec, w, senders, receivers, grad_out, rowptr=None, sender_perm=None,
+                     colptr=None, grad_x=True, grad_vec=True, grad_w=True, workspace=None, stream=None):
+    """Returns (grad_x, grad_vec, grad_w); each grad_* argument is True (allocate), False/None or a tensor."""
+    torch = _torch()
+    n, e = x.shape[0], senders.numel()
+    f32, i32 = torch.float32, torch.int32
+
+    def alloc(flag, shape):
+        if flag is True:
+            return torch.empty(shape, dtype=f32, device=x.device)
+        return flag if isinstance(flag, torch.Tensor) else None
+
+    grad_x = alloc(grad_x, (n, plan.d_in, plan.n_channels))
+    grad_vec = alloc(grad_vec, (e, 3))
+    grad_w = alloc(grad_w, (e, plan.n_paths, plan.n_channels))
+    workspace = _workspace(e3j_conv_vec_bwd_workspace_bytes(plan, n, e), x, workspace)
+    _check(_load().e3j_conv_vec_bwd(
+        plan.handle, n, e, _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"),
+        _dev_ptr(edge_vec, f32, (e, 3), "edge_vec"), _dev_ptr(w, f32, (e, plan.n_paths, plan.n_channels), "w"),
+        _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
+        _dev_ptr(rowptr, i32, (n + 1,), "rowptr"), _dev_ptr(sender_perm, i32, (e,), "sender_perm"),
+        _dev_ptr(colptr, i32, (n + 1,), "colptr"),
+        _dev_ptr(grad_out, f32, (n, plan.d_out, plan.n_channels), "grad_out"),
+        _dev_ptr(grad_x, f32, (n, plan.d_in, plan.n_channels), "grad_x"), _dev_ptr(grad_vec, f32, (e, 3), "grad_vec"),
+        _dev_ptr(grad_w, f32, (e, plan.n_paths, plan.n_channels), "grad_w"),
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_vec_bwd")
+    return grad_x, grad_vec, grad_w
 
 
 def e3j_conv_fwd_f64(plan: Plan, x, sh, w, senders, receivers, rowptr=None, out=None, stream=None):

@@ -312,16 +312,22 @@ size_t e3j_conv_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64
 
 }  // extern "C"
 
+bool e3j::has_fast_forward(const e3j_plan* plan) {
+    const FastKernels* fk = fast_lookup(plan);
+    return fk && fk->conv_fwd;
+}
+
 int e3j::conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x,
                        const float* sh, const float* w, const int32_t* senders,
                        const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
-                       size_t workspace_bytes, void* stream, bool padded) {
+                       size_t workspace_bytes, void* stream, bool padded, const float* edge_vec) {
     if (!plan || n_nodes < 0 || n_edges < 0 || n_nodes >= (1ll << 31) - 1 || n_edges >= (1ll << 31) - 1)
         return E3J_ERR_INVALID_ARG;
     if (plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;  // the kernels work on groups of four channels
     if (n_nodes == 0) return E3J_OK;
     if (!out || !x) return E3J_ERR_INVALID_ARG;
-    if (n_edges > 0 && (!sh || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    if (n_edges > 0 && ((!sh && !edge_vec) || !w || !senders || !receivers)) return E3J_ERR_INVALID_ARG;
+    if (edge_vec && !has_fast_forward(plan)) return E3J_ERR_UNSUPPORTED;   // the table-driven kernel reads sh
     if (!aligned16({x, w, out})) return E3J_ERR_INVALID_ARG;
     if (padded && !rowptr) return E3J_ERR_INVALID_ARG;  // rowptr[n_nodes] is where the kernels learn the edge count
     const int32_t* n_real = padded ? rowptr + n_nodes : nullptr;
@@ -340,6 +346,7 @@ int e3j::conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, c
         a.workspace = ws + L.scratch; a.workspace_bytes = workspace_bytes - L.scratch; a.stream = st;
         a.status = t.status;
         a.n_real = n_real;
+        a.vec = edge_vec;
         return fk->conv_fwd(a);
     }
     if (!rowptr) {

@@ -50,6 +50,7 @@ struct ConvArgs {
     cudaStream_t stream;
     int32_t* status;  // device status word of the plan on this device
     const int32_t* n_real;  // padded call: device word with the number of real edges (rowptr[n_nodes]); else null
+    const float* vec;       // forward: edge vectors [E][3] in place of sh (the kernel forms the harmonics); else null
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -73,7 +74,10 @@ inline int sm_count() {
 // The bodies of e3j_conv_fwd / e3j_conv_bwd (and their padded forms), for entry points that compose them.
 int conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x, const float* sh,
                   const float* w, const int32_t* senders, const int32_t* receivers, const int32_t* rowptr,
-                  float* out, void* workspace, size_t workspace_bytes, void* stream, bool padded);
+                  float* out, void* workspace, size_t workspace_bytes, void* stream, bool padded,
+                  const float* edge_vec = nullptr);   // edge_vec: specialised kernels only, in place of sh
+// Does the plan run on signature-specialised kernels (which can form the harmonics from edge vectors themselves)?
+bool has_fast_forward(const e3j_plan* plan);
 int conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x, const float* sh,
                   const float* w, const int32_t* senders, const int32_t* receivers, const int32_t* rowptr,
                   const int32_t* sender_perm, const int32_t* colptr, const float* grad_out, float* grad_x,

@@ -26,6 +26,7 @@ namespace fast {
 
 struct BwdParams {
     const float* x; const float* sh; const float* w;
+    const float* vec;                  // (forward only; always null here)
     const int32_t* senders; const int32_t* receivers;
     const float* grad_out;
     float* grad_sh; float* grad_w;

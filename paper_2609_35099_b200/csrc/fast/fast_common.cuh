@@ -143,6 +143,7 @@ struct PairRec {
 
 struct FwdParams {
     const float* x; const float* sh; const float* w;
+    const float* vec;                  // edge vectors [E][3]: the kernel forms the harmonics itself (then sh is unused)
     const int32_t* senders; const int32_t* receivers;
     float* out;
     int64_t n_nodes, n_edges, chunk;   // chunk = edges per CTA (multiple of 4)

@@ -41,6 +41,7 @@ int launch_fwd(const ConvArgs& a) {
     }
     FwdParams p{};
     p.x = a.x; p.sh = a.sh; p.w = a.w; p.senders = a.senders; p.receivers = a.receivers; p.out = a.out;
+    p.vec = a.vec;
     p.n_nodes = a.n_nodes; p.n_edges = a.n_edges;
     const int64_t per = (a.n_edges + n_cta - 1) / n_cta;
     p.chunk = (per + 3) / 4 * 4;

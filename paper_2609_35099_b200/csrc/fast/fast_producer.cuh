@@ -12,6 +12,7 @@
 // (APAD, DSH, pair_rec, rec_val, rec_i2); P is the kernel's parameter struct (x, sh, w, senders, receivers,
 // identity, status).
 #pragma once
+#include "harmonics.cuh"
 #include "fast_common.cuh"
 
 namespace e3j {
@@ -83,6 +84,7 @@ struct TablePart {
     ASlot tab[NA];              // this lane's A slots (lane, lane + 32, ...)
     int rcv_a = -1, rcv_b = -1; // receiver ids of the next two tiles
     float y_a[YPL], y_b[YPL];   // harmonics of the next two tiles
+    float v_a[3], v_b[3];       // or, when the call gives edge vectors instead, lane j's vector of each tile
     float uy_a[L::DBL ? YPL : 1], uy_b[L::DBL ? YPL : 1];   // and their cotangents (double backward)
     int last_rcv = -1;
 
@@ -99,8 +101,8 @@ struct TablePart {
             }
             tab[i] = a;
         }
-        load(0, rcv_a, y_a);
-        load(1, rcv_b, y_b);
+        load(0, rcv_a, y_a, v_a);
+        load(1, rcv_b, y_b, v_b);
         if constexpr (L::DBL) { load_ct(0, uy_a); load_ct(1, uy_b); }
     }
     __device__ __forceinline__ void load_ct(int t, float (&yv)[L::DBL ? YPL : 1]) {
@@ -113,11 +115,18 @@ struct TablePart {
             if (idx < n_e * Tab::DSH) yv[i] = p.ct_sh[e0 * Tab::DSH + idx];
         }
     }
-    __device__ __forceinline__ void load(int t, int& rcv, float (&yv)[YPL]) {
+    __device__ __forceinline__ void load(int t, int& rcv, float (&yv)[YPL], float (&vv)[3]) {
         if (t >= n_tiles) return;
         const int64_t e0 = e_begin + (int64_t)t * T;
         const int n_e = (int)min((int64_t)T, e_end - e0);
         if (lane < n_e) rcv = p.identity ? (int)(e0 + lane) : p.receivers[e0 + lane];
+        if (p.vec) {
+            if (lane < n_e) {
+#pragma unroll
+                for (int i = 0; i < 3; ++i) vv[i] = p.vec[(e0 + lane) * 3 + i];
+            }
+            return;
+        }
 #pragma unroll
         for (int i = 0; i < YPL; ++i) {
             const int idx = i * 32 + lane;
@@ -136,10 +145,20 @@ struct TablePart {
         last_rcv = __shfl_sync(0xffffffffu, rcv_a, n_e - 1);
         if (lane < n_e) recv_t[lane] = rcv_a;
         if (lane == 0) recv_t[T] = (int)mask;
+        if (p.vec) {   // harmonics of the edge direction, formed here
+            if (lane < n_e) {
+                float ux, uy, uz, inv_r, Y[Tab::DSH];
+                unit_vector(v_a[0], v_a[1], v_a[2], ux, uy, uz, inv_r);
+                harmonics<Tab::DSH>(ux, uy, uz, Y);
 #pragma unroll
-        for (int i = 0; i < YPL; ++i) {
-            const int idx = i * 32 + lane;
-            if (idx < n_e * Tab::DSH) y_t[idx] = y_a[i];
+                for (int i = 0; i < Tab::DSH; ++i) y_t[lane * Tab::DSH + i] = Y[i];
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < YPL; ++i) {
+                const int idx = i * 32 + lane;
+                if (idx < n_e * Tab::DSH) y_t[idx] = y_a[i];
+            }
         }
         if constexpr (L::DBL) {
             float* uy_t = reinterpret_cast<float*>(st + L::st_uy);
@@ -194,7 +213,9 @@ struct TablePart {
         rcv_a = rcv_b;
 #pragma unroll
         for (int i = 0; i < YPL; ++i) y_a[i] = y_b[i];
-        load(t + 2, rcv_b, y_b);
+#pragma unroll
+        for (int i = 0; i < 3; ++i) v_a[i] = v_b[i];
+        load(t + 2, rcv_b, y_b, v_b);
         if constexpr (L::DBL) {
 #pragma unroll
             for (int i = 0; i < YPL; ++i) uy_a[i] = uy_b[i];
