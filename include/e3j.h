@@ -331,6 +331,17 @@ int e3j_conv_vec_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, con
                      const int32_t* sender_perm, const int32_t* colptr, const float* grad_out, float* grad_x,
                      float* grad_vec, float* grad_w, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Both at once: the forward convolution from edge vectors and the radial layer, out = conv_fwd(x, Y(edge_vec), h W).
+ * Where the plan has the kernel that forms the edge scalars itself (see e3j_conv_radial_fwd) that kernel forms the
+ * harmonics too, and the call reads x, edge_vec, h, W and the graph only; otherwise the call is composed
+ * (e3j_harmonics_fwd and e3j_radial_weights into the workspace, then e3j_conv_fwd).  Arguments as for
+ * e3j_conv_radial_fwd with edge_vec [n_edges, 3] in place of sh. */
+size_t e3j_conv_radial_vec_fwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden);
+int e3j_conv_radial_vec_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
+                            const float* edge_vec, const float* h, const float* W, const int32_t* senders,
+                            const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
 /* Float64 convolution (paper, appendix on the benchmark setup: float64 builds of the kernels are shipped beside
  * the float32 ones).  Same operation, layouts, graph arguments and conventions as e3j_conv_fwd / e3j_conv_bwd with
  * every tensor in float64 and the coupling coefficients in float64 as the plan builder computed them.  Table-driven

@@ -24,7 +24,7 @@ __all__ = [
     "e3j_conv_bwd", "e3j_graph_prepare_padded", "e3j_conv_fwd_padded", "e3j_conv_bwd_padded",
     "e3j_conv_bwd_bwd_workspace_bytes", "e3j_conv_bwd_bwd",
     "e3j_radial_weights", "e3j_conv_radial_fwd_workspace_bytes", "e3j_conv_radial_bwd_workspace_bytes",
-    "e3j_conv_radial_fwd", "e3j_conv_radial_bwd",
+    "e3j_conv_radial_fwd", "e3j_conv_radial_bwd", "e3j_conv_radial_vec_fwd", "e3j_conv_radial_vec_fwd_workspace_bytes",
     "e3j_tp_fwd", "e3j_tp_bwd", "e3j_harmonics_fwd", "e3j_harmonics_bwd", "e3j_conv_vec_fwd", "e3j_conv_vec_bwd",
     "e3j_conv_vec_fwd_workspace_bytes", "e3j_conv_vec_bwd_workspace_bytes", "e3j_conv_fwd_f64", "e3j_conv_bwd_f64", "e3j_shard_prepare", "e3j_rows_gather", "e3j_rows_add", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
     "E3J_PLAN_COLLAPSE_OUTPUTS",
@@ -109,6 +109,10 @@ def _load():
     lib.e3j_conv_radial_bwd_workspace_bytes.restype = sz
     lib.e3j_conv_radial_fwd.argtypes = [vp, i64, i64, i32] + [vp] * 9 + [sz, vp]
     lib.e3j_conv_radial_fwd.restype = i32
+    lib.e3j_conv_radial_vec_fwd_workspace_bytes.argtypes = [vp, i64, i64, i32]
+    lib.e3j_conv_radial_vec_fwd_workspace_bytes.restype = sz
+    lib.e3j_conv_radial_vec_fwd.argtypes = [vp, i64, i64, i32] + [vp] * 9 + [sz, vp]
+    lib.e3j_conv_radial_vec_fwd.restype = i32
     lib.e3j_conv_radial_bwd.argtypes = [vp, i64, i64, i32] + [vp] * 15 + [sz, vp]
     lib.e3j_conv_radial_bwd.restype = i32
     lib.e3j_tp_fwd.argtypes = [vp, i64] + [vp] * 5
@@ -472,6 +476,31 @@ def e3j_conv_radial_fwd(plan: Plan, x, sh, h, W, senders, receivers, rowptr=None
         _dev_ptr(rowptr, i32, (n + 1,), "rowptr"),
         _dev_ptr(out, f32, (n, plan.d_out, plan.n_channels), "out"),
         ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_radial_fwd")
+    return out
+
+
+def e3j_conv_radial_vec_fwd_workspace_bytes(plan: Plan, n_nodes: int, n_edges: int, hidden: int) -> int:
+    return int(_load().e3j_conv_radial_vec_fwd_workspace_bytes(plan.handle, n_nodes, n_edges, hidden))
+
+
+def e3j_conv_radial_vec_fwd(plan: Plan, x, edge_vec, h, W, senders, receivers, rowptr=None, out=None, workspace=None,
+                            stream=None):
+    """Forward convolution from edge vectors [E, 3] and the radial layer (h, W): neither the harmonics nor the
+    edge weights exist as arrays where the plan has the kernel for it."""
+    torch = _torch()
+    n, e, hidden = x.shape[0], senders.numel(), W.shape[0]
+    f32, i32 = torch.float32, torch.int32
+    if out is None:
+        out = torch.empty((n, plan.d_out, plan.n_channels), dtype=f32, device=x.device)
+    workspace = _workspace(e3j_conv_radial_vec_fwd_workspace_bytes(plan, n, e, hidden), x, workspace)
+    _check(_load().e3j_conv_radial_vec_fwd(
+        plan.handle, n, e, hidden,
+        _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"), _dev_ptr(edge_vec, f32, (e, 3), "edge_vec"),
+        _dev_ptr(h, f32, (e, hidden), "h"), _dev_ptr(W, f32, (hidden, plan.n_paths * plan.n_channels), "W"),
+        _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
+        _dev_ptr(rowptr, i32, (n + 1,), "rowptr"),
+        _dev_ptr(out, f32, (n, plan.d_out, plan.n_channels), "out"),
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_radial_vec_fwd")
     return out
 
 

@@ -76,6 +76,10 @@ int conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const 
                   const float* w, const int32_t* senders, const int32_t* receivers, const int32_t* rowptr,
                   float* out, void* workspace, size_t workspace_bytes, void* stream, bool padded,
                   const float* edge_vec = nullptr);   // edge_vec: specialised kernels only, in place of sh
+// Harmonics of edge vectors (harmonics.cu): sh [n, (lmax+1)^2] from vec [n, 3] and the gradient back; lmax <= 3.
+int harmonics_fwd(int lmax, int64_t n, const float* vec, float* sh, cudaStream_t st);
+int harmonics_bwd(int lmax, int64_t n, const float* vec, const float* grad_sh, float* grad_vec, cudaStream_t st);
+int plan_sh_lmax(const e3j_plan* plan);   // lmax of the plan's harmonics if they are the full set l <= 3, else -1
 // Does the plan run on signature-specialised kernels (which can form the harmonics from edge vectors themselves)?
 bool has_fast_forward(const e3j_plan* plan);
 int conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x, const float* sh,

@@ -27,6 +27,7 @@
 // Stages hold a quarter tile (4 groups); two stages.  Registers are moved from the helper warps to the
 // consumers (setmaxnreg).  Every wait is bounded.
 #pragma once
+#include "harmonics.cuh"
 #include "../umma.cuh"
 #include "fast_common.cuh"
 
@@ -46,6 +47,7 @@ static_assert(4 * 32 * (kRegsTile + 2 * kRegsCons + kRegsAux) <= 65536, "registe
 
 struct RadialFwdParams {
     const float* x; const float* sh; const float* h; const float* W;
+    const float* vec;   // edge vectors [E][3]: the table warp forms the harmonics itself (then sh is unused)
     const int32_t* senders;
     const int32_t* slotptr; const int32_t* slot_edge; const int32_t* group_recv;
     float* out;
@@ -293,8 +295,19 @@ __device__ __forceinline__ void radial_table_warp(const RadialFwdParams& p, unsi
     float y[S::DSH];
     int recv = -1;
     auto load_data = [&](int qi, int edge) {
+        if (p.vec) {
+            if (edge >= 0) {
+                float ux, uy, uz, inv_r;
+                unit_vector(p.vec[(size_t)edge * 3], p.vec[(size_t)edge * 3 + 1], p.vec[(size_t)edge * 3 + 2], ux, uy, uz, inv_r);
+                harmonics<S::DSH>(ux, uy, uz, y);
+            } else {
 #pragma unroll
-        for (int i = 0; i < S::DSH; ++i) y[i] = (edge >= 0) ? p.sh[(size_t)edge * S::DSH + i] : 0.f;
+                for (int i = 0; i < S::DSH; ++i) y[i] = 0.f;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < S::DSH; ++i) y[i] = (edge >= 0) ? p.sh[(size_t)edge * S::DSH + i] : 0.f;
+        }
         recv = (qi < rg.n_quarters && lane < rg.valid_groups(qi)) ? p.group_recv[rg.g_begin + 4 * qi + lane] : -1;
     };
     load_data(0, rg.edge_of(p, 0, lane));
@@ -605,7 +618,7 @@ int launch_radial_fwd(const ConvArgs& a, const RadialArgs& r) {
         attr_dev = dev;
     }
     RadialFwdParams p{};
-    p.x = a.x; p.sh = a.sh; p.h = r.h; p.W = r.W; p.senders = a.senders;
+    p.x = a.x; p.sh = a.sh; p.vec = a.vec; p.h = r.h; p.W = r.W; p.senders = a.senders;
     p.slotptr = r.slotptr; p.slot_edge = r.slot_edge; p.group_recv = r.group_recv;
     p.out = a.out;
     p.part_recv = reinterpret_cast<int32_t*>(r.scratch);

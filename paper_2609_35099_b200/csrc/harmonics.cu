@@ -60,6 +60,8 @@ harmonics_bwd_kernel(int64_t n, const float* __restrict__ vec, const float* __re
 
 inline int grid_for(int64_t n) { return (int)std::min<int64_t>((n + 255) / 256, (int64_t)sm_count() * 16); }
 
+}  // namespace
+
 int harmonics_fwd(int lmax, int64_t n, const float* vec, float* sh, cudaStream_t st) {
     if (n == 0) return E3J_OK;
     switch (lmax) {
@@ -90,6 +92,8 @@ int plan_sh_lmax(const e3j_plan* plan) {
         if ((l + 1) * (l + 1) == plan->dp) return l;
     return -1;
 }
+
+namespace {
 
 // workspace of the calls on edge vectors: [convolution workspace | sh | grad_sh]
 struct VecLayout { size_t conv, conv_bytes, sh, gsh, total; };

@@ -179,10 +179,13 @@ size_t e3j_conv_radial_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes
     return radial::radial_layout(plan, n_nodes, n_edges, hidden, true).total;
 }
 
-int e3j_conv_radial_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
-                        const float* sh, const float* h, const float* W, const int32_t* senders,
-                        const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
-                        size_t workspace_bytes, void* stream) {
+}  // extern "C"
+
+// sh, or edge_vec with sh_scratch (room for [n_edges, d'] floats, used where no kernel forms the harmonics itself)
+static int radial_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
+                           const float* sh, const float* edge_vec, float* sh_scratch, const float* h, const float* W,
+                           const int32_t* senders, const int32_t* receivers, const int32_t* rowptr, float* out,
+                           void* workspace, size_t workspace_bytes, void* stream) {
     if (!radial::radial_args_ok(plan, n_nodes, n_edges, hidden)) return E3J_ERR_INVALID_ARG;
     if (hidden % 4 != 0 || plan->nq % 4 != 0) return E3J_ERR_UNSUPPORTED;
     if (n_nodes == 0) return E3J_OK;
@@ -193,7 +196,7 @@ int e3j_conv_radial_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, 
     char* ws = (char*)workspace;
     if (L.fused && n_edges > 0) {
         // edge scalars formed inside the kernel: slot tables of the graph, then one sweep
-        if (!x || !out || !sh || !senders || !receivers) return E3J_ERR_INVALID_ARG;
+        if (!x || !out || (!sh && !edge_vec) || !senders || !receivers) return E3J_ERR_INVALID_ARG;
         if (((uintptr_t)x | (uintptr_t)out) & 15u) return E3J_ERR_INVALID_ARG;
         cudaStream_t st = (cudaStream_t)stream;
         if (!rowptr) {
@@ -210,6 +213,7 @@ int e3j_conv_radial_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, 
         ConvArgs a{};
         a.n_nodes = n_nodes; a.n_edges = n_edges; a.x = x; a.sh = sh; a.senders = senders; a.receivers = receivers;
         a.rowptr = rowptr; a.out = out; a.stream = st; a.status = t.status;
+        a.vec = sh ? nullptr : edge_vec;
         RadialArgs r{};
         r.h = h; r.W = W; r.hidden = hidden; r.slotptr = slotptr; r.slot_edge = slot_edge; r.group_recv = group_recv;
         r.scratch = ws + L.scratch; r.scratch_bytes = L.scratch_bytes;
@@ -226,9 +230,46 @@ int e3j_conv_radial_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, 
         if (int st = get_device_tables(plan, t)) return st;
         if (int st = radial::radial_weights(n_edges, hidden, plan->P * plan->nq, h, W, s, t.status, (cudaStream_t)stream))
             return st;
+        if (!sh) {   // composed form on edge vectors: the harmonics go through the caller's scratch
+            if (!edge_vec || !sh_scratch) return E3J_ERR_INVALID_ARG;
+            if (int st = harmonics_fwd(plan_sh_lmax(plan), n_edges, edge_vec, sh_scratch, (cudaStream_t)stream)) return st;
+            sh = sh_scratch;
+        }
     }
     return conv_fwd_impl(plan, n_nodes, n_edges, x, sh, s, senders, receivers, rowptr, out, ws + L.conv, L.conv_bytes,
                          stream, false);
+}
+
+extern "C" {
+
+int e3j_conv_radial_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
+                        const float* sh, const float* h, const float* W, const int32_t* senders,
+                        const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    if (n_edges > 0 && !sh) return E3J_ERR_INVALID_ARG;
+    return radial_fwd_impl(plan, n_nodes, n_edges, hidden, x, sh, nullptr, nullptr, h, W, senders, receivers, rowptr, out,
+                           workspace, workspace_bytes, stream);
+}
+
+size_t e3j_conv_radial_vec_fwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden) {
+    if (!radial::radial_args_ok(plan, n_nodes, n_edges, hidden)) return 0;
+    return align_up(radial::radial_layout(plan, n_nodes, n_edges, hidden, false).total, 256) +
+           align_up(4 * (size_t)std::max<int64_t>(n_edges, 1) * plan->dp, 256);
+}
+
+int e3j_conv_radial_vec_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
+                            const float* edge_vec, const float* h, const float* W, const int32_t* senders,
+                            const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
+                            size_t workspace_bytes, void* stream) {
+    if (!radial::radial_args_ok(plan, n_nodes, n_edges, hidden)) return E3J_ERR_INVALID_ARG;
+    if (plan_sh_lmax(plan) < 0) return E3J_ERR_UNSUPPORTED;
+    if (n_edges > 0 && !edge_vec) return E3J_ERR_INVALID_ARG;
+    const size_t inner = align_up(radial::radial_layout(plan, n_nodes, n_edges, hidden, false).total, 256);
+    if (!workspace || ((uintptr_t)workspace & 255u) ||
+        workspace_bytes < e3j_conv_radial_vec_fwd_workspace_bytes(plan, n_nodes, n_edges, hidden))
+        return E3J_ERR_WORKSPACE;
+    return radial_fwd_impl(plan, n_nodes, n_edges, hidden, x, nullptr, edge_vec, (float*)((char*)workspace + inner), h, W,
+                           senders, receivers, rowptr, out, workspace, inner, stream);
 }
 
 int e3j_conv_radial_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,

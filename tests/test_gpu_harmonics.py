@@ -102,6 +102,31 @@ def test_convolution_on_edge_vectors(config, n_atoms, flags):
     assert_blockwise_close(only_vec[1].cpu().numpy(), rvec, [(0, 3)], what="grad_vec alone")
 
 
+@pytest.mark.parametrize("config,n_atoms,hidden", [(2, 192, 64), (2, 648, 32), (1, None, 16), (3, 300, 64)])
+def test_radial_forward_on_edge_vectors(config, n_atoms, hidden):
+    """e3j_conv_radial_vec_fwd against the oracle's conv_radial_fwd on the oracle's harmonics of the vectors, and
+    against the call that takes ready-made harmonics."""
+    c = workloads.CONFIGS[config]
+    wl = workloads.make_graph(config, n_atoms)
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"], 0)
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"])
+    x, _, _, _ = workloads.make_features(wl, plan.n_paths, plan.d_out)
+    h, W = workloads.make_radial(wl, plan.n_paths, hidden)
+    vec = wl.vectors.astype(np.float32)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    out = e3j.e3j_conv_radial_vec_fwd(plan, _cuda(x), _cuda(vec), _cuda(h), _cuda(W), snd, rcv)
+    out2 = e3j.e3j_conv_radial_vec_fwd(plan, _cuda(x), _cuda(vec), _cuda(h), _cuda(W), snd, rcv)
+    torch.cuda.synchronize()
+    assert e3j.e3j_plan_device_status(plan) == 0
+    assert torch.equal(out, out2)
+    y = osh.real_sh_all_of_vectors(c["sh_lmax"], vec.astype(np.float64)).astype(np.float32)
+    ref = oconv.conv_radial_fwd(cp, x, y, h, W, wl.senders, wl.receivers)
+    assert_blockwise_close(out.cpu().numpy(), ref, blocks_of_paths(cp.paths, "out"), what="out")
+    with_sh = e3j.e3j_conv_radial_fwd(plan, _cuda(x), e3j.e3j_harmonics_fwd(c["sh_lmax"], _cuda(vec)), _cuda(h), _cuda(W),
+                                      snd, rcv)
+    assert torch.allclose(out, with_sh, rtol=0, atol=1e-6 * float(out.abs().max()))
+
+
 def test_convolution_on_edge_vectors_checks_its_workspace():
     """The binding refuses a short workspace; the library itself answers E3J_ERR_WORKSPACE (called directly)."""
     import ctypes
