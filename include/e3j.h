@@ -342,6 +342,31 @@ int e3j_conv_radial_vec_fwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edg
                             const int32_t* receivers, const int32_t* rowptr, float* out, void* workspace,
                             size_t workspace_bytes, void* stream);
 
+/* Scheduled backward (no counterpart in the paper; it replaces the atomics of the paper's GPU backward and most of the
+ * per-edge share array of e3j_conv_bwd's fixed-order sender sum).  The schedule is a processing order of the edges,
+ * built once per neighbour list: inside every CTA's edge range, edges with the same sender and neighbouring receivers
+ * follow one another in one consumer warp, which adds their shares of grad_x in registers and writes one row per run;
+ * the sender sum then reads 1.6 times fewer rows (water box) in a fixed order.  Results are bit-identical from run to
+ * run; they differ from e3j_conv_bwd's in the rounding of grad_x only (another, equally fixed, summation order).
+ *   e3j_bwd_schedule_bytes      device bytes a schedule may need (0: the plan has no scheduled kernel)
+ *   e3j_bwd_schedule_build      senders / receivers are HOST arrays here (receiver-sorted, as everywhere); the order
+ *                               is computed on the host and copied to schedule_dev (256-byte aligned) on the stream;
+ *                               E3J_ERR_INVALID_ARG for an unsorted list or an index out of range.  The schedule
+ *                               belongs to the plan's signature and to the device's SM count.
+ *   e3j_conv_bwd_scheduled      e3j_conv_bwd on a schedule: x, sh, w, grad_out and the three gradients as there (all
+ *                               three required), workspace as for e3j_conv_bwd.
+ *   e3j_bwd_schedule_build_host host-only form for tests and tools: T = edges per tile, writes the schedule's words
+ *                               (layout: csrc/bwd_schedule.hpp) to host memory; -2 with *n_words = need if it does
+ *                               not fit. */
+size_t e3j_bwd_schedule_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges);
+int e3j_bwd_schedule_build(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const int32_t* senders_host,
+                           const int32_t* receivers_host, void* schedule_dev, size_t schedule_bytes, void* stream);
+int e3j_conv_bwd_scheduled(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, const float* x, const float* sh,
+                           const float* w, const void* schedule_dev, const float* grad_out, float* grad_x,
+                           float* grad_sh, float* grad_w, void* workspace, size_t workspace_bytes, void* stream);
+int e3j_bwd_schedule_build_host(int T, int n_ranges, int64_t n_nodes, int64_t n_edges, const int32_t* senders,
+                                const int32_t* receivers, int32_t* out_words, size_t capacity_words, size_t* n_words);
+
 /* Float64 convolution (paper, appendix on the benchmark setup: float64 builds of the kernels are shipped beside
  * the float32 ones).  Same operation, layouts, graph arguments and conventions as e3j_conv_fwd / e3j_conv_bwd with
  * every tensor in float64 and the coupling coefficients in float64 as the plan builder computed them.  Table-driven
