@@ -575,6 +575,32 @@ def main():
         }
         del ws_rf, ws_rb, w_mat, hh, WW, gh, gW
 
+    # ---- the backward over a processing order built once per neighbour list (runs of one sender summed in registers)
+    sched_block = None
+    if want_radial and not args.pad and not args.collapse and not args.generic and \
+            e3j.e3j_bwd_schedule_bytes(plan, n, e) > 0:
+        t_b = time.perf_counter()
+        sched = e3j.e3j_bwd_schedule_build(plan, n, d["snd"], d["rcv"])
+        torch.cuda.synchronize()
+        build_ms = (time.perf_counter() - t_b) * 1e3
+        hdr = sched[:64].view(torch.int32).cpu()
+        k_s = max(3, min(args.steps, 50))
+        for _ in range(3):
+            e3j.e3j_conv_bwd_scheduled(plan, d["x"], d["y"], d["w"], sched, d["g"], grad_x=gx, grad_sh=gy, grad_w=gw, workspace=ws_b)
+        a_, b_ = ev(), ev()
+        torch.cuda.synchronize()
+        a_.record(stream)
+        for _ in range(k_s):
+            e3j.e3j_conv_bwd_scheduled(plan, d["x"], d["y"], d["w"], sched, d["g"], grad_x=gx, grad_sh=gy, grad_w=gw, workspace=ws_b)
+        b_.record(stream)
+        torch.cuda.synchronize()
+        sched_block = {"bwd_ms": a_.elapsed_time(b_) / k_s, "schedule_build_ms": build_ms,
+                       "schedule_build": "host (graph arrays copied to the host, order copied back), once per neighbour list",
+                       "rows_written": int(hdr[5]), "edges_per_row": e / max(int(hdr[5]), 1), "tiles": int(hdr[4]),
+                       "note": "e3j_conv_bwd_scheduled: same gradients, grad_x summed in another fixed order; "
+                               "the headline backward is the unscheduled call"}
+        del sched
+
     # ---- the convolution on edge vectors: harmonics formed in the kernel's table warp, beside the two-step form
     vec_block = None
     if want_radial and not args.pad and not args.collapse and not args.generic and plan.d_sh in (1, 4, 9, 16):
@@ -713,7 +739,7 @@ def main():
             # 20 % of the runs, as in its efficiency-comparison section), minimum and maximum
             "call_stats_ms": {"fwd": call_stats(fwd_ms), "bwd": call_stats(bwd_ms)},
             "outside_the_step_ms": {"plan_build_host": plan_build_ms, "graph_prepare_device": graph_prepare_ms},
-            "double_backward": dbl, "radial": radial, "edge_vectors": vec_block, "sustained": sustained,
+            "double_backward": dbl, "radial": radial, "edge_vectors": vec_block, "scheduled_backward": sched_block, "sustained": sustained,
             "roofline": dominant, "roofline_fwd": roofs["fwd"], "roofline_bwd": roofs["bwd"],
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         }

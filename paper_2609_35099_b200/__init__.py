@@ -25,7 +25,7 @@ __all__ = [
     "e3j_conv_bwd_bwd_workspace_bytes", "e3j_conv_bwd_bwd",
     "e3j_radial_weights", "e3j_conv_radial_fwd_workspace_bytes", "e3j_conv_radial_bwd_workspace_bytes",
     "e3j_conv_radial_fwd", "e3j_conv_radial_bwd", "e3j_conv_radial_vec_fwd", "e3j_conv_radial_vec_fwd_workspace_bytes",
-    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_harmonics_fwd", "e3j_harmonics_bwd", "e3j_conv_vec_fwd", "e3j_conv_vec_bwd",
+    "e3j_tp_fwd", "e3j_tp_bwd", "e3j_bwd_schedule_bytes", "e3j_bwd_schedule_build", "e3j_conv_bwd_scheduled", "e3j_harmonics_fwd", "e3j_harmonics_bwd", "e3j_conv_vec_fwd", "e3j_conv_vec_bwd",
     "e3j_conv_vec_fwd_workspace_bytes", "e3j_conv_vec_bwd_workspace_bytes", "e3j_conv_fwd_f64", "e3j_conv_bwd_f64", "e3j_shard_prepare", "e3j_rows_gather", "e3j_rows_add", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
     "E3J_PLAN_COLLAPSE_OUTPUTS",
 ]
@@ -128,6 +128,12 @@ def _load():
     lib.e3j_conv_vec_fwd.restype = i32
     lib.e3j_conv_vec_bwd.argtypes = [vp, i64, i64] + [vp] * 13 + [sz, vp]
     lib.e3j_conv_vec_bwd.restype = i32
+    lib.e3j_bwd_schedule_bytes.argtypes = [vp, i64, i64]
+    lib.e3j_bwd_schedule_bytes.restype = sz
+    lib.e3j_bwd_schedule_build.argtypes = [vp, i64, i64, vp, vp, vp, sz, vp]
+    lib.e3j_bwd_schedule_build.restype = i32
+    lib.e3j_conv_bwd_scheduled.argtypes = [vp, i64, i64] + [vp] * 9 + [sz, vp]
+    lib.e3j_conv_bwd_scheduled.restype = i32
     lib.e3j_conv_f64_workspace_bytes.argtypes = [vp, i64, i64]
     lib.e3j_conv_f64_workspace_bytes.restype = sz
     lib.e3j_conv_fwd_f64.argtypes = [vp, i64, i64] + [vp] * 8 + [sz, vp]
@@ -572,6 +578,55 @@ def e3j_tp_bwd(plan: Plan, x1, x2, w, grad_out, grad_x1=True, grad_x2=True, grad
         _dev_ptr(grad_x1, f32, None, "grad_x1"), _dev_ptr(grad_x2, f32, None, "grad_x2"),
         _dev_ptr(grad_w, f32, None, "grad_w"), _stream(stream)), "e3j_tp_bwd")
     return grad_x1, grad_x2, grad_w
+
+
+def e3j_bwd_schedule_bytes(plan: Plan, n_nodes: int, n_edges: int) -> int:
+    """Device bytes a backward schedule may need; 0 if the plan has no scheduled kernel."""
+    return int(_load().e3j_bwd_schedule_bytes(plan.handle, n_nodes, n_edges))
+
+
+def e3j_bwd_schedule_build(plan: Plan, n_nodes: int, senders, receivers, stream=None):
+    """The processing order of e3j_conv_bwd_scheduled for this graph (a device uint8 tensor).  The graph arrays may
+    live on the device or the host; the order is computed on the host."""
+    torch = _torch()
+    e = senders.numel()
+    dev = senders.device if senders.is_cuda else torch.device("cuda", torch.cuda.current_device())
+    nbytes = e3j_bwd_schedule_bytes(plan, n_nodes, e)
+    if nbytes == 0:
+        raise RuntimeError("e3j_bwd_schedule_build: the plan has no scheduled backward kernel")
+    snd = senders.detach().to("cpu", torch.int32).contiguous()
+    rcv = receivers.detach().to("cpu", torch.int32).contiguous()
+    sched = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        _check(_load().e3j_bwd_schedule_build(plan.handle, n_nodes, e, ctypes.c_void_p(snd.data_ptr()),
+                                              ctypes.c_void_p(rcv.data_ptr()), ctypes.c_void_p(sched.data_ptr()), nbytes,
+                                              _stream(stream)), "e3j_bwd_schedule_build")
+    return sched
+
+
+def e3j_conv_bwd_scheduled(plan: Plan, x, sh, w, schedule, grad_out, grad_x=None, grad_sh=None, grad_w=None,
+                           workspace=None, stream=None):
+    """e3j_conv_bwd over a schedule from e3j_bwd_schedule_build: (grad_x, grad_sh, grad_w), all three always."""
+    torch = _torch()
+    n, e = x.shape[0], w.shape[0]
+    f32 = torch.float32
+    if grad_x is None:
+        grad_x = torch.empty((n, plan.d_in, plan.n_channels), dtype=f32, device=x.device)
+    if grad_sh is None:
+        grad_sh = torch.empty((e, plan.d_sh), dtype=f32, device=x.device)
+    if grad_w is None:
+        grad_w = torch.empty((e, plan.n_paths, plan.n_channels), dtype=f32, device=x.device)
+    workspace = _workspace(e3j_conv_bwd_workspace_bytes(plan, n, e), x, workspace)
+    if schedule.dtype != torch.uint8 or not schedule.is_cuda:
+        raise ValueError("schedule must be the CUDA uint8 tensor returned by e3j_bwd_schedule_build")
+    _check(_load().e3j_conv_bwd_scheduled(
+        plan.handle, n, e, _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"), _dev_ptr(sh, f32, (e, plan.d_sh), "sh"),
+        _dev_ptr(w, f32, (e, plan.n_paths, plan.n_channels), "w"), ctypes.c_void_p(schedule.data_ptr()),
+        _dev_ptr(grad_out, f32, (n, plan.d_out, plan.n_channels), "grad_out"),
+        _dev_ptr(grad_x, f32, (n, plan.d_in, plan.n_channels), "grad_x"), _dev_ptr(grad_sh, f32, (e, plan.d_sh), "grad_sh"),
+        _dev_ptr(grad_w, f32, (e, plan.n_paths, plan.n_channels), "grad_w"),
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_bwd_scheduled")
+    return grad_x, grad_sh, grad_w
 
 
 def e3j_harmonics_fwd(lmax: int, edge_vec, out=None, stream=None):

@@ -69,6 +69,29 @@ __global__ void bwd_dx_reduce_kernel(int64_t n_nodes, int row_f4, const float4* 
     }
 }
 
+__global__ void bwd_rows_reduce_kernel(int64_t n_nodes, int row_f4, const float4* __restrict__ dx_rows,
+                                       const int32_t* __restrict__ row_ptr, float4* __restrict__ grad_x) {
+    for (int64_t a = blockIdx.x; a < n_nodes; a += gridDim.x) {
+        const int j0 = row_ptr[a], j1 = row_ptr[a + 1];
+        for (int i = threadIdx.x; i < row_f4; i += blockDim.x) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            int j = j0;
+            for (; j + 8 <= j1; j += 8) {   // eight independent loads in flight; the additions stay in row order
+                float4 v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = dx_rows[(size_t)(j + u) * row_f4 + i];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+            }
+            for (; j < j1; ++j) {
+                const float4 v = dx_rows[(size_t)j * row_f4 + i];
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
+            grad_x[(size_t)a * row_f4 + i] = acc;
+        }
+    }
+}
+
 }  // namespace fast
 }  // namespace e3j
 

@@ -37,6 +37,10 @@ struct FastKernels {
     // forward with the edge scalars formed in the kernel from the radial layer (null: the caller materialises
     // them first); see fast/fast_radial.cuh
     int (*radial_fwd)(const ConvArgs&, const RadialArgs&);
+    // backward over a processing order built once per neighbour list (fast/fast_bwd1s.cuh, bwd_schedule.hpp);
+    // null: the signature has no scheduled kernel.  sched_T = edges per tile the order must be built for.
+    int (*conv_bwd_sched)(const ConvArgs&, const int32_t* schedule);
+    int sched_T;
 };
 
 // Index of the entry generated for `signature`, or -1.

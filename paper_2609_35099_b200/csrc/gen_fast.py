@@ -643,6 +643,8 @@ class Sig:
         o.append('#include "fast_fwd.cuh"')
         o.append('#include "fast_bwd.cuh"')
         o.append('#include "fast_launch.cuh"')
+        if self.cfg.get("SB", 0):
+            o.append('#include "fast_bwd1s.cuh"')
         if self.cfg.get("RF", 0):
             o.append('#include "fast_radial.cuh"')
         o.append("")
@@ -804,8 +806,9 @@ class Sig:
                      f"&fast::launch_tp_bwd<fast::{S}>,")
             dbl_e = f"&fast::launch_dbl_edges<fast::{S}>" if self.cfg.get("DT", 0) else "nullptr"
             dbl_o = f"&fast::launch_dbl_out<fast::{S}>" if self.cfg.get("DFT", 0) else "nullptr"
-            rf = f", &fast::launch_radial_fwd<fast::{S}>" if self.cfg.get("RF", 0) else ""
-            o.append(f"    {dbl_e}, {dbl_o}{rf}}};")
+            rf = f"&fast::launch_radial_fwd<fast::{S}>" if self.cfg.get("RF", 0) else "nullptr"
+            sb = (f"&fast::launch_bwd_sched<fast::{S}>, {self.cfg['ET']}" if self.cfg.get("SB", 0) else "nullptr, 0")
+            o.append(f"    {dbl_e}, {dbl_o}, {rf}, {sb}}};")
         else:
             o.append(f"    &fast::fwd_scratch_bytes<fast::{S}>, nullptr, &fast::launch_fwd<fast::{S}>, nullptr, nullptr, nullptr, "
                      f"nullptr, nullptr}};")
