@@ -723,6 +723,18 @@ def test_config5_full_size_sampled():
         rx, _, _ = oconv.conv_bwd(cp, xs, y[ids], ws, l_snd, l_rcv.astype(np.int32), gs)
         assert_blockwise_close(gx[a].cpu().numpy()[None], rx[-1][None], blocks_of_paths(cp.paths, "x"), what=f"grad_x[{a}]")
 
+    # the scheduled backward at the same size, into the same tensors: per-edge gradients bit-identical to the call
+    # checked above, grad_x equal to rounding (its rows are summed in another fixed order)
+    sums_plain = [_checksum(t) for t in (gy, gw)]
+    gx_plain = gx.clone()
+    sched = e3j.e3j_bwd_schedule_build(plan, n, snd, rcv)
+    gx.zero_(); gy.zero_()
+    e3j.e3j_conv_bwd_scheduled(plan, dx_, dy_, dw_, sched, dg_, grad_x=gx, grad_sh=gy, grad_w=gw)
+    torch.cuda.synchronize()
+    assert e3j.e3j_plan_device_status(plan) == 0
+    assert sums_plain == [_checksum(t) for t in (gy, gw)]
+    assert float((gx - gx_plain).abs().max()) <= 2e-6 * float(gx_plain.abs().max())
+
 
 def test_tensor_product_full_size_sampled():
     """Config 4 at 2^20 rows (75 GB of forward I/O); sampled rows against the oracle."""
