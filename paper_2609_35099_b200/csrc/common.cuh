@@ -30,6 +30,21 @@ inline int after_launch() {
     return cuda_status(cudaGetLastError());
 }
 
+// Launch of a kernel that follows another one on the same stream and starts with fast::grid_dependency_wait(): the
+// launch itself (and the scheduling of its first CTAs) overlaps the tail of its predecessor; the wait inside the
+// kernel holds it until the predecessor has finished and its writes are visible (programmatic dependent launch).
+template <class... KArgs, class... Args>
+inline int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return cuda_status(err != cudaSuccess ? err : cudaGetLastError());
+}
 // Device tables of `plan` on the current device (uploaded on first use).
 int get_device_tables(const e3j_plan* plan, DeviceTables& out);
 

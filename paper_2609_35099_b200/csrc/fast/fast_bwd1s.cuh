@@ -292,9 +292,8 @@ int launch_bwd_sched(const ConvArgs& a, const int32_t* sched) {
     if (int s = after_launch()) return s;
     const int32_t* row_ptr = sched + 16 + n_cta + 1;   // header, tile_ptr[n_cta + 1], then row_ptr (bwd_schedule.hpp)
     const int64_t blocks = std::min<int64_t>(a.n_nodes, (int64_t)1 << 30);
-    bwd_rows_reduce_kernel<<<(int)blocks, S::DIN * S::NQ / 4, 0, a.stream>>>(a.n_nodes, S::DIN * S::NQ / 4,
+    return launch_dependent(bwd_rows_reduce_kernel, dim3((int)blocks), dim3(S::DIN * S::NQ / 4), 0, a.stream, a.n_nodes, S::DIN * S::NQ / 4,
         reinterpret_cast<const float4*>(p.dx_rows), row_ptr, reinterpret_cast<float4*>(a.grad_x));
-    return after_launch();
 }
 
 }  // namespace fast

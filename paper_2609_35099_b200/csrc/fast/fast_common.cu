@@ -6,6 +6,7 @@ namespace fast {
 
 __global__ void fwd_fixup_kernel(int n_cta, int row_f4, const float4* __restrict__ partial,
                                  const int32_t* __restrict__ part_recv, float4* __restrict__ out) {
+    grid_dependency_wait();
     const int c = blockIdx.x;
     const int b = part_recv[2 * c + 1];  // a row whose first piece is this CTA's tail
     if (b < 0) return;
@@ -47,6 +48,7 @@ __global__ void bwd_zero_padding_kernel(const int32_t* __restrict__ n_real, int6
 __global__ void bwd_dx_reduce_kernel(int64_t n_nodes, int row_f4, const float4* __restrict__ dx_edge,
                                      const int32_t* __restrict__ sender_perm, const int32_t* __restrict__ colptr,
                                      float4* __restrict__ grad_x) {
+    grid_dependency_wait();
     for (int64_t a = blockIdx.x; a < n_nodes; a += gridDim.x) {
         const int j0 = colptr[a], j1 = colptr[a + 1];
         for (int i = threadIdx.x; i < row_f4; i += blockDim.x) {
@@ -71,6 +73,7 @@ __global__ void bwd_dx_reduce_kernel(int64_t n_nodes, int row_f4, const float4* 
 
 __global__ void bwd_rows_reduce_kernel(int64_t n_nodes, int row_f4, const float4* __restrict__ dx_rows,
                                        const int32_t* __restrict__ row_ptr, float4* __restrict__ grad_x) {
+    grid_dependency_wait();
     for (int64_t a = blockIdx.x; a < n_nodes; a += gridDim.x) {
         const int j0 = row_ptr[a], j1 = row_ptr[a + 1];
         for (int i = threadIdx.x; i < row_f4; i += blockDim.x) {

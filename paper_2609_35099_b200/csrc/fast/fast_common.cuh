@@ -20,6 +20,10 @@ namespace fast {
 constexpr uint32_t kSpinLimit = 1u << 22;  // polls of mbarrier.try_wait before giving up
 constexpr int kStatusTimeout = 1;          // value stored in the device status word
 
+// First statement of a kernel that is launched with launch_dependent (common.cuh): holds the kernel until the
+// one before it on the stream has finished and its writes are visible; a no-op under an ordinary launch.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- channel vectors
 // A lane owns V consecutive channels (float2 or float4): one 8- or 16-byte shared-memory
 // load feeds V FMAs.

@@ -52,9 +52,8 @@ int launch_fwd(const ConvArgs& a) {
     constexpr int threads = (S::FW * (S::NQ / (32 * S::V)) + 2) * 32;  // consumers + two producer warps
     fast_fwd_kernel<S><<<n_cta, threads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
-    fwd_fixup_kernel<<<n_cta, 256, 0, a.stream>>>(n_cta, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),
+    return launch_dependent(fwd_fixup_kernel, dim3(n_cta), dim3(256), 0, a.stream, n_cta, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),
                                                  p.part_recv, reinterpret_cast<float4*>(a.out));
-    return after_launch();
 }
 
 // Standalone tensor product = the forward kernel with every row its own sender and receiver: no row
@@ -161,9 +160,8 @@ int launch_bwd(const ConvArgs& a) {
     }
     // one CTA per sender: the hardware hands them out as CTAs finish, so uneven degrees do not leave a tail
     const int64_t blocks = std::min<int64_t>(a.n_nodes, (int64_t)1 << 30);
-    bwd_dx_reduce_kernel<<<(int)blocks, S::DIN * S::NQ / 4, 0, a.stream>>>(a.n_nodes, S::DIN * S::NQ / 4,
+    return launch_dependent(bwd_dx_reduce_kernel, dim3((int)blocks), dim3(S::DIN * S::NQ / 4), 0, a.stream, a.n_nodes, S::DIN * S::NQ / 4,
         reinterpret_cast<const float4*>(p.dx_edge), a.sender_perm, a.colptr, reinterpret_cast<float4*>(a.grad_x));
-    return after_launch();
 }
 
 // Fused double backward, edge outputs: the edge-wise sweep over (x, sh, w) and their cotangents, then the
@@ -193,9 +191,8 @@ int launch_dbl_edges(const ConvArgs& a, const float* ct_x, const float* ct_sh, c
     fast_bwd1_kernel<S, false, true><<<n_cta, (L1::T * L1::CH + 1) * 32, L1::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
     const int64_t blocks = std::min<int64_t>(a.n_nodes, (int64_t)1 << 30);
-    bwd_dx_reduce_kernel<<<(int)blocks, S::DIN * S::NQ / 4, 0, a.stream>>>(a.n_nodes, S::DIN * S::NQ / 4,
+    return launch_dependent(bwd_dx_reduce_kernel, dim3((int)blocks), dim3(S::DIN * S::NQ / 4), 0, a.stream, a.n_nodes, S::DIN * S::NQ / 4,
         reinterpret_cast<const float4*>(p.dx_edge), a.sender_perm, a.colptr, reinterpret_cast<float4*>(a.grad_x));
-    return after_launch();
 }
 
 // Fused double backward, cotangent of grad_out: the forward sweep with two terms per coefficient pair, written
@@ -227,9 +224,8 @@ int launch_dbl_out(const ConvArgs& a, const float* ct_x, const float* ct_sh, con
     constexpr int threads = (L::NCONS + 2) * 32;  // consumers + two producer warps
     fast_fwd_kernel<S, true><<<n_cta, threads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
-    fwd_fixup_kernel<<<n_cta, 256, 0, a.stream>>>(n_cta, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),
+    return launch_dependent(fwd_fixup_kernel, dim3(n_cta), dim3(256), 0, a.stream, n_cta, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),
                                                  p.part_recv, reinterpret_cast<float4*>(a.out));
-    return after_launch();
 }
 
 }  // namespace fast

@@ -630,9 +630,8 @@ int launch_radial_fwd(const ConvArgs& a, const RadialArgs& r) {
 #endif
     radial_fwd_kernel<S><<<n_ranges * NCG, kRadialThreads, L::total, a.stream>>>(p);
     if (int s = after_launch()) return s;
-    fwd_fixup_kernel<<<n_ranges, 256, 0, a.stream>>>(n_ranges, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),
+    return launch_dependent(fwd_fixup_kernel, dim3(n_ranges), dim3(256), 0, a.stream, n_ranges, S::D * S::NQ / 4, reinterpret_cast<const float4*>(p.partial),
                                                     p.part_recv, reinterpret_cast<float4*>(a.out));
-    return after_launch();
 }
 
 }  // namespace fast
