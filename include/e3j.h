@@ -367,6 +367,16 @@ int e3j_conv_bwd_scheduled(const e3j_plan* plan, int64_t n_nodes, int64_t n_edge
 int e3j_bwd_schedule_build_host(int T, int n_ranges, int64_t n_nodes, int64_t n_edges, const int32_t* senders,
                                 const int32_t* receivers, int32_t* out_words, size_t capacity_words, size_t* n_words);
 
+/* Backward of the call above, composed: harmonics into the workspace, e3j_conv_radial_bwd with the harmonics' cotangent
+ * kept as scratch, e3j_harmonics_bwd.  grad_vec [n_edges, 3] in place of grad_sh; any of grad_x, grad_vec, grad_h,
+ * grad_W may be NULL. */
+size_t e3j_conv_radial_vec_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden);
+int e3j_conv_radial_vec_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
+                            const float* edge_vec, const float* h, const float* W, const int32_t* senders,
+                            const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                            const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_vec,
+                            float* grad_h, float* grad_W, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Float64 convolution (paper, appendix on the benchmark setup: float64 builds of the kernels are shipped beside
  * the float32 ones).  Same operation, layouts, graph arguments and conventions as e3j_conv_fwd / e3j_conv_bwd with
  * every tensor in float64 and the coupling coefficients in float64 as the plan builder computed them.  Table-driven

@@ -24,7 +24,7 @@ __all__ = [
     "e3j_conv_bwd", "e3j_graph_prepare_padded", "e3j_conv_fwd_padded", "e3j_conv_bwd_padded",
     "e3j_conv_bwd_bwd_workspace_bytes", "e3j_conv_bwd_bwd",
     "e3j_radial_weights", "e3j_conv_radial_fwd_workspace_bytes", "e3j_conv_radial_bwd_workspace_bytes",
-    "e3j_conv_radial_fwd", "e3j_conv_radial_bwd", "e3j_conv_radial_vec_fwd", "e3j_conv_radial_vec_fwd_workspace_bytes",
+    "e3j_conv_radial_fwd", "e3j_conv_radial_bwd", "e3j_conv_radial_vec_fwd", "e3j_conv_radial_vec_fwd_workspace_bytes", "e3j_conv_radial_vec_bwd", "e3j_conv_radial_vec_bwd_workspace_bytes",
     "e3j_tp_fwd", "e3j_tp_bwd", "e3j_bwd_schedule_bytes", "e3j_bwd_schedule_build", "e3j_conv_bwd_scheduled", "e3j_harmonics_fwd", "e3j_harmonics_bwd", "e3j_conv_vec_fwd", "e3j_conv_vec_bwd",
     "e3j_conv_vec_fwd_workspace_bytes", "e3j_conv_vec_bwd_workspace_bytes", "e3j_conv_fwd_f64", "e3j_conv_bwd_f64", "e3j_shard_prepare", "e3j_rows_gather", "e3j_rows_add", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
     "E3J_PLAN_COLLAPSE_OUTPUTS",
@@ -113,6 +113,10 @@ def _load():
     lib.e3j_conv_radial_vec_fwd_workspace_bytes.restype = sz
     lib.e3j_conv_radial_vec_fwd.argtypes = [vp, i64, i64, i32] + [vp] * 9 + [sz, vp]
     lib.e3j_conv_radial_vec_fwd.restype = i32
+    lib.e3j_conv_radial_vec_bwd_workspace_bytes.argtypes = [vp, i64, i64, i32]
+    lib.e3j_conv_radial_vec_bwd_workspace_bytes.restype = sz
+    lib.e3j_conv_radial_vec_bwd.argtypes = [vp, i64, i64, i32] + [vp] * 15 + [sz, vp]
+    lib.e3j_conv_radial_vec_bwd.restype = i32
     lib.e3j_conv_radial_bwd.argtypes = [vp, i64, i64, i32] + [vp] * 15 + [sz, vp]
     lib.e3j_conv_radial_bwd.restype = i32
     lib.e3j_tp_fwd.argtypes = [vp, i64] + [vp] * 5
@@ -543,6 +547,44 @@ def e3j_conv_radial_bwd(plan: Plan, x, sh, h, W, senders, receivers, grad_out, r
         _dev_ptr(grad_h, f32, (e, hidden), "grad_h"), _dev_ptr(grad_W, f32, s_w, "grad_W"),
         ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_radial_bwd")
     return grad_x, grad_sh, grad_h, grad_W
+
+
+def e3j_conv_radial_vec_bwd_workspace_bytes(plan: Plan, n_nodes: int, n_edges: int, hidden: int) -> int:
+    return int(_load().e3j_conv_radial_vec_bwd_workspace_bytes(plan.handle, n_nodes, n_edges, hidden))
+
+
+def e3j_conv_radial_vec_bwd(plan: Plan, x, edge_vec, h, W, senders, receivers, grad_out, rowptr=None, sender_perm=None,
+                            colptr=None, grad_x=True, grad_vec=True, grad_h=True, grad_W=True, workspace=None,
+                            stream=None):
+    """Backward of e3j_conv_radial_vec_fwd: (grad_x, grad_vec, grad_h, grad_W); each grad_* argument is True
+    (allocate), False/None (not wanted) or a preallocated tensor."""
+    torch = _torch()
+    n, e, hidden = x.shape[0], senders.numel(), W.shape[0]
+    f32, i32 = torch.float32, torch.int32
+
+    def alloc(flag, shape):
+        if flag is True:
+            return torch.empty(shape, dtype=f32, device=x.device)
+        return flag if isinstance(flag, torch.Tensor) else None
+
+    s_w = (hidden, plan.n_paths * plan.n_channels)
+    grad_x = alloc(grad_x, (n, plan.d_in, plan.n_channels))
+    grad_vec = alloc(grad_vec, (e, 3))
+    grad_h = alloc(grad_h, (e, hidden))
+    grad_W = alloc(grad_W, s_w)
+    workspace = _workspace(e3j_conv_radial_vec_bwd_workspace_bytes(plan, n, e, hidden), x, workspace)
+    _check(_load().e3j_conv_radial_vec_bwd(
+        plan.handle, n, e, hidden,
+        _dev_ptr(x, f32, (n, plan.d_in, plan.n_channels), "x"), _dev_ptr(edge_vec, f32, (e, 3), "edge_vec"),
+        _dev_ptr(h, f32, (e, hidden), "h"), _dev_ptr(W, f32, s_w, "W"),
+        _dev_ptr(senders, i32, (e,), "senders"), _dev_ptr(receivers, i32, (e,), "receivers"),
+        _dev_ptr(rowptr, i32, (n + 1,), "rowptr"),
+        _dev_ptr(sender_perm, i32, (e,), "sender_perm"), _dev_ptr(colptr, i32, (n + 1,), "colptr"),
+        _dev_ptr(grad_out, f32, (n, plan.d_out, plan.n_channels), "grad_out"),
+        _dev_ptr(grad_x, f32, (n, plan.d_in, plan.n_channels), "grad_x"), _dev_ptr(grad_vec, f32, (e, 3), "grad_vec"),
+        _dev_ptr(grad_h, f32, (e, hidden), "grad_h"), _dev_ptr(grad_W, f32, s_w, "grad_W"),
+        ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)), "e3j_conv_radial_vec_bwd")
+    return grad_x, grad_vec, grad_h, grad_W
 
 
 def e3j_tp_fwd(plan: Plan, x1, x2, w, out=None, stream=None):

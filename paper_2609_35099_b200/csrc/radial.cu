@@ -305,4 +305,34 @@ int e3j_conv_radial_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, 
     return E3J_OK;
 }
 
+size_t e3j_conv_radial_vec_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden) {
+    if (!radial::radial_args_ok(plan, n_nodes, n_edges, hidden)) return 0;
+    return align_up(radial::radial_layout(plan, n_nodes, n_edges, hidden, true).total, 256) +
+           2 * align_up(4 * (size_t)std::max<int64_t>(n_edges, 1) * plan->dp, 256);
+}
+
+int e3j_conv_radial_vec_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, int hidden, const float* x,
+                            const float* edge_vec, const float* h, const float* W, const int32_t* senders,
+                            const int32_t* receivers, const int32_t* rowptr, const int32_t* sender_perm,
+                            const int32_t* colptr, const float* grad_out, float* grad_x, float* grad_vec,
+                            float* grad_h, float* grad_W, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!radial::radial_args_ok(plan, n_nodes, n_edges, hidden)) return E3J_ERR_INVALID_ARG;
+    const int lmax = plan_sh_lmax(plan);
+    if (lmax < 0) return E3J_ERR_UNSUPPORTED;
+    if (n_edges > 0 && !edge_vec) return E3J_ERR_INVALID_ARG;
+    const size_t inner = align_up(radial::radial_layout(plan, n_nodes, n_edges, hidden, true).total, 256);
+    const size_t sh_bytes = align_up(4 * (size_t)std::max<int64_t>(n_edges, 1) * plan->dp, 256);
+    if (!workspace || ((uintptr_t)workspace & 255u) || workspace_bytes < inner + 2 * sh_bytes) return E3J_ERR_WORKSPACE;
+    float* sh = (float*)((char*)workspace + inner);
+    float* gsh = (float*)((char*)workspace + inner + sh_bytes);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (int rc = harmonics_fwd(lmax, n_edges, edge_vec, sh, st)) return rc;
+    if (int rc = e3j_conv_radial_bwd(plan, n_nodes, n_edges, hidden, x, sh, h, W, senders, receivers, rowptr, sender_perm,
+                                     colptr, grad_out, grad_x, grad_vec ? gsh : nullptr, grad_h, grad_W, workspace, inner,
+                                     stream)) return rc;
+    if (grad_vec && n_nodes > 0)
+        if (int rc = harmonics_bwd(lmax, n_edges, edge_vec, gsh, grad_vec, st)) return rc;
+    return E3J_OK;
+}
+
 }  // extern "C"

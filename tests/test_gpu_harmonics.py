@@ -125,6 +125,17 @@ def test_radial_forward_on_edge_vectors(config, n_atoms, hidden):
     with_sh = e3j.e3j_conv_radial_fwd(plan, _cuda(x), e3j.e3j_harmonics_fwd(c["sh_lmax"], _cuda(vec)), _cuda(h), _cuda(W),
                                       snd, rcv)
     assert torch.allclose(out, with_sh, rtol=0, atol=1e-6 * float(out.abs().max()))
+    # the backward: grad_x, grad_h, grad_W as the oracle's radial backward on those harmonics, grad_vec through its
+    # harmonics gradient
+    g = workloads.make_features(wl, plan.n_paths, plan.d_out)[3]
+    gx, gvec, gh, gW = e3j.e3j_conv_radial_vec_bwd(plan, _cuda(x), _cuda(vec), _cuda(h), _cuda(W), snd, rcv, _cuda(g))
+    torch.cuda.synchronize()
+    rx, ry, rh, rW = oconv.conv_radial_bwd(cp, x, y, h, W, wl.senders, wl.receivers, g)
+    rvec = osh.real_sh_all_vjp(c["sh_lmax"], vec.astype(np.float64), ry)
+    assert_blockwise_close(gx.cpu().numpy(), rx, blocks_of_paths(cp.paths, "x"), what="grad_x")
+    assert_blockwise_close(gvec.cpu().numpy(), rvec, [(0, 3)], what="grad_vec")
+    assert_blockwise_close(gh.cpu().numpy(), rh, [(0, hidden)], what="grad_h")
+    assert np.abs(gW.cpu().numpy() - rW).max() <= 1e-5 * np.abs(rW).max()
 
 
 def test_convolution_on_edge_vectors_checks_its_workspace():
