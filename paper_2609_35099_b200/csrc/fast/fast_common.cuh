@@ -5,7 +5,8 @@
 // counted on an mbarrier); sender rows are gathered into the same stage by one bulk
 // copy per edge.  One producer warp issues the copies, the consumer warps wait on the
 // stage's "full" barrier and hand the stage back through its "empty" barrier.
-// No multicast, no tensor maps: every copy is a contiguous, 16-byte aligned range.
+// Plain bulk copies only (no tensor maps, nothing shared across a cluster): every copy is a contiguous,
+// 16-byte aligned range.
 //
 // Every wait is bounded: after kSpinLimit failed polls a warp records an error in the
 // status word, and the CTA drains and returns instead of spinning forever.
