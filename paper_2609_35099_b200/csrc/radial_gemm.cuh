@@ -7,6 +7,10 @@
 // core-matrix layout that the tensor cores read.  Roles: warps 0-3 read finished tiles out of tensor memory
 // and store them, eight warps convert, the last warp issues the tcgen05.mma instructions (one lane).
 //
+// Where the A operand does not depend on the tile (Prob::A_RESIDENT: the weights product, whose CTA keeps one block
+// of W^T for all of its edge tiles) it is converted once into a resident region of shared memory and the stage
+// ring carries the B operand alone, with more chunks of loads in flight per converter thread (Prob::PREFETCH).
+//
 // A Problem type describes one product: which output tiles a CTA owns, how many K chunks a tile has, where
 // operand values come from (zero outside the matrices) and where results go.  Three instances are used:
 //   s^T      = W^T h^T      edge scalars from the hidden activations            (RadialWeights)
