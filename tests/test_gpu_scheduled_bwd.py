@@ -77,3 +77,26 @@ def test_a_schedule_of_another_shape_is_refused_not_followed():
     c = workloads.CONFIGS[3]
     other = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"], 0)
     assert e3j.e3j_bwd_schedule_bytes(other, 10, 10) == 0
+
+
+def test_scheduled_backward_on_sparse_and_empty_graphs():
+    """Isolated nodes, senders without a run in most ranges, duplicate edges, and no edges at all."""
+    c = workloads.CONFIGS[2]
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"], 0)
+    rng = np.random.default_rng(5)
+    for n, e in ((400, 900), (50, 2000), (7, 3), (300, 0)):
+        snd = rng.integers(0, n, size=e).astype(np.int32)
+        rcv = np.sort(rng.integers(0, max(n // 2, 1), size=e)).astype(np.int32)   # the upper half receives nothing
+        x = rng.standard_normal((n, plan.d_in, plan.n_channels)).astype(np.float32)
+        y = rng.standard_normal((e, plan.d_sh)).astype(np.float32)
+        w = rng.standard_normal((e, plan.n_paths, plan.n_channels)).astype(np.float32)
+        g = rng.standard_normal((n, plan.d_out, plan.n_channels)).astype(np.float32)
+        ds, dr = _cuda(snd), _cuda(rcv)
+        sched = e3j.e3j_bwd_schedule_build(plan, n, ds, dr)
+        gx, gy, gw = e3j.e3j_conv_bwd_scheduled(plan, _cuda(x), _cuda(y), _cuda(w), sched, _cuda(g))
+        px, py, pw = e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), ds, dr, _cuda(g))
+        torch.cuda.synchronize()
+        assert e3j.e3j_plan_device_status(plan) == 0
+        assert torch.equal(gy, py) and torch.equal(gw, pw)
+        scale = max(float(px.abs().max()), 1e-30)
+        assert float((gx - px).abs().max()) <= 2e-6 * scale, (n, e)
