@@ -84,6 +84,11 @@ enum {
  * kernels where a collapsed signature has been generated (the water-box signature), the table-driven kernels
  * otherwise. */
 #define E3J_PLAN_COLLAPSE_OUTPUTS 2u
+/* e3j_conv_radial_fwd / e3j_conv_radial_vec_fwd take the two-step form (edge weights written to the workspace by the
+ * tensor-core product, then the plain forward) even where the plan has the kernel that forms them itself: faster
+ * where the [n_edges, P, N_q] array fits in memory (bench workload: 0.49 against 0.71 ms), at the price of that
+ * array in the workspace. */
+#define E3J_PLAN_RADIAL_MATERIALISE 4u
 
 typedef struct e3j_plan e3j_plan; /* opaque; immutable after creation; usable from several streams */
 

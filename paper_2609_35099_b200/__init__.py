@@ -27,11 +27,12 @@ __all__ = [
     "e3j_conv_radial_fwd", "e3j_conv_radial_bwd", "e3j_conv_radial_vec_fwd", "e3j_conv_radial_vec_fwd_workspace_bytes", "e3j_conv_radial_vec_bwd", "e3j_conv_radial_vec_bwd_workspace_bytes",
     "e3j_tp_fwd", "e3j_tp_bwd", "e3j_bwd_schedule_bytes", "e3j_bwd_schedule_build", "e3j_conv_bwd_scheduled", "e3j_harmonics_fwd", "e3j_harmonics_bwd", "e3j_conv_vec_fwd", "e3j_conv_vec_bwd",
     "e3j_conv_vec_fwd_workspace_bytes", "e3j_conv_vec_bwd_workspace_bytes", "e3j_conv_fwd_f64", "e3j_conv_bwd_f64", "e3j_shard_prepare", "e3j_rows_gather", "e3j_rows_add", "e3j_status_string", "e3j_selftest_bounded_wait", "e3j_launch_count", "E3J_PLAN_GENERIC_ONLY",
-    "E3J_PLAN_COLLAPSE_OUTPUTS",
+    "E3J_PLAN_COLLAPSE_OUTPUTS", "E3J_PLAN_RADIAL_MATERIALISE",
 ]
 
 E3J_PLAN_GENERIC_ONLY = 1
 E3J_PLAN_COLLAPSE_OUTPUTS = 2
+E3J_PLAN_RADIAL_MATERIALISE = 4
 # status codes of include/e3j.h
 E3J_OK, E3J_ERR_INVALID_ARG, E3J_ERR_BAD_IRREPS, E3J_ERR_MUL_NOT_UNIFORM = 0, -1, -2, -3
 E3J_ERR_UNSUPPORTED, E3J_ERR_WORKSPACE, E3J_ERR_CUDA, E3J_ERR_GRAPH = -4, -5, -6, -7

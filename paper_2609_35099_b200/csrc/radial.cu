@@ -107,6 +107,7 @@ namespace {
 
 // Does the plan have a kernel that forms the edge scalars itself, for this hidden width?
 const FastKernels* fused_forward(const e3j_plan* plan, int H) {
+    if (plan->flags & E3J_PLAN_RADIAL_MATERIALISE) return nullptr;
     const FastKernels* fk = fast_lookup(plan);
     return (fk && fk->radial_fwd && fk->fwd_scratch_bytes && H % 8 == 0 && H <= fast::kMaxHidden) ? fk : nullptr;
 }

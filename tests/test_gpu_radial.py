@@ -108,6 +108,7 @@ def run_radial_parity(wl, plan, cp, x, y, h, W, g, prepared=True):
     (2, 192, 64, 0),
     (2, 648, 64, 0),
     (2, 192, 64, e3j.E3J_PLAN_GENERIC_ONLY),
+    (2, 648, 64, e3j.E3J_PLAN_RADIAL_MATERIALISE),   # two-step form although the plan has the in-kernel one
     (3, 300, 64, 0),
     (5, 3000, 32, 0),
 ])
