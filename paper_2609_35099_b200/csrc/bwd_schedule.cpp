@@ -63,24 +63,50 @@ int build_bwd_schedule(int T, int n_ranges, int64_t n_nodes, int64_t n_edges, co
     std::vector<std::vector<int32_t>> col((size_t)T);
     for (int c = 0; c < n_ranges; ++c) {
         base.clear();
+        for (auto& v : col) v.clear();
+        // Columns run on from step to step (no padding to the step's fullest column): a tile may hold edges of two
+        // neighbouring steps, i.e. of up to kSchedWindow + 1 receivers, which is what the slots hold.  What must
+        // not happen is a receiver sharing a tile (or the kSchedStages tiles before it) with the previous occupant
+        // of its slot: the rows of a step start no earlier than that.
+        std::vector<int64_t> last_row;   // last row (tile of the range) that uses receiver r_first + i
+        const int32_t r_first = (run_pos < runs.size() && runs[run_pos].range == c) ? runs[run_pos].start : 0;
+        auto last_row_of = [&](int32_t r) -> int64_t {
+            const int64_t i = (int64_t)r - r_first;
+            return (i >= 0 && i < (int64_t)last_row.size()) ? last_row[i] : -1;
+        };
         while (run_pos < runs.size() && runs[run_pos].range == c) {
             size_t end = run_pos;
-            while (end < runs.size() && runs[end].range == c && runs[end].start == runs[run_pos].start) ++end;
+            const int32_t k = runs[run_pos].start;
+            while (end < runs.size() && runs[end].range == c && runs[end].start == k) ++end;
+            int64_t guard = 0;
+            for (int q = k; q < k + kSchedWindow; ++q) {
+                const int64_t lr = last_row_of(q - kSchedSlots);
+                if (lr >= 0) guard = std::max(guard, lr + 1 + kSchedStages);
+            }
+            for (auto& v : col)
+                if ((int64_t)v.size() < guard) v.resize((size_t)guard, -1);
             std::vector<int32_t> order(end - run_pos);
             std::iota(order.begin(), order.end(), (int32_t)run_pos);
             std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return runs[a].len > runs[b].len; });
-            for (auto& v : col) v.clear();
             for (int32_t id : order) {
                 int best = 0;
                 for (int j = 1; j < T; ++j)
                     if (col[j].size() < col[best].size()) best = j;
-                for (int64_t k = run_off[id]; k < run_off[id + 1]; ++k) col[best].push_back(run_edges[k]);
+                for (int64_t kk = run_off[id]; kk < run_off[id + 1]; ++kk) {
+                    const int32_t e = run_edges[kk];
+                    const size_t i = (size_t)(receivers[e] - r_first);
+                    if (last_row.size() <= i) last_row.resize(i + 1, -1);
+                    last_row[i] = std::max<int64_t>(last_row[i], (int64_t)col[best].size());
+                    col[best].push_back(e);
+                }
             }
+            run_pos = end;
+        }
+        {
             size_t h = 0;
             for (auto& v : col) h = std::max(h, v.size());
             for (size_t i = 0; i < h; ++i)
                 for (int j = 0; j < T; ++j) base.push_back(i < col[j].size() ? col[j][i] : -1);
-            run_pos = end;
         }
         const int n_base = (int)(base.size() / T);
         // first / last use of every receiver of the range (base tile index), receivers are a contiguous id range

@@ -9,8 +9,10 @@
 // Order of a range: steps k = receivers in ascending order.  Step k holds every edge into k that no earlier step
 // took, plus the edges of the same senders into receivers k+1 .. k+window-1 (a run: one sender, consecutive
 // processing positions in one column).  The runs of a step are dealt to the T columns (= consumer warps) longest
-// first onto the least loaded column; the step is as many tiles as its fullest column has edges, empty slots
-// hold -1.  The grad_out rows of the receivers in use sit in n_slots shared-memory slots (receiver % n_slots);
+// first onto the least loaded column; the columns run on from step to step, so a tile (= one row across the
+// columns) may hold edges of two neighbouring steps, and slots are empty (-1) only where a step has to wait for a
+// grad_out slot and at the end of the range.  The grad_out rows of the receivers in use sit in n_slots
+// shared-memory slots (receiver % n_slots);
 // a row is loaded with the first tile at which its slot is free again (n_stages tiles after the last use of the
 // previous occupant), empty tiles are inserted where that is later than the row's first use.
 //
