@@ -594,7 +594,10 @@ def main():
             e3j.e3j_conv_bwd_scheduled(plan, d["x"], d["y"], d["w"], sched, d["g"], grad_x=gx, grad_sh=gy, grad_w=gw, workspace=ws_b)
         b_.record(stream)
         torch.cuda.synchronize()
-        sched_block = {"bwd_ms": a_.elapsed_time(b_) / k_s, "schedule_build_ms": build_ms,
+        sb_ms = a_.elapsed_time(b_) / k_s
+        sched_block = {"bwd_ms": sb_ms, "fwd_plus_bwd_ms": statistics.mean(fwd_ms) + sb_ms,
+                       "fwd_plus_bwd_edges_per_s": e / ((statistics.mean(fwd_ms) + sb_ms) * 1e-3),
+                       "schedule_build_ms": build_ms,
                        "schedule_build": "host (graph arrays copied to the host, order copied back), once per neighbour list",
                        "rows_written": int(hdr[5]), "edges_per_row": e / max(int(hdr[5]), 1), "tiles": int(hdr[4]),
                        "note": "e3j_conv_bwd_scheduled: same gradients, grad_x summed in another fixed order; "

@@ -7,8 +7,12 @@
 // edge instead of once per edge and path group, and all warps of an SM run the same instructions.
 //
 // Ring: NS tiles of up to T edges (T = number of consumer warps, warp j takes edge j of the tile).  A tile
-// never spans a receiver change, so it needs one staged row block of grad_out; the NS blocks form a ring of
-// their own that advances only when the receiver changes (the tiles in flight use at most NS - 1 of them).
+// holds the edges of at most two neighbouring receivers (one in the fused double backward), so that the last
+// tile of a receiver is filled up with the first edges of the next one instead of leaving warps idle; the
+// staged row blocks of grad_out form a ring of their own (three for two receivers per tile, NS for one) that
+// advances when the receiver changes.  With NS = 2 tiles in flight a new receiver's block must not be one that
+// the tile before reads: three blocks allow that as long as a tile that starts a new receiver right after a
+// two-receiver tile stays with that one receiver (graphs with one or two edges per receiver).
 // The producer warp cuts the tiles, issues the bulk copies (weights, sender rows, the receiver's block when
 // it is new) and contracts the A entries; the metadata it needs (receiver and sender ids, harmonics) arrives
 // two 32-edge windows ahead through 4-byte asynchronous copies.
@@ -59,13 +63,12 @@ struct Bwd1Smem {
     static constexpr size_t off_bar = 0;                                   // full[NS], empty[NS]
     static constexpr size_t off_join = off_bar + 16 * NS;                  // join[NS][T]: the CH warps of an edge
     static constexpr size_t off_abort = off_join + 8 * NS * T;
-    static constexpr size_t off_meta = up(off_abort + 4, 16);              // int[NS][4]: first edge, n_e | last << 8, block
+    static constexpr size_t off_meta = up(off_abort + 4, 16);              // int[NS][4]: first edge, n_e | last << 8, block a | block b << 8 | edges of a << 16
     static constexpr size_t off_rcv = off_meta + 16 * NS;                  // int[2 * WIN]
     static constexpr size_t off_snd = off_rcv + 4 * 2 * WIN;               // int[2 * WIN]
     static constexpr size_t off_y = off_snd + 4 * 2 * WIN;                 // float[2 * WIN][DSH]
     static constexpr size_t off_uy = off_y + 4 * 2 * WIN * S::DSH;         // float[2 * WIN][DSH] (DBL)
     static constexpr size_t off_dm = up(off_uy + (DBL ? 4 * 2 * WIN * S::DSH : 0), 128);  // float[NS][D][NQ] (graph calls)
-    static constexpr size_t off_stage = up(off_dm + (ROWS ? 0 : 4 * (size_t)NS * DM_ROW), 128);
     static constexpr int NIN = DBL ? 2 : 1;         // copies of every per-edge input (DBL: primal and cotangent)
     static constexpr size_t st_s = 0;
     static constexpr size_t st_us = st_s + 4 * (size_t)T * S_EDGE;               // (DBL)
@@ -76,6 +79,14 @@ struct Bwd1Smem {
     static constexpr size_t st_dy = st_A + 4 * (size_t)NIN * T * S::B_APAD;      // float[T][CH][16] (CH > 1)
     static constexpr size_t st_dm = up(st_dy + (CH > 1 ? 4 * (size_t)T * CH * 16 : 0), 128);   // float[T][D][NQ] (ROWS)
     static constexpr size_t stage_bytes = up(st_dm + (ROWS ? 4 * (size_t)T * DM_ROW : 0), 128);
+    // Receivers a tile may hold and staged grad_out row blocks: two receivers per tile need three blocks (see the
+    // head of this file); signatures whose rows are too large for a third block keep one receiver per tile.
+    static constexpr size_t total_with(int nd) {
+        return up(off_dm + (ROWS ? 0 : 4 * (size_t)nd * DM_ROW), 128) + NS * stage_bytes;
+    }
+    static constexpr int MAXR = (!ROWS && !DBL && NS == 2 && T < 29 && total_with(3) + 1024 <= 228 * 1024) ? 2 : 1;
+    static constexpr int ND = MAXR == 2 ? 3 : NS;
+    static constexpr size_t off_stage = up(off_dm + (ROWS ? 0 : 4 * (size_t)ND * DM_ROW), 128);
     static constexpr size_t total = off_stage + NS * stage_bytes;
 };
 
@@ -102,7 +113,8 @@ __device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char*
     while (my_tiles > 0) {
         if (!mbar_wait(&full[stage], phase, abort_flag, p.status)) break;
         const int* meta = reinterpret_cast<const int*>(smem + L::off_meta) + 4 * stage;
-        const int first = meta[0], n_e = meta[1] & 0xff, last = meta[1] >> 8, block = meta[2];
+        const int first = meta[0], n_e = meta[1] & 0xff, last = meta[1] >> 8;
+        const int block = j < (meta[2] >> 16) ? (meta[2] & 0xff) : ((meta[2] >> 8) & 0xff);   // this edge's receiver
         if (j < n_e) {
             const unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
             const int64_t e = e_begin + first + j;
@@ -217,7 +229,8 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
     }
     int wbase = 0;               // windows wbase and wbase + 1 are in the ring or on their way
     int done = 0;                // edges handed out so far
-    int block = NS - 1;          // ring position of the current receiver's grad_out block
+    int block = L::ND - 1;       // ring position of the current receiver's grad_out block
+    bool prev_second = false;    // the tile before held edges of two receivers
     int last_rcv = -1;
     int stage = 0, phase = 0, armed = 0;
 #pragma unroll 1
@@ -229,32 +242,47 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
         // the newest group may stay in flight unless this tile reaches into it
         if ((done & 31) + T > WIN) cp_async_wait<0>(); else cp_async_wait<1>();
         __syncwarp();
-        // the tile: edges done .. done + n_e - 1, all of one receiver (ROWS: the next T rows)
+        // the tile: edges done .. done + n_e - 1 of at most MAXR receivers (ROWS: the next T rows)
         const int i = done + lane;
-        int r0 = -1, n_e;
+        int r0 = -1, r1 = -1, n_e, n_a = 0;   // n_a: edges of the first receiver
         if (ROWS) {
             n_e = min(T, n_tot - done);
         } else {
             const int r = (lane < T && i < n_tot) ? rcv_ring[i & (2 * WIN - 1)] : -2;
             r0 = __shfl_sync(0xffffffffu, r, 0);
             const unsigned differs = __ballot_sync(0xffffffffu, r != r0);   // lane T always differs
-            n_e = n_tot > 0 ? __ffs((int)differs) - 1 : 0;
+            n_a = n_tot > 0 ? __ffs((int)differs) - 1 : 0;
+            n_e = n_a;
+            // fill up with the next receiver's edges -- unless that receiver's row block would land on one that the
+            // tile before (still in flight) reads: the case when that tile held two receivers and this one starts a third
+            if (L::MAXR == 2 && n_a > 0 && n_a < T && done + n_a < n_tot && !(prev_second && r0 != last_rcv)) {
+                r1 = __shfl_sync(0xffffffffu, r, n_a);
+                const unsigned differs2 = __ballot_sync(0xffffffffu, lane >= n_a && r != r1);
+                n_e = __ffs((int)differs2) - 1;
+            }
         }
         const int last = done + n_e >= n_tot;
         // phase of `empty` that ends the previous use of this ring slot
         if (t >= NS && !mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status)) break;
         const bool new_block = !ROWS && n_e > 0 && r0 != last_rcv;
         if (new_block) {
-            block = block + 1 == NS ? 0 : block + 1;
+            block = block + 1 == L::ND ? 0 : block + 1;
             last_rcv = r0;
         }
+        const int block_a = block;
+        const bool second = r1 >= 0;   // the tile goes on into the next receiver: its block is new by definition
+        if (second) {
+            block = block + 1 == L::ND ? 0 : block + 1;
+            last_rcv = r1;
+        }
+        prev_second = second;
         unsigned char* st = smem + L::off_stage + stage * (int)L::stage_bytes;
         if (lane == 0) {
             int* meta = reinterpret_cast<int*>(smem + L::off_meta) + 4 * stage;
-            meta[0] = done; meta[1] = n_e | (last << 8); meta[2] = block;
+            meta[0] = done; meta[1] = n_e | (last << 8); meta[2] = block_a | (block << 8) | (n_a << 16);
             // arrival and byte count in one step: the phase cannot complete before the bytes are expected
             mbar_arrive_expect_tx(&full[stage], (uint32_t)n_e * 4u * (L::NIN * (L::S_EDGE + L::X_EDGE) + (ROWS ? L::DM_ROW : 0)) +
-                                                    (new_block ? 4u * L::DM_ROW : 0u));
+                                                    ((new_block ? 4u : 0u) + (second ? 4u : 0u)) * L::DM_ROW);
             if (n_e > 0)
                 bulk_g2s(st + L::st_s, p.w + (size_t)(e_begin + done) * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE,
                          &full[stage]);
@@ -277,8 +305,11 @@ __device__ __forceinline__ void bwd1_producer(const BwdParams& p, unsigned char*
             if (DBL && lane == 30 && n_e > 0)
                 bulk_g2s(st + L::st_us, p.ct_w + (size_t)(e_begin + done) * L::S_EDGE, (uint32_t)n_e * 4u * L::S_EDGE,
                          &full[stage]);
+            if (lane == 29 && second)
+                bulk_g2s(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW, p.grad_out + (size_t)r1 * L::DM_ROW,
+                         4u * L::DM_ROW, &full[stage]);
             if (lane == 31 && new_block)
-                bulk_g2s(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW, p.grad_out + (size_t)r0 * L::DM_ROW,
+                bulk_g2s(smem + L::off_dm + (size_t)block_a * 4 * L::DM_ROW, p.grad_out + (size_t)r0 * L::DM_ROW,
                          4u * L::DM_ROW, &full[stage]);
         }
         armed = t + 1;
