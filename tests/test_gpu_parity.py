@@ -736,6 +736,68 @@ def test_config5_full_size_sampled():
     assert float((gx - gx_plain).abs().max()) <= 2e-6 * float(gx_plain.abs().max())
 
 
+def _assert_blockwise_close_on_device(got, want, blocks, tol=1e-5, what=""):
+    """parity_util.assert_blockwise_close for a CUDA tensor and a float64 oracle array, evaluated on the GPU (the
+    host version spends seconds per gigabyte on conversions)."""
+    w = torch.from_numpy(np.ascontiguousarray(want)).to(DEV)
+    assert tuple(got.shape) == tuple(w.shape), (what, got.shape, w.shape)
+    assert bool(torch.isfinite(got).all()), what
+    for lo, hi in blocks:
+        gb, wb = got[:, lo:hi].double(), w[:, lo:hi]
+        if wb.numel() == 0:
+            continue
+        scale, err = float(wb.abs().max()), float((gb - wb).abs().max())
+        assert err <= tol * scale, f"{what} block {lo}:{hi}: err {err:.3e} > {tol} * {scale:.3e}"
+
+
+def test_config5_full_size_every_element():
+    """Config 5 at full size, every output element: the receivers are taken in chunks of 2500, every chunk's edges
+    go to the oracle with locally renumbered nodes; out, grad_w and grad_sh are compared chunk by chunk, grad_x is
+    accumulated over the chunks in float64 and compared at the end (about a minute of host time)."""
+    c = workloads.CONFIGS[5]
+    wl = workloads.make_graph(5)
+    n, e = wl.n_nodes, wl.n_edges
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], None, c["out_lmax"])
+    cp = oconv.Coupling(c["irreps_in"], c["sh_lmax"], None, c["out_lmax"])
+    rng = np.random.Generator(np.random.PCG64([5, 2]))
+    x = rng.standard_normal((n, plan.d_in, plan.n_channels), dtype=np.float32)
+    y = workloads.edge_harmonics(wl)
+    dx_, dy_ = _cuda(x), _cuda(y)
+    dw_ = _seeded_normal((e, plan.n_paths, plan.n_channels), 61)
+    dg_ = _seeded_normal((n, plan.d_out, plan.n_channels), 62)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    rowptr, perm, colptr = e3j.e3j_graph_prepare(n, snd, rcv)
+    out = e3j.e3j_conv_fwd(plan, dx_, dy_, dw_, snd, rcv, rowptr)
+    gx, gy, gw = e3j.e3j_conv_bwd(plan, dx_, dy_, dw_, snd, rcv, dg_, rowptr, perm, colptr)
+    torch.cuda.synchronize()
+    assert e3j.e3j_plan_device_status(plan) == 0
+    rp = rowptr.cpu().numpy()
+    g_host = dg_.cpu().numpy()
+    out_blocks, w_blocks, sh_blocks = (blocks_of_paths(cp.paths, k) for k in ("out", "w", "sh"))
+    ref_gx = np.zeros((n, plan.d_in, plan.n_channels))
+    step = 2500
+    for b0 in range(0, n, step):
+        b1 = min(n, b0 + step)
+        e0, e1 = int(rp[b0]), int(rp[b1])
+        s_ids, r_ids = wl.senders[e0:e1], wl.receivers[e0:e1]
+        nodes, local = np.unique(np.concatenate([s_ids, np.arange(b0, b1)]), return_inverse=True)
+        l_snd = local[:e1 - e0].astype(np.int32)
+        pos = np.searchsorted(nodes, np.arange(b0, b1))            # local ids of the chunk's receivers (ascending)
+        l_rcv = pos[r_ids - b0].astype(np.int32)
+        # the oracle wants receivers non-decreasing in its own numbering: local ids of b0..b1-1 ascend with b
+        xs = x[nodes]
+        gs = np.zeros((len(nodes), plan.d_out, plan.n_channels), np.float32)
+        gs[pos] = g_host[b0:b1]
+        ws = dw_[e0:e1].cpu().numpy()
+        ref = oconv.conv_fwd(cp, xs, y[e0:e1], ws, l_snd, l_rcv)
+        _assert_blockwise_close_on_device(out[b0:b1], ref[pos], out_blocks, what=f"out[{b0}:{b1}]")
+        rx, ry, rw = oconv.conv_bwd(cp, xs, y[e0:e1], ws, l_snd, l_rcv, gs)
+        _assert_blockwise_close_on_device(gw[e0:e1], rw, w_blocks, what=f"grad_w[{e0}:{e1}]")
+        _assert_blockwise_close_on_device(gy[e0:e1], ry, sh_blocks, what=f"grad_sh[{e0}:{e1}]")
+        ref_gx[nodes] += rx
+    _assert_blockwise_close_on_device(gx, ref_gx, blocks_of_paths(cp.paths, "x"), what="grad_x")
+
+
 def test_tensor_product_full_size_sampled():
     """Config 4 at 2^20 rows (75 GB of forward I/O); sampled rows against the oracle."""
     c = workloads.CONFIGS[4]
