@@ -29,7 +29,7 @@ struct BwdParams {
     const float* vec;                  // (forward only; always null here)
     const int32_t* senders; const int32_t* receivers;
     const float* grad_out;
-    float* grad_sh; float* grad_w;
+    float* grad_sh; float* grad_w;     // grad_sh may be null: computed all the same, not stored
     float* dx_edge;                    // scratch [E][d][N_q]
     int64_t n_nodes, n_edges, chunk;   // chunk = edges per CTA
     int32_t* status;
@@ -172,7 +172,7 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
                 float sum = 0.f;
 #pragma unroll
                 for (int w2 = 0; w2 < NCONS; ++w2) sum += dyp[(buf * NCONS + w2) * L::DYP + lane];
-                p.grad_sh[(size_t)e * S::DSH + lane] = sum;
+                if (p.grad_sh) p.grad_sh[(size_t)e * S::DSH + lane] = sum;
             }
             buf ^= 1;
         }

@@ -141,7 +141,7 @@ __device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char*
             const float dy_tot = reduce16_over_lanes(dyl, lane);
             const int idx = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
             if constexpr (CH == 1) {
-                if ((lane & 1) == 0 && idx < S::DSH) p.grad_sh[(size_t)e * S::DSH + idx] = dy_tot;
+                if ((lane & 1) == 0 && idx < S::DSH && p.grad_sh) p.grad_sh[(size_t)e * S::DSH + idx] = dy_tot;
             } else {
                 float* dyx = const_cast<float*>(reinterpret_cast<const float*>(st + L::st_dy)) + j * CH * 16;
                 if ((lane & 1) == 0) dyx[c * 16 + idx] = dy_tot;
@@ -153,7 +153,7 @@ __device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char*
                         float sum = 0.f;
 #pragma unroll
                         for (int c2 = 0; c2 < CH; ++c2) sum += dyx[c2 * 16 + lane];
-                        p.grad_sh[(size_t)e * S::DSH + lane] = sum;
+                        if (p.grad_sh) p.grad_sh[(size_t)e * S::DSH + lane] = sum;
                     }
                 }
                 join_phase ^= 1u << stage;   // (a short tile leaves the barriers of its unused edge slots alone)

@@ -158,6 +158,7 @@ int launch_bwd(const ConvArgs& a) {
                                                               reinterpret_cast<float4*>(a.grad_w), a.grad_sh);
         if (int s = after_launch()) return s;
     }
+    if (!a.grad_x) return E3J_OK;   // the shares stay in the scratch
     // one CTA per sender: the hardware hands them out as CTAs finish, so uneven degrees do not leave a tail
     const int64_t blocks = std::min<int64_t>(a.n_nodes, (int64_t)1 << 30);
     return launch_dependent(bwd_dx_reduce_kernel, dim3((int)blocks), dim3(S::DIN * S::NQ / 4), 0, a.stream, a.n_nodes, S::DIN * S::NQ / 4,

@@ -857,3 +857,22 @@ def test_float64_entry_points(config, n_atoms, collapse):
     assert_blockwise_close(gx.cpu().numpy(), rx, blocks_of_paths(cp.paths, "x"), tol=1e-12, what="f64 grad_x")
     assert_blockwise_close(gy.cpu().numpy(), ry, blocks_of_paths(cp.paths, "sh"), tol=1e-12, what="f64 grad_sh")
     assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), tol=1e-12, what="f64 grad_w")
+
+
+def test_backward_without_grad_sh_or_grad_x_takes_the_specialised_sweep():
+    """Leaving grad_sh and / or grad_x out must not change the gradients that are asked for (same kernel, the store
+    or the sender sum skipped): bit-identical to the full call, with the launches of the specialised path."""
+    wl, plan, cp, x, y, w, g = make_case(2, 192)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    graph = e3j.e3j_graph_prepare(wl.n_nodes, snd, rcv)
+    d = [_cuda(a) for a in (x, y, w, g)]
+    full = e3j.e3j_conv_bwd(plan, d[0], d[1], d[2], snd, rcv, d[3], *graph)
+    l0 = e3j.e3j_launch_count()
+    no_sh = e3j.e3j_conv_bwd(plan, d[0], d[1], d[2], snd, rcv, d[3], *graph, grad_sh=False)
+    assert e3j.e3j_launch_count() - l0 == 2
+    l0 = e3j.e3j_launch_count()
+    only_w = e3j.e3j_conv_bwd(plan, d[0], d[1], d[2], snd, rcv, d[3], *graph, grad_sh=False, grad_x=False)
+    assert e3j.e3j_launch_count() - l0 == 1
+    torch.cuda.synchronize()
+    assert no_sh[1] is None and torch.equal(no_sh[0], full[0]) and torch.equal(no_sh[2], full[2])
+    assert only_w[0] is None and only_w[1] is None and torch.equal(only_w[2], full[2])
