@@ -200,9 +200,8 @@ int e3j_noalloc_status(int32_t* status);
 
 /* Convolution backward.  grad_out [n_nodes,D,N_q]; grad_x [n_nodes,d,N_q],
  * grad_sh [n_edges,d'], grad_w [n_edges,P,N_q]; any of the three may be NULL (not
- * returned; plans with signature-specialised kernels keep their one sweep as long as
- * grad_w is asked for and skip the store of grad_sh / the sender sum of grad_x, a call
- * without grad_w runs on the table-driven kernels).  rowptr, sender_perm, colptr as produced by e3j_graph_prepare, or NULL
+ * returned; plans with signature-specialised kernels keep their one sweep and skip the
+ * stores of grad_sh / grad_w and the sender sum of grad_x).  rowptr, sender_perm, colptr as produced by e3j_graph_prepare, or NULL
  * (then derived into the workspace on every call).  A node that sends nothing gets
  * a zero grad_x row. */
 size_t e3j_conv_bwd_workspace_bytes(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges);

@@ -407,9 +407,9 @@ int e3j::conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, c
         sender_perm = pm; colptr = cp;
     }
     const FastKernels* fk = fast_lookup(plan);
-    // the specialised sweep produces all three cotangents at once: grad_sh and grad_x may be left out (computed, not
-    // stored / not summed); a call without grad_w uses the table-driven kernels
-    if (fk && fk->conv_bwd && n_edges > 0 && grad_w) {
+    // the specialised sweep produces all three cotangents at once; those that are not asked for are computed all the
+    // same and not stored (grad_sh, grad_w) or not summed (grad_x)
+    if (fk && fk->conv_bwd && n_edges > 0 && (grad_x || grad_sh || grad_w)) {
         DeviceTables t;
         if (int s = get_device_tables(plan, t)) return s;
         ConvArgs a{};

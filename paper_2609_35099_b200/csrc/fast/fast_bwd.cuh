@@ -141,7 +141,7 @@ __device__ __forceinline__ void bwd_consumer(const BwdParams& p, unsigned char* 
             mask >>= 1;
             Vec dxp[S::DIN];   // both are assigned (not accumulated into) by bwd_edge
             float dyl[16];
-            Vec* gw = reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + vlane;
+            Vec* gw = p.grad_w ? reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + vlane : nullptr;   // null: not wanted
             S::bwd_edge(G, dm, xs, ss, As, dxp, dyl, gw);
             xs += L::X_EDGE / S::BV; ss += L::S_EDGE / S::BV; As += S::B_APAD;
 

@@ -125,7 +125,7 @@ __device__ __forceinline__ void bwd1_consumer(const BwdParams& p, unsigned char*
                                    : reinterpret_cast<const Vec*>(smem + L::off_dm + (size_t)block * 4 * L::DM_ROW)) + vlane;
             Vec dxp[S::DIN];   // both are assigned (not accumulated into) by bwd_edge_all
             float dyl[16];
-            Vec* gw = reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + vlane;
+            Vec* gw = p.grad_w ? reinterpret_cast<Vec*>(p.grad_w + (size_t)e * L::S_EDGE) + vlane : nullptr;   // null: not wanted
             if constexpr (DBL) {
                 const Vec* uxs = reinterpret_cast<const Vec*>(st + L::st_ux) + j * (L::X_EDGE / VW) + vlane;
                 const Vec* uss = reinterpret_cast<const Vec*>(st + L::st_us) + j * (L::S_EDGE / VW) + vlane;

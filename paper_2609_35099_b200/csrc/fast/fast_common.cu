@@ -40,7 +40,8 @@ __global__ void bwd_zero_padding_kernel(const int32_t* __restrict__ n_real, int6
     const int64_t first = min((int64_t)*n_real, n_edges);
     const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int64_t e = first + blockIdx.x; e < n_edges; e += gridDim.x) {
-        for (int i = threadIdx.x; i < w_row_f4; i += blockDim.x) grad_w[(size_t)e * w_row_f4 + i] = z;
+        if (grad_w)
+            for (int i = threadIdx.x; i < w_row_f4; i += blockDim.x) grad_w[(size_t)e * w_row_f4 + i] = z;
         if (grad_sh)
             for (int i = threadIdx.x; i < sh_row; i += blockDim.x) grad_sh[(size_t)e * sh_row + i] = 0.f;
     }

@@ -374,7 +374,7 @@ class Sig:
                 F, M = self.ops("bwd"); o.append(f"            BVec ds{k} = {M}(x{first}, u{k}_{first});")
                 for i1 in used[1:]:
                     F, M = self.ops("bwd"); o.append(f"            {F}(ds{k}, x{i1}, u{k}_{i1});")
-                o.append(f"            gw[{k} * NQV] = ds{k};")
+                o.append(f"            if (gw) gw[{k} * NQV] = ds{k};")
                 for i1 in used:
                     if i1 in dx_touched:
                         F, M = self.ops("bwd"); o.append(f"            {F}(dxp[{i1}], s{k}, u{k}_{i1});")
@@ -451,7 +451,7 @@ class Sig:
             F, M = self.ops("bwd"); o.append(f"        EVec ds{k} = {M}(x{first}, u{k}_{first});")
             for i1 in used[1:]:
                 F, M = self.ops("bwd"); o.append(f"        {F}(ds{k}, x{i1}, u{k}_{i1});")
-            o.append(f"        gw[{k} * NQV] = ds{k};")
+            o.append(f"        if (gw) gw[{k} * NQV] = ds{k};")
             for i1 in used:
                 if i1 in dx_touched:
                     F, M = self.ops("bwd"); o.append(f"        {F}(dxp[{i1}], s{k}, u{k}_{i1});")
@@ -524,7 +524,7 @@ class Sig:
             F, M = self.ops("bwd2"); o.append(f"        DVec ds{k} = {M}(ux{first}, v{k}_{first}); {F}(ds{k}, x{first}, w{k}_{first});")
             for i1 in used[1:]:
                 F, M = self.ops("bwd2"); o.append(f"        {F}(ds{k}, ux{i1}, v{k}_{i1}); {F}(ds{k}, x{i1}, w{k}_{i1});")
-            o.append(f"        gw[{k} * NQV] = ds{k};")
+            o.append(f"        if (gw) gw[{k} * NQV] = ds{k};")
             for i1 in used:
                 if i1 in dx_touched:
                     F, M = self.ops("bwd2"); o.append(f"        {F}(dxp[{i1}], us{k}, v{k}_{i1}); {F}(dxp[{i1}], s{k}, w{k}_{i1});")

@@ -876,3 +876,8 @@ def test_backward_without_grad_sh_or_grad_x_takes_the_specialised_sweep():
     torch.cuda.synchronize()
     assert no_sh[1] is None and torch.equal(no_sh[0], full[0]) and torch.equal(no_sh[2], full[2])
     assert only_w[0] is None and only_w[1] is None and torch.equal(only_w[2], full[2])
+    l0 = e3j.e3j_launch_count()
+    no_w = e3j.e3j_conv_bwd(plan, d[0], d[1], d[2], snd, rcv, d[3], *graph, grad_w=False)
+    assert e3j.e3j_launch_count() - l0 == 2
+    torch.cuda.synchronize()
+    assert no_w[2] is None and torch.equal(no_w[0], full[0]) and torch.equal(no_w[1], full[1])
