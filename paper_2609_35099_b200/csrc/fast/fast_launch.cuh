@@ -82,7 +82,7 @@ template <class S>
 int launch_tp_bwd(int64_t rows, const float* x1, const float* x2, const float* w, const float* g, float* gx1,
                   float* gx2, float* gw, cudaStream_t st) {
     using L = BwdSmem<S>;
-    if (!gx1 || !gx2 || !gw) return E3J_ERR_UNSUPPORTED;  // caller falls back to the generic kernels
+    if (!gx1) return E3J_ERR_UNSUPPORTED;  // (the row's share of grad_x1 is stored unconditionally) caller falls back to the generic kernels
     constexpr bool kRowwise = S::ETR > 0;   // one warp per row, one CTA per SM (fast_bwd1.cuh)
     const int n_cta = sm_count() * (kRowwise ? 1 : S::BC);
     BwdParams p{};
