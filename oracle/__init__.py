@@ -10,7 +10,12 @@ Modules
 -------
 cg    Clebsch-Gordan coefficients from the Racah closed form, the change to the
       real basis, the canonical sign, path enumeration, dense coupling tensor.
-sh    Real spherical harmonics of any degree from the complex definition.
+sh    Real spherical harmonics of any degree from the complex definition; of edge
+      vectors (direction only) and their vector-Jacobian product by central
+      differences in float64.
 conv  Naive edge loops (plain C, fp64) for the convolution forward / backward
-      and the standalone channelwise tensor product.
+      and the standalone channelwise tensor product; on top of them, written
+      from their definitions: padded edge lists, collapsed output
+      multiplicities, the double backward, the radial network's last layer
+      (s = h W in float64) and the convolution on edge vectors.
 """
