@@ -122,14 +122,6 @@ def test_lmax2_signature():
     assert_blockwise_close(gx1.cpu().numpy(), rx, blocks_of_paths(cp.paths, "x"), what="tp grad_x1")
     assert_blockwise_close(gx2.cpu().numpy(), ry, blocks_of_paths(cp.paths, "sh"), what="tp grad_x2")
     assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="tp grad_w")
-    # partial requests: the same numbers for what is asked for
-    p1 = e3j.e3j_tp_bwd(plan, d[0], d[1], d[2], d[3], grad_x2=False, grad_w=False)
-    p2 = e3j.e3j_tp_bwd(plan, d[0], d[1], d[2], d[3], grad_x1=False)
-    torch.cuda.synchronize()
-    assert p1[1] is None and p1[2] is None and p2[0] is None
-    assert_blockwise_close(p1[0].cpu().numpy(), r1, blocks_of_paths(cp.paths, "x"), what="tp grad_x1 alone")
-    assert_blockwise_close(p2[1].cpu().numpy(), r2, blocks_of_paths(cp.paths, "sh"), what="tp grad_x2 without grad_x1")
-    assert_blockwise_close(p2[2].cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="tp grad_w without grad_x1")
 
 
 @pytest.mark.parametrize("irreps,lmax", [("96x0e+96x1o", 3), ("128x0e+128x1o+128x2e+128x3o", 2)])
@@ -256,6 +248,14 @@ def test_tensor_product(rows, flags):
     assert_blockwise_close(g1.cpu().numpy(), r1, blocks_of_paths(cp.paths, "x"), what="tp grad_x1")
     assert_blockwise_close(g2.cpu().numpy(), r2, blocks_of_paths(cp.paths, "sh"), what="tp grad_x2")
     assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="tp grad_w")
+    # partial requests: the same numbers for what is asked for
+    p1 = e3j.e3j_tp_bwd(plan, d[0], d[1], d[2], d[3], grad_x2=False, grad_w=False)
+    p2 = e3j.e3j_tp_bwd(plan, d[0], d[1], d[2], d[3], grad_x1=False)
+    torch.cuda.synchronize()
+    assert p1[1] is None and p1[2] is None and p2[0] is None
+    assert_blockwise_close(p1[0].cpu().numpy(), r1, blocks_of_paths(cp.paths, "x"), what="tp grad_x1 alone")
+    assert_blockwise_close(p2[1].cpu().numpy(), r2, blocks_of_paths(cp.paths, "sh"), what="tp grad_x2 without grad_x1")
+    assert_blockwise_close(p2[2].cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="tp grad_w without grad_x1")
 
 
 @pytest.mark.parametrize("flags", [0, e3j.E3J_PLAN_GENERIC_ONLY])
