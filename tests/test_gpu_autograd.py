@@ -1,0 +1,44 @@
+"""The torch.autograd wrapper returns what the direct calls return: first derivatives = e3j_conv_bwd, second
+derivatives = e3j_conv_bwd_bwd (bit-identical: same kernels, same inputs)."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+import paper_2609_35099_b200 as e3j
+from paper_2609_35099_b200 import workloads
+from paper_2609_35099_b200.autograd import Graph, conv
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _cuda(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+@pytest.mark.parametrize("config,n_atoms", [(2, 192), (1, None)])
+def test_autograd_first_and_second_order(config, n_atoms):
+    c = workloads.CONFIGS[config]
+    wl = workloads.make_graph(config, n_atoms)
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"], 0)
+    x, y, w, g = (_cuda(a) for a in workloads.make_features(wl, plan.n_paths, plan.d_out))
+    graph = Graph(wl.n_nodes, _cuda(wl.senders), _cuda(wl.receivers))
+    xs, ys, ws = (t.clone().requires_grad_(True) for t in (x, y, w))
+    out = conv(plan, graph, xs, ys, ws)
+    assert torch.equal(out, e3j.e3j_conv_fwd(plan, x, y, w, graph.senders, graph.receivers, graph.rowptr))
+    gx, gy, gw = torch.autograd.grad(out, (xs, ys, ws), grad_outputs=g, create_graph=True)
+    dx, dy, dw = e3j.e3j_conv_bwd(plan, x, y, w, graph.senders, graph.receivers, g, graph.rowptr, graph.sender_perm,
+                                  graph.colptr)
+    assert torch.equal(gx, dx) and torch.equal(gy, dy) and torch.equal(gw, dw)
+    # a loss on the gradients (what force matching does): its derivatives are the double backward
+    gen = torch.Generator(device=DEV); gen.manual_seed(3)
+    ux, uy, uw = (torch.randn(t.shape, generator=gen, device=DEV) for t in (x, y, w))
+    loss = (gx * ux).sum() + (gy * uy).sum() + (gw * uw).sum()
+    hx, hy, hw = torch.autograd.grad(loss, (xs, ys, ws))
+    _, rx, ry, rw = e3j.e3j_conv_bwd_bwd(plan, x, y, w, graph.senders, graph.receivers, g, graph.rowptr,
+                                         graph.sender_perm, graph.colptr, ux, uy, uw, gg_out=False)
+    torch.cuda.synchronize()
+    for a, b, name in ((hx, rx, "x"), (hy, ry, "sh"), (hw, rw, "w")):
+        assert float((a - b).abs().max()) <= 1e-6 * float(b.abs().max()), name
