@@ -7,7 +7,7 @@ torch = pytest.importorskip("torch")
 
 import paper_2609_35099_b200 as e3j
 from paper_2609_35099_b200 import workloads
-from paper_2609_35099_b200.autograd import Graph, conv
+from paper_2609_35099_b200.autograd import Graph, conv, conv_radial, conv_vec
 
 pytestmark = pytest.mark.gpu
 
@@ -42,3 +42,28 @@ def test_autograd_first_and_second_order(config, n_atoms):
     torch.cuda.synchronize()
     for a, b, name in ((hx, rx, "x"), (hy, ry, "sh"), (hw, rw, "w")):
         assert float((a - b).abs().max()) <= 1e-6 * float(b.abs().max()), name
+
+
+def test_autograd_radial_and_edge_vector_forms():
+    c = workloads.CONFIGS[2]
+    wl = workloads.make_graph(2, 192)
+    plan = e3j.e3j_plan_create(c["irreps_in"], c["sh_lmax"], c["irreps_out"], c["out_lmax"], 0)
+    x, y, w, g = (_cuda(a) for a in workloads.make_features(wl, plan.n_paths, plan.d_out))
+    h, W = (_cuda(a) for a in workloads.make_radial(wl, plan.n_paths, 64))
+    vec = _cuda(wl.vectors.astype(np.float32))
+    graph = Graph(wl.n_nodes, _cuda(wl.senders), _cuda(wl.receivers))
+    args = (graph.senders, graph.receivers)
+    prep = (graph.rowptr, graph.sender_perm, graph.colptr)
+    # radial layer; W frozen: its gradient is not asked for and not computed
+    xs, hs = x.clone().requires_grad_(True), h.clone().requires_grad_(True)
+    out = conv_radial(plan, graph, xs, y, hs, W)
+    gx, gh = torch.autograd.grad(out, (xs, hs), grad_outputs=g)
+    rx, _, rh, _ = e3j.e3j_conv_radial_bwd(plan, x, y, h, W, *args, g, *prep, grad_sh=False, grad_W=False)
+    assert torch.equal(gx, rx) and torch.equal(gh, rh)
+    # edge vectors
+    vs, ws = vec.clone().requires_grad_(True), w.clone().requires_grad_(True)
+    out = conv_vec(plan, graph, x, vs, ws)
+    gv, gw = torch.autograd.grad(out, (vs, ws), grad_outputs=g)
+    _, rv, rw = e3j.e3j_conv_vec_bwd(plan, x, vec, w, *args, g, *prep, grad_x=False)
+    torch.cuda.synchronize()
+    assert torch.equal(gv, rv) and torch.equal(gw, rw)
