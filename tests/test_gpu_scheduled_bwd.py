@@ -100,3 +100,32 @@ def test_scheduled_backward_on_sparse_and_empty_graphs():
         assert torch.equal(gy, py) and torch.equal(gw, pw)
         scale = max(float(px.abs().max()), 1e-30)
         assert float((gx - px).abs().max()) <= 2e-6 * scale, (n, e)
+
+
+@pytest.mark.parametrize("irreps,lmax,irreps_out,out_lmax", [
+    ("128x0e+128x1o", 3, "0e+1o+2e+3o", -1),   # natural-parity outputs
+    ("64x0e+64x1o", 3, None, 3),                # two channels per lane, ten edges per tile
+    ("128x0e+128x1o", 2, None, 2),              # nine harmonics (4-byte gathers)
+])
+def test_scheduled_backward_of_the_other_signatures(irreps, lmax, irreps_out, out_lmax):
+    wl = workloads.make_graph(2, 648)
+    plan = e3j.e3j_plan_create(irreps, lmax, irreps_out, out_lmax, 0)
+    assert e3j.e3j_bwd_schedule_bytes(plan, wl.n_nodes, wl.n_edges) > 0
+    cp = oconv.Coupling(irreps, lmax, irreps_out, None if out_lmax < 0 else out_lmax)
+    rng = np.random.default_rng(17)
+    n, e = wl.n_nodes, wl.n_edges
+    x = rng.standard_normal((n, plan.d_in, plan.n_channels)).astype(np.float32)
+    y = rng.standard_normal((e, plan.d_sh)).astype(np.float32)
+    w = rng.standard_normal((e, plan.n_paths, plan.n_channels)).astype(np.float32)
+    g = rng.standard_normal((n, plan.d_out, plan.n_channels)).astype(np.float32)
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    sched = e3j.e3j_bwd_schedule_build(plan, n, snd, rcv)
+    gx, gy, gw = e3j.e3j_conv_bwd_scheduled(plan, _cuda(x), _cuda(y), _cuda(w), sched, _cuda(g))
+    px, py, pw = e3j.e3j_conv_bwd(plan, _cuda(x), _cuda(y), _cuda(w), snd, rcv, _cuda(g))
+    torch.cuda.synchronize()
+    assert e3j.e3j_plan_device_status(plan) == 0
+    assert torch.equal(gy, py) and torch.equal(gw, pw)
+    rx, ry, rw = oconv.conv_bwd(cp, x, y, w, wl.senders, wl.receivers, g)
+    assert_blockwise_close(gx.cpu().numpy(), rx, blocks_of_paths(cp.paths, "x"), what="grad_x")
+    assert_blockwise_close(gy.cpu().numpy(), ry, blocks_of_paths(cp.paths, "sh"), what="grad_sh")
+    assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="grad_w")
