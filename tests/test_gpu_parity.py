@@ -124,10 +124,12 @@ def test_lmax2_signature():
     assert_blockwise_close(gw.cpu().numpy(), rw, blocks_of_paths(cp.paths, "w"), what="tp grad_w")
 
 
-@pytest.mark.parametrize("irreps,lmax", [("96x0e+96x1o", 3), ("128x0e+128x1o+128x2e+128x3o", 2)])
+@pytest.mark.parametrize("irreps,lmax", [("96x0e+96x1o", 3), ("128x0e+128x1o+128x2e+128x3o", 2),
+                                         ("64x0e+64x1o+64x2e", 3), ("32x0e+32x1o", 3)])
 def test_signatures_generated_with_automatic_tile_parameters(irreps, lmax):
-    """Two signatures that were not tuned by hand: the generator chose their tiles (96 channels: one channel per
-    lane and three warps per row group; four input irreps with harmonics up to l = 2: 18 paths, 64 rows)."""
+    """Signatures that were not tuned by hand: the generator chose their tiles (96 channels: one channel per lane
+    and three warps per row group; four input irreps with harmonics up to l = 2: 18 paths, 64 rows; three input
+    irreps at 64 channels: 24 paths; 32 channels: one warp covers an edge with one channel per lane)."""
     import dataclasses
     wl = dataclasses.replace(workloads.make_graph(2, 300), irreps_in=irreps, sh_lmax=lmax, out_lmax=lmax)
     plan = e3j.e3j_plan_create(irreps, lmax, None, lmax)
