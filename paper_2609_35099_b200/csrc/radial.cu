@@ -35,7 +35,9 @@ int launch_gemm(const Prob& prob, dim3 grid, cudaStream_t st, int resident_chunk
     static_assert(L::total <= 227 * 1024, "stage ring does not fit in shared memory");
     static_assert(L::res_total(kMaxResidentChunks) <= 227 * 1024, "resident operand does not fit in shared memory");
     constexpr bool kResident = ProbTraits<Prob>::A_RESIDENT;
-    constexpr size_t most = kResident ? L::res_total(kMaxResidentChunks) : L::total;
+    constexpr bool kTma = TmaTraits<Prob>::TMA;
+    static_assert(!kTma || L::tma_total <= 227 * 1024, "ring of raw boxes does not fit in shared memory");
+    constexpr size_t most = kResident ? L::res_total(kMaxResidentChunks) : kTma ? L::tma_total : L::total;
     static thread_local int attr_dev = -1;
     int dev = 0;
     E3J_CUDA_TRY(cudaGetDevice(&dev));
@@ -43,9 +45,39 @@ int launch_gemm(const Prob& prob, dim3 grid, cudaStream_t st, int resident_chunk
         E3J_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32x3_kernel<Prob>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most));
         attr_dev = dev;
     }
-    const size_t bytes = kResident ? L::res_total(resident_chunks) : L::total;
-    gemm_tf32x3_kernel<Prob><<<grid, kGemmThreads, bytes, st>>>(prob);
+    const size_t bytes = kResident ? L::res_total(resident_chunks) : most;
+    gemm_tf32x3_kernel<Prob><<<grid, gemm_threads<Prob>(), bytes, st>>>(prob);
     return after_launch();
+}
+
+// Tensor map of a row-major float32 matrix [rows][cols] with `pitch` floats between rows, fetched in boxes of
+// box_cols x box_rows.  False where the matrix does not meet the copy engine's alignment rules (the caller
+// then takes the kernel that loads through registers) or the driver has no encoder.
+using EncodeTiled = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiled tensor_map_encoder() {
+    static const EncodeTiled fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiled>(p);
+    }();
+    return fn;
+}
+bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t cols, int64_t pitch, int box_cols, int box_rows,
+              bool swizzle128) {
+    const EncodeTiled encode = tensor_map_encoder();
+    if (!encode || (reinterpret_cast<uintptr_t>(base) & 15) || (pitch & 3) || rows <= 0 || cols <= 0) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)pitch * sizeof(float)};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, elem,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
@@ -82,6 +114,10 @@ int grad_hidden(int64_t n_edges, int H, int C, const float* gs, const float* W, 
     GradHidden p{};
     p.gs = gs; p.W = W; p.gh = gh; p.n_edges = n_edges; p.H = H; p.C = C; p.status = status;
     p.chunk = round_up((n_edges + n_cta - 1) / n_cta, 128);
+    GradHiddenTma q{};
+    static_cast<GradHidden&>(q) = p;
+    if (make_map(&q.map_a, gs, n_edges, C, C, kChunkK, 128, true) && make_map(&q.map_b, W, H, C, C, kChunkK, 64, true))
+        return launch_gemm(q, dim3(n_cta, (H + 63) / 64), st);
     return launch_gemm(p, dim3(n_cta, (H + 63) / 64), st);
 }
 
@@ -97,7 +133,12 @@ int grad_layer(int64_t n_edges, int H, int C, const float* gs, const float* h, f
     GradLayer p{};
     p.gs = gs; p.h = h; p.partial = partial; p.n_edges = n_edges; p.H = H; p.C = C; p.status = status;
     p.chunk = round_up((n_edges + n_ranges - 1) / n_ranges, kChunkK);
-    if (int s = launch_gemm(p, dim3(n_cb, n_ranges, (H + 63) / 64), st)) return s;
+    GradLayerTma q{};
+    static_cast<GradLayer&>(q) = p;
+    const dim3 grid(n_cb, n_ranges, (H + 63) / 64);
+    const bool boxes = make_map(&q.map_a, gs, n_edges, C, C, 128, kChunkK, false) &&
+                       make_map(&q.map_b, h, n_edges, H, H, 64, kChunkK, false);
+    if (int s = boxes ? launch_gemm(q, grid, st) : launch_gemm(p, grid, st)) return s;
     const int blocks = (int)std::min<int64_t>((n_elems + 255) / 256, 4 * fast::sm_count());
     layer_sum_kernel<<<blocks, 256, 0, st>>>(n_ranges, n_elems, partial, gW);
     return after_launch();

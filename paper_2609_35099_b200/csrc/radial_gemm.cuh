@@ -11,6 +11,14 @@
 // of W^T for all of its edge tiles) it is converted once into a resident region of shared memory and the stage
 // ring carries the B operand alone, with more chunks of loads in flight per converter thread (Prob::PREFETCH).
 //
+// Where the operands lie in global memory with 16-byte aligned rows (Prob::TMA: the two gradient products), one more
+// warp brings them in as raw float32 boxes with tiled bulk copies (cp.async.bulk.tensor through a tensor map; rows
+// past the end of a matrix arrive as zeros), a ring of kRawStages boxes deep, and the converter warps read the boxes
+// from shared memory instead of loading from global memory: the loads in flight no longer depend on the
+// converters' registers, and they stay off the load/store pipe that the converters' shared-memory stores and the
+// tensor cores' operand reads already fill.  Boxes whose rows are 128 bytes use the 128-byte swizzle, so that the
+// eight rows a converter quarter-warp reads lie in different banks.
+//
 // A Problem type describes one product: which output tiles a CTA owns, how many K chunks a tile has, where
 // operand values come from (zero outside the matrices) and where results go.  Three instances are used:
 //   s^T      = W^T h^T      edge scalars from the hidden activations            (RadialWeights)
@@ -26,6 +34,8 @@
 // Every wait is bounded (fast::mbar_wait): on a time-out the CTA records the failure in the status word,
 // stops issuing work, lets the tensor cores drain, frees its tensor memory and returns.
 #pragma once
+#include <cuda.h>   // CUtensorMap (the type only: the encoder is looked up at run time)
+
 #include "fast/fast_common.cuh"
 #include "umma.cuh"
 
@@ -40,6 +50,8 @@ constexpr int kConvWarps = 8;     // converter warps
 constexpr int kPrefetch = 2;      // chunks of loads in flight per converter thread (Prob::PREFETCH where given)
 constexpr int kMaxResidentChunks = 4;   // K chunks of a resident A operand (Prob::A_RESIDENT): K <= 128
 constexpr int kGemmThreads = (4 + kConvWarps + 1) * 32;   // epilogue, converters, tensor-core issue
+constexpr int kStagesTma = 2;     // operand stages of the products whose inputs arrive as raw boxes (Prob::TMA) ...
+constexpr int kRawStages = 4;     // ... and their ring of raw boxes
 
 template <int N>
 struct GemmSmem {
@@ -54,6 +66,12 @@ struct GemmSmem {
     // A operand resident (converted once per CTA): [chunks][A_hi, A_lo] first, then stages of B alone
     static constexpr size_t res_stage_bytes = 2 * b_bytes;
     static constexpr size_t res_total(int chunks) { return off_stage + (size_t)chunks * 2 * a_bytes + kStages * res_stage_bytes; }
+    // raw boxes (Prob::TMA): raw_full[kRawStages], raw_empty[kRawStages] behind the other barriers; the ring starts
+    // at the first 1024-byte boundary behind the operand stages (the swizzle is a function of the address)
+    static constexpr size_t off_raw_bar = 128;
+    static constexpr size_t raw_bytes = a_bytes + b_bytes;
+    static constexpr size_t tma_total = off_stage + kStagesTma * stage_bytes + 1024 + kRawStages * raw_bytes;
+    static_assert(off_raw_bar + 16 * kRawStages <= off_stage && off_abort + 4 <= off_raw_bar, "barrier area");
 };
 
 template <class P, class = void> struct ProbTraits {
@@ -64,6 +82,17 @@ template <class P> struct ProbTraits<P, decltype((void)P::A_RESIDENT)> {
     static constexpr bool A_RESIDENT = P::A_RESIDENT;
     static constexpr int PREFETCH = P::PREFETCH;
 };
+
+template <class P, class = void> struct TmaTraits { static constexpr bool TMA = false; };
+template <class P> struct TmaTraits<P, decltype((void)P::TMA)> { static constexpr bool TMA = P::TMA; };
+template <class P> constexpr int gemm_threads() { return kGemmThreads + (TmaTraits<P>::TMA ? 32 : 0); }
+
+// One box of a rank-2 tensor map into shared memory; x is the coordinate along the contiguous dimension and must
+// be a multiple of four elements.  Completes on the barrier with the box's bytes, whatever part of it lay outside.
+__device__ __forceinline__ void tma_load_2d(void* dst_smem, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(fast::smem_u32(dst_smem)), "l"(map), "r"(x), "r"(y), "r"(fast::smem_u32(bar)) : "memory");
+}
 
 // Converters: an operand of a stage is rows [0, ROWS) x k [0, 32).  LANE_ROWS = 8: a warp item is 8 rows x 4 k-quads
 // (sources with k contiguous); LANE_ROWS = 32: 32 rows x 1 k-quad (sources with rows contiguous).  Either way 8
@@ -109,18 +138,22 @@ struct OperandItems {
 };
 
 template <class Prob>
-__global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob prob) {
+__global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(const __grid_constant__ Prob prob) {
     constexpr int N = Prob::N;
+    constexpr bool kTma = TmaTraits<Prob>::TMA;
+    constexpr int NSTAGE = kTma ? kStagesTma : kStages;
     using L = GemmSmem<N>;
     constexpr uint32_t kTmemCols = 2 * N;   // two accumulator tiles
     static_assert(kTmemCols == 128 || kTmemCols == 256, "tensor-memory allocation must be a power of two");
     extern __shared__ __align__(1024) unsigned char smem[];
     uint64_t* stage_full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
-    uint64_t* stage_empty = stage_full + kStages;
+    uint64_t* stage_empty = stage_full + kStages;   // (the barrier area is laid out for kStages whatever NSTAGE is)
     uint64_t* d_full = stage_empty + kStages;
     uint64_t* d_empty = d_full + 2;
     uint64_t* drain = d_empty + 2;
     uint64_t* a_ready = drain + 1;
+    uint64_t* raw_full = reinterpret_cast<uint64_t*>(smem + L::off_raw_bar);
+    uint64_t* raw_empty = raw_full + kRawStages;
     constexpr bool kResident = ProbTraits<Prob>::A_RESIDENT;   // A does not depend on the tile: converted once
     constexpr int kPre = ProbTraits<Prob>::PREFETCH;
     const int res_chunks = kResident ? prob.n_chunks(0) : 0;
@@ -133,6 +166,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { fast::mbar_init(&stage_full[s], kConvWarps); fast::mbar_init(&stage_empty[s], 1); }
+        if constexpr (kTma)
+            for (int s = 0; s < kRawStages; ++s) { fast::mbar_init(&raw_full[s], 1); fast::mbar_init(&raw_empty[s], kConvWarps); }
         for (int b = 0; b < 2; ++b) { fast::mbar_init(&d_full[b], 1); fast::mbar_init(&d_empty[b], 4); }
         fast::mbar_init(drain, 1);
         fast::mbar_init(a_ready, kConvWarps);
@@ -144,6 +179,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
     __syncthreads();
     umma::fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // raw boxes: behind the operand stages, at a 1024-byte boundary of the shared-memory window
+    unsigned char* const raw_ring =
+        smem + (((fast::smem_u32(stages + (size_t)NSTAGE * kStageBytes) + 1023u) & ~1023u) - fast::smem_u32(smem));
 
     const int n_tiles = prob.n_tiles();
     if (warp < 4) {
@@ -192,6 +230,31 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
             __syncwarp();
             if (lane == 0) fast::mbar_arrive(a_ready);
         }
+        if constexpr (kTma) {
+            // the operands arrive as raw boxes: read, split, store; one arrival frees the box, one fills the stage
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; ok && t < n_tiles; ++t) {
+                const int n_chunks = prob.n_chunks(t);
+#pragma unroll 1
+                for (int kc = 0; kc < n_chunks; ++kc, ++it) {
+                    const int rs = it % kRawStages, s = it % NSTAGE;
+                    if (!fast::mbar_wait(&raw_full[rs], (it / kRawStages) & 1, abort_flag, prob.status)) { ok = false; break; }
+                    const unsigned char* ra = raw_ring + (size_t)rs * L::raw_bytes;
+                    const unsigned char* rb = ra + L::a_bytes;
+                    float4 a[OA::NI], b[OB::NI];
+                    OA::load(a, cwarp, lane, [&](int row, int k) { return Prob::raw_a(ra, row, k); });
+                    OB::load(b, cwarp, lane, [&](int row, int k) { return Prob::raw_b(rb, row, k); });
+                    if (it >= NSTAGE && !fast::mbar_wait(&stage_empty[s], ((it / NSTAGE) + 1) & 1, abort_flag, prob.status)) { ok = false; break; }
+                    unsigned char* st = stages + (size_t)s * kStageBytes;
+                    OA::store(a, st, st + L::a_bytes, cwarp, lane);
+                    OB::store(b, st + kStageB, st + kStageB + L::b_bytes, cwarp, lane);
+                    umma::fence_smem_to_async();
+                    __syncwarp();   // every lane's stores are out, so every lane's reads of the box have returned
+                    if (lane == 0) { fast::mbar_arrive(&stage_full[s]); fast::mbar_arrive(&raw_empty[rs]); }
+                }
+            }
+        } else {
         float4 va[kPre][kResident ? 1 : OA::NI], vb[kPre][OB::NI];
         int tf = 0, kf = 0;                      // next chunk to fetch
         int ts = 0, ks = 0;                      // next chunk to convert and store
@@ -222,8 +285,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
                 fetch(va[u], vb[u]);             // refill this register set with the chunk kPre ahead
             }
         }
-    } else {
-        // ------------------------------------------------ tensor-core issue (lane 0 of warp 8)
+        }
+    } else if (warp == 4 + kConvWarps) {
+        // ------------------------------------------------ tensor-core issue (one lane)
         constexpr uint32_t idesc = umma::idesc_tf32(kTileM, N);
         const uint32_t sbo = umma::sbo_bytes(kChunkK);
         int it = 0;
@@ -234,8 +298,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
             const int n_chunks = prob.n_chunks(t);
             if (t >= 2 && !fast::mbar_wait(&d_empty[db], ((t >> 1) + 1) & 1, abort_flag, prob.status)) break;
             for (int kc = 0; kc < n_chunks; ++kc, ++it) {
-                const int s = it % kStages;
-                if (!fast::mbar_wait(&stage_full[s], (it / kStages) & 1, abort_flag, prob.status)) { ok = false; break; }
+                const int s = it % NSTAGE;
+                if (!fast::mbar_wait(&stage_full[s], (it / NSTAGE) & 1, abort_flag, prob.status)) { ok = false; break; }
                 umma::fence_after_sync();
                 if (lane == 0) {
                     const uint32_t st = umma::smem_addr(stages + (size_t)s * kStageBytes);
@@ -266,10 +330,53 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tf32x3_kernel(const Prob
             for (uint32_t spin = 0; spin < fast::kSpinLimit; ++spin)
                 if (fast::mbar_try_wait(drain, 0)) break;
         }
+    } else {
+        // ------------------------------------------------ raw boxes (Prob::TMA): tiled bulk copies, one lane
+        if constexpr (kTma) {
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; ok && t < n_tiles; ++t) {
+                const int n_chunks = prob.n_chunks(t);
+#pragma unroll 1
+                for (int kc = 0; kc < n_chunks; ++kc, ++it) {
+                    const int rs = it % kRawStages;
+                    if (it >= kRawStages && !fast::mbar_wait(&raw_empty[rs], ((it / kRawStages) + 1) & 1, abort_flag, prob.status)) { ok = false; break; }
+                    if (lane == 0) {
+                        unsigned char* ra = raw_ring + (size_t)rs * L::raw_bytes;
+                        int x, y;
+                        fast::mbar_arrive_expect_tx(&raw_full[rs], (uint32_t)L::raw_bytes);
+                        prob.box_a(t, kc, x, y);
+                        tma_load_2d(ra, &prob.map_a, x, y, &raw_full[rs]);
+                        prob.box_b(t, kc, x, y);
+                        tma_load_2d(ra + L::a_bytes, &prob.map_b, x, y, &raw_full[rs]);
+                    }
+                    __syncwarp();
+                }
+            }
+            // abort path only: the copies still in flight must land before the CTA gives its shared memory back
+            if (*abort_flag) {
+                for (int j = max(0, it - kRawStages); j < it; ++j) {
+#pragma unroll 1
+                    for (uint32_t spin = 0; spin < fast::kSpinLimit; ++spin)
+                        if (fast::mbar_try_wait(&raw_full[j % kRawStages], (j / kRawStages) & 1)) break;
+                }
+            }
+        }
     }
     umma::fence_before_sync();
     __syncthreads();
     if (warp == 4 + kConvWarps) umma::tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// Reads of a raw box by the converters.  Rows of 128 bytes under the 128-byte swizzle: the 16-byte piece j of
+// row r lies at piece j ^ (r % 8) of that row (the box starts at a 1024-byte boundary).
+__device__ __forceinline__ float4 raw_swizzled(const unsigned char* box, int row, int k) {
+    return *reinterpret_cast<const float4*>(box + row * 128 + ((((k >> 2) ^ row) & 7) << 4));
+}
+// Plain boxes of `pitch` floats per row, read across the rows: element (k + i, row) for i < 4.
+__device__ __forceinline__ float4 raw_transposed(const unsigned char* box, int pitch, int row, int k) {
+    const float* b = reinterpret_cast<const float*>(box) + k * pitch + row;
+    return make_float4(b[0], b[pitch], b[2 * pitch], b[3 * pitch]);
 }
 
 // ------------------------------------------------------------------------------------------------ problems
@@ -373,6 +480,19 @@ struct GradHidden {
     }
 };
 
+// the same with both operands fetched as boxes of 32 c: (128 edges of grad_s | 64 rows of W), 128-byte swizzle
+struct GradHiddenTma : GradHidden {
+    static constexpr bool TMA = true;
+    alignas(64) CUtensorMap map_a, map_b;
+    __device__ __forceinline__ int first_c(int t, int kc) const { return ((t % groups()) * kGroupChunks + kc) * kChunkK; }
+    __device__ __forceinline__ void box_a(int t, int kc, int& x, int& y) const {
+        x = first_c(t, kc); y = (int)(e_begin() + (int64_t)(t / groups()) * 128);
+    }
+    __device__ __forceinline__ void box_b(int t, int kc, int& x, int& y) const { x = first_c(t, kc); y = blockIdx.y * 64; }
+    __device__ static __forceinline__ float4 raw_a(const unsigned char* box, int row, int k) { return raw_swizzled(box, row, k); }
+    __device__ static __forceinline__ float4 raw_b(const unsigned char* box, int row, int k) { return raw_swizzled(box, row, k); }
+};
+
 // partial[r, j, c] = sum over the edges of range r of h[e, j] grad_s[e, c]: one tile per CTA,
 // m = c (column block of 128), n = j (block blockIdx.z of 64), k = edge.  grad_W = sum_r partial[r] in range
 // order (layer_sum_kernel).
@@ -425,6 +545,17 @@ struct GradLayer {
                 if (j0 + i < H) dst[(size_t)i * C] = v[i];
         }
     }
+};
+
+// the same with both operands fetched as boxes of 32 edges: (128 c of grad_s | 64 j of h), read across the rows
+struct GradLayerTma : GradLayer {
+    static constexpr bool TMA = true;
+    alignas(64) CUtensorMap map_a, map_b;
+    __device__ __forceinline__ int first_e(int t, int kc) const { return (int)(e_begin() + (int64_t)(t * kGroupChunks + kc) * kChunkK); }
+    __device__ __forceinline__ void box_a(int t, int kc, int& x, int& y) const { x = blockIdx.x * 128; y = first_e(t, kc); }
+    __device__ __forceinline__ void box_b(int t, int kc, int& x, int& y) const { x = blockIdx.z * 64; y = first_e(t, kc); }
+    __device__ static __forceinline__ float4 raw_a(const unsigned char* box, int row, int k) { return raw_transposed(box, 128, row, k); }
+    __device__ static __forceinline__ float4 raw_b(const unsigned char* box, int row, int k) { return raw_transposed(box, 64, row, k); }
 };
 
 // grad_W[j, c] = sum_r partial[r, j, c], r ascending.
