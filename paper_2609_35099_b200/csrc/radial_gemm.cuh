@@ -50,16 +50,17 @@ constexpr int kConvWarps = 8;     // converter warps
 constexpr int kPrefetch = 2;      // chunks of loads in flight per converter thread (Prob::PREFETCH where given)
 constexpr int kMaxResidentChunks = 4;   // K chunks of a resident A operand (Prob::A_RESIDENT): K <= 128
 constexpr int kGemmThreads = (4 + kConvWarps + 1) * 32;   // epilogue, converters, tensor-core issue
-constexpr int kStagesTma = 2;     // operand stages of the products whose inputs arrive as raw boxes (Prob::TMA) ...
-constexpr int kRawStages = 4;     // ... and their ring of raw boxes
+constexpr int kStagesTma = 4;     // operand stages of the products whose inputs arrive as raw boxes (Prob::TMA) ...
+constexpr int kRawStages = 5;     // ... and their ring of raw boxes
+constexpr int kMaxStages = 4;     // the barrier area holds this many stage barriers of each kind
 
 template <int N>
 struct GemmSmem {
     static constexpr size_t a_bytes = (size_t)kTileM * kChunkK * 4;   // one of hi / lo
     static constexpr size_t b_bytes = (size_t)N * kChunkK * 4;
     static constexpr size_t stage_bytes = 2 * a_bytes + 2 * b_bytes;  // A_hi, A_lo, B_hi, B_lo
-    static constexpr size_t off_bar = 0;       // stage_full[kStages], stage_empty[kStages], d_full[2], d_empty[2], drain, a_ready
-    static constexpr size_t off_tmem = 8 * (2 * kStages + 6);
+    static constexpr size_t off_bar = 0;       // stage_full[kMaxStages], stage_empty[kMaxStages], d_full[2], d_empty[2], drain, a_ready
+    static constexpr size_t off_tmem = 8 * (2 * kMaxStages + 6);
     static constexpr size_t off_abort = off_tmem + 4;
     static constexpr size_t off_stage = 1024;
     static constexpr size_t total = off_stage + kStages * stage_bytes;
@@ -70,7 +71,10 @@ struct GemmSmem {
     // at the first 1024-byte boundary behind the operand stages (the swizzle is a function of the address)
     static constexpr size_t off_raw_bar = 128;
     static constexpr size_t raw_bytes = a_bytes + b_bytes;
-    static constexpr size_t tma_total = off_stage + kStagesTma * stage_bytes + 1024 + kRawStages * raw_bytes;
+    static constexpr size_t tma_total = off_stage + kStagesTma * res_stage_bytes + 1024 + kRawStages * raw_bytes;
+    // tensor memory of those products: two accumulator tiles, then per stage the A operand as (hi | lo) of 32 k each
+    static constexpr uint32_t tma_col_a = 2 * N, tma_cols = 512;
+    static_assert(tma_col_a + kStagesTma * 2 * kChunkK <= tma_cols, "tensor memory");
     static_assert(off_raw_bar + 16 * kRawStages <= off_stage && off_abort + 4 <= off_raw_bar, "barrier area");
 };
 
@@ -143,12 +147,12 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
     constexpr bool kTma = TmaTraits<Prob>::TMA;
     constexpr int NSTAGE = kTma ? kStagesTma : kStages;
     using L = GemmSmem<N>;
-    constexpr uint32_t kTmemCols = 2 * N;   // two accumulator tiles
-    static_assert(kTmemCols == 128 || kTmemCols == 256, "tensor-memory allocation must be a power of two");
+    constexpr uint32_t kTmemCols = TmaTraits<Prob>::TMA ? L::tma_cols : 2 * N;   // two accumulator tiles (+ the A stages)
+    static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "tensor-memory allocation must be a power of two");
     extern __shared__ __align__(1024) unsigned char smem[];
     uint64_t* stage_full = reinterpret_cast<uint64_t*>(smem + L::off_bar);
-    uint64_t* stage_empty = stage_full + kStages;   // (the barrier area is laid out for kStages whatever NSTAGE is)
-    uint64_t* d_full = stage_empty + kStages;
+    uint64_t* stage_empty = stage_full + kMaxStages;
+    uint64_t* d_full = stage_empty + kMaxStages;
     uint64_t* d_empty = d_full + 2;
     uint64_t* drain = d_empty + 2;
     uint64_t* a_ready = drain + 1;
@@ -158,14 +162,15 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
     constexpr int kPre = ProbTraits<Prob>::PREFETCH;
     const int res_chunks = kResident ? prob.n_chunks(0) : 0;
     unsigned char* const stages = smem + L::off_stage + (size_t)res_chunks * 2 * L::a_bytes;
-    constexpr size_t kStageBytes = kResident ? L::res_stage_bytes : L::stage_bytes;
-    constexpr size_t kStageB = kResident ? 0 : 2 * L::a_bytes;   // where B_hi starts inside a stage
+    static_assert(!(kResident && kTma) && NSTAGE <= kMaxStages, "one way of keeping A out of the stages at a time");
+    constexpr size_t kStageBytes = (kResident || kTma) ? L::res_stage_bytes : L::stage_bytes;
+    constexpr size_t kStageB = (kResident || kTma) ? 0 : 2 * L::a_bytes;   // where B_hi starts inside a stage
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::off_tmem);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::off_abort);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { fast::mbar_init(&stage_full[s], kConvWarps); fast::mbar_init(&stage_empty[s], 1); }
+        for (int s = 0; s < kMaxStages; ++s) { fast::mbar_init(&stage_full[s], kConvWarps); fast::mbar_init(&stage_empty[s], 1); }
         if constexpr (kTma)
             for (int s = 0; s < kRawStages; ++s) { fast::mbar_init(&raw_full[s], 1); fast::mbar_init(&raw_empty[s], kConvWarps); }
         for (int b = 0; b < 2; ++b) { fast::mbar_init(&d_full[b], 1); fast::mbar_init(&d_empty[b], 4); }
@@ -231,7 +236,12 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
             if (lane == 0) fast::mbar_arrive(a_ready);
         }
         if constexpr (kTma) {
-            // the operands arrive as raw boxes: read, split, store; one arrival frees the box, one fills the stage
+            // The operands arrive as raw boxes.  A goes to tensor memory, where the tensor cores read it without
+            // touching shared memory: lane m of tensor memory is row m of the tile, and a warp reaches the 32 lanes
+            // of its quarter only, so warp w converts rows 32 (w % 4) ... and columns 16 (w / 4) ... of every
+            // chunk.  B is split into the shared-memory stage as before.
+            const int a_row = (cwarp & 3) * 32 + lane, a_k0 = (cwarp >> 2) * 16;
+            const uint32_t a_taddr = tmem_base + ((uint32_t)((cwarp & 3) * 32) << 16) + L::tma_col_a + (uint32_t)a_k0;
             int it = 0;
             bool ok = true;
             for (int t = 0; ok && t < n_tiles; ++t) {
@@ -242,13 +252,26 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
                     if (!fast::mbar_wait(&raw_full[rs], (it / kRawStages) & 1, abort_flag, prob.status)) { ok = false; break; }
                     const unsigned char* ra = raw_ring + (size_t)rs * L::raw_bytes;
                     const unsigned char* rb = ra + L::a_bytes;
-                    float4 a[OA::NI], b[OB::NI];
-                    OA::load(a, cwarp, lane, [&](int row, int k) { return Prob::raw_a(ra, row, k); });
+                    float4 a[4], b[OB::NI];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) a[i] = Prob::raw_a(ra, a_row, a_k0 + 4 * i);
                     OB::load(b, cwarp, lane, [&](int row, int k) { return Prob::raw_b(rb, row, k); });
                     if (it >= NSTAGE && !fast::mbar_wait(&stage_empty[s], ((it / NSTAGE) + 1) & 1, abort_flag, prob.status)) { ok = false; break; }
+                    umma::fence_after_sync();
+                    float hi[16], lo[16];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        float4 h4, l4;
+                        umma::split_tf32(a[i], h4, l4);
+                        hi[4 * i] = h4.x; hi[4 * i + 1] = h4.y; hi[4 * i + 2] = h4.z; hi[4 * i + 3] = h4.w;
+                        lo[4 * i] = l4.x; lo[4 * i + 1] = l4.y; lo[4 * i + 2] = l4.z; lo[4 * i + 3] = l4.w;
+                    }
+                    umma::tmem_st16(a_taddr + (uint32_t)(s * 2 * kChunkK), hi);
+                    umma::tmem_st16(a_taddr + (uint32_t)(s * 2 * kChunkK + kChunkK), lo);
                     unsigned char* st = stages + (size_t)s * kStageBytes;
-                    OA::store(a, st, st + L::a_bytes, cwarp, lane);
-                    OB::store(b, st + kStageB, st + kStageB + L::b_bytes, cwarp, lane);
+                    OB::store(b, st, st + L::b_bytes, cwarp, lane);
+                    umma::tmem_st_wait();
+                    umma::fence_before_sync();
                     umma::fence_smem_to_async();
                     __syncwarp();   // every lane's stores are out, so every lane's reads of the box have returned
                     if (lane == 0) { fast::mbar_arrive(&stage_full[s]); fast::mbar_arrive(&raw_empty[rs]); }
@@ -303,19 +326,31 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
                 umma::fence_after_sync();
                 if (lane == 0) {
                     const uint32_t st = umma::smem_addr(stages + (size_t)s * kStageBytes);
-                    const uint32_t a_hi = kResident ? umma::smem_addr(smem + L::off_stage + (size_t)kc * 2 * L::a_bytes) : st;
-                    const uint32_t a_lo = a_hi + (uint32_t)L::a_bytes;
                     const uint32_t b_hi = st + (uint32_t)kStageB, b_lo = b_hi + (uint32_t)L::b_bytes;
                     const uint32_t d = tmem_base + (uint32_t)(db * N);
                     // small terms first: a_lo b_hi, a_hi b_lo, then a_hi b_hi
-                    const uint32_t pa[3] = {a_lo, a_hi, a_hi}, pb[3] = {b_hi, b_lo, b_hi};
+                    const uint32_t pb[3] = {b_hi, b_lo, b_hi};
+                    if constexpr (kTma) {   // A in tensor memory: columns (hi | lo) of the stage
+                        const uint32_t a_hi = tmem_base + L::tma_col_a + (uint32_t)(s * 2 * kChunkK), a_lo = a_hi + kChunkK;
+                        const uint32_t pa[3] = {a_lo, a_hi, a_hi};
 #pragma unroll
-                    for (int pass = 0; pass < 3; ++pass)
+                        for (int pass = 0; pass < 3; ++pass)
 #pragma unroll
-                        for (int ks = 0; ks < kChunkK / 8; ++ks)
-                            umma::mma_tf32(d, umma::make_desc(pa[pass] + ks * 2 * umma::kLbo, umma::kLbo, sbo),
-                                           umma::make_desc(pb[pass] + ks * 2 * umma::kLbo, umma::kLbo, sbo), idesc,
-                                           (kc > 0 || pass > 0 || ks > 0) ? 1u : 0u);
+                            for (int ks = 0; ks < kChunkK / 8; ++ks)
+                                umma::mma_tf32_ts(d, pa[pass] + ks * 8, umma::make_desc(pb[pass] + ks * 2 * umma::kLbo, umma::kLbo, sbo),
+                                                  idesc, (kc > 0 || pass > 0 || ks > 0) ? 1u : 0u);
+                    } else {
+                        const uint32_t a_hi = kResident ? umma::smem_addr(smem + L::off_stage + (size_t)kc * 2 * L::a_bytes) : st;
+                        const uint32_t a_lo = a_hi + (uint32_t)L::a_bytes;
+                        const uint32_t pa[3] = {a_lo, a_hi, a_hi};
+#pragma unroll
+                        for (int pass = 0; pass < 3; ++pass)
+#pragma unroll
+                            for (int ks = 0; ks < kChunkK / 8; ++ks)
+                                umma::mma_tf32(d, umma::make_desc(pa[pass] + ks * 2 * umma::kLbo, umma::kLbo, sbo),
+                                               umma::make_desc(pb[pass] + ks * 2 * umma::kLbo, umma::kLbo, sbo), idesc,
+                                               (kc > 0 || pass > 0 || ks > 0) ? 1u : 0u);
+                    }
                     umma::commit(&stage_empty[s]);                       // the stage may be refilled
                     if (kc == n_chunks - 1) umma::commit(&d_full[db]);   // the tile is complete
                 }
