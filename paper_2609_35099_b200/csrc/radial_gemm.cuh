@@ -51,7 +51,9 @@ constexpr int kPrefetch = 2;      // chunks of loads in flight per converter thr
 constexpr int kMaxResidentChunks = 4;   // K chunks of a resident A operand (Prob::A_RESIDENT): K <= 128
 constexpr int kGemmThreads = (4 + kConvWarps + 1) * 32;   // epilogue, converters, tensor-core issue
 constexpr int kStagesTma = 4;     // operand stages of the products whose inputs arrive as raw boxes (Prob::TMA) ...
-constexpr int kRawStages = 5;     // ... and their ring of raw boxes
+constexpr int kRawStages = 6;     // ... and their ring of raw boxes (both even: a stage always meets the same converter group,
+                                  // so every waiter sees each of its barriers' phases one after the other)
+static_assert(kStagesTma % 2 == 0 && kRawStages % 2 == 0, "stages alternate between the two converter groups");
 constexpr int kMaxStages = 4;     // the barrier area holds this many stage barriers of each kind
 
 template <int N>
@@ -73,8 +75,9 @@ struct GemmSmem {
     static constexpr size_t raw_bytes = a_bytes + b_bytes;
     static constexpr size_t tma_total = off_stage + kStagesTma * res_stage_bytes + 1024 + kRawStages * raw_bytes;
     // tensor memory of those products: two accumulator tiles, then per stage the A operand as (hi | lo) of 32 k each
-    static constexpr uint32_t tma_col_a = 2 * N, tma_cols = 512;
-    static_assert(tma_col_a + kStagesTma * 2 * kChunkK <= tma_cols, "tensor memory");
+    // (an accumulator tile of those products is two: the product of the hi parts, and the two cross terms)
+    static constexpr uint32_t tma_col_a = 4 * N, tma_cols = 512;
+    static_assert(N > 64 || tma_col_a + kStagesTma * 2 * kChunkK <= tma_cols, "tensor memory");
     static_assert(off_raw_bar + 16 * kRawStages <= off_stage && off_abort + 4 <= off_raw_bar, "barrier area");
 };
 
@@ -103,16 +106,16 @@ __device__ __forceinline__ void tma_load_2d(void* dst_smem, const CUtensorMap* m
 // consecutive lanes write 128 contiguous bytes of shared memory.  The work is two halves: all loads of a chunk go
 // out first (into registers), the conversion and the stores follow one chunk later, so that the loads of chunk
 // i + 1 are in flight while chunk i is converted.
-template <int ROWS, int LANE_ROWS>
+template <int ROWS, int LANE_ROWS, int NW = kConvWarps>
 struct OperandItems {
     static constexpr int QUADS = kChunkK / 4;
     static constexpr int LANE_QUADS = 32 / LANE_ROWS;
     static constexpr int ITEMS = (ROWS / LANE_ROWS) * (QUADS / LANE_QUADS);   // warp items of the operand
     static_assert(ROWS % LANE_ROWS == 0 && QUADS % LANE_QUADS == 0, "operand does not tile");
-    static_assert(ITEMS % kConvWarps == 0, "the converter warps share the items");
-    static constexpr int NI = ITEMS / kConvWarps;
+    static_assert(ITEMS % NW == 0, "the converter warps share the items");
+    static constexpr int NI = ITEMS / NW;
     __device__ static __forceinline__ void coords(int i, int cwarp, int lane, int& row, int& k) {
-        const int item = cwarp + kConvWarps * i;
+        const int item = cwarp + NW * i;
         const int rg = item / (QUADS / LANE_QUADS), qg = item % (QUADS / LANE_QUADS);
         row = rg * LANE_ROWS + lane % LANE_ROWS;
         k = (qg * LANE_QUADS + lane / LANE_ROWS) * 4;
@@ -146,6 +149,7 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
     constexpr int N = Prob::N;
     constexpr bool kTma = TmaTraits<Prob>::TMA;
     constexpr int NSTAGE = kTma ? kStagesTma : kStages;
+    constexpr int DN = kTma ? 2 * N : N;   // tensor-memory columns of one accumulator tile
     using L = GemmSmem<N>;
     constexpr uint32_t kTmemCols = TmaTraits<Prob>::TMA ? L::tma_cols : 2 * N;   // two accumulator tiles (+ the A stages)
     static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "tensor-memory allocation must be a power of two");
@@ -170,9 +174,9 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMaxStages; ++s) { fast::mbar_init(&stage_full[s], kConvWarps); fast::mbar_init(&stage_empty[s], 1); }
+        for (int s = 0; s < kMaxStages; ++s) { fast::mbar_init(&stage_full[s], kTma ? kConvWarps / 2 : kConvWarps); fast::mbar_init(&stage_empty[s], 1); }
         if constexpr (kTma)
-            for (int s = 0; s < kRawStages; ++s) { fast::mbar_init(&raw_full[s], 1); fast::mbar_init(&raw_empty[s], kConvWarps); }
+            for (int s = 0; s < kRawStages; ++s) { fast::mbar_init(&raw_full[s], 1); fast::mbar_init(&raw_empty[s], kConvWarps / 2); }
         for (int b = 0; b < 2; ++b) { fast::mbar_init(&d_full[b], 1); fast::mbar_init(&d_empty[b], 4); }
         fast::mbar_init(drain, 1);
         fast::mbar_init(a_ready, kConvWarps);
@@ -198,8 +202,30 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
             const int db = t & 1;
             if (!fast::mbar_wait(&d_full[db], (t >> 1) & 1, abort_flag, prob.status)) break;
             umma::fence_after_sync();
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(db * N);
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(db * DN);
             const bool flush = prob.flush(t);
+            if constexpr (kTma) {
+                // two accumulators per tile: a_hi b_hi in columns [0, N), the cross terms in [N, 2 N)
+#pragma unroll
+                for (int c0 = 0; c0 < N; c0 += 16) {
+                    float v[16], u[16];
+                    umma::tmem_ld16(taddr + c0, v);
+                    umma::tmem_ld16(taddr + N + c0, u);
+                    umma::tmem_ld_wait();
+                    if (c0 + 16 == N) {
+                        umma::fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) fast::mbar_arrive(&d_empty[db]);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] += u[i];
+                    if constexpr (Prob::ACCUMULATE) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) { v[i] += acc[c0 + i]; acc[c0 + i] = flush ? 0.f : v[i]; }
+                    }
+                    if (flush) prob.store(t, warp * 32 + lane, c0, v);
+                }
+            } else {
 #pragma unroll
             for (int c0 = 0; c0 < N; c0 += 32) {
                 float v[32];
@@ -215,6 +241,7 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
                     for (int i = 0; i < 32; ++i) { v[i] += acc[c0 + i]; acc[c0 + i] = flush ? 0.f : v[i]; }
                 }
                 if (flush) prob.store(t, warp * 32 + lane, c0, v);
+            }
             }
         }
     } else if (warp < 4 + kConvWarps) {
@@ -238,38 +265,47 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
         if constexpr (kTma) {
             // The operands arrive as raw boxes.  A goes to tensor memory, where the tensor cores read it without
             // touching shared memory: lane m of tensor memory is row m of the tile, and a warp reaches the 32 lanes
-            // of its quarter only, so warp w converts rows 32 (w % 4) ... and columns 16 (w / 4) ... of every
-            // chunk.  B is split into the shared-memory stage as before.
-            const int a_row = (cwarp & 3) * 32 + lane, a_k0 = (cwarp >> 2) * 16;
-            const uint32_t a_taddr = tmem_base + ((uint32_t)((cwarp & 3) * 32) << 16) + L::tma_col_a + (uint32_t)a_k0;
+            // of its quarter only, so a warp converts rows 32 (w % 4) ... of a chunk.  B is split into the
+            // shared-memory stage as before.  The eight warps are two groups of four that take alternate chunks:
+            // a chunk's way through a warp is a chain of latencies (box, tensor-memory store, proxy fence), and two
+            // chunks on their way at a time hide half of it.
+            using OB4 = OperandItems<N, Prob::B_LANE_ROWS, kConvWarps / 2>;
+            static_assert(kConvWarps == 8, "two groups of one warp per tensor-memory quarter");
+            const int grp = cwarp >> 2, qw = cwarp & 3;
+            const int a_row = qw * 32 + lane;
+            const uint32_t a_taddr = tmem_base + ((uint32_t)(qw * 32) << 16) + L::tma_col_a;
             int it = 0;
             bool ok = true;
             for (int t = 0; ok && t < n_tiles; ++t) {
                 const int n_chunks = prob.n_chunks(t);
 #pragma unroll 1
                 for (int kc = 0; kc < n_chunks; ++kc, ++it) {
+                    if ((it & 1) != grp) continue;
                     const int rs = it % kRawStages, s = it % NSTAGE;
                     if (!fast::mbar_wait(&raw_full[rs], (it / kRawStages) & 1, abort_flag, prob.status)) { ok = false; break; }
                     const unsigned char* ra = raw_ring + (size_t)rs * L::raw_bytes;
                     const unsigned char* rb = ra + L::a_bytes;
-                    float4 a[4], b[OB::NI];
+                    float4 a[8], b[OB4::NI];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) a[i] = Prob::raw_a(ra, a_row, a_k0 + 4 * i);
-                    OB::load(b, cwarp, lane, [&](int row, int k) { return Prob::raw_b(rb, row, k); });
+                    for (int i = 0; i < 8; ++i) a[i] = Prob::raw_a(ra, a_row, 4 * i);
+                    OB4::load(b, qw, lane, [&](int row, int k) { return Prob::raw_b(rb, row, k); });
                     if (it >= NSTAGE && !fast::mbar_wait(&stage_empty[s], ((it / NSTAGE) + 1) & 1, abort_flag, prob.status)) { ok = false; break; }
                     umma::fence_after_sync();
-                    float hi[16], lo[16];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        float4 h4, l4;
-                        umma::split_tf32(a[i], h4, l4);
-                        hi[4 * i] = h4.x; hi[4 * i + 1] = h4.y; hi[4 * i + 2] = h4.z; hi[4 * i + 3] = h4.w;
-                        lo[4 * i] = l4.x; lo[4 * i + 1] = l4.y; lo[4 * i + 2] = l4.z; lo[4 * i + 3] = l4.w;
+                    for (int half = 0; half < 2; ++half) {
+                        float hi[16], lo[16];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            float4 h4, l4;
+                            umma::split_tf32(a[4 * half + i], h4, l4);
+                            hi[4 * i] = h4.x; hi[4 * i + 1] = h4.y; hi[4 * i + 2] = h4.z; hi[4 * i + 3] = h4.w;
+                            lo[4 * i] = l4.x; lo[4 * i + 1] = l4.y; lo[4 * i + 2] = l4.z; lo[4 * i + 3] = l4.w;
+                        }
+                        umma::tmem_st16(a_taddr + (uint32_t)(s * 2 * kChunkK + 16 * half), hi);
+                        umma::tmem_st16(a_taddr + (uint32_t)(s * 2 * kChunkK + kChunkK + 16 * half), lo);
                     }
-                    umma::tmem_st16(a_taddr + (uint32_t)(s * 2 * kChunkK), hi);
-                    umma::tmem_st16(a_taddr + (uint32_t)(s * 2 * kChunkK + kChunkK), lo);
                     unsigned char* st = stages + (size_t)s * kStageBytes;
-                    OB::store(b, st, st + L::b_bytes, cwarp, lane);
+                    OB4::store(b, st, st + L::b_bytes, qw, lane);
                     umma::tmem_st_wait();
                     umma::fence_before_sync();
                     umma::fence_smem_to_async();
@@ -327,18 +363,24 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
                 if (lane == 0) {
                     const uint32_t st = umma::smem_addr(stages + (size_t)s * kStageBytes);
                     const uint32_t b_hi = st + (uint32_t)kStageB, b_lo = b_hi + (uint32_t)L::b_bytes;
-                    const uint32_t d = tmem_base + (uint32_t)(db * N);
+                    const uint32_t d = tmem_base + (uint32_t)(db * DN);
                     // small terms first: a_lo b_hi, a_hi b_lo, then a_hi b_hi
                     const uint32_t pb[3] = {b_hi, b_lo, b_hi};
-                    if constexpr (kTma) {   // A in tensor memory: columns (hi | lo) of the stage
+                    if constexpr (kTma) {
+                        // A in tensor memory: columns (hi | lo) of the stage.  The issuing thread is what bounds
+                        // these products (an instruction of N = 64 is over before the next one is out), so the
+                        // passes are folded: B_hi and B_lo lie behind each other in the stage and serve as one
+                        // operand of 2 N rows, a_hi [b_hi | b_lo] lands in the tile's two accumulators at once,
+                        // and a_lo b_hi joins the second one.
                         const uint32_t a_hi = tmem_base + L::tma_col_a + (uint32_t)(s * 2 * kChunkK), a_lo = a_hi + kChunkK;
-                        const uint32_t pa[3] = {a_lo, a_hi, a_hi};
+                        constexpr uint32_t idesc2 = umma::idesc_tf32(kTileM, 2 * N);
 #pragma unroll
-                        for (int pass = 0; pass < 3; ++pass)
+                        for (int ks = 0; ks < kChunkK / 8; ++ks)
+                            umma::mma_tf32_ts(d, a_hi + ks * 8, umma::make_desc(b_hi + ks * 2 * umma::kLbo, umma::kLbo, sbo), idesc2,
+                                              (kc > 0 || ks > 0) ? 1u : 0u);
 #pragma unroll
-                            for (int ks = 0; ks < kChunkK / 8; ++ks)
-                                umma::mma_tf32_ts(d, pa[pass] + ks * 8, umma::make_desc(pb[pass] + ks * 2 * umma::kLbo, umma::kLbo, sbo),
-                                                  idesc, (kc > 0 || pass > 0 || ks > 0) ? 1u : 0u);
+                        for (int ks = 0; ks < kChunkK / 8; ++ks)
+                            umma::mma_tf32_ts(d + N, a_lo + ks * 8, umma::make_desc(b_hi + ks * 2 * umma::kLbo, umma::kLbo, sbo), idesc, 1u);
                     } else {
                         const uint32_t a_hi = kResident ? umma::smem_addr(smem + L::off_stage + (size_t)kc * 2 * L::a_bytes) : st;
                         const uint32_t a_lo = a_hi + (uint32_t)L::a_bytes;
@@ -449,18 +491,19 @@ struct RadialWeights {
         if (e >= n_edges || e >= e_begin() + chunk || j >= H) return make_float4(0.f, 0.f, 0.f, 0.f);
         return *reinterpret_cast<const float4*>(h + (size_t)e * H + j);   // H % 4 == 0
     }
-    __device__ __forceinline__ void store(int t, int m, int n0, const float (&v)[32]) const {
+    template <int W>
+    __device__ __forceinline__ void store(int t, int m, int n0, const float (&v)[W]) const {
         const int c = blockIdx.x * 128 + m;
         if (c >= C) return;
         const int64_t e0 = e_begin() + (int64_t)t * 128 + n0;
         const int64_t e_end = min(n_edges, e_begin() + chunk);
         float* dst = s + (size_t)e0 * C + c;   // lanes: consecutive c; one row of s further per value
-        if (e0 + 32 <= e_end) {                // whole piece inside the range: no per-store test
+        if (e0 + W <= e_end) {                 // whole piece inside the range: no per-store test
 #pragma unroll
-            for (int i = 0; i < 32; ++i) dst[(size_t)i * C] = v[i];
+            for (int i = 0; i < W; ++i) dst[(size_t)i * C] = v[i];
         } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
+            for (int i = 0; i < W; ++i)
                 if (e0 + i < e_end) dst[(size_t)i * C] = v[i];
         }
     }
@@ -504,12 +547,13 @@ struct GradHidden {
         if (j >= H || c >= C) return make_float4(0.f, 0.f, 0.f, 0.f);
         return *reinterpret_cast<const float4*>(W + (size_t)j * C + c);
     }
-    __device__ __forceinline__ void store(int t, int m, int n0, const float (&v)[32]) const {
+    template <int W>
+    __device__ __forceinline__ void store(int t, int m, int n0, const float (&v)[W]) const {
         const int64_t e = e_begin() + (int64_t)(t / groups()) * 128 + m;
         if (e >= n_edges || e >= e_begin() + chunk) return;
         const int j0 = blockIdx.y * 64 + n0;
 #pragma unroll
-        for (int i = 0; i < 32; i += 4)
+        for (int i = 0; i < W; i += 4)
             if (j0 + i < H)   // H % 4 == 0
                 *reinterpret_cast<float4*>(gh + (size_t)e * H + j0 + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
     }
@@ -566,17 +610,18 @@ struct GradLayer {
         const int j = blockIdx.z * 64 + row;
         return column(h, H, j, j < H, t * kGroupChunks + kc, k);
     }
-    __device__ __forceinline__ void store(int, int m, int n0, const float (&v)[32]) const {
+    template <int W>
+    __device__ __forceinline__ void store(int, int m, int n0, const float (&v)[W]) const {
         const int c = blockIdx.x * 128 + m;
         if (c >= C) return;
         const int j0 = blockIdx.z * 64 + n0;
         float* dst = partial + (size_t)blockIdx.y * H * C + (size_t)j0 * C + c;   // lanes: consecutive c
-        if (j0 + 32 <= H) {
+        if (j0 + W <= H) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) dst[(size_t)i * C] = v[i];
+            for (int i = 0; i < W; ++i) dst[(size_t)i * C] = v[i];
         } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
+            for (int i = 0; i < W; ++i)
                 if (j0 + i < H) dst[(size_t)i * C] = v[i];
         }
     }
