@@ -50,7 +50,7 @@ constexpr int kConvWarps = 8;     // converter warps
 constexpr int kPrefetch = 2;      // chunks of loads in flight per converter thread (Prob::PREFETCH where given)
 constexpr int kMaxResidentChunks = 4;   // K chunks of a resident A operand (Prob::A_RESIDENT): K <= 128
 constexpr int kGemmThreads = (4 + kConvWarps + 1) * 32;   // epilogue, converters, tensor-core issue
-constexpr int kStagesTma = 4;     // operand stages of the products whose inputs arrive as raw boxes (Prob::TMA) ...
+constexpr int kStagesTma = 2;     // operand stages of the products whose inputs arrive as raw boxes (Prob::TMA) ...
 constexpr int kRawStages = 6;     // ... and their ring of raw boxes (both even: a stage always meets the same converter group,
                                   // so every waiter sees each of its barriers' phases one after the other)
 static_assert(kStagesTma % 2 == 0 && kRawStages % 2 == 0, "stages alternate between the two converter groups");
@@ -62,7 +62,7 @@ struct GemmSmem {
     static constexpr size_t b_bytes = (size_t)N * kChunkK * 4;
     static constexpr size_t stage_bytes = 2 * a_bytes + 2 * b_bytes;  // A_hi, A_lo, B_hi, B_lo
     static constexpr size_t off_bar = 0;       // stage_full[kMaxStages], stage_empty[kMaxStages], d_full[2], d_empty[2], drain, a_ready
-    static constexpr size_t off_tmem = 8 * (2 * kMaxStages + 6);
+    static constexpr size_t off_tmem = 8 * (2 * kMaxStages + 7);   // (... a_ready, drain of the second issuing warp)
     static constexpr size_t off_abort = off_tmem + 4;
     static constexpr size_t off_stage = 1024;
     static constexpr size_t total = off_stage + kStages * stage_bytes;
@@ -75,8 +75,8 @@ struct GemmSmem {
     static constexpr size_t raw_bytes = a_bytes + b_bytes;
     static constexpr size_t tma_total = off_stage + kStagesTma * res_stage_bytes + 1024 + kRawStages * raw_bytes;
     // tensor memory of those products: two accumulator tiles, then per stage the A operand as (hi | lo) of 32 k each
-    // (an accumulator tile of those products is two: the product of the hi parts, and the two cross terms)
-    static constexpr uint32_t tma_col_a = 4 * N, tma_cols = 512;
+    // (an accumulator tile of those products is three: a_hi b_hi, a_hi b_lo and a_lo b_hi)
+    static constexpr uint32_t tma_col_a = 6 * N, tma_cols = 512;
     static_assert(N > 64 || tma_col_a + kStagesTma * 2 * kChunkK <= tma_cols, "tensor memory");
     static_assert(off_raw_bar + 16 * kRawStages <= off_stage && off_abort + 4 <= off_raw_bar, "barrier area");
 };
@@ -92,7 +92,8 @@ template <class P> struct ProbTraits<P, decltype((void)P::A_RESIDENT)> {
 
 template <class P, class = void> struct TmaTraits { static constexpr bool TMA = false; };
 template <class P> struct TmaTraits<P, decltype((void)P::TMA)> { static constexpr bool TMA = P::TMA; };
-template <class P> constexpr int gemm_threads() { return kGemmThreads + (TmaTraits<P>::TMA ? 32 : 0); }
+// (Prob::TMA: one warp more for the bulk copies and one for the second half of the tensor-core instructions)
+template <class P> constexpr int gemm_threads() { return kGemmThreads + (TmaTraits<P>::TMA ? 64 : 0); }
 
 // One box of a rank-2 tensor map into shared memory; x is the coordinate along the contiguous dimension and must
 // be a multiple of four elements.  Completes on the barrier with the box's bytes, whatever part of it lay outside.
@@ -149,7 +150,7 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
     constexpr int N = Prob::N;
     constexpr bool kTma = TmaTraits<Prob>::TMA;
     constexpr int NSTAGE = kTma ? kStagesTma : kStages;
-    constexpr int DN = kTma ? 2 * N : N;   // tensor-memory columns of one accumulator tile
+    constexpr int DN = kTma ? 3 * N : N;   // tensor-memory columns of one accumulator tile
     using L = GemmSmem<N>;
     constexpr uint32_t kTmemCols = TmaTraits<Prob>::TMA ? L::tma_cols : 2 * N;   // two accumulator tiles (+ the A stages)
     static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "tensor-memory allocation must be a power of two");
@@ -160,6 +161,7 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
     uint64_t* d_empty = d_full + 2;
     uint64_t* drain = d_empty + 2;
     uint64_t* a_ready = drain + 1;
+    uint64_t* drain2 = a_ready + 1;
     uint64_t* raw_full = reinterpret_cast<uint64_t*>(smem + L::off_raw_bar);
     uint64_t* raw_empty = raw_full + kRawStages;
     constexpr bool kResident = ProbTraits<Prob>::A_RESIDENT;   // A does not depend on the tile: converted once
@@ -174,11 +176,13 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMaxStages; ++s) { fast::mbar_init(&stage_full[s], kTma ? kConvWarps / 2 : kConvWarps); fast::mbar_init(&stage_empty[s], 1); }
+        // (Prob::TMA: two issuing warps commit to stage_empty and d_full)
+        for (int s = 0; s < kMaxStages; ++s) { fast::mbar_init(&stage_full[s], kTma ? kConvWarps / 2 : kConvWarps); fast::mbar_init(&stage_empty[s], kTma ? 2 : 1); }
         if constexpr (kTma)
             for (int s = 0; s < kRawStages; ++s) { fast::mbar_init(&raw_full[s], 1); fast::mbar_init(&raw_empty[s], kConvWarps / 2); }
-        for (int b = 0; b < 2; ++b) { fast::mbar_init(&d_full[b], 1); fast::mbar_init(&d_empty[b], 4); }
+        for (int b = 0; b < 2; ++b) { fast::mbar_init(&d_full[b], kTma ? 2 : 1); fast::mbar_init(&d_empty[b], 4); }
         fast::mbar_init(drain, 1);
+        fast::mbar_init(drain2, 1);
         fast::mbar_init(a_ready, kConvWarps);
         *abort_flag = 0;
         fast::mbar_fence_init();
@@ -205,12 +209,16 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
             const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(db * DN);
             const bool flush = prob.flush(t);
             if constexpr (kTma) {
-                // two accumulators per tile: a_hi b_hi in columns [0, N), the cross terms in [N, 2 N)
+                // three accumulators per tile: a_hi b_hi in columns [0, N), a_hi b_lo in [N, 2 N), a_lo b_hi behind
 #pragma unroll
                 for (int c0 = 0; c0 < N; c0 += 16) {
                     float v[16], u[16];
-                    umma::tmem_ld16(taddr + c0, v);
                     umma::tmem_ld16(taddr + N + c0, u);
+                    umma::tmem_ld16(taddr + 2 * N + c0, v);
+                    umma::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) u[i] += v[i];   // the small terms first
+                    umma::tmem_ld16(taddr + c0, v);
                     umma::tmem_ld_wait();
                     if (c0 + 16 == N) {
                         umma::fence_before_sync();
@@ -345,8 +353,9 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
             }
         }
         }
-    } else if (warp == 4 + kConvWarps) {
-        // ------------------------------------------------ tensor-core issue (one lane)
+    } else if (warp == 4 + kConvWarps || (kTma && warp == 4 + kConvWarps + 2)) {
+        // ------------------------------------------------ tensor-core issue (one lane; Prob::TMA: of two warps)
+        const bool second = warp != 4 + kConvWarps;
         constexpr uint32_t idesc = umma::idesc_tf32(kTileM, N);
         const uint32_t sbo = umma::sbo_bytes(kChunkK);
         int it = 0;
@@ -369,18 +378,24 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
                     if constexpr (kTma) {
                         // A in tensor memory: columns (hi | lo) of the stage.  The issuing thread is what bounds
                         // these products (an instruction of N = 64 is over before the next one is out), so the
-                        // passes are folded: B_hi and B_lo lie behind each other in the stage and serve as one
-                        // operand of 2 N rows, a_hi [b_hi | b_lo] lands in the tile's two accumulators at once,
-                        // and a_lo b_hi joins the second one.
+                        // passes are folded and shared between two warps.  B_hi and B_lo lie behind each other
+                        // in the stage and serve as one operand of 2 N rows: the first warp issues
+                        // a_hi [b_hi | b_lo] into the tile's first two accumulators, the second a_lo b_hi into
+                        // the third (accumulators of their own, so the order of the sums does not depend on
+                        // which warp is ahead); the epilogue adds the three.
                         const uint32_t a_hi = tmem_base + L::tma_col_a + (uint32_t)(s * 2 * kChunkK), a_lo = a_hi + kChunkK;
                         constexpr uint32_t idesc2 = umma::idesc_tf32(kTileM, 2 * N);
+                        if (!second) {
 #pragma unroll
-                        for (int ks = 0; ks < kChunkK / 8; ++ks)
-                            umma::mma_tf32_ts(d, a_hi + ks * 8, umma::make_desc(b_hi + ks * 2 * umma::kLbo, umma::kLbo, sbo), idesc2,
-                                              (kc > 0 || ks > 0) ? 1u : 0u);
+                            for (int ks = 0; ks < kChunkK / 8; ++ks)
+                                umma::mma_tf32_ts(d, a_hi + ks * 8, umma::make_desc(b_hi + ks * 2 * umma::kLbo, umma::kLbo, sbo), idesc2,
+                                                  (kc > 0 || ks > 0) ? 1u : 0u);
+                        } else {
 #pragma unroll
-                        for (int ks = 0; ks < kChunkK / 8; ++ks)
-                            umma::mma_tf32_ts(d + N, a_lo + ks * 8, umma::make_desc(b_hi + ks * 2 * umma::kLbo, umma::kLbo, sbo), idesc, 1u);
+                            for (int ks = 0; ks < kChunkK / 8; ++ks)
+                                umma::mma_tf32_ts(d + 2 * N, a_lo + ks * 8, umma::make_desc(b_hi + ks * 2 * umma::kLbo, umma::kLbo, sbo), idesc,
+                                                  (kc > 0 || ks > 0) ? 1u : 0u);
+                        }
                     } else {
                         const uint32_t a_hi = kResident ? umma::smem_addr(smem + L::off_stage + (size_t)kc * 2 * L::a_bytes) : st;
                         const uint32_t a_lo = a_hi + (uint32_t)L::a_bytes;
@@ -401,11 +416,12 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
         }
         // abort path only: let the products still in flight finish before tensor memory is freed
         if (*abort_flag) {
-            if (lane == 0) umma::commit(drain);
+            uint64_t* const mine = second ? drain2 : drain;
+            if (lane == 0) umma::commit(mine);
             __syncwarp();
 #pragma unroll 1
             for (uint32_t spin = 0; spin < fast::kSpinLimit; ++spin)
-                if (fast::mbar_try_wait(drain, 0)) break;
+                if (fast::mbar_try_wait(mine, 0)) break;
         }
     } else {
         // ------------------------------------------------ raw boxes (Prob::TMA): tiled bulk copies, one lane
