@@ -114,8 +114,10 @@ int grad_hidden(int64_t n_edges, int H, int C, const float* gs, const float* W, 
     GradHidden p{};
     p.gs = gs; p.W = W; p.gh = gh; p.n_edges = n_edges; p.H = H; p.C = C; p.status = status;
     p.chunk = round_up((n_edges + n_cta - 1) / n_cta, 128);
+    p.gc = kGroupChunks;
     GradHiddenTma q{};
     static_cast<GradHidden&>(q) = p;
+    q.gc = kGroupChunksTma;
     if (make_map(&q.map_a, gs, n_edges, C, C, kChunkK, 128, true) && make_map(&q.map_b, W, H, C, C, kChunkK, 64, true))
         return launch_gemm(q, dim3(n_cta, (H + 63) / 64), st);
     return launch_gemm(p, dim3(n_cta, (H + 63) / 64), st);
@@ -133,8 +135,10 @@ int grad_layer(int64_t n_edges, int H, int C, const float* gs, const float* h, f
     GradLayer p{};
     p.gs = gs; p.h = h; p.partial = partial; p.n_edges = n_edges; p.H = H; p.C = C; p.status = status;
     p.chunk = round_up((n_edges + n_ranges - 1) / n_ranges, kChunkK);
+    p.gc = kGroupChunks;
     GradLayerTma q{};
     static_cast<GradLayer&>(q) = p;
+    q.gc = kGroupChunksTma;
     const dim3 grid(n_cb, n_ranges, (H + 63) / 64);
     const bool boxes = make_map(&q.map_a, gs, n_edges, C, C, 128, kChunkK, false) &&
                        make_map(&q.map_b, h, n_edges, H, H, 64, kChunkK, false);

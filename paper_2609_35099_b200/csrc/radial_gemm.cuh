@@ -46,6 +46,7 @@ constexpr int kTileM = 128;      // rows of an output tile = tensor-memory lanes
 constexpr int kChunkK = 32;      // k per shared-memory stage (four tcgen05.mma steps of 8)
 constexpr int kStages = 3;
 constexpr int kGroupChunks = 8;  // K chunks accumulated inside tensor memory before the tile is read out
+constexpr int kGroupChunksTma = 16;   // the same where every term of the split has an accumulator of its own (Prob::TMA)
 constexpr int kConvWarps = 8;     // converter warps
 constexpr int kPrefetch = 2;      // chunks of loads in flight per converter thread (Prob::PREFETCH where given)
 constexpr int kMaxResidentChunks = 4;   // K chunks of a resident A operand (Prob::A_RESIDENT): K <= 128
@@ -538,28 +539,29 @@ struct GradHidden {
     const float* gs; const float* W; float* gh;
     int64_t n_edges, chunk;   // chunk: edges per CTA (multiple of 128)
     int H, C;
+    int gc;                   // K chunks summed inside tensor memory before a tile is read out (see the head of the file)
     int32_t* status;
-    // pipeline tile t = (edge tile t / groups, group t % groups of kGroupChunks chunks of c)
+    // pipeline tile t = (edge tile t / groups, group t % groups of gc chunks of c)
     __device__ __forceinline__ int total_chunks() const { return (C + kChunkK - 1) / kChunkK; }
-    __device__ __forceinline__ int groups() const { return (total_chunks() + kGroupChunks - 1) / kGroupChunks; }
+    __device__ __forceinline__ int groups() const { return (total_chunks() + gc - 1) / gc; }
     __device__ __forceinline__ int64_t e_begin() const { return min(n_edges, (int64_t)blockIdx.x * chunk); }
     __device__ __forceinline__ int n_tiles() const {
         const int64_t e0 = e_begin(), e1 = min(n_edges, e0 + chunk);
         return (int)((e1 - e0 + 127) / 128) * groups();
     }
     __device__ __forceinline__ int n_chunks(int t) const {
-        return min(kGroupChunks, total_chunks() - (t % groups()) * kGroupChunks);
+        return min(gc, total_chunks() - (t % groups()) * gc);
     }
     __device__ __forceinline__ bool flush(int t) const { return t % groups() == groups() - 1; }
     __device__ __forceinline__ float4 load_a(int t, int kc, int row, int k) const {   // grad_s: row = edge, k = c
         const int g = groups();
         const int64_t e = e_begin() + (int64_t)(t / g) * 128 + row;
-        const int c = ((t % g) * kGroupChunks + kc) * kChunkK + k;
+        const int c = ((t % g) * gc + kc) * kChunkK + k;
         if (e >= n_edges || e >= e_begin() + chunk || c >= C) return make_float4(0.f, 0.f, 0.f, 0.f);
         return *reinterpret_cast<const float4*>(gs + (size_t)e * C + c);   // C % 4 == 0
     }
     __device__ __forceinline__ float4 load_b(int t, int kc, int row, int k) const {   // W: row = j, k = c
-        const int c = ((t % groups()) * kGroupChunks + kc) * kChunkK + k, j = blockIdx.y * 64 + row;
+        const int c = ((t % groups()) * gc + kc) * kChunkK + k, j = blockIdx.y * 64 + row;
         if (j >= H || c >= C) return make_float4(0.f, 0.f, 0.f, 0.f);
         return *reinterpret_cast<const float4*>(W + (size_t)j * C + c);
     }
@@ -579,7 +581,7 @@ struct GradHidden {
 struct GradHiddenTma : GradHidden {
     static constexpr bool TMA = true;
     alignas(64) CUtensorMap map_a, map_b;
-    __device__ __forceinline__ int first_c(int t, int kc) const { return ((t % groups()) * kGroupChunks + kc) * kChunkK; }
+    __device__ __forceinline__ int first_c(int t, int kc) const { return ((t % groups()) * gc + kc) * kChunkK; }
     __device__ __forceinline__ void box_a(int t, int kc, int& x, int& y) const {
         x = first_c(t, kc); y = (int)(e_begin() + (int64_t)(t / groups()) * 128);
     }
@@ -597,15 +599,16 @@ struct GradLayer {
     const float* gs; const float* h; float* partial;
     int64_t n_edges, chunk;   // chunk: edges per range (multiple of 32)
     int H, C;
+    int gc;                   // K chunks summed inside tensor memory before a tile is read out
     int32_t* status;
     __device__ __forceinline__ int64_t e_begin() const { return min(n_edges, (int64_t)blockIdx.y * chunk); }
-    // pipeline tile t = group t of kGroupChunks chunks of the range's edges; one output tile per CTA
+    // pipeline tile t = group t of gc chunks of the range's edges; one output tile per CTA
     __device__ __forceinline__ int total_chunks() const {
         const int64_t e0 = e_begin(), e1 = min(n_edges, e0 + chunk);
         return (int)max((int64_t)1, (e1 - e0 + kChunkK - 1) / kChunkK);   // an empty range still writes a zero tile
     }
-    __device__ __forceinline__ int n_tiles() const { return (total_chunks() + kGroupChunks - 1) / kGroupChunks; }
-    __device__ __forceinline__ int n_chunks(int t) const { return min(kGroupChunks, total_chunks() - t * kGroupChunks); }
+    __device__ __forceinline__ int n_tiles() const { return (total_chunks() + gc - 1) / gc; }
+    __device__ __forceinline__ int n_chunks(int t) const { return min(gc, total_chunks() - t * gc); }
     __device__ __forceinline__ bool flush(int t) const { return t == n_tiles() - 1; }
     __device__ __forceinline__ float4 column(const float* base, int ld, int col, bool col_ok, int kc, int k) const {
         const int64_t e = e_begin() + (int64_t)kc * kChunkK + k, e_end = min(n_edges, e_begin() + chunk);
@@ -620,11 +623,11 @@ struct GradLayer {
     }
     __device__ __forceinline__ float4 load_a(int t, int kc, int row, int k) const {   // grad_s^T: row = c, k = edge
         const int c = blockIdx.x * 128 + row;
-        return column(gs, C, c, c < C, t * kGroupChunks + kc, k);
+        return column(gs, C, c, c < C, t * gc + kc, k);
     }
     __device__ __forceinline__ float4 load_b(int t, int kc, int row, int k) const {   // h^T: row = j, k = edge
         const int j = blockIdx.z * 64 + row;
-        return column(h, H, j, j < H, t * kGroupChunks + kc, k);
+        return column(h, H, j, j < H, t * gc + kc, k);
     }
     template <int W>
     __device__ __forceinline__ void store(int, int m, int n0, const float (&v)[W]) const {
@@ -647,7 +650,7 @@ struct GradLayer {
 struct GradLayerTma : GradLayer {
     static constexpr bool TMA = true;
     alignas(64) CUtensorMap map_a, map_b;
-    __device__ __forceinline__ int first_e(int t, int kc) const { return (int)(e_begin() + (int64_t)(t * kGroupChunks + kc) * kChunkK); }
+    __device__ __forceinline__ int first_e(int t, int kc) const { return (int)(e_begin() + (int64_t)(t * gc + kc) * kChunkK); }
     __device__ __forceinline__ void box_a(int t, int kc, int& x, int& y) const { x = blockIdx.x * 128; y = first_e(t, kc); }
     __device__ __forceinline__ void box_b(int t, int kc, int& x, int& y) const { x = blockIdx.z * 64; y = first_e(t, kc); }
     __device__ static __forceinline__ float4 raw_a(const unsigned char* box, int row, int k) { return raw_transposed(box, 128, row, k); }
