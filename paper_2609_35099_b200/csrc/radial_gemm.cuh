@@ -131,6 +131,7 @@ struct OperandItems {
             v[i] = ld(row, k);
         }
     }
+    template <bool BITS = false>   // BITS: the split with integer instructions (umma::split_tf32_bits)
     __device__ static __forceinline__ void store(const float4 (&v)[NI], unsigned char* hi, unsigned char* lo, int cwarp,
                                                  int lane) {
 #pragma unroll
@@ -138,7 +139,8 @@ struct OperandItems {
             int row, k;
             coords(i, cwarp, lane, row, k);
             float4 h, l;
-            umma::split_tf32(v[i], h, l);
+            if constexpr (BITS) umma::split_tf32_bits(v[i], h, l);
+            else umma::split_tf32(v[i], h, l);
             const uint32_t off = umma::tile_offset(row, k, kChunkK);
             *reinterpret_cast<float4*>(hi + off) = h;
             *reinterpret_cast<float4*>(lo + off) = l;
@@ -306,7 +308,7 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             float4 h4, l4;
-                            umma::split_tf32(a[4 * half + i], h4, l4);
+                            umma::split_tf32_bits(a[4 * half + i], h4, l4);
                             hi[4 * i] = h4.x; hi[4 * i + 1] = h4.y; hi[4 * i + 2] = h4.z; hi[4 * i + 3] = h4.w;
                             lo[4 * i] = l4.x; lo[4 * i + 1] = l4.y; lo[4 * i + 2] = l4.z; lo[4 * i + 3] = l4.w;
                         }
@@ -314,7 +316,7 @@ __global__ void __launch_bounds__(gemm_threads<Prob>(), 1) gemm_tf32x3_kernel(co
                         umma::tmem_st16(a_taddr + (uint32_t)(s * 2 * kChunkK + kChunkK + 16 * half), lo);
                     }
                     unsigned char* st = stages + (size_t)s * kStageBytes;
-                    OB4::store(b, st, st + L::b_bytes, qw, lane);
+                    OB4::template store<true>(b, st, st + L::b_bytes, qw, lane);
                     umma::tmem_st_wait();
                     umma::fence_before_sync();
                     umma::fence_smem_to_async();

@@ -149,18 +149,27 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // float32 -> (hi, lo) TF32 pair, both rounded to nearest (ties away from zero); v = hi + lo up to 2^-22 |v|.
-// The rounding is done on the bit pattern (add half a TF32 unit to the magnitude, clear the 13 low bits), which
-// gives what cvt.rna.tf32.f32 gives for finite values but runs on the integer pipe at full rate: the conversion
-// instruction issues at an eighth of that, and the converter warps of the products were bound by it.
-__device__ __forceinline__ float round_tf32(float v) {
-    return __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
-}
 __device__ __forceinline__ void split_tf32(float v, float& hi, float& lo) {
-    hi = round_tf32(v);
-    lo = round_tf32(v - hi);
+    uint32_t h, l;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(v));
+    hi = __uint_as_float(h);
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(l) : "f"(v - hi));
+    lo = __uint_as_float(l);
 }
 __device__ __forceinline__ void split_tf32(const float4 v, float4& hi, float4& lo) {
     split_tf32(v.x, hi.x, lo.x); split_tf32(v.y, hi.y, lo.y); split_tf32(v.z, hi.z, lo.z); split_tf32(v.w, hi.w, lo.w);
+}
+// The same split with the rounding done on the bit pattern (add half a TF32 unit to the magnitude, clear the 13
+// low bits): what the conversion instruction gives for finite values, on the integer pipe.  The conversion
+// instruction issues at an eighth of the integer rate, which bounds warps that do little else (the converters of
+// the gradient products); where the integer pipe is the busy one (the other kernels) the instruction is the cheaper.
+__device__ __forceinline__ float round_tf32_bits(float v) {
+    return __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
+}
+__device__ __forceinline__ void split_tf32_bits(const float4 v, float4& hi, float4& lo) {
+    hi = make_float4(round_tf32_bits(v.x), round_tf32_bits(v.y), round_tf32_bits(v.z), round_tf32_bits(v.w));
+    lo = make_float4(round_tf32_bits(v.x - hi.x), round_tf32_bits(v.y - hi.y), round_tf32_bits(v.z - hi.z),
+                     round_tf32_bits(v.w - hi.w));
 }
 
 }  // namespace umma
