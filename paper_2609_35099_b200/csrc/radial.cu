@@ -51,8 +51,8 @@ int launch_gemm(const Prob& prob, dim3 grid, cudaStream_t st, int resident_chunk
 }
 
 // Tensor map of a row-major float32 matrix [rows][cols] with `pitch` floats between rows, fetched in boxes of
-// box_cols x box_rows.  False where the matrix does not meet the copy engine's alignment rules (the caller
-// then takes the kernel that loads through registers) or the driver has no encoder.
+// box_cols x box_rows.  False where the matrix does not meet the copy engine's alignment rules (16-byte aligned
+// base and rows) or the driver has no encoder.
 using EncodeTiled = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -114,12 +114,9 @@ int grad_hidden(int64_t n_edges, int H, int C, const float* gs, const float* W, 
     GradHidden p{};
     p.gs = gs; p.W = W; p.gh = gh; p.n_edges = n_edges; p.H = H; p.C = C; p.status = status;
     p.chunk = round_up((n_edges + n_cta - 1) / n_cta, 128);
-    p.gc = kGroupChunks;
-    GradHiddenTma q{};
-    static_cast<GradHidden&>(q) = p;
-    q.gc = kGroupChunksTma;
-    if (make_map(&q.map_a, gs, n_edges, C, C, kChunkK, 128, true) && make_map(&q.map_b, W, H, C, C, kChunkK, 64, true))
-        return launch_gemm(q, dim3(n_cta, (H + 63) / 64), st);
+    p.gc = kGroupChunksTma;
+    if (!make_map(&p.map_a, gs, n_edges, C, C, kChunkK, 128, true) || !make_map(&p.map_b, W, H, C, C, kChunkK, 64, true))
+        return E3J_ERR_UNSUPPORTED;   // (the entry points have checked the alignment: the driver has no encoder)
     return launch_gemm(p, dim3(n_cta, (H + 63) / 64), st);
 }
 
@@ -135,14 +132,10 @@ int grad_layer(int64_t n_edges, int H, int C, const float* gs, const float* h, f
     GradLayer p{};
     p.gs = gs; p.h = h; p.partial = partial; p.n_edges = n_edges; p.H = H; p.C = C; p.status = status;
     p.chunk = round_up((n_edges + n_ranges - 1) / n_ranges, kChunkK);
-    p.gc = kGroupChunks;
-    GradLayerTma q{};
-    static_cast<GradLayer&>(q) = p;
-    q.gc = kGroupChunksTma;
-    const dim3 grid(n_cb, n_ranges, (H + 63) / 64);
-    const bool boxes = make_map(&q.map_a, gs, n_edges, C, C, 128, kChunkK, false) &&
-                       make_map(&q.map_b, h, n_edges, H, H, 64, kChunkK, false);
-    if (int s = boxes ? launch_gemm(q, grid, st) : launch_gemm(p, grid, st)) return s;
+    p.gc = kGroupChunksTma;
+    if (!make_map(&p.map_a, gs, n_edges, C, C, 128, kChunkK, false) || !make_map(&p.map_b, h, n_edges, H, H, 64, kChunkK, false))
+        return E3J_ERR_UNSUPPORTED;
+    if (int s = launch_gemm(p, dim3(n_cb, n_ranges, (H + 63) / 64), st)) return s;
     const int blocks = (int)std::min<int64_t>((n_elems + 255) / 256, 4 * fast::sm_count());
     layer_sum_kernel<<<blocks, 256, 0, st>>>(n_ranges, n_elems, partial, gW);
     return after_launch();

@@ -11,13 +11,21 @@
 // of W^T for all of its edge tiles) it is converted once into a resident region of shared memory and the stage
 // ring carries the B operand alone, with more chunks of loads in flight per converter thread (Prob::PREFETCH).
 //
-// Where the operands lie in global memory with 16-byte aligned rows (Prob::TMA: the two gradient products), one more
-// warp brings them in as raw float32 boxes with tiled bulk copies (cp.async.bulk.tensor through a tensor map; rows
-// past the end of a matrix arrive as zeros), a ring of kRawStages boxes deep, and the converter warps read the boxes
-// from shared memory instead of loading from global memory: the loads in flight no longer depend on the
-// converters' registers, and they stay off the load/store pipe that the converters' shared-memory stores and the
-// tensor cores' operand reads already fill.  Boxes whose rows are 128 bytes use the 128-byte swizzle, so that the
-// eight rows a converter quarter-warp reads lie in different banks.
+// The two gradient products (Prob::TMA) are built differently, because they read 1 GB each and little else:
+//   * One more warp brings the operands in as raw float32 boxes with tiled bulk copies (cp.async.bulk.tensor
+//     through a tensor map; rows past the end of a matrix arrive as zeros), a ring of kRawStages boxes deep.  The
+//     converter warps read the boxes from shared memory: the loads in flight no longer depend on the converters'
+//     registers, and they stay off the load/store pipe.  Boxes whose rows are 128 bytes use the 128-byte
+//     swizzle, so that the eight rows a converter quarter-warp reads lie in different banks.
+//   * The A operand goes to tensor memory (tcgen05.st, lane = row of the tile) instead of a shared-memory stage:
+//     the tensor cores read it without touching shared memory.  The converters are two groups of four warps (one
+//     per quarter of the lanes) that take alternate chunks.
+//   * A tcgen05.mma of N = 64 is over before its issuing thread has the next one out, so the thread, not the
+//     tensor cores, bounds the product.  The three passes are therefore folded into two instructions per k-step:
+//     B_hi and B_lo lie behind each other in the stage and serve as one operand of 2 N rows, so that
+//     a_hi [b_hi | b_lo] is one instruction, a_lo b_hi the other; two warps issue one of them each, into
+//     accumulators of their own (the order of the floating-point sums does not depend on which warp is ahead),
+//     and the epilogue adds the three accumulators of a tile, small terms first.
 //
 // A Problem type describes one product: which output tiles a CTA owns, how many K chunks a tile has, where
 // operand values come from (zero outside the matrices) and where results go.  Three instances are used:
@@ -27,9 +35,9 @@
 //
 // Accumulation: the tensor cores add into their float32 accumulators with truncation, so a long chain of
 // products drifts (measured: 2e-5 relative after 1200 accumulation steps).  A tile of the pipeline therefore
-// covers at most kGroupChunks K chunks (96 steps); where a sum is longer, the epilogue warps add the finished
-// partial tiles in float32 registers (round to nearest) and store once the last group has arrived
-// (Prob::ACCUMULATE, Prob::flush).
+// covers at most kGroupChunks K chunks (96 steps; kGroupChunksTma where every term has its own accumulator: 64
+// steps); where a sum is longer, the epilogue warps add the finished partial tiles in float32 registers (round
+// to nearest) and store once the last group has arrived (Prob::ACCUMULATE, Prob::flush).
 //
 // Every wait is bounded (fast::mbar_wait): on a time-out the CTA records the failure in the status word,
 // stops issuing work, lets the tensor cores drain, frees its tensor memory and returns.
@@ -538,6 +546,8 @@ struct RadialWeightsWide : RadialWeights {
 struct GradHidden {
     static constexpr int N = 64, A_LANE_ROWS = 8, B_LANE_ROWS = 8;
     static constexpr bool ACCUMULATE = true;
+    static constexpr bool TMA = true;
+    alignas(64) CUtensorMap map_a, map_b;   // grad_s [n_edges][C], W [H][C]
     const float* gs; const float* W; float* gh;
     int64_t n_edges, chunk;   // chunk: edges per CTA (multiple of 128)
     int H, C;
@@ -555,18 +565,14 @@ struct GradHidden {
         return min(gc, total_chunks() - (t % groups()) * gc);
     }
     __device__ __forceinline__ bool flush(int t) const { return t % groups() == groups() - 1; }
-    __device__ __forceinline__ float4 load_a(int t, int kc, int row, int k) const {   // grad_s: row = edge, k = c
-        const int g = groups();
-        const int64_t e = e_begin() + (int64_t)(t / g) * 128 + row;
-        const int c = ((t % g) * gc + kc) * kChunkK + k;
-        if (e >= n_edges || e >= e_begin() + chunk || c >= C) return make_float4(0.f, 0.f, 0.f, 0.f);
-        return *reinterpret_cast<const float4*>(gs + (size_t)e * C + c);   // C % 4 == 0
+    // operands: boxes of 32 c (128 edges of grad_s | 64 rows of W), 128-byte swizzle
+    __device__ __forceinline__ int first_c(int t, int kc) const { return ((t % groups()) * gc + kc) * kChunkK; }
+    __device__ __forceinline__ void box_a(int t, int kc, int& x, int& y) const {
+        x = first_c(t, kc); y = (int)(e_begin() + (int64_t)(t / groups()) * 128);
     }
-    __device__ __forceinline__ float4 load_b(int t, int kc, int row, int k) const {   // W: row = j, k = c
-        const int c = ((t % groups()) * gc + kc) * kChunkK + k, j = blockIdx.y * 64 + row;
-        if (j >= H || c >= C) return make_float4(0.f, 0.f, 0.f, 0.f);
-        return *reinterpret_cast<const float4*>(W + (size_t)j * C + c);
-    }
+    __device__ __forceinline__ void box_b(int t, int kc, int& x, int& y) const { x = first_c(t, kc); y = blockIdx.y * 64; }
+    __device__ static __forceinline__ float4 raw_a(const unsigned char* box, int row, int k) { return raw_swizzled(box, row, k); }
+    __device__ static __forceinline__ float4 raw_b(const unsigned char* box, int row, int k) { return raw_swizzled(box, row, k); }
     template <int W>
     __device__ __forceinline__ void store(int t, int m, int n0, const float (&v)[W]) const {
         const int64_t e = e_begin() + (int64_t)(t / groups()) * 128 + m;
@@ -579,25 +585,14 @@ struct GradHidden {
     }
 };
 
-// the same with both operands fetched as boxes of 32 c: (128 edges of grad_s | 64 rows of W), 128-byte swizzle
-struct GradHiddenTma : GradHidden {
-    static constexpr bool TMA = true;
-    alignas(64) CUtensorMap map_a, map_b;
-    __device__ __forceinline__ int first_c(int t, int kc) const { return ((t % groups()) * gc + kc) * kChunkK; }
-    __device__ __forceinline__ void box_a(int t, int kc, int& x, int& y) const {
-        x = first_c(t, kc); y = (int)(e_begin() + (int64_t)(t / groups()) * 128);
-    }
-    __device__ __forceinline__ void box_b(int t, int kc, int& x, int& y) const { x = first_c(t, kc); y = blockIdx.y * 64; }
-    __device__ static __forceinline__ float4 raw_a(const unsigned char* box, int row, int k) { return raw_swizzled(box, row, k); }
-    __device__ static __forceinline__ float4 raw_b(const unsigned char* box, int row, int k) { return raw_swizzled(box, row, k); }
-};
-
 // partial[r, j, c] = sum over the edges of range r of h[e, j] grad_s[e, c]: one tile per CTA,
 // m = c (column block of 128), n = j (block blockIdx.z of 64), k = edge.  grad_W = sum_r partial[r] in range
 // order (layer_sum_kernel).
 struct GradLayer {
     static constexpr int N = 64, A_LANE_ROWS = 32, B_LANE_ROWS = 32;
     static constexpr bool ACCUMULATE = true;
+    static constexpr bool TMA = true;
+    alignas(64) CUtensorMap map_a, map_b;   // grad_s [n_edges][C], h [n_edges][H]
     const float* gs; const float* h; float* partial;
     int64_t n_edges, chunk;   // chunk: edges per range (multiple of 32)
     int H, C;
@@ -612,25 +607,12 @@ struct GradLayer {
     __device__ __forceinline__ int n_tiles() const { return (total_chunks() + gc - 1) / gc; }
     __device__ __forceinline__ int n_chunks(int t) const { return min(gc, total_chunks() - t * gc); }
     __device__ __forceinline__ bool flush(int t) const { return t == n_tiles() - 1; }
-    __device__ __forceinline__ float4 column(const float* base, int ld, int col, bool col_ok, int kc, int k) const {
-        const int64_t e = e_begin() + (int64_t)kc * kChunkK + k, e_end = min(n_edges, e_begin() + chunk);
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (col_ok) {
-            if (e + 0 < e_end) v.x = base[(size_t)(e + 0) * ld + col];
-            if (e + 1 < e_end) v.y = base[(size_t)(e + 1) * ld + col];
-            if (e + 2 < e_end) v.z = base[(size_t)(e + 2) * ld + col];
-            if (e + 3 < e_end) v.w = base[(size_t)(e + 3) * ld + col];
-        }
-        return v;
-    }
-    __device__ __forceinline__ float4 load_a(int t, int kc, int row, int k) const {   // grad_s^T: row = c, k = edge
-        const int c = blockIdx.x * 128 + row;
-        return column(gs, C, c, c < C, t * gc + kc, k);
-    }
-    __device__ __forceinline__ float4 load_b(int t, int kc, int row, int k) const {   // h^T: row = j, k = edge
-        const int j = blockIdx.z * 64 + row;
-        return column(h, H, j, j < H, t * gc + kc, k);
-    }
+    // operands: boxes of 32 edges (128 c of grad_s | 64 j of h), read across the rows
+    __device__ __forceinline__ int first_e(int t, int kc) const { return (int)(e_begin() + (int64_t)(t * gc + kc) * kChunkK); }
+    __device__ __forceinline__ void box_a(int t, int kc, int& x, int& y) const { x = blockIdx.x * 128; y = first_e(t, kc); }
+    __device__ __forceinline__ void box_b(int t, int kc, int& x, int& y) const { x = blockIdx.z * 64; y = first_e(t, kc); }
+    __device__ static __forceinline__ float4 raw_a(const unsigned char* box, int row, int k) { return raw_transposed(box, 128, row, k); }
+    __device__ static __forceinline__ float4 raw_b(const unsigned char* box, int row, int k) { return raw_transposed(box, 64, row, k); }
     template <int W>
     __device__ __forceinline__ void store(int, int m, int n0, const float (&v)[W]) const {
         const int c = blockIdx.x * 128 + m;
@@ -646,17 +628,6 @@ struct GradLayer {
                 if (j0 + i < H) dst[(size_t)i * C] = v[i];
         }
     }
-};
-
-// the same with both operands fetched as boxes of 32 edges: (128 c of grad_s | 64 j of h), read across the rows
-struct GradLayerTma : GradLayer {
-    static constexpr bool TMA = true;
-    alignas(64) CUtensorMap map_a, map_b;
-    __device__ __forceinline__ int first_e(int t, int kc) const { return (int)(e_begin() + (int64_t)(t * gc + kc) * kChunkK); }
-    __device__ __forceinline__ void box_a(int t, int kc, int& x, int& y) const { x = blockIdx.x * 128; y = first_e(t, kc); }
-    __device__ __forceinline__ void box_b(int t, int kc, int& x, int& y) const { x = blockIdx.z * 64; y = first_e(t, kc); }
-    __device__ static __forceinline__ float4 raw_a(const unsigned char* box, int row, int k) { return raw_transposed(box, 128, row, k); }
-    __device__ static __forceinline__ float4 raw_b(const unsigned char* box, int row, int k) { return raw_transposed(box, 64, row, k); }
 };
 
 // grad_W[j, c] = sum_r partial[r, j, c], r ascending.
