@@ -281,6 +281,8 @@ int e3j_conv_bwd_bwd(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, con
  *   e3j_conv_fwd / e3j_conv_bwd; any of grad_x, grad_sh, grad_h, grad_W may be NULL.
  *   Workspace: 256-byte aligned, at least e3j_conv_radial_*_workspace_bytes(); calls that overlap on the GPU
  *   must not share it.
+ *   The two gradient products fetch their operands through tensor maps (tiled bulk copies); a driver that has no
+ *   encoder for them (cuTensorMapEncodeTiled, CUDA 12) makes the backward return E3J_ERR_UNSUPPORTED.
  * e3j_radial_weights writes the product itself, w_out [n_edges, P, N_q] (for callers that want the weights, and
  * as the unfused baseline in measurements). */
 int e3j_radial_weights(const e3j_plan* plan, int64_t n_edges, int hidden, const float* h, const float* W,
