@@ -29,7 +29,7 @@ __device__ __forceinline__ float4 f4_mul(const float4 a, const float4 b) {
 __device__ __forceinline__ float4 f4_zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
 
 template <bool IDENT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 conv_fwd_kernel(DeviceTables t, Dims dm, int64_t n_nodes, const float* __restrict__ x,
                 const float* __restrict__ sh, const float* __restrict__ w,
                 const int32_t* __restrict__ senders, const int32_t* __restrict__ rowptr,
@@ -103,7 +103,7 @@ conv_fwd_kernel(DeviceTables t, Dims dm, int64_t n_nodes, const float* __restric
 
 // Edge-local cotangents: grad_w[e,k,q] and grad_sh[e,i2]; one block per edge.
 template <bool IDENT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 conv_bwd_edge_kernel(DeviceTables t, Dims dm, int64_t n_edges, const float* __restrict__ x,
                      const float* __restrict__ sh, const float* __restrict__ w,
                      const int32_t* __restrict__ senders, const int32_t* __restrict__ receivers,
@@ -167,7 +167,7 @@ conv_bwd_edge_kernel(DeviceTables t, Dims dm, int64_t n_edges, const float* __re
 
 // Sender cotangent: grad_x[a,i1,q] gathers over the edges sent by a, in edge order.
 template <bool IDENT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 conv_bwd_node_kernel(DeviceTables t, Dims dm, int64_t n_nodes, const float* __restrict__ sh,
                      const float* __restrict__ w, const int32_t* __restrict__ receivers,
                      const int32_t* __restrict__ sender_perm, const int32_t* __restrict__ colptr,
