@@ -111,6 +111,8 @@ def run_radial_parity(wl, plan, cp, x, y, h, W, g, prepared=True):
     (2, 648, 64, e3j.E3J_PLAN_RADIAL_MATERIALISE),   # two-step form although the plan has the in-kernel one
     (3, 300, 64, 0),
     (5, 3000, 32, 0),
+    (2, 192, 128, 0),                              # two blocks of 64 hidden units in the gradient products
+    (2, 192, 160, 0),                              # three, the last one half full; W^T converted per tile
 ])
 def test_conv_radial_small(config, n_atoms, hidden, flags):
     run_radial_parity(*_radial_case(config, n_atoms, hidden, flags))
