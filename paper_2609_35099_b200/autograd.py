@@ -14,16 +14,21 @@ from __future__ import annotations
 import torch
 
 from . import (e3j_conv_bwd, e3j_conv_bwd_bwd, e3j_conv_fwd, e3j_conv_radial_bwd, e3j_conv_radial_fwd, e3j_conv_vec_bwd,
-               e3j_conv_vec_fwd, e3j_graph_prepare)
+               e3j_conv_vec_fwd, e3j_graph_prepare, e3j_graph_validate)
 
 
 class Graph:
     """Receiver-sorted edge list with the index arrays the kernels want (e3j_graph_prepare), on the device."""
 
-    def __init__(self, n_nodes: int, senders: torch.Tensor, receivers: torch.Tensor):
+    def __init__(self, n_nodes: int, senders: torch.Tensor, receivers: torch.Tensor, validate: bool = True):
+        """validate: check on the device, before anything indexes with them, that the ids lie in [0, n_nodes) and the
+        receivers do not decrease (one small kernel and a synchronisation per edge list).  The compute calls
+        trust the list: an id outside the range makes them read or write outside their arrays."""
         self.n_nodes = int(n_nodes)
         self.senders = senders.to(torch.int32).contiguous()
         self.receivers = receivers.to(torch.int32).contiguous()
+        if validate and e3j_graph_validate(self.n_nodes, self.senders, self.receivers) != 0:
+            raise ValueError("edge list: an id outside [0, n_nodes) or receivers that decrease")
         self.rowptr, self.sender_perm, self.colptr = e3j_graph_prepare(self.n_nodes, self.senders, self.receivers)
 
 

@@ -67,3 +67,13 @@ def test_autograd_radial_and_edge_vector_forms():
     _, rv, rw = e3j.e3j_conv_vec_bwd(plan, x, vec, w, *args, g, *prep, grad_x=False)
     torch.cuda.synchronize()
     assert torch.equal(gv, rv) and torch.equal(gw, rw)
+
+
+def test_graph_refuses_bad_edge_lists_before_anything_indexes_with_them():
+    snd = torch.tensor([0, 1, 2, 1], dtype=torch.int32, device=DEV)
+    rcv = torch.tensor([0, 0, 1, 2], dtype=torch.int32, device=DEV)
+    assert Graph(3, snd, rcv).rowptr.tolist() == [0, 2, 3, 4]
+    with pytest.raises(ValueError):
+        Graph(2, snd, rcv)                       # ids up to 2 with two nodes
+    with pytest.raises(ValueError):
+        Graph(3, snd, torch.tensor([0, 1, 0, 2], dtype=torch.int32, device=DEV))   # receivers decrease
