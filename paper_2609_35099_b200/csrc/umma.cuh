@@ -159,17 +159,17 @@ __device__ __forceinline__ void split_tf32(float v, float& hi, float& lo) {
 __device__ __forceinline__ void split_tf32(const float4 v, float4& hi, float4& lo) {
     split_tf32(v.x, hi.x, lo.x); split_tf32(v.y, hi.y, lo.y); split_tf32(v.z, hi.z, lo.z); split_tf32(v.w, hi.w, lo.w);
 }
-// The same split with the rounding done on the bit pattern (add half a TF32 unit to the magnitude, clear the 13
-// low bits): what the conversion instruction gives for finite values, on the integer pipe.  The conversion
-// instruction issues at an eighth of the integer rate, which bounds warps that do little else (the converters of
-// the gradient products); where the integer pipe is the busy one (the other kernels) the instruction is the cheaper.
+// A cheaper split for warps that do little else (the converters of the gradient products, which the conversion
+// instruction bounds: it issues at an eighth of the integer rate).  hi is rounded on the bit pattern (add half a
+// TF32 unit to the magnitude, clear the 13 low bits: what the instruction gives for finite values); lo = v - hi
+// is exact in float32 and left as it is: the tensor cores drop its low bits themselves, an error of 2^-21 |v| at
+// most, of the size of the a_lo b_lo term that the three-term product leaves out anyway.
 __device__ __forceinline__ float round_tf32_bits(float v) {
     return __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
 }
 __device__ __forceinline__ void split_tf32_bits(const float4 v, float4& hi, float4& lo) {
     hi = make_float4(round_tf32_bits(v.x), round_tf32_bits(v.y), round_tf32_bits(v.z), round_tf32_bits(v.w));
-    lo = make_float4(round_tf32_bits(v.x - hi.x), round_tf32_bits(v.y - hi.y), round_tf32_bits(v.z - hi.z),
-                     round_tf32_bits(v.w - hi.w));
+    lo = make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);
 }
 
 }  // namespace umma
