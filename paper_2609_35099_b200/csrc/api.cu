@@ -120,6 +120,14 @@ inline int grid_for(int64_t n) {
     return (int)g;
 }
 
+// Threads per block for a kernel whose blocks work through `items` items block-wide: whole warps, at most 256, and
+// as few idle threads in the last pass as the warp granularity allows (128 items: 128 threads, 416: two passes of 224).
+inline int block_for(int64_t items) {
+    const int64_t passes = (std::max<int64_t>(items, 1) + 255) / 256;
+    const int64_t per_pass = (std::max<int64_t>(items, 1) + passes - 1) / passes;
+    return (int)std::min<int64_t>(256, std::max<int64_t>(64, (per_pass + 31) / 32 * 32));
+}
+
 inline Dims dims_of(const e3j_plan* p) {
     return Dims{p->nq, p->d, p->dp, p->P, p->D, (p->flags & E3J_PLAN_COLLAPSE_OUTPUTS) ? 1 : 0};
 }
@@ -356,7 +364,7 @@ int e3j::conv_fwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, c
     }
     DeviceTables t;
     if (int s = get_device_tables(plan, t)) return s;
-    generic::conv_fwd_kernel<false><<<grid_for(n_nodes), 256, 0, st>>>(t, dims_of(plan), n_nodes, x, sh, w,
+    generic::conv_fwd_kernel<false><<<grid_for(n_nodes), block_for((int64_t)plan->D * plan->nq / 4), 0, st>>>(t, dims_of(plan), n_nodes, x, sh, w,
                                                                       senders, rowptr, out);
     return after_launch();
 }
@@ -426,12 +434,12 @@ int e3j::conv_bwd_impl(const e3j_plan* plan, int64_t n_nodes, int64_t n_edges, c
     if (int s = get_device_tables(plan, t)) return s;
     const Dims dm = dims_of(plan);
     if ((grad_w || grad_sh) && n_edges > 0) {
-        generic::conv_bwd_edge_kernel<false><<<grid_for(n_edges), 256, 0, st>>>(
+        generic::conv_bwd_edge_kernel<false><<<grid_for(n_edges), block_for((int64_t)dm.P * dm.nq / 4), 0, st>>>(
             t, dm, n_edges, x, sh, w, senders, receivers, grad_out, grad_w, grad_sh, n_real);
         if (int s = after_launch()) return s;
     }
     if (grad_x) {
-        generic::conv_bwd_node_kernel<false><<<grid_for(n_nodes), 256, 0, st>>>(
+        generic::conv_bwd_node_kernel<false><<<grid_for(n_nodes), block_for((int64_t)dm.d * dm.nq / 4), 0, st>>>(
             t, dm, n_nodes, sh, w, receivers, sender_perm, colptr, grad_out, grad_x);
         if (int s = after_launch()) return s;
     }
@@ -584,7 +592,7 @@ int e3j_tp_fwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
     if (fk && fk->tp_fwd) return fk->tp_fwd(rows, x1, x2, w, out, st);
     DeviceTables t;
     if (int s = get_device_tables(plan, t)) return s;
-    generic::conv_fwd_kernel<true><<<grid_for(rows), 256, 0, st>>>(t, dims_of(plan), rows, x1, x2, w, nullptr,
+    generic::conv_fwd_kernel<true><<<grid_for(rows), block_for((int64_t)plan->D * plan->nq / 4), 0, st>>>(t, dims_of(plan), rows, x1, x2, w, nullptr,
                                                                   nullptr, out);
     return after_launch();
 }
@@ -605,12 +613,12 @@ int e3j_tp_bwd(const e3j_plan* plan, int64_t rows, const float* x1, const float*
     if (int s = get_device_tables(plan, t)) return s;
     const Dims dm = dims_of(plan);
     if (grad_w || grad_x2) {
-        generic::conv_bwd_edge_kernel<true><<<grid_for(rows), 256, 0, st>>>(t, dm, rows, x1, x2, w, nullptr,
+        generic::conv_bwd_edge_kernel<true><<<grid_for(rows), block_for((int64_t)dm.P * dm.nq / 4), 0, st>>>(t, dm, rows, x1, x2, w, nullptr,
                                                                            nullptr, grad_out, grad_w, grad_x2, nullptr);
         if (int s = after_launch()) return s;
     }
     if (grad_x1) {
-        generic::conv_bwd_node_kernel<true><<<grid_for(rows), 256, 0, st>>>(t, dm, rows, x2, w, nullptr, nullptr,
+        generic::conv_bwd_node_kernel<true><<<grid_for(rows), block_for((int64_t)dm.d * dm.nq / 4), 0, st>>>(t, dm, rows, x2, w, nullptr, nullptr,
                                                                            nullptr, grad_out, grad_x1);
         if (int s = after_launch()) return s;
     }
