@@ -239,3 +239,38 @@ def test_conv_radial_config5_full_size_sampled():
     via_h = float((gh.double() * dh_.double()).sum().item())
     scale = float((dg_.double() * out.double()).abs().sum().item())
     assert abs(via_W - ref) <= 1e-6 * scale and abs(via_h - ref) <= 1e-6 * scale, (ref, via_W, via_h, scale)
+
+
+def test_radial_calls_can_be_captured_in_a_cuda_graph():
+    """The calls through (h, W) only enqueue kernels once the graph is prepared and the caller owns outputs and
+    workspaces (the tensor maps of the gradient products travel as kernel arguments): a captured forward +
+    backward replays to the bits of the eager calls."""
+    wl, plan, cp, x, y, h, W, g = _radial_case(2, 192, 64)
+    n, e = wl.n_nodes, wl.n_edges
+    snd, rcv = _cuda(wl.senders), _cuda(wl.receivers)
+    dx, dy, dh, dW, dg = _cuda(x), _cuda(y), _cuda(h), _cuda(W), _cuda(g)
+    rowptr, perm, colptr = e3j.e3j_graph_prepare(n, snd, rcv)
+    u8 = lambda nbytes: torch.empty(max(nbytes, 256), dtype=torch.uint8, device=DEV)
+    ws_f = u8(e3j.e3j_conv_radial_fwd_workspace_bytes(plan, n, e, 64))
+    ws_b = u8(e3j.e3j_conv_radial_bwd_workspace_bytes(plan, n, e, 64))
+    out = torch.empty_like(dg)
+    grads = [torch.empty_like(t) for t in (dx, dy, dh, dW)]
+
+    def step():
+        e3j.e3j_conv_radial_fwd(plan, dx, dy, dh, dW, snd, rcv, rowptr, out=out, workspace=ws_f)
+        e3j.e3j_conv_radial_bwd(plan, dx, dy, dh, dW, snd, rcv, dg, rowptr, perm, colptr, grad_x=grads[0],
+                                grad_sh=grads[1], grad_h=grads[2], grad_W=grads[3], workspace=ws_b)
+
+    step()   # eager: first use sets the kernels' attributes, uploads the tables and looks the map encoder up
+    torch.cuda.synchronize()
+    eager = [t.clone() for t in (out, *grads)]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for t in (out, *grads):
+        t.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    for a, b in zip(eager, (out, *grads)):
+        assert torch.equal(a, b)
+    assert e3j.e3j_plan_device_status(plan) == 0
