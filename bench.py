@@ -683,7 +683,7 @@ def main():
                 if evd is not None:
                     stream.wait_event(evd)
 
-        e2e_run(2); torch.cuda.synchronize()
+        e2e_run(max(3, args.warmup)); torch.cuda.synchronize()   # untimed warm-up steps of the same pipeline
         k_e2e = args.steps
         barrier(); torch.cuda.synchronize()
         s0, s1 = ev(), ev()
