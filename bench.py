@@ -573,6 +573,66 @@ def main():
                 "tensor_frac_of_tf32_peak": flop_tensor / (rf_ms * 1e-3) / 1e12 / (0.5 * bf16_peak),
                 "tensor_peak_note": "TF32 peak taken as half the measured bf16 peak (nominal ratio)"},
         }
+        # The same two calls end to end from pinned host memory: with (h, W) in place of w a step moves a tenth of the
+        # bytes over the bus, which is what bounds `e2e` of the headline calls.
+        if not args.no_e2e and world == 1:
+            keys_in = ("x", "y", "snd", "rcv", "g")
+            host_in = {k: pinned[k] for k in keys_in}
+            host_in["h"], host_in["W"] = hh.cpu().pin_memory(), WW.cpu().pin_memory()
+            dev_res = dict(out=out, gx=gx, gy=gy, gh=gh, gW=gW)
+            host_res = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in dev_res.items()}
+            sets = [{k: torch.empty(v.shape, dtype=v.dtype, device=dev) for k, v in host_in.items()} for _ in range(2)]
+            results = [{k: torch.empty_like(v) for k, v in dev_res.items()} for _ in range(2)]
+            r_h2d = sum(v.numel() * v.element_size() for v in host_in.values())
+            r_d2h = sum(v.numel() * v.element_size() for v in host_res.values())
+            q_in, q_out = torch.cuda.Stream(), torch.cuda.Stream()
+            done_c, done_o = [None, None], [None, None]
+
+            def radial_step(i):
+                b = i % 2
+                s, r = sets[b], results[b]
+                with torch.cuda.stream(q_in):
+                    if done_c[b] is not None:
+                        q_in.wait_event(done_c[b])
+                    for k in s:
+                        s[k].copy_(host_in[k], non_blocking=True)
+                    arrived = torch.cuda.Event(); arrived.record(q_in)
+                stream.wait_event(arrived)
+                if done_o[b] is not None:
+                    stream.wait_event(done_o[b])
+                e3j.e3j_conv_radial_fwd(plan, s["x"], s["y"], s["h"], s["W"], s["snd"], s["rcv"], rowptr, out=r["out"],
+                                        workspace=ws_rf)
+                e3j.e3j_conv_radial_bwd(plan, s["x"], s["y"], s["h"], s["W"], s["snd"], s["rcv"], s["g"], rowptr, perm,
+                                        colptr, grad_x=r["gx"], grad_sh=r["gy"], grad_h=r["gh"], grad_W=r["gW"],
+                                        workspace=ws_rb)
+                done_c[b] = torch.cuda.Event(); done_c[b].record(stream)
+                with torch.cuda.stream(q_out):
+                    q_out.wait_event(done_c[b])
+                    for k in host_res:
+                        host_res[k].copy_(r[k], non_blocking=True)
+                    done_o[b] = torch.cuda.Event(); done_o[b].record(q_out)
+
+            def radial_run(k):
+                for i in range(k):
+                    radial_step(i)
+                for evd in done_o:
+                    if evd is not None:
+                        stream.wait_event(evd)
+
+            radial_run(max(3, args.warmup)); torch.cuda.synchronize()
+            k_re = max(3, min(args.steps, 50))
+            a0, a1 = ev(), ev()
+            a0.record(stream)
+            q_in.wait_event(a0)
+            radial_run(k_re)
+            a1.record(stream)
+            torch.cuda.synchronize()
+            re_ms = a0.elapsed_time(a1) / k_re
+            radial["e2e"] = {"value": e / (re_ms * 1e-3), "unit": "edges/s", "ms_per_step": re_ms, "steps": k_re,
+                             "h2d_bytes_per_step": r_h2d, "d2h_bytes_per_step": r_d2h,
+                             "note": "e3j_conv_radial_fwd + e3j_conv_radial_bwd from pinned host buffers, copies inside "
+                                     "the timed region on streams of their own, two buffer sets"}
+            del sets, results, host_res
         del ws_rf, ws_rb, w_mat, hh, WW, gh, gW
 
     # ---- the backward over a processing order built once per neighbour list (runs of one sender summed in registers)
